@@ -1,0 +1,162 @@
+"""TEST INFRASTRUCTURE ONLY: ctypes front end of the plain-C collectives oracle.
+
+The arithmetic lives in ``collectives_oracle.c`` (naive fp64 / wrapping-int / byte
+loops written from the collective definitions of the paper, Sec. 2 and Sec. 3.1,
+and the rank-order sum of Sec. 3.3).  This wrapper only marshals numpy arrays.
+Nothing in the product package imports this module; only the tests, the smoke
+check and the benchmark's cpu_baseline / reference legs do.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "collectives_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+BF16, F32, I32, U8 = 0, 1, 2, 3
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle (gcc -O2, OpenMP when available)."""
+    if not force and os.path.exists(_LIB) and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC):
+        return _LIB
+    cmd = ["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-fopenmp", _SRC, "-o", _LIB, "-lm"]
+    try:
+        subprocess.run(cmd, check=True, capture_output=True)
+    except subprocess.CalledProcessError:
+        cmd.remove("-fopenmp")
+        subprocess.run(cmd, check=True, capture_output=True)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.orc_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().orc_num_threads())
+
+
+def _ptrs(arrs):
+    for a in arrs:
+        assert a.flags["C_CONTIGUOUS"]
+    return (ctypes.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise RuntimeError(f"oracle {what} failed with code {rc}")
+
+
+def allgather(inputs):
+    """inputs[r]: any dtype, m bytes each -> out[r] = concatenation over ranks."""
+    R = len(inputs)
+    m = inputs[0].nbytes
+    outs = [np.empty(R * inputs[0].size, dtype=inputs[0].dtype) for _ in range(R)]
+    _check(lib().orc_allgather(R, ctypes.c_size_t(m), _ptrs(inputs), _ptrs(outs)), "allgather")
+    return outs
+
+
+def alltoall(inputs):
+    R = len(inputs)
+    assert inputs[0].nbytes % R == 0
+    m = inputs[0].nbytes // R
+    outs = [np.empty_like(inputs[0]) for _ in range(R)]
+    _check(lib().orc_alltoall(R, ctypes.c_size_t(m), _ptrs(inputs), _ptrs(outs)), "alltoall")
+    return outs
+
+
+def alltoallv(inputs, counts_elems):
+    """counts_elems[p][r] = elements p sends to r (element = inputs dtype)."""
+    R = len(inputs)
+    C = np.ascontiguousarray(np.asarray(counts_elems, dtype=np.uint64) * np.uint64(inputs[0].itemsize))
+    outs = [np.zeros(int(np.asarray(counts_elems)[:, r].sum()), dtype=inputs[0].dtype) for r in range(R)]
+    # keep zero-size buffers addressable
+    outs_c = [o if o.size else np.zeros(1, dtype=o.dtype) for o in outs]
+    ins_c = [a if a.size else np.zeros(1, dtype=a.dtype) for a in inputs]
+    _check(lib().orc_alltoallv(R, C.ctypes.data_as(ctypes.c_void_p), _ptrs(ins_c), _ptrs(outs_c)), "alltoallv")
+    return [oc[:o.size] for oc, o in zip(outs_c, outs)]
+
+
+def _dtype_code(a, dtype):
+    if dtype == "bf16":
+        assert a.dtype == np.uint16
+        return BF16
+    if dtype == "f32":
+        assert a.dtype == np.float32
+        return F32
+    raise ValueError(dtype)
+
+
+def reduce_scatter(inputs, dtype):
+    """dtype 'bf16' (uint16 bits) / 'f32' -> fp64 outputs; 'i32' -> int32 outputs."""
+    R = len(inputs)
+    n = inputs[0].size
+    assert n % R == 0
+    m = n // R
+    if dtype == "i32":
+        outs = [np.empty(m, dtype=np.int32) for _ in range(R)]
+        _check(lib().orc_reduce_scatter_i32(R, ctypes.c_size_t(m), _ptrs(inputs), _ptrs(outs)), "rs_i32")
+        return outs
+    outs = [np.empty(m, dtype=np.float64) for _ in range(R)]
+    _check(lib().orc_reduce_scatter_f64(R, _dtype_code(inputs[0], dtype), ctypes.c_size_t(m),
+                                        _ptrs(inputs), _ptrs(outs)), "rs_f64")
+    return outs
+
+
+def allreduce(inputs, dtype):
+    R = len(inputs)
+    n = inputs[0].size
+    if dtype == "i32":
+        outs = [np.empty(n, dtype=np.int32) for _ in range(R)]
+        _check(lib().orc_allreduce_i32(R, ctypes.c_size_t(n), _ptrs(inputs), _ptrs(outs)), "ar_i32")
+        return outs
+    outs = [np.empty(n, dtype=np.float64) for _ in range(R)]
+    _check(lib().orc_allreduce_f64(R, _dtype_code(inputs[0], dtype), ctypes.c_size_t(n),
+                                   _ptrs(inputs), _ptrs(outs)), "ar_f64")
+    return outs
+
+
+def moe_dispatch(x, idx, E, recv_capacity_rows=None):
+    """x[p]: [T, W] row arrays (any dtype), idx[p]: int32 [T, K].
+    Returns dict(recv, meta, pos, counts, expert_counts); recv[r] has capacity rows,
+    of which counts[:, r].sum() are valid."""
+    R = len(x)
+    T, K = idx[0].shape
+    row_bytes = x[0].shape[1] * x[0].itemsize
+    cap = recv_capacity_rows if recv_capacity_rows is not None else R * T * K
+    recv = [np.zeros((cap, x[0].shape[1]), dtype=x[0].dtype) for _ in range(R)]
+    meta = [np.full((cap, 4), -1, dtype=np.int32) for _ in range(R)]
+    pos = [np.full((T, K), -1, dtype=np.int32) for _ in range(R)]
+    counts = np.zeros((R, R), dtype=np.int64)
+    ecounts = np.zeros((R, E), dtype=np.int64)
+    rc = lib().orc_moe_dispatch(R, T, E, K, ctypes.c_size_t(row_bytes), ctypes.c_size_t(cap),
+                                _ptrs(x), _ptrs(idx), _ptrs(recv), _ptrs(meta), _ptrs(pos),
+                                counts.ctypes.data_as(ctypes.c_void_p),
+                                ecounts.ctypes.data_as(ctypes.c_void_p))
+    _check(rc, "moe_dispatch")
+    return dict(recv=recv, meta=meta, pos=pos, counts=counts, expert_counts=ecounts)
+
+
+def moe_combine(y, idx, pos, gates, E, H):
+    """y[r]: uint16 bf16 rows [cap, H]; returns fp64 out[p] of shape [T, H]."""
+    R = len(y)
+    T, K = idx[0].shape
+    outs = [np.empty((T, H), dtype=np.float64) for _ in range(R)]
+    for a in y:
+        assert a.dtype == np.uint16
+    for g in gates:
+        assert g.dtype == np.float32
+    rc = lib().orc_moe_combine_f64(R, T, H, E, K, _ptrs(y), _ptrs(idx), _ptrs(pos), _ptrs(gates), _ptrs(outs))
+    _check(rc, "moe_combine")
+    return outs
