@@ -1,0 +1,321 @@
+/*
+ * purlin.h -- C ABI of the B200 collectives executor.
+ *
+ * The library follows the paper's split into semantics, orchestration and datapath
+ * (Sec. 1, "three-layer design"; Sec. 3.1-3.3):
+ *
+ *   semantics      a collective is named by (consume op, input layout, output layout)
+ *                  (Listing 1) -> pl_collective_t;
+ *   orchestration  where and when chunks move: the host lowers a collective into a flat
+ *                  list of chunk-granular copy / reduce / copy-reduce ops with wait and
+ *                  signal edges (Sec. 3.2, Listing 2, Algorithm 1) -> pl_schedule_build*;
+ *   datapath       how bytes move: one persistent sm_100a kernel interprets the per-CTA op
+ *                  queues (Sec. 3.3, Listing 3, Algorithm 2) -> pl_execute.
+ *
+ * R logical ranks are R sets of buffers in ONE GPU's memory; every rank's buffers are
+ * visible to every other rank, i.e. the executor is the paper's variant that skips the
+ * staging copy because application buffers are already peer accessible (Sec. 3.2,
+ * "SNAC omits staging"; Sec. 5 "-ZS").
+ *
+ * Conventions
+ *   - Plain C99 ABI, opaque handles, every call returns pl_status_t (PL_OK == 0).
+ *   - All buffer pointers handed to pl_execute / pl_moe_* are DEVICE pointers unless a
+ *     parameter is documented as host memory.  The library never owns, frees or writes
+ *     input buffers; inputs are const, so repeating an execute repeats its result.
+ *   - Errors are found on the host before any launch.  The device never traps: a wait
+ *     that exceeds the schedule's time limit records a pl_devstatus_t and the kernel
+ *     returns (see pl_comm_status).
+ *   - pl_execute enqueues exactly one kernel on `stream`; it allocates nothing, copies
+ *     nothing and never synchronises.  A schedule may be executed any number of times
+ *     (flags carry a device-resident epoch; nothing is reset between executes).
+ *   - One stream at a time per schedule: two executes of the same schedule must not
+ *     overlap on the GPU.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ */
+#ifndef PURLIN_H_
+#define PURLIN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PL_MAX_RANKS 16
+#define PL_MAX_SRC 16   /* sources of one reduce op */
+#define PL_MAX_WAITS 16 /* flags one op may wait on */
+
+typedef enum {
+  PL_OK = 0,
+  PL_ERR_INVALID_ARG = 1,
+  PL_ERR_UNSUPPORTED = 2,
+  PL_ERR_ALIGNMENT = 3,
+  PL_ERR_OOM = 4,
+  PL_ERR_CUDA = 5,
+  PL_ERR_TIMEOUT = 6,
+  PL_ERR_OVERSUBSCRIBED = 7,
+  PL_ERR_INVALID_SCHEDULE = 8,
+  PL_ERR_OVERFLOW = 9
+} pl_status_t;
+
+/* Element types.  Reductions convert each element to fp32, accumulate in fp32 and
+ * convert once at the end (Sec. 3.3, Eq. "rank-order"); int32 sums wrap.  PL_U8 is
+ * valid for copy-only collectives. */
+typedef enum { PL_BF16 = 0, PL_F32 = 1, PL_I32 = 2, PL_U8 = 3 } pl_dtype_t;
+
+/* Collectives (Listing 1): reduce-scatter = reduce, scattered->packed; all-gather = copy,
+ * packed->scattered; all-to-all = copy, scattered->transposed; all-to-all-v its runtime-
+ * sized twin; all-reduce = compose<reduce-scatter, all-gather>. */
+typedef enum {
+  PL_ALLREDUCE = 0,
+  PL_REDUCE_SCATTER = 1,
+  PL_ALLGATHER = 2,
+  PL_ALLTOALL = 3,
+  PL_ALLTOALLV = 4
+} pl_collective_t;
+
+/* Algorithms.
+ *   PL_ALGO_DIRECT        every consumer pulls straight from the producers' buffers.  For
+ *                         all-reduce this is Algorithm 1 without the staging role: rank k
+ *                         reduces partition k from all inputs into its own output,
+ *                         publishes reduced(k, c), and every other rank copies that chunk.
+ *   PL_ALGO_ONESHOT       all-reduce only: every rank reduces the whole message itself.
+ *   PL_ALGO_DIRECT_FUSED  all-reduce only: the reducer of partition k writes the result
+ *                         into all R outputs (no gather step, fewest bytes).
+ *   PL_ALGO_RING          textbook ring; partial sums travel in fp32 (int32 for ints).
+ *   PL_ALGO_TREE          all-reduce only: binomial reduce to rank 0, binomial broadcast.
+ * Ring and tree are not in the paper (its only pattern is the direct pull); they are the
+ * classical algorithms the benchmark configurations name. */
+typedef enum {
+  PL_ALGO_RING = 0,
+  PL_ALGO_TREE = 1,
+  PL_ALGO_DIRECT = 2,
+  PL_ALGO_ONESHOT = 3,
+  PL_ALGO_DIRECT_FUSED = 4
+} pl_algo_t;
+
+typedef enum { PL_OP_COPY = 0, PL_OP_REDUCE = 1, PL_OP_COPY_REDUCE = 2 } pl_op_kind_t;
+typedef enum { PL_BUF_IN = 0, PL_BUF_OUT = 1, PL_BUF_SCRATCH = 2 } pl_buf_kind_t;
+/* How an op body moves bytes (Sec. 3.3).  TMA = cp.async.bulk staged through a
+ * shared-memory ring of `stages` slots of `stage_bytes` (Algorithm 2: prime / steady /
+ * drain).  LDST = 128-bit register loads/stores, unrolled (the paper's register path). */
+typedef enum { PL_DP_AUTO = 0, PL_DP_LDST = 1, PL_DP_TMA = 2 } pl_datapath_t;
+
+typedef struct pl_comm_s* pl_comm_t;
+typedef struct pl_schedule_s* pl_schedule_t;
+typedef struct pl_moe_plan_s* pl_moe_plan_t;
+
+/* Tuning knobs of one schedule ("codesign policy", Sec. 3.2/3.3).  Zero = take the
+ * library's sm_100a default for the message size.  struct_size must be sizeof(). */
+typedef struct {
+  uint32_t struct_size;
+  int32_t n_ctas;        /* persistent CTAs = op queues; rounded down to a multiple of R  */
+  int32_t threads;       /* threads per CTA (multiple of 32, <= 1024)                     */
+  int32_t datapath;      /* pl_datapath_t                                                 */
+  int32_t stages;        /* shared-memory ring depth S of the TMA pipeline                */
+  uint32_t stage_bytes;  /* bytes per ring slot B_stage (multiple of 16)                  */
+  uint32_t slice_bytes;  /* a chunk larger than this is split into slices run by several  */
+                         /* CTAs; the chunk's flag then counts slices (Sec. 3.2, "last    */
+                         /* staging CTA ... announces")                                   */
+  uint64_t timeout_ns;   /* bound of every device-side wait; 0 = 2 s                      */
+  uint32_t flags;        /* PL_OPT_*                                                      */
+} pl_sched_opts_t;
+#define PL_OPT_SKIP_VALIDATE 1u /* do not run the static validator inside build */
+
+/* A buffer reference inside an op: rank's in/out/scratch buffer, byte offset, and the
+ * element type stored there (partials of a bf16 reduction are PL_F32). */
+typedef struct {
+  int32_t rank;
+  int32_t buf;   /* pl_buf_kind_t */
+  int32_t dtype; /* pl_dtype_t */
+  int32_t pad_;
+  uint64_t offset; /* bytes */
+} pl_ref_t;
+
+/* One op of a schedule as reported by pl_schedule_dump (host copy, for inspection and
+ * for replaying a schedule on the CPU in tests). */
+typedef struct {
+  int32_t kind;      /* pl_op_kind_t */
+  int32_t exec_rank; /* rank whose CTAs run the op (the consumer that pulls) */
+  int32_t queue;     /* CTA / op queue the op is placed on */
+  int32_t topo;      /* position in the global topological order */
+  int32_t layer;     /* layer of a multi-layer schedule, else 0 */
+  int32_t n_src;
+  int32_t n_wait;
+  int32_t signal_flag; /* flag incremented (release) when the op's writes are done, -1 none */
+  int32_t signal_flag2;/* optional second flag incremented the same way, -1 none */
+  int32_t dst_bcast;   /* 1: dst is replicated at the same offset into out[0..R) */
+  uint64_t count;      /* elements; COPY ops count bytes (dtype PL_U8) */
+  pl_ref_t dst;
+  pl_ref_t src[PL_MAX_SRC];
+  int32_t wait_flag[PL_MAX_WAITS];
+  uint32_t wait_need[PL_MAX_WAITS]; /* signals per execute the flag must have received */
+} pl_op_t;
+
+typedef struct {
+  uint64_t n_ops, n_queues, n_flags, n_waits, n_layers;
+  uint64_t bytes_read, bytes_written;  /* summed over ops: the schedule's algorithmic bytes */
+  uint64_t message_bytes;              /* per-rank message size in the paper's convention  */
+                                       /* (Sec. 5: gathered output for all-gather, per-rank */
+                                       /* input otherwise)                                  */
+  uint64_t scratch_bytes;              /* device scratch the schedule owns (all ranks)      */
+  uint64_t in_bytes[PL_MAX_RANKS];     /* bytes pl_execute requires in bufs->in[r]          */
+  uint64_t out_bytes[PL_MAX_RANKS];    /* bytes pl_execute requires in bufs->out[r]         */
+  int32_t grid, threads, smem_bytes, datapath, stages;
+  uint32_t stage_bytes, slice_bytes;
+} pl_sched_info_t;
+
+/* Device buffers of one execute: in[r] / out[r] for r < R, 16-byte aligned, non-overlapping. */
+typedef struct {
+  const void* in[PL_MAX_RANKS];
+  void* out[PL_MAX_RANKS];
+  size_t in_bytes[PL_MAX_RANKS];
+  size_t out_bytes[PL_MAX_RANKS];
+} pl_bufs_t;
+
+/* Device-side status record (first writer wins).  code == PL_OK when nothing happened. */
+typedef struct {
+  int32_t code;   /* PL_OK or PL_ERR_TIMEOUT */
+  int32_t queue;  /* CTA that gave up */
+  int32_t op;     /* index of the op inside the schedule (topological index) */
+  int32_t flag;   /* flag it was waiting on */
+  uint64_t expected, observed;
+} pl_devstatus_t;
+
+/* ---- communicator ------------------------------------------------------------------ */
+
+/* Create a communicator of R emulated ranks (2 <= R <= PL_MAX_RANKS) with element type
+ * `dtype` on the CURRENT CUDA device.  Allocates a few device words (status, abort).
+ * Errors: PL_ERR_INVALID_ARG (R, dtype, out), PL_ERR_CUDA (no usable device). */
+pl_status_t pl_comm_create(int R, pl_dtype_t dtype, pl_comm_t* out);
+
+/* Same, but host-only: schedules can be built, validated, inspected and dumped; nothing is
+ * placed on a device and pl_execute returns PL_ERR_UNSUPPORTED.  Needs no GPU. */
+pl_status_t pl_comm_create_planner(int R, pl_dtype_t dtype, pl_comm_t* out);
+
+/* Destroy a communicator.  Its schedules and plans must be destroyed first
+ * (PL_ERR_INVALID_ARG otherwise). */
+pl_status_t pl_comm_destroy(pl_comm_t comm);
+
+/* Read the device status record.  Synchronises the device.  Returns PL_OK and fills *out;
+ * out->code tells whether a wait timed out since the last reset. */
+pl_status_t pl_comm_status(pl_comm_t comm, pl_devstatus_t* out);
+
+/* Clear the status record and re-zero the flags and epochs of every schedule of `comm`
+ * (asynchronously on `stream`).  Required after a timeout before executing again. */
+pl_status_t pl_comm_reset(pl_comm_t comm, void* stream);
+
+/* ---- orchestration ----------------------------------------------------------------- */
+
+/* Lower a fixed-size collective into a schedule.
+ *   count_per_rank  elements of the per-rank message: the INPUT element count for
+ *                   all-reduce, reduce-scatter and all-to-all; the per-rank CONTRIBUTION
+ *                   for all-gather (output = R * count_per_rank).
+ *   chunk_bytes     chunk size in bytes of the element type (multiple of 16); clipped to
+ *                   the partition size; the last chunk of a partition may be short.
+ * Partitioned collectives need count_per_rank * elem_size divisible by R*16
+ * (PL_ERR_INVALID_ARG).  PL_ERR_UNSUPPORTED for algorithm/collective pairs that do not
+ * exist (tree, one-shot and fused are all-reduce only; PL_U8 cannot be reduced).
+ * PL_ERR_OVERSUBSCRIBED when the requested CTAs cannot all be co-resident (the executor
+ * spins on flags, so every queue must be running).  PL_ERR_OOM / PL_ERR_CUDA on device
+ * allocation failure.  The schedule owns its device op list, flags and scratch. */
+pl_status_t pl_schedule_build(pl_comm_t comm, pl_collective_t coll, pl_algo_t algo,
+                              size_t count_per_rank, size_t chunk_bytes,
+                              const pl_sched_opts_t* opts, pl_schedule_t* out);
+
+/* Variable-size all-to-all: counts is a HOST array R*R, row-major [src][dst], in elements.
+ * counts[p][r]*elem_size must be a multiple of 16 (PL_ERR_ALIGNMENT).  Only
+ * PL_ALLTOALLV with PL_ALGO_DIRECT. */
+pl_status_t pl_schedule_build_v(pl_comm_t comm, pl_collective_t coll, pl_algo_t algo,
+                                const size_t* counts, size_t chunk_bytes,
+                                const pl_sched_opts_t* opts, pl_schedule_t* out);
+
+/* n_layers back-to-back all-reduces in ONE launch (the latency path: no kernel launch,
+ * memset or host round trip per layer).  Layer l reads in[r] + l*M and writes out[r] + l*M
+ * (M = count_per_rank * elem_size).  Rank r's layer-(l+1) contribution counts as published
+ * only when r's layer-l output is complete, and no consumer reads it earlier.  Algorithms:
+ * PL_ALGO_ONESHOT, PL_ALGO_DIRECT, PL_ALGO_DIRECT_FUSED. */
+pl_status_t pl_schedule_build_layers(pl_comm_t comm, pl_algo_t algo, size_t count_per_rank,
+                                     int n_layers, const pl_sched_opts_t* opts,
+                                     pl_schedule_t* out);
+
+pl_status_t pl_schedule_info(pl_schedule_t s, pl_sched_info_t* out);
+
+/* Copy up to `cap` ops (topological order) into `ops`; *n receives the total op count.
+ * ops may be NULL to query the count. */
+pl_status_t pl_schedule_dump(pl_schedule_t s, pl_op_t* ops, size_t cap, size_t* n);
+
+/* Static check of a schedule (also run by build unless PL_OPT_SKIP_VALIDATE): every output
+ * byte written exactly once, every read of a byte the schedule writes is ordered after that
+ * write by a wait edge (or by queue order), every flag's signals precede its waiters in
+ * the topological order, queue order embeds in that order.  On failure returns
+ * PL_ERR_INVALID_SCHEDULE and writes a message into msg (may be NULL). */
+pl_status_t pl_schedule_validate(pl_schedule_t s, char* msg, size_t msg_cap);
+
+/* TEST HOOK: corrupt one wait edge of a built schedule so that it can never be satisfied
+ * (raises the needed count of op `op_index`'s first wait).  Used with a short timeout_ns to
+ * exercise the bounded-wait path without hanging a GPU. */
+pl_status_t pl_schedule_debug_break_wait(pl_schedule_t s, size_t op_index);
+
+pl_status_t pl_schedule_destroy(pl_schedule_t s);
+
+/* ---- datapath ---------------------------------------------------------------------- */
+
+/* Run the schedule once over `bufs` on `stream` (asynchronous, one kernel launch).
+ * Errors (all before launch): PL_ERR_INVALID_ARG (NULL pointer, buffer smaller than
+ * pl_schedule_info reports, in/out ranges that overlap), PL_ERR_ALIGNMENT (a pointer not
+ * 16-byte aligned), PL_ERR_UNSUPPORTED (planner communicator), PL_ERR_CUDA (launch). */
+pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream);
+
+/* End-to-end form for callers whose data lives in HOST memory: copies host->in[r] into
+ * dev->in[r] (cudaMemcpyAsync on `stream`; pinned memory makes it truly asynchronous), runs
+ * the schedule, and copies dev->out[r] back into host->out[r].  `dev` supplies the device
+ * staging buffers (caller-owned).  Sizes come from pl_schedule_info. */
+pl_status_t pl_execute_host(pl_schedule_t s, const pl_bufs_t* host, const pl_bufs_t* dev,
+                            void* stream);
+
+/* ---- MoE expert-parallel dispatch / combine (all-to-all-v of token rows) ------------ */
+
+/* Plan for R ranks x tokens_per_rank tokens of `hidden` elements (comm dtype, row bytes a
+ * multiple of 16), n_experts experts (n_experts % R == 0, expert e lives on rank
+ * e / (n_experts/R)), topk distinct experts per token (topk <= 32).  recv_capacity_rows =
+ * rows each rank's receive buffer can hold.  The plan owns device scratch for counts,
+ * offsets and the row positions that combine reuses. */
+pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, int n_experts,
+                               int topk, size_t recv_capacity_rows, pl_moe_plan_t* out);
+pl_status_t pl_moe_plan_destroy(pl_moe_plan_t plan);
+
+/* Dispatch (Table 2, expert parallelism: scatteredV -> transposedV).  Host arrays of R
+ * DEVICE pointers: x[p] rows [T][hidden]; topk_idx[p] int32 [T][topk]; recv[r] rows
+ * [recv_capacity_rows][hidden]; recv_meta[r] int32 [recv_capacity_rows][4] =
+ * (source rank, token, slot, expert) per received row (may be NULL to skip).
+ * One row is sent per (token, slot); rank r receives rows ordered by (source rank,
+ * expert, token).  Counts and offsets are computed on the device (histogram + exclusive
+ * scans).  Rows beyond recv_capacity_rows are dropped and flagged (pl_moe_plan_read
+ * returns PL_ERR_OVERFLOW). */
+pl_status_t pl_moe_dispatch(pl_moe_plan_t plan, const void* const* x,
+                            const int32_t* const* topk_idx, void* const* recv,
+                            int32_t* const* recv_meta, void* stream);
+
+/* Combine: out[p][t][:] = sum_{j<topk} gates[p][t][j] * y[rank(e_j)][pos(p,t,j)][:] in fp32,
+ * ascending j, one final conversion; y has the layout dispatch produced, pos is the row
+ * dispatch wrote for (p,t,j).  Must follow a dispatch on the same plan (it reuses pos). */
+pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float* const* gates,
+                           void* const* out, void* stream);
+
+/* Synchronise `stream` and copy the plan's bookkeeping to HOST arrays (any may be NULL):
+ * pos int32 [R][T][topk]; counts int64 [R][R] rows src->dst; expert_counts int64
+ * [R][n_experts].  Returns PL_ERR_OVERFLOW if the last dispatch dropped rows. */
+pl_status_t pl_moe_plan_read(pl_moe_plan_t plan, int32_t* pos, int64_t* counts,
+                             int64_t* expert_counts, void* stream);
+
+const char* pl_status_string(pl_status_t st);
+
+/* Number of kernels this library has launched in the calling process (all entry points). */
+uint64_t pl_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PURLIN_H_ */

@@ -1,0 +1,513 @@
+// C-ABI layer: handles, argument checks, device upload of a lowered schedule, launches.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "pl_api_internal.h"
+#include "pl_internal.h"
+#include "pl_kernels.h"
+
+using namespace pl;
+
+namespace pl {
+std::atomic<uint64_t> g_launches{0};
+}
+
+struct pl_schedule_s {
+  pl_comm_t comm = nullptr;
+  Lowered L;
+  Policy pol{};
+  pl_sched_info_t info{};
+  uint64_t timeout_ns = 0;
+  // host copies in device (queue-major) order
+  std::vector<DevOp> dev_ops;
+  std::vector<uint32_t> queue_begin;
+  std::vector<uint64_t> srcs;
+  std::vector<DevWait> waits;
+  std::vector<int> topo_to_dev;  // topological index -> position in dev_ops
+  uint32_t src_stride = 1, wait_stride = 1;
+  // device
+  char* d_blob = nullptr;
+  size_t blob_bytes = 0;
+  size_t off_ops = 0, off_qb = 0, off_srcs = 0, off_waits = 0, off_flags = 0, off_epoch = 0;
+  size_t sync_bytes = 0;  // flags + epoch, zeroed at build and by reset
+  char* d_scratch = nullptr;
+  uint64_t scratch_off[PL_MAX_RANKS] = {0};
+};
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+uint64_t pack(const pl_schedule_s& S, const pl_ref_t& r) {
+  int slot = r.buf == PL_BUF_IN ? kSlotIn + r.rank : r.buf == PL_BUF_OUT ? kSlotOut + r.rank : kSlotScratch + r.rank;
+  return ((uint64_t)slot << 48) | r.offset;
+}
+
+void fill_info(pl_schedule_s* S, int R) {
+  pl_sched_info_t& I = S->info;
+  std::memset(&I, 0, sizeof(I));
+  const Lowered& L = S->L;
+  I.n_ops = L.ops.size();
+  I.n_queues = S->pol.n_ctas;
+  I.n_flags = L.n_flags;
+  I.n_layers = L.n_layers;
+  for (const HostOp& op : L.ops) {
+    I.n_waits += op.waits.size();
+    for (const pl_ref_t& s : op.src) I.bytes_read += op.count * elem_size(s.dtype);
+    I.bytes_written += op.count * elem_size(op.dst.dtype) * (op.bcast ? R : 1);
+  }
+  I.message_bytes = L.message_bytes;
+  for (int r = 0; r < R; ++r) {
+    I.scratch_bytes += L.scratch_per_rank[r];
+    I.in_bytes[r] = L.in_bytes[r];
+    I.out_bytes[r] = L.out_bytes[r];
+  }
+  I.grid = S->pol.n_ctas;
+  I.threads = S->pol.threads;
+  I.smem_bytes = 0;
+  I.datapath = S->pol.datapath;
+  I.stages = S->pol.stages;
+  I.stage_bytes = S->pol.stage_bytes;
+  I.slice_bytes = S->pol.slice_bytes;
+}
+
+// Flatten the lowered ops into the queue-major device arrays (host side).
+void flatten(pl_schedule_s* S, int dtype) {
+  const Lowered& L = S->L;
+  const int nq = S->pol.n_ctas;
+  size_t max_src = 1, max_wait = 1;
+  std::vector<uint32_t> qcount(nq + 1, 0);
+  for (const HostOp& op : L.ops) {
+    max_src = std::max(max_src, op.src.size());
+    max_wait = std::max(max_wait, op.waits.size());
+    qcount[op.queue + 1]++;
+  }
+  S->src_stride = (uint32_t)max_src;
+  S->wait_stride = (uint32_t)max_wait;
+  S->queue_begin.assign(nq + 1, 0);
+  for (int q = 0; q < nq; ++q) S->queue_begin[q + 1] = S->queue_begin[q] + qcount[q + 1];
+  std::vector<uint32_t> cursor(S->queue_begin.begin(), S->queue_begin.end() - 1);
+  const size_t n = L.ops.size();
+  S->dev_ops.assign(n, DevOp{});
+  S->srcs.assign(n * max_src, 0);
+  S->waits.assign(n * max_wait, DevWait{0, 0});
+  S->topo_to_dev.assign(n, 0);
+  for (const HostOp& op : L.ops) {  // topological order => per-queue order is a subsequence
+    const uint32_t pos = cursor[op.queue]++;
+    S->topo_to_dev[op.topo] = (int)pos;
+    DevOp& d = S->dev_ops[pos];
+    d.kind = op.kind;
+    d.n_src = (uint32_t)op.src.size();
+    d.n_wait = (uint32_t)op.waits.size();
+    d.signal = op.signal >= 0 ? (uint32_t)op.signal : kNoFlag;
+    d.signal2 = op.signal2 >= 0 ? (uint32_t)op.signal2 : kNoFlag;
+    d.flags = (op.bcast ? kDstBcast : 0u) | ((dtype == PL_BF16 && op.dst.dtype == PL_F32) ? kDstF32 : 0u);
+    d.count = op.count;
+    d.dst = pack(*S, op.dst);
+    d.topo = (uint32_t)op.topo;
+    for (size_t k = 0; k < op.src.size(); ++k) {
+      S->srcs[pos * max_src + k] = pack(*S, op.src[k]);
+      if (dtype == PL_BF16 && op.src[k].dtype == PL_F32) d.src_f32_mask |= 1u << k;
+    }
+    for (size_t k = 0; k < op.waits.size(); ++k)
+      S->waits[pos * max_wait + k] = DevWait{(uint32_t)op.waits[k], L.flag_need[op.waits[k]]};
+  }
+}
+
+pl_status_t upload(pl_schedule_s* S, int R) {
+  size_t off = 0;
+  auto place = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + std::max<size_t>(bytes, 16), 256);
+    return o;
+  };
+  S->off_ops = place(S->dev_ops.size() * sizeof(DevOp));
+  S->off_qb = place(S->queue_begin.size() * sizeof(uint32_t));
+  S->off_srcs = place(S->srcs.size() * sizeof(uint64_t));
+  S->off_waits = place(S->waits.size() * sizeof(DevWait));
+  S->off_flags = place((size_t)std::max(1, S->L.n_flags) * sizeof(unsigned long long));
+  S->off_epoch = place(2 * sizeof(unsigned long long));
+  S->sync_bytes = off - S->off_flags;
+  S->blob_bytes = off;
+  if (cudaMalloc(&S->d_blob, S->blob_bytes) != cudaSuccess) { cudaGetLastError(); return PL_ERR_OOM; }
+  std::vector<char> host(S->blob_bytes, 0);
+  std::memcpy(host.data() + S->off_ops, S->dev_ops.data(), S->dev_ops.size() * sizeof(DevOp));
+  std::memcpy(host.data() + S->off_qb, S->queue_begin.data(), S->queue_begin.size() * sizeof(uint32_t));
+  std::memcpy(host.data() + S->off_srcs, S->srcs.data(), S->srcs.size() * sizeof(uint64_t));
+  std::memcpy(host.data() + S->off_waits, S->waits.data(), S->waits.size() * sizeof(DevWait));
+  if (cudaMemcpy(S->d_blob, host.data(), S->blob_bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    return PL_ERR_CUDA;
+  }
+  uint64_t total = 0;
+  for (int r = 0; r < R; ++r) {
+    S->scratch_off[r] = total;
+    total += align_up(S->L.scratch_per_rank[r], 256);
+  }
+  if (total) {
+    if (cudaMalloc(&S->d_scratch, total) != cudaSuccess) { cudaGetLastError(); return PL_ERR_OOM; }
+  }
+  return PL_OK;
+}
+
+pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t* opts, pl_schedule_t* out) {
+  if (!comm || !out) return PL_ERR_INVALID_ARG;
+  *out = nullptr;
+  Policy pol{};
+  uint64_t timeout = 2000000000ull;
+  uint32_t flags = 0;
+  if (opts) {
+    if (opts->struct_size != sizeof(pl_sched_opts_t)) return PL_ERR_INVALID_ARG;
+    pol.n_ctas = opts->n_ctas;
+    pol.threads = opts->threads;
+    pol.datapath = opts->datapath;
+    pol.stages = opts->stages;
+    pol.stage_bytes = opts->stage_bytes;
+    pol.slice_bytes = opts->slice_bytes;
+    if (opts->timeout_ns) timeout = opts->timeout_ns;
+    flags = opts->flags;
+    if (pol.threads < 0 || pol.threads % 32 || pol.threads > exec_max_threads()) return PL_ERR_INVALID_ARG;
+    if (pol.n_ctas < 0 || pol.stages < 0 || pol.stage_bytes % 16 || pol.slice_bytes % 16) return PL_ERR_INVALID_ARG;
+    if (pol.datapath < PL_DP_AUTO || pol.datapath > PL_DP_TMA) return PL_ERR_INVALID_ARG;
+  }
+  rq.R = comm->R;
+  rq.dtype = comm->dtype;
+  rq.pol = pol;
+  const int threads = pol.threads > 0 ? pol.threads : 512;
+  int capacity = 148;
+  if (!comm->planner) {
+    int per_sm = exec_max_ctas_per_sm(comm->dtype, threads);
+    if (per_sm <= 0) return PL_ERR_CUDA;
+    capacity = per_sm * comm->sm_count;
+  }
+  const int requested = pol.n_ctas;
+  pol = default_policy(rq, capacity);
+  if (requested > capacity) return PL_ERR_OVERSUBSCRIBED;
+  if (pol.n_ctas > capacity) return PL_ERR_OVERSUBSCRIBED;
+  rq.pol = pol;
+
+  pl_schedule_s* S = new (std::nothrow) pl_schedule_s();
+  if (!S) return PL_ERR_OOM;
+  S->comm = comm;
+  S->pol = pol;
+  S->timeout_ns = timeout;
+  std::string err;
+  pl_status_t st = lower(rq, &S->L, &err);
+  if (st != PL_OK) {
+    comm->last_error = err;
+    delete S;
+    return st;
+  }
+  assign_queues(&S->L, comm->R, pol.n_ctas);
+  if (!(flags & PL_OPT_SKIP_VALIDATE)) {
+    st = validate(S->L, comm->R, &err);
+    if (st != PL_OK) {
+      comm->last_error = err;
+      delete S;
+      return st;
+    }
+  }
+  fill_info(S, comm->R);
+  flatten(S, comm->dtype);
+  if (!comm->planner) {
+    st = upload(S, comm->R);
+    if (st != PL_OK) {
+      pl_schedule_destroy(S);
+      return st;
+    }
+  }
+  {
+    std::lock_guard<std::mutex> g(comm->mu);
+    comm->schedules.push_back(S);
+  }
+  *out = S;
+  return PL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pl_status_string(pl_status_t st) {
+  switch (st) {
+    case PL_OK: return "ok";
+    case PL_ERR_INVALID_ARG: return "invalid argument";
+    case PL_ERR_UNSUPPORTED: return "unsupported";
+    case PL_ERR_ALIGNMENT: return "misaligned pointer or size";
+    case PL_ERR_OOM: return "out of memory";
+    case PL_ERR_CUDA: return "CUDA error";
+    case PL_ERR_TIMEOUT: return "device-side wait timed out";
+    case PL_ERR_OVERSUBSCRIBED: return "more CTAs than can be co-resident";
+    case PL_ERR_INVALID_SCHEDULE: return "schedule failed validation";
+    case PL_ERR_OVERFLOW: return "receive capacity exceeded";
+    default: return "unknown status";
+  }
+}
+
+uint64_t pl_launch_count(void) { return g_launches.load(); }
+
+static pl_status_t comm_create(int R, pl_dtype_t dtype, bool planner, pl_comm_t* out) {
+  if (!out) return PL_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (R < 2 || R > PL_MAX_RANKS) return PL_ERR_INVALID_ARG;
+  if (dtype < PL_BF16 || dtype > PL_U8) return PL_ERR_INVALID_ARG;
+  pl_comm_s* c = new (std::nothrow) pl_comm_s();
+  if (!c) return PL_ERR_OOM;
+  c->R = R;
+  c->dtype = dtype;
+  c->planner = planner;
+  if (!planner) {
+    if (cudaGetDevice(&c->device) != cudaSuccess) { cudaGetLastError(); delete c; return PL_ERR_CUDA; }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) { cudaGetLastError(); delete c; return PL_ERR_CUDA; }
+    c->sm_count = prop.multiProcessorCount;
+    if (cudaMalloc(&c->d_status, kStatusWords * sizeof(int)) != cudaSuccess) { cudaGetLastError(); delete c; return PL_ERR_OOM; }
+    if (cudaMemset(c->d_status, 0, kStatusWords * sizeof(int)) != cudaSuccess) { cudaGetLastError(); cudaFree(c->d_status); delete c; return PL_ERR_CUDA; }
+  }
+  *out = c;
+  return PL_OK;
+}
+
+pl_status_t pl_comm_create(int R, pl_dtype_t dtype, pl_comm_t* out) { return comm_create(R, dtype, false, out); }
+pl_status_t pl_comm_create_planner(int R, pl_dtype_t dtype, pl_comm_t* out) { return comm_create(R, dtype, true, out); }
+
+pl_status_t pl_comm_destroy(pl_comm_t comm) {
+  if (!comm) return PL_ERR_INVALID_ARG;
+  if (!comm->schedules.empty() || comm->n_plans != 0) return PL_ERR_INVALID_ARG;
+  if (comm->d_status) cudaFree(comm->d_status);
+  delete comm;
+  return PL_OK;
+}
+
+pl_status_t pl_comm_status(pl_comm_t comm, pl_devstatus_t* out) {
+  if (!comm || !out) return PL_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  if (comm->planner) return PL_OK;
+  int words[kStatusWords];
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  if (cudaMemcpy(words, comm->d_status, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  out->code = words[0];
+  out->queue = words[1];
+  out->op = words[2];
+  out->flag = words[3];
+  std::memcpy(&out->expected, words + 4, 8);
+  std::memcpy(&out->observed, words + 6, 8);
+  return PL_OK;
+}
+
+pl_status_t pl_comm_reset(pl_comm_t comm, void* stream) {
+  if (!comm) return PL_ERR_INVALID_ARG;
+  if (comm->planner) return PL_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(comm->d_status, 0, kStatusWords * sizeof(int), st) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  std::lock_guard<std::mutex> g(comm->mu);
+  for (pl_schedule_s* S : comm->schedules)
+    if (S->d_blob && cudaMemsetAsync(S->d_blob + S->off_flags, 0, S->sync_bytes, st) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  return PL_OK;
+}
+
+pl_status_t pl_schedule_build(pl_comm_t comm, pl_collective_t coll, pl_algo_t algo, size_t count_per_rank,
+                              size_t chunk_bytes, const pl_sched_opts_t* opts, pl_schedule_t* out) {
+  if (coll == PL_ALLTOALLV) return PL_ERR_INVALID_ARG;
+  BuildRequest rq{};
+  rq.coll = coll;
+  rq.algo = algo;
+  rq.count_per_rank = count_per_rank;
+  rq.chunk_bytes = chunk_bytes;
+  return build_common(comm, rq, opts, out);
+}
+
+pl_status_t pl_schedule_build_v(pl_comm_t comm, pl_collective_t coll, pl_algo_t algo, const size_t* counts,
+                                size_t chunk_bytes, const pl_sched_opts_t* opts, pl_schedule_t* out) {
+  if (!comm || !counts) return PL_ERR_INVALID_ARG;
+  if (coll != PL_ALLTOALLV) return PL_ERR_UNSUPPORTED;
+  std::vector<uint64_t> c((size_t)comm->R * comm->R);
+  for (size_t i = 0; i < c.size(); ++i) c[i] = counts[i];
+  BuildRequest rq{};
+  rq.coll = coll;
+  rq.algo = algo;
+  rq.chunk_bytes = chunk_bytes;
+  rq.counts_v = c.data();
+  return build_common(comm, rq, opts, out);
+}
+
+pl_status_t pl_schedule_build_layers(pl_comm_t comm, pl_algo_t algo, size_t count_per_rank, int n_layers,
+                                     const pl_sched_opts_t* opts, pl_schedule_t* out) {
+  if (n_layers < 1) return PL_ERR_INVALID_ARG;
+  BuildRequest rq{};
+  rq.coll = PL_ALLREDUCE;
+  rq.algo = algo;
+  rq.count_per_rank = count_per_rank;
+  rq.n_layers = n_layers;
+  // a layer is one chunk per partition: the latency path does not pipeline inside a layer
+  rq.chunk_bytes = ((uint64_t)1 << 40);
+  return build_common(comm, rq, opts, out);
+}
+
+pl_status_t pl_schedule_info(pl_schedule_t s, pl_sched_info_t* out) {
+  if (!s || !out) return PL_ERR_INVALID_ARG;
+  *out = s->info;
+  return PL_OK;
+}
+
+pl_status_t pl_schedule_dump(pl_schedule_t s, pl_op_t* ops, size_t cap, size_t* n) {
+  if (!s || !n) return PL_ERR_INVALID_ARG;
+  *n = s->L.ops.size();
+  if (!ops) return PL_OK;
+  const size_t m = std::min(cap, s->L.ops.size());
+  for (size_t i = 0; i < m; ++i) {
+    const HostOp& h = s->L.ops[i];
+    pl_op_t& o = ops[i];
+    std::memset(&o, 0, sizeof(o));
+    o.kind = h.kind;
+    o.exec_rank = h.exec_rank;
+    o.queue = h.queue;
+    o.topo = h.topo;
+    o.layer = h.layer;
+    o.n_src = (int32_t)h.src.size();
+    o.n_wait = (int32_t)h.waits.size();
+    o.signal_flag = h.signal;
+    o.signal_flag2 = h.signal2;
+    o.dst_bcast = h.bcast ? 1 : 0;
+    o.count = h.count;
+    o.dst = h.dst;
+    for (size_t k = 0; k < h.src.size(); ++k) o.src[k] = h.src[k];
+    for (size_t k = 0; k < h.waits.size(); ++k) {
+      o.wait_flag[k] = h.waits[k];
+      o.wait_need[k] = s->L.flag_need[h.waits[k]];
+    }
+  }
+  return PL_OK;
+}
+
+pl_status_t pl_schedule_validate(pl_schedule_t s, char* msg, size_t msg_cap) {
+  if (!s) return PL_ERR_INVALID_ARG;
+  std::string err;
+  pl_status_t st = validate(s->L, s->comm->R, &err);
+  if (msg && msg_cap) {
+    std::snprintf(msg, msg_cap, "%s", err.c_str());
+  }
+  return st;
+}
+
+pl_status_t pl_schedule_debug_break_wait(pl_schedule_t s, size_t op_index) {
+  if (!s || op_index >= s->L.ops.size()) return PL_ERR_INVALID_ARG;
+  const HostOp& h = s->L.ops[op_index];
+  if (h.waits.empty()) return PL_ERR_INVALID_ARG;
+  const size_t pos = (size_t)s->topo_to_dev[op_index];
+  DevWait& w = s->waits[pos * s->wait_stride];
+  w.need += 1;  // one more signal than the schedule will ever produce
+  if (s->d_blob) {
+    if (cudaMemcpy(s->d_blob + s->off_waits + (pos * s->wait_stride) * sizeof(DevWait), &w, sizeof(DevWait),
+                   cudaMemcpyHostToDevice) != cudaSuccess) {
+      cudaGetLastError();
+      return PL_ERR_CUDA;
+    }
+  }
+  return PL_OK;
+}
+
+pl_status_t pl_schedule_destroy(pl_schedule_t s) {
+  if (!s) return PL_ERR_INVALID_ARG;
+  if (s->d_blob) cudaFree(s->d_blob);
+  if (s->d_scratch) cudaFree(s->d_scratch);
+  if (s->comm) {
+    std::lock_guard<std::mutex> g(s->comm->mu);
+    auto& v = s->comm->schedules;
+    for (size_t i = 0; i < v.size(); ++i)
+      if (v[i] == s) { v.erase(v.begin() + i); break; }
+  }
+  delete s;
+  return PL_OK;
+}
+
+static pl_status_t check_bufs(pl_schedule_t s, const pl_bufs_t* b) {
+  const int R = s->comm->R;
+  for (int r = 0; r < R; ++r) {
+    const bool need_in = s->info.in_bytes[r] > 0, need_out = s->info.out_bytes[r] > 0;
+    if ((need_in && !b->in[r]) || (need_out && !b->out[r])) return PL_ERR_INVALID_ARG;
+    if (((uintptr_t)b->in[r] & 15) || ((uintptr_t)b->out[r] & 15)) return PL_ERR_ALIGNMENT;
+    if (b->in_bytes[r] < s->info.in_bytes[r] || b->out_bytes[r] < s->info.out_bytes[r]) return PL_ERR_INVALID_ARG;
+  }
+  // outputs must not overlap any input or another output (all collectives are out of place)
+  for (int r = 0; r < R; ++r) {
+    const uintptr_t olo = (uintptr_t)b->out[r], ohi = olo + s->info.out_bytes[r];
+    if (olo == ohi) continue;
+    for (int p = 0; p < R; ++p) {
+      const uintptr_t ilo = (uintptr_t)b->in[p], ihi = ilo + s->info.in_bytes[p];
+      if (ilo < ohi && olo < ihi) return PL_ERR_INVALID_ARG;
+      if (p != r) {
+        const uintptr_t qlo = (uintptr_t)b->out[p], qhi = qlo + s->info.out_bytes[p];
+        if (qlo < ohi && olo < qhi) return PL_ERR_INVALID_ARG;
+      }
+    }
+  }
+  return PL_OK;
+}
+
+pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
+  if (!s || !bufs) return PL_ERR_INVALID_ARG;
+  if (s->comm->planner || !s->d_blob) return PL_ERR_UNSUPPORTED;
+  pl_status_t st = check_bufs(s, bufs);
+  if (st != PL_OK) return st;
+  ExecParams P;
+  std::memset(&P, 0, sizeof(P));
+  const int R = s->comm->R;
+  for (int r = 0; r < R; ++r) {
+    P.base[kSlotIn + r] = const_cast<void*>(bufs->in[r]);
+    P.base[kSlotOut + r] = bufs->out[r];
+    P.base[kSlotScratch + r] = s->d_scratch ? s->d_scratch + s->scratch_off[r] : nullptr;
+  }
+  P.ops = reinterpret_cast<const DevOp*>(s->d_blob + s->off_ops);
+  P.queue_begin = reinterpret_cast<const uint32_t*>(s->d_blob + s->off_qb);
+  P.srcs = reinterpret_cast<const uint64_t*>(s->d_blob + s->off_srcs);
+  P.waits = reinterpret_cast<const DevWait*>(s->d_blob + s->off_waits);
+  P.src_stride = s->src_stride;
+  P.wait_stride = s->wait_stride;
+  P.flags = reinterpret_cast<unsigned long long*>(s->d_blob + s->off_flags);
+  P.epoch = reinterpret_cast<unsigned long long*>(s->d_blob + s->off_epoch);
+  P.status = s->comm->d_status;
+  P.timeout_ns = s->timeout_ns;
+  P.n_ranks = R;
+  if (launch_exec(s->comm->dtype, P, s->pol.n_ctas, s->pol.threads, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return PL_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return PL_OK;
+}
+
+pl_status_t pl_execute_host(pl_schedule_t s, const pl_bufs_t* host, const pl_bufs_t* dev, void* stream) {
+  if (!s || !host || !dev) return PL_ERR_INVALID_ARG;
+  if (s->comm->planner || !s->d_blob) return PL_ERR_UNSUPPORTED;
+  pl_status_t st = check_bufs(s, dev);
+  if (st != PL_OK) return st;
+  const int R = s->comm->R;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  for (int r = 0; r < R; ++r) {
+    if (host->in_bytes[r] < s->info.in_bytes[r] || host->out_bytes[r] < s->info.out_bytes[r]) return PL_ERR_INVALID_ARG;
+    if ((s->info.in_bytes[r] && !host->in[r]) || (s->info.out_bytes[r] && !host->out[r])) return PL_ERR_INVALID_ARG;
+  }
+  for (int r = 0; r < R; ++r)
+    if (s->info.in_bytes[r] &&
+        cudaMemcpyAsync(const_cast<void*>(dev->in[r]), host->in[r], s->info.in_bytes[r], cudaMemcpyHostToDevice, cs) != cudaSuccess) {
+      cudaGetLastError();
+      return PL_ERR_CUDA;
+    }
+  st = pl_execute(s, dev, stream);
+  if (st != PL_OK) return st;
+  for (int r = 0; r < R; ++r)
+    if (s->info.out_bytes[r] &&
+        cudaMemcpyAsync(host->out[r], dev->out[r], s->info.out_bytes[r], cudaMemcpyDeviceToHost, cs) != cudaSuccess) {
+      cudaGetLastError();
+      return PL_ERR_CUDA;
+    }
+  return PL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,437 @@
+// Datapath: one persistent kernel; CTA q interprets op queue q.
+//
+// Per op: wait (acquire) on the op's flags -> body (copy / reduce / copy-reduce with 128-bit
+// accesses, fp32 accumulation in ascending source order, Sec. 3.3 Eq. "rank-order") ->
+// signal (release).  Flags are 64-bit counters that only grow: execute number e expects
+// e * need signals, so nothing is reset between executes and the epoch lives on the device
+// (Sec. 4.2 keeps a persistent epoch for the same reason).  Every wait is bounded by a
+// globaltimer limit; on expiry the CTA records a status, raises the abort word that every
+// waiter also polls, and the kernel returns normally.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "pl_internal.h"
+#include "pl_kernels.h"
+
+namespace pl {
+namespace {
+
+constexpr int kMaxThreads = 512;
+
+// ---- small PTX helpers ---------------------------------------------------------------
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ int ld_volatile_s32(const int* p) {
+  int v;
+  asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint4 ld16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st16(void* p, const uint4& v) {
+  asm volatile("st.global.cg.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+__device__ __forceinline__ char* resolve(const ExecParams& P, uint64_t packed) {
+  return static_cast<char*>(P.base[packed >> 48]) + (packed & 0xFFFFFFFFFFFFull);
+}
+
+// ---- element arithmetic ----------------------------------------------------------------
+// A "unit" is the group of elements one 16-byte vector of the narrowest operand holds:
+// 8 elements for bf16 schedules, 4 for fp32 / int32.
+template <int DT>
+struct Acc;
+
+template <>
+struct Acc<PL_BF16> {
+  static constexpr int kElems = 8;
+  float v[8];
+  __device__ __forceinline__ void zero() {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = 0.f;
+  }
+  __device__ __forceinline__ void add_bf16(const uint4& q) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] += __uint_as_float(w[i] << 16);
+      v[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+  __device__ __forceinline__ void add_f32(const uint4& lo, const uint4& hi) {
+    v[0] += __uint_as_float(lo.x); v[1] += __uint_as_float(lo.y);
+    v[2] += __uint_as_float(lo.z); v[3] += __uint_as_float(lo.w);
+    v[4] += __uint_as_float(hi.x); v[5] += __uint_as_float(hi.y);
+    v[6] += __uint_as_float(hi.z); v[7] += __uint_as_float(hi.w);
+  }
+  __device__ __forceinline__ uint4 to_bf16() const {
+    uint4 q;
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
+    __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
+    __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]);
+    __nv_bfloat162 d = __floats2bfloat162_rn(v[6], v[7]);
+    q.x = *reinterpret_cast<uint32_t*>(&a);
+    q.y = *reinterpret_cast<uint32_t*>(&b);
+    q.z = *reinterpret_cast<uint32_t*>(&c);
+    q.w = *reinterpret_cast<uint32_t*>(&d);
+    return q;
+  }
+};
+
+// fp32 data: compensated (Kahan-Neumaier style two-sum) accumulation, still one
+// accumulator per element and ascending source order; the correction is folded in once at
+// the end.  Keeps the result inside the fp32 tolerance for any input mantissas.
+template <>
+struct Acc<PL_F32> {
+  static constexpr int kElems = 4;
+  float v[4], c[4];
+  __device__ __forceinline__ void zero() {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = c[i] = 0.f;
+  }
+  __device__ __forceinline__ void add(const uint4& q) {
+    const float x[4] = {__uint_as_float(q.x), __uint_as_float(q.y), __uint_as_float(q.z), __uint_as_float(q.w)};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float s = __fadd_rn(v[i], x[i]);
+      float bp = __fsub_rn(s, v[i]);
+      float err = __fadd_rn(__fsub_rn(v[i], __fsub_rn(s, bp)), __fsub_rn(x[i], bp));
+      c[i] = __fadd_rn(c[i], err);
+      v[i] = s;
+    }
+  }
+  __device__ __forceinline__ uint4 result() const {
+    uint4 q;
+    q.x = __float_as_uint(__fadd_rn(v[0], c[0]));
+    q.y = __float_as_uint(__fadd_rn(v[1], c[1]));
+    q.z = __float_as_uint(__fadd_rn(v[2], c[2]));
+    q.w = __float_as_uint(__fadd_rn(v[3], c[3]));
+    return q;
+  }
+};
+
+template <>
+struct Acc<PL_I32> {
+  static constexpr int kElems = 4;
+  uint32_t v[4];
+  __device__ __forceinline__ void zero() { v[0] = v[1] = v[2] = v[3] = 0u; }
+  __device__ __forceinline__ void add(const uint4& q) {
+    v[0] += q.x; v[1] += q.y; v[2] += q.z; v[3] += q.w;
+  }
+  __device__ __forceinline__ uint4 result() const { return make_uint4(v[0], v[1], v[2], v[3]); }
+};
+
+// ---- op bodies (register path: unrolled 128-bit loads, then stores) -----------------------
+__device__ __forceinline__ void body_copy(char* dst, const char* src, uint64_t bytes, int tid, int nthr) {
+  const uint64_t n = bytes >> 4;
+  constexpr int U = 8;
+  uint64_t i = tid;
+  for (; i + (uint64_t)(U - 1) * nthr < n; i += (uint64_t)U * nthr) {
+    uint4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) v[u] = ld16(src + ((i + (uint64_t)u * nthr) << 4));
+#pragma unroll
+    for (int u = 0; u < U; ++u) st16(dst + ((i + (uint64_t)u * nthr) << 4), v[u]);
+  }
+  for (; i < n; i += nthr) st16(dst + (i << 4), ld16(src + (i << 4)));
+}
+
+// Add NB same-typed sources (ascending) for U units at once: all loads first, then the adds.
+template <int DT, int NB, int U>
+__device__ __forceinline__ void accumulate_batch(Acc<DT> (&acc)[U], const char* const* src, const uint64_t (&off)[U]) {
+  uint4 q[U][NB];
+#pragma unroll
+  for (int u = 0; u < U; ++u)
+#pragma unroll
+    for (int s = 0; s < NB; ++s) q[u][s] = ld16(src[s] + off[u]);
+#pragma unroll
+  for (int u = 0; u < U; ++u)
+#pragma unroll
+    for (int s = 0; s < NB; ++s) {
+      if constexpr (DT == PL_BF16) acc[u].add_bf16(q[u][s]);
+      else acc[u].add(q[u][s]);
+    }
+}
+
+// Reduce U units (unit index first + u*stride) from ns sources and store the result.
+template <int DT, int U>
+__device__ __forceinline__ void reduce_units(const ExecParams& P, const char* const* s_src, int ns, char* dst,
+                                             uint64_t dst_off, bool bcast, uint64_t first, uint64_t stride) {
+  Acc<DT> acc[U];
+  uint64_t off[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    acc[u].zero();
+    off[u] = (first + (uint64_t)u * stride) << 4;
+  }
+  int s = 0;
+#pragma unroll 1
+  for (; s + 4 <= ns; s += 4) accumulate_batch<DT, 4, U>(acc, s_src + s, off);
+  if (s + 2 <= ns) { accumulate_batch<DT, 2, U>(acc, s_src + s, off); s += 2; }
+  if (s < ns) accumulate_batch<DT, 1, U>(acc, s_src + s, off);
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    uint4 r;
+    if constexpr (DT == PL_BF16) r = acc[u].to_bf16();
+    else r = acc[u].result();
+    if (!bcast) {
+      st16(dst + off[u], r);
+    } else {
+      for (int k = 0; k < P.n_ranks; ++k) st16(static_cast<char*>(P.base[kSlotOut + k]) + dst_off + off[u], r);
+    }
+  }
+}
+
+// REDUCE with n same-typed sources -> element-typed destination (optionally replicated to
+// every rank's output).  s_src holds the resolved source pointers in shared memory.
+template <int DT>
+__device__ __forceinline__ void body_reduce(const ExecParams& P, const DevOp& op, const char* const* s_src, int tid,
+                                            int nthr) {
+  constexpr int U = 2;
+  const uint64_t n_units = op.count / Acc<DT>::kElems;  // 16 bytes of every operand each
+  const bool bcast = op.flags & kDstBcast;
+  char* dst = resolve(P, op.dst);
+  const uint64_t dst_off = op.dst & 0xFFFFFFFFFFFFull;
+  const int ns = op.n_src;
+  uint64_t base = tid;
+  for (; base + (uint64_t)(U - 1) * nthr < n_units; base += (uint64_t)U * nthr)
+    reduce_units<DT, U>(P, s_src, ns, dst, dst_off, bcast, base, nthr);
+  for (; base < n_units; base += nthr) reduce_units<DT, 1>(P, s_src, ns, dst, dst_off, bcast, base, nthr);
+}
+
+// COPY_REDUCE: dst = a + b where a and/or b may hold fp32 partials of a bf16 reduction and
+// dst may be a partial too.  For fp32 / int32 data every operand has the element type.
+template <int DT>
+__device__ __forceinline__ void body_copy_reduce(const ExecParams& P, const DevOp& op, const char* const* s_src,
+                                                 int tid, int nthr) {
+  const uint64_t n_units = op.count / Acc<DT>::kElems;
+  char* dst = resolve(P, op.dst);
+  const char* a = s_src[0];
+  const char* b = s_src[1];
+  if constexpr (DT != PL_BF16) {
+    constexpr int U = 4;
+    for (uint64_t base = tid; base < n_units; base += (uint64_t)U * nthr) {
+      uint4 qa[U], qb[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint64_t i = base + (uint64_t)u * nthr;
+        if (i < n_units) { qa[u] = ld16(a + (i << 4)); qb[u] = ld16(b + (i << 4)); }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint64_t i = base + (uint64_t)u * nthr;
+        if (i < n_units) {
+          Acc<DT> acc;
+          acc.zero();
+          acc.add(qa[u]);
+          acc.add(qb[u]);
+          st16(dst + (i << 4), acc.result());
+        }
+      }
+    }
+  } else {
+    const bool a32 = op.src_f32_mask & 1u, b32 = op.src_f32_mask & 2u, d32 = op.flags & kDstF32;
+    constexpr int U = 2;
+    for (uint64_t base = tid; base < n_units; base += (uint64_t)U * nthr) {
+      uint4 qa[U][2], qb[U][2];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint64_t i = base + (uint64_t)u * nthr;
+        if (i < n_units) {
+          if (a32) { qa[u][0] = ld16(a + (i << 5)); qa[u][1] = ld16(a + (i << 5) + 16); }
+          else qa[u][0] = ld16(a + (i << 4));
+          if (b32) { qb[u][0] = ld16(b + (i << 5)); qb[u][1] = ld16(b + (i << 5) + 16); }
+          else qb[u][0] = ld16(b + (i << 4));
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint64_t i = base + (uint64_t)u * nthr;
+        if (i < n_units) {
+          Acc<PL_BF16> acc;
+          acc.zero();
+          if (a32) acc.add_f32(qa[u][0], qa[u][1]); else acc.add_bf16(qa[u][0]);
+          if (b32) acc.add_f32(qb[u][0], qb[u][1]); else acc.add_bf16(qb[u][0]);
+          if (d32) {
+            uint4 lo = make_uint4(__float_as_uint(acc.v[0]), __float_as_uint(acc.v[1]), __float_as_uint(acc.v[2]), __float_as_uint(acc.v[3]));
+            uint4 hi = make_uint4(__float_as_uint(acc.v[4]), __float_as_uint(acc.v[5]), __float_as_uint(acc.v[6]), __float_as_uint(acc.v[7]));
+            st16(dst + (i << 5), lo);
+            st16(dst + (i << 5) + 16, hi);
+          } else {
+            st16(dst + (i << 4), acc.to_bf16());
+          }
+        }
+      }
+    }
+  }
+}
+
+// ---- the executor -------------------------------------------------------------------------
+struct OpSlot {
+  DevOp op;
+  const char* src[PL_MAX_SRC];
+  DevWait wait[PL_MAX_WAITS];
+};
+
+// Record a timeout (first writer wins) and raise the abort word.
+__device__ __noinline__ void record_timeout(const ExecParams& P, int queue, uint32_t topo, uint32_t flag,
+                                            unsigned long long expected, unsigned long long observed) {
+  if (atomicCAS(P.status, 0, (int)PL_ERR_TIMEOUT) == 0) {
+    P.status[1] = queue;
+    P.status[2] = (int)topo;
+    P.status[3] = (int)flag;
+    *reinterpret_cast<unsigned long long*>(P.status + 4) = expected;
+    *reinterpret_cast<unsigned long long*>(P.status + 6) = observed;
+  }
+  __threadfence();
+  atomicExch(P.status + 8, 1);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_constant__ ExecParams P) {
+  __shared__ OpSlot s_slot[2];
+  __shared__ int s_abort[2];  // indexed by iteration parity: written during wait i, read after barrier i
+  const int tid = threadIdx.x, nthr = blockDim.x, q = blockIdx.x;
+  const uint32_t qb = P.queue_begin[q], qe = P.queue_begin[q + 1];
+  // every CTA reads the epoch before it reports completion, and the epoch word is only
+  // advanced after all CTAs reported, so all of them see the same value
+  const unsigned long long epoch = *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull;
+  if (tid == 0) s_abort[0] = s_abort[1] = 0;
+  bool aborted = false;
+
+  // descriptor fetch by warp 0: lanes 0-3 carry the op, lane k source k and wait entry k
+  auto fetch = [&](uint32_t i, uint4& r_op, uint64_t& r_src, DevWait& r_wait) {
+    if (tid < 4) r_op = reinterpret_cast<const uint4*>(P.ops + i)[tid];
+    if (tid < (int)P.src_stride) r_src = P.srcs[(uint64_t)i * P.src_stride + tid];
+    if (tid < (int)P.wait_stride) r_wait = P.waits[(uint64_t)i * P.wait_stride + tid];
+  };
+  auto stash = [&](int slot, const uint4& r_op, uint64_t r_src, const DevWait& r_wait) {
+    if (tid < 4) reinterpret_cast<uint4*>(&s_slot[slot].op)[tid] = r_op;
+    if (tid < (int)P.src_stride) s_slot[slot].src[tid] = resolve(P, r_src);
+    if (tid < (int)P.wait_stride) s_slot[slot].wait[tid] = r_wait;
+  };
+
+  uint4 r_op = make_uint4(0, 0, 0, 0);
+  uint64_t r_src = 0;
+  DevWait r_wait = {0, 0};
+  if (tid < 32 && qb < qe) {
+    fetch(qb, r_op, r_src, r_wait);
+    stash(0, r_op, r_src, r_wait);
+  }
+  __syncthreads();
+
+  for (uint32_t i = qb; i < qe; ++i) {
+    const int slot = (i - qb) & 1;
+    OpSlot& S = s_slot[slot];
+    if (tid < 32) {
+      // ---- wait: lane k polls wait entry k (acquire), bounded by the time limit
+      const uint32_t nw = S.op.n_wait;
+      if (tid < (int)nw) {
+        const DevWait w = S.wait[tid];
+        const unsigned long long need = epoch * (unsigned long long)w.need;
+        const unsigned long long* fp = P.flags + w.flag;
+        unsigned long long seen = ld_acquire_u64(fp);
+        if (seen < need) {
+          const unsigned long long t0 = globaltimer_ns();
+          uint32_t spins = 0;
+          while ((seen = ld_acquire_u64(fp)) < need) {
+            if ((++spins & 63u) == 0) {
+              if (ld_volatile_s32(P.status + 8)) { s_abort[slot] = 1; break; }
+              if (globaltimer_ns() - t0 > P.timeout_ns) {
+                record_timeout(P, q, S.op.topo, w.flag, need, seen);
+                s_abort[slot] = 1;
+                break;
+              }
+            }
+          }
+        }
+      }
+      __syncwarp();
+    }
+    __syncthreads();  // descriptor + satisfied waits visible to the CTA; previous body finished
+    if (s_abort[slot]) { aborted = true; break; }
+    const bool has_next = i + 1 < qe;
+    if (tid < 32 && has_next) fetch(i + 1, r_op, r_src, r_wait);
+
+    const DevOp& op = S.op;
+    if (op.kind == PL_OP_COPY) {
+      body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
+    } else if (op.kind == PL_OP_REDUCE) {
+      if constexpr (DT != PL_U8) body_reduce<DT>(P, op, S.src, tid, nthr);
+    } else {
+      if constexpr (DT != PL_U8) body_copy_reduce<DT>(P, op, S.src, tid, nthr);
+    }
+
+    if (op.signal != kNoFlag) {
+      __syncthreads();  // every thread's writes are done
+      if (tid == 0) {
+        __threadfence();
+        red_release_add_u64(P.flags + op.signal, 1ull);
+        if (op.signal2 != kNoFlag) red_release_add_u64(P.flags + op.signal2, 1ull);
+      }
+    }
+    if (tid < 32 && has_next) {
+      stash(slot ^ 1, r_op, r_src, r_wait);
+      __syncwarp();
+    }
+  }
+
+  __syncthreads();
+  if (tid == 0 && !aborted) {
+    // last CTA to finish advances the epoch for the next execute
+    const unsigned long long prev = atomicAdd(P.epoch + 1, 1ull);
+    if (prev == (unsigned long long)gridDim.x - 1ull) {
+      P.epoch[1] = 0ull;
+      __threadfence();
+      *reinterpret_cast<volatile unsigned long long*>(P.epoch) = epoch;
+    }
+  }
+}
+
+template <int DT>
+cudaError_t launch_t(const ExecParams& P, int grid, int threads, cudaStream_t stream) {
+  pl_exec_kernel<DT><<<grid, threads, 0, stream>>>(P);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_exec(int dtype, const ExecParams& P, int grid, int threads, cudaStream_t stream) {
+  switch (dtype) {
+    case PL_BF16: return launch_t<PL_BF16>(P, grid, threads, stream);
+    case PL_F32: return launch_t<PL_F32>(P, grid, threads, stream);
+    case PL_I32: return launch_t<PL_I32>(P, grid, threads, stream);
+    default: return launch_t<PL_U8>(P, grid, threads, stream);
+  }
+}
+
+int exec_max_ctas_per_sm(int dtype, int threads) {
+  int n = 0;
+  cudaError_t e;
+  switch (dtype) {
+    case PL_BF16: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_BF16>, threads, 0); break;
+    case PL_F32: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_F32>, threads, 0); break;
+    case PL_I32: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_I32>, threads, 0); break;
+    default: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_U8>, threads, 0); break;
+  }
+  if (e != cudaSuccess) { cudaGetLastError(); return 0; }
+  return n;
+}
+
+int exec_max_threads() { return kMaxThreads; }
+
+}  // namespace pl

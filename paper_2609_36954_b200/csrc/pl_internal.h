@@ -1,0 +1,113 @@
+// Internal types shared by the host orchestrator, the C-ABI layer and the kernels.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <utility>
+#include <vector>
+
+#include "purlin.h"
+
+namespace pl {
+
+inline int elem_size(int dtype) {
+  switch (dtype) {
+    case PL_BF16: return 2;
+    case PL_F32: return 4;
+    case PL_I32: return 4;
+    default: return 1;
+  }
+}
+// Element type of partial sums that travel between ops (ring hops, tree levels).
+inline int partial_dtype(int dtype) { return dtype == PL_BF16 ? PL_F32 : dtype; }
+
+struct HostOp {
+  int kind = PL_OP_COPY;
+  int exec_rank = 0;
+  int layer = 0;
+  uint64_t count = 0;  // elements (bytes for COPY)
+  pl_ref_t dst{};
+  bool bcast = false;
+  std::vector<pl_ref_t> src;
+  std::vector<int> waits;  // flag ids
+  int signal = -1;
+  int signal2 = -1;
+  int queue = -1;
+  int topo = -1;
+};
+
+// ---- device-resident schedule ------------------------------------------------------
+// A buffer address is packed as (slot << 48) | byte offset; slot indexes the pointer
+// table passed by value in the kernel parameters: in[0..16), out[16..32), scratch[32..48).
+constexpr int kSlotIn = 0, kSlotOut = PL_MAX_RANKS, kSlotScratch = 2 * PL_MAX_RANKS;
+constexpr int kNumSlots = 3 * PL_MAX_RANKS;
+constexpr uint32_t kNoFlag = 0xFFFFFFFFu;
+
+struct alignas(16) DevOp {
+  uint32_t kind;        // pl_op_kind_t
+  uint32_t n_src;
+  uint32_t rsv0;
+  uint32_t src_f32_mask;  // bit p set: source p holds fp32 partials (bf16 schedules only)
+  uint32_t rsv1;
+  uint32_t n_wait;
+  uint32_t signal;      // flag index or kNoFlag
+  uint32_t flags;       // bit0: dst holds fp32 partials (bf16 schedules); bit1: dst broadcast
+  uint64_t count;       // elements (bytes for COPY)
+  uint64_t dst;         // packed address
+  uint32_t topo;
+  uint32_t signal2;     // second flag index or kNoFlag
+  uint32_t pad[2];
+};
+static_assert(sizeof(DevOp) == 64, "DevOp must stay 64 bytes");
+constexpr uint32_t kDstF32 = 1u, kDstBcast = 2u;
+
+struct DevWait {
+  uint32_t flag;
+  uint32_t need;
+};
+
+struct ExecParams {
+  void* base[kNumSlots];
+  const DevOp* ops;             // queue-major order
+  const uint32_t* queue_begin;  // n_queues + 1 entries
+  const uint64_t* srcs;         // src_stride packed addresses per op (same order as ops)
+  const DevWait* waits;         // wait_stride entries per op
+  uint32_t src_stride, wait_stride;
+  unsigned long long* flags;    // one 64-bit counter per flag, monotone across executes
+  unsigned long long* epoch;    // [0] executes completed, [1] CTAs finished in this execute
+  int* status;                  // pl_devstatus_t words + abort word (comm-owned)
+  unsigned long long timeout_ns;
+  int n_ranks;
+};
+
+struct Policy {
+  int n_ctas, threads, datapath, stages;
+  uint32_t stage_bytes, slice_bytes;
+};
+
+struct Lowered {
+  std::vector<HostOp> ops;  // topological order
+  int n_flags = 0;
+  std::vector<uint32_t> flag_need;  // signals per execute, per flag
+  uint64_t scratch_per_rank[PL_MAX_RANKS] = {0};
+  uint64_t in_bytes[PL_MAX_RANKS] = {0};
+  uint64_t out_bytes[PL_MAX_RANKS] = {0};
+  uint64_t message_bytes = 0;
+  int n_layers = 1;
+};
+
+struct BuildRequest {
+  int R, dtype, coll, algo;
+  uint64_t count_per_rank;
+  uint64_t chunk_bytes;
+  const uint64_t* counts_v;  // R*R for all-to-all-v, else null
+  int n_layers;              // 0: single collective
+  Policy pol;
+};
+
+// orchestrator (host only, no CUDA)
+pl_status_t lower(const BuildRequest& rq, Lowered* out, std::string* err);
+void assign_queues(Lowered* L, int R, int n_queues);
+pl_status_t validate(const Lowered& L, int R, std::string* err);
+Policy default_policy(const BuildRequest& rq, int max_resident_ctas);
+
+}  // namespace pl

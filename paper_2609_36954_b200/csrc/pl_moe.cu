@@ -1,0 +1,448 @@
+// MoE expert-parallel dispatch / combine: an all-to-all-v of token rows whose counts are
+// only known on the device (Table 2 of the paper names the pattern; Sec. 4 uses prefix sums
+// for the variable-length offsets).
+//
+// dispatch = count (per 256-token block, per expert, via bit masks) -> scan (exclusive
+// prefix sums: receive offsets in (source rank, expert, token) order) -> place (row index
+// of every (token, slot) + receive metadata) -> move (each token row is read once into
+// shared memory by a bulk async copy and written to its K destinations by K bulk stores).
+// combine = gate-weighted fp32 sum of the K expert rows of every token, ascending slot.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstring>
+#include <new>
+
+#include "pl_api_internal.h"
+#include "pl_internal.h"
+#include "pl_ptx.cuh"
+
+using namespace pl;
+
+namespace {
+
+constexpr int kTB = 256;             // tokens per count/place block
+constexpr int kMaskWords = kTB / 32;
+constexpr int kMaxTopk = 32;
+constexpr uint32_t kMaxTile = 16384;  // bytes of a row moved per bulk copy
+
+struct DispatchPtrs {
+  const void* x[PL_MAX_RANKS];
+  const int32_t* idx[PL_MAX_RANKS];
+  void* recv[PL_MAX_RANKS];
+  int32_t* meta[PL_MAX_RANKS];
+};
+struct CombinePtrs {
+  const void* y[PL_MAX_RANKS];
+  const float* gates[PL_MAX_RANKS];
+  void* out[PL_MAX_RANKS];
+};
+struct MoeGeo {
+  int R, T, E, K, NB, epr;
+  uint32_t row_bytes, tile_bytes, n_tiles, slots;
+  unsigned long long cap;
+  int32_t* blockcnt;   // [R][NB][E]: per-block counts, turned into exclusive block offsets by scan
+  int32_t* base;       // [R][E]: first row of segment (p, e) in the destination's receive buffer
+  long long* counts;   // [R][R]
+  long long* ecounts;  // [R][E]
+  int32_t* pos;        // [R][T][K] row in the destination's receive buffer, -1 if dropped
+  int32_t* prank;      // [R][T][K] destination rank
+  int* flags;          // [0] overflow, [1] invalid expert id, [2] copy engine wait gave up
+};
+
+__device__ __forceinline__ void build_mask(const MoeGeo& g, const int32_t* idx, uint32_t* mask, int t, int tid) {
+  for (int i = tid; i < g.E * kMaskWords; i += kTB) mask[i] = 0u;
+  __syncthreads();
+  if (t < g.T)
+    for (int j = 0; j < g.K; ++j) {
+      const int e = idx[(size_t)t * g.K + j];
+      if ((unsigned)e < (unsigned)g.E) atomicOr(&mask[e * kMaskWords + (tid >> 5)], 1u << (tid & 31));
+      else g.flags[1] = 1;
+    }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kTB) moe_count_kernel(const __grid_constant__ DispatchPtrs P, const __grid_constant__ MoeGeo g) {
+  extern __shared__ uint32_t mask[];
+  const int b = blockIdx.x, p = blockIdx.y, tid = threadIdx.x;
+  build_mask(g, P.idx[p], mask, b * kTB + tid, tid);
+  for (int e = tid; e < g.E; e += kTB) {
+    int c = 0;
+#pragma unroll
+    for (int w = 0; w < kMaskWords; ++w) c += __popc(mask[e * kMaskWords + w]);
+    g.blockcnt[((size_t)p * g.NB + b) * g.E + e] = c;
+  }
+}
+
+__global__ void __launch_bounds__(1024) moe_scan_kernel(const __grid_constant__ MoeGeo g) {
+  const int tid = threadIdx.x, n = blockDim.x;
+  if (tid < 3) g.flags[tid] = 0;
+  for (int pe = tid; pe < g.R * g.E; pe += n) {
+    const int p = pe / g.E, e = pe % g.E;
+    int run = 0;
+    for (int b = 0; b < g.NB; ++b) {
+      int32_t* c = g.blockcnt + ((size_t)p * g.NB + b) * g.E + e;
+      const int v = *c;
+      *c = run;
+      run += v;
+    }
+    g.ecounts[pe] = run;
+  }
+  __syncthreads();
+  for (int pr = tid; pr < g.R * g.R; pr += n) {
+    const int p = pr / g.R, r = pr % g.R;
+    long long s = 0;
+    for (int e = r * g.epr; e < (r + 1) * g.epr; ++e) s += g.ecounts[p * g.E + e];
+    g.counts[pr] = s;
+  }
+  __syncthreads();
+  for (int pe = tid; pe < g.R * g.E; pe += n) {
+    const int p = pe / g.E, e = pe % g.E, r = e / g.epr;
+    long long off = 0;
+    for (int q = 0; q < p; ++q) off += g.counts[q * g.R + r];
+    for (int e2 = r * g.epr; e2 < e; ++e2) off += g.ecounts[p * g.E + e2];
+    g.base[pe] = (int32_t)off;
+  }
+  for (int r = tid; r < g.R; r += n) {
+    long long total = 0;
+    for (int p = 0; p < g.R; ++p) total += g.counts[p * g.R + r];
+    if ((unsigned long long)total > g.cap) g.flags[0] = 1;
+  }
+}
+
+__global__ void __launch_bounds__(kTB) moe_place_kernel(const __grid_constant__ DispatchPtrs P, const __grid_constant__ MoeGeo g) {
+  extern __shared__ uint32_t mask[];
+  const int b = blockIdx.x, p = blockIdx.y, tid = threadIdx.x, t = b * kTB + tid;
+  const int32_t* idx = P.idx[p];
+  build_mask(g, idx, mask, t, tid);
+  if (t >= g.T) return;
+  const int w = tid >> 5;
+  const uint32_t below = (1u << (tid & 31)) - 1u;
+  for (int j = 0; j < g.K; ++j) {
+    const int e = idx[(size_t)t * g.K + j];
+    const size_t o = ((size_t)p * g.T + t) * g.K + j;
+    if ((unsigned)e >= (unsigned)g.E) { g.pos[o] = -1; g.prank[o] = 0; continue; }
+    int rank = __popc(mask[e * kMaskWords + w] & below);
+    for (int w2 = 0; w2 < w; ++w2) rank += __popc(mask[e * kMaskWords + w2]);
+    const long long row = (long long)g.base[p * g.E + e] + g.blockcnt[((size_t)p * g.NB + b) * g.E + e] + rank;
+    const int r = e / g.epr;
+    g.prank[o] = r;
+    if ((unsigned long long)row < g.cap) {
+      g.pos[o] = (int32_t)row;
+      if (P.meta[r]) reinterpret_cast<int4*>(P.meta[r])[row] = make_int4(p, t, j, e);
+    } else {
+      g.pos[o] = -1;
+    }
+  }
+}
+
+// One warp per CTA drives a ring of `slots` shared-memory tiles: lane 0 issues the bulk loads
+// (prime, then refill as tiles drain: the paper's Algorithm 2 with the processing step being
+// "store to K places"), lane j issues the bulk store to destination j.
+__global__ void __launch_bounds__(32) moe_move_kernel(const __grid_constant__ DispatchPtrs P, const __grid_constant__ MoeGeo g) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int lane = threadIdx.x;
+  const uint32_t S = g.slots;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);
+  unsigned char* tiles = smem + 128;
+  if (lane == 0) {
+    for (uint32_t s = 0; s < S; ++s) ptx::mbar_init(full + s, 1);
+    ptx::mbar_init_fence();
+  }
+  __syncwarp();
+  const unsigned long long n_items = (unsigned long long)g.R * g.T * g.n_tiles;
+  const unsigned long long c = blockIdx.x, G = gridDim.x;
+  if (c >= n_items) return;
+  const unsigned long long n_my = (n_items - c + G - 1) / G;
+  constexpr int L = 2;  // store groups allowed to be still reading shared memory
+
+  auto item = [&](unsigned long long n, unsigned long long& tok, uint32_t& off, uint32_t& bytes) {
+    const unsigned long long w = c + n * G;
+    tok = w / g.n_tiles;
+    const uint32_t tile = (uint32_t)(w % g.n_tiles);
+    off = tile * g.tile_bytes;
+    bytes = min(g.tile_bytes, g.row_bytes - off);
+  };
+  auto issue_load = [&](unsigned long long n) {
+    unsigned long long tok;
+    uint32_t off, bytes;
+    item(n, tok, off, bytes);
+    const int p = (int)(tok / g.T);
+    const unsigned long long t = tok % g.T;
+    const char* src = static_cast<const char*>(P.x[p]) + t * g.row_bytes + off;
+    const uint32_t s = (uint32_t)(n % S);
+    ptx::mbar_expect_tx(full + s, bytes);
+    ptx::bulk_g2s(tiles + (size_t)s * g.tile_bytes, src, bytes, full + s);
+  };
+
+  unsigned long long issued = 0;
+  if (lane == 0)
+    for (; issued < n_my && issued < S; ++issued) issue_load(issued);
+  issued = min(n_my, (unsigned long long)S);
+  bool failed = false;
+  unsigned long long n = 0;
+  for (; n < n_my; ++n) {
+    unsigned long long tok;
+    uint32_t off, bytes;
+    item(n, tok, off, bytes);
+    int row = -1, r = 0;
+    if (lane < g.K) {
+      row = g.pos[tok * g.K + lane];
+      r = g.prank[tok * g.K + lane];
+    }
+    const uint32_t s = (uint32_t)(n % S), parity = (uint32_t)((n / S) & 1);
+    // bounded wait for the tile to land
+    bool ok = ptx::mbar_try_wait(full + s, parity);
+    if (!ok) {
+      unsigned long long t0 = 0;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+      for (uint32_t tries = 1; !(ok = ptx::mbar_try_wait(full + s, parity)); ++tries) {
+        if ((tries & 1023u) == 0) {
+          unsigned long long t1;
+          asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+          if (t1 - t0 > 2000000000ull) break;
+        }
+      }
+    }
+    ok = __all_sync(0xFFFFFFFFu, ok);
+    if (!ok) { failed = true; break; }
+    if (row >= 0) ptx::bulk_s2g(static_cast<char*>(P.recv[r]) + (size_t)row * g.row_bytes + off,
+                                tiles + (size_t)s * g.tile_bytes, bytes);
+    ptx::bulk_commit();
+    if (n >= (unsigned long long)L) {
+      ptx::bulk_wait_read<L>();
+      __syncwarp();
+      const unsigned long long m = n - L;  // its tile is no longer being read
+      if (lane == 0 && m + S < n_my) issue_load(m + S);
+    }
+  }
+  ptx::bulk_wait<0>();
+  if (failed && lane == 0) {
+    g.flags[2] = 1;
+    // loads already issued may still land: give each a bounded chance before leaving
+    const unsigned long long last = min(n_my, n + S);
+    for (unsigned long long k = n; k < last; ++k) {
+      const uint32_t s = (uint32_t)(k % S), parity = (uint32_t)((k / S) & 1);
+      for (uint32_t tries = 0; tries < (1u << 20) && !ptx::mbar_try_wait(full + s, parity); ++tries) {}
+    }
+  }
+}
+
+// combine: CTA per token (grid-strided), 16-byte column units across threads, the K source
+// rows and gates of the next token are fetched while the current one is summed.
+__global__ void __launch_bounds__(256) moe_combine_kernel(const __grid_constant__ CombinePtrs P, const __grid_constant__ MoeGeo g) {
+  __shared__ const char* s_row[2][kMaxTopk];
+  __shared__ float s_gate[2][kMaxTopk];
+  const int tid = threadIdx.x;
+  const unsigned long long n_tok = (unsigned long long)g.R * g.T;
+  auto load_meta = [&](unsigned long long tok, int buf) {
+    if (tid < g.K) {
+      const int p = (int)(tok / g.T);
+      const unsigned long long t = tok % g.T;
+      const int row = g.pos[tok * g.K + tid];
+      const int r = g.prank[tok * g.K + tid];
+      s_row[buf][tid] = row >= 0 ? static_cast<const char*>(P.y[r]) + (size_t)row * g.row_bytes : nullptr;
+      s_gate[buf][tid] = P.gates[p][t * g.K + tid];
+    }
+  };
+  unsigned long long tok = blockIdx.x;
+  if (tok < n_tok) load_meta(tok, 0);
+  __syncthreads();
+  const uint32_t units = g.row_bytes >> 4;
+  for (int it = 0; tok < n_tok; tok += gridDim.x, ++it) {
+    const int buf = it & 1;
+    if (tok + gridDim.x < n_tok) load_meta(tok + gridDim.x, buf ^ 1);
+    const int p = (int)(tok / g.T);
+    char* out = static_cast<char*>(P.out[p]) + (tok % g.T) * g.row_bytes;
+    for (uint32_t u = tid; u < units; u += 256) {
+      float acc[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+      for (int j0 = 0; j0 < g.K; j0 += 8) {
+        uint4 q[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const char* rowp = (j0 + j < g.K) ? s_row[buf][j0 + j] : nullptr;
+          q[j] = rowp ? __ldcg(reinterpret_cast<const uint4*>(rowp) + u) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (j0 + j < g.K) {
+            const float gt = s_gate[buf][j0 + j];
+            const uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              acc[2 * i] = fmaf(gt, __uint_as_float(w[i] << 16), acc[2 * i]);
+              acc[2 * i + 1] = fmaf(gt, __uint_as_float(w[i] & 0xFFFF0000u), acc[2 * i + 1]);
+            }
+          }
+        }
+      }
+      uint4 o;
+      __nv_bfloat162 a = __floats2bfloat162_rn(acc[0], acc[1]);
+      __nv_bfloat162 b = __floats2bfloat162_rn(acc[2], acc[3]);
+      __nv_bfloat162 c2 = __floats2bfloat162_rn(acc[4], acc[5]);
+      __nv_bfloat162 d = __floats2bfloat162_rn(acc[6], acc[7]);
+      o.x = *reinterpret_cast<uint32_t*>(&a);
+      o.y = *reinterpret_cast<uint32_t*>(&b);
+      o.z = *reinterpret_cast<uint32_t*>(&c2);
+      o.w = *reinterpret_cast<uint32_t*>(&d);
+      __stcg(reinterpret_cast<uint4*>(out) + u, o);
+    }
+    __syncthreads();
+  }
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+struct pl_moe_plan_s {
+  pl_comm_t comm = nullptr;
+  MoeGeo g{};
+  char* d_blob = nullptr;
+  size_t blob_bytes = 0;
+  int sm_count = 148;
+  size_t move_smem = 0;
+  bool dispatched = false;
+};
+
+extern "C" {
+
+pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, int n_experts, int topk,
+                               size_t recv_capacity_rows, pl_moe_plan_t* out) {
+  if (!comm || !out) return PL_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (comm->planner) return PL_ERR_UNSUPPORTED;
+  const int R = comm->R;
+  if (tokens_per_rank < 1 || hidden < 1 || n_experts < R || topk < 1 || topk > kMaxTopk) return PL_ERR_INVALID_ARG;
+  if (n_experts % R || n_experts > 4096 || topk > n_experts) return PL_ERR_INVALID_ARG;
+  if (recv_capacity_rows == 0 || recv_capacity_rows > 0x7FFFFFFFull) return PL_ERR_INVALID_ARG;
+  const size_t row_bytes = (size_t)hidden * elem_size(comm->dtype);
+  if (row_bytes % 16) return PL_ERR_ALIGNMENT;
+  if (row_bytes > (1u << 30)) return PL_ERR_INVALID_ARG;
+  pl_moe_plan_s* pl = new (std::nothrow) pl_moe_plan_s();
+  if (!pl) return PL_ERR_OOM;
+  pl->comm = comm;
+  pl->sm_count = comm->sm_count;
+  MoeGeo& g = pl->g;
+  g.R = R;
+  g.T = tokens_per_rank;
+  g.E = n_experts;
+  g.K = topk;
+  g.NB = (tokens_per_rank + kTB - 1) / kTB;
+  g.epr = n_experts / R;
+  g.row_bytes = (uint32_t)row_bytes;
+  g.n_tiles = (uint32_t)((row_bytes + kMaxTile - 1) / kMaxTile);
+  g.tile_bytes = (uint32_t)align_up((row_bytes + g.n_tiles - 1) / g.n_tiles, 16);
+  g.slots = (uint32_t)std::min<size_t>(8, std::max<size_t>(2, (96 * 1024) / g.tile_bytes));
+  g.cap = recv_capacity_rows;
+  pl->move_smem = 128 + (size_t)g.slots * g.tile_bytes;
+  size_t off = 0;
+  auto place = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t o_bc = place((size_t)R * g.NB * g.E * 4), o_base = place((size_t)R * g.E * 4);
+  const size_t o_cnt = place((size_t)R * R * 8), o_ecnt = place((size_t)R * g.E * 8);
+  const size_t o_pos = place((size_t)R * g.T * g.K * 4), o_prank = place((size_t)R * g.T * g.K * 4);
+  const size_t o_flags = place(16);
+  pl->blob_bytes = off;
+  if (cudaMalloc(&pl->d_blob, off) != cudaSuccess) { cudaGetLastError(); delete pl; return PL_ERR_OOM; }
+  if (cudaMemset(pl->d_blob, 0, off) != cudaSuccess) { cudaGetLastError(); cudaFree(pl->d_blob); delete pl; return PL_ERR_CUDA; }
+  g.blockcnt = reinterpret_cast<int32_t*>(pl->d_blob + o_bc);
+  g.base = reinterpret_cast<int32_t*>(pl->d_blob + o_base);
+  g.counts = reinterpret_cast<long long*>(pl->d_blob + o_cnt);
+  g.ecounts = reinterpret_cast<long long*>(pl->d_blob + o_ecnt);
+  g.pos = reinterpret_cast<int32_t*>(pl->d_blob + o_pos);
+  g.prank = reinterpret_cast<int32_t*>(pl->d_blob + o_prank);
+  g.flags = reinterpret_cast<int*>(pl->d_blob + o_flags);
+  if (cudaFuncSetAttribute(moe_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->move_smem) != cudaSuccess ||
+      cudaFuncSetAttribute(moe_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.E * kMaskWords * 4) != cudaSuccess ||
+      cudaFuncSetAttribute(moe_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.E * kMaskWords * 4) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(pl->d_blob);
+    delete pl;
+    return PL_ERR_CUDA;
+  }
+  comm->n_plans += 1;
+  *out = pl;
+  return PL_OK;
+}
+
+pl_status_t pl_moe_plan_destroy(pl_moe_plan_t plan) {
+  if (!plan) return PL_ERR_INVALID_ARG;
+  if (plan->d_blob) cudaFree(plan->d_blob);
+  plan->comm->n_plans -= 1;
+  delete plan;
+  return PL_OK;
+}
+
+pl_status_t pl_moe_dispatch(pl_moe_plan_t plan, const void* const* x, const int32_t* const* topk_idx,
+                            void* const* recv, int32_t* const* recv_meta, void* stream) {
+  if (!plan || !x || !topk_idx || !recv) return PL_ERR_INVALID_ARG;
+  const MoeGeo& g = plan->g;
+  DispatchPtrs P;
+  std::memset(&P, 0, sizeof(P));
+  for (int r = 0; r < g.R; ++r) {
+    if (!x[r] || !topk_idx[r] || !recv[r]) return PL_ERR_INVALID_ARG;
+    if (((uintptr_t)x[r] & 15) || ((uintptr_t)recv[r] & 15) || ((uintptr_t)topk_idx[r] & 3)) return PL_ERR_ALIGNMENT;
+    if (recv_meta && recv_meta[r] && ((uintptr_t)recv_meta[r] & 15)) return PL_ERR_ALIGNMENT;
+    P.x[r] = x[r];
+    P.idx[r] = topk_idx[r];
+    P.recv[r] = recv[r];
+    P.meta[r] = recv_meta ? recv_meta[r] : nullptr;
+  }
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const size_t mask_smem = (size_t)g.E * kMaskWords * 4;
+  dim3 grid(g.NB, g.R);
+  moe_count_kernel<<<grid, kTB, mask_smem, cs>>>(P, g);
+  moe_scan_kernel<<<1, 1024, 0, cs>>>(g);
+  moe_place_kernel<<<grid, kTB, mask_smem, cs>>>(P, g);
+  const unsigned long long items = (unsigned long long)g.R * g.T * g.n_tiles;
+  const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, (200 * 1024) / plan->move_smem));
+  const int mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)plan->sm_count * per_sm);
+  moe_move_kernel<<<mgrid, 32, plan->move_smem, cs>>>(P, g);
+  if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
+  g_launches.fetch_add(4);
+  plan->dispatched = true;
+  return PL_OK;
+}
+
+pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float* const* gates, void* const* out,
+                           void* stream) {
+  if (!plan || !y || !gates || !out) return PL_ERR_INVALID_ARG;
+  if (plan->comm->dtype != PL_BF16) return PL_ERR_UNSUPPORTED;
+  if (!plan->dispatched) return PL_ERR_INVALID_ARG;
+  const MoeGeo& g = plan->g;
+  CombinePtrs P;
+  std::memset(&P, 0, sizeof(P));
+  for (int r = 0; r < g.R; ++r) {
+    if (!y[r] || !gates[r] || !out[r]) return PL_ERR_INVALID_ARG;
+    if (((uintptr_t)y[r] & 15) || ((uintptr_t)out[r] & 15) || ((uintptr_t)gates[r] & 3)) return PL_ERR_ALIGNMENT;
+    P.y[r] = y[r];
+    P.gates[r] = gates[r];
+    P.out[r] = out[r];
+  }
+  const unsigned long long n_tok = (unsigned long long)g.R * g.T;
+  const int grid = (int)std::min<unsigned long long>(n_tok, (unsigned long long)plan->sm_count * 6);
+  moe_combine_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(P, g);
+  if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return PL_OK;
+}
+
+pl_status_t pl_moe_plan_read(pl_moe_plan_t plan, int32_t* pos, int64_t* counts, int64_t* expert_counts, void* stream) {
+  if (!plan) return PL_ERR_INVALID_ARG;
+  const MoeGeo& g = plan->g;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  int flags[4] = {0, 0, 0, 0};
+  bool ok = cudaMemcpy(flags, g.flags, 12, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (ok && pos) ok = cudaMemcpy(pos, g.pos, (size_t)g.R * g.T * g.K * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (ok && counts) ok = cudaMemcpy(counts, g.counts, (size_t)g.R * g.R * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (ok && expert_counts) ok = cudaMemcpy(expert_counts, g.ecounts, (size_t)g.R * g.E * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return PL_ERR_CUDA; }
+  if (flags[2]) return PL_ERR_TIMEOUT;
+  if (flags[1]) return PL_ERR_INVALID_ARG;
+  if (flags[0]) return PL_ERR_OVERFLOW;
+  return PL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,700 @@
+// Host orchestrator: lowers (collective, algorithm, chunk size) into a flat list of
+// chunk-granular ops with wait / signal edges.  It plays the role the paper gives to its
+// orchestration tier (Sec. 3.2): dependencies are derived from the input and output
+// layouts (Listing 2), the composed all-reduce follows Algorithm 1 without the staging
+// role, and the consume operation (copy or reduce) selects the op kind.  Everything here
+// is plain host C++: no CUDA calls.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <numeric>
+
+#include "pl_internal.h"
+
+namespace pl {
+namespace {
+
+pl_ref_t ref(int rank, int buf, int dtype, uint64_t off) {
+  pl_ref_t r;
+  std::memset(&r, 0, sizeof(r));
+  r.rank = rank;
+  r.buf = buf;
+  r.dtype = dtype;
+  r.offset = off;
+  return r;
+}
+
+struct Emitter {
+  Lowered* L;
+  uint32_t slice_bytes;
+  int queues_per_rank = 1;
+  // Chunks each rank runs in the phase being emitted (0 = unknown).  When known, the slice
+  // count is nudged upwards so that a rank's work items divide evenly over its queues.
+  uint64_t phase_chunks = 0;
+
+  int new_flag() { return L->n_flags++; }
+
+  // Emit one chunk-granular op.  A chunk wider than slice_bytes is cut into slices that
+  // different CTAs of the executing rank run; every slice signals the chunk's flag, so the
+  // flag counts finished slices and a waiter needs all of them (Sec. 3.2: the last CTA of a
+  // group to finish a chunk is the one that makes it visible).
+  void chunk_op(int kind, int exec_rank, int layer, pl_ref_t dst, bool bcast,
+                const std::vector<pl_ref_t>& src, uint64_t count, const std::vector<int>& waits,
+                int signal, int signal2 = -1) {
+    int min_es = elem_size(dst.dtype), max_es = min_es;
+    for (const pl_ref_t& s : src) {
+      min_es = std::min(min_es, elem_size(s.dtype));
+      max_es = std::max(max_es, elem_size(s.dtype));
+    }
+    const uint64_t unit16 = 16 / min_es;  // elements that keep every operand 16-byte aligned
+    uint64_t wide = count * max_es;
+    uint64_t n_slices = 1;
+    if (slice_bytes && wide > slice_bytes + slice_bytes / 2) n_slices = (wide + slice_bytes - 1) / slice_bytes;
+    if (n_slices > 1 && phase_chunks && queues_per_rank > 1) {
+      for (uint64_t k = n_slices; k <= 4 * n_slices; ++k)
+        if ((phase_chunks * k) % (uint64_t)queues_per_rank == 0 && wide / k >= 4096) {
+          n_slices = k;
+          break;
+        }
+    }
+    uint64_t per = (count + n_slices - 1) / n_slices;
+    uint64_t unit = (per >= 8 * (128 / min_es)) ? uint64_t(128 / min_es) : unit16;
+    per = (per + unit - 1) / unit * unit;
+    for (uint64_t b = 0; b < count; b += per) {
+      HostOp op;
+      op.kind = kind;
+      op.exec_rank = exec_rank;
+      op.layer = layer;
+      op.count = std::min(per, count - b);
+      op.dst = dst;
+      op.dst.offset += b * elem_size(dst.dtype);
+      op.bcast = bcast;
+      for (pl_ref_t s : src) {
+        s.offset += b * elem_size(s.dtype);
+        op.src.push_back(s);
+      }
+      op.waits = waits;
+      op.signal = signal;
+      op.signal2 = signal2;
+      L->ops.push_back(std::move(op));
+    }
+  }
+};
+
+struct Geo {
+  int R, dtype, es;
+  uint64_t n;            // elements per rank message
+  uint64_t P;            // elements per partition
+  uint64_t chunk;        // elements per chunk (clipped to P)
+  uint64_t n_c;          // chunks per partition
+  uint64_t clen(uint64_t c) const { return std::min(chunk, P - c * chunk); }
+};
+
+Geo make_geo(int R, int dtype, uint64_t n, uint64_t part_elems, uint64_t chunk_bytes) {
+  Geo g;
+  g.R = R;
+  g.dtype = dtype;
+  g.es = elem_size(dtype);
+  g.n = n;
+  g.P = part_elems;
+  g.chunk = std::max<uint64_t>(1, std::min<uint64_t>(chunk_bytes / g.es, g.P));
+  g.n_c = g.P ? (g.P + g.chunk - 1) / g.chunk : 0;
+  return g;
+}
+
+// Cross-layer edges of a multi-layer schedule: `pub[p]` is the flag that tells that rank p's
+// contribution to this layer may be read (its previous layer's output is complete), -1 when
+// there is nothing to wait for; `done[r]` is the flag every op that writes rank r's output
+// in this layer must signal, -1 when nobody will ask.
+struct LayerEdges {
+  std::vector<int> pub;
+  std::vector<int> done;
+};
+
+std::vector<int> waits_on(const LayerEdges* le, const std::vector<int>& ranks) {
+  std::vector<int> w;
+  if (!le) return w;
+  for (int p : ranks)
+    if (le->pub[p] >= 0 && std::find(w.begin(), w.end(), le->pub[p]) == w.end()) w.push_back(le->pub[p]);
+  return w;
+}
+
+std::vector<int> all_ranks(int R) {
+  std::vector<int> v(R);
+  std::iota(v.begin(), v.end(), 0);
+  return v;
+}
+
+// reduce-scatter, direct: rank r reduces chunk c of partition r from all R inputs in
+// ascending rank order (Listing 2: packed output => out = dst + offset, reduce waits for
+// all producers; with peer-visible inputs there is nothing to wait for).
+void rs_direct(Emitter& em, const Geo& g) {
+  em.phase_chunks = g.n_c;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int r = 0; r < g.R; ++r) {
+      std::vector<pl_ref_t> src;
+      for (int p = 0; p < g.R; ++p) src.push_back(ref(p, PL_BUF_IN, g.dtype, (r * g.P + c * g.chunk) * g.es));
+      em.chunk_op(PL_OP_REDUCE, r, 0, ref(r, PL_BUF_OUT, g.dtype, c * g.chunk * g.es), false, src, g.clen(c), {}, -1);
+    }
+}
+
+// all-gather, direct: rank r copies chunk c of every peer's packed input to
+// out + peer*partBytes + offset (Listing 2, scattered output).  Peers are visited starting
+// at r so that the R consumers do not all hit the same producer at once.
+void ag_direct(Emitter& em, const Geo& g) {
+  em.phase_chunks = g.n_c * g.R;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int i = 0; i < g.R; ++i)
+      for (int r = 0; r < g.R; ++r) {
+        int p = (r + i) % g.R;
+        uint64_t bytes = g.clen(c) * g.es;
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, (p * g.P + c * g.chunk) * g.es), false,
+                    {ref(p, PL_BUF_IN, PL_U8, c * g.chunk * g.es)}, bytes, {}, -1);
+      }
+}
+
+// all-to-all, direct: rank r copies partition r of every source p to slot p of its output.
+void a2a_direct(Emitter& em, const Geo& g) {
+  em.phase_chunks = g.n_c * g.R;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int i = 0; i < g.R; ++i)
+      for (int r = 0; r < g.R; ++r) {
+        int p = (r + i) % g.R;
+        uint64_t bytes = g.clen(c) * g.es;
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, (p * g.P + c * g.chunk) * g.es), false,
+                    {ref(p, PL_BUF_IN, PL_U8, (r * g.P + c * g.chunk) * g.es)}, bytes, {}, -1);
+      }
+}
+
+// all-to-all-v: counts[p][r] elements from p to r; sender offsets are prefix sums over
+// destinations, receiver offsets prefix sums over sources (transposedV layout).
+void a2av_direct(Emitter& em, int R, int dtype, const uint64_t* counts, uint64_t chunk_bytes) {
+  const int es = elem_size(dtype);
+  std::vector<uint64_t> soff(R * R), roff(R * R);
+  for (int p = 0; p < R; ++p) {
+    uint64_t a = 0;
+    for (int r = 0; r < R; ++r) { soff[p * R + r] = a; a += counts[p * R + r]; }
+  }
+  for (int r = 0; r < R; ++r) {
+    uint64_t a = 0;
+    for (int p = 0; p < R; ++p) { roff[p * R + r] = a; a += counts[p * R + r]; }
+  }
+  uint64_t max_seg = 0;
+  for (int i = 0; i < R * R; ++i) max_seg = std::max(max_seg, counts[i] * es);
+  uint64_t chunk = std::max<uint64_t>(16, chunk_bytes);
+  for (uint64_t b = 0; b < max_seg; b += chunk)
+    for (int i = 0; i < R; ++i)
+      for (int r = 0; r < R; ++r) {
+        int p = (r + i) % R;
+        uint64_t seg = counts[p * R + r] * es;
+        if (b >= seg) continue;
+        uint64_t bytes = std::min(chunk, seg - b);
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, roff[p * R + r] * es + b), false,
+                    {ref(p, PL_BUF_IN, PL_U8, soff[p * R + r] * es + b)}, bytes, {}, -1);
+      }
+}
+
+// all-reduce, one-shot: every rank reduces the whole message from all R inputs.
+void ar_oneshot(Emitter& em, const Geo& g, int layer, uint64_t in_off, uint64_t out_off, const LayerEdges* le) {
+  // g.P == g.n here: the "partition" is the whole message, chunked.
+  em.phase_chunks = g.n_c;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int r = 0; r < g.R; ++r) {
+      std::vector<pl_ref_t> src;
+      for (int p = 0; p < g.R; ++p) src.push_back(ref(p, PL_BUF_IN, g.dtype, in_off + c * g.chunk * g.es));
+      em.chunk_op(PL_OP_REDUCE, r, layer, ref(r, PL_BUF_OUT, g.dtype, out_off + c * g.chunk * g.es), false, src,
+                  g.clen(c), waits_on(le, all_ranks(g.R)), le ? le->done[r] : -1);
+    }
+}
+
+// all-reduce, direct fused: the reducer of partition k writes each result into all R outputs.
+void ar_fused(Emitter& em, const Geo& g, int layer, uint64_t in_off, uint64_t out_off, const LayerEdges* le) {
+  em.phase_chunks = g.n_c;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int k = 0; k < g.R; ++k) {
+      std::vector<pl_ref_t> src;
+      uint64_t off = (k * g.P + c * g.chunk) * g.es;
+      for (int p = 0; p < g.R; ++p) src.push_back(ref(p, PL_BUF_IN, g.dtype, in_off + off));
+      // every output is complete only when every reducer is: one shared flag per layer
+      em.chunk_op(PL_OP_REDUCE, k, layer, ref(k, PL_BUF_OUT, g.dtype, out_off + off), true, src, g.clen(c),
+                  waits_on(le, all_ranks(g.R)), le ? le->done[0] : -1);
+    }
+}
+
+// all-reduce, direct two-shot = compose<reduce-scatter, all-gather> in one launch
+// (Algorithm 1 without the staging role): rank k reduces chunk c of partition k into its own
+// output and publishes reduced(k,c) to all ranks; every other rank then copies that chunk.
+void ar_direct(Emitter& em, const Geo& g, int layer, uint64_t in_off, uint64_t out_off, const LayerEdges* le) {
+  std::vector<int> reduced(g.R * g.n_c);
+  em.phase_chunks = g.n_c;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int k = 0; k < g.R; ++k) {
+      int f = reduced[k * g.n_c + c] = em.new_flag();
+      std::vector<pl_ref_t> src;
+      uint64_t off = (k * g.P + c * g.chunk) * g.es;
+      for (int p = 0; p < g.R; ++p) src.push_back(ref(p, PL_BUF_IN, g.dtype, in_off + off));
+      em.chunk_op(PL_OP_REDUCE, k, layer, ref(k, PL_BUF_OUT, g.dtype, out_off + off), false, src, g.clen(c),
+                  waits_on(le, all_ranks(g.R)), f, le ? le->done[k] : -1);
+    }
+  em.phase_chunks = g.n_c * (g.R - 1);
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int i = 1; i < g.R; ++i)
+      for (int r = 0; r < g.R; ++r) {
+        int k = (r + i) % g.R;
+        uint64_t off = (k * g.P + c * g.chunk) * g.es;
+        em.chunk_op(PL_OP_COPY, r, layer, ref(r, PL_BUF_OUT, PL_U8, out_off + off), false,
+                    {ref(k, PL_BUF_OUT, PL_U8, out_off + off)}, g.clen(c) * g.es, {reduced[k * g.n_c + c]},
+                    le ? le->done[r] : -1);
+      }
+}
+
+// Ring reduce-scatter.  Partition k's chain starts with rank k+1's own input and visits
+// k+2, ..., k (mod R).  At step s in [0, R-2] rank r handles k = (r - s - 2) mod R:
+//   part_r[k] = part_{r-1}[k] + in_r[k]      (step 0 reads in_{r-1}[k] directly)
+// and the last step writes rank r's result.  Partials are kept in the partial dtype
+// (fp32 for bf16 data) in per-step scratch slots.  `final_to_out_partition`: write the last
+// hop to out_r + r*P (all-reduce) instead of out_r + 0 (reduce-scatter).  Returns the flag
+// of (r, last step, c) in final_flags when asked.
+void rs_ring(Emitter& em, const Geo& g, bool final_to_out_partition, std::vector<int>* final_flags) {
+  const int R = g.R, pd = partial_dtype(g.dtype), ps = elem_size(pd);
+  std::vector<int> prev(R * g.n_c, -1), cur(R * g.n_c, -1);
+  em.phase_chunks = g.n_c;
+  for (int s = 0; s <= R - 2; ++s) {
+    const bool last = (s == R - 2);
+    for (uint64_t c = 0; c < g.n_c; ++c)
+      for (int r = 0; r < R; ++r) {
+        const int k = ((r - s - 2) % R + R) % R, q = (r - 1 + R) % R;
+        const uint64_t in_off = (k * g.P + c * g.chunk) * g.es;
+        pl_ref_t a = (s == 0) ? ref(q, PL_BUF_IN, g.dtype, in_off)
+                              : ref(q, PL_BUF_SCRATCH, pd, ((s - 1) * g.P + c * g.chunk) * ps);
+        pl_ref_t b = ref(r, PL_BUF_IN, g.dtype, in_off);
+        pl_ref_t d = last ? ref(r, PL_BUF_OUT, g.dtype, ((final_to_out_partition ? r * g.P : 0) + c * g.chunk) * g.es)
+                          : ref(r, PL_BUF_SCRATCH, pd, (s * g.P + c * g.chunk) * ps);
+        std::vector<int> w;
+        if (s > 0) w.push_back(prev[q * g.n_c + c]);
+        int f = -1;
+        if (!last || final_flags) f = em.new_flag();
+        cur[r * g.n_c + c] = f;
+        em.chunk_op(PL_OP_COPY_REDUCE, r, 0, d, false, {a, b}, g.clen(c), w, f);
+      }
+    prev = cur;
+  }
+  if (final_flags) *final_flags = prev;
+  if (R > 2)
+    for (int r = 0; r < R; ++r) em.L->scratch_per_rank[r] = (uint64_t)(R - 2) * g.P * ps;
+}
+
+// Ring all-gather.  Rank r first places its own contribution, then at step s in [0, R-2]
+// copies partition (r - s - 1) mod R from rank r-1 (from r-1's input at step 0, from its
+// output afterwards).  `own_from_out`: the own partition already sits in out_r (all-reduce);
+// own_flags then carries the flags that say so.
+void ag_ring(Emitter& em, const Geo& g, bool own_from_out, const std::vector<int>* own_flags) {
+  const int R = g.R;
+  std::vector<int> prev(R * g.n_c, -1), cur(R * g.n_c, -1);
+  em.phase_chunks = g.n_c;
+  if (!own_from_out)
+    for (uint64_t c = 0; c < g.n_c; ++c)
+      for (int r = 0; r < R; ++r)
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, (r * g.P + c * g.chunk) * g.es), false,
+                    {ref(r, PL_BUF_IN, PL_U8, c * g.chunk * g.es)}, g.clen(c) * g.es, {}, -1);
+  for (int s = 0; s <= R - 2; ++s) {
+    for (uint64_t c = 0; c < g.n_c; ++c)
+      for (int r = 0; r < R; ++r) {
+        const int k = ((r - s - 1) % R + R) % R, q = (r - 1 + R) % R;
+        const uint64_t off = (k * g.P + c * g.chunk) * g.es;
+        pl_ref_t src = (s == 0 && !own_from_out) ? ref(q, PL_BUF_IN, PL_U8, c * g.chunk * g.es)
+                                                 : ref(q, PL_BUF_OUT, PL_U8, off);
+        std::vector<int> w;
+        if (s == 0) {
+          if (own_from_out) w.push_back((*own_flags)[q * g.n_c + c]);
+        } else {
+          w.push_back(prev[q * g.n_c + c]);
+        }
+        int f = (s < R - 2) ? em.new_flag() : -1;
+        cur[r * g.n_c + c] = f;
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, off), false, {src}, g.clen(c) * g.es, w, f);
+      }
+    prev = cur;
+  }
+}
+
+// Binomial-tree all-reduce, chunk-pipelined.  Reduce: at level l every rank r that is a
+// multiple of 2^(l+1) adds the running sum of rank r + 2^l (skipped when that rank does not
+// exist) to its own; running sums live in fp32 scratch (one slot per level, never
+// overwritten); the root's last addition writes the output.  Broadcast: the same tree in
+// reverse, child r + 2^l copies the finished chunk from r's output.
+void ar_tree(Emitter& em, const Geo& g) {
+  const int R = g.R, pd = partial_dtype(g.dtype), ps = elem_size(pd);
+  int levels = 0;
+  while ((1 << levels) < R) ++levels;
+  em.phase_chunks = 0;  // the ranks active per level differ
+  // g.P == g.n: chunks run over the whole message
+  std::vector<int> slots(R, 0);                        // scratch slots used so far per rank
+  std::vector<pl_ref_t> acc(R);                        // where rank r's running sum lives (chunk 0)
+  std::vector<std::vector<int>> acc_flag(R, std::vector<int>(g.n_c, -1));
+  for (int r = 0; r < R; ++r) acc[r] = ref(r, PL_BUF_IN, g.dtype, 0);
+  // the root's last reducing level
+  int root_last = -1;
+  for (int l = 0; l < levels; ++l)
+    if ((1 << l) < R) root_last = l;
+  std::vector<std::vector<int>> has(R, std::vector<int>(g.n_c, -1));  // "out_r chunk c is final"
+  for (int l = 0; l < levels; ++l) {
+    for (uint64_t c = 0; c < g.n_c; ++c)
+      for (int r = 0; r < R; r += (1 << (l + 1))) {
+        int q = r + (1 << l);
+        if (q >= R) continue;
+        const bool to_out = (r == 0 && l == root_last);
+        pl_ref_t a = acc[r], b = acc[q];
+        a.offset += c * g.chunk * elem_size(a.dtype);
+        b.offset += c * g.chunk * elem_size(b.dtype);
+        pl_ref_t d = to_out ? ref(0, PL_BUF_OUT, g.dtype, c * g.chunk * g.es)
+                            : ref(r, PL_BUF_SCRATCH, pd, ((uint64_t)slots[r] * g.n + c * g.chunk) * ps);
+        std::vector<int> w;
+        if (acc_flag[r][c] >= 0) w.push_back(acc_flag[r][c]);
+        if (acc_flag[q][c] >= 0) w.push_back(acc_flag[q][c]);
+        int f = em.new_flag();
+        em.chunk_op(PL_OP_COPY_REDUCE, r, 0, d, false, {a, b}, g.clen(c), w, f);
+        acc_flag[r][c] = f;
+        if (to_out) has[0][c] = f;
+      }
+    // after finishing the level, move acc[] of the reducing ranks to the slot just written
+    for (int r = 0; r < R; r += (1 << (l + 1))) {
+      int q = r + (1 << l);
+      if (q >= R) continue;
+      const bool to_out = (r == 0 && l == root_last);
+      if (!to_out) {
+        acc[r] = ref(r, PL_BUF_SCRATCH, pd, (uint64_t)slots[r] * g.n * ps);
+        slots[r] += 1;
+      }
+    }
+  }
+  for (int r = 0; r < R; ++r) em.L->scratch_per_rank[r] = (uint64_t)slots[r] * g.n * ps;
+  for (int l = levels - 1; l >= 0; --l)
+    for (uint64_t c = 0; c < g.n_c; ++c)
+      for (int r = 0; r < R; r += (1 << (l + 1))) {
+        int q = r + (1 << l);
+        if (q >= R) continue;
+        int f = em.new_flag();
+        em.chunk_op(PL_OP_COPY, q, 0, ref(q, PL_BUF_OUT, PL_U8, c * g.chunk * g.es), false,
+                    {ref(r, PL_BUF_OUT, PL_U8, c * g.chunk * g.es)}, g.clen(c) * g.es, {has[r][c]}, f);
+        has[q][c] = f;
+      }
+}
+
+}  // namespace
+
+Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
+  Policy p = rq.pol;
+  const int es = elem_size(rq.dtype);
+  uint64_t msg = rq.count_per_rank * es;
+  if (rq.counts_v) {
+    msg = 0;
+    for (int i = 0; i < rq.R * rq.R; ++i) msg += rq.counts_v[i] * es;
+    msg /= rq.R;
+  }
+  if (rq.coll == PL_ALLGATHER) msg *= rq.R;
+  if (p.threads <= 0) p.threads = 512;
+  if (p.datapath == PL_DP_AUTO) p.datapath = PL_DP_LDST;
+  if (p.stages <= 0) p.stages = 4;
+  if (p.stage_bytes == 0) p.stage_bytes = 16384;
+  if (p.slice_bytes == 0) {
+    // latency regime: few, small slices; throughput regime: 64 KiB slices
+    p.slice_bytes = msg <= (1u << 20) ? 16384 : 65536;
+  }
+  if (p.n_ctas <= 0) {
+    const int full = std::max(rq.R, max_resident_ctas / rq.R * rq.R);
+    // work items per rank under this slicing (output bytes a rank produces / slice)
+    uint64_t per_rank_out = msg;
+    if (rq.coll == PL_REDUCE_SCATTER) per_rank_out = msg / rq.R;
+    uint64_t per_rank_slices = std::max<uint64_t>(1, (per_rank_out + p.slice_bytes - 1) / p.slice_bytes);
+    uint64_t want = per_rank_slices * rq.R;
+    p.n_ctas = (int)std::min<uint64_t>(full, std::max<uint64_t>(rq.R, want));
+  }
+  p.n_ctas = std::max(rq.R, p.n_ctas / rq.R * rq.R);
+  return p;
+}
+
+pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
+  const int R = rq.R, dt = rq.dtype, es = elem_size(dt);
+  auto fail = [&](pl_status_t st, const char* m) {
+    if (err) *err = m;
+    return st;
+  };
+  if (R < 2 || R > PL_MAX_RANKS) return fail(PL_ERR_INVALID_ARG, "R out of range");
+  if (rq.chunk_bytes == 0 || rq.chunk_bytes % 16) return fail(PL_ERR_INVALID_ARG, "chunk_bytes must be a positive multiple of 16");
+  const bool reduces = rq.coll == PL_ALLREDUCE || rq.coll == PL_REDUCE_SCATTER;
+  if (reduces && dt == PL_U8) return fail(PL_ERR_UNSUPPORTED, "bytes cannot be reduced");
+  Emitter em{L, rq.pol.slice_bytes};
+  em.queues_per_rank = std::max(1, rq.pol.n_ctas / R);
+  L->n_layers = 1;
+
+  if (rq.coll == PL_ALLTOALLV) {
+    if (rq.algo != PL_ALGO_DIRECT) return fail(PL_ERR_UNSUPPORTED, "all-to-all-v is direct only");
+    if (!rq.counts_v) return fail(PL_ERR_INVALID_ARG, "counts missing");
+    uint64_t total = 0;
+    for (int i = 0; i < R * R; ++i) {
+      if ((rq.counts_v[i] * es) % 16) return fail(PL_ERR_ALIGNMENT, "every (src,dst) segment must be a multiple of 16 bytes");
+      total += rq.counts_v[i] * es;
+    }
+    for (int p = 0; p < R; ++p)
+      for (int r = 0; r < R; ++r) {
+        L->in_bytes[p] += rq.counts_v[p * R + r] * es;
+        L->out_bytes[r] += rq.counts_v[p * R + r] * es;
+      }
+    L->message_bytes = total / R;
+    em.phase_chunks = 0;
+    a2av_direct(em, R, dt, rq.counts_v, rq.chunk_bytes);
+    return PL_OK;
+  }
+  if (rq.counts_v) return fail(PL_ERR_INVALID_ARG, "counts only apply to all-to-all-v");
+  const uint64_t n = rq.count_per_rank;
+  if (n == 0) return fail(PL_ERR_INVALID_ARG, "count_per_rank is zero");
+  const uint64_t bytes = n * es;
+
+  if (rq.n_layers > 0) {
+    if (rq.coll != PL_ALLREDUCE) return fail(PL_ERR_UNSUPPORTED, "layered schedules are all-reduce only");
+    if (rq.algo != PL_ALGO_ONESHOT && rq.algo != PL_ALGO_DIRECT && rq.algo != PL_ALGO_DIRECT_FUSED)
+      return fail(PL_ERR_UNSUPPORTED, "layered schedules support one-shot, direct and direct-fused");
+  }
+  const int n_layers = std::max(1, rq.n_layers);
+  L->n_layers = n_layers;
+
+  switch (rq.coll) {
+    case PL_ALLGATHER: {
+      if (bytes % 16) return fail(PL_ERR_INVALID_ARG, "all-gather contribution must be a multiple of 16 bytes");
+      Geo g = make_geo(R, dt, n * R, n, rq.chunk_bytes);
+      for (int r = 0; r < R; ++r) { L->in_bytes[r] = bytes; L->out_bytes[r] = bytes * R; }
+      L->message_bytes = bytes * R;
+      if (rq.algo == PL_ALGO_DIRECT) ag_direct(em, g);
+      else if (rq.algo == PL_ALGO_RING) ag_ring(em, g, false, nullptr);
+      else return fail(PL_ERR_UNSUPPORTED, "all-gather supports direct and ring");
+      return PL_OK;
+    }
+    case PL_ALLTOALL: {
+      if (bytes % (16 * R)) return fail(PL_ERR_INVALID_ARG, "message bytes must be divisible by 16*R");
+      if (rq.algo != PL_ALGO_DIRECT) return fail(PL_ERR_UNSUPPORTED, "all-to-all is direct only");
+      Geo g = make_geo(R, dt, n, n / R, rq.chunk_bytes);
+      for (int r = 0; r < R; ++r) L->in_bytes[r] = L->out_bytes[r] = bytes;
+      L->message_bytes = bytes;
+      a2a_direct(em, g);
+      return PL_OK;
+    }
+    case PL_REDUCE_SCATTER: {
+      if (bytes % (16 * R)) return fail(PL_ERR_INVALID_ARG, "message bytes must be divisible by 16*R");
+      Geo g = make_geo(R, dt, n, n / R, rq.chunk_bytes);
+      for (int r = 0; r < R; ++r) { L->in_bytes[r] = bytes; L->out_bytes[r] = bytes / R; }
+      L->message_bytes = bytes;
+      if (rq.algo == PL_ALGO_DIRECT) rs_direct(em, g);
+      else if (rq.algo == PL_ALGO_RING) rs_ring(em, g, false, nullptr);
+      else return fail(PL_ERR_UNSUPPORTED, "reduce-scatter supports direct and ring");
+      return PL_OK;
+    }
+    case PL_ALLREDUCE: {
+      const bool partitioned = rq.algo == PL_ALGO_DIRECT || rq.algo == PL_ALGO_DIRECT_FUSED || rq.algo == PL_ALGO_RING;
+      if (partitioned && bytes % (16 * R)) return fail(PL_ERR_INVALID_ARG, "message bytes must be divisible by 16*R");
+      if (bytes % 16) return fail(PL_ERR_INVALID_ARG, "message bytes must be a multiple of 16");
+      for (int r = 0; r < R; ++r) L->in_bytes[r] = L->out_bytes[r] = bytes * n_layers;
+      L->message_bytes = bytes;
+      Geo gp = make_geo(R, dt, n, n / R, rq.chunk_bytes);  // partitioned view
+      Geo gw = make_geo(R, dt, n, n, rq.chunk_bytes);      // whole-message view
+      if (rq.n_layers > 0) {
+        LayerEdges le;
+        le.pub.assign(R, -1);
+        for (int l = 0; l < n_layers; ++l) {
+          le.done.assign(R, -1);
+          if (l + 1 < n_layers) {
+            if (rq.algo == PL_ALGO_DIRECT_FUSED) {
+              int f = em.new_flag();
+              le.done.assign(R, f);
+            } else {
+              for (int r = 0; r < R; ++r) le.done[r] = em.new_flag();
+            }
+          }
+          const uint64_t off = (uint64_t)l * bytes;
+          if (rq.algo == PL_ALGO_ONESHOT) ar_oneshot(em, gw, l, off, off, &le);
+          else if (rq.algo == PL_ALGO_DIRECT) ar_direct(em, gp, l, off, off, &le);
+          else ar_fused(em, gp, l, off, off, &le);
+          le.pub = le.done;
+        }
+        return PL_OK;
+      }
+      switch (rq.algo) {
+        case PL_ALGO_ONESHOT: ar_oneshot(em, gw, 0, 0, 0, nullptr); return PL_OK;
+        case PL_ALGO_DIRECT: ar_direct(em, gp, 0, 0, 0, nullptr); return PL_OK;
+        case PL_ALGO_DIRECT_FUSED: ar_fused(em, gp, 0, 0, 0, nullptr); return PL_OK;
+        case PL_ALGO_RING: {
+          std::vector<int> fin;
+          rs_ring(em, gp, true, &fin);
+          ag_ring(em, gp, true, &fin);
+          return PL_OK;
+        }
+        case PL_ALGO_TREE: ar_tree(em, gw); return PL_OK;
+        default: return fail(PL_ERR_INVALID_ARG, "unknown algorithm");
+      }
+    }
+    default: return fail(PL_ERR_INVALID_ARG, "unknown collective");
+  }
+}
+
+// Place ops on queues.  Rank r owns queues {q : q % R == r}; its ops go, in topological
+// order, to the least-loaded of its queues (ties to the lowest queue).  Each queue's order is
+// therefore a subsequence of the topological order, which is what makes a co-resident grid
+// deadlock free: the unfinished op with the smallest topological index is always at the head
+// of its queue and all it waits for has already run.
+void assign_queues(Lowered* L, int R, int n_queues) {
+  const int per_rank = std::max(1, n_queues / R);
+  std::vector<uint64_t> load((size_t)per_rank * R, 0);
+  L->flag_need.assign(L->n_flags, 0);
+  int topo = 0;
+  for (HostOp& op : L->ops) {
+    op.topo = topo++;
+    uint64_t cost = op.count * elem_size(op.dst.dtype) * (op.bcast ? R : 1);
+    for (const pl_ref_t& s : op.src) cost += op.count * elem_size(s.dtype);
+    cost += 2048;  // fixed per-op overhead so that many tiny ops still spread out
+    int best = 0;
+    for (int j = 1; j < per_rank; ++j)
+      if (load[(size_t)j * R + op.exec_rank] < load[(size_t)best * R + op.exec_rank]) best = j;
+    load[(size_t)best * R + op.exec_rank] += cost;
+    op.queue = best * R + op.exec_rank;
+    if (op.signal >= 0) L->flag_need[op.signal] += 1;
+    if (op.signal2 >= 0) L->flag_need[op.signal2] += 1;
+  }
+}
+
+namespace {
+struct Interval {
+  uint64_t lo, hi;
+  int op;
+};
+using Key = std::pair<int, int>;  // (buf kind, rank)
+}  // namespace
+
+pl_status_t validate(const Lowered& L, int R, std::string* err) {
+  char msg[256];
+  auto fail = [&](const char* m) {
+    if (err) *err = m;
+    return PL_ERR_INVALID_SCHEDULE;
+  };
+  const size_t n = L.ops.size();
+  // 1. topological sanity: each flag's signals all come from ops before any waiter
+  std::vector<int> last_signal(L.n_flags, -1), first_wait(L.n_flags, INT32_MAX);
+  std::vector<uint32_t> need(L.n_flags, 0);
+  for (size_t i = 0; i < n; ++i) {
+    const HostOp& op = L.ops[i];
+    if (op.topo != (int)i) return fail("ops are not stored in topological order");
+    for (int s : {op.signal, op.signal2})
+      if (s >= 0) {
+        if (s >= L.n_flags) return fail("signal flag out of range");
+        last_signal[s] = std::max(last_signal[s], (int)i);
+        need[s]++;
+      }
+    if (op.signal >= 0 && op.signal == op.signal2) return fail("op signals the same flag twice");
+    if (op.waits.size() > PL_MAX_WAITS) return fail("too many waits on one op");
+    if (op.src.size() > PL_MAX_SRC || op.src.empty()) return fail("bad source count");
+    for (int w : op.waits) {
+      if (w < 0 || w >= L.n_flags) return fail("wait flag out of range");
+      first_wait[w] = std::min(first_wait[w], (int)i);
+    }
+  }
+  for (int f = 0; f < L.n_flags; ++f) {
+    if (need[f] != L.flag_need[f]) return fail("flag_need does not match the number of signals");
+    if (first_wait[f] != INT32_MAX && need[f] == 0) return fail("a flag is waited on but never signalled");
+    if (first_wait[f] != INT32_MAX && last_signal[f] >= first_wait[f]) return fail("a waiter precedes one of its signals in the topological order");
+  }
+  // 2. queue order embeds in the topological order (ops are appended per queue in topo order
+  //    by construction; check exec_rank / queue agreement)
+  for (const HostOp& op : L.ops) {
+    if (op.queue < 0) return fail("op without a queue");
+    if (op.queue % R != op.exec_rank) return fail("op placed on another rank's queue");
+  }
+  // 3. alignment and bounds
+  for (const HostOp& op : L.ops) {
+    auto check = [&](const pl_ref_t& r, uint64_t limit_bytes) -> const char* {
+      uint64_t b = op.count * elem_size(r.dtype);
+      if (r.offset % 16 || b % 16) return "operand not 16-byte aligned";
+      if (r.rank < 0 || r.rank >= R) return "rank out of range";
+      if (r.offset + b > limit_bytes) return "operand exceeds its buffer";
+      return nullptr;
+    };
+    auto limit = [&](const pl_ref_t& r) {
+      return r.buf == PL_BUF_IN ? L.in_bytes[r.rank] : r.buf == PL_BUF_OUT ? L.out_bytes[r.rank] : L.scratch_per_rank[r.rank];
+    };
+    if (op.dst.buf == PL_BUF_IN) return fail("an op writes an input buffer");
+    if (op.bcast) {
+      if (op.dst.buf != PL_BUF_OUT) return fail("broadcast destination must be an output");
+      for (int r = 0; r < R; ++r) {
+        pl_ref_t d = op.dst;
+        d.rank = r;
+        if (const char* m = check(d, L.out_bytes[r])) return fail(m);
+      }
+    } else if (const char* m = check(op.dst, limit(op.dst))) {
+      return fail(m);
+    }
+    for (const pl_ref_t& s : op.src)
+      if (const char* m = check(s, limit(s))) return fail(m);
+  }
+  // 4. every written byte written once; outputs fully covered
+  std::map<Key, std::vector<Interval>> writes;
+  for (size_t i = 0; i < n; ++i) {
+    const HostOp& op = L.ops[i];
+    uint64_t b = op.count * elem_size(op.dst.dtype);
+    if (op.bcast) {
+      for (int r = 0; r < R; ++r) writes[{op.dst.buf, r}].push_back({op.dst.offset, op.dst.offset + b, (int)i});
+    } else {
+      writes[{op.dst.buf, op.dst.rank}].push_back({op.dst.offset, op.dst.offset + b, (int)i});
+    }
+  }
+  for (auto& kv : writes) {
+    auto& v = kv.second;
+    std::sort(v.begin(), v.end(), [](const Interval& a, const Interval& b) { return a.lo < b.lo; });
+    for (size_t i = 1; i < v.size(); ++i)
+      if (v[i].lo < v[i - 1].hi) {
+        std::snprintf(msg, sizeof msg, "ops %d and %d write overlapping bytes of buffer kind %d rank %d", v[i - 1].op,
+                      v[i].op, kv.first.first, kv.first.second);
+        return fail(msg);
+      }
+  }
+  for (int r = 0; r < R; ++r) {
+    uint64_t covered = 0;
+    auto it = writes.find({PL_BUF_OUT, r});
+    if (it != writes.end())
+      for (const Interval& iv : it->second) {
+        if (iv.lo != covered) break;
+        covered = iv.hi;
+      }
+    if (covered != L.out_bytes[r]) {
+      std::snprintf(msg, sizeof msg, "output of rank %d is covered up to byte %llu of %llu", r,
+                    (unsigned long long)covered, (unsigned long long)L.out_bytes[r]);
+      return fail(msg);
+    }
+  }
+  // 5. reads of bytes the schedule writes must be ordered after the write: the reader waits
+  //    on a flag the writer signals, or both sit on one queue (program order)
+  for (size_t i = 0; i < n; ++i) {
+    const HostOp& op = L.ops[i];
+    for (const pl_ref_t& s : op.src) {
+      auto it = writes.find({s.buf, s.rank});
+      if (it == writes.end()) continue;
+      const auto& v = it->second;
+      uint64_t lo = s.offset, hi = s.offset + op.count * elem_size(s.dtype);
+      auto first = std::upper_bound(v.begin(), v.end(), lo, [](uint64_t x, const Interval& iv) { return x < iv.hi; });
+      for (auto w = first; w != v.end() && w->lo < hi; ++w) {
+        const HostOp& wr = L.ops[w->op];
+        bool ordered = false;
+        if (w->op < (int)i) {
+          for (int f : op.waits)
+            if (f == wr.signal || f == wr.signal2) ordered = true;
+          if (wr.queue == op.queue) ordered = true;
+        }
+        if (!ordered) {
+          std::snprintf(msg, sizeof msg, "op %zu reads bytes written by op %d without a wait edge", i, w->op);
+          return fail(msg);
+        }
+      }
+    }
+  }
+  return PL_OK;
+}
+
+}  // namespace pl

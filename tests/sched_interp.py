@@ -1,0 +1,91 @@
+"""Test tool: replays a dumped schedule on the CPU with numpy.
+
+It is neither the oracle nor the product: it executes the op list produced by the host
+orchestrator (pl_schedule_dump) queue by queue in a *random* interleaving that honours only
+the wait/signal edges, over poison-filled output and scratch buffers.  A missing dependency
+edge therefore shows up as a wrong result (or as a deadlock) without any GPU.
+"""
+from __future__ import annotations
+
+import random
+
+import numpy as np
+
+from paper_2609_36954_b200 import binding as B
+from paper_2609_36954_b200 import inputs as gen
+
+_ES = {B.PL_BF16: 2, B.PL_F32: 4, B.PL_I32: 4, B.PL_U8: 1}
+
+
+def _load(buf, off, count, dtype):
+    raw = buf[off:off + count * _ES[dtype]]
+    if dtype == B.PL_BF16:
+        return gen.bf16_bits_to_f32(raw.view(np.uint16))
+    if dtype == B.PL_F32:
+        return raw.view(np.float32).copy()
+    if dtype == B.PL_I32:
+        return raw.view(np.uint32).copy()
+    return raw.copy()
+
+
+def _store(buf, off, vals, dtype):
+    if dtype == B.PL_BF16:
+        raw = gen.f32_to_bf16_bits(vals.astype(np.float32)).view(np.uint8)
+    elif dtype == B.PL_F32:
+        raw = vals.astype(np.float32).view(np.uint8)
+    elif dtype == B.PL_I32:
+        raw = vals.astype(np.uint32).view(np.uint8)
+    else:
+        raw = vals
+    buf[off:off + raw.size] = raw
+
+
+def run(ops, info, R, ins, seed=0, max_steps=None):
+    """ins[r]: numpy arrays (any dtype).  Returns list of uint8 output buffers."""
+    rng = random.Random(seed)
+    bufs = {B.PL_BUF_IN: [np.ascontiguousarray(a).view(np.uint8).reshape(-1) for a in ins],
+            B.PL_BUF_OUT: [np.full(int(info.out_bytes[r]), 0xFF, np.uint8) for r in range(R)],
+            B.PL_BUF_SCRATCH: [np.full(int(info.scratch_bytes) + 16, 0xFF, np.uint8) for _ in range(R)]}
+    for r in range(R):
+        assert bufs[B.PL_BUF_IN][r].size >= int(info.in_bytes[r])
+    nq = int(info.n_queues)
+    queues = [[] for _ in range(nq)]
+    for op in sorted(ops, key=lambda o: o.topo):
+        queues[op.queue].append(op)
+    heads = [0] * nq
+    flags = [0] * int(info.n_flags)
+    remaining = len(ops)
+    while remaining:
+        runnable = []
+        for q in range(nq):
+            if heads[q] < len(queues[q]):
+                op = queues[q][heads[q]]
+                if all(flags[op.wait_flag[k]] >= op.wait_need[k] for k in range(op.n_wait)):
+                    runnable.append(q)
+        if not runnable:
+            raise AssertionError("schedule deadlocks: no queue head is runnable")
+        q = rng.choice(runnable)
+        op = queues[q][heads[q]]
+        heads[q] += 1
+        remaining -= 1
+        n = int(op.count)
+        if op.kind == B.PL_OP_COPY:
+            data = _load(bufs[op.src[0].buf][op.src[0].rank], int(op.src[0].offset), n, B.PL_U8)
+            result, rdt = data, B.PL_U8
+        else:
+            first = op.src[0]
+            if first.dtype == B.PL_I32:
+                acc = np.zeros(n, np.uint32)
+            else:
+                acc = np.zeros(n, np.float32)
+            for k in range(op.n_src):
+                s = op.src[k]
+                acc = acc + _load(bufs[s.buf][s.rank], int(s.offset), n, s.dtype)
+            result, rdt = acc, op.dst.dtype
+        targets = range(R) if op.dst_bcast else [op.dst.rank]
+        for r in targets:
+            _store(bufs[op.dst.buf][r], int(op.dst.offset), result, rdt)
+        for f in (op.signal_flag, op.signal_flag2):
+            if f >= 0:
+                flags[f] += 1
+    return bufs[B.PL_BUF_OUT]

@@ -1,0 +1,284 @@
+"""Host orchestrator (planner communicator, no GPU): lowering, validation, error rules, and
+replay of the dumped op lists on the CPU against the oracle."""
+import numpy as np
+import pytest
+
+from oracle import oracle
+from paper_2609_36954_b200 import binding as B
+from paper_2609_36954_b200 import inputs as gen
+
+from sched_interp import run as interp_run
+
+DT = {"bf16": B.PL_BF16, "f32": B.PL_F32, "i32": B.PL_I32, "u8": B.PL_U8}
+NP = {"bf16": np.uint16, "f32": np.float32, "i32": np.int32, "u8": np.uint8}
+
+
+def check_float(got_f64, ref_f64, dtype):
+    if dtype == "bf16":
+        tol = 2.0 ** -7 * np.abs(ref_f64) + 1e-6
+    else:
+        tol = 1e-6 * np.abs(ref_f64) + 1e-7
+    err = np.abs(got_f64 - ref_f64)
+    assert np.all(err <= tol), f"max err/tol {np.max(err / tol)}"
+
+
+def compare_reduce(outs_u8, ref, dtype):
+    for r, o in enumerate(outs_u8):
+        if dtype == "i32":
+            assert np.array_equal(o.view(np.int32), ref[r])
+        elif dtype == "bf16":
+            check_float(gen.bf16_bits_to_f64(o.view(np.uint16)), ref[r], dtype)
+        else:
+            check_float(o.view(np.float32).astype(np.float64), ref[r], dtype)
+
+
+class Planner:
+    def __init__(self, R, dtype):
+        self.R, self.dtype = R, dtype
+        self.comm = B.pl_comm_create_planner(R, DT[dtype])
+        self.scheds = []
+
+    def build(self, coll, algo, count, chunk, **kw):
+        s = B.pl_schedule_build(self.comm, coll, algo, count, chunk, B.make_opts(**kw) if kw else None)
+        self.scheds.append(s)
+        return s
+
+    def close(self):
+        for s in self.scheds:
+            B.pl_schedule_destroy(s)
+        B.pl_comm_destroy(self.comm)
+
+
+ALLREDUCE_ALGOS = [B.PL_ALGO_RING, B.PL_ALGO_TREE, B.PL_ALGO_DIRECT, B.PL_ALGO_ONESHOT, B.PL_ALGO_DIRECT_FUSED]
+
+
+@pytest.mark.parametrize("R", [2, 3, 4, 5, 8])
+@pytest.mark.parametrize("algo", ALLREDUCE_ALGOS)
+@pytest.mark.parametrize("dtype", ["i32", "bf16", "f32"])
+def test_allreduce_schedules_replay_to_oracle(R, algo, dtype):
+    es = B.DTYPE_SIZE[DT[dtype]]
+    n = R * (16 // es) * 13  # 13 vectors per partition: ragged against every chunk size below
+    x = gen.rank_inputs(R, n, dtype, seed=R)
+    ref = oracle.allreduce(x, dtype)
+    pl = Planner(R, dtype)
+    try:
+        for chunk, slice_b in [(16, 16), (48, 32), (1 << 20, 64), (64, 0)]:
+            s = pl.build(B.PL_ALLREDUCE, algo, n, chunk, slice_bytes=slice_b, n_ctas=3 * R)
+            st, msg = B.pl_schedule_validate(s)
+            assert st == B.PL_OK, msg
+            info = B.pl_schedule_info(s)
+            ops = B.pl_schedule_dump(s)
+            assert len(ops) == info.n_ops
+            for seed in (0, 1):
+                outs = interp_run(ops, info, R, x, seed=seed)
+                compare_reduce(outs, ref, dtype)
+    finally:
+        pl.close()
+
+
+@pytest.mark.parametrize("R", [2, 3, 5, 8])
+@pytest.mark.parametrize("algo", [B.PL_ALGO_RING, B.PL_ALGO_DIRECT])
+def test_reduce_scatter_and_allgather_replay(R, algo):
+    for dtype in ("i32", "bf16"):
+        es = B.DTYPE_SIZE[DT[dtype]]
+        n = R * (16 // es) * 7
+        x = gen.rank_inputs(R, n, dtype, seed=7)
+        pl = Planner(R, dtype)
+        try:
+            s = pl.build(B.PL_REDUCE_SCATTER, algo, n, 48, slice_bytes=32, n_ctas=2 * R)
+            info = B.pl_schedule_info(s)
+            outs = interp_run(B.pl_schedule_dump(s), info, R, x, seed=3)
+            compare_reduce(outs, oracle.reduce_scatter(x, dtype), dtype)
+            assert info.message_bytes == n * es
+            # all-gather of the same buffers (contribution = n elements)
+            s = pl.build(B.PL_ALLGATHER, algo, n, 48, slice_bytes=32, n_ctas=2 * R)
+            info = B.pl_schedule_info(s)
+            outs = interp_run(B.pl_schedule_dump(s), info, R, x, seed=4)
+            ref = oracle.allgather(x)
+            for r in range(R):
+                assert np.array_equal(outs[r], ref[r].view(np.uint8))
+            assert info.message_bytes == n * es * R
+        finally:
+            pl.close()
+
+
+@pytest.mark.parametrize("R", [2, 4, 7])
+def test_alltoall_and_alltoallv_replay(R):
+    pl = Planner(R, "u8")
+    try:
+        m = 16 * 5
+        x = gen.rank_coded_bytes(R, R * m)
+        s = pl.build(B.PL_ALLTOALL, B.PL_ALGO_DIRECT, R * m, 32, slice_bytes=16)
+        outs = interp_run(B.pl_schedule_dump(s), B.pl_schedule_info(s), R, x)
+        ref = oracle.alltoall(x)
+        for r in range(R):
+            assert np.array_equal(outs[r], ref[r])
+        rng = np.random.default_rng(R)
+        C = rng.integers(0, 6, size=(R, R)) * 16
+        C[0, R - 1] = 0
+        xs = [gen.rank_coded_bytes(R, max(16, int(C[p].sum())))[p][: int(C[p].sum())] for p in range(R)]
+        s = B.pl_schedule_build_v(pl.comm, B.PL_ALLTOALLV, B.PL_ALGO_DIRECT, C.tolist(), 48, None)
+        pl.scheds.append(s)
+        info = B.pl_schedule_info(s)
+        outs = interp_run(B.pl_schedule_dump(s), info, R, xs)
+        ref = oracle.alltoallv(xs, C)
+        for r in range(R):
+            assert int(info.out_bytes[r]) == int(C[:, r].sum())
+            assert np.array_equal(outs[r], ref[r])
+    finally:
+        pl.close()
+
+
+@pytest.mark.parametrize("algo", [B.PL_ALGO_ONESHOT, B.PL_ALGO_DIRECT, B.PL_ALGO_DIRECT_FUSED])
+def test_layered_allreduce_replay_and_program_order(algo):
+    R, n, Lyr = 4, 4 * 8 * 3, 5
+    dtype = "bf16"
+    pl = Planner(R, dtype)
+    try:
+        x = [np.concatenate([gen.normal_bf16(n, 0, l * R + r) for l in range(Lyr)]) for r in range(R)]
+        s = B.pl_schedule_build_layers(pl.comm, algo, n, Lyr, B.make_opts(slice_bytes=32, n_ctas=2 * R))
+        pl.scheds.append(s)
+        st, msg = B.pl_schedule_validate(s)
+        assert st == B.PL_OK, msg
+        info = B.pl_schedule_info(s)
+        assert info.n_layers == Lyr
+        ops = B.pl_schedule_dump(s)
+        outs = interp_run(ops, info, R, x, seed=5)
+        for l in range(Lyr):
+            xl = [a[l * n:(l + 1) * n] for a in x]
+            ref = oracle.allreduce(xl, dtype)
+            for r in range(R):
+                got = gen.bf16_bits_to_f64(outs[r].view(np.uint16)[l * n:(l + 1) * n])
+                check_float(got, ref[r], dtype)
+        # program order: an op of layer l+1 that reads rank p's input waits on a flag that is
+        # only complete once every op writing out_p in layer l has signalled
+        writers = {}
+        for o in ops:
+            for f in (o.signal_flag, o.signal_flag2):
+                if f >= 0:
+                    writers.setdefault(f, []).append(o)
+        for o in ops:
+            if o.layer == 0 or o.kind == B.PL_OP_COPY:
+                continue
+            waited = {o.wait_flag[k] for k in range(o.n_wait)}
+            for k in range(o.n_src):
+                p = o.src[k].rank
+                prev_writers = [w for w in ops if w.layer == o.layer - 1 and
+                                (w.dst_bcast or w.dst.rank == p) and w.dst.buf == B.PL_BUF_OUT]
+                assert prev_writers
+                for w in prev_writers:
+                    assert {w.signal_flag, w.signal_flag2} & waited, "missing cross-layer edge"
+    finally:
+        pl.close()
+
+
+def test_config1_op_counts_and_bytes():
+    # all-reduce, R=4, 262144 fp32 per rank, ring, 64 KiB chunks, unsliced:
+    # 3 reduce-scatter hops + 3 all-gather hops, 4 ranks, 4 chunks per partition
+    pl = Planner(4, "f32")
+    try:
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, 262144, 65536, slice_bytes=65536)
+        info = B.pl_schedule_info(s)
+        ops = B.pl_schedule_dump(s)
+        assert sum(o.kind == B.PL_OP_COPY_REDUCE for o in ops) == 48
+        assert sum(o.kind == B.PL_OP_COPY for o in ops) == 48
+        M = 1 << 20
+        assert info.bytes_read + info.bytes_written == 5 * 3 * M  # 5(R-1)M
+        assert info.message_bytes == M
+    finally:
+        pl.close()
+
+
+def test_schedule_bytes_match_closed_forms_bf16_R8():
+    R, M = 8, 1 << 20
+    n = M // 2
+    pl = Planner(R, "bf16")
+    try:
+        def total(coll, algo, count=n):
+            i = B.pl_schedule_info(pl.build(coll, algo, count, 1 << 16))
+            return i.bytes_read + i.bytes_written
+        assert total(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT) == (R + 1) * M
+        assert total(B.PL_REDUCE_SCATTER, B.PL_ALGO_RING) == 33 * M  # fp32 partials: (16+10(R-3))/2 per byte
+        assert total(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R) == 2 * R * M  # per-rank-message M = gathered size
+        assert total(B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT) == R * (R + 1) * M
+        assert total(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT) == (3 * R - 1) * M
+        assert total(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT_FUSED) == 2 * R * M
+        assert total(B.PL_ALLREDUCE, B.PL_ALGO_RING) == 47 * M
+        assert total(B.PL_ALLREDUCE, B.PL_ALGO_TREE) == 47 * M
+    finally:
+        pl.close()
+
+
+def test_error_rules():
+    with pytest.raises(B.PurlinError) as e:
+        B.pl_comm_create_planner(1, B.PL_BF16)
+    assert e.value.status == B.PL_ERR_INVALID_ARG
+    with pytest.raises(B.PurlinError):
+        B.pl_comm_create_planner(17, B.PL_BF16)
+    pl = Planner(8, "bf16")
+    try:
+        def status(fn):
+            with pytest.raises(B.PurlinError) as ei:
+                fn()
+            return ei.value.status
+        # bytes not divisible by R*16
+        assert status(lambda: pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, 8 * 8 + 8, 64)) == B.PL_ERR_INVALID_ARG
+        # chunk not a multiple of 16 / zero
+        assert status(lambda: pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 24)) == B.PL_ERR_INVALID_ARG
+        assert status(lambda: pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 0)) == B.PL_ERR_INVALID_ARG
+        # tree on a non-allreduce, fused all-gather
+        assert status(lambda: pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_TREE, 1024, 64)) == B.PL_ERR_UNSUPPORTED
+        assert status(lambda: pl.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT_FUSED, 1024, 64)) == B.PL_ERR_UNSUPPORTED
+        assert status(lambda: pl.build(B.PL_ALLTOALL, B.PL_ALGO_RING, 1024, 64)) == B.PL_ERR_UNSUPPORTED
+        # more CTAs than can be co-resident
+        assert status(lambda: pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1 << 20, 1 << 16, n_ctas=100000)) == B.PL_ERR_OVERSUBSCRIBED
+        # all-to-all-v segment not 16-byte aligned
+        C = [[4] * 8 for _ in range(8)]
+        assert status(lambda: B.pl_schedule_build_v(pl.comm, B.PL_ALLTOALLV, B.PL_ALGO_DIRECT, C, 64)) == B.PL_ERR_ALIGNMENT
+        # planner communicators cannot execute
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 64)
+        bufs = B.make_bufs([16] * 8, [16] * 8, [1 << 20] * 8, [1 << 20] * 8)
+        assert status(lambda: B.pl_execute(s, bufs)) == B.PL_ERR_UNSUPPORTED
+        # layered schedules: ring is not offered
+        assert status(lambda: B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_RING, 1024, 4)) == B.PL_ERR_UNSUPPORTED
+        # a communicator with live schedules cannot be destroyed
+        assert status(lambda: B.pl_comm_destroy(pl.comm)) == B.PL_ERR_INVALID_ARG
+    finally:
+        pl.close()
+    plu = Planner(4, "u8")
+    try:
+        with pytest.raises(B.PurlinError) as ei:
+            plu.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 64)
+        assert ei.value.status == B.PL_ERR_UNSUPPORTED
+    finally:
+        plu.close()
+
+
+def test_validator_catches_a_broken_edge():
+    # raising one wait's needed count makes the replay deadlock: the interpreter notices
+    pl = Planner(4, "i32")
+    try:
+        n = 4 * 4 * 4
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 16)
+        ops = B.pl_schedule_dump(s)
+        victim = next(o for o in ops if o.n_wait > 0)
+        victim.wait_need[0] += 1
+        with pytest.raises(AssertionError):
+            interp_run(ops, B.pl_schedule_info(s), 4, gen.rank_coded_i32(4, n))
+    finally:
+        pl.close()
+
+
+def test_queues_are_rank_owned_and_balanced():
+    pl = Planner(8, "bf16")
+    try:
+        s = pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, 8 << 20, 1 << 20, n_ctas=144, slice_bytes=65536)
+        ops = B.pl_schedule_dump(s)
+        load = {}
+        for o in ops:
+            assert o.queue % 8 == o.exec_rank
+            load[o.queue] = load.get(o.queue, 0) + o.count
+        assert len(load) == 144
+        assert max(load.values()) <= 1.25 * min(load.values())
+    finally:
+        pl.close()
