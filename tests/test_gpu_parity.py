@@ -1,0 +1,294 @@
+"""GPU parity: the CUDA path (through the C-ABI) against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+
+from oracle import oracle
+from paper_2609_36954_b200 import binding as B
+from paper_2609_36954_b200 import inputs as gen
+
+from gpu_harness import Session, check_float, to_dev
+
+pytestmark = pytest.mark.gpu
+
+ALL_AR = [B.PL_ALGO_RING, B.PL_ALGO_TREE, B.PL_ALGO_DIRECT, B.PL_ALGO_ONESHOT, B.PL_ALGO_DIRECT_FUSED]
+ALGO_NAME = {B.PL_ALGO_RING: "ring", B.PL_ALGO_TREE: "tree", B.PL_ALGO_DIRECT: "direct",
+             B.PL_ALGO_ONESHOT: "oneshot", B.PL_ALGO_DIRECT_FUSED: "fused"}
+
+
+def as_f64(out_u8, dtype):
+    if dtype == "bf16":
+        return gen.bf16_bits_to_f64(out_u8.view(np.uint16))
+    return out_u8.view(np.float32).astype(np.float64)
+
+
+def compare_reduce(outs, ref, dtype):
+    worst = 0.0
+    for r, o in enumerate(outs):
+        if dtype == "i32":
+            assert np.array_equal(o.view(np.int32), ref[r]), f"rank {r} differs"
+        else:
+            worst = max(worst, check_float(as_f64(o, dtype), ref[r], dtype))
+    return worst
+
+
+# ---- config 1: all-reduce R=4, 262144 fp32 + int32 twin, ring, 64 KiB chunks ------------
+@pytest.mark.parametrize("dtype", ["f32", "i32"])
+def test_config1_allreduce_ring(dtype):
+    R, n = 4, 262144
+    x = gen.rank_inputs(R, n, dtype, seed=0)
+    ref = oracle.allreduce(x, dtype)
+    ses = Session(R, dtype)
+    try:
+        for slice_bytes in (65536, 16384):
+            s = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 65536, slice_bytes=slice_bytes)
+            outs, info = ses.execute(s, x, repeats=3)  # repeats exercise epoch reuse of the flags
+            compare_reduce(outs, ref, dtype)
+            if dtype == "i32":  # closed form: 4 i + 262144 * (0+1+2+3)
+                i = np.arange(n, dtype=np.int64)
+                assert np.array_equal(outs[2].view(np.int32).astype(np.int64), 4 * i + 1572864)
+    finally:
+        ses.close()
+
+
+# ---- every all-reduce algorithm, ragged sizes, several R, every dtype ---------------------
+@pytest.mark.parametrize("algo", ALL_AR)
+@pytest.mark.parametrize("dtype", ["bf16", "f32", "i32"])
+@pytest.mark.parametrize("R", [2, 3, 8])
+def test_allreduce_all_algorithms(algo, dtype, R):
+    es = B.DTYPE_SIZE[{"bf16": B.PL_BF16, "f32": B.PL_F32, "i32": B.PL_I32}[dtype]]
+    # partition = 37 KiB + 16 B: not a multiple of the chunk, the slice or the CTA width
+    n = R * ((37 * 1024 + 16) // es)
+    # Single-op reductions (direct, one-shot, fused) use a compensated fp32 accumulator and
+    # meet the fp32 tolerance for any mantissas, so they get full-mantissa N(0,1) data.  Ring
+    # and tree round the travelling fp32 partial once per hop: they get the configuration's
+    # own data (uniform on the 2^-23 grid) under the strict tolerance, and N(0,1) data under
+    # the textbook bound of recursive summation, (R-1) * 2^-24 * sum_p |x_p|.
+    multi_hop = algo in (B.PL_ALGO_RING, B.PL_ALGO_TREE)
+    x = gen.rank_inputs(R, n, "f32n" if (dtype == "f32" and not multi_hop) else dtype, seed=11)
+    ref = oracle.allreduce(x, dtype)
+    ses = Session(R, dtype)
+    try:
+        for chunk, sl in [(8192, 4096), (1 << 20, 16384)]:
+            s = ses.build(B.PL_ALLREDUCE, algo, n, chunk, slice_bytes=sl)
+            outs, _ = ses.execute(s, x, repeats=2)
+            compare_reduce(outs, ref, dtype)
+        if dtype == "f32" and multi_hop:
+            xn = gen.rank_inputs(R, n, "f32n", seed=12)
+            refn = oracle.allreduce(xn, "f32")
+            bound = (R - 1) * 2.0 ** -24 * np.sum([np.abs(a.astype(np.float64)) for a in xn], axis=0)
+            outs, _ = ses.execute(s, xn)
+            for r in range(R):
+                err = np.abs(outs[r].view(np.float32).astype(np.float64) - refn[r])
+                assert np.all(err <= bound + 1e-12)
+    finally:
+        ses.close()
+
+
+def test_allreduce_tiny_and_single_vector():
+    for R in (2, 5):
+        for dtype in ("bf16", "i32"):
+            es = 2 if dtype == "bf16" else 4
+            n = R * (16 // es)  # one 16-byte vector per partition
+            x = gen.rank_inputs(R, n, dtype, seed=1)
+            ref = oracle.allreduce(x, dtype)
+            ses = Session(R, dtype)
+            try:
+                for algo in ALL_AR:
+                    s = ses.build(B.PL_ALLREDUCE, algo, n, 16)
+                    outs, _ = ses.execute(s, x)
+                    compare_reduce(outs, ref, dtype)
+            finally:
+                ses.close()
+
+
+@pytest.mark.parametrize("algo", [B.PL_ALGO_RING, B.PL_ALGO_DIRECT])
+@pytest.mark.parametrize("dtype", ["bf16", "i32", "f32"])
+def test_reduce_scatter_and_allgather(algo, dtype):
+    R = 8
+    es = 2 if dtype == "bf16" else 4
+    n = R * (300 * 1024 + 48) // es // 1  # partition 300 KiB + 48 B
+    n -= n % (R * 16 // es)
+    x = gen.rank_inputs(R, n, dtype, seed=3)  # fp32: the 2^-23 grid of the fp32 configuration
+    ses = Session(R, dtype)
+    try:
+        for chunk in (256 * 1024, 1 << 20):
+            s = ses.build(B.PL_REDUCE_SCATTER, algo, n, chunk)
+            outs, _ = ses.execute(s, x, repeats=2)
+            compare_reduce(outs, oracle.reduce_scatter(x, dtype), dtype)
+            m = n // R
+            contrib = [a[:m].copy() for a in x]
+            s = ses.build(B.PL_ALLGATHER, algo, m, chunk)
+            outs, _ = ses.execute(s, contrib, repeats=2)
+            ref = oracle.allgather(contrib)
+            for r in range(R):
+                assert np.array_equal(outs[r], ref[r].view(np.uint8))
+    finally:
+        ses.close()
+
+
+def test_alltoall_and_alltoallv_bit_exact():
+    R = 8
+    ses = Session(R, "u8")
+    try:
+        m = 100 * 1024 + 16
+        x = gen.rank_coded_bytes(R, R * m)
+        s = ses.build(B.PL_ALLTOALL, B.PL_ALGO_DIRECT, R * m, 65536)
+        outs, _ = ses.execute(s, x)
+        ref = oracle.alltoall(x)
+        for r in range(R):
+            assert np.array_equal(outs[r], ref[r])
+        # the paper's Zipf(0.125) split rotated per rank, T = 1 MiB, plus a matrix with empty segments
+        for C in (gen.alltoallv_counts_bytes(1 << 20), None):
+            if C is None:
+                rng = np.random.default_rng(5)
+                C = rng.integers(0, 5000, size=(R, R)) * 16
+                C[2, :] = 0
+                C[:, 5] = 0
+            xs = [gen.rank_coded_bytes(R, max(16, int(C[p].sum())))[p][: int(C[p].sum())] for p in range(R)]
+            s = ses.build_v(C.tolist(), 65536)
+            outs, info = ses.execute(s, xs)
+            ref = oracle.alltoallv(xs, C)
+            for r in range(R):
+                assert outs[r].size == int(C[:, r].sum())
+                assert np.array_equal(outs[r], ref[r])
+    finally:
+        ses.close()
+
+
+def test_float_special_cases_on_gpu():
+    R, n = 8, 8 * 4096
+    base = gen.normal_bf16(n, 11, 0)
+    ses = Session(R, "bf16")
+    try:
+        s = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, n, 65536)
+        # all ranks equal -> 8x exactly (power of two), bit-exact even in bf16
+        outs, _ = ses.execute(s, [base.copy() for _ in range(R)])
+        want = gen.f32_to_bf16_bits((gen.bf16_bits_to_f32(base) * 8).astype(np.float32))
+        assert np.array_equal(outs[3].view(np.uint16), want)
+        # +x / -x pairs cancel to zero
+        neg = base ^ np.uint16(0x8000)
+        outs, _ = ses.execute(s, [base if p % 2 == 0 else neg for p in range(R)])
+        assert np.all(gen.bf16_bits_to_f32(outs[0].view(np.uint16)) == 0.0)
+        # one non-zero rank -> copy of it
+        zero = np.zeros(n, np.uint16)
+        outs, _ = ses.execute(s, [base if p == 6 else zero for p in range(R)])
+        assert np.array_equal(outs[1].view(np.uint16), base)
+    finally:
+        ses.close()
+
+
+def test_bf16_direct_sum_is_the_correctly_rounded_sum():
+    # fp32 accumulation of 8 bf16 values followed by one rounding reproduces
+    # bf16_rne(exact sum) on (nearly) every element; report the fraction, require 99.9 %
+    R, n = 8, 8 * 65536
+    x = gen.rank_inputs(R, n, "bf16", seed=0)
+    ref = oracle.allreduce(x, "bf16")
+    ses = Session(R, "bf16")
+    try:
+        s = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT, n, 1 << 20)
+        outs, _ = ses.execute(s, x)
+        want = gen.f32_to_bf16_bits(ref[0].astype(np.float32))
+        frac = float(np.mean(outs[0].view(np.uint16) == want))
+        assert frac > 0.999, frac
+    finally:
+        ses.close()
+
+
+def test_run_to_run_determinism():
+    R, n = 8, 8 * 40000
+    x = gen.rank_inputs(R, n, "bf16", seed=4)
+    ses = Session(R, "bf16")
+    try:
+        for algo in (B.PL_ALGO_RING, B.PL_ALGO_DIRECT):
+            s = ses.build(B.PL_ALLREDUCE, algo, n, 32768)
+            a, _ = ses.execute(s, x)
+            b, _ = ses.execute(s, x, repeats=3)
+            for r in range(R):
+                assert np.array_equal(a[r], b[r])
+    finally:
+        ses.close()
+
+
+@pytest.mark.parametrize("algo", [B.PL_ALGO_ONESHOT, B.PL_ALGO_DIRECT, B.PL_ALGO_DIRECT_FUSED])
+@pytest.mark.parametrize("batch", [1, 8])
+def test_layered_decode_allreduce(algo, batch):
+    # tensor-parallel decode shape: batch x hidden 8192 bf16, several layers in one launch
+    R, hidden, Lyr = 8, 8192, 6
+    n = batch * hidden
+    x = [np.concatenate([gen.normal_bf16(n, 0, l * R + r) for l in range(Lyr)]) for r in range(R)]
+    ses = Session(R, "bf16")
+    try:
+        s = ses.build_layers(algo, n, Lyr)
+        for rep in range(3):  # back-to-back executes with poisoned outputs: epoch reuse
+            outs, info = ses.execute(s, x)
+            assert info.n_layers == Lyr
+            for l in range(Lyr):
+                ref = oracle.allreduce([a[l * n:(l + 1) * n] for a in x], "bf16")
+                for r in range(R):
+                    check_float(as_f64(outs[r], "bf16")[l * n:(l + 1) * n], ref[r], "bf16")
+            x = [np.roll(a, 8 * (rep + 1)) for a in x]  # new inputs next time
+    finally:
+        ses.close()
+
+
+def test_execute_argument_errors():
+    R, n = 4, 4 * 64
+    ses = Session(R, "f32")
+    try:
+        s = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT, n, 1024)
+        info = B.pl_schedule_info(s)
+        d_in = [to_dev(np.zeros(n, np.float32)) for _ in range(R)]
+        d_out = [to_dev(np.zeros(n + 8, np.float32)) for _ in range(R)]
+        ib = [int(info.in_bytes[r]) for r in range(R)]
+        ob = [int(info.out_bytes[r]) for r in range(R)]
+
+        def status(bufs):
+            with pytest.raises(B.PurlinError) as e:
+                B.pl_execute(s, bufs)
+            return e.value.status
+        ins = [t.data_ptr() for t in d_in]
+        outs = [t.data_ptr() for t in d_out]
+        assert status(B.make_bufs(ins, [o + 4 for o in outs], ib, ob)) == B.PL_ERR_ALIGNMENT
+        assert status(B.make_bufs(ins, outs, ib, [b - 16 for b in ob])) == B.PL_ERR_INVALID_ARG
+        assert status(B.make_bufs(ins, [ins[0]] + outs[1:], ib, ob)) == B.PL_ERR_INVALID_ARG  # in/out overlap
+        assert status(B.make_bufs([0] + ins[1:], outs, ib, ob)) == B.PL_ERR_INVALID_ARG
+        with pytest.raises(B.PurlinError) as e:
+            ses.build(B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT, n, 1024, n_ctas=1 << 20)
+        assert e.value.status == B.PL_ERR_OVERSUBSCRIBED
+    finally:
+        ses.close()
+
+
+def test_bounded_wait_reports_timeout_and_recovers():
+    # host-made failure: one wait edge is raised beyond what the schedule will ever signal;
+    # with a 20 ms limit the kernel must return, report PL_ERR_TIMEOUT, and the GPU must stay
+    # usable: after pl_comm_reset an intact schedule runs and matches the oracle.
+    R, n = 4, 4 * 4096
+    x = gen.rank_inputs(R, n, "i32")
+    ref = oracle.allreduce(x, "i32")
+    ses = Session(R, "i32")
+    try:
+        bad = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 4096, timeout_ns=20_000_000)
+        ops = B.pl_schedule_dump(bad)
+        victim = next(o.topo for o in ops if o.n_wait > 0)
+        B.pl_schedule_debug_break_wait(bad, victim)
+        info = B.pl_schedule_info(bad)
+        import torch
+        from gpu_harness import poison, stream_handle
+        d_in = [to_dev(a) for a in x]
+        d_out = [poison(info.out_bytes[r]) for r in range(R)]
+        bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                           [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
+        B.pl_execute(bad, bufs, stream_handle())
+        torch.cuda.synchronize()
+        st = B.pl_comm_status(ses.comm)
+        assert st.code == B.PL_ERR_TIMEOUT
+        assert st.expected > st.observed
+        B.pl_comm_reset(ses.comm, stream_handle())
+        torch.cuda.synchronize()
+        assert B.pl_comm_status(ses.comm).code == B.PL_OK
+        good = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 4096)
+        outs, _ = ses.execute(good, x)
+        compare_reduce(outs, ref, "i32")
+    finally:
+        ses.close()
