@@ -62,7 +62,17 @@ typedef enum {
 /* Element types.  Reductions convert each element to fp32, accumulate in fp32 and
  * convert once at the end (Sec. 3.3, Eq. "rank-order"); int32 sums wrap.  PL_U8 is
  * valid for copy-only collectives. */
-typedef enum { PL_BF16 = 0, PL_F32 = 1, PL_I32 = 2, PL_U8 = 3 } pl_dtype_t;
+typedef enum {
+  PL_BF16 = 0,
+  PL_F32 = 1,
+  PL_I32 = 2,
+  PL_U8 = 3,
+  /* Internal, appears only in op dumps: partial sums of an fp32 reduction that travel
+   * between ops (ring hops, tree levels) as a (sum, correction) pair of fp32 per element,
+   * 8 bytes, stored in blocks of 4 sums followed by their 4 corrections.  Not a valid
+   * communicator dtype. */
+  PL_F32X2 = 4
+} pl_dtype_t;
 
 /* Collectives (Listing 1): reduce-scatter = reduce, scattered->packed; all-gather = copy,
  * packed->scattered; all-to-all = copy, scattered->transposed; all-to-all-v its runtime-
@@ -83,7 +93,8 @@ typedef enum {
  *   PL_ALGO_ONESHOT       all-reduce only: every rank reduces the whole message itself.
  *   PL_ALGO_DIRECT_FUSED  all-reduce only: the reducer of partition k writes the result
  *                         into all R outputs (no gather step, fewest bytes).
- *   PL_ALGO_RING          textbook ring; partial sums travel in fp32 (int32 for ints).
+ *   PL_ALGO_RING          textbook ring; partial sums of bf16 data travel in fp32, of fp32
+ *                         data as compensated fp32 pairs (PL_F32X2), of int32 data in int32.
  *   PL_ALGO_TREE          all-reduce only: binomial reduce to rank 0, binomial broadcast.
  * Ring and tree are not in the paper (its only pattern is the direct pull); they are the
  * classical algorithms the benchmark configurations name. */

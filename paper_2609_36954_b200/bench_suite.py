@@ -1,0 +1,183 @@
+"""Timing of every benchmark configuration on one GPU (CUDA events, C-ABI calls only).
+
+Used by ``bench.py --suite``.  One JSON line per measured point:
+effective GB/s (message size / time, the paper's algorithm bandwidth), schedule GB/s
+(bytes the schedule reads + writes / time), fraction of the HBM peak, and microseconds.
+Inputs are seeded synthetic data of the configuration's shape; values do not influence
+timing, so large buffers are filled by tiling a generated block.
+"""
+from __future__ import annotations
+
+import json
+import os
+import sys
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import inputs as gen
+
+MIB = 1 << 20
+ALGO = {"ring": B.PL_ALGO_RING, "tree": B.PL_ALGO_TREE, "direct": B.PL_ALGO_DIRECT,
+        "oneshot": B.PL_ALGO_ONESHOT, "fused": B.PL_ALGO_DIRECT_FUSED}
+
+
+def _peak():
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    try:
+        return float(json.load(open(os.path.join(root, "MEASURED_PEAKS.json")))["hbm_gbs"])
+    except Exception:
+        return 6650.0
+
+
+def _fill(nbytes, stream_id):
+    """Device buffer of nbytes filled with tiled bf16 N(0,1) bits."""
+    blk = gen.normal_bf16(min(nbytes // 2, 1 << 20) or 8, 0, stream_id)
+    t = torch.from_numpy(blk.view(np.int16)).cuda()
+    reps = (nbytes // 2 + t.numel() - 1) // t.numel()
+    return t.repeat(reps)[: max(8, nbytes // 2)].contiguous()
+
+
+def _time(fn, iters, warmup=3, per_call_events=False):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if per_call_events:
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+        ev[0].record()
+        for i in range(iters):
+            fn()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        ms = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(iters)])
+        return float(np.median(ms) * 1e3), float(np.percentile(ms, 10) * 1e3), float(np.percentile(ms, 90) * 1e3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / iters
+    return us, us, us
+
+
+class Bench:
+    def __init__(self, out_path=None, opts_kw=None):
+        self.peak = _peak()
+        self.out = open(out_path, "w") if out_path else None
+        self.stream = torch.cuda.current_stream().cuda_stream
+        self.opts_kw = opts_kw or {}
+
+    def emit(self, rec):
+        line = json.dumps(rec)
+        print(line, flush=True)
+        if self.out:
+            self.out.write(line + "\n")
+            self.out.flush()
+
+    def collective(self, cfg, R, dtype, coll, algo, count, chunk, iters=20, layers=0, **kw):
+        comm = B.pl_comm_create(R, dtype)
+        okw = dict(self.opts_kw)
+        okw.update(kw)
+        opts = B.make_opts(**okw)
+        try:
+            if layers:
+                s = B.pl_schedule_build_layers(comm, ALGO[algo], count, layers, opts)
+            else:
+                s = B.pl_schedule_build(comm, coll, ALGO[algo], count, chunk, opts)
+        except B.PurlinError as e:
+            B.pl_comm_destroy(comm)
+            self.emit({"cfg": cfg, "algo": algo, "error": str(e)})
+            return None
+        info = B.pl_schedule_info(s)
+        d_in = [_fill(int(info.in_bytes[r]), r) for r in range(R)]
+        d_out = [torch.empty(max(16, int(info.out_bytes[r])), dtype=torch.uint8, device="cuda") for r in range(R)]
+        bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                           [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
+        p50, p10, p90 = _time(lambda: B.pl_execute(s, bufs, self.stream), iters, per_call_events=True)
+        st = B.pl_comm_status(comm)
+        nl = max(1, layers)
+        sched_bytes = info.bytes_read + info.bytes_written
+        rec = {"cfg": cfg, "coll": int(coll), "algo": algo, "R": R, "dtype": int(dtype),
+               "message_bytes": int(info.message_bytes), "chunk": int(min(chunk, 1 << 40)), "layers": layers,
+               "us": p50 / nl, "us_p10": p10 / nl, "us_p90": p90 / nl,
+               "eff_gbs": info.message_bytes * nl / p50 / 1e3, "sched_gbs": sched_bytes / p50 / 1e3,
+               "hbm_frac_measured": sched_bytes / p50 / 1e3 / self.peak, "hbm_frac_8TBps": sched_bytes / p50 / 1e3 / 8000.0,
+               "n_ops": int(info.n_ops), "grid": int(info.grid), "threads": int(info.threads),
+               "slice_bytes": int(info.slice_bytes), "datapath": int(info.datapath), "status": int(st.code)}
+        self.emit(rec)
+        B.pl_schedule_destroy(s)
+        B.pl_comm_destroy(comm)
+        del d_in, d_out
+        return rec
+
+    def moe(self, cfg, R=8, T=4096, H=7168, E=256, K=8, identity=False, iters=10):
+        idx, gates = gen.moe_routing(R, T, E, K, identity_perm=identity)
+        counts = np.zeros((R, R), np.int64)
+        for p in range(R):
+            counts[p] = np.bincount(idx[p].ravel() // (E // R), minlength=R)
+        cap = int(counts.sum(axis=0).max())
+        comm = B.pl_comm_create(R, B.PL_BF16)
+        plan = B.pl_moe_plan_create(comm, T, H, E, K, cap)
+        d_x = [_fill(T * H * 2, r) for r in range(R)]
+        d_i = [torch.from_numpy(a).cuda() for a in idx]
+        d_g = [torch.from_numpy(a).cuda() for a in gates]
+        d_recv = [torch.empty(cap * H, dtype=torch.int16, device="cuda") for _ in range(R)]
+        d_meta = [torch.empty(cap * 4, dtype=torch.int32, device="cuda") for _ in range(R)]
+        d_out = [torch.empty(T * H, dtype=torch.int16, device="cuda") for _ in range(R)]
+        px = [t.data_ptr() for t in d_x]
+        pi = [t.data_ptr() for t in d_i]
+        pr = [t.data_ptr() for t in d_recv]
+        pm = [t.data_ptr() for t in d_meta]
+        pg = [t.data_ptr() for t in d_g]
+        po = [t.data_ptr() for t in d_out]
+        disp, _, _ = _time(lambda: B.pl_moe_dispatch(plan, px, pi, pr, pm, self.stream), iters, per_call_events=True)
+        comb, _, _ = _time(lambda: B.pl_moe_combine(plan, pr, pg, po, self.stream), iters, per_call_events=True)
+        st = B.pl_moe_plan_read(plan, 0, 0, 0, self.stream)
+        rows = R * T * K
+        row_b = H * 2
+        d_bytes = R * T * row_b + rows * row_b
+        c_bytes = rows * row_b + R * T * row_b
+        self.emit({"cfg": cfg, "routing": "identity" if identity else "permuted", "rows": rows, "cap": cap,
+                   "max_over_mean_rows": float(counts.sum(axis=0).max() / counts.sum(axis=0).mean()),
+                   "dispatch_us": disp, "combine_us": comb,
+                   "dispatch_gbs": d_bytes / disp / 1e3, "combine_gbs": c_bytes / comb / 1e3,
+                   "dispatch_frac_measured": d_bytes / disp / 1e3 / self.peak,
+                   "combine_frac_measured": c_bytes / comb / 1e3 / self.peak, "status": int(st)})
+        B.pl_moe_plan_destroy(plan)
+        B.pl_comm_destroy(comm)
+
+
+def main(args=None):
+    which = os.environ.get("PL_SUITE", "c1,c2,c3,c4,c5").split(",")
+    os.makedirs("gpurun_out", exist_ok=True)
+    b = Bench(os.environ.get("PL_SUITE_OUT", "gpurun_out/suite.jsonl"))
+    if "c1" in which:
+        for dt in (B.PL_F32, B.PL_I32):
+            b.collective("C1", 4, dt, B.PL_ALLREDUCE, "ring", 262144, 65536, iters=50)
+    if "c2" in which:
+        n = 32 * MIB  # 64 MiB bf16 per rank
+        for algo in ("direct", "ring"):
+            for chunk in (256 * 1024, MIB):
+                b.collective("C2-RS", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, algo, n, chunk)
+                b.collective("C2-AG", 8, B.PL_BF16, B.PL_ALLGATHER, algo, n // 8, chunk)
+    if "c3" in which:
+        for lg in range(12, 29):
+            size = 1 << lg
+            for algo in ("ring", "tree", "oneshot", "direct", "fused"):
+                if algo == "oneshot" and size > 64 * MIB:
+                    continue
+                chunk = max(16, min(MIB, size // 8))
+                b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30 if lg < 24 else 10)
+    if "c4" in which:
+        b.moe("C4", identity=False)
+        b.moe("C4", identity=True)
+    if "c5" in which:
+        for batch in (1, 8, 64):
+            for algo in ("oneshot", "direct", "fused"):
+                b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, batch * 8192, 0, iters=50, layers=80)
+
+
+if __name__ == "__main__":
+    main()

@@ -22,8 +22,8 @@ PL_MAX_WAITS = 16
 PL_OK, PL_ERR_INVALID_ARG, PL_ERR_UNSUPPORTED, PL_ERR_ALIGNMENT, PL_ERR_OOM, PL_ERR_CUDA, \
     PL_ERR_TIMEOUT, PL_ERR_OVERSUBSCRIBED, PL_ERR_INVALID_SCHEDULE, PL_ERR_OVERFLOW = range(10)
 # dtypes
-PL_BF16, PL_F32, PL_I32, PL_U8 = range(4)
-DTYPE_SIZE = {PL_BF16: 2, PL_F32: 4, PL_I32: 4, PL_U8: 1}
+PL_BF16, PL_F32, PL_I32, PL_U8, PL_F32X2 = range(5)
+DTYPE_SIZE = {PL_BF16: 2, PL_F32: 4, PL_I32: 4, PL_U8: 1, PL_F32X2: 8}
 # collectives
 PL_ALLREDUCE, PL_REDUCE_SCATTER, PL_ALLGATHER, PL_ALLTOALL, PL_ALLTOALLV = range(5)
 # algorithms

@@ -71,7 +71,7 @@ void fill_info(pl_schedule_s* S, int R) {
   }
   I.grid = S->pol.n_ctas;
   I.threads = S->pol.threads;
-  I.smem_bytes = 0;
+  I.smem_bytes = S->pol.datapath == PL_DP_TMA ? (int32_t)exec_tma_smem_bytes(S->pol.stages, S->pol.stage_bytes) : 0;
   I.datapath = S->pol.datapath;
   I.stages = S->pol.stages;
   I.stage_bytes = S->pol.stage_bytes;
@@ -108,13 +108,13 @@ void flatten(pl_schedule_s* S, int dtype) {
     d.n_wait = (uint32_t)op.waits.size();
     d.signal = op.signal >= 0 ? (uint32_t)op.signal : kNoFlag;
     d.signal2 = op.signal2 >= 0 ? (uint32_t)op.signal2 : kNoFlag;
-    d.flags = (op.bcast ? kDstBcast : 0u) | ((dtype == PL_BF16 && op.dst.dtype == PL_F32) ? kDstF32 : 0u);
+    d.flags = (op.bcast ? kDstBcast : 0u) | ((op.kind != PL_OP_COPY && op.dst.dtype != dtype) ? kDstF32 : 0u);
     d.count = op.count;
     d.dst = pack(*S, op.dst);
     d.topo = (uint32_t)op.topo;
     for (size_t k = 0; k < op.src.size(); ++k) {
       S->srcs[pos * max_src + k] = pack(*S, op.src[k]);
-      if (dtype == PL_BF16 && op.src[k].dtype == PL_F32) d.src_f32_mask |= 1u << k;
+      if (op.kind != PL_OP_COPY && op.src[k].dtype != dtype) d.src_f32_mask |= 1u << k;
     }
     for (size_t k = 0; k < op.waits.size(); ++k)
       S->waits[pos * max_wait + k] = DevWait{(uint32_t)op.waits[k], L.flag_need[op.waits[k]]};
@@ -180,14 +180,23 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   rq.R = comm->R;
   rq.dtype = comm->dtype;
   rq.pol = pol;
-  const int threads = pol.threads > 0 ? pol.threads : 512;
-  int capacity = 148;
+  const int requested = pol.n_ctas;
+  pol = default_policy(rq, 0);  // datapath, threads, ring geometry
+  rq.pol = pol;
+  rq.pol.n_ctas = requested;
+  if (pol.datapath == PL_DP_TMA) {
+    if (pol.stages < 2 || pol.stages > 8 || pol.stage_bytes < 1024 || exec_tma_smem_bytes(pol.stages, pol.stage_bytes) > 227 * 1024)
+      return PL_ERR_INVALID_ARG;
+    pol.threads = exec_tma_threads();
+    rq.pol.threads = pol.threads;
+  }
+  int capacity = 148 * (pol.datapath == PL_DP_TMA ? 2 : 1);
   if (!comm->planner) {
-    int per_sm = exec_max_ctas_per_sm(comm->dtype, threads);
+    int per_sm = pol.datapath == PL_DP_TMA ? exec_tma_max_ctas_per_sm(comm->dtype, pol.stages, pol.stage_bytes)
+                                           : exec_max_ctas_per_sm(comm->dtype, pol.threads);
     if (per_sm <= 0) return PL_ERR_CUDA;
     capacity = per_sm * comm->sm_count;
   }
-  const int requested = pol.n_ctas;
   pol = default_policy(rq, capacity);
   if (requested > capacity) return PL_ERR_OVERSUBSCRIBED;
   if (pol.n_ctas > capacity) return PL_ERR_OVERSUBSCRIBED;
@@ -257,7 +266,7 @@ static pl_status_t comm_create(int R, pl_dtype_t dtype, bool planner, pl_comm_t*
   if (!out) return PL_ERR_INVALID_ARG;
   *out = nullptr;
   if (R < 2 || R > PL_MAX_RANKS) return PL_ERR_INVALID_ARG;
-  if (dtype < PL_BF16 || dtype > PL_U8) return PL_ERR_INVALID_ARG;
+  if (dtype < PL_BF16 || dtype > PL_U8) return PL_ERR_INVALID_ARG;  // PL_F32X2 is internal
   pl_comm_s* c = new (std::nothrow) pl_comm_s();
   if (!c) return PL_ERR_OOM;
   c->R = R;
@@ -476,8 +485,12 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   P.status = s->comm->d_status;
   P.timeout_ns = s->timeout_ns;
   P.n_ranks = R;
-  if (launch_exec(s->comm->dtype, P, s->pol.n_ctas, s->pol.threads, static_cast<cudaStream_t>(stream)) != cudaSuccess)
-    return PL_ERR_CUDA;
+  P.stages = s->pol.stages;
+  P.stage_bytes = s->pol.stage_bytes;
+  cudaError_t le = s->pol.datapath == PL_DP_TMA
+                       ? launch_exec_tma(s->comm->dtype, P, s->pol.n_ctas, static_cast<cudaStream_t>(stream))
+                       : launch_exec(s->comm->dtype, P, s->pol.n_ctas, s->pol.threads, static_cast<cudaStream_t>(stream));
+  if (le != cudaSuccess) return PL_ERR_CUDA;
   g_launches.fetch_add(1);
   return PL_OK;
 }

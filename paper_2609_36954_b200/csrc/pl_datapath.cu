@@ -10,130 +10,16 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "pl_device.cuh"
 #include "pl_internal.h"
 #include "pl_kernels.h"
 
 namespace pl {
 namespace {
 
+using namespace dev;
+
 constexpr int kMaxThreads = 512;
-
-// ---- small PTX helpers ---------------------------------------------------------------
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
-  unsigned long long v;
-  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
-  asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ int ld_volatile_s32(const int* p) {
-  int v;
-  asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ uint4 ld16(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
-__device__ __forceinline__ void st16(void* p, const uint4& v) {
-  asm volatile("st.global.cg.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
-__device__ __forceinline__ char* resolve(const ExecParams& P, uint64_t packed) {
-  return static_cast<char*>(P.base[packed >> 48]) + (packed & 0xFFFFFFFFFFFFull);
-}
-
-// ---- element arithmetic ----------------------------------------------------------------
-// A "unit" is the group of elements one 16-byte vector of the narrowest operand holds:
-// 8 elements for bf16 schedules, 4 for fp32 / int32.
-template <int DT>
-struct Acc;
-
-template <>
-struct Acc<PL_BF16> {
-  static constexpr int kElems = 8;
-  float v[8];
-  __device__ __forceinline__ void zero() {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = 0.f;
-  }
-  __device__ __forceinline__ void add_bf16(const uint4& q) {
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      v[2 * i] += __uint_as_float(w[i] << 16);
-      v[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
-    }
-  }
-  __device__ __forceinline__ void add_f32(const uint4& lo, const uint4& hi) {
-    v[0] += __uint_as_float(lo.x); v[1] += __uint_as_float(lo.y);
-    v[2] += __uint_as_float(lo.z); v[3] += __uint_as_float(lo.w);
-    v[4] += __uint_as_float(hi.x); v[5] += __uint_as_float(hi.y);
-    v[6] += __uint_as_float(hi.z); v[7] += __uint_as_float(hi.w);
-  }
-  __device__ __forceinline__ uint4 to_bf16() const {
-    uint4 q;
-    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
-    __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
-    __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]);
-    __nv_bfloat162 d = __floats2bfloat162_rn(v[6], v[7]);
-    q.x = *reinterpret_cast<uint32_t*>(&a);
-    q.y = *reinterpret_cast<uint32_t*>(&b);
-    q.z = *reinterpret_cast<uint32_t*>(&c);
-    q.w = *reinterpret_cast<uint32_t*>(&d);
-    return q;
-  }
-};
-
-// fp32 data: compensated (Kahan-Neumaier style two-sum) accumulation, still one
-// accumulator per element and ascending source order; the correction is folded in once at
-// the end.  Keeps the result inside the fp32 tolerance for any input mantissas.
-template <>
-struct Acc<PL_F32> {
-  static constexpr int kElems = 4;
-  float v[4], c[4];
-  __device__ __forceinline__ void zero() {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) v[i] = c[i] = 0.f;
-  }
-  __device__ __forceinline__ void add(const uint4& q) {
-    const float x[4] = {__uint_as_float(q.x), __uint_as_float(q.y), __uint_as_float(q.z), __uint_as_float(q.w)};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float s = __fadd_rn(v[i], x[i]);
-      float bp = __fsub_rn(s, v[i]);
-      float err = __fadd_rn(__fsub_rn(v[i], __fsub_rn(s, bp)), __fsub_rn(x[i], bp));
-      c[i] = __fadd_rn(c[i], err);
-      v[i] = s;
-    }
-  }
-  __device__ __forceinline__ uint4 result() const {
-    uint4 q;
-    q.x = __float_as_uint(__fadd_rn(v[0], c[0]));
-    q.y = __float_as_uint(__fadd_rn(v[1], c[1]));
-    q.z = __float_as_uint(__fadd_rn(v[2], c[2]));
-    q.w = __float_as_uint(__fadd_rn(v[3], c[3]));
-    return q;
-  }
-};
-
-template <>
-struct Acc<PL_I32> {
-  static constexpr int kElems = 4;
-  uint32_t v[4];
-  __device__ __forceinline__ void zero() { v[0] = v[1] = v[2] = v[3] = 0u; }
-  __device__ __forceinline__ void add(const uint4& q) {
-    v[0] += q.x; v[1] += q.y; v[2] += q.z; v[3] += q.w;
-  }
-  __device__ __forceinline__ uint4 result() const { return make_uint4(v[0], v[1], v[2], v[3]); }
-};
 
 // ---- op bodies (register path: unrolled 128-bit loads, then stores) -----------------------
 __device__ __forceinline__ void body_copy(char* dst, const char* src, uint64_t bytes, int tid, int nthr) {
@@ -222,7 +108,7 @@ __device__ __forceinline__ void body_copy_reduce(const ExecParams& P, const DevO
   char* dst = resolve(P, op.dst);
   const char* a = s_src[0];
   const char* b = s_src[1];
-  if constexpr (DT != PL_BF16) {
+  if constexpr (DT == PL_I32) {
     constexpr int U = 4;
     for (uint64_t base = tid; base < n_units; base += (uint64_t)U * nthr) {
       uint4 qa[U], qb[U];
@@ -240,6 +126,39 @@ __device__ __forceinline__ void body_copy_reduce(const ExecParams& P, const DevO
           acc.add(qa[u]);
           acc.add(qb[u]);
           st16(dst + (i << 4), acc.result());
+        }
+      }
+    }
+  } else if constexpr (DT == PL_F32) {
+    // operands are fp32 vectors (16 B per unit) or (sum, correction) pairs (32 B per unit)
+    const bool ap = op.src_f32_mask & 1u, bp = op.src_f32_mask & 2u, dp = op.flags & kDstF32;
+    constexpr int U = 2;
+    for (uint64_t base = tid; base < n_units; base += (uint64_t)U * nthr) {
+      uint4 qa[U][2], qb[U][2];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint64_t i = base + (uint64_t)u * nthr;
+        if (i < n_units) {
+          if (ap) { qa[u][0] = ld16(a + (i << 5)); qa[u][1] = ld16(a + (i << 5) + 16); }
+          else qa[u][0] = ld16(a + (i << 4));
+          if (bp) { qb[u][0] = ld16(b + (i << 5)); qb[u][1] = ld16(b + (i << 5) + 16); }
+          else qb[u][0] = ld16(b + (i << 4));
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint64_t i = base + (uint64_t)u * nthr;
+        if (i < n_units) {
+          Acc<PL_F32> acc;
+          acc.zero();
+          if (ap) acc.add_pair(qa[u][0], qa[u][1]); else acc.add(qa[u][0]);
+          if (bp) acc.add_pair(qb[u][0], qb[u][1]); else acc.add(qb[u][0]);
+          if (dp) {
+            st16(dst + (i << 5), acc.sums());
+            st16(dst + (i << 5) + 16, acc.corrections());
+          } else {
+            st16(dst + (i << 4), acc.result());
+          }
         }
       }
     }
@@ -286,20 +205,6 @@ struct OpSlot {
   const char* src[PL_MAX_SRC];
   DevWait wait[PL_MAX_WAITS];
 };
-
-// Record a timeout (first writer wins) and raise the abort word.
-__device__ __noinline__ void record_timeout(const ExecParams& P, int queue, uint32_t topo, uint32_t flag,
-                                            unsigned long long expected, unsigned long long observed) {
-  if (atomicCAS(P.status, 0, (int)PL_ERR_TIMEOUT) == 0) {
-    P.status[1] = queue;
-    P.status[2] = (int)topo;
-    P.status[3] = (int)flag;
-    *reinterpret_cast<unsigned long long*>(P.status + 4) = expected;
-    *reinterpret_cast<unsigned long long*>(P.status + 6) = observed;
-  }
-  __threadfence();
-  atomicExch(P.status + 8, 1);
-}
 
 template <int DT>
 __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_constant__ ExecParams P) {

@@ -1,0 +1,421 @@
+// Throughput datapath: the op-queue executor built around bulk asynchronous copies (TMA).
+//
+// One CTA per op queue, warp specialised:
+//   warp 0  producer  walks the queue, waits on the op's flags (acquire, bounded), cuts the
+//                     op into stages and fills a ring of shared-memory slots with
+//                     cp.async.bulk loads (one per source), running ahead of the consumers
+//                     across op boundaries (Algorithm 2 of the paper: prime / steady / drain,
+//                     here as a free-running ring with full / empty mbarriers);
+//   warp 1  copier    for COPY stages: one bulk store shared -> global per stage, no
+//                     registers touched by the payload;
+//   warps 2..9 consumers  for REDUCE / COPY_REDUCE stages: read the source tiles from
+//                     shared memory 16 bytes at a time, accumulate in fp32 in ascending
+//                     source order, store the result with 128-bit global stores.
+// A stage descriptor travels with every slot.  The last stage of an op carries its signal:
+// the warps that wrote report on an mbarrier, then one thread fences and does the release
+// increment.  Every wait (flag, full, empty, done) is bounded; on expiry the CTA records a
+// status, raises the abort word and leaves after draining its own copies.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "pl_device.cuh"
+#include "pl_internal.h"
+#include "pl_kernels.h"
+#include "pl_ptx.cuh"
+
+namespace pl {
+namespace {
+
+using namespace dev;
+
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = 32 * kConsumerWarps;
+constexpr int kThreads = 32 * (2 + kConsumerWarps);
+constexpr int kMaxStages = 8;
+constexpr uint32_t kEnd = 0xFFFFFFFFu;
+constexpr uint32_t kLastOfOp = 0x100u;  // stage flag (above the DevOp flag bits)
+constexpr int kCtrlBytes = 1024;        // barriers + stage descriptors ahead of the slots
+
+struct StageDesc {
+  uint32_t kind;   // pl_op_kind_t or kEnd
+  uint32_t n_src;
+  uint32_t units;  // 16-byte units of the element type in this stage (COPY: bytes / 16)
+  uint32_t ucap;   // unit capacity of a slot for this op (tile k starts at a multiple of it)
+  uint32_t pmask;  // sources that hold partials (twice as wide)
+  uint32_t flags;  // kDstF32 | kDstBcast | kLastOfOp
+  uint32_t signal, signal2;
+  char* dst;       // destination of this stage
+  uint64_t dst_off;  // byte offset inside every rank's output (broadcast destinations)
+};
+static_assert(sizeof(StageDesc) == 48, "StageDesc layout");
+
+struct Ctrl {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t done;  // consumer warps that finished writing the last stage of an op
+  int abort;
+  int pad;
+  StageDesc desc[kMaxStages];
+};
+static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
+
+// Bounded mbarrier wait.  Returns false when the CTA is aborting or the time limit passed.
+__device__ __forceinline__ bool wait_bar(const ExecParams& P, Ctrl* c, uint64_t* bar, uint32_t parity) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  for (uint32_t spins = 1;; ++spins) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((spins & 255u) == 0) {
+      if (*reinterpret_cast<volatile int*>(&c->abort)) return false;
+      if (globaltimer_ns() - t0 > P.timeout_ns) {
+        record_timeout(P, blockIdx.x, 0xFFFFFFFFu, 0xFFFFFFFFu, parity, 0);
+        *reinterpret_cast<volatile int*>(&c->abort) = 1;
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ uint4 lds16(const unsigned char* p) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(ptx::smem_u32(p)));
+  return v;
+}
+
+// Consumer work for one stage of a REDUCE / COPY_REDUCE op.
+template <int DT>
+__device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDesc& d, const unsigned char* slot, int ctid) {
+  const uint32_t units = d.units, ns = d.n_src, pmask = d.pmask;
+  const uint32_t tile = d.ucap * 16u;  // bytes of an element-typed tile; partial tiles are twice that
+  const bool dpart = d.flags & kDstF32, bcast = d.flags & kDstBcast;
+  for (uint32_t u = ctid; u < units; u += kConsumerThreads) {
+    Acc<DT> acc;
+    acc.zero();
+    if (pmask == 0) {
+      // all sources element-typed: loads of four sources at a time, then the adds (ascending)
+      const unsigned char* p = slot + (size_t)u * 16u;
+      uint32_t s = 0;
+      for (; s + 4 <= ns; s += 4) {
+        uint4 q0 = lds16(p), q1 = lds16(p + tile), q2 = lds16(p + 2 * tile), q3 = lds16(p + 3 * tile);
+        p += 4 * (size_t)tile;
+        if constexpr (DT == PL_BF16) { acc.add_bf16(q0); acc.add_bf16(q1); acc.add_bf16(q2); acc.add_bf16(q3); }
+        else { acc.add(q0); acc.add(q1); acc.add(q2); acc.add(q3); }
+      }
+      for (; s < ns; ++s) {
+        uint4 q = lds16(p);
+        p += tile;
+        if constexpr (DT == PL_BF16) acc.add_bf16(q);
+        else acc.add(q);
+      }
+    } else {
+      const unsigned char* base = slot;
+      for (uint32_t s = 0; s < ns; ++s) {
+        const bool part = (pmask >> s) & 1u;
+        if constexpr (DT == PL_I32) {
+          acc.add(lds16(base + (size_t)u * 16u));
+          base += tile;
+        } else if (part) {
+          const uint4 lo = lds16(base + (size_t)u * 32u), hi = lds16(base + (size_t)u * 32u + 16u);
+          if constexpr (DT == PL_BF16) acc.add_f32(lo, hi);
+          else acc.add_pair(lo, hi);
+          base += 2 * (size_t)tile;
+        } else {
+          const uint4 q = lds16(base + (size_t)u * 16u);
+          if constexpr (DT == PL_BF16) acc.add_bf16(q);
+          else acc.add(q);
+          base += tile;
+        }
+      }
+    }
+    if (dpart) {
+      if constexpr (DT == PL_BF16) {
+        st16(d.dst + (size_t)u * 32u, make_uint4(__float_as_uint(acc.v[0]), __float_as_uint(acc.v[1]),
+                                                  __float_as_uint(acc.v[2]), __float_as_uint(acc.v[3])));
+        st16(d.dst + (size_t)u * 32u + 16u, make_uint4(__float_as_uint(acc.v[4]), __float_as_uint(acc.v[5]),
+                                                        __float_as_uint(acc.v[6]), __float_as_uint(acc.v[7])));
+      } else if constexpr (DT == PL_F32) {
+        st16(d.dst + (size_t)u * 32u, acc.sums());
+        st16(d.dst + (size_t)u * 32u + 16u, acc.corrections());
+      }
+    } else {
+      uint4 r;
+      if constexpr (DT == PL_BF16) r = acc.to_bf16();
+      else r = acc.result();
+      if (!bcast) {
+        st16(d.dst + (size_t)u * 16u, r);
+      } else {
+        for (int k = 0; k < P.n_ranks; ++k)
+          st16(static_cast<char*>(P.base[kSlotOut + k]) + d.dst_off + (size_t)u * 16u, r);
+      }
+    }
+  }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_constant__ ExecParams P) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  Ctrl* c = reinterpret_cast<Ctrl*>(smem);
+  unsigned char* slots = smem + kCtrlBytes;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, q = blockIdx.x;
+  const uint32_t S = (uint32_t)P.stages, slot_bytes = P.stage_bytes;
+  const unsigned long long epoch = *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull;
+
+  if (tid == 0) {
+    for (uint32_t s = 0; s < S; ++s) {
+      ptx::mbar_init(&c->full[s], 1);
+      ptx::mbar_init(&c->empty[s], 1 + kConsumerWarps);  // copier + every consumer warp
+    }
+    ptx::mbar_init(&c->done, kConsumerWarps);
+    c->abort = 0;
+    ptx::mbar_init_fence();
+  }
+  __syncthreads();
+
+  if (warp == 0) {
+    // ================================ producer =========================================
+    const uint32_t qb = P.queue_begin[q], qe = P.queue_begin[q + 1];
+    uint32_t n = 0;  // stages produced
+    bool ok = true;
+    uint4 r_op = make_uint4(0, 0, 0, 0), r_op_next = r_op;
+    uint64_t r_src = 0, r_src_next = 0;
+    DevWait r_wait = {0, 0}, r_wait_next = {0, 0};
+    auto fetch = [&](uint32_t i, uint4& o, uint64_t& sr, DevWait& w) {
+      if (lane < 4) o = reinterpret_cast<const uint4*>(P.ops + i)[lane];
+      if (lane < (int)P.src_stride) sr = P.srcs[(uint64_t)i * P.src_stride + lane];
+      if (lane < (int)P.wait_stride) w = P.waits[(uint64_t)i * P.wait_stride + lane];
+    };
+    if (qb < qe) fetch(qb, r_op_next, r_src_next, r_wait_next);
+    for (uint32_t i = qb; i < qe && ok; ++i) {
+      r_op = r_op_next;
+      r_src = r_src_next;
+      r_wait = r_wait_next;
+      if (i + 1 < qe) fetch(i + 1, r_op_next, r_src_next, r_wait_next);
+      // op words: lane 0: kind n_src rsv pmask | lane 1: rsv n_wait signal flags | lane 2: count dst | lane 3: topo signal2
+      const uint32_t kind = __shfl_sync(0xFFFFFFFFu, r_op.x, 0), n_src = __shfl_sync(0xFFFFFFFFu, r_op.y, 0);
+      const uint32_t pmask = __shfl_sync(0xFFFFFFFFu, r_op.w, 0);
+      const uint32_t n_wait = __shfl_sync(0xFFFFFFFFu, r_op.y, 1), signal = __shfl_sync(0xFFFFFFFFu, r_op.z, 1);
+      const uint32_t oflags = __shfl_sync(0xFFFFFFFFu, r_op.w, 1);
+      const uint64_t count = ((uint64_t)__shfl_sync(0xFFFFFFFFu, r_op.y, 2) << 32) | __shfl_sync(0xFFFFFFFFu, r_op.x, 2);
+      const uint64_t dstp = ((uint64_t)__shfl_sync(0xFFFFFFFFu, r_op.w, 2) << 32) | __shfl_sync(0xFFFFFFFFu, r_op.z, 2);
+      const uint32_t topo = __shfl_sync(0xFFFFFFFFu, r_op.x, 3), signal2 = __shfl_sync(0xFFFFFFFFu, r_op.y, 3);
+
+      // ---- wait (acquire) on the op's flags: lane k polls entry k
+      bool lane_ok = true;
+      if (lane < (int)n_wait) {
+        const unsigned long long need = epoch * (unsigned long long)r_wait.need;
+        const unsigned long long* fp = P.flags + r_wait.flag;
+        unsigned long long seen = ld_acquire_u64(fp);
+        if (seen < need) {
+          const unsigned long long t0 = globaltimer_ns();
+          uint32_t spins = 0;
+          while ((seen = ld_acquire_u64(fp)) < need) {
+            if ((++spins & 63u) == 0) {
+              if (ld_volatile_s32(P.status + 8) || *reinterpret_cast<volatile int*>(&c->abort)) { lane_ok = false; break; }
+              if (globaltimer_ns() - t0 > P.timeout_ns) {
+                record_timeout(P, q, topo, r_wait.flag, need, seen);
+                lane_ok = false;
+                break;
+              }
+            }
+          }
+        }
+      }
+      ok = __all_sync(0xFFFFFFFFu, lane_ok);
+      if (!ok) break;
+      if (n_wait) ptx::fence_proxy_async();  // data released by other CTAs' generic stores -> our bulk loads
+
+      // ---- cut the op into stages
+      const char* my_src = (lane < (int)n_src) ? resolve(P, r_src) : nullptr;
+      const bool my_part = (pmask >> lane) & 1u;
+      const uint32_t unit_b = (kind == PL_OP_COPY) ? 16u : 16u * (n_src + __popc(pmask));  // slot bytes per unit
+      const uint32_t ucap = slot_bytes / unit_b;
+      const uint64_t n_units = (kind == PL_OP_COPY) ? (count >> 4) : count / Acc<DT == PL_U8 ? PL_I32 : DT>::kElems;
+      // tile offset of my source inside a slot, and my bytes per unit
+      const uint32_t my_w = my_part ? 32u : 16u;
+      const uint32_t my_tile_off = ucap * 16u * (lane + __popc(pmask & ((1u << lane) - 1u)));
+      const uint32_t dst_w = (kind == PL_OP_COPY) ? 16u : ((oflags & kDstF32) ? 32u : 16u);
+      char* dst = resolve(P, dstp);
+      const uint64_t dst_off = dstp & 0xFFFFFFFFFFFFull;
+      for (uint64_t u0 = 0; u0 < n_units; u0 += ucap) {
+        const uint32_t units = (uint32_t)min((uint64_t)ucap, n_units - u0);
+        const uint32_t s = n % S, ph = (n / S) & 1u;
+        bool w_ok = true;
+        if (lane == 0) w_ok = wait_bar(P, c, &c->empty[s], ph ^ 1u);
+        ok = __shfl_sync(0xFFFFFFFFu, (int)w_ok, 0);
+        if (!ok) break;
+        if (lane == 0) {
+          StageDesc& d = c->desc[s];
+          d.kind = kind;
+          d.n_src = n_src;
+          d.units = units;
+          d.ucap = ucap;
+          d.pmask = pmask;
+          d.flags = oflags | ((u0 + ucap >= n_units) ? kLastOfOp : 0u);
+          d.signal = signal;
+          d.signal2 = signal2;
+          d.dst = dst + u0 * dst_w;
+          d.dst_off = dst_off + u0 * dst_w;
+          ptx::mbar_expect_tx(&c->full[s], units * unit_b);
+        }
+        __syncwarp();
+        if (lane < (int)n_src)
+          ptx::bulk_g2s(slots + (size_t)s * slot_bytes + my_tile_off, my_src + u0 * my_w, units * my_w, &c->full[s]);
+        ++n;
+      }
+    }
+    // ---- end of queue (or abort): tell the other warps, then make sure nothing is in flight
+    if (lane == 0) {
+      if (!ok) {
+        *reinterpret_cast<volatile int*>(&c->abort) = 1;
+        // loads already issued must land before the CTA may leave: bounded drain
+        for (uint32_t k = (n > S ? n - S : 0u); k < n; ++k)
+          for (uint32_t tries = 0; tries < (1u << 22) && !ptx::mbar_try_wait(&c->full[k % S], (k / S) & 1u); ++tries) {}
+      }
+      const uint32_t s = n % S, ph = (n / S) & 1u;
+      if (ok && wait_bar(P, c, &c->empty[s], ph ^ 1u)) {
+        c->desc[s].kind = kEnd;
+        ptx::mbar_arrive(&c->full[s]);
+      }
+    }
+  } else if (warp == 1) {
+    // ================================ copier ============================================
+    int prev = -1;  // slot whose bulk store may still be reading shared memory
+    for (uint32_t n = 0;; ++n) {
+      const uint32_t s = n % S, ph = (n / S) & 1u;
+      bool go = true;
+      if (lane == 0) go = wait_bar(P, c, &c->full[s], ph);
+      go = __shfl_sync(0xFFFFFFFFu, (int)go, 0);
+      __syncwarp();  // lane 0's acquire on the barrier covers the whole warp's reads below
+      if (!go) break;
+      const StageDesc& d = c->desc[s];
+      const uint32_t kind = d.kind;
+      if (kind == kEnd) break;
+      if (lane == 0) {
+        if (kind == PL_OP_COPY) {
+          ptx::bulk_s2g(d.dst, slots + (size_t)s * slot_bytes, d.units * 16u);
+          ptx::bulk_commit();
+          if (prev >= 0) {
+            ptx::bulk_wait_read<1>();
+            ptx::mbar_arrive(&c->empty[prev]);
+          }
+          prev = (int)s;
+          if ((d.flags & kLastOfOp) && d.signal != kNoFlag) {
+            ptx::bulk_wait<0>();        // the op's bytes have landed
+            ptx::fence_proxy_async();   // async-proxy writes before the generic-proxy release
+            __threadfence();
+            red_release_add_u64(P.flags + d.signal, 1ull);
+            if (d.signal2 != kNoFlag) red_release_add_u64(P.flags + d.signal2, 1ull);
+          }
+        } else {
+          if (prev >= 0) {
+            ptx::bulk_wait_read<0>();
+            ptx::mbar_arrive(&c->empty[prev]);
+            prev = -1;
+          }
+          ptx::mbar_arrive(&c->empty[s]);
+        }
+      }
+    }
+    if (lane == 0) {
+      ptx::bulk_wait<0>();
+      if (prev >= 0) ptx::mbar_arrive(&c->empty[prev]);
+    }
+  } else {
+    // ================================ consumers =========================================
+    const int ctid = tid - 64;
+    uint32_t n_done = 0;  // completed phases of the done barrier
+    for (uint32_t n = 0;; ++n) {
+      const uint32_t s = n % S, ph = (n / S) & 1u;
+      bool go = true;
+      if (lane == 0) go = wait_bar(P, c, &c->full[s], ph);
+      go = __shfl_sync(0xFFFFFFFFu, (int)go, 0);
+      __syncwarp();  // lane 0's acquire on the barrier covers the whole warp's reads below
+      if (!go) break;
+      const StageDesc& d = c->desc[s];
+      const uint32_t kind = d.kind;
+      if (kind == kEnd) break;
+      if (kind != PL_OP_COPY) {
+        if constexpr (DT != PL_U8) consume_stage<DT>(P, d, slots + (size_t)s * slot_bytes, ctid);
+        const bool last = d.flags & kLastOfOp;
+        const uint32_t signal = d.signal, signal2 = d.signal2;
+        __syncwarp();
+        if (last && signal != kNoFlag) {
+          // every consumer warp reports its stores; consumer thread 0 then publishes
+          if (lane == 0) ptx::mbar_arrive(&c->done);
+          if (ctid == 0) {
+            if (wait_bar(P, c, &c->done, n_done & 1u)) {
+              __threadfence();
+              red_release_add_u64(P.flags + signal, 1ull);
+              if (signal2 != kNoFlag) red_release_add_u64(P.flags + signal2, 1ull);
+            }
+          }
+          ++n_done;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&c->empty[s]);
+    }
+  }
+
+  __syncthreads();
+  if (tid == 0 && !*reinterpret_cast<volatile int*>(&c->abort)) {
+    const unsigned long long prev = atomicAdd(P.epoch + 1, 1ull);
+    if (prev == (unsigned long long)gridDim.x - 1ull) {
+      P.epoch[1] = 0ull;
+      __threadfence();
+      *reinterpret_cast<volatile unsigned long long*>(P.epoch) = epoch;
+    }
+  }
+}
+
+template <int DT>
+cudaError_t launch_t(const ExecParams& P, int grid, cudaStream_t stream) {
+  const size_t smem = exec_tma_smem_bytes(P.stages, P.stage_bytes);
+  static bool configured = false;  // per instantiation
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(pl_exec_tma_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  pl_exec_tma_kernel<DT><<<grid, kThreads, smem, stream>>>(P);
+  return cudaGetLastError();
+}
+
+template <int DT>
+int occupancy_t(size_t smem) {
+  int n = 0;
+  if (cudaFuncSetAttribute(pl_exec_tma_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_tma_kernel<DT>, kThreads, smem) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return n;
+}
+
+}  // namespace
+
+size_t exec_tma_smem_bytes(int stages, uint32_t stage_bytes) { return kCtrlBytes + (size_t)stages * stage_bytes; }
+int exec_tma_threads() { return kThreads; }
+
+cudaError_t launch_exec_tma(int dtype, const ExecParams& P, int grid, cudaStream_t stream) {
+  if (P.stages < 2 || P.stages > kMaxStages) return cudaErrorInvalidValue;
+  switch (dtype) {
+    case PL_BF16: return launch_t<PL_BF16>(P, grid, stream);
+    case PL_F32: return launch_t<PL_F32>(P, grid, stream);
+    case PL_I32: return launch_t<PL_I32>(P, grid, stream);
+    default: return launch_t<PL_U8>(P, grid, stream);
+  }
+}
+
+int exec_tma_max_ctas_per_sm(int dtype, int stages, uint32_t stage_bytes) {
+  const size_t smem = exec_tma_smem_bytes(stages, stage_bytes);
+  if (smem > 227 * 1024) return 0;
+  switch (dtype) {
+    case PL_BF16: return occupancy_t<PL_BF16>(smem);
+    case PL_F32: return occupancy_t<PL_F32>(smem);
+    case PL_I32: return occupancy_t<PL_I32>(smem);
+    default: return occupancy_t<PL_U8>(smem);
+  }
+}
+
+}  // namespace pl

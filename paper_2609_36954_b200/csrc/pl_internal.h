@@ -14,11 +14,14 @@ inline int elem_size(int dtype) {
     case PL_BF16: return 2;
     case PL_F32: return 4;
     case PL_I32: return 4;
+    case PL_F32X2: return 8;
     default: return 1;
   }
 }
 // Element type of partial sums that travel between ops (ring hops, tree levels).
-inline int partial_dtype(int dtype) { return dtype == PL_BF16 ? PL_F32 : dtype; }
+// bf16 data: fp32.  fp32 data: a compensated (sum, correction) fp32 pair, so that rounding once
+// per hop does not eat the fp32 tolerance.  int32: int32.
+inline int partial_dtype(int dtype) { return dtype == PL_BF16 ? PL_F32 : dtype == PL_F32 ? PL_F32X2 : dtype; }
 
 struct HostOp {
   int kind = PL_OP_COPY;
@@ -46,11 +49,11 @@ struct alignas(16) DevOp {
   uint32_t kind;        // pl_op_kind_t
   uint32_t n_src;
   uint32_t rsv0;
-  uint32_t src_f32_mask;  // bit p set: source p holds fp32 partials (bf16 schedules only)
+  uint32_t src_f32_mask;  // bit p set: source p holds partials (fp32 for bf16 data, fp32 pairs for fp32 data)
   uint32_t rsv1;
   uint32_t n_wait;
   uint32_t signal;      // flag index or kNoFlag
-  uint32_t flags;       // bit0: dst holds fp32 partials (bf16 schedules); bit1: dst broadcast
+  uint32_t flags;       // bit0: dst holds partials; bit1: dst broadcast
   uint64_t count;       // elements (bytes for COPY)
   uint64_t dst;         // packed address
   uint32_t topo;
@@ -77,6 +80,8 @@ struct ExecParams {
   int* status;                  // pl_devstatus_t words + abort word (comm-owned)
   unsigned long long timeout_ns;
   int n_ranks;
+  int stages;            // shared-memory ring depth of the TMA executor
+  uint32_t stage_bytes;  // bytes per ring slot
 };
 
 struct Policy {

@@ -7,8 +7,15 @@
 
 namespace pl {
 
+// register (ld/st) executor
 cudaError_t launch_exec(int dtype, const ExecParams& P, int grid, int threads, cudaStream_t stream);
 int exec_max_ctas_per_sm(int dtype, int threads);
 int exec_max_threads();
+
+// TMA (bulk-copy, shared-memory ring) executor
+cudaError_t launch_exec_tma(int dtype, const ExecParams& P, int grid, cudaStream_t stream);
+int exec_tma_max_ctas_per_sm(int dtype, int stages, uint32_t stage_bytes);
+int exec_tma_threads();
+size_t exec_tma_smem_bytes(int stages, uint32_t stage_bytes);
 
 }  // namespace pl

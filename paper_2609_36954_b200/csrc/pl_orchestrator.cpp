@@ -28,6 +28,7 @@ pl_ref_t ref(int rank, int buf, int dtype, uint64_t off) {
 struct Emitter {
   Lowered* L;
   uint32_t slice_bytes;
+  int dtype = PL_U8;  // the schedule's element type
   int queues_per_rank = 1;
   // Chunks each rank runs in the phase being emitted (0 = unknown).  When known, the slice
   // count is nudged upwards so that a rank's work items divide evenly over its queues.
@@ -42,12 +43,11 @@ struct Emitter {
   void chunk_op(int kind, int exec_rank, int layer, pl_ref_t dst, bool bcast,
                 const std::vector<pl_ref_t>& src, uint64_t count, const std::vector<int>& waits,
                 int signal, int signal2 = -1) {
-    int min_es = elem_size(dst.dtype), max_es = min_es;
-    for (const pl_ref_t& s : src) {
-      min_es = std::min(min_es, elem_size(s.dtype));
-      max_es = std::max(max_es, elem_size(s.dtype));
-    }
-    const uint64_t unit16 = 16 / min_es;  // elements that keep every operand 16-byte aligned
+    int max_es = elem_size(dst.dtype);
+    for (const pl_ref_t& s : src) max_es = std::max(max_es, elem_size(s.dtype));
+    // elements per 16-byte vector of the schedule's element type: the kernel's unit of work,
+    // which also keeps every (wider) partial operand aligned
+    const uint64_t unit16 = kind == PL_OP_COPY ? 16 : 16 / elem_size(dtype);
     uint64_t wide = count * max_es;
     uint64_t n_slices = 1;
     if (slice_bytes && wide > slice_bytes + slice_bytes / 2) n_slices = (wide + slice_bytes - 1) / slice_bytes;
@@ -59,7 +59,7 @@ struct Emitter {
         }
     }
     uint64_t per = (count + n_slices - 1) / n_slices;
-    uint64_t unit = (per >= 8 * (128 / min_es)) ? uint64_t(128 / min_es) : unit16;
+    uint64_t unit = (per >= 64 * unit16) ? 8 * unit16 : unit16;
     per = (per + unit - 1) / unit * unit;
     for (uint64_t b = 0; b < count; b += per) {
       HostOp op;
@@ -384,6 +384,9 @@ void ar_tree(Emitter& em, const Geo& g) {
 
 }  // namespace
 
+// Default knobs for sm_100a ("codesign policy", Sec. 3.2-3.3).  Called twice by the build:
+// first with max_resident_ctas == 0 to settle the datapath and its shared-memory ring (which
+// decide how many CTAs fit on an SM), then with the resulting capacity to settle the grid.
 Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
   Policy p = rq.pol;
   const int es = elem_size(rq.dtype);
@@ -394,14 +397,14 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
     msg /= rq.R;
   }
   if (rq.coll == PL_ALLGATHER) msg *= rq.R;
+  // latency regime (register path, small slices) below 1 MiB per rank, layered schedules too
+  const bool small = msg <= (1u << 20) || rq.n_layers > 0;
+  if (p.datapath == PL_DP_AUTO) p.datapath = small ? PL_DP_LDST : PL_DP_TMA;
   if (p.threads <= 0) p.threads = 512;
-  if (p.datapath == PL_DP_AUTO) p.datapath = PL_DP_LDST;
-  if (p.stages <= 0) p.stages = 4;
-  if (p.stage_bytes == 0) p.stage_bytes = 16384;
-  if (p.slice_bytes == 0) {
-    // latency regime: few, small slices; throughput regime: 64 KiB slices
-    p.slice_bytes = msg <= (1u << 20) ? 16384 : 65536;
-  }
+  if (p.stages <= 0) p.stages = 3;
+  if (p.stage_bytes == 0) p.stage_bytes = 32768;
+  if (p.slice_bytes == 0) p.slice_bytes = small ? 16384 : (p.datapath == PL_DP_TMA ? 262144 : 65536);
+  if (max_resident_ctas <= 0) return p;
   if (p.n_ctas <= 0) {
     const int full = std::max(rq.R, max_resident_ctas / rq.R * rq.R);
     // work items per rank under this slicing (output bytes a rank produces / slice)
@@ -426,6 +429,7 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
   const bool reduces = rq.coll == PL_ALLREDUCE || rq.coll == PL_REDUCE_SCATTER;
   if (reduces && dt == PL_U8) return fail(PL_ERR_UNSUPPORTED, "bytes cannot be reduced");
   Emitter em{L, rq.pol.slice_bytes};
+  em.dtype = dt;
   em.queues_per_rank = std::max(1, rq.pol.n_ctas / R);
   L->n_layers = 1;
 

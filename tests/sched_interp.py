@@ -14,7 +14,7 @@ import numpy as np
 from paper_2609_36954_b200 import binding as B
 from paper_2609_36954_b200 import inputs as gen
 
-_ES = {B.PL_BF16: 2, B.PL_F32: 4, B.PL_I32: 4, B.PL_U8: 1}
+_ES = {B.PL_BF16: 2, B.PL_F32: 4, B.PL_I32: 4, B.PL_U8: 1, B.PL_F32X2: 8}
 
 
 def _load(buf, off, count, dtype):
@@ -25,6 +25,9 @@ def _load(buf, off, count, dtype):
         return raw.view(np.float32).copy()
     if dtype == B.PL_I32:
         return raw.view(np.uint32).copy()
+    if dtype == B.PL_F32X2:  # blocks of 4 sums then 4 corrections; value = sum + correction
+        blk = raw.view(np.float32).reshape(-1, 2, 4).astype(np.float64)
+        return (blk[:, 0, :] + blk[:, 1, :]).reshape(-1)
     return raw.copy()
 
 
@@ -35,6 +38,11 @@ def _store(buf, off, vals, dtype):
         raw = vals.astype(np.float32).view(np.uint8)
     elif dtype == B.PL_I32:
         raw = vals.astype(np.uint32).view(np.uint8)
+    elif dtype == B.PL_F32X2:
+        v = vals.astype(np.float64).reshape(-1, 4)
+        hi = v.astype(np.float32)
+        lo = (v - hi.astype(np.float64)).astype(np.float32)
+        raw = np.stack([hi, lo], axis=1).reshape(-1).view(np.uint8)
     else:
         raw = vals
     buf[off:off + raw.size] = raw
@@ -74,8 +82,11 @@ def run(ops, info, R, ins, seed=0, max_steps=None):
             result, rdt = data, B.PL_U8
         else:
             first = op.src[0]
+            kinds = {op.src[k].dtype for k in range(op.n_src)} | {op.dst.dtype}
             if first.dtype == B.PL_I32:
                 acc = np.zeros(n, np.uint32)
+            elif B.PL_F32X2 in kinds:
+                acc = np.zeros(n, np.float64)  # stands in for the compensated fp32 pair
             else:
                 acc = np.zeros(n, np.float32)
             for k in range(op.n_src):

@@ -51,35 +51,28 @@ def test_config1_allreduce_ring(dtype):
 
 
 # ---- every all-reduce algorithm, ragged sizes, several R, every dtype ---------------------
+DATAPATHS = [B.PL_DP_LDST, B.PL_DP_TMA]
+
+
+@pytest.mark.parametrize("dp", DATAPATHS)
 @pytest.mark.parametrize("algo", ALL_AR)
 @pytest.mark.parametrize("dtype", ["bf16", "f32", "i32"])
 @pytest.mark.parametrize("R", [2, 3, 8])
-def test_allreduce_all_algorithms(algo, dtype, R):
+def test_allreduce_all_algorithms(algo, dtype, R, dp):
     es = B.DTYPE_SIZE[{"bf16": B.PL_BF16, "f32": B.PL_F32, "i32": B.PL_I32}[dtype]]
     # partition = 37 KiB + 16 B: not a multiple of the chunk, the slice or the CTA width
     n = R * ((37 * 1024 + 16) // es)
-    # Single-op reductions (direct, one-shot, fused) use a compensated fp32 accumulator and
-    # meet the fp32 tolerance for any mantissas, so they get full-mantissa N(0,1) data.  Ring
-    # and tree round the travelling fp32 partial once per hop: they get the configuration's
-    # own data (uniform on the 2^-23 grid) under the strict tolerance, and N(0,1) data under
-    # the textbook bound of recursive summation, (R-1) * 2^-24 * sum_p |x_p|.
-    multi_hop = algo in (B.PL_ALGO_RING, B.PL_ALGO_TREE)
-    x = gen.rank_inputs(R, n, "f32n" if (dtype == "f32" and not multi_hop) else dtype, seed=11)
+    # fp32 data gets full-mantissa N(0,1) values: single-op reductions use a compensated fp32
+    # accumulator and multi-hop ones (ring, tree) carry (sum, correction) pairs, so the fp32
+    # tolerance holds for any mantissas, not only for the configuration's 2^-23 grid.
+    x = gen.rank_inputs(R, n, "f32n" if dtype == "f32" else dtype, seed=11)
     ref = oracle.allreduce(x, dtype)
     ses = Session(R, dtype)
     try:
-        for chunk, sl in [(8192, 4096), (1 << 20, 16384)]:
-            s = ses.build(B.PL_ALLREDUCE, algo, n, chunk, slice_bytes=sl)
+        for chunk, sl, stage in [(8192, 4096, 2048), (1 << 20, 16384, 32768)]:
+            s = ses.build(B.PL_ALLREDUCE, algo, n, chunk, slice_bytes=sl, datapath=dp, stage_bytes=stage, stages=3)
             outs, _ = ses.execute(s, x, repeats=2)
             compare_reduce(outs, ref, dtype)
-        if dtype == "f32" and multi_hop:
-            xn = gen.rank_inputs(R, n, "f32n", seed=12)
-            refn = oracle.allreduce(xn, "f32")
-            bound = (R - 1) * 2.0 ** -24 * np.sum([np.abs(a.astype(np.float64)) for a in xn], axis=0)
-            outs, _ = ses.execute(s, xn)
-            for r in range(R):
-                err = np.abs(outs[r].view(np.float32).astype(np.float64) - refn[r])
-                assert np.all(err <= bound + 1e-12)
     finally:
         ses.close()
 
@@ -94,30 +87,32 @@ def test_allreduce_tiny_and_single_vector():
             ses = Session(R, dtype)
             try:
                 for algo in ALL_AR:
-                    s = ses.build(B.PL_ALLREDUCE, algo, n, 16)
-                    outs, _ = ses.execute(s, x)
-                    compare_reduce(outs, ref, dtype)
+                    for dp in DATAPATHS:
+                        s = ses.build(B.PL_ALLREDUCE, algo, n, 16, datapath=dp)
+                        outs, _ = ses.execute(s, x)
+                        compare_reduce(outs, ref, dtype)
             finally:
                 ses.close()
 
 
+@pytest.mark.parametrize("dp", DATAPATHS)
 @pytest.mark.parametrize("algo", [B.PL_ALGO_RING, B.PL_ALGO_DIRECT])
 @pytest.mark.parametrize("dtype", ["bf16", "i32", "f32"])
-def test_reduce_scatter_and_allgather(algo, dtype):
+def test_reduce_scatter_and_allgather(algo, dtype, dp):
     R = 8
     es = 2 if dtype == "bf16" else 4
     n = R * (300 * 1024 + 48) // es // 1  # partition 300 KiB + 48 B
     n -= n % (R * 16 // es)
-    x = gen.rank_inputs(R, n, dtype, seed=3)  # fp32: the 2^-23 grid of the fp32 configuration
+    x = gen.rank_inputs(R, n, "f32n" if dtype == "f32" else dtype, seed=3)
     ses = Session(R, dtype)
     try:
         for chunk in (256 * 1024, 1 << 20):
-            s = ses.build(B.PL_REDUCE_SCATTER, algo, n, chunk)
+            s = ses.build(B.PL_REDUCE_SCATTER, algo, n, chunk, datapath=dp)
             outs, _ = ses.execute(s, x, repeats=2)
             compare_reduce(outs, oracle.reduce_scatter(x, dtype), dtype)
             m = n // R
             contrib = [a[:m].copy() for a in x]
-            s = ses.build(B.PL_ALLGATHER, algo, m, chunk)
+            s = ses.build(B.PL_ALLGATHER, algo, m, chunk, datapath=dp)
             outs, _ = ses.execute(s, contrib, repeats=2)
             ref = oracle.allgather(contrib)
             for r in range(R):
@@ -126,13 +121,14 @@ def test_reduce_scatter_and_allgather(algo, dtype):
         ses.close()
 
 
-def test_alltoall_and_alltoallv_bit_exact():
+@pytest.mark.parametrize("dp", DATAPATHS)
+def test_alltoall_and_alltoallv_bit_exact(dp):
     R = 8
     ses = Session(R, "u8")
     try:
         m = 100 * 1024 + 16
         x = gen.rank_coded_bytes(R, R * m)
-        s = ses.build(B.PL_ALLTOALL, B.PL_ALGO_DIRECT, R * m, 65536)
+        s = ses.build(B.PL_ALLTOALL, B.PL_ALGO_DIRECT, R * m, 65536, datapath=dp)
         outs, _ = ses.execute(s, x)
         ref = oracle.alltoall(x)
         for r in range(R):
@@ -145,7 +141,7 @@ def test_alltoall_and_alltoallv_bit_exact():
                 C[2, :] = 0
                 C[:, 5] = 0
             xs = [gen.rank_coded_bytes(R, max(16, int(C[p].sum())))[p][: int(C[p].sum())] for p in range(R)]
-            s = ses.build_v(C.tolist(), 65536)
+            s = ses.build_v(C.tolist(), 65536, datapath=dp)
             outs, info = ses.execute(s, xs)
             ref = oracle.alltoallv(xs, C)
             for r in range(R):
@@ -194,13 +190,14 @@ def test_bf16_direct_sum_is_the_correctly_rounded_sum():
         ses.close()
 
 
-def test_run_to_run_determinism():
+@pytest.mark.parametrize("dp", DATAPATHS)
+def test_run_to_run_determinism(dp):
     R, n = 8, 8 * 40000
     x = gen.rank_inputs(R, n, "bf16", seed=4)
     ses = Session(R, "bf16")
     try:
         for algo in (B.PL_ALGO_RING, B.PL_ALGO_DIRECT):
-            s = ses.build(B.PL_ALLREDUCE, algo, n, 32768)
+            s = ses.build(B.PL_ALLREDUCE, algo, n, 32768, datapath=dp)
             a, _ = ses.execute(s, x)
             b, _ = ses.execute(s, x, repeats=3)
             for r in range(R):
@@ -259,7 +256,8 @@ def test_execute_argument_errors():
         ses.close()
 
 
-def test_bounded_wait_reports_timeout_and_recovers():
+@pytest.mark.parametrize("dp", DATAPATHS)
+def test_bounded_wait_reports_timeout_and_recovers(dp):
     # host-made failure: one wait edge is raised beyond what the schedule will ever signal;
     # with a 20 ms limit the kernel must return, report PL_ERR_TIMEOUT, and the GPU must stay
     # usable: after pl_comm_reset an intact schedule runs and matches the oracle.
@@ -268,7 +266,7 @@ def test_bounded_wait_reports_timeout_and_recovers():
     ref = oracle.allreduce(x, "i32")
     ses = Session(R, "i32")
     try:
-        bad = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 4096, timeout_ns=20_000_000)
+        bad = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 4096, timeout_ns=20_000_000, datapath=dp)
         ops = B.pl_schedule_dump(bad)
         victim = next(o.topo for o in ops if o.n_wait > 0)
         B.pl_schedule_debug_break_wait(bad, victim)
@@ -287,7 +285,7 @@ def test_bounded_wait_reports_timeout_and_recovers():
         B.pl_comm_reset(ses.comm, stream_handle())
         torch.cuda.synchronize()
         assert B.pl_comm_status(ses.comm).code == B.PL_OK
-        good = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 4096)
+        good = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 4096, datapath=dp)
         outs, _ = ses.execute(good, x)
         compare_reduce(outs, ref, "i32")
     finally:

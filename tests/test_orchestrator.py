@@ -177,14 +177,23 @@ def test_config1_op_counts_and_bytes():
     # 3 reduce-scatter hops + 3 all-gather hops, 4 ranks, 4 chunks per partition
     pl = Planner(4, "f32")
     try:
-        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, 262144, 65536, slice_bytes=65536)
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, 262144, 65536, slice_bytes=131072)
         info = B.pl_schedule_info(s)
         ops = B.pl_schedule_dump(s)
         assert sum(o.kind == B.PL_OP_COPY_REDUCE for o in ops) == 48
         assert sum(o.kind == B.PL_OP_COPY for o in ops) == 48
         M = 1 << 20
-        assert info.bytes_read + info.bytes_written == 5 * 3 * M  # 5(R-1)M
+        # fp32 partials travel as (sum, correction) pairs: per partition element the three
+        # reduce-scatter hops move 16 + 20 + 16 bytes, the all-gather hops 2 * 4 * 3
+        assert info.bytes_read + info.bytes_written == 13 * M + 6 * M
         assert info.message_bytes == M
+    finally:
+        pl.close()
+    pl = Planner(4, "i32")
+    try:
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, 262144, 65536, slice_bytes=65536)
+        info = B.pl_schedule_info(s)
+        assert info.bytes_read + info.bytes_written == 5 * 3 * (1 << 20)  # 5(R-1)M with same-width partials
     finally:
         pl.close()
 
