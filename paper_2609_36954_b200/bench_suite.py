@@ -62,6 +62,28 @@ def _time(fn, iters, warmup=3, per_call_events=False):
     return us, us, us
 
 
+def _time_graph(launch, calls=128, replays=8):
+    """The paper's microbenchmark method (Sec. 5): capture `calls` invocations in a CUDA graph,
+    replay once to warm up, time `replays` replays with CUDA events, divide by calls*replays.
+    `launch(stream_handle)` must enqueue exactly one invocation on the given stream."""
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(g, stream=side):
+        h = torch.cuda.current_stream().cuda_stream
+        for _ in range(calls):
+            launch(h)
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / (calls * replays)
+
+
 class Bench:
     def __init__(self, out_path=None, opts_kw=None):
         self.peak = _peak()
@@ -76,7 +98,7 @@ class Bench:
             self.out.write(line + "\n")
             self.out.flush()
 
-    def collective(self, cfg, R, dtype, coll, algo, count, chunk, iters=20, layers=0, **kw):
+    def collective(self, cfg, R, dtype, coll, algo, count, chunk, iters=20, layers=0, graph=False, **kw):
         comm = B.pl_comm_create(R, dtype)
         okw = dict(self.opts_kw)
         okw.update(kw)
@@ -96,12 +118,15 @@ class Bench:
         bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
                            [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
         p50, p10, p90 = _time(lambda: B.pl_execute(s, bufs, self.stream), iters, per_call_events=True)
+        graph_us = None
+        if graph:
+            graph_us = _time_graph(lambda h: B.pl_execute(s, bufs, h)) / max(1, layers)
         st = B.pl_comm_status(comm)
         nl = max(1, layers)
         sched_bytes = info.bytes_read + info.bytes_written
         rec = {"cfg": cfg, "coll": int(coll), "algo": algo, "R": R, "dtype": int(dtype),
                "message_bytes": int(info.message_bytes), "chunk": int(min(chunk, 1 << 40)), "layers": layers,
-               "us": p50 / nl, "us_p10": p10 / nl, "us_p90": p90 / nl,
+               "us": p50 / nl, "us_p10": p10 / nl, "us_p90": p90 / nl, "us_graph128": graph_us,
                "eff_gbs": info.message_bytes * nl / p50 / 1e3, "sched_gbs": sched_bytes / p50 / 1e3,
                "hbm_frac_measured": sched_bytes / p50 / 1e3 / self.peak, "hbm_frac_8TBps": sched_bytes / p50 / 1e3 / 8000.0,
                "n_ops": int(info.n_ops), "grid": int(info.grid), "threads": int(info.threads),
@@ -149,13 +174,31 @@ class Bench:
         B.pl_comm_destroy(comm)
 
 
+def probe(b):
+    """Reference points from library kernels on the same GPU (context for the roofline
+    fractions, not part of the product path): plain copy, fill and read over 1 GiB."""
+    n = 1 << 30
+    a = torch.empty(n, dtype=torch.uint8, device="cuda")
+    c = torch.empty(n, dtype=torch.uint8, device="cuda")
+    a.zero_()
+    c.zero_()
+    af = a.view(torch.float32)
+    for name, fn, nbytes in (("torch copy_ (read+write)", lambda: c.copy_(a), 2 * n),
+                             ("torch fill_ (write)", lambda: a.fill_(1), n),
+                             ("torch sum fp32 (read)", lambda: af.sum(), n)):
+        us, _, _ = _time(fn, 20)
+        b.emit({"cfg": "probe", "what": name, "gbs": nbytes / us / 1e3})
+
+
 def main(args=None):
-    which = os.environ.get("PL_SUITE", "c1,c2,c3,c4,c5").split(",")
+    which = os.environ.get("PL_SUITE", "probe,c1,c2,c3,c4,c5").split(",")
     os.makedirs("gpurun_out", exist_ok=True)
     b = Bench(os.environ.get("PL_SUITE_OUT", "gpurun_out/suite.jsonl"))
+    if "probe" in which:
+        probe(b)
     if "c1" in which:
         for dt in (B.PL_F32, B.PL_I32):
-            b.collective("C1", 4, dt, B.PL_ALLREDUCE, "ring", 262144, 65536, iters=50)
+            b.collective("C1", 4, dt, B.PL_ALLREDUCE, "ring", 262144, 65536, iters=50, graph=True)
     if "c2" in which:
         n = 32 * MIB  # 64 MiB bf16 per rank
         for algo in ("direct", "ring"):
@@ -169,7 +212,8 @@ def main(args=None):
                 if algo == "oneshot" and size > 64 * MIB:
                     continue
                 chunk = max(16, min(MIB, size // 8))
-                b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30 if lg < 24 else 10)
+                b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30 if lg < 24 else 10,
+                             graph=lg <= 21)
     if "c4" in which:
         b.moe("C4", identity=False)
         b.moe("C4", identity=True)

@@ -8,7 +8,7 @@
 //                     here as a free-running ring with full / empty mbarriers);
 //   warp 1  copier    for COPY stages: one bulk store shared -> global per stage, no
 //                     registers touched by the payload;
-//   warps 2..9 consumers  for REDUCE / COPY_REDUCE stages: read the source tiles from
+//   warps 2..17 consumers  for REDUCE / COPY_REDUCE stages: read the source tiles from
 //                     shared memory 16 bytes at a time, accumulate in fp32 in ascending
 //                     source order, store the result with 128-bit global stores.
 // A stage descriptor travels with every slot.  The last stage of an op carries its signal:
@@ -28,7 +28,7 @@ namespace {
 
 using namespace dev;
 
-constexpr int kConsumerWarps = 8;
+constexpr int kConsumerWarps = 16;
 constexpr int kConsumerThreads = 32 * kConsumerWarps;
 constexpr int kThreads = 32 * (2 + kConsumerWarps);
 constexpr int kMaxStages = 8;
@@ -52,7 +52,10 @@ static_assert(sizeof(StageDesc) == 48, "StageDesc layout");
 struct Ctrl {
   uint64_t full[kMaxStages];
   uint64_t empty[kMaxStages];
-  uint64_t done;  // consumer warps that finished writing the last stage of an op
+  // consumer warps that finished writing the last stage of an op.  One barrier per slot: a
+  // fast warp can be a whole stage ahead of a slow one, and arrivals for two different
+  // stages must never meet on one barrier.
+  uint64_t done[kMaxStages];
   int abort;
   int pad;
   StageDesc desc[kMaxStages];
@@ -165,7 +168,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
       ptx::mbar_init(&c->full[s], 1);
       ptx::mbar_init(&c->empty[s], 1 + kConsumerWarps);  // copier + every consumer warp
     }
-    ptx::mbar_init(&c->done, kConsumerWarps);
+    for (uint32_t s = 0; s < S; ++s) ptx::mbar_init(&c->done[s], kConsumerWarps);
     c->abort = 0;
     ptx::mbar_init_fence();
   }
@@ -323,7 +326,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
   } else {
     // ================================ consumers =========================================
     const int ctid = tid - 64;
-    uint32_t n_done = 0;  // completed phases of the done barrier
+    uint32_t done_parity = 0;  // bit s: parity of the next phase of done[s]
     for (uint32_t n = 0;; ++n) {
       const uint32_t s = n % S, ph = (n / S) & 1u;
       bool go = true;
@@ -341,15 +344,15 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
         __syncwarp();
         if (last && signal != kNoFlag) {
           // every consumer warp reports its stores; consumer thread 0 then publishes
-          if (lane == 0) ptx::mbar_arrive(&c->done);
+          if (lane == 0) ptx::mbar_arrive(&c->done[s]);
           if (ctid == 0) {
-            if (wait_bar(P, c, &c->done, n_done & 1u)) {
+            if (wait_bar(P, c, &c->done[s], (done_parity >> s) & 1u)) {
               __threadfence();
               red_release_add_u64(P.flags + signal, 1ull);
               if (signal2 != kNoFlag) red_release_add_u64(P.flags + signal2, 1ull);
             }
           }
-          ++n_done;
+          done_parity ^= 1u << s;
         }
       }
       __syncwarp();

@@ -33,6 +33,9 @@ struct Emitter {
   // Chunks each rank runs in the phase being emitted (0 = unknown).  When known, the slice
   // count is nudged upwards so that a rank's work items divide evenly over its queues.
   uint64_t phase_chunks = 0;
+  // slice_bytes == 0: pick the slice per phase so that every queue of the rank gets about
+  // two work items, within [min_slice, max_slice]
+  uint32_t min_slice = 16384, max_slice = 131072;
 
   int new_flag() { return L->n_flags++; }
 
@@ -50,7 +53,13 @@ struct Emitter {
     const uint64_t unit16 = kind == PL_OP_COPY ? 16 : 16 / elem_size(dtype);
     uint64_t wide = count * max_es;
     uint64_t n_slices = 1;
-    if (slice_bytes && wide > slice_bytes + slice_bytes / 2) n_slices = (wide + slice_bytes - 1) / slice_bytes;
+    uint64_t slice = slice_bytes;
+    if (slice == 0) {
+      const uint64_t phase_bytes = std::max<uint64_t>(1, phase_chunks) * wide;
+      slice = phase_bytes / (2 * (uint64_t)queues_per_rank);
+      slice = std::min<uint64_t>(max_slice, std::max<uint64_t>(min_slice, slice / 4096 * 4096));
+    }
+    if (wide > slice + slice / 2) n_slices = (wide + slice - 1) / slice;
     if (n_slices > 1 && phase_chunks && queues_per_rank > 1) {
       for (uint64_t k = n_slices; k <= 4 * n_slices; ++k)
         if ((phase_chunks * k) % (uint64_t)queues_per_rank == 0 && wide / k >= 4096) {
@@ -397,21 +406,26 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
     msg /= rq.R;
   }
   if (rq.coll == PL_ALLGATHER) msg *= rq.R;
-  // latency regime (register path, small slices) below 1 MiB per rank, layered schedules too
-  const bool small = msg <= (1u << 20) || rq.n_layers > 0;
-  if (p.datapath == PL_DP_AUTO) p.datapath = small ? PL_DP_LDST : PL_DP_TMA;
+  // bytes of all ranks' inputs and outputs: decides whether the working set lives in L2
+  uint64_t footprint = 2 * (uint64_t)rq.R * msg;
+  if (rq.coll == PL_REDUCE_SCATTER || rq.coll == PL_ALLGATHER) footprint = (uint64_t)(rq.R + 1) * msg;
+  if (rq.coll == PL_ALLTOALLV) footprint = 2 * (uint64_t)rq.R * msg;
+  // Register path while the working set is L2 sized (and for layered latency schedules);
+  // bulk-copy ring once it has to stream from HBM.  Measured crossover on B200: all-reduce of
+  // 16-32 MiB per rank at R=8.
+  const bool stream = footprint >= (256ull << 20) && rq.n_layers == 0;
+  if (p.datapath == PL_DP_AUTO) p.datapath = stream ? PL_DP_TMA : PL_DP_LDST;
   if (p.threads <= 0) p.threads = 512;
-  if (p.stages <= 0) p.stages = 3;
-  if (p.stage_bytes == 0) p.stage_bytes = 32768;
-  if (p.slice_bytes == 0) p.slice_bytes = small ? 16384 : (p.datapath == PL_DP_TMA ? 262144 : 65536);
+  if (p.stages <= 0) p.stages = 4;
+  if (p.stage_bytes == 0) p.stage_bytes = 49152;
   if (max_resident_ctas <= 0) return p;
   if (p.n_ctas <= 0) {
     const int full = std::max(rq.R, max_resident_ctas / rq.R * rq.R);
-    // work items per rank under this slicing (output bytes a rank produces / slice)
+    // queues a rank can keep busy: one per 16 KiB of what it produces
     uint64_t per_rank_out = msg;
     if (rq.coll == PL_REDUCE_SCATTER) per_rank_out = msg / rq.R;
-    uint64_t per_rank_slices = std::max<uint64_t>(1, (per_rank_out + p.slice_bytes - 1) / p.slice_bytes);
-    uint64_t want = per_rank_slices * rq.R;
+    const uint64_t unit = p.slice_bytes ? p.slice_bytes : 16384;
+    uint64_t want = std::max<uint64_t>(1, (per_rank_out + unit - 1) / unit) * rq.R;
     p.n_ctas = (int)std::min<uint64_t>(full, std::max<uint64_t>(rq.R, want));
   }
   p.n_ctas = std::max(rq.R, p.n_ctas / rq.R * rq.R);
@@ -430,6 +444,7 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
   if (reduces && dt == PL_U8) return fail(PL_ERR_UNSUPPORTED, "bytes cannot be reduced");
   Emitter em{L, rq.pol.slice_bytes};
   em.dtype = dt;
+  em.max_slice = rq.pol.datapath == PL_DP_TMA ? 262144 : 131072;
   em.queues_per_rank = std::max(1, rq.pol.n_ctas / R);
   L->n_layers = 1;
 
