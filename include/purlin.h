@@ -321,6 +321,42 @@ pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float
 pl_status_t pl_moe_plan_read(pl_moe_plan_t plan, int32_t* pos, int64_t* counts,
                              int64_t* expert_counts, void* stream);
 
+/* ---- for callers that cannot allocate ------------------------------------------------ */
+
+/* Ring reduce-scatter with no allocation of any kind (the paper has no counterpart; this
+ * entry point exists for deployments, not for the method).
+ *
+ * Who needs it: code that must not call cudaMalloc where the collective happens -- a
+ * serving loop that cannot afford cudaMalloc's device-wide synchronisation, a component
+ * living under a pre-planned memory arena, a plugin that only ever receives buffers.  The
+ * schedule-based path (pl_schedule_build + pl_execute) allocates its op list, flags and the
+ * scratch for travelling partial sums at build time; this call instead keeps the partial
+ * sums in a fixed 32 MiB array that is part of the library image on every GPU that loads
+ * the library (it stays resident until the process exits), and launches exactly one kernel.
+ *
+ *   in[r]   DEVICE pointer, count_per_rank elements (R partitions), 16-byte aligned
+ *   out[r]  DEVICE pointer, count_per_rank / R elements: sum over ranks of partition r
+ *   status  optional DEVICE word owned by the caller: cleared on `stream` before the launch,
+ *           set to PL_ERR_TIMEOUT if a wait inside the kernel gave up (2 s); may be NULL
+ * in / out are HOST arrays of R pointers.  dtype: PL_BF16, PL_F32 or PL_I32; results are the
+ * same as the ring reduce-scatter schedule's (fp32 partial sums for bf16, compensated pairs
+ * for fp32, ascending ring order).
+ *
+ * Limits and rules
+ *   - R * (R-2) * (count_per_rank / R) * partial_size must fit the 32 MiB array (partial_size
+ *     4 bytes for bf16 and int32, 8 for fp32); larger messages return PL_ERR_OVERFLOW before
+ *     anything is launched.  Other errors as pl_schedule_build / pl_execute
+ *     (PL_ERR_INVALID_ARG, PL_ERR_ALIGNMENT, PL_ERR_UNSUPPORTED, PL_ERR_CUDA).
+ *   - The first call on a device looks up the device address of the built-in array (a one-
+ *     time set-up with that device current); make that first call outside any stream capture.
+ *   - All calls on a GPU share the array, and it keeps whatever the last call left there.
+ *     Nothing in it needs clearing between calls, but two calls that overlap in time on the
+ *     same GPU (e.g. on two streams) race on it: issue them on one stream or order them.
+ *   - Calls no cudaMalloc, cudaFree or other allocating routine. */
+pl_status_t pl_reduce_scatter_ring_static(int R, pl_dtype_t dtype, size_t count_per_rank,
+                                          const void* const* in, void* const* out,
+                                          int32_t* status, void* stream);
+
 const char* pl_status_string(pl_status_t st);
 
 /* Number of kernels this library has launched in the calling process (all entry points). */

@@ -87,7 +87,7 @@ EXPORTS = [
     "pl_schedule_dump", "pl_schedule_validate", "pl_schedule_debug_break_wait", "pl_schedule_destroy",
     "pl_execute", "pl_execute_host",
     "pl_moe_plan_create", "pl_moe_plan_destroy", "pl_moe_dispatch", "pl_moe_combine", "pl_moe_plan_read",
-    "pl_status_string", "pl_launch_count",
+    "pl_status_string", "pl_launch_count", "pl_reduce_scatter_ring_static",
 ]
 
 _lib = None
@@ -131,6 +131,7 @@ def load():
         "pl_moe_dispatch": [vp, P(vp), P(vp), P(vp), P(vp), vp],
         "pl_moe_combine": [vp, P(vp), P(vp), P(vp), vp],
         "pl_moe_plan_read": [vp, vp, vp, vp, vp],
+        "pl_reduce_scatter_ring_static": [i32, i32, sz, P(vp), P(vp), vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -292,6 +293,14 @@ def pl_moe_combine(plan, y, gates, out, stream=0):
 def pl_moe_plan_read(plan, pos=0, counts=0, expert_counts=0, stream=0):
     """pos / counts / expert_counts: host addresses (e.g. numpy ``arr.ctypes.data``) or 0."""
     return load().pl_moe_plan_read(plan, pos or None, counts or None, expert_counts or None, stream)
+
+
+def pl_reduce_scatter_ring_static(R, dtype, count_per_rank, ins, outs, status=0, stream=0):
+    """Ring reduce-scatter that allocates nothing (see include/purlin.h).  ins / outs are
+    device addresses per rank; status an optional device address of an int32.  Returns the
+    pl_status_t instead of raising, so that callers can test the size limit."""
+    return load().pl_reduce_scatter_ring_static(R, dtype, count_per_rank, _ptr_array(ins), _ptr_array(outs),
+                                                status or None, stream)
 
 
 def pl_launch_count() -> int:
