@@ -33,6 +33,9 @@ if ROOT not in sys.path:
 MIB = 1 << 20
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one reduce-scatter launch of this workload,
+# from the ncu capture summarised in profiles/pl_exec_tma_kernel_bf16_c2_reduce_scatter_all_gather.md
+NCU_RS_TRAFFIC_BYTES = 594786560.0
 
 
 def measured_peak():
@@ -115,18 +118,15 @@ def c2_inputs(R, n, seed=0, unique=None):
 
 def run_purlin(args):
     import torch
-    import torch.distributed as dist
 
     from paper_2609_36954_b200 import binding as B
+    from paper_2609_36954_b200 import replicas
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = replicas.world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    replicas.init("nccl")
 
     R, Mb, chunk = C2["R"], C2["bytes_per_rank"], C2["chunk"]
     n = Mb // 2
@@ -167,8 +167,7 @@ def run_purlin(args):
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
     sampler = ClockSampler(local)
     launches0 = B.pl_launch_count()
-    if world > 1:
-        dist.barrier()
+    replicas.barrier()
     torch.cuda.synchronize()
     sampler.start()
     t_begin = torch.cuda.Event(enable_timing=True)
@@ -188,14 +187,12 @@ def run_purlin(args):
     rs_ms = np.array([ev[i][0].elapsed_time(ev[i][1]) for i in range(K)])
     ag_ms = np.array([ev[i][1].elapsed_time(ev[i][2]) for i in range(K)])
     assert B.pl_comm_status(comm).code == B.PL_OK
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    replicas.barrier()
+    total_ms = replicas.max_over_ranks(total_ms)
 
     ms_per_step = total_ms / K
     eff_bytes = irs.message_bytes + iag.message_bytes  # 64 MiB + 64 MiB per step
-    value = world * eff_bytes / (ms_per_step * 1e-3) / 1e9
+    value = replicas.aggregate_throughput(eff_bytes, ms_per_step, world) / 1e9
 
     # ---- end to end through the host-buffer entry point -----------------------------------
     e2e = None
@@ -211,22 +208,17 @@ def run_purlin(args):
         for _ in range(2):
             e2e_step()
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(Ke):
             e2e_step()
         e1.record()
         torch.cuda.synchronize()
-        e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([e_ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = replicas.max_over_ranks(e0.elapsed_time(e1))
         h2d = sum(int(irs.in_bytes[r]) + int(iag.in_bytes[r]) for r in range(R))
         d2h = sum(int(irs.out_bytes[r]) + int(iag.out_bytes[r]) for r in range(R))
-        e2e = {"value": world * eff_bytes / (e_ms / Ke * 1e-3) / 1e9, "unit": "GB/s", "steps": Ke,
+        e2e = {"value": replicas.aggregate_throughput(eff_bytes, e_ms / Ke, world) / 1e9, "unit": "GB/s", "steps": Ke,
                "ms_per_step": e_ms / Ke, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "api": "pl_execute_host (pinned host buffers in and out)"}
         # parity spot check of the e2e result on sampled elements against the definition
@@ -242,7 +234,7 @@ def run_purlin(args):
     ag_floor = iag.in_bytes[0] * R + iag.bytes_written     # compulsory DRAM traffic (R+1) * M
     rs_gbs = rs_alg / (rs_ms.mean() * 1e-3) / 1e9
     ag_gbs = ag_floor / (ag_ms.mean() * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "pl_exec_kernel<bf16> (reduce-scatter launch)",
+    roofline = {"bound": "hbm", "kernel": "pl_exec_tma_kernel<bf16> (reduce-scatter launch)",
                 "achieved": rs_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": rs_gbs / peak, "frac_of_nominal_8TBps": rs_gbs / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_launch": int(rs_alg), "avg_launch_us": float(rs_ms.mean() * 1e3),
@@ -280,8 +272,7 @@ def run_purlin(args):
     B.pl_schedule_destroy(rs)
     B.pl_schedule_destroy(ag)
     B.pl_comm_destroy(comm)
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.finalize()
 
 
 # ------------------------------------------------------------------------------------------
@@ -374,7 +365,7 @@ def main():
     ap.add_argument("--datapath", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--stage-bytes", type=int, default=0)
-    ap.add_argument("--ncu-traffic", type=float, default=None,
+    ap.add_argument("--ncu-traffic", type=float, default=NCU_RS_TRAFFIC_BYTES,
                     help="dram bytes per reduce-scatter launch from the committed ncu capture")
     args = ap.parse_args()
     if args.impl == "reference":

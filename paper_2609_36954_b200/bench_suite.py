@@ -192,8 +192,10 @@ def probe(b):
 
 def main(args=None):
     which = os.environ.get("PL_SUITE", "probe,c1,c2,c3,c4,c5").split(",")
-    os.makedirs("gpurun_out", exist_ok=True)
-    b = Bench(os.environ.get("PL_SUITE_OUT", "gpurun_out/suite.jsonl"))
+    out = os.environ.get("PL_SUITE_OUT")  # optional file that receives the JSON lines too
+    if out and os.path.dirname(out):
+        os.makedirs(os.path.dirname(out), exist_ok=True)
+    b = Bench(out)
     if "probe" in which:
         probe(b)
     if "c1" in which:
