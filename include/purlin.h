@@ -133,6 +133,8 @@ typedef struct {
   uint32_t flags;        /* PL_OPT_*                                                      */
 } pl_sched_opts_t;
 #define PL_OPT_SKIP_VALIDATE 1u /* do not run the static validator inside build */
+#define PL_OPT_NO_L2_HINTS 2u  /* bulk copies without L2 eviction hints (default: stores evict-first,
+                                  sources of copy ops evict-last; measured 7 % on all-gather) */
 
 /* A buffer reference inside an op: rank's in/out/scratch buffer, byte offset, and the
  * element type stored there (partials of a bf16 reduction are PL_F32). */

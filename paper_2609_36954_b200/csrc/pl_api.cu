@@ -25,6 +25,7 @@ struct pl_schedule_s {
   Policy pol{};
   pl_sched_info_t info{};
   uint64_t timeout_ns = 0;
+  bool no_l2_hints = false;
   // host copies in device (queue-major) order
   std::vector<DevOp> dev_ops;
   std::vector<uint32_t> queue_begin;
@@ -207,6 +208,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   S->comm = comm;
   S->pol = pol;
   S->timeout_ns = timeout;
+  S->no_l2_hints = (flags & PL_OPT_NO_L2_HINTS) != 0;
   std::string err;
   pl_status_t st = lower(rq, &S->L, &err);
   if (st != PL_OK) {
@@ -487,6 +489,8 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   P.n_ranks = R;
   P.stages = s->pol.stages;
   P.stage_bytes = s->pol.stage_bytes;
+  // bulk stores stream out (evict-first), sources of copies are re-read by other ranks (evict-last)
+  P.hints = s->no_l2_hints ? 0u : 6u;
   cudaError_t le = s->pol.datapath == PL_DP_TMA
                        ? launch_exec_tma(s->comm->dtype, P, s->pol.n_ctas, static_cast<cudaStream_t>(stream))
                        : launch_exec(s->comm->dtype, P, s->pol.n_ctas, s->pol.threads, static_cast<cudaStream_t>(stream));

@@ -63,6 +63,9 @@ struct Ctrl {
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
 // Bounded mbarrier wait.  Returns false when the CTA is aborting or the time limit passed.
+// Waits inside a CTA get twice the limit of a flag wait: when a dependency never arrives, the
+// warps starved behind the producer started waiting earlier than the producer itself, and the
+// record should name the flag (the cause), not a starved barrier.
 __device__ __forceinline__ bool wait_bar(const ExecParams& P, Ctrl* c, uint64_t* bar, uint32_t parity) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
@@ -70,7 +73,7 @@ __device__ __forceinline__ bool wait_bar(const ExecParams& P, Ctrl* c, uint64_t*
     if (ptx::mbar_try_wait(bar, parity)) return true;
     if ((spins & 255u) == 0) {
       if (*reinterpret_cast<volatile int*>(&c->abort)) return false;
-      if (globaltimer_ns() - t0 > P.timeout_ns) {
+      if (globaltimer_ns() - t0 > 2ull * P.timeout_ns + 1000000ull) {
         record_timeout(P, blockIdx.x, 0xFFFFFFFFu, 0xFFFFFFFFu, parity, 0);
         *reinterpret_cast<volatile int*>(&c->abort) = 1;
         return false;
@@ -261,8 +264,12 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
           ptx::mbar_expect_tx(&c->full[s], units * unit_b);
         }
         __syncwarp();
-        if (lane < (int)n_src)
-          ptx::bulk_g2s(slots + (size_t)s * slot_bytes + my_tile_off, my_src + u0 * my_w, units * my_w, &c->full[s]);
+        if (lane < (int)n_src) {
+          void* sdst = slots + (size_t)s * slot_bytes + my_tile_off;
+          if ((P.hints & 4u) && kind == PL_OP_COPY) ptx::bulk_g2s_hint(sdst, my_src + u0 * my_w, units * my_w, &c->full[s], ptx::policy_evict_last());
+          else if (P.hints & 1u) ptx::bulk_g2s_hint(sdst, my_src + u0 * my_w, units * my_w, &c->full[s], ptx::policy_evict_first());
+          else ptx::bulk_g2s(sdst, my_src + u0 * my_w, units * my_w, &c->full[s]);
+        }
         ++n;
       }
     }
@@ -295,7 +302,8 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
       if (kind == kEnd) break;
       if (lane == 0) {
         if (kind == PL_OP_COPY) {
-          ptx::bulk_s2g(d.dst, slots + (size_t)s * slot_bytes, d.units * 16u);
+          if (P.hints & 2u) ptx::bulk_s2g_hint(d.dst, slots + (size_t)s * slot_bytes, d.units * 16u, ptx::policy_evict_first());
+          else ptx::bulk_s2g(d.dst, slots + (size_t)s * slot_bytes, d.units * 16u);
           ptx::bulk_commit();
           if (prev >= 0) {
             ptx::bulk_wait_read<1>();

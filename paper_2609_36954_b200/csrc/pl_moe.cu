@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(32) moe_move_kernel(const __grid_constant__ Di
     const char* src = static_cast<const char*>(P.x[p]) + t * g.row_bytes + off;
     const uint32_t s = (uint32_t)(n % S);
     ptx::mbar_expect_tx(full + s, bytes);
-    ptx::bulk_g2s(tiles + (size_t)s * g.tile_bytes, src, bytes, full + s);
+    ptx::bulk_g2s_hint(tiles + (size_t)s * g.tile_bytes, src, bytes, full + s, ptx::policy_evict_first());
   };
 
   unsigned long long issued = 0;
@@ -206,8 +206,9 @@ __global__ void __launch_bounds__(32) moe_move_kernel(const __grid_constant__ Di
     }
     ok = __all_sync(0xFFFFFFFFu, ok);
     if (!ok) { failed = true; break; }
-    if (row >= 0) ptx::bulk_s2g(static_cast<char*>(P.recv[r]) + (size_t)row * g.row_bytes + off,
-                                tiles + (size_t)s * g.tile_bytes, bytes);
+    // every token row is read once and every received row written once: both stream through L2
+    if (row >= 0) ptx::bulk_s2g_hint(static_cast<char*>(P.recv[r]) + (size_t)row * g.row_bytes + off,
+                                     tiles + (size_t)s * g.tile_bytes, bytes, ptx::policy_evict_first());
     ptx::bulk_commit();
     if (n >= (unsigned long long)L) {
       ptx::bulk_wait_read<L>();
