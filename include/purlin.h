@@ -131,8 +131,20 @@ typedef struct {
                          /* staging CTA ... announces")                                   */
   uint64_t timeout_ns;   /* bound of every device-side wait; 0 = 2 s                      */
   uint32_t flags;        /* PL_OPT_*                                                      */
+  uint64_t staging_bytes; /* PL_OPT_STAGED: staging capacity per rank; 0 = min(256 MiB, need) */
 } pl_sched_opts_t;
 #define PL_OPT_SKIP_VALIDATE 1u /* do not run the static validator inside build */
+/* Treat in/out as ORDINARY application buffers that peers must not touch (Sec. 3.2, "Protocol
+ * operations": stage -> notify -> consume; Algorithm 1 with its staging role).  Every rank
+ * first copies its contribution chunk by chunk into schedule-owned staging memory and
+ * publishes staged(r,k,c); consumers pull only from staging; a composed all-reduce also keeps
+ * its reduced chunks Y_k[c] in staging and the gather role publishes consumed(r,k,c).  Staging
+ * holds staging_bytes per rank: when the message needs more, chunk slots are reused cyclically
+ * (Sec. 4.1) and a stage op waits until the slot's previous chunk has been consumed.  Only
+ * PL_ALGO_DIRECT.  (The paper alternates two staging buffers by epoch parity so that a rank
+ * can start the next call early; here a launch ends only when every rank has drained, so one
+ * buffer is enough.) */
+#define PL_OPT_STAGED 4u
 #define PL_OPT_NO_L2_HINTS 2u  /* bulk copies without L2 eviction hints (default: stores evict-first,
                                   sources of copy ops evict-last; measured 7 % on all-gather) */
 
@@ -265,6 +277,11 @@ pl_status_t pl_schedule_dump(pl_schedule_t s, pl_op_t* ops, size_t cap, size_t* 
  * the topological order, queue order embeds in that order.  On failure returns
  * PL_ERR_INVALID_SCHEDULE and writes a message into msg (may be NULL). */
 pl_status_t pl_schedule_validate(pl_schedule_t s, char* msg, size_t msg_cap);
+
+/* TEST HOOK: remove the first wait edge of op `op_index` from the host copy of the schedule,
+ * so that pl_schedule_validate can be shown to notice the missing ordering.  The device copy
+ * is left alone; do not execute the schedule afterwards. */
+pl_status_t pl_schedule_debug_drop_wait(pl_schedule_t s, size_t op_index);
 
 /* TEST HOOK: corrupt one wait edge of a built schedule so that it can never be satisfied
  * (raises the needed count of op `op_index`'s first wait).  Used with a short timeout_ns to

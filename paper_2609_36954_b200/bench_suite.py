@@ -191,7 +191,7 @@ def probe(b):
 
 
 def main(args=None):
-    which = os.environ.get("PL_SUITE", "probe,c1,c2,c3,c4,c5").split(",")
+    which = os.environ.get("PL_SUITE", "probe,c1,c2,staged,c3,c4,c5").split(",")
     out = os.environ.get("PL_SUITE_OUT")  # optional file that receives the JSON lines too
     if out and os.path.dirname(out):
         os.makedirs(os.path.dirname(out), exist_ok=True)
@@ -207,6 +207,19 @@ def main(args=None):
             for chunk in (256 * 1024, MIB):
                 b.collective("C2-RS", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, algo, n, chunk)
                 b.collective("C2-AG", 8, B.PL_BF16, B.PL_ALLGATHER, algo, n // 8, chunk)
+    if "staged" in which:
+        # the paper's default setting: ordinary application buffers, so the work of staging is
+        # included (Sec. 5, "Collective Microbenchmarks"); full and restricted staging capacity
+        n = 32 * MIB
+        for cap in (0, 32 * MIB):
+            kw = dict(flags=B.PL_OPT_STAGED, staging_bytes=cap)
+            b.collective("staged-RS cap=%d" % cap, 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "direct", n, MIB, **kw)
+            b.collective("staged-AG cap=%d" % cap, 8, B.PL_BF16, B.PL_ALLGATHER, "direct", n // 8, MIB,
+                         flags=B.PL_OPT_STAGED, staging_bytes=cap // 8)
+            b.collective("staged-A2A cap=%d" % cap, 8, B.PL_BF16, B.PL_ALLTOALL, "direct", n, MIB, **kw)
+            for size in (MIB, 16 * MIB, 64 * MIB, 256 * MIB):
+                b.collective("staged-AR cap=%d" % cap, 8, B.PL_BF16, B.PL_ALLREDUCE, "direct", size // 2,
+                             max(16, min(MIB, size // 8)), iters=10, **kw)
     if "c3" in which:
         for lg in range(12, 29):
             size = 1 << lg

@@ -34,6 +34,7 @@ PL_BUF_IN, PL_BUF_OUT, PL_BUF_SCRATCH = range(3)
 PL_DP_AUTO, PL_DP_LDST, PL_DP_TMA = range(3)
 PL_OPT_SKIP_VALIDATE = 1
 PL_OPT_NO_L2_HINTS = 2
+PL_OPT_STAGED = 4
 
 
 class PurlinError(RuntimeError):
@@ -45,7 +46,8 @@ class PurlinError(RuntimeError):
 class pl_sched_opts_t(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("n_ctas", C.c_int32), ("threads", C.c_int32),
                 ("datapath", C.c_int32), ("stages", C.c_int32), ("stage_bytes", C.c_uint32),
-                ("slice_bytes", C.c_uint32), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32)]
+                ("slice_bytes", C.c_uint32), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32),
+                ("staging_bytes", C.c_uint64)]
 
 
 class pl_ref_t(C.Structure):
@@ -85,7 +87,8 @@ class pl_devstatus_t(C.Structure):
 EXPORTS = [
     "pl_comm_create", "pl_comm_create_planner", "pl_comm_destroy", "pl_comm_status", "pl_comm_reset",
     "pl_schedule_build", "pl_schedule_build_v", "pl_schedule_build_layers", "pl_schedule_info",
-    "pl_schedule_dump", "pl_schedule_validate", "pl_schedule_debug_break_wait", "pl_schedule_destroy",
+    "pl_schedule_dump", "pl_schedule_validate", "pl_schedule_debug_break_wait", "pl_schedule_debug_drop_wait",
+    "pl_schedule_destroy",
     "pl_execute", "pl_execute_host",
     "pl_moe_plan_create", "pl_moe_plan_destroy", "pl_moe_dispatch", "pl_moe_combine", "pl_moe_plan_read",
     "pl_status_string", "pl_launch_count", "pl_reduce_scatter_ring_static",
@@ -124,6 +127,7 @@ def load():
         "pl_schedule_dump": [vp, P(pl_op_t), sz, P(sz)],
         "pl_schedule_validate": [vp, C.c_char_p, sz],
         "pl_schedule_debug_break_wait": [vp, sz],
+        "pl_schedule_debug_drop_wait": [vp, sz],
         "pl_schedule_destroy": [vp],
         "pl_execute": [vp, P(pl_bufs_t), vp],
         "pl_execute_host": [vp, P(pl_bufs_t), P(pl_bufs_t), vp],
@@ -156,11 +160,12 @@ def _check(st, where):
 
 
 def make_opts(n_ctas=0, threads=0, datapath=PL_DP_AUTO, stages=0, stage_bytes=0, slice_bytes=0,
-              timeout_ns=0, flags=0):
+              timeout_ns=0, flags=0, staging_bytes=0):
     o = pl_sched_opts_t()
     o.struct_size = C.sizeof(pl_sched_opts_t)
     o.n_ctas, o.threads, o.datapath, o.stages = n_ctas, threads, datapath, stages
     o.stage_bytes, o.slice_bytes, o.timeout_ns, o.flags = stage_bytes, slice_bytes, timeout_ns, flags
+    o.staging_bytes = staging_bytes
     return o
 
 
@@ -251,6 +256,10 @@ def pl_schedule_validate(s):
 
 def pl_schedule_debug_break_wait(s, op_index):
     _check(load().pl_schedule_debug_break_wait(s, op_index), "pl_schedule_debug_break_wait")
+
+
+def pl_schedule_debug_drop_wait(s, op_index):
+    _check(load().pl_schedule_debug_drop_wait(s, op_index), "pl_schedule_debug_drop_wait")
 
 
 def pl_schedule_destroy(s):

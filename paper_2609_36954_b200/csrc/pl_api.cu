@@ -174,6 +174,8 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
     pol.slice_bytes = opts->slice_bytes;
     if (opts->timeout_ns) timeout = opts->timeout_ns;
     flags = opts->flags;
+    rq.staged = (flags & PL_OPT_STAGED) != 0;
+    rq.staging_bytes = opts->staging_bytes;
     if (pol.threads < 0 || pol.threads % 32 || pol.threads > exec_max_threads()) return PL_ERR_INVALID_ARG;
     if (pol.n_ctas < 0 || pol.stages < 0 || pol.stage_bytes % 16 || pol.slice_bytes % 16) return PL_ERR_INVALID_ARG;
     if (pol.datapath < PL_DP_AUTO || pol.datapath > PL_DP_TMA) return PL_ERR_INVALID_ARG;
@@ -406,6 +408,14 @@ pl_status_t pl_schedule_validate(pl_schedule_t s, char* msg, size_t msg_cap) {
     std::snprintf(msg, msg_cap, "%s", err.c_str());
   }
   return st;
+}
+
+pl_status_t pl_schedule_debug_drop_wait(pl_schedule_t s, size_t op_index) {
+  if (!s || op_index >= s->L.ops.size()) return PL_ERR_INVALID_ARG;
+  HostOp& h = s->L.ops[op_index];
+  if (h.waits.empty()) return PL_ERR_INVALID_ARG;
+  h.waits.erase(h.waits.begin());
+  return PL_OK;
 }
 
 pl_status_t pl_schedule_debug_break_wait(pl_schedule_t s, size_t op_index) {

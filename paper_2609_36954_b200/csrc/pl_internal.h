@@ -34,6 +34,7 @@ struct HostOp {
   std::vector<int> waits;  // flag ids
   int signal = -1;
   int signal2 = -1;
+  int role = 0;  // 0 = any queue of the rank; 1 stage, 2 reduce, 3 gather: CTA groups per role (Sec. 3.2)
   int queue = -1;
   int topo = -1;
 };
@@ -99,6 +100,7 @@ struct Lowered {
   uint64_t out_bytes[PL_MAX_RANKS] = {0};
   uint64_t message_bytes = 0;
   int n_layers = 1;
+  int role_queues[4] = {0, 0, 0, 0};  // queues per rank reserved for each role (0 = roles unused)
 };
 
 struct BuildRequest {
@@ -107,6 +109,8 @@ struct BuildRequest {
   uint64_t chunk_bytes;
   const uint64_t* counts_v;  // R*R for all-to-all-v, else null
   int n_layers;              // 0: single collective
+  bool staged;               // stage through schedule-owned memory (ordinary application buffers)
+  uint64_t staging_bytes;    // staging capacity per rank (0 = default)
   Policy pol;
 };
 

@@ -36,6 +36,7 @@ struct Emitter {
   // slice_bytes == 0: pick the slice per phase so that every queue of the rank gets about
   // two work items, within [min_slice, max_slice]
   uint32_t min_slice = 16384, max_slice = 131072;
+  int role = 0;  // role stamped on emitted ops
 
   int new_flag() { return L->n_flags++; }
 
@@ -86,6 +87,7 @@ struct Emitter {
       op.waits = waits;
       op.signal = signal;
       op.signal2 = signal2;
+      op.role = role;
       L->ops.push_back(std::move(op));
     }
   }
@@ -391,6 +393,192 @@ void ar_tree(Emitter& em, const Geo& g) {
       }
 }
 
+// ---- staged variants: ordinary application buffers (Sec. 3.2 protocol, Algorithm 1) --------
+// Peers never touch in/out: every rank copies its contribution chunk by chunk into its own
+// staging memory (stage role) and publishes it; consumers pull from staging only.  Staging has
+// `ns` chunk slots per partition; chunk c lives in slot c % ns and a stage op for chunk c waits
+// until chunk c - ns has been consumed (cyclic staging, Sec. 4.1).  Roles get their own CTA
+// groups so that staging runs ahead of reduction and gathering.
+struct Staging {
+  uint64_t ns;      // chunk slots per partition
+  uint64_t chunkB;  // bytes per chunk slot
+};
+
+Staging staging_geo(const Geo& g, uint64_t capacity, uint64_t partitions) {
+  Staging s;
+  s.chunkB = g.chunk * g.es;
+  if (capacity == 0) capacity = 256ull << 20;
+  s.ns = std::max<uint64_t>(1, std::min<uint64_t>(g.n_c, capacity / std::max<uint64_t>(1, partitions * s.chunkB)));
+  return s;
+}
+
+void set_roles(Emitter& em, int R, const double (&cost)[4]) {
+  // split a rank's queues between the roles in proportion to the bytes each role moves
+  const int Q = em.queues_per_rank;
+  int n_roles = 0;
+  double total = 0;
+  for (int i = 1; i < 4; ++i)
+    if (cost[i] > 0) { ++n_roles; total += cost[i]; }
+  if (Q < n_roles) return;  // too few queues: every op may run anywhere
+  int left = Q;
+  for (int i = 1; i < 4; ++i)
+    if (cost[i] > 0) {
+      em.L->role_queues[i] = std::max(1, (int)(Q * cost[i] / total));
+      left -= em.L->role_queues[i];
+    }
+  for (int i = 1; left != 0; i = i % 3 + 1)  // hand out / take back the rounding remainder
+    if (cost[i] > 0 && (left > 0 || em.L->role_queues[i] > 1)) {
+      em.L->role_queues[i] += left > 0 ? 1 : -1;
+      left += left > 0 ? -1 : 1;
+    }
+  (void)R;
+}
+
+void begin_role(Emitter& em, int role, uint64_t phase_chunks) {
+  em.role = em.L->role_queues[role] ? role : 0;
+  em.phase_chunks = phase_chunks;
+}
+
+void ar_direct_staged(Emitter& em, const Geo& g, uint64_t capacity) {
+  const int R = g.R;
+  const Staging st = staging_geo(g, capacity, R);
+  const double cost[4] = {0, 2.0, (R + 1.0) / R, 2.0};
+  set_roles(em, R, cost);
+  const int q_all = em.queues_per_rank;
+  auto S_off = [&](int k, uint64_t c) { return ((uint64_t)k * st.ns + c % st.ns) * st.chunkB; };
+  auto Y_off = [&](uint64_t c) { return ((uint64_t)R * st.ns + c % st.ns) * st.chunkB; };
+  std::vector<int> staged(R * g.n_c), reduced(R * g.n_c), consumed(R * g.n_c);
+  for (size_t i = 0; i < staged.size(); ++i) { staged[i] = em.new_flag(); reduced[i] = em.new_flag(); consumed[i] = em.new_flag(); }
+  for (uint64_t c = 0; c < g.n_c; ++c) {
+    begin_role(em, 1, (uint64_t)R);
+    if (em.role) em.queues_per_rank = em.L->role_queues[1];
+    for (int k = 0; k < R; ++k)
+      for (int r = 0; r < R; ++r) {
+        std::vector<int> w;
+        if (c >= st.ns) w.push_back(reduced[k * g.n_c + c - st.ns]);  // slot still holds live data
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_SCRATCH, PL_U8, S_off(k, c)), false,
+                    {ref(r, PL_BUF_IN, PL_U8, (k * g.P + c * g.chunk) * g.es)}, g.clen(c) * g.es, w, staged[k * g.n_c + c]);
+      }
+    begin_role(em, 2, 1);
+    if (em.role) em.queues_per_rank = em.L->role_queues[2];
+    for (int k = 0; k < R; ++k) {
+      std::vector<pl_ref_t> src;
+      for (int p = 0; p < R; ++p) src.push_back(ref(p, PL_BUF_SCRATCH, g.dtype, S_off(k, c)));
+      std::vector<int> w{staged[k * g.n_c + c]};
+      if (c >= st.ns) w.push_back(consumed[k * g.n_c + c - st.ns]);
+      em.chunk_op(PL_OP_REDUCE, k, 0, ref(k, PL_BUF_SCRATCH, g.dtype, Y_off(c)), false, src, g.clen(c), w, reduced[k * g.n_c + c]);
+    }
+    begin_role(em, 3, (uint64_t)R);
+    if (em.role) em.queues_per_rank = em.L->role_queues[3];
+    for (int i = 0; i < R; ++i)
+      for (int r = 0; r < R; ++r) {
+        const int k = (r + i) % R;
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, (k * g.P + c * g.chunk) * g.es), false,
+                    {ref(k, PL_BUF_SCRATCH, PL_U8, Y_off(c))}, g.clen(c) * g.es, {reduced[k * g.n_c + c]},
+                    consumed[k * g.n_c + c]);
+      }
+    em.queues_per_rank = q_all;
+  }
+  for (int r = 0; r < R; ++r) em.L->scratch_per_rank[r] = ((uint64_t)R * st.ns + st.ns) * st.chunkB;
+}
+
+void rs_direct_staged(Emitter& em, const Geo& g, uint64_t capacity) {
+  const int R = g.R;
+  const Staging st = staging_geo(g, capacity, R);
+  const double cost[4] = {0, 2.0, (R + 1.0) / R, 0};
+  set_roles(em, R, cost);
+  const int q_all = em.queues_per_rank;
+  auto S_off = [&](int k, uint64_t c) { return ((uint64_t)k * st.ns + c % st.ns) * st.chunkB; };
+  std::vector<int> staged(R * g.n_c), reduced(R * g.n_c);
+  for (size_t i = 0; i < staged.size(); ++i) { staged[i] = em.new_flag(); reduced[i] = em.new_flag(); }
+  for (uint64_t c = 0; c < g.n_c; ++c) {
+    begin_role(em, 1, (uint64_t)R);
+    if (em.role) em.queues_per_rank = em.L->role_queues[1];
+    for (int k = 0; k < R; ++k)
+      for (int r = 0; r < R; ++r) {
+        std::vector<int> w;
+        if (c >= st.ns) w.push_back(reduced[k * g.n_c + c - st.ns]);
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_SCRATCH, PL_U8, S_off(k, c)), false,
+                    {ref(r, PL_BUF_IN, PL_U8, (k * g.P + c * g.chunk) * g.es)}, g.clen(c) * g.es, w, staged[k * g.n_c + c]);
+      }
+    begin_role(em, 2, 1);
+    if (em.role) em.queues_per_rank = em.L->role_queues[2];
+    for (int k = 0; k < R; ++k) {
+      std::vector<pl_ref_t> src;
+      for (int p = 0; p < R; ++p) src.push_back(ref(p, PL_BUF_SCRATCH, g.dtype, S_off(k, c)));
+      em.chunk_op(PL_OP_REDUCE, k, 0, ref(k, PL_BUF_OUT, g.dtype, c * g.chunk * g.es), false, src, g.clen(c),
+                  {staged[k * g.n_c + c]}, reduced[k * g.n_c + c]);
+    }
+    em.queues_per_rank = q_all;
+  }
+  for (int r = 0; r < R; ++r) em.L->scratch_per_rank[r] = (uint64_t)R * st.ns * st.chunkB;
+}
+
+void ag_direct_staged(Emitter& em, const Geo& g, uint64_t capacity) {
+  const int R = g.R;
+  const Staging st = staging_geo(g, capacity, 1);
+  const double cost[4] = {0, 2.0, 0, 2.0 * R};
+  set_roles(em, R, cost);
+  const int q_all = em.queues_per_rank;
+  std::vector<int> staged(R * g.n_c), consumed(R * g.n_c);
+  for (size_t i = 0; i < staged.size(); ++i) { staged[i] = em.new_flag(); consumed[i] = em.new_flag(); }
+  for (uint64_t c = 0; c < g.n_c; ++c) {
+    begin_role(em, 1, 1);
+    if (em.role) em.queues_per_rank = em.L->role_queues[1];
+    for (int r = 0; r < R; ++r) {
+      std::vector<int> w;
+      if (c >= st.ns) w.push_back(consumed[r * g.n_c + c - st.ns]);
+      em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_SCRATCH, PL_U8, (c % st.ns) * st.chunkB), false,
+                  {ref(r, PL_BUF_IN, PL_U8, c * g.chunk * g.es)}, g.clen(c) * g.es, w, staged[r * g.n_c + c]);
+    }
+    begin_role(em, 3, (uint64_t)R);
+    if (em.role) em.queues_per_rank = em.L->role_queues[3];
+    for (int i = 0; i < R; ++i)
+      for (int r = 0; r < R; ++r) {
+        const int p = (r + i) % R;
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, (p * g.P + c * g.chunk) * g.es), false,
+                    {ref(p, PL_BUF_SCRATCH, PL_U8, (c % st.ns) * st.chunkB)}, g.clen(c) * g.es, {staged[p * g.n_c + c]},
+                    consumed[p * g.n_c + c]);
+      }
+    em.queues_per_rank = q_all;
+  }
+  for (int r = 0; r < R; ++r) em.L->scratch_per_rank[r] = st.ns * st.chunkB;
+}
+
+void a2a_direct_staged(Emitter& em, const Geo& g, uint64_t capacity) {
+  const int R = g.R;
+  const Staging st = staging_geo(g, capacity, R);
+  const double cost[4] = {0, 2.0, 0, 2.0};
+  set_roles(em, R, cost);
+  const int q_all = em.queues_per_rank;
+  auto S_off = [&](int k, uint64_t c) { return ((uint64_t)k * st.ns + c % st.ns) * st.chunkB; };
+  std::vector<int> staged((size_t)R * R * g.n_c), consumed((size_t)R * R * g.n_c);
+  for (size_t i = 0; i < staged.size(); ++i) { staged[i] = em.new_flag(); consumed[i] = em.new_flag(); }
+  auto fi = [&](int r, int k, uint64_t c) { return ((size_t)r * R + k) * g.n_c + c; };
+  for (uint64_t c = 0; c < g.n_c; ++c) {
+    begin_role(em, 1, (uint64_t)R);
+    if (em.role) em.queues_per_rank = em.L->role_queues[1];
+    for (int k = 0; k < R; ++k)
+      for (int r = 0; r < R; ++r) {
+        std::vector<int> w;
+        if (c >= st.ns) w.push_back(consumed[fi(r, k, c - st.ns)]);
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_SCRATCH, PL_U8, S_off(k, c)), false,
+                    {ref(r, PL_BUF_IN, PL_U8, (k * g.P + c * g.chunk) * g.es)}, g.clen(c) * g.es, w, staged[fi(r, k, c)]);
+      }
+    begin_role(em, 3, (uint64_t)R);
+    if (em.role) em.queues_per_rank = em.L->role_queues[3];
+    for (int i = 0; i < R; ++i)
+      for (int k = 0; k < R; ++k) {
+        const int r = (k + i) % R;  // source rank
+        em.chunk_op(PL_OP_COPY, k, 0, ref(k, PL_BUF_OUT, PL_U8, (r * g.P + c * g.chunk) * g.es), false,
+                    {ref(r, PL_BUF_SCRATCH, PL_U8, S_off(k, c))}, g.clen(c) * g.es, {staged[fi(r, k, c)]},
+                    consumed[fi(r, k, c)]);
+      }
+    em.queues_per_rank = q_all;
+  }
+  for (int r = 0; r < R; ++r) em.L->scratch_per_rank[r] = (uint64_t)R * st.ns * st.chunkB;
+}
+
 }  // namespace
 
 // Default knobs for sm_100a ("codesign policy", Sec. 3.2-3.3).  Called twice by the build:
@@ -471,6 +659,7 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
   if (n == 0) return fail(PL_ERR_INVALID_ARG, "count_per_rank is zero");
   const uint64_t bytes = n * es;
 
+  if (rq.staged && (rq.n_layers > 0 || rq.coll == PL_ALLTOALLV)) return fail(PL_ERR_UNSUPPORTED, "staging is offered for the four fixed-size direct collectives");
   if (rq.n_layers > 0) {
     if (rq.coll != PL_ALLREDUCE) return fail(PL_ERR_UNSUPPORTED, "layered schedules are all-reduce only");
     if (rq.algo != PL_ALGO_ONESHOT && rq.algo != PL_ALGO_DIRECT && rq.algo != PL_ALGO_DIRECT_FUSED)
@@ -485,7 +674,9 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
       Geo g = make_geo(R, dt, n * R, n, rq.chunk_bytes);
       for (int r = 0; r < R; ++r) { L->in_bytes[r] = bytes; L->out_bytes[r] = bytes * R; }
       L->message_bytes = bytes * R;
-      if (rq.algo == PL_ALGO_DIRECT) ag_direct(em, g);
+      if (rq.staged && rq.algo != PL_ALGO_DIRECT) return fail(PL_ERR_UNSUPPORTED, "staged schedules are direct only");
+      if (rq.staged) ag_direct_staged(em, g, rq.staging_bytes);
+      else if (rq.algo == PL_ALGO_DIRECT) ag_direct(em, g);
       else if (rq.algo == PL_ALGO_RING) ag_ring(em, g, false, nullptr);
       else return fail(PL_ERR_UNSUPPORTED, "all-gather supports direct and ring");
       return PL_OK;
@@ -496,7 +687,8 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
       Geo g = make_geo(R, dt, n, n / R, rq.chunk_bytes);
       for (int r = 0; r < R; ++r) L->in_bytes[r] = L->out_bytes[r] = bytes;
       L->message_bytes = bytes;
-      a2a_direct(em, g);
+      if (rq.staged) a2a_direct_staged(em, g, rq.staging_bytes);
+      else a2a_direct(em, g);
       return PL_OK;
     }
     case PL_REDUCE_SCATTER: {
@@ -504,7 +696,9 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
       Geo g = make_geo(R, dt, n, n / R, rq.chunk_bytes);
       for (int r = 0; r < R; ++r) { L->in_bytes[r] = bytes; L->out_bytes[r] = bytes / R; }
       L->message_bytes = bytes;
-      if (rq.algo == PL_ALGO_DIRECT) rs_direct(em, g);
+      if (rq.staged && rq.algo != PL_ALGO_DIRECT) return fail(PL_ERR_UNSUPPORTED, "staged schedules are direct only");
+      if (rq.staged) rs_direct_staged(em, g, rq.staging_bytes);
+      else if (rq.algo == PL_ALGO_DIRECT) rs_direct(em, g);
       else if (rq.algo == PL_ALGO_RING) rs_ring(em, g, false, nullptr);
       else return fail(PL_ERR_UNSUPPORTED, "reduce-scatter supports direct and ring");
       return PL_OK;
@@ -538,6 +732,11 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
         }
         return PL_OK;
       }
+      if (rq.staged) {
+        if (rq.algo != PL_ALGO_DIRECT) return fail(PL_ERR_UNSUPPORTED, "staged schedules are direct only");
+        ar_direct_staged(em, gp, rq.staging_bytes);
+        return PL_OK;
+      }
       switch (rq.algo) {
         case PL_ALGO_ONESHOT: ar_oneshot(em, gw, 0, 0, 0, nullptr); return PL_OK;
         case PL_ALGO_DIRECT: ar_direct(em, gp, 0, 0, 0, nullptr); return PL_OK;
@@ -565,14 +764,25 @@ void assign_queues(Lowered* L, int R, int n_queues) {
   const int per_rank = std::max(1, n_queues / R);
   std::vector<uint64_t> load((size_t)per_rank * R, 0);
   L->flag_need.assign(L->n_flags, 0);
+  // queue index ranges [lo, hi) inside a rank for each role (role 0 = all of them)
+  int lo[4] = {0, 0, 0, 0}, hi[4] = {per_rank, per_rank, per_rank, per_rank};
+  if (L->role_queues[1] + L->role_queues[2] + L->role_queues[3] == per_rank) {
+    int at = 0;
+    for (int i = 1; i < 4; ++i) {
+      lo[i] = at;
+      at += L->role_queues[i];
+      hi[i] = at;
+    }
+  }
   int topo = 0;
   for (HostOp& op : L->ops) {
     op.topo = topo++;
     uint64_t cost = op.count * elem_size(op.dst.dtype) * (op.bcast ? R : 1);
     for (const pl_ref_t& s : op.src) cost += op.count * elem_size(s.dtype);
     cost += 2048;  // fixed per-op overhead so that many tiny ops still spread out
-    int best = 0;
-    for (int j = 1; j < per_rank; ++j)
+    const int role = (op.role >= 0 && op.role < 4 && hi[op.role] > lo[op.role]) ? op.role : 0;
+    int best = lo[role];
+    for (int j = lo[role] + 1; j < hi[role]; ++j)
       if (load[(size_t)j * R + op.exec_rank] < load[(size_t)best * R + op.exec_rank]) best = j;
     load[(size_t)best * R + op.exec_rank] += cost;
     op.queue = best * R + op.exec_rank;
@@ -582,10 +792,6 @@ void assign_queues(Lowered* L, int R, int n_queues) {
 }
 
 namespace {
-struct Interval {
-  uint64_t lo, hi;
-  int op;
-};
 using Key = std::pair<int, int>;  // (buf kind, rank)
 }  // namespace
 
@@ -653,64 +859,120 @@ pl_status_t validate(const Lowered& L, int R, std::string* err) {
     for (const pl_ref_t& s : op.src)
       if (const char* m = check(s, limit(s))) return fail(m);
   }
-  // 4. every written byte written once; outputs fully covered
-  std::map<Key, std::vector<Interval>> writes;
+  // 4. memory hazards, replayed in topological order over a map of disjoint segments per
+  //    buffer.  Outputs: every byte written exactly once and fully covered.  Scratch (staging
+  //    slots may be reused within one execute): a write must happen after the previous write
+  //    of those bytes and after every read of that previous version.  Every read of bytes the
+  //    schedule writes must happen after that write.  "Happens after" = reachable through
+  //    wait edges (a wait on a flag orders the waiter after ALL of the flag's signallers) or
+  //    program order on one queue.
+  std::vector<std::vector<int>> signallers(L.n_flags);
+  for (size_t i = 0; i < n; ++i)
+    for (int f : {L.ops[i].signal, L.ops[i].signal2})
+      if (f >= 0) signallers[f].push_back((int)i);
+  std::vector<int> stamp(n, -1);
+  int query = 0;
+  auto happens_before = [&](int a, int x) -> bool {
+    if (a >= x) return false;
+    ++query;
+    std::vector<std::pair<int, int>> stack{{x, 0}};
+    stamp[x] = query;
+    size_t visited = 0;
+    while (!stack.empty()) {
+      auto [y, depth] = stack.back();
+      stack.pop_back();
+      const HostOp& oy = L.ops[y];
+      if (oy.queue == L.ops[a].queue && a < y) return true;
+      if (depth >= 6 || ++visited > 200000) continue;
+      for (int f : oy.waits)
+        for (int sgn : signallers[f]) {
+          if (sgn == a) return true;
+          if (sgn > a && stamp[sgn] != query) {
+            stamp[sgn] = query;
+            stack.push_back({sgn, depth + 1});
+          }
+        }
+    }
+    return false;
+  };
+  struct Seg {
+    uint64_t hi;
+    int writer;
+    std::vector<int> readers;
+  };
+  std::map<Key, std::map<uint64_t, Seg>> mem;
+  // split so that `at` is a segment boundary
+  auto split = [](std::map<uint64_t, Seg>& m, uint64_t at) {
+    auto it = m.upper_bound(at);
+    if (it == m.begin()) return;
+    --it;
+    if (it->first < at && at < it->second.hi) {
+      Seg right = it->second;
+      it->second.hi = at;
+      m[at] = right;
+    }
+  };
   for (size_t i = 0; i < n; ++i) {
     const HostOp& op = L.ops[i];
-    uint64_t b = op.count * elem_size(op.dst.dtype);
-    if (op.bcast) {
-      for (int r = 0; r < R; ++r) writes[{op.dst.buf, r}].push_back({op.dst.offset, op.dst.offset + b, (int)i});
-    } else {
-      writes[{op.dst.buf, op.dst.rank}].push_back({op.dst.offset, op.dst.offset + b, (int)i});
-    }
-  }
-  for (auto& kv : writes) {
-    auto& v = kv.second;
-    std::sort(v.begin(), v.end(), [](const Interval& a, const Interval& b) { return a.lo < b.lo; });
-    for (size_t i = 1; i < v.size(); ++i)
-      if (v[i].lo < v[i - 1].hi) {
-        std::snprintf(msg, sizeof msg, "ops %d and %d write overlapping bytes of buffer kind %d rank %d", v[i - 1].op,
-                      v[i].op, kv.first.first, kv.first.second);
-        return fail(msg);
+    for (const pl_ref_t& src : op.src) {
+      auto mit = mem.find({src.buf, src.rank});
+      if (mit == mem.end()) continue;
+      auto& m = mit->second;
+      const uint64_t lo = src.offset, hi = src.offset + op.count * elem_size(src.dtype);
+      auto it = m.upper_bound(lo);
+      if (it != m.begin()) --it;
+      for (; it != m.end() && it->first < hi; ++it) {
+        if (it->second.hi <= lo) continue;
+        const int w = it->second.writer;
+        bool direct = false;
+        for (int f : op.waits)
+          if (f == L.ops[w].signal || f == L.ops[w].signal2) direct = true;
+        if (!direct && !happens_before(w, (int)i)) {
+          std::snprintf(msg, sizeof msg, "op %zu reads bytes written by op %d without being ordered after it", i, w);
+          return fail(msg);
+        }
+        if (src.buf == PL_BUF_SCRATCH) it->second.readers.push_back((int)i);
       }
+    }
+    const uint64_t b = op.count * elem_size(op.dst.dtype);
+    for (int r = 0; r < R; ++r) {
+      if (!op.bcast && r != op.dst.rank) continue;
+      auto& m = mem[{op.dst.buf, r}];
+      const uint64_t lo = op.dst.offset, hi = lo + b;
+      split(m, lo);
+      split(m, hi);
+      auto it = m.lower_bound(lo);
+      while (it != m.end() && it->first < hi) {
+        if (op.dst.buf == PL_BUF_OUT) {
+          std::snprintf(msg, sizeof msg, "ops %d and %zu write overlapping bytes of the output of rank %d", it->second.writer, i, r);
+          return fail(msg);
+        }
+        if (!happens_before(it->second.writer, (int)i)) {
+          std::snprintf(msg, sizeof msg, "op %zu overwrites scratch written by op %d without being ordered after it", i, it->second.writer);
+          return fail(msg);
+        }
+        for (int rd : it->second.readers)
+          if (rd != (int)i && !happens_before(rd, (int)i)) {
+            std::snprintf(msg, sizeof msg, "op %zu overwrites scratch that op %d may still be reading", i, rd);
+            return fail(msg);
+          }
+        it = m.erase(it);
+      }
+      m[lo] = Seg{hi, (int)i, {}};
+    }
   }
   for (int r = 0; r < R; ++r) {
     uint64_t covered = 0;
-    auto it = writes.find({PL_BUF_OUT, r});
-    if (it != writes.end())
-      for (const Interval& iv : it->second) {
-        if (iv.lo != covered) break;
-        covered = iv.hi;
+    auto mit = mem.find({PL_BUF_OUT, r});
+    if (mit != mem.end())
+      for (const auto& kv : mit->second) {
+        if (kv.first != covered) break;
+        covered = kv.second.hi;
       }
     if (covered != L.out_bytes[r]) {
       std::snprintf(msg, sizeof msg, "output of rank %d is covered up to byte %llu of %llu", r,
                     (unsigned long long)covered, (unsigned long long)L.out_bytes[r]);
       return fail(msg);
-    }
-  }
-  // 5. reads of bytes the schedule writes must be ordered after the write: the reader waits
-  //    on a flag the writer signals, or both sit on one queue (program order)
-  for (size_t i = 0; i < n; ++i) {
-    const HostOp& op = L.ops[i];
-    for (const pl_ref_t& s : op.src) {
-      auto it = writes.find({s.buf, s.rank});
-      if (it == writes.end()) continue;
-      const auto& v = it->second;
-      uint64_t lo = s.offset, hi = s.offset + op.count * elem_size(s.dtype);
-      auto first = std::upper_bound(v.begin(), v.end(), lo, [](uint64_t x, const Interval& iv) { return x < iv.hi; });
-      for (auto w = first; w != v.end() && w->lo < hi; ++w) {
-        const HostOp& wr = L.ops[w->op];
-        bool ordered = false;
-        if (w->op < (int)i) {
-          for (int f : op.waits)
-            if (f == wr.signal || f == wr.signal2) ordered = true;
-          if (wr.queue == op.queue) ordered = true;
-        }
-        if (!ordered) {
-          std::snprintf(msg, sizeof msg, "op %zu reads bytes written by op %d without a wait edge", i, w->op);
-          return fail(msg);
-        }
-      }
     }
   }
   return PL_OK;

@@ -290,3 +290,40 @@ def test_bounded_wait_reports_timeout_and_recovers(dp):
         compare_reduce(outs, ref, "i32")
     finally:
         ses.close()
+
+
+# ---- staged schedules (ordinary application buffers, cyclic staging) -----------------------
+@pytest.mark.parametrize("dp", DATAPATHS)
+@pytest.mark.parametrize("dtype", ["bf16", "i32"])
+def test_staged_direct_collectives(dp, dtype):
+    R = 8
+    es = 2 if dtype == "bf16" else 4
+    part = 300 * 1024 + 48                      # 5 chunks of 64 KiB (last one short)
+    n = R * part // es
+    x = gen.rank_inputs(R, n, dtype, seed=9)
+    ses = Session(R, dtype)
+    try:
+        for cap_chunks in (2, 1000):            # 2 slots per partition: every slot is reused; 1000: never
+            kw = dict(flags=B.PL_OPT_STAGED, staging_bytes=cap_chunks * R * 65536, datapath=dp)
+            s = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, n, 65536, **kw)
+            outs, info = ses.execute(s, x, repeats=3)
+            compare_reduce(outs, oracle.allreduce(x, dtype), dtype)
+            if cap_chunks == 2:
+                assert info.scratch_bytes == R * (R * 2 + 2) * 65536
+            s = ses.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, 65536, **kw)
+            outs, _ = ses.execute(s, x, repeats=2)
+            compare_reduce(outs, oracle.reduce_scatter(x, dtype), dtype)
+            s = ses.build(B.PL_ALLTOALL, B.PL_ALGO_DIRECT, n, 65536, **kw)
+            outs, _ = ses.execute(s, x, repeats=2)
+            ref = oracle.alltoall(x)
+            for r in range(R):
+                assert np.array_equal(outs[r], ref[r].view(np.uint8))
+            contrib = [a[: n // R].copy() for a in x]
+            s = ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 65536,
+                          flags=B.PL_OPT_STAGED, staging_bytes=cap_chunks * 65536, datapath=dp)
+            outs, _ = ses.execute(s, contrib, repeats=2)
+            ref = oracle.allgather(contrib)
+            for r in range(R):
+                assert np.array_equal(outs[r], ref[r].view(np.uint8))
+    finally:
+        ses.close()

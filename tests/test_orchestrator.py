@@ -291,3 +291,112 @@ def test_queues_are_rank_owned_and_balanced():
         assert max(load.values()) <= 1.25 * min(load.values())
     finally:
         pl.close()
+
+
+# ---- staged schedules: ordinary application buffers, cyclic staging, role-specialised queues ----
+@pytest.mark.parametrize("R", [2, 3, 8])
+@pytest.mark.parametrize("cap_chunks", [1, 2, 100])
+def test_staged_collectives_replay_to_oracle(R, cap_chunks):
+    chunk = 48
+    for dtype in ("i32", "bf16"):
+        es = B.DTYPE_SIZE[DT[dtype]]
+        n = R * (16 // es) * 13                     # 13 vectors per partition: 5 chunks of 48 B, last one short
+        x = gen.rank_inputs(R, n, dtype, seed=R + 1)
+        pl = Planner(R, dtype)
+        try:
+            kw = dict(flags=B.PL_OPT_STAGED, staging_bytes=cap_chunks * R * chunk, slice_bytes=32, n_ctas=6 * R)
+            s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, n, chunk, **kw)
+            st, msg = B.pl_schedule_validate(s)
+            assert st == B.PL_OK, msg
+            info = B.pl_schedule_info(s)
+            ops = B.pl_schedule_dump(s)
+            # nothing but the staging copies reads an input, nothing but the rank itself reads it
+            for o in ops:
+                for k in range(o.n_src):
+                    if o.src[k].buf == B.PL_BUF_IN:
+                        assert o.kind == B.PL_OP_COPY and o.src[k].rank == o.exec_rank and o.dst.buf == B.PL_BUF_SCRATCH
+                if o.dst.buf == B.PL_BUF_OUT:
+                    assert o.dst.rank == o.exec_rank
+            if cap_chunks < 5:
+                # cyclic staging: scratch is smaller than the message and some stage op waits
+                assert info.scratch_bytes < R * (n * es + n * es // R)
+                assert any(o.n_wait > 0 and o.dst.buf == B.PL_BUF_SCRATCH and o.kind == B.PL_OP_COPY for o in ops)
+            for seed in (0, 1, 2):
+                compare_reduce(interp_run(ops, info, R, x, seed=seed), oracle.allreduce(x, dtype), dtype)
+            s = pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, chunk, **kw)
+            assert B.pl_schedule_validate(s)[0] == B.PL_OK
+            compare_reduce(interp_run(B.pl_schedule_dump(s), B.pl_schedule_info(s), R, x, seed=3),
+                           oracle.reduce_scatter(x, dtype), dtype)
+            kw_ag = dict(kw, staging_bytes=cap_chunks * chunk)
+            s = pl.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n, chunk, **kw_ag)
+            assert B.pl_schedule_validate(s)[0] == B.PL_OK
+            outs = interp_run(B.pl_schedule_dump(s), B.pl_schedule_info(s), R, x, seed=4)
+            ref = oracle.allgather(x)
+            for r in range(R):
+                assert np.array_equal(outs[r], ref[r].view(np.uint8))
+            s = pl.build(B.PL_ALLTOALL, B.PL_ALGO_DIRECT, n, chunk, **kw)
+            assert B.pl_schedule_validate(s)[0] == B.PL_OK
+            outs = interp_run(B.pl_schedule_dump(s), B.pl_schedule_info(s), R, x, seed=5)
+            ref = oracle.alltoall(x)
+            for r in range(R):
+                assert np.array_equal(outs[r], ref[r].view(np.uint8))
+        finally:
+            pl.close()
+
+
+def test_staged_roles_get_their_own_queues():
+    R = 8
+    pl = Planner(R, "bf16")
+    try:
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 8 << 20, 1 << 20, flags=B.PL_OPT_STAGED, n_ctas=144)
+        ops = B.pl_schedule_dump(s)
+        kinds = {}
+        for o in ops:
+            role = "stage" if o.dst.buf == B.PL_BUF_SCRATCH and o.kind == B.PL_OP_COPY else \
+                   "reduce" if o.kind == B.PL_OP_REDUCE else "gather"
+            kinds.setdefault(o.queue, set()).add(role)
+        assert all(len(v) == 1 for v in kinds.values())       # a queue serves one role only
+        per_role = {}
+        for q, v in kinds.items():
+            if q % R == 0:
+                per_role[next(iter(v))] = per_role.get(next(iter(v)), 0) + 1
+        assert sum(per_role.values()) == 18 and per_role["stage"] >= 6 and per_role["gather"] >= 6 and per_role["reduce"] >= 3
+    finally:
+        pl.close()
+
+
+def test_staged_rejections():
+    pl = Planner(4, "bf16")
+    try:
+        for coll, algo in ((B.PL_ALLREDUCE, B.PL_ALGO_RING), (B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT), (B.PL_REDUCE_SCATTER, B.PL_ALGO_RING)):
+            with pytest.raises(B.PurlinError) as e:
+                pl.build(coll, algo, 4096, 256, flags=B.PL_OPT_STAGED)
+            assert e.value.status == B.PL_ERR_UNSUPPORTED
+    finally:
+        pl.close()
+
+
+def test_validator_notices_a_dropped_wait_edge():
+    pl = Planner(4, "i32")
+    try:
+        n = 4 * 4 * 6
+        # a ring: dropping the wait of a hop leaves a read of the travelling partial unordered
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 32)
+        assert B.pl_schedule_validate(s)[0] == B.PL_OK
+        victim = next(o.topo for o in B.pl_schedule_dump(s) if o.n_wait > 0)
+        B.pl_schedule_debug_drop_wait(s, victim)
+        st, msg = B.pl_schedule_validate(s)
+        assert st == B.PL_ERR_INVALID_SCHEDULE and "without being ordered" in msg
+        # cyclic staging: dropping the "slot is free again" wait of a stage op is a write-after-read hazard
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, n, 32, flags=B.PL_OPT_STAGED, staging_bytes=4 * 32)
+        assert B.pl_schedule_validate(s)[0] == B.PL_OK
+        # one slot of 32 bytes per partition: the slot of partition k starts at byte 32*k; take a
+        # stage op whose consumer is another rank (on the same rank queue order would still protect it)
+        victim = next(o.topo for o in B.pl_schedule_dump(s)
+                      if o.n_wait > 0 and o.kind == B.PL_OP_COPY and o.dst.buf == B.PL_BUF_SCRATCH
+                      and o.dst.offset // 32 != o.exec_rank)
+        B.pl_schedule_debug_drop_wait(s, victim)
+        st, msg = B.pl_schedule_validate(s)
+        assert st == B.PL_ERR_INVALID_SCHEDULE and "overwrites scratch" in msg
+    finally:
+        pl.close()
