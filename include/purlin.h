@@ -82,7 +82,9 @@ typedef enum {
   PL_REDUCE_SCATTER = 1,
   PL_ALLGATHER = 2,
   PL_ALLTOALL = 3,
-  PL_ALLTOALLV = 4
+  PL_ALLTOALLV = 4,
+  PL_ALLGATHERV = 5,      /* copy, packedV -> scatteredV: rank p contributes n[p] elements */
+  PL_REDUCE_SCATTERV = 6  /* reduce, scatteredV -> packedV: rank k receives partition k of n[k] elements */
 } pl_collective_t;
 
 /* Algorithms.
@@ -249,9 +251,13 @@ pl_status_t pl_schedule_build(pl_comm_t comm, pl_collective_t coll, pl_algo_t al
                               size_t count_per_rank, size_t chunk_bytes,
                               const pl_sched_opts_t* opts, pl_schedule_t* out);
 
-/* Variable-size all-to-all: counts is a HOST array R*R, row-major [src][dst], in elements.
- * counts[p][r]*elem_size must be a multiple of 16 (PL_ERR_ALIGNMENT).  Only
- * PL_ALLTOALLV with PL_ALGO_DIRECT. */
+/* Variable-size collectives (Listing 1's V namings; partition sizes given at run time).
+ * counts is a HOST array in elements:
+ *   PL_ALLTOALLV        R*R entries, row-major [src][dst];
+ *   PL_ALLGATHERV       R entries: n[p] = contribution of rank p (output = their concatenation);
+ *   PL_REDUCE_SCATTERV  R entries: n[k] = partition k of every rank's input, reduced to rank k.
+ * Every size times elem_size must be a multiple of 16 (PL_ERR_ALIGNMENT); zero is allowed.
+ * PL_ALGO_DIRECT only.  The reported message size is the total T (as the paper plots it). */
 pl_status_t pl_schedule_build_v(pl_comm_t comm, pl_collective_t coll, pl_algo_t algo,
                                 const size_t* counts, size_t chunk_bytes,
                                 const pl_sched_opts_t* opts, pl_schedule_t* out);

@@ -9,7 +9,8 @@
  * leg may call into this file.
  *
  * Definitions follow the paper's statement of the collective contracts
- * (Sec. 2, "Stable communication semantics"), its layouts (Sec. 3.1: packed,
+ * (Sec. 2, "Stable communication semantics", including the V variants whose partition sizes
+ * are given at run time), its layouts (Sec. 3.1: packed,
  * scattered, transposed and their V variants), and its reduction rule
  * (Sec. 3.3, Eq. "rank-order": one accumulator per element, starting from zero,
  * adding rank 0, 1, ..., n-1).  The MoE dispatch/combine pair is the expert-
@@ -91,6 +92,50 @@ int orc_alltoallv(int R, const uint64_t *counts, const void *const *in, void *co
 #pragma omp parallel for schedule(static)
       for (size_t i = 0; i < n; ++i) d[i] = s[i];
     }
+  return 0;
+}
+
+/* AllGatherV (packedV -> scatteredV): rank p contributes n[p] bytes; every rank's output is
+ * the contributions in rank order: out_r[off_p + i] = in_p[i], off_p = sum_{q<p} n[q]. */
+int orc_allgatherv(int R, const uint64_t *n_bytes, const void *const *in, void *const *out) {
+  for (int r = 0; r < R; ++r) {
+    size_t off = 0;
+    for (int p = 0; p < R; ++p) {
+      const uint8_t *s = (const uint8_t *)in[p];
+      uint8_t *d = (uint8_t *)out[r] + off;
+      for (size_t i = 0; i < n_bytes[p]; ++i) d[i] = s[i];
+      off += n_bytes[p];
+    }
+  }
+  return 0;
+}
+
+/* ReduceScatterV (scatteredV -> packedV): every rank holds T = sum n[k] elements cut into
+ * partitions of n[k] elements; rank k receives out_k[i] = sum_p in_p[off_k + i], i < n[k]. */
+int orc_reduce_scatterv_f64(int R, int dtype, const uint64_t *n_elems, const void *const *in, double *const *out) {
+  if (dtype != ORC_BF16 && dtype != ORC_F32) return 1;
+  size_t off = 0;
+  for (int k = 0; k < R; ++k) {
+    for (size_t i = 0; i < n_elems[k]; ++i) {
+      double acc = 0.0;
+      for (int p = 0; p < R; ++p) acc += load_as_f64(in[p], dtype, off + i);
+      out[k][i] = acc;
+    }
+    off += n_elems[k];
+  }
+  return 0;
+}
+
+int orc_reduce_scatterv_i32(int R, const uint64_t *n_elems, const void *const *in, int32_t *const *out) {
+  size_t off = 0;
+  for (int k = 0; k < R; ++k) {
+    for (size_t i = 0; i < n_elems[k]; ++i) {
+      uint32_t acc = 0;
+      for (int p = 0; p < R; ++p) acc += ((const uint32_t *)in[p])[off + i];
+      out[k][i] = (int32_t)acc;
+    }
+    off += n_elems[k];
+  }
   return 0;
 }
 

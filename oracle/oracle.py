@@ -88,6 +88,32 @@ def alltoallv(inputs, counts_elems):
     return [oc[:o.size] for oc, o in zip(outs_c, outs)]
 
 
+def allgatherv(inputs):
+    """inputs[p]: rank p's contribution (sizes may differ, may be empty) -> out[r] = concatenation."""
+    R = len(inputs)
+    nb = np.array([a.nbytes for a in inputs], dtype=np.uint64)
+    total = sum(a.size for a in inputs)
+    outs = [np.zeros(max(1, total), dtype=inputs[0].dtype) for _ in range(R)]
+    ins_c = [a if a.size else np.zeros(1, dtype=a.dtype) for a in inputs]
+    _check(lib().orc_allgatherv(R, nb.ctypes.data_as(ctypes.c_void_p), _ptrs(ins_c), _ptrs(outs)), "allgatherv")
+    return [o[:total] for o in outs]
+
+
+def reduce_scatterv(inputs, sizes, dtype):
+    """inputs[p]: T = sum(sizes) elements; returns out[k] of sizes[k] elements (fp64 or int32)."""
+    R = len(inputs)
+    ne = np.array(sizes, dtype=np.uint64)
+    assert inputs[0].size == int(ne.sum())
+    if dtype == "i32":
+        outs = [np.zeros(max(1, int(k)), dtype=np.int32) for k in sizes]
+        _check(lib().orc_reduce_scatterv_i32(R, ne.ctypes.data_as(ctypes.c_void_p), _ptrs(inputs), _ptrs(outs)), "rsv_i32")
+    else:
+        outs = [np.zeros(max(1, int(k)), dtype=np.float64) for k in sizes]
+        _check(lib().orc_reduce_scatterv_f64(R, _dtype_code(inputs[0], dtype), ne.ctypes.data_as(ctypes.c_void_p),
+                                             _ptrs(inputs), _ptrs(outs)), "rsv_f64")
+    return [o[: int(k)] for o, k in zip(outs, sizes)]
+
+
 def _dtype_code(a, dtype):
     if dtype == "bf16":
         assert a.dtype == np.uint16

@@ -137,6 +137,26 @@ class Bench:
         del d_in, d_out
         return rec
 
+    def collective_v(self, cfg, R, dtype, coll, counts, chunk, iters=20, **kw):
+        """Variable-size collectives (counts as pl_schedule_build_v takes them)."""
+        comm = B.pl_comm_create(R, dtype)
+        s = B.pl_schedule_build_v(comm, coll, B.PL_ALGO_DIRECT, counts, chunk, B.make_opts(**kw))
+        info = B.pl_schedule_info(s)
+        d_in = [_fill(int(info.in_bytes[r]), r) for r in range(R)]
+        d_out = [torch.empty(max(16, int(info.out_bytes[r])), dtype=torch.uint8, device="cuda") for r in range(R)]
+        bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                           [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
+        p50, _, _ = _time(lambda: B.pl_execute(s, bufs, self.stream), iters, per_call_events=True)
+        graph_us = _time_graph(lambda h: B.pl_execute(s, bufs, h)) if info.message_bytes <= 2 * MIB else None
+        sched_bytes = info.bytes_read + info.bytes_written
+        self.emit({"cfg": cfg, "coll": int(coll), "algo": "direct", "R": R, "message_bytes": int(info.message_bytes),
+                   "us": p50, "us_graph128": graph_us, "eff_gbs": info.message_bytes / p50 / 1e3,
+                   "sched_gbs": sched_bytes / p50 / 1e3, "hbm_frac_measured": sched_bytes / p50 / 1e3 / self.peak,
+                   "n_ops": int(info.n_ops), "grid": int(info.grid), "datapath": int(info.datapath),
+                   "status": int(B.pl_comm_status(comm).code)})
+        B.pl_schedule_destroy(s)
+        B.pl_comm_destroy(comm)
+
     def moe(self, cfg, R=8, T=4096, H=7168, E=256, K=8, identity=False, iters=10):
         idx, gates = gen.moe_routing(R, T, E, K, identity_perm=identity)
         counts = np.zeros((R, R), np.int64)
@@ -191,7 +211,7 @@ def probe(b):
 
 
 def main(args=None):
-    which = os.environ.get("PL_SUITE", "probe,c1,c2,staged,c3,c4,c5").split(",")
+    which = os.environ.get("PL_SUITE", "probe,c1,c2,staged,varlen,c3,c4,c5").split(",")
     out = os.environ.get("PL_SUITE_OUT")  # optional file that receives the JSON lines too
     if out and os.path.dirname(out):
         os.makedirs(os.path.dirname(out), exist_ok=True)
@@ -220,6 +240,15 @@ def main(args=None):
             for size in (MIB, 16 * MIB, 64 * MIB, 256 * MIB):
                 b.collective("staged-AR cap=%d" % cap, 8, B.PL_BF16, B.PL_ALLREDUCE, "direct", size // 2,
                              max(16, min(MIB, size // 8)), iters=10, **kw)
+    if "varlen" in which:
+        # the paper's variable-length workload (Appendix C): Zipf(s=0.125) split of T bytes over
+        # 8 ranks; all-to-all-v rotates the split per rank so every rank sends and receives T
+        for T in (64 * 1024, MIB, 64 * MIB, 1024 * MIB):
+            n = (gen.zipf_split(T) // 2).tolist()
+            b.collective_v("AGV", 8, B.PL_BF16, B.PL_ALLGATHERV, n, MIB)
+            b.collective_v("RSV", 8, B.PL_BF16, B.PL_REDUCE_SCATTERV, n, MIB)
+            if T <= 256 * MIB:
+                b.collective_v("A2AV", 8, B.PL_BF16, B.PL_ALLTOALLV, (gen.alltoallv_counts_bytes(T) // 2).tolist(), MIB)
     if "c3" in which:
         for lg in range(12, 29):
             size = 1 << lg

@@ -25,7 +25,7 @@ PL_OK, PL_ERR_INVALID_ARG, PL_ERR_UNSUPPORTED, PL_ERR_ALIGNMENT, PL_ERR_OOM, PL_
 PL_BF16, PL_F32, PL_I32, PL_U8, PL_F32X2 = range(5)
 DTYPE_SIZE = {PL_BF16: 2, PL_F32: 4, PL_I32: 4, PL_U8: 1, PL_F32X2: 8}
 # collectives
-PL_ALLREDUCE, PL_REDUCE_SCATTER, PL_ALLGATHER, PL_ALLTOALL, PL_ALLTOALLV = range(5)
+PL_ALLREDUCE, PL_REDUCE_SCATTER, PL_ALLGATHER, PL_ALLTOALL, PL_ALLTOALLV, PL_ALLGATHERV, PL_REDUCE_SCATTERV = range(7)
 # algorithms
 PL_ALGO_RING, PL_ALGO_TREE, PL_ALGO_DIRECT, PL_ALGO_ONESHOT, PL_ALGO_DIRECT_FUSED = range(5)
 # op kinds / buffer kinds / datapaths
@@ -217,7 +217,7 @@ def pl_schedule_build(comm, coll, algo, count_per_rank, chunk_bytes, opts=None):
 
 
 def pl_schedule_build_v(comm, coll, algo, counts, chunk_bytes, opts=None):
-    flat = [int(v) for row in counts for v in row]
+    flat = [int(v) for row in counts for v in (row if hasattr(row, "__len__") else [row])]
     arr = (C.c_size_t * len(flat))(*flat)
     h = C.c_void_p()
     _check(load().pl_schedule_build_v(comm, coll, algo, arr, chunk_bytes,

@@ -328,7 +328,7 @@ pl_status_t pl_comm_reset(pl_comm_t comm, void* stream) {
 
 pl_status_t pl_schedule_build(pl_comm_t comm, pl_collective_t coll, pl_algo_t algo, size_t count_per_rank,
                               size_t chunk_bytes, const pl_sched_opts_t* opts, pl_schedule_t* out) {
-  if (coll == PL_ALLTOALLV) return PL_ERR_INVALID_ARG;
+  if (coll == PL_ALLTOALLV || coll == PL_ALLGATHERV || coll == PL_REDUCE_SCATTERV) return PL_ERR_INVALID_ARG;
   BuildRequest rq{};
   rq.coll = coll;
   rq.algo = algo;
@@ -340,8 +340,8 @@ pl_status_t pl_schedule_build(pl_comm_t comm, pl_collective_t coll, pl_algo_t al
 pl_status_t pl_schedule_build_v(pl_comm_t comm, pl_collective_t coll, pl_algo_t algo, const size_t* counts,
                                 size_t chunk_bytes, const pl_sched_opts_t* opts, pl_schedule_t* out) {
   if (!comm || !counts) return PL_ERR_INVALID_ARG;
-  if (coll != PL_ALLTOALLV) return PL_ERR_UNSUPPORTED;
-  std::vector<uint64_t> c((size_t)comm->R * comm->R);
+  if (coll != PL_ALLTOALLV && coll != PL_ALLGATHERV && coll != PL_REDUCE_SCATTERV) return PL_ERR_UNSUPPORTED;
+  std::vector<uint64_t> c(coll == PL_ALLTOALLV ? (size_t)comm->R * comm->R : (size_t)comm->R);
   for (size_t i = 0; i < c.size(); ++i) c[i] = counts[i];
   BuildRequest rq{};
   rq.coll = coll;

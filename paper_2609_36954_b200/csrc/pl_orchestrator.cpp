@@ -206,6 +206,39 @@ void a2av_direct(Emitter& em, int R, int dtype, const uint64_t* counts, uint64_t
       }
 }
 
+// reduce-scatter-v / all-gather-v: the fixed-size rules with run-time partition sizes n[k]
+// (offsets are prefix sums, Sec. 3.1 "V variants").
+void rsv_direct(Emitter& em, int R, int dtype, const uint64_t* n, uint64_t chunk_bytes) {
+  const int es = elem_size(dtype);
+  const uint64_t chunk = std::max<uint64_t>(16 / es, chunk_bytes / es);
+  uint64_t max_n = 0;
+  std::vector<uint64_t> off(R, 0);
+  for (int k = 0; k < R; ++k) { max_n = std::max(max_n, n[k]); if (k) off[k] = off[k - 1] + n[k - 1]; }
+  for (uint64_t b = 0; b < max_n; b += chunk)
+    for (int k = 0; k < R; ++k) {
+      if (b >= n[k]) continue;
+      std::vector<pl_ref_t> src;
+      for (int p = 0; p < R; ++p) src.push_back(ref(p, PL_BUF_IN, dtype, (off[k] + b) * es));
+      em.chunk_op(PL_OP_REDUCE, k, 0, ref(k, PL_BUF_OUT, dtype, b * es), false, src, std::min(chunk, n[k] - b), {}, -1);
+    }
+}
+
+void agv_direct(Emitter& em, int R, int dtype, const uint64_t* n, uint64_t chunk_bytes) {
+  const int es = elem_size(dtype);
+  const uint64_t chunk = std::max<uint64_t>(16, chunk_bytes);
+  uint64_t max_b = 0;
+  std::vector<uint64_t> off(R, 0);
+  for (int p = 0; p < R; ++p) { max_b = std::max(max_b, n[p] * es); if (p) off[p] = off[p - 1] + n[p - 1] * es; }
+  for (uint64_t b = 0; b < max_b; b += chunk)
+    for (int i = 0; i < R; ++i)
+      for (int r = 0; r < R; ++r) {
+        const int p = (r + i) % R;
+        if (b >= n[p] * es) continue;
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, off[p] + b), false, {ref(p, PL_BUF_IN, PL_U8, b)},
+                    std::min(chunk, n[p] * es - b), {}, -1);
+      }
+}
+
 // all-reduce, one-shot: every rank reduces the whole message from all R inputs.
 void ar_oneshot(Emitter& em, const Geo& g, int layer, uint64_t in_off, uint64_t out_off, const LayerEdges* le) {
   // g.P == g.n here: the "partition" is the whole message, chunked.
@@ -590,13 +623,15 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
   uint64_t msg = rq.count_per_rank * es;
   if (rq.counts_v) {
     msg = 0;
-    for (int i = 0; i < rq.R * rq.R; ++i) msg += rq.counts_v[i] * es;
-    msg /= rq.R;
+    const int entries = rq.coll == PL_ALLTOALLV ? rq.R * rq.R : rq.R;
+    for (int i = 0; i < entries; ++i) msg += rq.counts_v[i] * es;
+    if (rq.coll == PL_ALLTOALLV) msg /= rq.R;
   }
   if (rq.coll == PL_ALLGATHER) msg *= rq.R;
   // bytes of all ranks' inputs and outputs: decides whether the working set lives in L2
   uint64_t footprint = 2 * (uint64_t)rq.R * msg;
-  if (rq.coll == PL_REDUCE_SCATTER || rq.coll == PL_ALLGATHER) footprint = (uint64_t)(rq.R + 1) * msg;
+  if (rq.coll == PL_REDUCE_SCATTER || rq.coll == PL_ALLGATHER || rq.coll == PL_REDUCE_SCATTERV || rq.coll == PL_ALLGATHERV)
+    footprint = (uint64_t)(rq.R + 1) * msg;
   if (rq.coll == PL_ALLTOALLV) footprint = 2 * (uint64_t)rq.R * msg;
   // Register path while the working set is L2 sized (and for layered latency schedules);
   // bulk-copy ring once it has to stream from HBM.  Measured crossover on B200: all-reduce of
@@ -611,7 +646,7 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
     const int full = std::max(rq.R, max_resident_ctas / rq.R * rq.R);
     // queues a rank can keep busy: one per 16 KiB of what it produces
     uint64_t per_rank_out = msg;
-    if (rq.coll == PL_REDUCE_SCATTER) per_rank_out = msg / rq.R;
+    if (rq.coll == PL_REDUCE_SCATTER || rq.coll == PL_REDUCE_SCATTERV) per_rank_out = msg / rq.R;
     const uint64_t unit = p.slice_bytes ? p.slice_bytes : 16384;
     uint64_t want = std::max<uint64_t>(1, (per_rank_out + unit - 1) / unit) * rq.R;
     p.n_ctas = (int)std::min<uint64_t>(full, std::max<uint64_t>(rq.R, want));
@@ -636,6 +671,26 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
   em.queues_per_rank = std::max(1, rq.pol.n_ctas / R);
   L->n_layers = 1;
 
+  if (rq.coll == PL_ALLGATHERV || rq.coll == PL_REDUCE_SCATTERV) {
+    if (rq.algo != PL_ALGO_DIRECT) return fail(PL_ERR_UNSUPPORTED, "V collectives are direct only");
+    if (rq.staged) return fail(PL_ERR_UNSUPPORTED, "staging is offered for the four fixed-size direct collectives");
+    if (!rq.counts_v) return fail(PL_ERR_INVALID_ARG, "sizes missing");
+    if (rq.coll == PL_REDUCE_SCATTERV && dt == PL_U8) return fail(PL_ERR_UNSUPPORTED, "bytes cannot be reduced");
+    uint64_t total = 0;
+    for (int k = 0; k < R; ++k) {
+      if ((rq.counts_v[k] * es) % 16) return fail(PL_ERR_ALIGNMENT, "every partition must be a multiple of 16 bytes");
+      total += rq.counts_v[k] * es;
+    }
+    for (int r = 0; r < R; ++r) {
+      L->in_bytes[r] = rq.coll == PL_ALLGATHERV ? rq.counts_v[r] * es : total;
+      L->out_bytes[r] = rq.coll == PL_ALLGATHERV ? total : rq.counts_v[r] * es;
+    }
+    L->message_bytes = total;
+    em.phase_chunks = 0;
+    if (rq.coll == PL_ALLGATHERV) agv_direct(em, R, dt, rq.counts_v, rq.chunk_bytes);
+    else rsv_direct(em, R, dt, rq.counts_v, rq.chunk_bytes);
+    return PL_OK;
+  }
   if (rq.coll == PL_ALLTOALLV) {
     if (rq.algo != PL_ALGO_DIRECT) return fail(PL_ERR_UNSUPPORTED, "all-to-all-v is direct only");
     if (!rq.counts_v) return fail(PL_ERR_INVALID_ARG, "counts missing");

@@ -39,8 +39,8 @@ class Session:
         self.scheds.append(s)
         return s
 
-    def build_v(self, counts, chunk, **kw):
-        s = B.pl_schedule_build_v(self.comm, B.PL_ALLTOALLV, B.PL_ALGO_DIRECT, counts, chunk,
+    def build_v(self, counts, chunk, coll=B.PL_ALLTOALLV, **kw):
+        s = B.pl_schedule_build_v(self.comm, coll, B.PL_ALGO_DIRECT, counts, chunk,
                                   B.make_opts(**kw) if kw else None)
         self.scheds.append(s)
         return s

@@ -327,3 +327,35 @@ def test_staged_direct_collectives(dp, dtype):
                 assert np.array_equal(outs[r], ref[r].view(np.uint8))
     finally:
         ses.close()
+
+
+# ---- V variants with the paper's Zipf(0.125) split ------------------------------------------
+@pytest.mark.parametrize("dp", DATAPATHS)
+@pytest.mark.parametrize("dtype", ["bf16", "i32"])
+def test_allgatherv_and_reduce_scatterv(dp, dtype):
+    R = 8
+    es = 2 if dtype == "bf16" else 4
+    for sizes_b in (gen.zipf_split(4 << 20), np.array([0, 160, 65536 + 16, 0, 48, 300000 // 16 * 16, 16, 1024])):
+        sizes = (np.asarray(sizes_b) // es).tolist()
+        total = sum(sizes)
+        x = gen.rank_inputs(R, total, dtype, seed=13)
+        ses = Session(R, dtype)
+        try:
+            s = ses.build_v(sizes, 65536, coll=B.PL_REDUCE_SCATTERV, datapath=dp)
+            outs, info = ses.execute(s, x, repeats=2)
+            assert info.message_bytes == total * es
+            ref = oracle.reduce_scatterv(x, sizes, dtype)
+            for r in range(R):
+                assert outs[r].size == sizes[r] * es
+                if dtype == "i32":
+                    assert np.array_equal(outs[r].view(np.int32), ref[r])
+                elif sizes[r]:
+                    check_float(as_f64(outs[r], dtype), ref[r], dtype)
+            contrib = [x[p][: sizes[p]].copy() for p in range(R)]
+            s = ses.build_v(sizes, 65536, coll=B.PL_ALLGATHERV, datapath=dp)
+            outs, _ = ses.execute(s, contrib, repeats=2)
+            ref = oracle.allgatherv(contrib)
+            for r in range(R):
+                assert np.array_equal(outs[r], ref[r].view(np.uint8))
+        finally:
+            ses.close()

@@ -307,3 +307,44 @@ def test_moe_combine_identity_constant_and_onehot():
         y2.append(rows)
     out = oracle.moe_combine(y2, idx, d["pos"], g2, E, H)
     assert np.all(out[0] == 0.5 * 1 + 0.25 * 2 + 0.125 * 3 + 0.125 * 4)
+
+
+# ----------------------------------------------------------------------------- #
+# V variants of all-gather and reduce-scatter
+# ----------------------------------------------------------------------------- #
+def test_allgatherv_is_ragged_concatenation():
+    sizes = [5, 0, 12, 1, 7]
+    x = [(np.arange(n) + 100 * p).astype(np.int32) for p, n in enumerate(sizes)]
+    out = oracle.allgatherv(x)
+    want = np.concatenate(x)
+    for r in range(len(sizes)):
+        assert np.array_equal(out[r], want)
+    # equal sizes reduce to the fixed-size collective
+    y = inputs.rank_coded_bytes(4, 48)
+    a, b = oracle.allgatherv(y), oracle.allgather(y)
+    for r in range(4):
+        assert np.array_equal(a[r], b[r])
+
+
+def test_reduce_scatterv_closed_form_uniform_case_and_zipf_sizes():
+    R = 8
+    sizes_bytes = inputs.zipf_split(8192)                 # the paper's split: 128-byte units 9 9 8 8 8 8 7 7
+    sizes = (sizes_bytes // 4).tolist()
+    n = sum(sizes)
+    x = inputs.rank_coded_i32(R, n)                       # x_p[j] = p*n + j
+    out = oracle.reduce_scatterv(x, sizes, "i32")
+    off = 0
+    for k in range(R):
+        i = np.arange(sizes[k], dtype=np.int64)
+        assert np.array_equal(out[k].astype(np.int64), R * (off + i) + n * R * (R - 1) // 2)
+        off += sizes[k]
+    # uniform sizes: identical to reduce-scatter; a zero-size partition yields an empty output
+    xf = inputs.rank_inputs(4, 4 * 24, "bf16", seed=8)
+    a, b = oracle.reduce_scatterv(xf, [24] * 4, "bf16"), oracle.reduce_scatter(xf, "bf16")
+    for r in range(4):
+        assert np.array_equal(a[r], b[r])
+    c = oracle.reduce_scatterv(xf, [40, 0, 32, 24], "bf16")
+    full = oracle.allreduce(xf, "bf16")[0]
+    assert c[1].size == 0 and np.array_equal(c[2], full[40:72]) and np.array_equal(c[3], full[72:96])
+    # gathering what the V reduce-scatter scattered rebuilds the all-reduce (paper's composition identity)
+    assert np.array_equal(np.concatenate(c), full)

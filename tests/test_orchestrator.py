@@ -400,3 +400,52 @@ def test_validator_notices_a_dropped_wait_edge():
         assert st == B.PL_ERR_INVALID_SCHEDULE and "overwrites scratch" in msg
     finally:
         pl.close()
+
+
+# ---- V variants of all-gather / reduce-scatter ---------------------------------------------
+@pytest.mark.parametrize("R", [2, 5, 8])
+def test_allgatherv_reduce_scatterv_replay(R):
+    rng = np.random.default_rng(R)
+    sizes = (rng.integers(0, 6, size=R) * 8).tolist()      # elements; zero-size partitions included
+    sizes[0] = 40
+    total = sum(sizes)
+    for dtype in ("i32", "bf16"):
+        es = B.DTYPE_SIZE[DT[dtype]]
+        pl = Planner(R, dtype)
+        try:
+            x = gen.rank_inputs(R, total, dtype, seed=3)
+            s = B.pl_schedule_build_v(pl.comm, B.PL_REDUCE_SCATTERV, B.PL_ALGO_DIRECT, sizes, 48, B.make_opts(slice_bytes=32))
+            pl.scheds.append(s)
+            info = B.pl_schedule_info(s)
+            assert B.pl_schedule_validate(s)[0] == B.PL_OK
+            assert info.message_bytes == total * es
+            assert [int(info.out_bytes[r]) for r in range(R)] == [n * es for n in sizes]
+            outs = interp_run(B.pl_schedule_dump(s), info, R, x, seed=1)
+            ref = oracle.reduce_scatterv(x, sizes, dtype)
+            for r in range(R):
+                o = outs[r]
+                if dtype == "i32":
+                    assert np.array_equal(o.view(np.int32), ref[r])
+                else:
+                    check_float(gen.bf16_bits_to_f64(o.view(np.uint16)), ref[r], dtype)
+            contrib = [x[p][: sizes[p]].copy() for p in range(R)]
+            s = B.pl_schedule_build_v(pl.comm, B.PL_ALLGATHERV, B.PL_ALGO_DIRECT, sizes, 48, B.make_opts(slice_bytes=32))
+            pl.scheds.append(s)
+            info = B.pl_schedule_info(s)
+            assert [int(info.in_bytes[r]) for r in range(R)] == [n * es for n in sizes]
+            outs = interp_run(B.pl_schedule_dump(s), info, R, [c if c.size else np.zeros(0, c.dtype) for c in contrib], seed=2)
+            ref = oracle.allgatherv(contrib)
+            for r in range(R):
+                assert np.array_equal(outs[r], ref[r].view(np.uint8))
+        finally:
+            pl.close()
+    pl = Planner(4, "bf16")
+    try:
+        with pytest.raises(B.PurlinError) as e:
+            B.pl_schedule_build_v(pl.comm, B.PL_ALLGATHERV, B.PL_ALGO_DIRECT, [8, 4, 8, 8], 64)
+        assert e.value.status == B.PL_ERR_ALIGNMENT
+        with pytest.raises(B.PurlinError) as e:
+            B.pl_schedule_build_v(pl.comm, B.PL_REDUCE_SCATTERV, B.PL_ALGO_RING, [8, 8, 8, 8], 64)
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+    finally:
+        pl.close()
