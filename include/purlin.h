@@ -84,7 +84,13 @@ typedef enum {
   PL_ALLTOALL = 3,
   PL_ALLTOALLV = 4,
   PL_ALLGATHERV = 5,      /* copy, packedV -> scatteredV: rank p contributes n[p] elements */
-  PL_REDUCE_SCATTERV = 6  /* reduce, scatteredV -> packedV: rank k receives partition k of n[k] elements */
+  PL_REDUCE_SCATTERV = 6, /* reduce, scatteredV -> packedV: rank k receives partition k of n[k] elements */
+  /* Rooted collectives (the paper's Appendix B proposes them as layouts plus a Root role):
+   * only the root produces (scatter, broadcast) or only the root consumes (gather, reduce). */
+  PL_BROADCAST = 7,       /* compose<scatter, all-gather>: the root's buffer reaches every rank   */
+  PL_REDUCE = 8,          /* compose<reduce-scatter, gather>: the sum reaches the root only       */
+  PL_SCATTER = 9,         /* rank r receives partition r of the root's buffer                     */
+  PL_GATHER = 10          /* the root receives every rank's contribution in rank order            */
 } pl_collective_t;
 
 /* Algorithms.
@@ -261,6 +267,19 @@ pl_status_t pl_schedule_build(pl_comm_t comm, pl_collective_t coll, pl_algo_t al
 pl_status_t pl_schedule_build_v(pl_comm_t comm, pl_collective_t coll, pl_algo_t algo,
                                 const size_t* counts, size_t chunk_bytes,
                                 const pl_sched_opts_t* opts, pl_schedule_t* out);
+
+/* Rooted collectives, root given at run time (0 <= root < R).  count_per_rank: the root's
+ * message for PL_BROADCAST (every output has that size) and the per-rank message for PL_REDUCE
+ * (the root's output has that size); the per-rank partition for PL_SCATTER (root input =
+ * R * count) and PL_GATHER (root output = R * count).  Ranks that contribute nothing need no
+ * input buffer and ranks that receive nothing no output buffer (pl_schedule_info reports 0
+ * bytes for them).  Broadcast and reduce are the two-step compositions the paper names, in one
+ * launch: for broadcast rank k pulls partition k from the root and publishes it, every rank
+ * then pulls partition k from rank k; for reduce rank k reduces partition k into schedule-owned
+ * memory (the root straight into its output) and the root gathers.  Message bytes divisible by
+ * 16*R for broadcast and reduce, by 16 for scatter and gather.  PL_ALGO_DIRECT only. */
+pl_status_t pl_schedule_build_rooted(pl_comm_t comm, pl_collective_t coll, int root, size_t count_per_rank,
+                                     size_t chunk_bytes, const pl_sched_opts_t* opts, pl_schedule_t* out);
 
 /* n_layers back-to-back all-reduces in ONE launch (the latency path: no kernel launch,
  * memset or host round trip per layer).  Layer l reads in[r] + l*M and writes out[r] + l*M

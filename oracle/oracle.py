@@ -153,6 +153,52 @@ def allreduce(inputs, dtype):
     return outs
 
 
+# ---- rooted collectives (the paper's Appendix B: Broadcast copies the root's entire input to
+# every rank, Scatter gives rank r partition r of it, Gather concatenates the contributions in
+# rank order at the root, Reduce combines all contributions at the root; the root takes part
+# locally in each).  Written with plain numpy slicing; ranks that receive nothing get None.
+def broadcast(inputs, root):
+    return [np.array(inputs[root], copy=True) for _ in inputs]
+
+
+def scatter(inputs, root):
+    R = len(inputs)
+    src = inputs[root]
+    assert src.size % R == 0
+    m = src.size // R
+    return [np.array(src[r * m:(r + 1) * m], copy=True) for r in range(R)]
+
+
+def gather(inputs, root):
+    R = len(inputs)
+    out = [None] * R
+    out[root] = np.concatenate([inputs[p] for p in range(R)])
+    return out
+
+
+def reduce(inputs, root, dtype):
+    """Sum over ranks in ascending rank order from zero, delivered at the root only
+    (fp64 for 'bf16'/'f32' inputs, wrapping int32 for 'i32')."""
+    R = len(inputs)
+    out = [None] * R
+    if dtype == "i32":
+        acc = np.zeros(inputs[0].size, dtype=np.uint32)
+        for p in range(R):
+            acc = acc + inputs[p].view(np.uint32)
+        out[root] = acc.view(np.int32)
+        return out
+    acc = np.zeros(inputs[0].size, dtype=np.float64)
+    for p in range(R):
+        if dtype == "bf16":
+            assert inputs[p].dtype == np.uint16
+            f = (inputs[p].astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+        else:
+            f = inputs[p].astype(np.float64)
+        acc = acc + f
+    out[root] = acc
+    return out
+
+
 def moe_dispatch(x, idx, E, recv_capacity_rows=None):
     """x[p]: [T, W] row arrays (any dtype), idx[p]: int32 [T, K].
     Returns dict(recv, meta, pos, counts, expert_counts); recv[r] has capacity rows,

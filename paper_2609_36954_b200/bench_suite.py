@@ -98,13 +98,15 @@ class Bench:
             self.out.write(line + "\n")
             self.out.flush()
 
-    def collective(self, cfg, R, dtype, coll, algo, count, chunk, iters=20, layers=0, graph=False, **kw):
+    def collective(self, cfg, R, dtype, coll, algo, count, chunk, iters=20, layers=0, graph=False, root=None, **kw):
         comm = B.pl_comm_create(R, dtype)
         okw = dict(self.opts_kw)
         okw.update(kw)
         opts = B.make_opts(**okw)
         try:
-            if layers:
+            if root is not None:
+                s = B.pl_schedule_build_rooted(comm, coll, root, count, chunk, opts)
+            elif layers:
                 s = B.pl_schedule_build_layers(comm, ALGO[algo], count, layers, opts)
             else:
                 s = B.pl_schedule_build(comm, coll, ALGO[algo], count, chunk, opts)
@@ -211,7 +213,7 @@ def probe(b):
 
 
 def main(args=None):
-    which = os.environ.get("PL_SUITE", "probe,c1,c2,staged,varlen,c3,c4,c5").split(",")
+    which = os.environ.get("PL_SUITE", "probe,c1,c2,staged,varlen,rooted,c3,c4,c5").split(",")
     out = os.environ.get("PL_SUITE_OUT")  # optional file that receives the JSON lines too
     if out and os.path.dirname(out):
         os.makedirs(os.path.dirname(out), exist_ok=True)
@@ -240,6 +242,11 @@ def main(args=None):
             for size in (MIB, 16 * MIB, 64 * MIB, 256 * MIB):
                 b.collective("staged-AR cap=%d" % cap, 8, B.PL_BF16, B.PL_ALLREDUCE, "direct", size // 2,
                              max(16, min(MIB, size // 8)), iters=10, **kw)
+    if "rooted" in which:
+        for size in (64 * 1024, 64 * MIB):
+            for name, coll, count in (("broadcast", B.PL_BROADCAST, size // 2), ("reduce", B.PL_REDUCE, size // 2),
+                                      ("scatter", B.PL_SCATTER, size // 16), ("gather", B.PL_GATHER, size // 16)):
+                b.collective("rooted-" + name, 8, B.PL_BF16, coll, "direct", count, MIB, root=0, graph=size < MIB)
     if "varlen" in which:
         # the paper's variable-length workload (Appendix C): Zipf(s=0.125) split of T bytes over
         # 8 ranks; all-to-all-v rotates the split per rank so every rank sends and receives T

@@ -25,7 +25,8 @@ PL_OK, PL_ERR_INVALID_ARG, PL_ERR_UNSUPPORTED, PL_ERR_ALIGNMENT, PL_ERR_OOM, PL_
 PL_BF16, PL_F32, PL_I32, PL_U8, PL_F32X2 = range(5)
 DTYPE_SIZE = {PL_BF16: 2, PL_F32: 4, PL_I32: 4, PL_U8: 1, PL_F32X2: 8}
 # collectives
-PL_ALLREDUCE, PL_REDUCE_SCATTER, PL_ALLGATHER, PL_ALLTOALL, PL_ALLTOALLV, PL_ALLGATHERV, PL_REDUCE_SCATTERV = range(7)
+PL_ALLREDUCE, PL_REDUCE_SCATTER, PL_ALLGATHER, PL_ALLTOALL, PL_ALLTOALLV, PL_ALLGATHERV, PL_REDUCE_SCATTERV, \
+    PL_BROADCAST, PL_REDUCE, PL_SCATTER, PL_GATHER = range(11)
 # algorithms
 PL_ALGO_RING, PL_ALGO_TREE, PL_ALGO_DIRECT, PL_ALGO_ONESHOT, PL_ALGO_DIRECT_FUSED = range(5)
 # op kinds / buffer kinds / datapaths
@@ -86,7 +87,7 @@ class pl_devstatus_t(C.Structure):
 
 EXPORTS = [
     "pl_comm_create", "pl_comm_create_planner", "pl_comm_destroy", "pl_comm_status", "pl_comm_reset",
-    "pl_schedule_build", "pl_schedule_build_v", "pl_schedule_build_layers", "pl_schedule_info",
+    "pl_schedule_build", "pl_schedule_build_v", "pl_schedule_build_layers", "pl_schedule_build_rooted", "pl_schedule_info",
     "pl_schedule_dump", "pl_schedule_validate", "pl_schedule_debug_break_wait", "pl_schedule_debug_drop_wait",
     "pl_schedule_destroy",
     "pl_execute", "pl_execute_host",
@@ -123,6 +124,7 @@ def load():
         "pl_schedule_build": [vp, i32, i32, sz, sz, P(pl_sched_opts_t), P(vp)],
         "pl_schedule_build_v": [vp, i32, i32, P(sz), sz, P(pl_sched_opts_t), P(vp)],
         "pl_schedule_build_layers": [vp, i32, sz, i32, P(pl_sched_opts_t), P(vp)],
+        "pl_schedule_build_rooted": [vp, i32, i32, sz, sz, P(pl_sched_opts_t), P(vp)],
         "pl_schedule_info": [vp, P(pl_sched_info_t)],
         "pl_schedule_dump": [vp, P(pl_op_t), sz, P(sz)],
         "pl_schedule_validate": [vp, C.c_char_p, sz],
@@ -223,6 +225,14 @@ def pl_schedule_build_v(comm, coll, algo, counts, chunk_bytes, opts=None):
     _check(load().pl_schedule_build_v(comm, coll, algo, arr, chunk_bytes,
                                       C.byref(opts) if opts is not None else None, C.byref(h)),
            "pl_schedule_build_v")
+    return h
+
+
+def pl_schedule_build_rooted(comm, coll, root, count_per_rank, chunk_bytes, opts=None):
+    h = C.c_void_p()
+    _check(load().pl_schedule_build_rooted(comm, coll, root, count_per_rank, chunk_bytes,
+                                           C.byref(opts) if opts is not None else None, C.byref(h)),
+           "pl_schedule_build_rooted")
     return h
 
 

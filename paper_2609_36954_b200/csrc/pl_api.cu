@@ -328,7 +328,7 @@ pl_status_t pl_comm_reset(pl_comm_t comm, void* stream) {
 
 pl_status_t pl_schedule_build(pl_comm_t comm, pl_collective_t coll, pl_algo_t algo, size_t count_per_rank,
                               size_t chunk_bytes, const pl_sched_opts_t* opts, pl_schedule_t* out) {
-  if (coll == PL_ALLTOALLV || coll == PL_ALLGATHERV || coll == PL_REDUCE_SCATTERV) return PL_ERR_INVALID_ARG;
+  if (coll < PL_ALLREDUCE || coll > PL_ALLTOALL) return PL_ERR_INVALID_ARG;  // V and rooted forms have their own calls
   BuildRequest rq{};
   rq.coll = coll;
   rq.algo = algo;
@@ -348,6 +348,20 @@ pl_status_t pl_schedule_build_v(pl_comm_t comm, pl_collective_t coll, pl_algo_t 
   rq.algo = algo;
   rq.chunk_bytes = chunk_bytes;
   rq.counts_v = c.data();
+  return build_common(comm, rq, opts, out);
+}
+
+pl_status_t pl_schedule_build_rooted(pl_comm_t comm, pl_collective_t coll, int root, size_t count_per_rank,
+                                     size_t chunk_bytes, const pl_sched_opts_t* opts, pl_schedule_t* out) {
+  if (!comm) return PL_ERR_INVALID_ARG;
+  if (coll != PL_BROADCAST && coll != PL_REDUCE && coll != PL_SCATTER && coll != PL_GATHER) return PL_ERR_INVALID_ARG;
+  if (root < 0 || root >= comm->R) return PL_ERR_INVALID_ARG;
+  BuildRequest rq{};
+  rq.coll = coll;
+  rq.algo = PL_ALGO_DIRECT;
+  rq.root = root;
+  rq.count_per_rank = count_per_rank;
+  rq.chunk_bytes = chunk_bytes;
   return build_common(comm, rq, opts, out);
 }
 

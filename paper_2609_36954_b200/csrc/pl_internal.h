@@ -109,6 +109,7 @@ struct BuildRequest {
   uint64_t chunk_bytes;
   const uint64_t* counts_v;  // R*R for all-to-all-v, else null
   int n_layers;              // 0: single collective
+  int root;                  // rooted collectives
   bool staged;               // stage through schedule-owned memory (ordinary application buffers)
   uint64_t staging_bytes;    // staging capacity per rank (0 = default)
   Policy pol;

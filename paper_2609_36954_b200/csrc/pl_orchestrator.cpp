@@ -239,6 +239,74 @@ void agv_direct(Emitter& em, int R, int dtype, const uint64_t* n, uint64_t chunk
       }
 }
 
+// ---- rooted collectives (Appendix B of the paper: layouts plus a Root role) ----------------
+// scatter: only the root produces; rank r copies partition r of the root's input.
+void scatter_direct(Emitter& em, const Geo& g, int root) {
+  em.phase_chunks = g.n_c;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int r = 0; r < g.R; ++r)
+      em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, c * g.chunk * g.es), false,
+                  {ref(root, PL_BUF_IN, PL_U8, (r * g.P + c * g.chunk) * g.es)}, g.clen(c) * g.es, {}, -1);
+}
+
+// gather: only the root consumes; it copies every rank's packed contribution to slot p.
+void gather_direct(Emitter& em, const Geo& g, int root) {
+  em.phase_chunks = g.n_c * g.R;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int p = 0; p < g.R; ++p)
+      em.chunk_op(PL_OP_COPY, root, 0, ref(root, PL_BUF_OUT, PL_U8, (p * g.P + c * g.chunk) * g.es), false,
+                  {ref(p, PL_BUF_IN, PL_U8, c * g.chunk * g.es)}, g.clen(c) * g.es, {}, -1);
+}
+
+// broadcast = compose<scatter, all-gather>: rank k pulls chunk c of partition k from the root
+// into its own output and publishes it; every other rank then pulls it from rank k.
+void broadcast_composed(Emitter& em, const Geo& g, int root) {
+  std::vector<int> have(g.R * g.n_c);
+  em.phase_chunks = g.n_c;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int k = 0; k < g.R; ++k) {
+      const uint64_t off = (k * g.P + c * g.chunk) * g.es;
+      have[k * g.n_c + c] = em.new_flag();
+      em.chunk_op(PL_OP_COPY, k, 0, ref(k, PL_BUF_OUT, PL_U8, off), false, {ref(root, PL_BUF_IN, PL_U8, off)},
+                  g.clen(c) * g.es, {}, have[k * g.n_c + c]);
+    }
+  em.phase_chunks = g.n_c * (g.R - 1);
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int i = 1; i < g.R; ++i)
+      for (int r = 0; r < g.R; ++r) {
+        const int k = (r + i) % g.R;
+        const uint64_t off = (k * g.P + c * g.chunk) * g.es;
+        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, off), false, {ref(k, PL_BUF_OUT, PL_U8, off)},
+                    g.clen(c) * g.es, {have[k * g.n_c + c]}, -1);
+      }
+}
+
+// reduce = compose<reduce-scatter, gather>: rank k reduces chunk c of partition k (ascending
+// rank order) into its scratch -- the root straight into its output -- and the root gathers.
+void reduce_composed(Emitter& em, const Geo& g, int root) {
+  std::vector<int> reduced(g.R * g.n_c, -1);
+  em.phase_chunks = g.n_c;
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int k = 0; k < g.R; ++k) {
+      std::vector<pl_ref_t> src;
+      const uint64_t off = (k * g.P + c * g.chunk) * g.es;
+      for (int p = 0; p < g.R; ++p) src.push_back(ref(p, PL_BUF_IN, g.dtype, off));
+      pl_ref_t d = (k == root) ? ref(root, PL_BUF_OUT, g.dtype, off) : ref(k, PL_BUF_SCRATCH, g.dtype, c * g.chunk * g.es);
+      int f = -1;
+      if (k != root) f = reduced[k * g.n_c + c] = em.new_flag();
+      em.chunk_op(PL_OP_REDUCE, k, 0, d, false, src, g.clen(c), {}, f);
+    }
+  em.phase_chunks = g.n_c * (g.R - 1);
+  for (uint64_t c = 0; c < g.n_c; ++c)
+    for (int k = 0; k < g.R; ++k) {
+      if (k == root) continue;
+      em.chunk_op(PL_OP_COPY, root, 0, ref(root, PL_BUF_OUT, PL_U8, (k * g.P + c * g.chunk) * g.es), false,
+                  {ref(k, PL_BUF_SCRATCH, PL_U8, c * g.chunk * g.es)}, g.clen(c) * g.es, {reduced[k * g.n_c + c]}, -1);
+    }
+  for (int k = 0; k < g.R; ++k)
+    if (k != root) em.L->scratch_per_rank[k] = g.P * g.es;
+}
+
 // all-reduce, one-shot: every rank reduces the whole message from all R inputs.
 void ar_oneshot(Emitter& em, const Geo& g, int layer, uint64_t in_off, uint64_t out_off, const LayerEdges* le) {
   // g.P == g.n here: the "partition" is the whole message, chunked.
@@ -663,7 +731,7 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
   };
   if (R < 2 || R > PL_MAX_RANKS) return fail(PL_ERR_INVALID_ARG, "R out of range");
   if (rq.chunk_bytes == 0 || rq.chunk_bytes % 16) return fail(PL_ERR_INVALID_ARG, "chunk_bytes must be a positive multiple of 16");
-  const bool reduces = rq.coll == PL_ALLREDUCE || rq.coll == PL_REDUCE_SCATTER;
+  const bool reduces = rq.coll == PL_ALLREDUCE || rq.coll == PL_REDUCE_SCATTER || rq.coll == PL_REDUCE;
   if (reduces && dt == PL_U8) return fail(PL_ERR_UNSUPPORTED, "bytes cannot be reduced");
   Emitter em{L, rq.pol.slice_bytes};
   em.dtype = dt;
@@ -723,6 +791,33 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
   const int n_layers = std::max(1, rq.n_layers);
   L->n_layers = n_layers;
 
+  if (rq.coll == PL_BROADCAST || rq.coll == PL_REDUCE || rq.coll == PL_SCATTER || rq.coll == PL_GATHER) {
+    if (rq.algo != PL_ALGO_DIRECT || rq.staged || rq.n_layers > 0) return fail(PL_ERR_UNSUPPORTED, "rooted collectives are direct, unstaged, single layer");
+    if (rq.root < 0 || rq.root >= R) return fail(PL_ERR_INVALID_ARG, "root out of range");
+    const int root = rq.root;
+    if (rq.coll == PL_BROADCAST || rq.coll == PL_REDUCE) {
+      if (bytes % (16 * R)) return fail(PL_ERR_INVALID_ARG, "message bytes must be divisible by 16*R");
+      Geo g = make_geo(R, dt, n, n / R, rq.chunk_bytes);
+      L->message_bytes = bytes;
+      for (int r = 0; r < R; ++r) {
+        L->in_bytes[r] = rq.coll == PL_BROADCAST ? (r == root ? bytes : 0) : bytes;
+        L->out_bytes[r] = rq.coll == PL_BROADCAST ? bytes : (r == root ? bytes : 0);
+      }
+      if (rq.coll == PL_BROADCAST) broadcast_composed(em, g, root);
+      else reduce_composed(em, g, root);
+    } else {
+      if (bytes % 16) return fail(PL_ERR_INVALID_ARG, "partition bytes must be a multiple of 16");
+      Geo g = make_geo(R, dt, n * R, n, rq.chunk_bytes);
+      L->message_bytes = bytes * R;
+      for (int r = 0; r < R; ++r) {
+        L->in_bytes[r] = rq.coll == PL_SCATTER ? (r == root ? bytes * R : 0) : bytes;
+        L->out_bytes[r] = rq.coll == PL_SCATTER ? bytes : (r == root ? bytes * R : 0);
+      }
+      if (rq.coll == PL_SCATTER) scatter_direct(em, g, root);
+      else gather_direct(em, g, root);
+    }
+    return PL_OK;
+  }
   switch (rq.coll) {
     case PL_ALLGATHER: {
       if (bytes % 16) return fail(PL_ERR_INVALID_ARG, "all-gather contribution must be a multiple of 16 bytes");

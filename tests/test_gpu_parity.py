@@ -359,3 +359,41 @@ def test_allgatherv_and_reduce_scatterv(dp, dtype):
                 assert np.array_equal(outs[r], ref[r].view(np.uint8))
         finally:
             ses.close()
+
+
+# ---- rooted collectives -----------------------------------------------------------------------
+@pytest.mark.parametrize("dp", DATAPATHS)
+@pytest.mark.parametrize("root", [0, 5])
+def test_rooted_collectives(dp, root):
+    R = 8
+    for dtype in ("bf16", "i32"):
+        es = 2 if dtype == "bf16" else 4
+        m = (70 * 1024 + 32) // es
+        n = R * m
+        x = gen.rank_inputs(R, n, dtype, seed=23)
+        empty = np.zeros(0, x[0].dtype)
+        ses = Session(R, dtype)
+        try:
+            def run(coll, count, ins):
+                s = B.pl_schedule_build_rooted(ses.comm, coll, root, count, 32768, B.make_opts(datapath=dp))
+                ses.scheds.append(s)
+                return ses.execute(s, ins, repeats=2)
+            outs, _ = run(B.PL_BROADCAST, n, [x[r] if r == root else empty for r in range(R)])
+            for r in range(R):
+                assert np.array_equal(outs[r], x[root].view(np.uint8))
+            outs, info = run(B.PL_REDUCE, n, x)
+            ref = oracle.reduce(x, root, dtype)[root]
+            if dtype == "i32":
+                assert np.array_equal(outs[root].view(np.int32), ref)
+            else:
+                check_float(as_f64(outs[root], dtype), ref, dtype)
+            assert all(int(info.out_bytes[r]) == 0 for r in range(R) if r != root)
+            outs, _ = run(B.PL_SCATTER, m, [x[r] if r == root else empty for r in range(R)])
+            ref = oracle.scatter(x, root)
+            for r in range(R):
+                assert np.array_equal(outs[r], ref[r].view(np.uint8))
+            contrib = [a[:m].copy() for a in x]
+            outs, _ = run(B.PL_GATHER, m, contrib)
+            assert np.array_equal(outs[root], oracle.gather(contrib, root)[root].view(np.uint8))
+        finally:
+            ses.close()

@@ -348,3 +348,32 @@ def test_reduce_scatterv_closed_form_uniform_case_and_zipf_sizes():
     assert c[1].size == 0 and np.array_equal(c[2], full[40:72]) and np.array_equal(c[3], full[72:96])
     # gathering what the V reduce-scatter scattered rebuilds the all-reduce (paper's composition identity)
     assert np.array_equal(np.concatenate(c), full)
+
+
+# ----------------------------------------------------------------------------- #
+# rooted collectives
+# ----------------------------------------------------------------------------- #
+@pytest.mark.parametrize("root", [0, 2])
+def test_rooted_collectives_against_their_unrooted_relatives(root):
+    R, m = 4, 24
+    x = inputs.rank_inputs(R, R * m, "bf16", seed=21)
+    xi = inputs.rank_coded_i32(R, R * m)
+    # reduce = the all-reduce result, at the root only
+    red = oracle.reduce(x, root, "bf16")
+    assert np.array_equal(red[root], oracle.allreduce(x, "bf16")[root])
+    assert all(red[r] is None for r in range(R) if r != root)
+    assert np.array_equal(oracle.reduce(xi, root, "i32")[root], oracle.allreduce(xi, "i32")[root])
+    # gather = the all-gather result, at the root only
+    g = oracle.gather(xi, root)
+    assert np.array_equal(g[root], oracle.allgather(xi)[root]) and g[(root + 1) % R] is None
+    # scatter = what all-to-all delivers from the root: partition r of the root's buffer
+    sc = oracle.scatter(xi, root)
+    a2a = oracle.alltoall(xi)
+    for r in range(R):
+        assert np.array_equal(sc[r], a2a[r][root * m:(root + 1) * m])
+        assert sc[r][0] == root * R * m + r * m          # closed form on rank-coded ints
+    # broadcast: every rank ends with the root's buffer; gather(scatter(x)) rebuilds it at the root
+    bc = oracle.broadcast(xi, root)
+    for r in range(R):
+        assert np.array_equal(bc[r], xi[root])
+    assert np.array_equal(oracle.gather(sc, root)[root], xi[root])

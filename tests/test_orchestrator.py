@@ -449,3 +449,50 @@ def test_allgatherv_reduce_scatterv_replay(R):
         assert e.value.status == B.PL_ERR_UNSUPPORTED
     finally:
         pl.close()
+
+
+# ---- rooted collectives -----------------------------------------------------------------------
+@pytest.mark.parametrize("R,root", [(2, 1), (5, 0), (8, 3)])
+def test_rooted_collectives_replay(R, root):
+    for dtype in ("i32", "bf16"):
+        es = B.DTYPE_SIZE[DT[dtype]]
+        m = (16 // es) * 7
+        n = R * m
+        x = gen.rank_inputs(R, n, dtype, seed=17)
+        empty = np.zeros(0, x[0].dtype)
+        pl = Planner(R, dtype)
+        try:
+            def build(coll, count):
+                s = B.pl_schedule_build_rooted(pl.comm, coll, root, count, 48, B.make_opts(slice_bytes=32, n_ctas=2 * R))
+                pl.scheds.append(s)
+                st, msg = B.pl_schedule_validate(s)
+                assert st == B.PL_OK, msg
+                return s, B.pl_schedule_info(s)
+            s, info = build(B.PL_BROADCAST, n)
+            assert [int(info.in_bytes[r]) for r in range(R)] == [n * es if r == root else 0 for r in range(R)]
+            outs = interp_run(B.pl_schedule_dump(s), info, R, [x[r] if r == root else empty for r in range(R)], seed=1)
+            for r in range(R):
+                assert np.array_equal(outs[r], oracle.broadcast(x, root)[r].view(np.uint8))
+            s, info = build(B.PL_REDUCE, n)
+            assert [int(info.out_bytes[r]) for r in range(R)] == [n * es if r == root else 0 for r in range(R)]
+            outs = interp_run(B.pl_schedule_dump(s), info, R, x, seed=2)
+            ref = oracle.reduce(x, root, dtype)[root]
+            if dtype == "i32":
+                assert np.array_equal(outs[root].view(np.int32), ref)
+            else:
+                check_float(gen.bf16_bits_to_f64(outs[root].view(np.uint16)), ref, dtype)
+            s, info = build(B.PL_SCATTER, m)
+            outs = interp_run(B.pl_schedule_dump(s), info, R, [x[r] if r == root else empty for r in range(R)], seed=3)
+            for r in range(R):
+                assert np.array_equal(outs[r], oracle.scatter(x, root)[r].view(np.uint8))
+            contrib = [a[:m].copy() for a in x]
+            s, info = build(B.PL_GATHER, m)
+            outs = interp_run(B.pl_schedule_dump(s), info, R, contrib, seed=4)
+            assert np.array_equal(outs[root], oracle.gather(contrib, root)[root].view(np.uint8))
+            assert all(outs[r].size == 0 for r in range(R) if r != root)
+            with pytest.raises(B.PurlinError):
+                B.pl_schedule_build_rooted(pl.comm, B.PL_BROADCAST, R, n, 48, None)
+            with pytest.raises(B.PurlinError):
+                B.pl_schedule_build_rooted(pl.comm, B.PL_ALLREDUCE, 0, n, 48, None)
+        finally:
+            pl.close()
