@@ -247,6 +247,27 @@ def main(args=None):
             for name, coll, count in (("broadcast", B.PL_BROADCAST, size // 2), ("reduce", B.PL_REDUCE, size // 2),
                                       ("scatter", B.PL_SCATTER, size // 16), ("gather", B.PL_GATHER, size // 16)):
                 b.collective("rooted-" + name, 8, B.PL_BF16, coll, "direct", count, MIB, root=0, graph=size < MIB)
+    if "ablation" in which:
+        # (a) pipeline depth at a fixed CTA count: the analogue of the paper's copy ablation
+        #     (Sec. 5, "ablation": bandwidth vs. number of stages S at fixed stage size)
+        n = 32 * MIB
+        for sb in (16384, 32768):
+            for S in (2, 3, 4, 6, 8):
+                if 1024 + S * sb > 227 * 1024:
+                    continue
+                kw = dict(datapath=B.PL_DP_TMA, stages=S, stage_bytes=sb, n_ctas=144, slice_bytes=262144)
+                b.collective("depth-copy S=%d B=%d" % (S, sb), 8, B.PL_BF16, B.PL_ALLGATHER, "direct", n // 8, MIB, **kw)
+                b.collective("depth-reduce S=%d B=%d" % (S, sb), 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "direct", n, MIB, **kw)
+        # (b) CTA count at the default ring: the analogue of the paper's SM sweep (Sec. 2.2, Fig. 2)
+        for nct in (8, 16, 32, 64, 96, 128, 144):
+            kw = dict(datapath=B.PL_DP_TMA, n_ctas=nct, slice_bytes=65536)
+            b.collective("ctas-copy n=%d" % nct, 8, B.PL_BF16, B.PL_ALLGATHER, "direct", n // 8, MIB, **kw)
+            b.collective("ctas-reduce n=%d" % nct, 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "direct", n, MIB, **kw)
+        # (c) register path vs bulk-copy ring on the same schedules
+        for dp, name in ((B.PL_DP_LDST, "ldst"), (B.PL_DP_TMA, "tma")):
+            b.collective("datapath-copy " + name, 8, B.PL_BF16, B.PL_ALLGATHER, "direct", n // 8, MIB, datapath=dp)
+            b.collective("datapath-reduce " + name, 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "direct", n, MIB, datapath=dp)
+            b.collective("datapath-a2a " + name, 8, B.PL_BF16, B.PL_ALLTOALL, "direct", n, MIB, datapath=dp)
     if "varlen" in which:
         # the paper's variable-length workload (Appendix C): Zipf(s=0.125) split of T bytes over
         # 8 ranks; all-to-all-v rotates the split per rank so every rank sends and receives T
