@@ -1,0 +1,181 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py / the suite time.
+
+The oracle cannot redo a 4 GiB collective in seconds, so outputs are checked on samples: the
+oracle is run on the sampled input positions only (it computes those outputs one by one from
+the definition), and copy-only results are compared exactly on sampled blocks.  Large buffers
+are filled by tiling a seeded block and rolling it per rank, which keeps the N(0,1) value
+distribution.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_2609_36954_b200 import binding as B
+from paper_2609_36954_b200 import inputs as gen
+
+from gpu_harness import check_float, stream_handle
+
+pytestmark = pytest.mark.gpu
+MIB = 1 << 20
+
+
+def big_inputs(R, n, seed=0, block=1 << 20):
+    """Per-rank uint16 bf16 buffers of n elements on the GPU (tiled seeded block, rank-rolled)."""
+    outs = []
+    for r in range(R):
+        blk = torch.from_numpy(gen.normal_bf16(min(block, n), seed, r).view(np.int16)).cuda()
+        reps = (n + blk.numel() - 1) // blk.numel()
+        t = blk.repeat(reps)[:n]
+        outs.append(torch.roll(t, 977 * r + 13).contiguous())
+    return outs
+
+
+def sample_idx(n, k=4096, seed=1):
+    rng = np.random.default_rng(seed)
+    idx = np.unique(np.concatenate([rng.integers(0, n, size=k), np.arange(0, 64), np.arange(n - 64, n)]))
+    return idx
+
+
+def gather_samples(tensors, idx):
+    ti = torch.from_numpy(idx).cuda()
+    return [t[ti].cpu().numpy().view(np.uint16) for t in tensors]
+
+
+def run(sched, comm, R, d_in, d_out):
+    info = B.pl_schedule_info(sched)
+    bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                       [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
+    B.pl_execute(sched, bufs, stream_handle())
+    torch.cuda.synchronize()
+    assert B.pl_comm_status(comm).code == B.PL_OK
+    return info
+
+
+def test_c2_reduce_scatter_then_all_gather_full_size():
+    R, n = 8, 32 * MIB  # 64 MiB bf16 per rank
+    comm = B.pl_comm_create(R, B.PL_BF16)
+    try:
+        x = big_inputs(R, n)
+        for algo, chunk in ((B.PL_ALGO_DIRECT, MIB), (B.PL_ALGO_RING, 256 * 1024)):
+            rs = B.pl_schedule_build(comm, B.PL_REDUCE_SCATTER, algo, n, chunk, None)
+            ag = B.pl_schedule_build(comm, B.PL_ALLGATHER, algo, n // R, chunk, None)
+            mid = [torch.full((n // R,), -1, dtype=torch.int16, device="cuda") for _ in range(R)]
+            out = [torch.full((n,), -1, dtype=torch.int16, device="cuda") for _ in range(R)]
+            irs = run(rs, comm, R, x, mid)
+            run(ag, comm, R, mid, out)
+            assert irs.datapath == B.PL_DP_TMA
+            idx = sample_idx(n)
+            ref = oracle.allreduce(gather_samples(x, idx), "bf16")          # sums at the sampled positions
+            for r in (0, 3, 7):
+                got = gen.bf16_bits_to_f64(out[r][torch.from_numpy(idx).cuda()].cpu().numpy().view(np.uint16))
+                check_float(got, ref[r], "bf16")
+            # all-gather is a copy: every rank's output equals the concatenation of the mids, bit for bit
+            cat = torch.cat(mid)
+            for r in range(R):
+                assert torch.equal(out[r], cat)
+            B.pl_schedule_destroy(rs)
+            B.pl_schedule_destroy(ag)
+    finally:
+        B.pl_comm_destroy(comm)
+
+
+@pytest.mark.parametrize("algo", [B.PL_ALGO_DIRECT, B.PL_ALGO_DIRECT_FUSED, B.PL_ALGO_RING, B.PL_ALGO_TREE])
+def test_c3_allreduce_256mib_sampled(algo):
+    R, n = 8, 128 * MIB  # 256 MiB bf16 per rank
+    comm = B.pl_comm_create(R, B.PL_BF16)
+    try:
+        x = big_inputs(R, n)
+        s = B.pl_schedule_build(comm, B.PL_ALLREDUCE, algo, n, MIB, None)
+        out = [torch.full((n,), -1, dtype=torch.int16, device="cuda") for _ in range(R)]
+        run(s, comm, R, x, out)
+        idx = sample_idx(n)
+        ref = oracle.allreduce(gather_samples(x, idx), "bf16")
+        ti = torch.from_numpy(idx).cuda()
+        for r in (0, 5):
+            check_float(gen.bf16_bits_to_f64(out[r][ti].cpu().numpy().view(np.uint16)), ref[r], "bf16")
+        for r in range(1, R):  # every rank holds the same bits
+            assert torch.equal(out[r], out[0])
+        B.pl_schedule_destroy(s)
+    finally:
+        B.pl_comm_destroy(comm)
+
+
+@pytest.mark.parametrize("batch,algo", [(1, B.PL_ALGO_DIRECT_FUSED), (1, B.PL_ALGO_ONESHOT), (64, B.PL_ALGO_DIRECT_FUSED)])
+def test_c5_decode_allreduce_80_layers(batch, algo):
+    R, hidden, layers = 8, 8192, 80
+    n = batch * hidden
+    comm = B.pl_comm_create(R, B.PL_BF16)
+    try:
+        x = big_inputs(R, n * layers, seed=5, block=1 << 18)
+        s = B.pl_schedule_build_layers(comm, algo, n, layers, None)
+        out = [torch.full((n * layers,), -1, dtype=torch.int16, device="cuda") for _ in range(R)]
+        for _ in range(2):  # twice: flags carry over between executes
+            run(s, comm, R, x, out)
+        idx = sample_idx(n * layers, k=8192)  # spans every layer
+        ref = oracle.allreduce(gather_samples(x, idx), "bf16")
+        ti = torch.from_numpy(idx).cuda()
+        for r in (0, 7):
+            check_float(gen.bf16_bits_to_f64(out[r][ti].cpu().numpy().view(np.uint16)), ref[r], "bf16")
+        B.pl_schedule_destroy(s)
+    finally:
+        B.pl_comm_destroy(comm)
+
+
+@pytest.mark.parametrize("identity", [False, True])
+def test_c4_moe_full_size_sampled(identity):
+    R, T, H, E, K = 8, 4096, 7168, 256, 8
+    idx, gates = gen.moe_routing(R, T, E, K, identity_perm=identity)
+    # routing-only oracle run (token rows replaced by their ids) gives pos / meta / counts exactly
+    ids = [np.arange(T, dtype=np.int32).reshape(T, 1) + p * T for p in range(R)]
+    cap = int(max(np.bincount(np.concatenate([i.ravel() for i in idx]) // (E // R), minlength=R)))
+    ref = oracle.moe_dispatch(ids, idx, E, recv_capacity_rows=cap)
+    comm = B.pl_comm_create(R, B.PL_BF16)
+    plan = B.pl_moe_plan_create(comm, T, H, E, K, cap)
+    try:
+        x = [t.view(T, H) for t in big_inputs(R, T * H, seed=2, block=1 << 20)]
+        d_i = [torch.from_numpy(a).cuda() for a in idx]
+        d_g = [torch.from_numpy(a).cuda() for a in gates]
+        recv = [torch.full((cap, H), -1, dtype=torch.int16, device="cuda") for _ in range(R)]
+        meta = [torch.full((cap, 4), -1, dtype=torch.int32, device="cuda") for _ in range(R)]
+        out = [torch.full((T, H), -1, dtype=torch.int16, device="cuda") for _ in range(R)]
+        B.pl_moe_dispatch(plan, [t.data_ptr() for t in x], [t.data_ptr() for t in d_i],
+                          [t.data_ptr() for t in recv], [t.data_ptr() for t in meta], stream_handle())
+        pos = np.zeros((R, T, K), np.int32)
+        counts = np.zeros((R, R), np.int64)
+        ecounts = np.zeros((R, E), np.int64)
+        assert B.pl_moe_plan_read(plan, pos.ctypes.data, counts.ctypes.data, ecounts.ctypes.data, stream_handle()) == B.PL_OK
+        assert np.array_equal(counts, ref["counts"]) and np.array_equal(ecounts, ref["expert_counts"])
+        assert counts.sum() == R * T * K == 262144
+        for p in range(R):
+            assert np.array_equal(pos[p], ref["pos"][p])
+        rng = np.random.default_rng(3)
+        for r in range(R):
+            nrows = int(counts[:, r].sum())
+            assert np.array_equal(meta[r][:nrows].cpu().numpy(), ref["meta"][r][:nrows])
+            rows = np.unique(np.concatenate([rng.integers(0, nrows, size=256), [0, nrows - 1]]))
+            m = ref["meta"][r][rows]
+            for row, (p, t, _, _) in zip(rows.tolist(), m.tolist()):
+                assert torch.equal(recv[r][row], x[p][t]), (r, row)
+            assert bool((recv[r][nrows:] == -1).all())  # nothing written past the received rows
+        # combine over identity experts; reference per sampled token from the definition
+        B.pl_moe_combine(plan, [t.data_ptr() for t in recv], [t.data_ptr() for t in d_g],
+                         [t.data_ptr() for t in out], stream_handle())
+        torch.cuda.synchronize()
+        epr = E // R
+        for p in (0, 6):
+            toks = np.unique(rng.integers(0, T, size=64))
+            y_rows = []
+            for t in toks.tolist():
+                rows = [recv[idx[p][t, j] // epr][pos[p, t, j]].cpu().numpy().view(np.uint16) for j in range(K)]
+                y_rows.append(np.stack(rows))
+            # oracle combine on a miniature problem: one "rank" whose y holds the K rows of each sampled token
+            ymini = [np.concatenate(y_rows)]
+            idx_m = [np.zeros((len(toks), K), np.int32)]
+            pos_m = [np.arange(len(toks) * K, dtype=np.int32).reshape(len(toks), K)]
+            want = oracle.moe_combine(ymini, idx_m, pos_m, [np.ascontiguousarray(gates[p][toks])], 1, H)[0]
+            got = gen.bf16_bits_to_f64(out[p][torch.from_numpy(toks).cuda()].cpu().numpy().view(np.uint16))
+            check_float(got, want, "bf16")
+    finally:
+        B.pl_moe_plan_destroy(plan)
+        B.pl_comm_destroy(comm)
