@@ -150,3 +150,25 @@ def test_moe_argument_errors():
                 B.pl_moe_plan_create(comm, *args)
     finally:
         B.pl_comm_destroy(comm)
+
+
+def test_moe_sixteen_ranks_topk_32():
+    R, T, H, E, K = 16, 96, 64, 64, 32          # the widest top-k and communicator the plan accepts
+    idx, gates = gen.moe_routing(R, T, E, K, seed=8)
+    x = gen.moe_tokens_bf16(R, T, H, seed=9)
+    cap = R * T * K
+    ref = oracle.moe_dispatch(x, idx, E, recv_capacity_rows=cap)
+    run = MoeRun(R, T, H, E, K, cap)
+    try:
+        st, recv, meta, pos, counts, ecounts = run.dispatch(x, idx)
+        assert st == B.PL_OK and np.array_equal(counts, ref["counts"])
+        for r in range(R):
+            n = int(counts[:, r].sum())
+            assert np.array_equal(recv[r].view(np.uint16).reshape(cap, H)[:n], ref["recv"][r][:n])
+            assert np.array_equal(meta[r][:n], ref["meta"][r][:n])
+        out = run.combine(run.d_recv, gates)
+        want = oracle.moe_combine(ref["recv"], idx, ref["pos"], gates, E, H)
+        for p in range(R):
+            check_float(gen.bf16_bits_to_f64(out[p]), want[p], "bf16")
+    finally:
+        run.close()

@@ -397,3 +397,28 @@ def test_rooted_collectives(dp, root):
             assert np.array_equal(outs[root], oracle.gather(contrib, root)[root].view(np.uint8))
         finally:
             ses.close()
+
+
+# ---- the largest communicator the ABI allows ---------------------------------------------------
+@pytest.mark.parametrize("dp", DATAPATHS)
+def test_sixteen_ranks(dp):
+    R = B.PL_MAX_RANKS
+    for dtype in ("bf16", "i32"):
+        es = 2 if dtype == "bf16" else 4
+        n = R * ((20 * 1024 + 16) // es)
+        x = gen.rank_inputs(R, n, dtype, seed=31)
+        ref = oracle.allreduce(x, dtype)
+        ses = Session(R, dtype)
+        try:
+            for algo in ALL_AR:
+                s = ses.build(B.PL_ALLREDUCE, algo, n, 8192, datapath=dp)
+                outs, info = ses.execute(s, x, repeats=2)
+                assert info.grid % R == 0
+                compare_reduce(outs, ref, dtype)
+            s = ses.build(B.PL_ALLTOALL, B.PL_ALGO_DIRECT, n, 8192, datapath=dp)
+            outs, _ = ses.execute(s, x)
+            a2a = oracle.alltoall(x)
+            for r in range(R):
+                assert np.array_equal(outs[r], a2a[r].view(np.uint8))
+        finally:
+            ses.close()
