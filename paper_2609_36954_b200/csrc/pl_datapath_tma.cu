@@ -149,12 +149,25 @@ __device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDe
       else r = acc.result();
       if (!bcast) {
         st16(d.dst + (size_t)u * 16u, r);
+      } else if (pmask == 0) {
+        // Replicated destination: park the result in the slot, over unit u of the first source
+        // tile (this thread has already read unit u of every tile and nobody else reads it);
+        // the copier sends the tile to all R outputs with bulk stores.
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(ptx::smem_u32(slot + (size_t)u * 16u)), "r"(r.x),
+                     "r"(r.y), "r"(r.z), "r"(r.w)
+                     : "memory");
       } else {
         for (int k = 0; k < P.n_ranks; ++k)
           st16(static_cast<char*>(P.base[kSlotOut + k]) + d.dst_off + (size_t)u * 16u, r);
       }
     }
   }
+  if (bcast && pmask == 0) ptx::fence_proxy_async_smem();  // generic writes above -> the copier's bulk stores
+}
+
+// A REDUCE stage whose result leaves through shared memory (see consume_stage).
+__device__ __forceinline__ bool leaves_via_smem(uint32_t kind, uint32_t flags, uint32_t pmask) {
+  return kind != PL_OP_COPY && (flags & kDstBcast) && !(flags & kDstF32) && pmask == 0;
 }
 
 template <int DT>
@@ -290,6 +303,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
   } else if (warp == 1) {
     // ================================ copier ============================================
     int prev = -1;  // slot whose bulk store may still be reading shared memory
+    uint32_t done_parity = 0;  // tracked exactly as the consumers do
     for (uint32_t n = 0;; ++n) {
       const uint32_t s = n % S, ph = (n / S) & 1u;
       bool go = true;
@@ -300,10 +314,28 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
       const StageDesc& d = c->desc[s];
       const uint32_t kind = d.kind;
       if (kind == kEnd) break;
+      const bool via_smem = leaves_via_smem(kind, d.flags, d.pmask);
+      const bool uses_done = via_smem || (kind != PL_OP_COPY && (d.flags & kLastOfOp) && d.signal != kNoFlag);
+      if (via_smem) {
+        bool ready = true;
+        if (lane == 0) ready = wait_bar(P, c, &c->done[s], (done_parity >> s) & 1u);  // all consumer warps wrote
+        ready = __shfl_sync(0xFFFFFFFFu, (int)ready, 0);
+        if (!ready) break;
+      }
+      if (uses_done) done_parity ^= 1u << s;
       if (lane == 0) {
-        if (kind == PL_OP_COPY) {
-          if (P.hints & 2u) ptx::bulk_s2g_hint(d.dst, slots + (size_t)s * slot_bytes, d.units * 16u, ptx::policy_evict_first());
-          else ptx::bulk_s2g(d.dst, slots + (size_t)s * slot_bytes, d.units * 16u);
+        if (kind == PL_OP_COPY || via_smem) {
+          if (via_smem) {
+            for (int k = 0; k < P.n_ranks; ++k) {
+              void* dk = static_cast<char*>(P.base[kSlotOut + k]) + d.dst_off;
+              if (P.hints & 2u) ptx::bulk_s2g_hint(dk, slots + (size_t)s * slot_bytes, d.units * 16u, ptx::policy_evict_first());
+              else ptx::bulk_s2g(dk, slots + (size_t)s * slot_bytes, d.units * 16u);
+            }
+          } else if (P.hints & 2u) {
+            ptx::bulk_s2g_hint(d.dst, slots + (size_t)s * slot_bytes, d.units * 16u, ptx::policy_evict_first());
+          } else {
+            ptx::bulk_s2g(d.dst, slots + (size_t)s * slot_bytes, d.units * 16u);
+          }
           ptx::bulk_commit();
           if (prev >= 0) {
             ptx::bulk_wait_read<1>();
@@ -350,7 +382,11 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
         const bool last = d.flags & kLastOfOp;
         const uint32_t signal = d.signal, signal2 = d.signal2;
         __syncwarp();
-        if (last && signal != kNoFlag) {
+        if (leaves_via_smem(kind, d.flags, d.pmask)) {
+          // the copier ships the tile (and signals, if this is the op's last stage)
+          if (lane == 0) ptx::mbar_arrive(&c->done[s]);
+          done_parity ^= 1u << s;
+        } else if (last && signal != kNoFlag) {
           // every consumer warp reports its stores; consumer thread 0 then publishes
           if (lane == 0) ptx::mbar_arrive(&c->done[s]);
           if (ctid == 0) {
