@@ -89,6 +89,8 @@ struct ExecParams {
 struct Policy {
   int n_ctas, threads, datapath, stages;
   uint32_t stage_bytes, slice_bytes;
+  // automatic slicing (slice_bytes == 0): bounds of a slice
+  uint32_t min_slice, max_slice;
 };
 
 struct Lowered {

@@ -5,6 +5,7 @@
 // role, and the consume operation (copy or reduce) selects the op kind.  Everything here
 // is plain host C++: no CUDA calls.
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <map>
@@ -33,9 +34,10 @@ struct Emitter {
   // Chunks each rank runs in the phase being emitted (0 = unknown).  When known, the slice
   // count is nudged upwards so that a rank's work items divide evenly over its queues.
   uint64_t phase_chunks = 0;
-  // slice_bytes == 0: pick the slice per phase so that every queue of the rank gets about
-  // two work items, within [min_slice, max_slice]
+  // slice_bytes == 0: the slice count is chosen per phase by a cost model, slices stay within
+  // [min_slice, max_slice]
   uint32_t min_slice = 16384, max_slice = 131072;
+  double op_overhead_us = 1.5, wait_overhead_us = 0.5;
   int role = 0;  // role stamped on emitted ops
 
   int new_flag() { return L->n_flags++; }
@@ -54,19 +56,31 @@ struct Emitter {
     const uint64_t unit16 = kind == PL_OP_COPY ? 16 : 16 / elem_size(dtype);
     uint64_t wide = count * max_es;
     uint64_t n_slices = 1;
-    uint64_t slice = slice_bytes;
-    if (slice == 0) {
-      const uint64_t phase_bytes = std::max<uint64_t>(1, phase_chunks) * wide;
-      slice = phase_bytes / (2 * (uint64_t)queues_per_rank);
-      slice = std::min<uint64_t>(max_slice, std::max<uint64_t>(min_slice, slice / 4096 * 4096));
-    }
-    if (wide > slice + slice / 2) n_slices = (wide + slice - 1) / slice;
-    if (n_slices > 1 && phase_chunks && queues_per_rank > 1) {
-      for (uint64_t k = n_slices; k <= 4 * n_slices; ++k)
-        if ((phase_chunks * k) % (uint64_t)queues_per_rank == 0 && wide / k >= 4096) {
+    if (slice_bytes) {
+      if (wide > (uint64_t)slice_bytes + slice_bytes / 2) n_slices = (wide + slice_bytes - 1) / slice_bytes;
+    } else {
+      // Pick the slice count that minimises the time of the phase under a simple model: a rank
+      // runs `chunks` chunks of this shape on `queues_per_rank` queues; a queue spends a fixed
+      // cost per op (descriptor hand-off, barrier, flag traffic: small for the bulk-copy ring,
+      // which runs ahead across ops, larger for the register path) plus its bytes at the
+      // per-SM share of the memory bandwidth.
+      uint64_t traffic = count * elem_size(dst.dtype) * (bcast ? 8 : 1);
+      for (const pl_ref_t& s : src) traffic += count * elem_size(s.dtype);
+      const double chunks = (double)std::max<uint64_t>(1, phase_chunks);
+      const double bytes_per_us = 40000.0;  // ~6 TB/s over 148 SMs
+      const uint64_t k_lo = std::max<uint64_t>(1, (wide + max_slice - 1) / max_slice);
+      const uint64_t k_hi = std::max<uint64_t>(k_lo, std::min<uint64_t>(wide / std::max<uint32_t>(16, min_slice), 8ull * queues_per_rank));
+      // an op that waits on a flag cannot hide that latency behind its predecessor
+      const double overhead = op_overhead_us + (waits.empty() ? 0.0 : wait_overhead_us);
+      double best = 1e300;
+      for (uint64_t k = k_lo; k <= k_hi; ++k) {
+        const double rounds = std::ceil(chunks * (double)k / (double)queues_per_rank);
+        const double cost = rounds * (overhead + (double)traffic / (double)k / bytes_per_us);
+        if (cost < best * 0.97) {  // more slices only for a clear gain
+          best = cost;
           n_slices = k;
-          break;
         }
+      }
     }
     uint64_t per = (count + n_slices - 1) / n_slices;
     uint64_t unit = (per >= 64 * unit16) ? 8 * unit16 : unit16;
@@ -709,14 +723,22 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
   if (p.threads <= 0) p.threads = 512;
   if (p.stages <= 0) p.stages = 4;
   if (p.stage_bytes == 0) p.stage_bytes = 49152;
+  // Latency regime (at most 1 MiB per rank, and every layered schedule): slices down to 2 KiB,
+  // one work item per queue, as many queues as there are items.  Measured on B200 with 80
+  // layers in one launch: 16 KiB one-shot is fastest with 8 queues per rank of 2 KiB each.
+  const bool latency = msg <= (1u << 20) || rq.n_layers > 0;
+  p.min_slice = latency ? 2048 : 16384;
+  p.max_slice = latency ? 32768 : (p.datapath == PL_DP_TMA ? 262144 : 131072);
   if (max_resident_ctas <= 0) return p;
   if (p.n_ctas <= 0) {
     const int full = std::max(rq.R, max_resident_ctas / rq.R * rq.R);
-    // queues a rank can keep busy: one per 16 KiB of what it produces
-    uint64_t per_rank_out = msg;
-    if (rq.coll == PL_REDUCE_SCATTER || rq.coll == PL_REDUCE_SCATTERV) per_rank_out = msg / rq.R;
-    const uint64_t unit = p.slice_bytes ? p.slice_bytes : 16384;
-    uint64_t want = std::max<uint64_t>(1, (per_rank_out + unit - 1) / unit) * rq.R;
+    // bytes a rank produces in its busiest phase
+    uint64_t per_rank = msg;
+    if (rq.coll == PL_REDUCE_SCATTER || rq.coll == PL_REDUCE_SCATTERV) per_rank = msg / rq.R;
+    if (rq.coll == PL_ALLREDUCE && rq.algo == PL_ALGO_DIRECT_FUSED) per_rank = msg / rq.R;
+    uint64_t unit = p.slice_bytes;
+    if (unit == 0) unit = std::min<uint64_t>(p.max_slice, std::max<uint64_t>(p.min_slice, per_rank / (full / rq.R)));
+    uint64_t want = std::max<uint64_t>(1, (per_rank + unit - 1) / unit) * rq.R;
     p.n_ctas = (int)std::min<uint64_t>(full, std::max<uint64_t>(rq.R, want));
   }
   p.n_ctas = std::max(rq.R, p.n_ctas / rq.R * rq.R);
@@ -735,7 +757,10 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
   if (reduces && dt == PL_U8) return fail(PL_ERR_UNSUPPORTED, "bytes cannot be reduced");
   Emitter em{L, rq.pol.slice_bytes};
   em.dtype = dt;
-  em.max_slice = rq.pol.datapath == PL_DP_TMA ? 262144 : 131072;
+  em.min_slice = rq.pol.min_slice;
+  em.max_slice = rq.pol.max_slice;
+  em.op_overhead_us = rq.pol.datapath == PL_DP_TMA ? 0.2 : 1.5;
+  em.wait_overhead_us = rq.pol.datapath == PL_DP_TMA ? 1.5 : 0.5;  // measured on ring schedules
   em.queues_per_rank = std::max(1, rq.pol.n_ctas / R);
   L->n_layers = 1;
 

@@ -281,7 +281,7 @@ def test_validator_catches_a_broken_edge():
 def test_queues_are_rank_owned_and_balanced():
     pl = Planner(8, "bf16")
     try:
-        s = pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, 8 << 20, 1 << 20, n_ctas=144, slice_bytes=65536)
+        s = pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, 8 << 20, 1 << 20, n_ctas=144)  # automatic slicing
         ops = B.pl_schedule_dump(s)
         load = {}
         for o in ops:
