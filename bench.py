@@ -229,6 +229,11 @@ def run_purlin(args):
         gotf = gen.bf16_bits_to_f64(got[idx])
         assert np.all(np.abs(gotf - exact) <= 2.0 ** -7 * np.abs(exact) + 1e-6), "e2e result is wrong"
 
+    # ---- p50 latency of the small all-reduce (the metric's second half) ----------------------
+    latency = None
+    if not args.no_latency:
+        latency = measure_small_allreduce(B, torch, stream)
+
     # ---- roofline of the dominant kernel (the reduce-scatter launch) -----------------------
     rs_alg = irs.bytes_read + irs.bytes_written            # (R+1) * M: every byte touched once
     ag_floor = iag.in_bytes[0] * R + iag.bytes_written     # compulsory DRAM traffic (R+1) * M
@@ -266,13 +271,48 @@ def run_purlin(args):
                        "l2": "inputs_larger_than_l2 (512 MiB of inputs per step; no flush)",
                        "replicas": world, "parallelism": "replicas only (no inter-GPU exchange on this path)"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "cpu_baseline": cpu, "detail": detail,
+            "cpu_baseline": cpu, "small_allreduce": latency, "detail": detail,
         }
         print(json.dumps(line))
     B.pl_schedule_destroy(rs)
     B.pl_schedule_destroy(ag)
     B.pl_comm_destroy(comm)
     replicas.finalize()
+
+
+def measure_small_allreduce(B, torch, stream, R=8, hidden=8192, layers=80, steps=200):
+    """Tensor-parallel decode shape: one token x hidden 8192 bf16 (16 KiB per rank), 80
+    back-to-back all-reduces in ONE launch, distinct inputs per layer.  p50 over steps of the
+    time per layer, CUDA events around each launch."""
+    from paper_2609_36954_b200 import inputs as gen
+    n = hidden
+    comm = B.pl_comm_create(R, B.PL_BF16)
+    out = {}
+    for name, algo in (("oneshot", B.PL_ALGO_ONESHOT), ("fused", B.PL_ALGO_DIRECT_FUSED)):
+        s = B.pl_schedule_build_layers(comm, algo, n, layers, None)
+        info = B.pl_schedule_info(s)
+        d_in = [torch.from_numpy(np.concatenate([gen.normal_bf16(n, 0, l * R + r) for l in range(layers)]).view(np.int16)).cuda()
+                for r in range(R)]
+        d_out = [torch.empty(n * layers, dtype=torch.int16, device="cuda") for _ in range(R)]
+        bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                           [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
+        for _ in range(5):
+            B.pl_execute(s, bufs, stream)
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        ev[0].record()
+        for i in range(steps):
+            B.pl_execute(s, bufs, stream)
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        us = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]) * 1e3 / layers
+        out[name] = {"p50_us": float(np.median(us)), "p10_us": float(np.percentile(us, 10)),
+                     "p90_us": float(np.percentile(us, 90)), "grid": int(info.grid)}
+        B.pl_schedule_destroy(s)
+    B.pl_comm_destroy(comm)
+    best = min(out, key=lambda k: out[k]["p50_us"])
+    return {"metric": "p50 us per 16 KiB all-reduce (R=8, bf16, 80 layers per launch, per layer)",
+            "p50_us": out[best]["p50_us"], "algorithm": best, "all": out, "steps": steps}
 
 
 # ------------------------------------------------------------------------------------------
@@ -357,6 +397,7 @@ def main():
     ap.add_argument("--suite", action="store_true", help="run every configuration (paper_2609_36954_b200/bench_suite.py)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-latency", action="store_true")
     ap.add_argument("--fast-inputs", action="store_true", help="tile 4 Mi generated elements instead of generating all")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--n-ctas", type=int, default=0)

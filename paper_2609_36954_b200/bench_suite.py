@@ -40,6 +40,7 @@ def _fill(nbytes, stream_id):
 
 
 def _time(fn, iters, warmup=3, per_call_events=False):
+    iters = int(os.environ.get("PL_SUITE_ITERS", iters))  # short runs for profiler captures
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
@@ -287,8 +288,9 @@ def main(args=None):
                 b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30 if lg < 24 else 10,
                              graph=lg <= 21)
     if "c4" in which:
-        b.moe("C4", identity=False)
-        b.moe("C4", identity=True)
+        T = int(os.environ.get("PL_MOE_TOKENS", 4096))  # fewer tokens per rank for profiler captures
+        b.moe("C4", T=T, identity=False)
+        b.moe("C4", T=T, identity=True)
     if "c5" in which:
         for batch in (1, 8, 64):
             for algo in ("oneshot", "direct", "fused"):

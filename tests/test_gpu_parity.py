@@ -422,3 +422,43 @@ def test_sixteen_ranks(dp):
                 assert np.array_equal(outs[r], a2a[r].view(np.uint8))
         finally:
             ses.close()
+
+
+# ---- CUDA-graph replay: the epoch lives on the device, so a captured execute replays correctly ----
+@pytest.mark.parametrize("dp", DATAPATHS)
+def test_cuda_graph_replay_keeps_results_right(dp):
+    import torch
+    from gpu_harness import poison
+    R, n = 8, 8 * 6000
+    x = gen.rank_inputs(R, n, "bf16", seed=41)
+    ref = oracle.allreduce(x, "bf16")
+    ses = Session(R, "bf16")
+    try:
+        for algo in (B.PL_ALGO_RING, B.PL_ALGO_DIRECT):
+            s = ses.build(B.PL_ALLREDUCE, algo, n, 4096, datapath=dp)
+            info = B.pl_schedule_info(s)
+            d_in = [to_dev(a) for a in x]
+            d_out = [poison(info.out_bytes[r]) for r in range(R)]
+            bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                               [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
+            B.pl_execute(s, bufs, torch.cuda.current_stream().cuda_stream)   # one plain execute first
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(4):                                           # four executes per replay
+                    B.pl_execute(s, bufs, torch.cuda.current_stream().cuda_stream)
+            for _ in range(3):
+                for t in d_out:
+                    t.fill_(0xFF)
+                g.replay()
+                torch.cuda.synchronize()
+                assert B.pl_comm_status(ses.comm).code == B.PL_OK
+                outs = [d_out[r][: int(info.out_bytes[r])].cpu().numpy() for r in range(R)]
+                compare_reduce(outs, ref, "bf16")
+            B.pl_execute(s, bufs, torch.cuda.current_stream().cuda_stream)   # and a plain one after the replays
+            torch.cuda.synchronize()
+            compare_reduce([d_out[r][: int(info.out_bytes[r])].cpu().numpy() for r in range(R)], ref, "bf16")
+    finally:
+        ses.close()
