@@ -140,6 +140,10 @@ typedef struct {
   uint64_t timeout_ns;   /* bound of every device-side wait; 0 = 2 s                      */
   uint32_t flags;        /* PL_OPT_*                                                      */
   uint64_t staging_bytes; /* PL_OPT_STAGED: staging capacity per rank; 0 = min(256 MiB, need) */
+  float out_scale;       /* processing hook (Sec. 3.3, "processing phase ... while resident in   */
+                         /* registers"): every final sum is multiplied by this in fp32 before   */
+                         /* the one conversion to the element type, e.g. 1/R for an average.    */
+                         /* 0 = no scaling.  Float element types only (PL_ERR_UNSUPPORTED).     */
 } pl_sched_opts_t;
 #define PL_OPT_SKIP_VALIDATE 1u /* do not run the static validator inside build */
 /* Treat in/out as ORDINARY application buffers that peers must not touch (Sec. 3.2, "Protocol

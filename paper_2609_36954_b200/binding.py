@@ -48,7 +48,7 @@ class pl_sched_opts_t(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("n_ctas", C.c_int32), ("threads", C.c_int32),
                 ("datapath", C.c_int32), ("stages", C.c_int32), ("stage_bytes", C.c_uint32),
                 ("slice_bytes", C.c_uint32), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32),
-                ("staging_bytes", C.c_uint64)]
+                ("staging_bytes", C.c_uint64), ("out_scale", C.c_float)]
 
 
 class pl_ref_t(C.Structure):
@@ -162,12 +162,13 @@ def _check(st, where):
 
 
 def make_opts(n_ctas=0, threads=0, datapath=PL_DP_AUTO, stages=0, stage_bytes=0, slice_bytes=0,
-              timeout_ns=0, flags=0, staging_bytes=0):
+              timeout_ns=0, flags=0, staging_bytes=0, out_scale=0.0):
     o = pl_sched_opts_t()
     o.struct_size = C.sizeof(pl_sched_opts_t)
     o.n_ctas, o.threads, o.datapath, o.stages = n_ctas, threads, datapath, stages
     o.stage_bytes, o.slice_bytes, o.timeout_ns, o.flags = stage_bytes, slice_bytes, timeout_ns, flags
     o.staging_bytes = staging_bytes
+    o.out_scale = out_scale
     return o
 
 

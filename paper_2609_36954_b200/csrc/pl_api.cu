@@ -26,6 +26,7 @@ struct pl_schedule_s {
   pl_sched_info_t info{};
   uint64_t timeout_ns = 0;
   bool no_l2_hints = false;
+  float out_scale = 1.0f;
   // host copies in device (queue-major) order
   std::vector<DevOp> dev_ops;
   std::vector<uint32_t> queue_begin;
@@ -164,6 +165,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   Policy pol{};
   uint64_t timeout = 2000000000ull;
   uint32_t flags = 0;
+  float out_scale = 1.0f;
   if (opts) {
     if (opts->struct_size != sizeof(pl_sched_opts_t)) return PL_ERR_INVALID_ARG;
     pol.n_ctas = opts->n_ctas;
@@ -176,6 +178,10 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
     flags = opts->flags;
     rq.staged = (flags & PL_OPT_STAGED) != 0;
     rq.staging_bytes = opts->staging_bytes;
+    if (opts->out_scale != 0.0f) {
+      if (comm && comm->dtype != PL_BF16 && comm->dtype != PL_F32) return PL_ERR_UNSUPPORTED;
+      out_scale = opts->out_scale;
+    }
     if (pol.threads < 0 || pol.threads % 32 || pol.threads > exec_max_threads()) return PL_ERR_INVALID_ARG;
     if (pol.n_ctas < 0 || pol.stages < 0 || pol.stage_bytes % 16 || pol.slice_bytes % 16) return PL_ERR_INVALID_ARG;
     if (pol.datapath < PL_DP_AUTO || pol.datapath > PL_DP_TMA) return PL_ERR_INVALID_ARG;
@@ -211,6 +217,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   S->pol = pol;
   S->timeout_ns = timeout;
   S->no_l2_hints = (flags & PL_OPT_NO_L2_HINTS) != 0;
+  S->out_scale = out_scale;
   std::string err;
   pl_status_t st = lower(rq, &S->L, &err);
   if (st != PL_OK) {
@@ -515,6 +522,7 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   P.stage_bytes = s->pol.stage_bytes;
   // bulk stores stream out (evict-first), sources of copies are re-read by other ranks (evict-last)
   P.hints = s->no_l2_hints ? 0u : 6u;
+  P.out_scale = s->out_scale;
   cudaError_t le = s->pol.datapath == PL_DP_TMA
                        ? launch_exec_tma(s->comm->dtype, P, s->pol.n_ctas, static_cast<cudaStream_t>(stream))
                        : launch_exec(s->comm->dtype, P, s->pol.n_ctas, s->pol.threads, static_cast<cudaStream_t>(stream));

@@ -72,8 +72,8 @@ __device__ __forceinline__ void reduce_units(const ExecParams& P, const char* co
 #pragma unroll
   for (int u = 0; u < U; ++u) {
     uint4 r;
-    if constexpr (DT == PL_BF16) r = acc[u].to_bf16();
-    else r = acc[u].result();
+    if constexpr (DT == PL_BF16) r = acc[u].to_bf16(P.out_scale);
+    else r = acc[u].result(P.out_scale);
     if (!bcast) {
       st16(dst + off[u], r);
     } else {
@@ -125,7 +125,7 @@ __device__ __forceinline__ void body_copy_reduce(const ExecParams& P, const DevO
           acc.zero();
           acc.add(qa[u]);
           acc.add(qb[u]);
-          st16(dst + (i << 4), acc.result());
+          st16(dst + (i << 4), acc.result(P.out_scale));
         }
       }
     }
@@ -157,7 +157,7 @@ __device__ __forceinline__ void body_copy_reduce(const ExecParams& P, const DevO
             st16(dst + (i << 5), acc.sums());
             st16(dst + (i << 5) + 16, acc.corrections());
           } else {
-            st16(dst + (i << 4), acc.result());
+            st16(dst + (i << 4), acc.result(P.out_scale));
           }
         }
       }
@@ -191,7 +191,7 @@ __device__ __forceinline__ void body_copy_reduce(const ExecParams& P, const DevO
             st16(dst + (i << 5), lo);
             st16(dst + (i << 5) + 16, hi);
           } else {
-            st16(dst + (i << 4), acc.to_bf16());
+            st16(dst + (i << 4), acc.to_bf16(P.out_scale));
           }
         }
       }

@@ -145,8 +145,8 @@ __device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDe
       }
     } else {
       uint4 r;
-      if constexpr (DT == PL_BF16) r = acc.to_bf16();
-      else r = acc.result();
+      if constexpr (DT == PL_BF16) r = acc.to_bf16(P.out_scale);
+      else r = acc.result(P.out_scale);
       if (!bcast) {
         st16(d.dst + (size_t)u * 16u, r);
       } else if (pmask == 0) {

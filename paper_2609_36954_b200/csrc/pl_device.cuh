@@ -71,12 +71,13 @@ struct Acc<PL_BF16> {
     v[4] += __uint_as_float(hi.x); v[5] += __uint_as_float(hi.y);
     v[6] += __uint_as_float(hi.z); v[7] += __uint_as_float(hi.w);
   }
-  __device__ __forceinline__ uint4 to_bf16() const {
+  // final conversion; `scale` is the schedule's output scale (1 = plain sum, exact)
+  __device__ __forceinline__ uint4 to_bf16(float scale = 1.0f) const {
     uint4 q;
-    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
-    __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
-    __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]);
-    __nv_bfloat162 d = __floats2bfloat162_rn(v[6], v[7]);
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0] * scale, v[1] * scale);
+    __nv_bfloat162 b = __floats2bfloat162_rn(v[2] * scale, v[3] * scale);
+    __nv_bfloat162 c = __floats2bfloat162_rn(v[4] * scale, v[5] * scale);
+    __nv_bfloat162 d = __floats2bfloat162_rn(v[6] * scale, v[7] * scale);
     q.x = *reinterpret_cast<uint32_t*>(&a);
     q.y = *reinterpret_cast<uint32_t*>(&b);
     q.z = *reinterpret_cast<uint32_t*>(&c);
@@ -121,12 +122,12 @@ struct Acc<PL_F32> {
   __device__ __forceinline__ uint4 corrections() const {
     return make_uint4(__float_as_uint(c[0]), __float_as_uint(c[1]), __float_as_uint(c[2]), __float_as_uint(c[3]));
   }
-  __device__ __forceinline__ uint4 result() const {
+  __device__ __forceinline__ uint4 result(float scale = 1.0f) const {
     uint4 q;
-    q.x = __float_as_uint(__fadd_rn(v[0], c[0]));
-    q.y = __float_as_uint(__fadd_rn(v[1], c[1]));
-    q.z = __float_as_uint(__fadd_rn(v[2], c[2]));
-    q.w = __float_as_uint(__fadd_rn(v[3], c[3]));
+    q.x = __float_as_uint(__fmul_rn(__fadd_rn(v[0], c[0]), scale));
+    q.y = __float_as_uint(__fmul_rn(__fadd_rn(v[1], c[1]), scale));
+    q.z = __float_as_uint(__fmul_rn(__fadd_rn(v[2], c[2]), scale));
+    q.w = __float_as_uint(__fmul_rn(__fadd_rn(v[3], c[3]), scale));
     return q;
   }
 };
@@ -139,7 +140,7 @@ struct Acc<PL_I32> {
   __device__ __forceinline__ void add(const uint4& q) {
     v[0] += q.x; v[1] += q.y; v[2] += q.z; v[3] += q.w;
   }
-  __device__ __forceinline__ uint4 result() const { return make_uint4(v[0], v[1], v[2], v[3]); }
+  __device__ __forceinline__ uint4 result(float = 1.0f) const { return make_uint4(v[0], v[1], v[2], v[3]); }
 };
 
 // Record a timeout (first writer wins) and raise the abort word.

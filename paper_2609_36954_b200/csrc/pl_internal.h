@@ -83,6 +83,7 @@ struct ExecParams {
   int n_ranks;
   int stages;            // shared-memory ring depth of the TMA executor
   uint32_t stage_bytes;  // bytes per ring slot
+  float out_scale;       // multiplies every final (element-typed) sum; 1 = plain sum
   uint32_t hints;        // L2 policy bits for bulk copies: 1 loads evict-first, 2 stores evict-first, 4 copy loads evict-last
 };
 

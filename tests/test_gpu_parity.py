@@ -462,3 +462,44 @@ def test_cuda_graph_replay_keeps_results_right(dp):
             compare_reduce([d_out[r][: int(info.out_bytes[r])].cpu().numpy() for r in range(R)], ref, "bf16")
     finally:
         ses.close()
+
+
+# ---- processing hook: scaled sums (e.g. an average) ---------------------------------------------
+@pytest.mark.parametrize("dp", DATAPATHS)
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_output_scale_hook(dp, dtype):
+    R = 8
+    es = 2 if dtype == "bf16" else 4
+    n = R * ((24 * 1024 + 16) // es)
+    x = gen.rank_inputs(R, n, "f32n" if dtype == "f32" else dtype, seed=51)
+    scale = np.float32(1.0 / R)
+    ses = Session(R, dtype)
+    try:
+        ref = [a * float(scale) for a in oracle.allreduce(x, dtype)]            # the fp64 sums, scaled
+        for algo in ALL_AR:
+            s = ses.build(B.PL_ALLREDUCE, algo, n, 8192, datapath=dp, out_scale=float(scale))
+            outs, _ = ses.execute(s, x)
+            compare_reduce(outs, ref, dtype)
+        rs_ref = [a * float(scale) for a in oracle.reduce_scatter(x, dtype)]
+        s = ses.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_RING, n, 8192, datapath=dp, out_scale=float(scale))
+        outs, _ = ses.execute(s, x)
+        compare_reduce(outs, rs_ref, dtype)
+        s = B.pl_schedule_build_rooted(ses.comm, B.PL_REDUCE, 2, n, 8192, B.make_opts(datapath=dp, out_scale=float(scale)))
+        ses.scheds.append(s)
+        outs, _ = ses.execute(s, x)
+        check_float(as_f64(outs[2], dtype), oracle.reduce(x, 2, dtype)[2] * float(scale), dtype)
+        # copies are untouched by the hook
+        s = ses.build(B.PL_ALLTOALL, B.PL_ALGO_DIRECT, n, 8192, datapath=dp, out_scale=float(scale))
+        outs, _ = ses.execute(s, x)
+        a2a = oracle.alltoall(x)
+        for r in range(R):
+            assert np.array_equal(outs[r], a2a[r].view(np.uint8))
+    finally:
+        ses.close()
+    si = Session(4, "i32")
+    try:
+        with pytest.raises(B.PurlinError) as e:
+            si.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 1024, out_scale=0.5)
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+    finally:
+        si.close()
