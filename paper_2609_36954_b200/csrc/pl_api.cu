@@ -29,7 +29,6 @@ struct pl_schedule_s {
   float out_scale = 1.0f;
   // host copies in device (queue-major) order
   std::vector<DevOp> dev_ops;
-  std::vector<uint32_t> queue_begin;
   std::vector<uint64_t> srcs;
   std::vector<DevWait> waits;
   std::vector<int> topo_to_dev;  // topological index -> position in dev_ops
@@ -37,7 +36,7 @@ struct pl_schedule_s {
   // device
   char* d_blob = nullptr;
   size_t blob_bytes = 0;
-  size_t off_ops = 0, off_qb = 0, off_srcs = 0, off_waits = 0, off_flags = 0, off_epoch = 0;
+  size_t off_ops = 0, off_srcs = 0, off_waits = 0, off_flags = 0, off_epoch = 0;
   size_t sync_bytes = 0;  // flags + epoch, zeroed at build and by reset
   char* d_scratch = nullptr;
   uint64_t scratch_off[PL_MAX_RANKS] = {0};
@@ -80,33 +79,39 @@ void fill_info(pl_schedule_s* S, int R) {
   I.slice_bytes = S->pol.slice_bytes;
 }
 
-// Flatten the lowered ops into the queue-major device arrays (host side).
+// Flatten the lowered ops into the device arrays (host side): op i of queue q at index
+// i * n_queues + q, queues padded to the longest one, empty queues get one placeholder.
 void flatten(pl_schedule_s* S, int dtype) {
   const Lowered& L = S->L;
   const int nq = S->pol.n_ctas;
   size_t max_src = 1, max_wait = 1;
-  std::vector<uint32_t> qcount(nq + 1, 0);
+  std::vector<uint32_t> qlen(nq, 0);
   for (const HostOp& op : L.ops) {
     max_src = std::max(max_src, op.src.size());
     max_wait = std::max(max_wait, op.waits.size());
-    qcount[op.queue + 1]++;
+    qlen[op.queue]++;
   }
   S->src_stride = (uint32_t)max_src;
   S->wait_stride = (uint32_t)max_wait;
-  S->queue_begin.assign(nq + 1, 0);
-  for (int q = 0; q < nq; ++q) S->queue_begin[q + 1] = S->queue_begin[q] + qcount[q + 1];
-  std::vector<uint32_t> cursor(S->queue_begin.begin(), S->queue_begin.end() - 1);
-  const size_t n = L.ops.size();
-  S->dev_ops.assign(n, DevOp{});
+  uint32_t max_len = 1;
+  for (int q = 0; q < nq; ++q) max_len = std::max(max_len, qlen[q]);
+  const size_t n = (size_t)max_len * nq;
+  DevOp nop{};
+  nop.kind = kNopKind;
+  nop.signal = nop.signal2 = kNoFlag;
+  S->dev_ops.assign(n, nop);
   S->srcs.assign(n * max_src, 0);
   S->waits.assign(n * max_wait, DevWait{0, 0});
-  S->topo_to_dev.assign(n, 0);
+  S->topo_to_dev.assign(L.ops.size(), 0);
+  std::vector<uint32_t> cursor(nq, 0);
   for (const HostOp& op : L.ops) {  // topological order => per-queue order is a subsequence
-    const uint32_t pos = cursor[op.queue]++;
+    const uint32_t i = cursor[op.queue]++;
+    const size_t pos = (size_t)i * nq + op.queue;
     S->topo_to_dev[op.topo] = (int)pos;
     DevOp& d = S->dev_ops[pos];
     d.kind = op.kind;
     d.n_src = (uint32_t)op.src.size();
+    d.remaining = qlen[op.queue] - 1 - i;
     d.n_wait = (uint32_t)op.waits.size();
     d.signal = op.signal >= 0 ? (uint32_t)op.signal : kNoFlag;
     d.signal2 = op.signal2 >= 0 ? (uint32_t)op.signal2 : kNoFlag;
@@ -131,7 +136,6 @@ pl_status_t upload(pl_schedule_s* S, int R) {
     return o;
   };
   S->off_ops = place(S->dev_ops.size() * sizeof(DevOp));
-  S->off_qb = place(S->queue_begin.size() * sizeof(uint32_t));
   S->off_srcs = place(S->srcs.size() * sizeof(uint64_t));
   S->off_waits = place(S->waits.size() * sizeof(DevWait));
   S->off_flags = place((size_t)std::max(1, S->L.n_flags) * sizeof(unsigned long long));
@@ -141,7 +145,6 @@ pl_status_t upload(pl_schedule_s* S, int R) {
   if (cudaMalloc(&S->d_blob, S->blob_bytes) != cudaSuccess) { cudaGetLastError(); return PL_ERR_OOM; }
   std::vector<char> host(S->blob_bytes, 0);
   std::memcpy(host.data() + S->off_ops, S->dev_ops.data(), S->dev_ops.size() * sizeof(DevOp));
-  std::memcpy(host.data() + S->off_qb, S->queue_begin.data(), S->queue_begin.size() * sizeof(uint32_t));
   std::memcpy(host.data() + S->off_srcs, S->srcs.data(), S->srcs.size() * sizeof(uint64_t));
   std::memcpy(host.data() + S->off_waits, S->waits.data(), S->waits.size() * sizeof(DevWait));
   if (cudaMemcpy(S->d_blob, host.data(), S->blob_bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -508,12 +511,12 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
     P.base[kSlotScratch + r] = s->d_scratch ? s->d_scratch + s->scratch_off[r] : nullptr;
   }
   P.ops = reinterpret_cast<const DevOp*>(s->d_blob + s->off_ops);
-  P.queue_begin = reinterpret_cast<const uint32_t*>(s->d_blob + s->off_qb);
+  P.n_queues = (uint32_t)s->pol.n_ctas;
   P.srcs = reinterpret_cast<const uint64_t*>(s->d_blob + s->off_srcs);
   P.waits = reinterpret_cast<const DevWait*>(s->d_blob + s->off_waits);
   P.src_stride = s->src_stride;
   P.wait_stride = s->wait_stride;
-  P.flags = reinterpret_cast<unsigned long long*>(s->d_blob + s->off_flags);
+  P.flags = s->L.n_flags ? reinterpret_cast<unsigned long long*>(s->d_blob + s->off_flags) : nullptr;
   P.epoch = reinterpret_cast<unsigned long long*>(s->d_blob + s->off_epoch);
   P.status = s->comm->d_status;
   P.timeout_ns = s->timeout_ns;

@@ -211,18 +211,21 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   __shared__ OpSlot s_slot[2];
   __shared__ int s_abort[2];  // indexed by iteration parity: written during wait i, read after barrier i
   const int tid = threadIdx.x, nthr = blockDim.x, q = blockIdx.x;
-  const uint32_t qb = P.queue_begin[q], qe = P.queue_begin[q + 1];
+  const uint32_t nq = P.n_queues;
   // every CTA reads the epoch before it reports completion, and the epoch word is only
-  // advanced after all CTAs reported, so all of them see the same value
-  const unsigned long long epoch = *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull;
+  // advanced after all CTAs reported, so all of them see the same value; a schedule without
+  // flags needs no epoch at all
+  const bool has_flags = P.flags != nullptr;
+  const unsigned long long epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
   if (tid == 0) s_abort[0] = s_abort[1] = 0;
   bool aborted = false;
 
   // descriptor fetch by warp 0: lanes 0-3 carry the op, lane k source k and wait entry k
   auto fetch = [&](uint32_t i, uint4& r_op, uint64_t& r_src, DevWait& r_wait) {
-    if (tid < 4) r_op = reinterpret_cast<const uint4*>(P.ops + i)[tid];
-    if (tid < (int)P.src_stride) r_src = P.srcs[(uint64_t)i * P.src_stride + tid];
-    if (tid < (int)P.wait_stride) r_wait = P.waits[(uint64_t)i * P.wait_stride + tid];
+    const uint64_t at = (uint64_t)i * nq + q;  // op i of this queue
+    if (tid < 4) r_op = reinterpret_cast<const uint4*>(P.ops + at)[tid];
+    if (tid < (int)P.src_stride) r_src = P.srcs[at * P.src_stride + tid];
+    if (tid < (int)P.wait_stride) r_wait = P.waits[at * P.wait_stride + tid];
   };
   auto stash = [&](int slot, const uint4& r_op, uint64_t r_src, const DevWait& r_wait) {
     if (tid < 4) reinterpret_cast<uint4*>(&s_slot[slot].op)[tid] = r_op;
@@ -233,14 +236,16 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   uint4 r_op = make_uint4(0, 0, 0, 0);
   uint64_t r_src = 0;
   DevWait r_wait = {0, 0};
-  if (tid < 32 && qb < qe) {
-    fetch(qb, r_op, r_src, r_wait);
+  if (tid < 32) {
+    fetch(0, r_op, r_src, r_wait);
     stash(0, r_op, r_src, r_wait);
   }
   __syncthreads();
+  // the first descriptor tells how many ops the queue holds (a placeholder marks an empty one)
+  const uint32_t n_ops = s_slot[0].op.kind == kNopKind ? 0u : s_slot[0].op.remaining + 1u;
 
-  for (uint32_t i = qb; i < qe; ++i) {
-    const int slot = (i - qb) & 1;
+  for (uint32_t i = 0; i < n_ops; ++i) {
+    const int slot = i & 1;
     OpSlot& S = s_slot[slot];
     if (tid < 32) {
       // ---- wait: lane k polls wait entry k (acquire), bounded by the time limit
@@ -269,7 +274,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
     }
     __syncthreads();  // descriptor + satisfied waits visible to the CTA; previous body finished
     if (s_abort[slot]) { aborted = true; break; }
-    const bool has_next = i + 1 < qe;
+    const bool has_next = i + 1 < n_ops;
     if (tid < 32 && has_next) fetch(i + 1, r_op, r_src, r_wait);
 
     const DevOp& op = S.op;
@@ -296,7 +301,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   }
 
   __syncthreads();
-  if (tid == 0 && !aborted) {
+  if (tid == 0 && !aborted && has_flags) {
     // last CTA to finish advances the epoch for the next execute
     const unsigned long long prev = atomicAdd(P.epoch + 1, 1ull);
     if (prev == (unsigned long long)gridDim.x - 1ull) {

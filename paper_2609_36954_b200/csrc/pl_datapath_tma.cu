@@ -177,7 +177,8 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
   unsigned char* slots = smem + kCtrlBytes;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, q = blockIdx.x;
   const uint32_t S = (uint32_t)P.stages, slot_bytes = P.stage_bytes;
-  const unsigned long long epoch = *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull;
+  const bool has_flags = P.flags != nullptr;
+  const unsigned long long epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
 
   if (tid == 0) {
     for (uint32_t s = 0; s < S; ++s) {
@@ -192,24 +193,28 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
 
   if (warp == 0) {
     // ================================ producer =========================================
-    const uint32_t qb = P.queue_begin[q], qe = P.queue_begin[q + 1];
+    const uint32_t nq = P.n_queues;
     uint32_t n = 0;  // stages produced
     bool ok = true;
     uint4 r_op = make_uint4(0, 0, 0, 0), r_op_next = r_op;
     uint64_t r_src = 0, r_src_next = 0;
     DevWait r_wait = {0, 0}, r_wait_next = {0, 0};
     auto fetch = [&](uint32_t i, uint4& o, uint64_t& sr, DevWait& w) {
-      if (lane < 4) o = reinterpret_cast<const uint4*>(P.ops + i)[lane];
-      if (lane < (int)P.src_stride) sr = P.srcs[(uint64_t)i * P.src_stride + lane];
-      if (lane < (int)P.wait_stride) w = P.waits[(uint64_t)i * P.wait_stride + lane];
+      const uint64_t at = (uint64_t)i * nq + q;  // op i of this queue
+      if (lane < 4) o = reinterpret_cast<const uint4*>(P.ops + at)[lane];
+      if (lane < (int)P.src_stride) sr = P.srcs[at * P.src_stride + lane];
+      if (lane < (int)P.wait_stride) w = P.waits[at * P.wait_stride + lane];
     };
-    if (qb < qe) fetch(qb, r_op_next, r_src_next, r_wait_next);
-    for (uint32_t i = qb; i < qe && ok; ++i) {
+    fetch(0, r_op_next, r_src_next, r_wait_next);
+    // the first descriptor tells how many ops the queue holds (a placeholder marks an empty one)
+    const uint32_t first_kind = __shfl_sync(0xFFFFFFFFu, r_op_next.x, 0);
+    const uint32_t n_ops = first_kind == kNopKind ? 0u : __shfl_sync(0xFFFFFFFFu, r_op_next.z, 0) + 1u;
+    for (uint32_t i = 0; i < n_ops && ok; ++i) {
       r_op = r_op_next;
       r_src = r_src_next;
       r_wait = r_wait_next;
-      if (i + 1 < qe) fetch(i + 1, r_op_next, r_src_next, r_wait_next);
-      // op words: lane 0: kind n_src rsv pmask | lane 1: rsv n_wait signal flags | lane 2: count dst | lane 3: topo signal2
+      if (i + 1 < n_ops) fetch(i + 1, r_op_next, r_src_next, r_wait_next);
+      // op words: lane 0: kind n_src remaining pmask | lane 1: rsv n_wait signal flags | lane 2: count dst | lane 3: topo signal2
       const uint32_t kind = __shfl_sync(0xFFFFFFFFu, r_op.x, 0), n_src = __shfl_sync(0xFFFFFFFFu, r_op.y, 0);
       const uint32_t pmask = __shfl_sync(0xFFFFFFFFu, r_op.w, 0);
       const uint32_t n_wait = __shfl_sync(0xFFFFFFFFu, r_op.y, 1), signal = __shfl_sync(0xFFFFFFFFu, r_op.z, 1);
@@ -405,7 +410,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
   }
 
   __syncthreads();
-  if (tid == 0 && !*reinterpret_cast<volatile int*>(&c->abort)) {
+  if (tid == 0 && has_flags && !*reinterpret_cast<volatile int*>(&c->abort)) {
     const unsigned long long prev = atomicAdd(P.epoch + 1, 1ull);
     if (prev == (unsigned long long)gridDim.x - 1ull) {
       P.epoch[1] = 0ull;

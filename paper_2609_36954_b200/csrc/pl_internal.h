@@ -45,11 +45,12 @@ struct HostOp {
 constexpr int kSlotIn = 0, kSlotOut = PL_MAX_RANKS, kSlotScratch = 2 * PL_MAX_RANKS;
 constexpr int kNumSlots = 3 * PL_MAX_RANKS;
 constexpr uint32_t kNoFlag = 0xFFFFFFFFu;
+constexpr uint32_t kNopKind = 0xFFu;  // placeholder op of an empty queue
 
 struct alignas(16) DevOp {
   uint32_t kind;        // pl_op_kind_t
   uint32_t n_src;
-  uint32_t rsv0;
+  uint32_t remaining;   // ops that follow this one in its queue
   uint32_t src_f32_mask;  // bit p set: source p holds partials (fp32 for bf16 data, fp32 pairs for fp32 data)
   uint32_t rsv1;
   uint32_t n_wait;
@@ -71,12 +72,15 @@ struct DevWait {
 
 struct ExecParams {
   void* base[kNumSlots];
-  const DevOp* ops;             // queue-major order
-  const uint32_t* queue_begin;  // n_queues + 1 entries
+  // Op i of queue q sits at index i * n_queues + q (queues padded to the longest one), so a
+  // CTA finds its first op from its block index alone and learns the queue length from that
+  // op: no dependent load in front of the first descriptor.
+  const DevOp* ops;
+  uint32_t n_queues;
   const uint64_t* srcs;         // src_stride packed addresses per op (same order as ops)
   const DevWait* waits;         // wait_stride entries per op
   uint32_t src_stride, wait_stride;
-  unsigned long long* flags;    // one 64-bit counter per flag, monotone across executes
+  unsigned long long* flags;    // one 64-bit counter per flag, monotone across executes; null if the schedule has none
   unsigned long long* epoch;    // [0] executes completed, [1] CTAs finished in this execute
   int* status;                  // pl_devstatus_t words + abort word (comm-owned)
   unsigned long long timeout_ns;
