@@ -29,7 +29,11 @@
  *     nothing and never synchronises.  A schedule may be executed any number of times
  *     (flags carry a device-resident epoch; nothing is reset between executes).
  *   - One stream at a time per schedule: two executes of the same schedule must not
- *     overlap on the GPU.
+ *     overlap on the GPU.  Executes of DIFFERENT schedules may overlap only if their grids
+ *     together are co-resident (pl_schedule_info reports each grid): the CTAs of a launch
+ *     wait on one another, so two launches that each hold part of the SMs could starve each
+ *     other until the wait limit reports PL_ERR_TIMEOUT.  Issuing all executes on one stream
+ *     is always safe.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  */
 #ifndef PURLIN_H_
