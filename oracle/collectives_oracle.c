@@ -266,3 +266,60 @@ int orc_moe_combine_f64(int R, int T, int H, int E, int K, const void *const *y,
   }
   return 0;
 }
+
+/*
+ * MoE dispatch / combine with per-rank deduplication (the variant used when several of a
+ * token's experts live on the same rank: the token row crosses to that rank once).
+ *
+ * Dispatch: rank r receives ONE row for every (source p, token t) that selects at least one
+ * expert on r, in (p, t) order.  meta[r][row] = {p, t, slot mask, r}: bit j of the mask is set
+ * when slot j's expert lives on r.  pos[p][t*R + r] = row at rank r, or -1.
+ * counts[p*R + r] = rows p -> r.  Returns 2 on receive overflow.
+ *
+ * Combine: each rank returns one row per received row (the expert layer has already applied
+ * the gates and summed its local experts); out_p[t][h] = sum over r ascending with
+ * pos[p][t*R+r] >= 0 of z_r[pos][h], in fp64.
+ */
+int orc_moe_dispatch_dedup(int R, int T, int E, int K, size_t row_bytes, size_t recv_capacity_rows,
+                           const void *const *x, const int32_t *const *idx, void *const *recv,
+                           int32_t *const *meta, int32_t *const *pos, int64_t *counts) {
+  const int epr = E / R;
+  if (epr * R != E || K > 32) return 1;
+  memset(counts, 0, sizeof(int64_t) * (size_t)R * R);
+  for (int r = 0; r < R; ++r) {
+    size_t row = 0;
+    for (int p = 0; p < R; ++p)
+      for (int t = 0; t < T; ++t) {
+        uint32_t mask = 0;
+        for (int j = 0; j < K; ++j)
+          if (idx[p][(size_t)t * K + j] / epr == r) mask |= 1u << j;
+        if (!mask) {
+          pos[p][(size_t)t * R + r] = -1;
+          continue;
+        }
+        if (row >= recv_capacity_rows) return 2;
+        memcpy((uint8_t *)recv[r] + row * row_bytes, (const uint8_t *)x[p] + (size_t)t * row_bytes, row_bytes);
+        int32_t *m = meta[r] + row * 4;
+        m[0] = p; m[1] = t; m[2] = (int32_t)mask; m[3] = r;
+        pos[p][(size_t)t * R + r] = (int32_t)row;
+        counts[(size_t)p * R + r] += 1;
+        ++row;
+      }
+  }
+  return 0;
+}
+
+int orc_moe_combine_dedup_f64(int R, int T, int H, const void *const *z, const int32_t *const *pos,
+                              double *const *out) {
+  for (int p = 0; p < R; ++p)
+    for (int t = 0; t < T; ++t)
+      for (int h = 0; h < H; ++h) {
+        double acc = 0.0;
+        for (int r = 0; r < R; ++r) {
+          int32_t row = pos[p][(size_t)t * R + r];
+          if (row >= 0) acc += load_as_f64(z[r], ORC_BF16, (size_t)row * H + h);
+        }
+        out[p][(size_t)t * H + h] = acc;
+      }
+  return 0;
+}

@@ -232,3 +232,30 @@ def moe_combine(y, idx, pos, gates, E, H):
     rc = lib().orc_moe_combine_f64(R, T, H, E, K, _ptrs(y), _ptrs(idx), _ptrs(pos), _ptrs(gates), _ptrs(outs))
     _check(rc, "moe_combine")
     return outs
+
+
+def moe_dispatch_dedup(x, idx, E, recv_capacity_rows=None):
+    """One row per (token, destination rank).  Returns dict(recv, meta, pos [T, R], counts)."""
+    R = len(x)
+    T, K = idx[0].shape
+    row_bytes = x[0].shape[1] * x[0].itemsize
+    cap = recv_capacity_rows if recv_capacity_rows is not None else R * T
+    recv = [np.zeros((cap, x[0].shape[1]), dtype=x[0].dtype) for _ in range(R)]
+    meta = [np.full((cap, 4), -1, dtype=np.int32) for _ in range(R)]
+    pos = [np.full((T, R), -1, dtype=np.int32) for _ in range(R)]
+    counts = np.zeros((R, R), dtype=np.int64)
+    rc = lib().orc_moe_dispatch_dedup(R, T, E, K, ctypes.c_size_t(row_bytes), ctypes.c_size_t(cap),
+                                      _ptrs(x), _ptrs(idx), _ptrs(recv), _ptrs(meta), _ptrs(pos),
+                                      counts.ctypes.data_as(ctypes.c_void_p))
+    _check(rc, "moe_dispatch_dedup")
+    return dict(recv=recv, meta=meta, pos=pos, counts=counts)
+
+
+def moe_combine_dedup(z, pos, H):
+    """z[r]: uint16 bf16 rows [cap, H] (one per received row); returns fp64 out[p] [T, H]."""
+    R = len(z)
+    T = pos[0].shape[0]
+    outs = [np.empty((T, H), dtype=np.float64) for _ in range(R)]
+    rc = lib().orc_moe_combine_dedup_f64(R, T, H, _ptrs(z), _ptrs(pos), _ptrs(outs))
+    _check(rc, "moe_combine_dedup")
+    return outs

@@ -183,6 +183,12 @@ class Bench:
         disp, _, _ = _time(lambda: B.pl_moe_dispatch(plan, px, pi, pr, pm, self.stream), iters, per_call_events=True)
         comb, _, _ = _time(lambda: B.pl_moe_combine(plan, pr, pg, po, self.stream), iters, per_call_events=True)
         st = B.pl_moe_plan_read(plan, 0, 0, 0, self.stream)
+        # deduplicated variant on the same plan: one row per (token, destination rank)
+        dd, _, _ = _time(lambda: B.pl_moe_dispatch_dedup(plan, px, pi, pr, pm, self.stream), iters, per_call_events=True)
+        dc, _, _ = _time(lambda: B.pl_moe_combine_dedup(plan, pr, po, self.stream), iters, per_call_events=True)
+        cnt = np.zeros((R, R), np.int64)
+        B.pl_moe_plan_read_dedup(plan, 0, cnt.ctypes.data, self.stream)
+        rows_dd = int(cnt.sum())
         rows = R * T * K
         row_b = H * 2
         d_bytes = R * T * row_b + rows * row_b
@@ -192,7 +198,10 @@ class Bench:
                    "dispatch_us": disp, "combine_us": comb,
                    "dispatch_gbs": d_bytes / disp / 1e3, "combine_gbs": c_bytes / comb / 1e3,
                    "dispatch_frac_measured": d_bytes / disp / 1e3 / self.peak,
-                   "combine_frac_measured": c_bytes / comb / 1e3 / self.peak, "status": int(st)})
+                   "combine_frac_measured": c_bytes / comb / 1e3 / self.peak, "status": int(st),
+                   "dedup_rows": rows_dd, "dedup_dispatch_us": dd, "dedup_combine_us": dc,
+                   "dedup_dispatch_gbs": (R * T + rows_dd) * H * 2 / dd / 1e3,
+                   "dedup_combine_gbs": (R * T + rows_dd) * H * 2 / dc / 1e3})
         B.pl_moe_plan_destroy(plan)
         B.pl_comm_destroy(comm)
 

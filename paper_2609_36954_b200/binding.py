@@ -92,6 +92,7 @@ EXPORTS = [
     "pl_schedule_destroy",
     "pl_execute", "pl_execute_host",
     "pl_moe_plan_create", "pl_moe_plan_destroy", "pl_moe_dispatch", "pl_moe_combine", "pl_moe_plan_read",
+    "pl_moe_dispatch_dedup", "pl_moe_combine_dedup", "pl_moe_plan_read_dedup",
     "pl_status_string", "pl_launch_count", "pl_reduce_scatter_ring_static",
 ]
 
@@ -138,6 +139,9 @@ def load():
         "pl_moe_dispatch": [vp, P(vp), P(vp), P(vp), P(vp), vp],
         "pl_moe_combine": [vp, P(vp), P(vp), P(vp), vp],
         "pl_moe_plan_read": [vp, vp, vp, vp, vp],
+        "pl_moe_dispatch_dedup": [vp, P(vp), P(vp), P(vp), P(vp), vp],
+        "pl_moe_combine_dedup": [vp, P(vp), P(vp), vp],
+        "pl_moe_plan_read_dedup": [vp, vp, vp, vp],
         "pl_reduce_scatter_ring_static": [i32, i32, sz, P(vp), P(vp), vp, vp],
     }
     for name, args in sig.items():
@@ -309,6 +313,20 @@ def pl_moe_dispatch(plan, x, topk_idx, recv, recv_meta=None, stream=0):
 def pl_moe_combine(plan, y, gates, out, stream=0):
     _check(load().pl_moe_combine(plan, _ptr_array(y), _ptr_array(gates), _ptr_array(out), stream),
            "pl_moe_combine")
+
+
+def pl_moe_dispatch_dedup(plan, x, topk_idx, recv, recv_meta=None, stream=0):
+    meta = _ptr_array(recv_meta) if recv_meta is not None else None
+    _check(load().pl_moe_dispatch_dedup(plan, _ptr_array(x), _ptr_array(topk_idx), _ptr_array(recv), meta, stream),
+           "pl_moe_dispatch_dedup")
+
+
+def pl_moe_combine_dedup(plan, z, out, stream=0):
+    _check(load().pl_moe_combine_dedup(plan, _ptr_array(z), _ptr_array(out), stream), "pl_moe_combine_dedup")
+
+
+def pl_moe_plan_read_dedup(plan, pos=0, counts=0, stream=0):
+    return load().pl_moe_plan_read_dedup(plan, pos or None, counts or None, stream)
 
 
 def pl_moe_plan_read(plan, pos=0, counts=0, expert_counts=0, stream=0):

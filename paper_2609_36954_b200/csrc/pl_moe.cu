@@ -12,6 +12,7 @@
 
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "pl_api_internal.h"
 #include "pl_internal.h"
@@ -48,6 +49,7 @@ struct MoeGeo {
   int32_t* pos;        // [R][T][K] row in the destination's receive buffer, -1 if dropped
   int32_t* prank;      // [R][T][K] destination rank
   int* flags;          // [0] overflow, [1] invalid expert id, [2] copy engine wait gave up
+  const int32_t* slotmask;  // optional [R][T][K]: written into the metadata instead of the slot index
 };
 
 __device__ __forceinline__ void build_mask(const MoeGeo& g, const int32_t* idx, uint32_t* mask, int t, int tid) {
@@ -56,7 +58,8 @@ __device__ __forceinline__ void build_mask(const MoeGeo& g, const int32_t* idx, 
   if (t < g.T)
     for (int j = 0; j < g.K; ++j) {
       const int e = idx[(size_t)t * g.K + j];
-      if ((unsigned)e < (unsigned)g.E) atomicOr(&mask[e * kMaskWords + (tid >> 5)], 1u << (tid & 31));
+      if (e < 0) continue;  // empty slot (deduplicated routing pads with -1)
+      if (e < g.E) atomicOr(&mask[e * kMaskWords + (tid >> 5)], 1u << (tid & 31));
       else g.flags[1] = 1;
     }
   __syncthreads();
@@ -129,10 +132,43 @@ __global__ void __launch_bounds__(kTB) moe_place_kernel(const __grid_constant__ 
     g.prank[o] = r;
     if ((unsigned long long)row < g.cap) {
       g.pos[o] = (int32_t)row;
-      if (P.meta[r]) reinterpret_cast<int4*>(P.meta[r])[row] = make_int4(p, t, j, e);
+      if (P.meta[r]) reinterpret_cast<int4*>(P.meta[r])[row] = make_int4(p, t, g.slotmask ? g.slotmask[o] : j, e);
     } else {
       g.pos[o] = -1;
     }
+  }
+}
+
+// Deduplicated routing: for every token the distinct destination ranks in ascending order
+// (padded with -1) and, per destination, the mask of slots whose expert lives there.
+__global__ void __launch_bounds__(256) moe_derive_ranks_kernel(const __grid_constant__ DispatchPtrs P, int R, int T, int K,
+                                                               int epr, int KR, int32_t* ridx, int32_t* rmask) {
+  const long long tok = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (tok >= (long long)R * T) return;
+  const int p = (int)(tok / T);
+  const long long t = tok % T;
+  const int32_t* idx = P.idx[p] + t * K;
+  unsigned masks[PL_MAX_RANKS];
+#pragma unroll
+  for (int r = 0; r < PL_MAX_RANKS; ++r) masks[r] = 0u;
+  for (int j = 0; j < K; ++j) {
+    const int e = idx[j];
+    const int r = (e >= 0) ? e / epr : -1;
+#pragma unroll
+    for (int q = 0; q < PL_MAX_RANKS; ++q)
+      if (q == r) masks[q] |= 1u << j;
+  }
+  int n = 0;
+#pragma unroll
+  for (int r = 0; r < PL_MAX_RANKS; ++r)
+    if (r < R && masks[r]) {
+      ridx[tok * KR + n] = r;
+      rmask[tok * KR + n] = (int32_t)masks[r];
+      ++n;
+    }
+  for (; n < KR; ++n) {
+    ridx[tok * KR + n] = -1;
+    rmask[tok * KR + n] = 0;
   }
 }
 
@@ -306,6 +342,13 @@ struct pl_moe_plan_s {
   int sm_count = 148;
   size_t move_smem = 0;
   bool dispatched = false;
+  // deduplicated variant: the same machinery run over "one expert per rank" routing
+  MoeGeo gd{};
+  int32_t* d_ridx = nullptr;   // [R][T][KR] distinct destination ranks, -1 padded
+  int32_t* d_rmask = nullptr;  // [R][T][KR] slot masks
+  float* d_ones = nullptr;     // [T][KR] unit gates
+  char* d_blob2 = nullptr;
+  bool dispatched_dedup = false;
 };
 
 extern "C" {
@@ -363,6 +406,43 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
     delete pl;
     return PL_ERR_CUDA;
   }
+  // second set of bookkeeping for the deduplicated variant: R "experts" (one per rank),
+  // at most min(topk, R) destinations per token
+  {
+    MoeGeo& d = pl->gd;
+    d = g;
+    d.E = R;
+    d.epr = 1;
+    d.K = std::min(topk, R);
+    size_t off2 = 0;
+    auto place2 = [&](size_t bytes) { size_t o = off2; off2 = align_up(off2 + bytes, 256); return o; };
+    const size_t tk = (size_t)R * g.T * d.K;
+    const size_t q_bc = place2((size_t)R * g.NB * R * 4), q_base = place2((size_t)R * R * 4);
+    const size_t q_cnt = place2((size_t)R * R * 8), q_ecnt = place2((size_t)R * R * 8);
+    const size_t q_pos = place2(tk * 4), q_prank = place2(tk * 4), q_ridx = place2(tk * 4), q_rmask = place2(tk * 4);
+    const size_t q_ones = place2((size_t)g.T * d.K * 4), q_flags = place2(16);
+    if (cudaMalloc(&pl->d_blob2, off2) != cudaSuccess) { cudaGetLastError(); cudaFree(pl->d_blob); delete pl; return PL_ERR_OOM; }
+    std::vector<float> ones((size_t)g.T * d.K, 1.0f);
+    if (cudaMemset(pl->d_blob2, 0, off2) != cudaSuccess ||
+        cudaMemcpy(pl->d_blob2 + q_ones, ones.data(), ones.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) {
+      cudaGetLastError();
+      cudaFree(pl->d_blob);
+      cudaFree(pl->d_blob2);
+      delete pl;
+      return PL_ERR_CUDA;
+    }
+    d.blockcnt = reinterpret_cast<int32_t*>(pl->d_blob2 + q_bc);
+    d.base = reinterpret_cast<int32_t*>(pl->d_blob2 + q_base);
+    d.counts = reinterpret_cast<long long*>(pl->d_blob2 + q_cnt);
+    d.ecounts = reinterpret_cast<long long*>(pl->d_blob2 + q_ecnt);
+    d.pos = reinterpret_cast<int32_t*>(pl->d_blob2 + q_pos);
+    d.prank = reinterpret_cast<int32_t*>(pl->d_blob2 + q_prank);
+    d.flags = reinterpret_cast<int*>(pl->d_blob2 + q_flags);
+    pl->d_ridx = reinterpret_cast<int32_t*>(pl->d_blob2 + q_ridx);
+    pl->d_rmask = reinterpret_cast<int32_t*>(pl->d_blob2 + q_rmask);
+    pl->d_ones = reinterpret_cast<float*>(pl->d_blob2 + q_ones);
+    d.slotmask = pl->d_rmask;
+  }
   comm->n_plans += 1;
   *out = pl;
   return PL_OK;
@@ -371,6 +451,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
 pl_status_t pl_moe_plan_destroy(pl_moe_plan_t plan) {
   if (!plan) return PL_ERR_INVALID_ARG;
   if (plan->d_blob) cudaFree(plan->d_blob);
+  if (plan->d_blob2) cudaFree(plan->d_blob2);
   plan->comm->n_plans -= 1;
   delete plan;
   return PL_OK;
@@ -439,6 +520,91 @@ pl_status_t pl_moe_plan_read(pl_moe_plan_t plan, int32_t* pos, int64_t* counts, 
   if (ok && pos) ok = cudaMemcpy(pos, g.pos, (size_t)g.R * g.T * g.K * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
   if (ok && counts) ok = cudaMemcpy(counts, g.counts, (size_t)g.R * g.R * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
   if (ok && expert_counts) ok = cudaMemcpy(expert_counts, g.ecounts, (size_t)g.R * g.E * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return PL_ERR_CUDA; }
+  if (flags[2]) return PL_ERR_TIMEOUT;
+  if (flags[1]) return PL_ERR_INVALID_ARG;
+  if (flags[0]) return PL_ERR_OVERFLOW;
+  return PL_OK;
+}
+
+pl_status_t pl_moe_dispatch_dedup(pl_moe_plan_t plan, const void* const* x, const int32_t* const* topk_idx,
+                                  void* const* recv, int32_t* const* recv_meta, void* stream) {
+  if (!plan || !x || !topk_idx || !recv) return PL_ERR_INVALID_ARG;
+  const MoeGeo& g = plan->g;
+  const MoeGeo& d = plan->gd;
+  DispatchPtrs P0, P;
+  std::memset(&P0, 0, sizeof(P0));
+  std::memset(&P, 0, sizeof(P));
+  for (int r = 0; r < g.R; ++r) {
+    if (!x[r] || !topk_idx[r] || !recv[r]) return PL_ERR_INVALID_ARG;
+    if (((uintptr_t)x[r] & 15) || ((uintptr_t)recv[r] & 15) || ((uintptr_t)topk_idx[r] & 3)) return PL_ERR_ALIGNMENT;
+    if (recv_meta && recv_meta[r] && ((uintptr_t)recv_meta[r] & 15)) return PL_ERR_ALIGNMENT;
+    P0.idx[r] = topk_idx[r];
+    P.x[r] = x[r];
+    P.idx[r] = plan->d_ridx + (size_t)r * g.T * d.K;  // the derived per-rank routing
+    P.recv[r] = recv[r];
+    P.meta[r] = recv_meta ? recv_meta[r] : nullptr;
+  }
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const long long n_tok = (long long)g.R * g.T;
+  moe_derive_ranks_kernel<<<(unsigned)((n_tok + 255) / 256), 256, 0, cs>>>(P0, g.R, g.T, g.K, g.epr, d.K, plan->d_ridx, plan->d_rmask);
+  const size_t mask_smem = (size_t)d.E * kMaskWords * 4;
+  dim3 grid(d.NB, d.R);
+  moe_count_kernel<<<grid, kTB, mask_smem, cs>>>(P, d);
+  moe_scan_kernel<<<1, 1024, 0, cs>>>(d);
+  moe_place_kernel<<<grid, kTB, mask_smem, cs>>>(P, d);
+  const unsigned long long items = (unsigned long long)d.R * d.T * d.n_tiles;
+  const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, (200 * 1024) / plan->move_smem));
+  const int mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)plan->sm_count * per_sm);
+  moe_move_kernel<<<mgrid, 32, plan->move_smem, cs>>>(P, d);
+  if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
+  g_launches.fetch_add(5);
+  plan->dispatched_dedup = true;
+  return PL_OK;
+}
+
+pl_status_t pl_moe_combine_dedup(pl_moe_plan_t plan, const void* const* z, void* const* out, void* stream) {
+  if (!plan || !z || !out) return PL_ERR_INVALID_ARG;
+  if (plan->comm->dtype != PL_BF16) return PL_ERR_UNSUPPORTED;
+  if (!plan->dispatched_dedup) return PL_ERR_INVALID_ARG;
+  const MoeGeo& d = plan->gd;
+  CombinePtrs P;
+  std::memset(&P, 0, sizeof(P));
+  for (int r = 0; r < d.R; ++r) {
+    if (!z[r] || !out[r]) return PL_ERR_INVALID_ARG;
+    if (((uintptr_t)z[r] & 15) || ((uintptr_t)out[r] & 15)) return PL_ERR_ALIGNMENT;
+    P.y[r] = z[r];
+    P.gates[r] = plan->d_ones;  // the expert layer has already applied the gates
+    P.out[r] = out[r];
+  }
+  const unsigned long long n_tok = (unsigned long long)d.R * d.T;
+  const int grid = (int)std::min<unsigned long long>(n_tok, (unsigned long long)plan->sm_count * 6);
+  moe_combine_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(P, d);
+  if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return PL_OK;
+}
+
+pl_status_t pl_moe_plan_read_dedup(pl_moe_plan_t plan, int32_t* pos, int64_t* counts, void* stream) {
+  if (!plan) return PL_ERR_INVALID_ARG;
+  const MoeGeo& d = plan->gd;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  int flags[4] = {0, 0, 0, 0};
+  bool ok = cudaMemcpy(flags, d.flags, 12, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (ok && counts) ok = cudaMemcpy(counts, d.counts, (size_t)d.R * d.R * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (ok && pos) {
+    const size_t tk = (size_t)d.R * d.T * d.K;
+    std::vector<int32_t> ridx(tk), rpos(tk);
+    ok = cudaMemcpy(ridx.data(), plan->d_ridx, tk * 4, cudaMemcpyDeviceToHost) == cudaSuccess &&
+         cudaMemcpy(rpos.data(), d.pos, tk * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (ok) {
+      const size_t n_tok = (size_t)d.R * d.T;
+      for (size_t i = 0; i < n_tok * d.R; ++i) pos[i] = -1;
+      for (size_t t = 0; t < n_tok; ++t)
+        for (int j = 0; j < d.K; ++j)
+          if (ridx[t * d.K + j] >= 0) pos[t * d.R + ridx[t * d.K + j]] = rpos[t * d.K + j];
+    }
+  }
   if (!ok) { cudaGetLastError(); return PL_ERR_CUDA; }
   if (flags[2]) return PL_ERR_TIMEOUT;
   if (flags[1]) return PL_ERR_INVALID_ARG;

@@ -172,3 +172,50 @@ def test_moe_sixteen_ranks_topk_32():
             check_float(gen.bf16_bits_to_f64(out[p]), want[p], "bf16")
     finally:
         run.close()
+
+
+# ---- deduplicated variant: one row per (token, destination rank) ------------------------------
+@pytest.mark.parametrize("R,T,H,E,K,ident", [(8, 300, 512, 64, 8, False), (4, 700, 7168, 32, 4, True), (2, 40, 8, 8, 4, False)])
+def test_dedup_dispatch_and_combine(R, T, H, E, K, ident):
+    idx, _ = gen.moe_routing(R, T, E, K, seed=4, identity_perm=ident)
+    x = gen.moe_tokens_bf16(R, T, H, seed=6)
+    cap = R * T
+    ref = oracle.moe_dispatch_dedup(x, idx, E, recv_capacity_rows=cap)
+    run = MoeRun(R, T, H, E, K, cap)
+    try:
+        d_x = [to_dev(a) for a in x]
+        d_i = [to_dev(a) for a in idx]
+        for rep in range(2):
+            d_recv = [poison(cap * H * 2) for _ in range(R)]
+            d_meta = [poison(cap * 16) for _ in range(R)]
+            B.pl_moe_dispatch_dedup(run.plan, [t.data_ptr() for t in d_x], [t.data_ptr() for t in d_i],
+                                    [t.data_ptr() for t in d_recv], [t.data_ptr() for t in d_meta], stream_handle())
+            pos = np.zeros((R, T, R), np.int32)
+            counts = np.zeros((R, R), np.int64)
+            assert B.pl_moe_plan_read_dedup(run.plan, pos.ctypes.data, counts.ctypes.data, stream_handle()) == B.PL_OK
+            assert np.array_equal(counts, ref["counts"])
+            for p in range(R):
+                assert np.array_equal(pos[p], ref["pos"][p])
+            for r in range(R):
+                n = int(counts[:, r].sum())
+                got = d_recv[r].cpu().numpy().view(np.uint16).reshape(cap, H)
+                assert np.array_equal(got[:n], ref["recv"][r][:n])
+                assert np.all(d_recv[r].cpu().numpy().reshape(cap, -1)[n:] == 0xFF)
+                assert np.array_equal(d_meta[r].cpu().numpy().view(np.int32).reshape(cap, 4)[:n], ref["meta"][r][:n])
+        # fewer rows cross than without deduplication
+        assert counts.sum() <= R * T * K
+        # combine: every destination returns one row per received row
+        z = [gen.normal_bf16(cap * H, 90, r).reshape(cap, H) for r in range(R)]
+        d_z = [to_dev(a) for a in z]
+        d_out = [poison(T * H * 2) for _ in range(R)]
+        B.pl_moe_combine_dedup(run.plan, [t.data_ptr() for t in d_z], [t.data_ptr() for t in d_out], stream_handle())
+        torch.cuda.synchronize()
+        want = oracle.moe_combine_dedup(z, ref["pos"], H)
+        for p in range(R):
+            got = gen.bf16_bits_to_f64(d_out[p].cpu().numpy().view(np.uint16).reshape(T, H))
+            check_float(got, want[p], "bf16")
+        # the plain dispatch on the same plan still works afterwards
+        st, recv, *_ = run.dispatch(x, idx, with_meta=False)
+        assert st == B.PL_OK or st == B.PL_ERR_OVERFLOW  # cap = R*T rows may be too small for K rows per token
+    finally:
+        run.close()

@@ -377,3 +377,53 @@ def test_rooted_collectives_against_their_unrooted_relatives(root):
     for r in range(R):
         assert np.array_equal(bc[r], xi[root])
     assert np.array_equal(oracle.gather(sc, root)[root], xi[root])
+
+
+# ----------------------------------------------------------------------------- #
+# MoE with per-rank deduplication
+# ----------------------------------------------------------------------------- #
+def test_moe_dedup_dispatch_and_combine():
+    R, T, E, K, H = 4, 48, 16, 4, 8
+    idx, _ = inputs.moe_routing(R, T, E, K, seed=12)
+    epr = E // R
+    x = [np.stack([np.full(2, p * 1000 + t, dtype=np.int32) for t in range(T)]) for p in range(R)]
+    d = oracle.moe_dispatch_dedup(x, idx, E)
+    plain = oracle.moe_dispatch(x, idx, E)
+    for r in range(R):
+        n = int(d["counts"][:, r].sum())
+        meta = d["meta"][r][:n]
+        # the (source, token) pairs that reach rank r: the distinct ones of the plain dispatch, in (p, t) order
+        pm = plain["meta"][r][: int(plain["counts"][:, r].sum())]
+        want = sorted({(int(a), int(b)) for a, b in pm[:, :2].tolist()})
+        assert [tuple(v) for v in meta[:, :2].tolist()] == want
+        assert np.array_equal(d["recv"][r][:n, 0], meta[:, 0] * 1000 + meta[:, 1])
+        # the slot mask names exactly the slots whose expert lives on r
+        for (p, t, mask, rr) in meta.tolist():
+            assert rr == r and mask == sum(1 << j for j in range(K) if idx[p][t, j] // epr == r)
+    # rows sent by p = number of distinct destination ranks over its tokens
+    for p in range(R):
+        distinct = sum(len(set((idx[p][t] // epr).tolist())) for t in range(T))
+        assert int(d["counts"][p].sum()) == distinct
+        assert distinct <= T * K
+    # pos is the inverse map, -1 where the token does not go
+    for p in range(R):
+        for t in (0, T - 1):
+            for r in range(R):
+                row = d["pos"][p][t, r]
+                assert (row >= 0) == (r in set((idx[p][t] // epr).tolist()))
+                if row >= 0:
+                    assert d["meta"][r][row][:2].tolist() == [p, t]
+    # combine over identity rows: every destination returns the token, so out = (#ranks) * x
+    xb = inputs.moe_tokens_bf16(R, T, H, seed=3)
+    db = oracle.moe_dispatch_dedup(xb, idx, E)
+    out = oracle.moe_combine_dedup(db["recv"], db["pos"], H)
+    for p in range(R):
+        nr = np.array([len(set((idx[p][t] // epr).tolist())) for t in range(T)], dtype=np.float64)
+        assert np.array_equal(out[p], inputs.bf16_bits_to_f64(xb[p]) * nr[:, None])
+    # one expert per rank and K = 1: deduplication changes nothing
+    idx1 = [np.random.default_rng(p).integers(0, R, size=(T, 1)).astype(np.int32) for p in range(R)]
+    a = oracle.moe_dispatch_dedup(x, idx1, R)
+    b = oracle.moe_dispatch(x, idx1, R)
+    for r in range(R):
+        n = int(a["counts"][:, r].sum())
+        assert np.array_equal(a["recv"][r][:n], b["recv"][r][:n]) and np.array_equal(a["counts"], b["counts"])
