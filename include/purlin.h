@@ -161,6 +161,9 @@ typedef struct {
  * can start the next call early; here a launch ends only when every rank has drained, so one
  * buffer is enough.) */
 #define PL_OPT_STAGED 4u
+/* Record, for every op, when its waits were satisfied and when its signal was about to be
+ * released (%globaltimer, ns) into a schedule-owned buffer: see pl_schedule_trace_read. */
+#define PL_OPT_TRACE 8u
 #define PL_OPT_NO_L2_HINTS 2u  /* bulk copies without L2 eviction hints (default: stores evict-first,
                                   sources of copy ops evict-last; measured 7 % on all-gather) */
 
@@ -310,6 +313,14 @@ pl_status_t pl_schedule_dump(pl_schedule_t s, pl_op_t* ops, size_t cap, size_t* 
  * the topological order, queue order embeds in that order.  On failure returns
  * PL_ERR_INVALID_SCHEDULE and writes a message into msg (may be NULL). */
 pl_status_t pl_schedule_validate(pl_schedule_t s, char* msg, size_t msg_cap);
+
+/* Copy the trace of the LAST execute to a HOST array of 2 * n_ops entries (index 2*i = start of
+ * op i in topological order: the moment its waits were satisfied; 2*i+1 = end: the moment just
+ * before its signal was released; the bulk-copy executor stamps the end only for ops that
+ * signal, others read 0).  Needs PL_OPT_TRACE at build (PL_ERR_INVALID_ARG otherwise).
+ * Synchronises `stream`.  Useful to see where a schedule's time goes and to check on the real
+ * device that every waiter started after all of its signallers ended. */
+pl_status_t pl_schedule_trace_read(pl_schedule_t s, uint64_t* out, size_t cap_entries, void* stream);
 
 /* TEST HOOK: remove the first wait edge of op `op_index` from the host copy of the schedule,
  * so that pl_schedule_validate can be shown to notice the missing ordering.  The device copy

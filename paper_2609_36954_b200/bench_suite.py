@@ -125,11 +125,23 @@ class Bench:
         if graph:
             graph_us = _time_graph(lambda h: B.pl_execute(s, bufs, h)) / max(1, layers)
         st = B.pl_comm_status(comm)
+        in_kernel = None
+        if layers and (okw.get("flags", 0) & B.PL_OPT_TRACE):
+            # per-layer latency from the in-kernel stamps of the last execute: a layer is
+            # complete when the last of its signalling ops is about to release its flag
+            ops = B.pl_schedule_dump(s)
+            tr = B.pl_schedule_trace_read(s, len(ops), self.stream)
+            done = np.zeros(layers, dtype=np.float64)
+            for o in ops:
+                done[o.layer] = max(done[o.layer], float(tr[o.topo, 1]), float(tr[o.topo, 0]))
+            gaps = np.diff(done[:-1]) / 1e3  # the last layer's ops do not signal
+            in_kernel = {"p50_us": float(np.median(gaps)), "p10_us": float(np.percentile(gaps, 10)),
+                         "p90_us": float(np.percentile(gaps, 90))}
         nl = max(1, layers)
         sched_bytes = info.bytes_read + info.bytes_written
         rec = {"cfg": cfg, "coll": int(coll), "algo": algo, "R": R, "dtype": int(dtype),
                "message_bytes": int(info.message_bytes), "chunk": int(min(chunk, 1 << 40)), "layers": layers,
-               "us": p50 / nl, "us_p10": p10 / nl, "us_p90": p90 / nl, "us_graph128": graph_us,
+               "us": p50 / nl, "us_p10": p10 / nl, "us_p90": p90 / nl, "us_graph128": graph_us, "layer_us_in_kernel": in_kernel,
                "eff_gbs": info.message_bytes * nl / p50 / 1e3, "sched_gbs": sched_bytes / p50 / 1e3,
                "hbm_frac_measured": sched_bytes / p50 / 1e3 / self.peak, "hbm_frac_8TBps": sched_bytes / p50 / 1e3 / 8000.0,
                "n_ops": int(info.n_ops), "grid": int(info.grid), "threads": int(info.threads),
@@ -153,7 +165,7 @@ class Bench:
         graph_us = _time_graph(lambda h: B.pl_execute(s, bufs, h)) if info.message_bytes <= 2 * MIB else None
         sched_bytes = info.bytes_read + info.bytes_written
         self.emit({"cfg": cfg, "coll": int(coll), "algo": "direct", "R": R, "message_bytes": int(info.message_bytes),
-                   "us": p50, "us_graph128": graph_us, "eff_gbs": info.message_bytes / p50 / 1e3,
+                   "us": p50, "us_graph128": graph_us, "layer_us_in_kernel": in_kernel, "eff_gbs": info.message_bytes / p50 / 1e3,
                    "sched_gbs": sched_bytes / p50 / 1e3, "hbm_frac_measured": sched_bytes / p50 / 1e3 / self.peak,
                    "n_ops": int(info.n_ops), "grid": int(info.grid), "datapath": int(info.datapath),
                    "status": int(B.pl_comm_status(comm).code)})
@@ -304,6 +316,10 @@ def main(args=None):
         for batch in (1, 8, 64):
             for algo in ("oneshot", "direct", "fused"):
                 b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, batch * 8192, 0, iters=50, layers=80)
+        # the same with in-kernel time stamps: distribution of the per-layer latency inside one launch
+        for batch in (1, 8, 64):
+            b.collective("C5-trace", 8, B.PL_BF16, B.PL_ALLREDUCE, "fused", batch * 8192, 0, iters=20, layers=80,
+                         flags=B.PL_OPT_TRACE)
 
 
 if __name__ == "__main__":

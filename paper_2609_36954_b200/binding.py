@@ -36,6 +36,7 @@ PL_DP_AUTO, PL_DP_LDST, PL_DP_TMA = range(3)
 PL_OPT_SKIP_VALIDATE = 1
 PL_OPT_NO_L2_HINTS = 2
 PL_OPT_STAGED = 4
+PL_OPT_TRACE = 8
 
 
 class PurlinError(RuntimeError):
@@ -89,7 +90,7 @@ EXPORTS = [
     "pl_comm_create", "pl_comm_create_planner", "pl_comm_destroy", "pl_comm_status", "pl_comm_reset",
     "pl_schedule_build", "pl_schedule_build_v", "pl_schedule_build_layers", "pl_schedule_build_rooted", "pl_schedule_info",
     "pl_schedule_dump", "pl_schedule_validate", "pl_schedule_debug_break_wait", "pl_schedule_debug_drop_wait",
-    "pl_schedule_destroy",
+    "pl_schedule_trace_read", "pl_schedule_destroy",
     "pl_execute", "pl_execute_host",
     "pl_moe_plan_create", "pl_moe_plan_destroy", "pl_moe_dispatch", "pl_moe_combine", "pl_moe_plan_read",
     "pl_moe_dispatch_dedup", "pl_moe_combine_dedup", "pl_moe_plan_read_dedup",
@@ -131,6 +132,7 @@ def load():
         "pl_schedule_validate": [vp, C.c_char_p, sz],
         "pl_schedule_debug_break_wait": [vp, sz],
         "pl_schedule_debug_drop_wait": [vp, sz],
+        "pl_schedule_trace_read": [vp, vp, sz, vp],
         "pl_schedule_destroy": [vp],
         "pl_execute": [vp, P(pl_bufs_t), vp],
         "pl_execute_host": [vp, P(pl_bufs_t), P(pl_bufs_t), vp],
@@ -271,6 +273,14 @@ def pl_schedule_validate(s):
 
 def pl_schedule_debug_break_wait(s, op_index):
     _check(load().pl_schedule_debug_break_wait(s, op_index), "pl_schedule_debug_break_wait")
+
+
+def pl_schedule_trace_read(s, n_ops, stream=0):
+    """Returns a numpy uint64 array [n_ops, 2] of (start, end) stamps in ns (see purlin.h)."""
+    import numpy as np
+    out = np.zeros((n_ops, 2), dtype=np.uint64)
+    _check(load().pl_schedule_trace_read(s, out.ctypes.data, out.size, stream), "pl_schedule_trace_read")
+    return out
 
 
 def pl_schedule_debug_drop_wait(s, op_index):

@@ -26,6 +26,8 @@ struct pl_schedule_s {
   pl_sched_info_t info{};
   uint64_t timeout_ns = 0;
   bool no_l2_hints = false;
+  bool trace = false;
+  size_t off_trace = 0;
   float out_scale = 1.0f;
   // host copies in device (queue-major) order
   std::vector<DevOp> dev_ops;
@@ -141,6 +143,7 @@ pl_status_t upload(pl_schedule_s* S, int R) {
   S->off_flags = place((size_t)std::max(1, S->L.n_flags) * sizeof(unsigned long long));
   S->off_epoch = place(2 * sizeof(unsigned long long));
   S->sync_bytes = off - S->off_flags;
+  if (S->trace) S->off_trace = place(2 * S->L.ops.size() * sizeof(unsigned long long));
   S->blob_bytes = off;
   if (cudaMalloc(&S->d_blob, S->blob_bytes) != cudaSuccess) { cudaGetLastError(); return PL_ERR_OOM; }
   std::vector<char> host(S->blob_bytes, 0);
@@ -220,6 +223,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   S->pol = pol;
   S->timeout_ns = timeout;
   S->no_l2_hints = (flags & PL_OPT_NO_L2_HINTS) != 0;
+  S->trace = (flags & PL_OPT_TRACE) != 0;
   S->out_scale = out_scale;
   std::string err;
   pl_status_t st = lower(rq, &S->L, &err);
@@ -434,6 +438,17 @@ pl_status_t pl_schedule_validate(pl_schedule_t s, char* msg, size_t msg_cap) {
   return st;
 }
 
+pl_status_t pl_schedule_trace_read(pl_schedule_t s, uint64_t* out, size_t cap_entries, void* stream) {
+  if (!s || !out || !s->trace || !s->d_blob) return PL_ERR_INVALID_ARG;
+  if (cap_entries < 2 * s->L.ops.size()) return PL_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess ||
+      cudaMemcpy(out, s->d_blob + s->off_trace, 2 * s->L.ops.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return PL_ERR_CUDA;
+  }
+  return PL_OK;
+}
+
 pl_status_t pl_schedule_debug_drop_wait(pl_schedule_t s, size_t op_index) {
   if (!s || op_index >= s->L.ops.size()) return PL_ERR_INVALID_ARG;
   HostOp& h = s->L.ops[op_index];
@@ -519,6 +534,7 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   P.flags = s->L.n_flags ? reinterpret_cast<unsigned long long*>(s->d_blob + s->off_flags) : nullptr;
   P.epoch = reinterpret_cast<unsigned long long*>(s->d_blob + s->off_epoch);
   P.status = s->comm->d_status;
+  P.trace = s->trace ? reinterpret_cast<unsigned long long*>(s->d_blob + s->off_trace) : nullptr;
   P.timeout_ns = s->timeout_ns;
   P.n_ranks = R;
   P.stages = s->pol.stages;

@@ -278,6 +278,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
     if (tid < 32 && has_next) fetch(i + 1, r_op, r_src, r_wait);
 
     const DevOp& op = S.op;
+    if (P.trace && tid == 0) P.trace[2ull * op.topo] = globaltimer_ns();  // waits satisfied
     if (op.kind == PL_OP_COPY) {
       body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
     } else if (op.kind == PL_OP_REDUCE) {
@@ -286,9 +287,10 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
       if constexpr (DT != PL_U8) body_copy_reduce<DT>(P, op, S.src, tid, nthr);
     }
 
-    if (op.signal != kNoFlag) {
+    if (op.signal != kNoFlag || P.trace) {
       __syncthreads();  // every thread's writes are done
-      if (tid == 0) {
+      if (tid == 0 && P.trace) P.trace[2ull * op.topo + 1] = globaltimer_ns();
+      if (tid == 0 && op.signal != kNoFlag) {
         __threadfence();
         red_release_add_u64(P.flags + op.signal, 1ull);
         if (op.signal2 != kNoFlag) red_release_add_u64(P.flags + op.signal2, 1ull);

@@ -46,8 +46,10 @@ struct StageDesc {
   uint32_t signal, signal2;
   char* dst;       // destination of this stage
   uint64_t dst_off;  // byte offset inside every rank's output (broadcast destinations)
+  uint32_t topo;   // the op's topological index (trace)
+  uint32_t pad;
 };
-static_assert(sizeof(StageDesc) == 48, "StageDesc layout");
+static_assert(sizeof(StageDesc) == 56, "StageDesc layout");
 
 struct Ctrl {
   uint64_t full[kMaxStages];
@@ -247,6 +249,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
       ok = __all_sync(0xFFFFFFFFu, lane_ok);
       if (!ok) break;
       if (n_wait) ptx::fence_proxy_async();  // data released by other CTAs' generic stores -> our bulk loads
+      if (P.trace && lane == 0) P.trace[2ull * topo] = globaltimer_ns();  // waits satisfied
 
       // ---- cut the op into stages
       const char* my_src = (lane < (int)n_src) ? resolve(P, r_src) : nullptr;
@@ -279,6 +282,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
           d.signal2 = signal2;
           d.dst = dst + u0 * dst_w;
           d.dst_off = dst_off + u0 * dst_w;
+          d.topo = topo;
           ptx::mbar_expect_tx(&c->full[s], units * unit_b);
         }
         __syncwarp();
@@ -350,6 +354,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
           if ((d.flags & kLastOfOp) && d.signal != kNoFlag) {
             ptx::bulk_wait<0>();        // the op's bytes have landed
             ptx::fence_proxy_async();   // async-proxy writes before the generic-proxy release
+            if (P.trace) P.trace[2ull * d.topo + 1] = globaltimer_ns();
             __threadfence();
             red_release_add_u64(P.flags + d.signal, 1ull);
             if (d.signal2 != kNoFlag) red_release_add_u64(P.flags + d.signal2, 1ull);
@@ -385,7 +390,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
       if (kind != PL_OP_COPY) {
         if constexpr (DT != PL_U8) consume_stage<DT>(P, d, slots + (size_t)s * slot_bytes, ctid);
         const bool last = d.flags & kLastOfOp;
-        const uint32_t signal = d.signal, signal2 = d.signal2;
+        const uint32_t signal = d.signal, signal2 = d.signal2, topo = d.topo;
         __syncwarp();
         if (leaves_via_smem(kind, d.flags, d.pmask)) {
           // the copier ships the tile (and signals, if this is the op's last stage)
@@ -396,6 +401,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
           if (lane == 0) ptx::mbar_arrive(&c->done[s]);
           if (ctid == 0) {
             if (wait_bar(P, c, &c->done[s], (done_parity >> s) & 1u)) {
+              if (P.trace) P.trace[2ull * topo + 1] = globaltimer_ns();
               __threadfence();
               red_release_add_u64(P.flags + signal, 1ull);
               if (signal2 != kNoFlag) red_release_add_u64(P.flags + signal2, 1ull);

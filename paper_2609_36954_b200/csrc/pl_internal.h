@@ -83,6 +83,7 @@ struct ExecParams {
   unsigned long long* flags;    // one 64-bit counter per flag, monotone across executes; null if the schedule has none
   unsigned long long* epoch;    // [0] executes completed, [1] CTAs finished in this execute
   int* status;                  // pl_devstatus_t words + abort word (comm-owned)
+  unsigned long long* trace;    // optional: per op (topological index) [start, end] %globaltimer stamps
   unsigned long long timeout_ns;
   int n_ranks;
   int stages;            // shared-memory ring depth of the TMA executor

@@ -503,3 +503,52 @@ def test_output_scale_hook(dp, dtype):
         assert e.value.status == B.PL_ERR_UNSUPPORTED
     finally:
         si.close()
+
+
+# ---- execution trace: on the real device every waiter starts after all of its signallers ended ----
+@pytest.mark.parametrize("dp", DATAPATHS)
+def test_trace_shows_dependencies_were_respected(dp):
+    R = 8
+    cases = []
+    ses = Session(R, "bf16")
+    try:
+        n = R * 24 * 1024
+        x = gen.rank_inputs(R, n, "bf16", seed=61)
+        for algo in (B.PL_ALGO_RING, B.PL_ALGO_TREE, B.PL_ALGO_DIRECT):
+            cases.append((ses.build(B.PL_ALLREDUCE, algo, n, 16384, datapath=dp, flags=B.PL_OPT_TRACE), x))
+        cases.append((ses.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, n, 16384, datapath=dp,
+                                flags=B.PL_OPT_TRACE | B.PL_OPT_STAGED, staging_bytes=2 * R * 16384), x))
+        if dp == B.PL_DP_LDST:
+            xl = [np.concatenate([gen.normal_bf16(8192, 0, l * R + r) for l in range(10)]) for r in range(R)]
+            cases.append((ses.build_layers(B.PL_ALGO_DIRECT_FUSED, 8192, 10, flags=B.PL_OPT_TRACE), xl))
+        for s, data in cases:
+            ses.execute(s, data, repeats=2)
+            ops = B.pl_schedule_dump(s)
+            tr = B.pl_schedule_trace_read(s, len(ops))
+            start, end = tr[:, 0].astype(np.int64), tr[:, 1].astype(np.int64)
+            signallers = {}
+            for o in ops:
+                for f in (o.signal_flag, o.signal_flag2):
+                    if f >= 0:
+                        signallers.setdefault(f, []).append(o.topo)
+            checked = 0
+            for o in ops:
+                assert start[o.topo] > 0
+                if o.signal_flag >= 0:
+                    assert end[o.topo] >= start[o.topo]
+                for k in range(o.n_wait):
+                    for sgn in signallers[o.wait_flag[k]]:
+                        assert 0 < end[sgn] <= start[o.topo], (o.topo, sgn)
+                        checked += 1
+            assert checked > 0
+            # a queue runs its ops in order
+            by_q = {}
+            for o in sorted(ops, key=lambda o: o.topo):
+                by_q.setdefault(o.queue, []).append(start[o.topo])
+            assert all(all(b >= a for a, b in zip(v, v[1:])) for v in by_q.values())
+        # without the option there is nothing to read
+        plain = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 16384, datapath=dp)
+        with pytest.raises(B.PurlinError):
+            B.pl_schedule_trace_read(plain, 10)
+    finally:
+        ses.close()
