@@ -552,3 +552,36 @@ def test_trace_shows_dependencies_were_respected(dp):
             B.pl_schedule_trace_read(plain, 10)
     finally:
         ses.close()
+
+
+# ---- the two executors run the same arithmetic in the same order: identical bits -------------
+def test_register_path_and_bulk_copy_ring_agree_bit_for_bit():
+    import torch
+    from gpu_harness import poison, stream_handle
+    R, n = 8, 8 * 3 * 1024 * 17
+    x = gen.rank_inputs(R, n, "bf16", seed=71)
+    d_in = [to_dev(a) for a in x]
+    ses = Session(R, "bf16")
+    try:
+        for algo, flags in [(B.PL_ALGO_RING, 0), (B.PL_ALGO_TREE, 0), (B.PL_ALGO_DIRECT, 0), (B.PL_ALGO_DIRECT_FUSED, 0),
+                            (B.PL_ALGO_DIRECT, B.PL_OPT_STAGED)]:
+            ref = None
+            for dp, n_ctas, sl in [(B.PL_DP_LDST, 0, 0), (B.PL_DP_TMA, 0, 0), (B.PL_DP_TMA, 4 * R, 4096), (B.PL_DP_LDST, 9 * R, 8192)]:
+                s = ses.build(B.PL_ALLREDUCE, algo, n, 12288, datapath=dp, n_ctas=n_ctas, slice_bytes=sl, flags=flags,
+                              staging_bytes=3 * R * 12288 if flags else 0)
+                info = B.pl_schedule_info(s)
+                d_out = [poison(info.out_bytes[r]) for r in range(R)]
+                bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                                   [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
+                for _ in range(20):
+                    B.pl_execute(s, bufs, stream_handle())
+                torch.cuda.synchronize()
+                assert B.pl_comm_status(ses.comm).code == B.PL_OK
+                out0 = d_out[0][: n * 2].clone()
+                assert all(torch.equal(d_out[r][: n * 2], out0) for r in range(1, R))
+                if ref is None:
+                    ref = out0
+                else:
+                    assert torch.equal(ref, out0), (algo, dp, n_ctas, sl)
+    finally:
+        ses.close()
