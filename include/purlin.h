@@ -378,6 +378,12 @@ pl_status_t pl_moe_dispatch(pl_moe_plan_t plan, const void* const* x,
 pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float* const* gates,
                            void* const* out, void* stream);
 
+/* Combine with the gates computed on the GPU: logits[p] holds, per token, the K logits of
+ * the selected experts (fp32 [T][topk], slot order); the kernel takes their softmax in fp32
+ * (maximum subtracted) and uses the result as gates.  Otherwise as pl_moe_combine. */
+pl_status_t pl_moe_combine_logits(pl_moe_plan_t plan, const void* const* y, const float* const* logits,
+                                  void* const* out, void* stream);
+
 /* Synchronise `stream` and copy the plan's bookkeeping to HOST arrays (any may be NULL):
  * pos int32 [R][T][topk]; counts int64 [R][R] rows src->dst; expert_counts int64
  * [R][n_experts].  Returns PL_ERR_OVERFLOW if the last dispatch dropped rows. */

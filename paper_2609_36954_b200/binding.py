@@ -93,7 +93,7 @@ EXPORTS = [
     "pl_schedule_trace_read", "pl_schedule_destroy",
     "pl_execute", "pl_execute_host",
     "pl_moe_plan_create", "pl_moe_plan_destroy", "pl_moe_dispatch", "pl_moe_combine", "pl_moe_plan_read",
-    "pl_moe_dispatch_dedup", "pl_moe_combine_dedup", "pl_moe_plan_read_dedup",
+    "pl_moe_dispatch_dedup", "pl_moe_combine_dedup", "pl_moe_plan_read_dedup", "pl_moe_combine_logits",
     "pl_status_string", "pl_launch_count", "pl_reduce_scatter_ring_static",
 ]
 
@@ -141,6 +141,7 @@ def load():
         "pl_moe_dispatch": [vp, P(vp), P(vp), P(vp), P(vp), vp],
         "pl_moe_combine": [vp, P(vp), P(vp), P(vp), vp],
         "pl_moe_plan_read": [vp, vp, vp, vp, vp],
+        "pl_moe_combine_logits": [vp, P(vp), P(vp), P(vp), vp],
         "pl_moe_dispatch_dedup": [vp, P(vp), P(vp), P(vp), P(vp), vp],
         "pl_moe_combine_dedup": [vp, P(vp), P(vp), vp],
         "pl_moe_plan_read_dedup": [vp, vp, vp, vp],
@@ -323,6 +324,11 @@ def pl_moe_dispatch(plan, x, topk_idx, recv, recv_meta=None, stream=0):
 def pl_moe_combine(plan, y, gates, out, stream=0):
     _check(load().pl_moe_combine(plan, _ptr_array(y), _ptr_array(gates), _ptr_array(out), stream),
            "pl_moe_combine")
+
+
+def pl_moe_combine_logits(plan, y, logits, out, stream=0):
+    _check(load().pl_moe_combine_logits(plan, _ptr_array(y), _ptr_array(logits), _ptr_array(out), stream),
+           "pl_moe_combine_logits")
 
 
 def pl_moe_dispatch_dedup(plan, x, topk_idx, recv, recv_meta=None, stream=0):

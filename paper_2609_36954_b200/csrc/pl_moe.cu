@@ -50,6 +50,7 @@ struct MoeGeo {
   int32_t* prank;      // [R][T][K] destination rank
   int* flags;          // [0] overflow, [1] invalid expert id, [2] copy engine wait gave up
   const int32_t* slotmask;  // optional [R][T][K]: written into the metadata instead of the slot index
+  int gates_are_logits;     // combine: the gate input holds the K selected logits; softmax them first
 };
 
 __device__ __forceinline__ void build_mask(const MoeGeo& g, const int32_t* idx, uint32_t* mask, int t, int tid) {
@@ -279,7 +280,18 @@ __global__ void __launch_bounds__(256) moe_combine_kernel(const __grid_constant_
       const int row = g.pos[tok * g.K + tid];
       const int r = g.prank[tok * g.K + tid];
       s_row[buf][tid] = row >= 0 ? static_cast<const char*>(P.y[r]) + (size_t)row * g.row_bytes : nullptr;
-      s_gate[buf][tid] = P.gates[p][t * g.K + tid];
+      float gate = P.gates[p][t * g.K + tid];
+      if (g.gates_are_logits) {
+        // fp32 softmax over the token's K logits (max-subtracted); K <= 32 lanes of warp 0
+        const unsigned lanes = (g.K >= 32) ? 0xFFFFFFFFu : ((1u << g.K) - 1u);
+        float m = gate;
+        for (int j = 0; j < g.K; ++j) m = fmaxf(m, __shfl_sync(lanes, gate, j));
+        const float e = expf(gate - m);
+        float sum = 0.f;
+        for (int j = 0; j < g.K; ++j) sum += __shfl_sync(lanes, e, j);  // ascending slot order on every lane
+        gate = e / sum;
+      }
+      s_gate[buf][tid] = gate;
     }
   };
   unsigned long long tok = blockIdx.x;
@@ -509,6 +521,15 @@ pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float
   if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
   g_launches.fetch_add(1);
   return PL_OK;
+}
+
+pl_status_t pl_moe_combine_logits(pl_moe_plan_t plan, const void* const* y, const float* const* logits,
+                                  void* const* out, void* stream) {
+  if (!plan) return PL_ERR_INVALID_ARG;
+  plan->g.gates_are_logits = 1;
+  pl_status_t st = pl_moe_combine(plan, y, logits, out, stream);
+  plan->g.gates_are_logits = 0;
+  return st;
 }
 
 pl_status_t pl_moe_plan_read(pl_moe_plan_t plan, int32_t* pos, int64_t* counts, int64_t* expert_counts, void* stream) {

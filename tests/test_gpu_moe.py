@@ -219,3 +219,33 @@ def test_dedup_dispatch_and_combine(R, T, H, E, K, ident):
         assert st == B.PL_OK or st == B.PL_ERR_OVERFLOW  # cap = R*T rows may be too small for K rows per token
     finally:
         run.close()
+
+
+@pytest.mark.parametrize("K", [8, 6, 1, 32])
+def test_combine_with_gates_from_logits(K):
+    R, T, H, E = 4, 96, 256, 64
+    idx, _ = gen.moe_routing(R, T, E, K, seed=14)
+    x = gen.moe_tokens_bf16(R, T, H, seed=15)
+    cap = R * T * K
+    ref = oracle.moe_dispatch(x, idx, E, recv_capacity_rows=cap)
+    logits = [gen.normal_f32(T * K, 33, p).reshape(T, K) * 3.0 for p in range(R)]
+    # reference gates: softmax in fp64, handed to the oracle as the fp32 values nearest to them
+    gates64 = [np.exp(l.astype(np.float64) - l.astype(np.float64).max(axis=1, keepdims=True)) for l in logits]
+    gates = [np.ascontiguousarray((g / g.sum(axis=1, keepdims=True)).astype(np.float32)) for g in gates64]
+    y = [gen.normal_bf16(cap * H, 77, r).reshape(cap, H) for r in range(R)]
+    want = oracle.moe_combine(y, idx, ref["pos"], gates, E, H)
+    run = MoeRun(R, T, H, E, K, cap)
+    try:
+        st, *_ = run.dispatch(x, idx, with_meta=False)
+        assert st == B.PL_OK
+        d_y = [to_dev(a) for a in y]
+        d_l = [to_dev(a) for a in logits]
+        d_out = [poison(T * H * 2) for _ in range(R)]
+        B.pl_moe_combine_logits(run.plan, [t.data_ptr() for t in d_y], [t.data_ptr() for t in d_l],
+                                [t.data_ptr() for t in d_out], stream_handle())
+        torch.cuda.synchronize()
+        for p in range(R):
+            got = gen.bf16_bits_to_f64(d_out[p].cpu().numpy().view(np.uint16).reshape(T, H))
+            check_float(got, want[p], "bf16")
+    finally:
+        run.close()
