@@ -250,6 +250,11 @@ pl_status_t pl_comm_status(pl_comm_t comm, pl_devstatus_t* out);
  * (asynchronously on `stream`).  Required after a timeout before executing again. */
 pl_status_t pl_comm_reset(pl_comm_t comm, void* stream);
 
+/* Text of the last build or validation failure on this communicator ("" if none): which
+ * rule of the size / algorithm / schedule checks was violated.  The pointer stays valid until
+ * the next failing call on the same communicator. */
+const char* pl_comm_last_error(pl_comm_t comm);
+
 /* ---- orchestration ----------------------------------------------------------------- */
 
 /* Lower a fixed-size collective into a schedule.

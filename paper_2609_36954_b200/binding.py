@@ -88,6 +88,7 @@ class pl_devstatus_t(C.Structure):
 
 EXPORTS = [
     "pl_comm_create", "pl_comm_create_planner", "pl_comm_destroy", "pl_comm_status", "pl_comm_reset",
+    "pl_comm_last_error",
     "pl_schedule_build", "pl_schedule_build_v", "pl_schedule_build_layers", "pl_schedule_build_rooted", "pl_schedule_info",
     "pl_schedule_dump", "pl_schedule_validate", "pl_schedule_debug_break_wait", "pl_schedule_debug_drop_wait",
     "pl_schedule_trace_read", "pl_schedule_destroy",
@@ -153,6 +154,8 @@ def load():
         fn.restype = C.c_int
     L.pl_status_string.argtypes = [C.c_int]
     L.pl_status_string.restype = C.c_char_p
+    L.pl_comm_last_error.argtypes = [vp]
+    L.pl_comm_last_error.restype = C.c_char_p
     L.pl_launch_count.argtypes = []
     L.pl_launch_count.restype = C.c_uint64
     _lib = L
@@ -212,6 +215,10 @@ def pl_comm_status(comm):
     s = pl_devstatus_t()
     _check(load().pl_comm_status(comm, C.byref(s)), "pl_comm_status")
     return s
+
+
+def pl_comm_last_error(comm) -> str:
+    return load().pl_comm_last_error(comm).decode()
 
 
 def pl_comm_reset(comm, stream=0):

@@ -185,7 +185,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
     rq.staged = (flags & PL_OPT_STAGED) != 0;
     rq.staging_bytes = opts->staging_bytes;
     if (opts->out_scale != 0.0f) {
-      if (comm && comm->dtype != PL_BF16 && comm->dtype != PL_F32) return PL_ERR_UNSUPPORTED;
+      if (comm->dtype != PL_BF16 && comm->dtype != PL_F32) return PL_ERR_UNSUPPORTED;
       out_scale = opts->out_scale;
     }
     if (pol.threads < 0 || pol.threads % 32 || pol.threads > exec_max_threads()) return PL_ERR_INVALID_ARG;
@@ -328,6 +328,8 @@ pl_status_t pl_comm_status(pl_comm_t comm, pl_devstatus_t* out) {
   std::memcpy(&out->observed, words + 6, 8);
   return PL_OK;
 }
+
+const char* pl_comm_last_error(pl_comm_t comm) { return comm ? comm->last_error.c_str() : ""; }
 
 pl_status_t pl_comm_reset(pl_comm_t comm, void* stream) {
   if (!comm) return PL_ERR_INVALID_ARG;

@@ -232,6 +232,7 @@ def test_error_rules():
             return ei.value.status
         # bytes not divisible by R*16
         assert status(lambda: pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, 8 * 8 + 8, 64)) == B.PL_ERR_INVALID_ARG
+        assert "divisible by 16*R" in B.pl_comm_last_error(pl.comm)
         # chunk not a multiple of 16 / zero
         assert status(lambda: pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 24)) == B.PL_ERR_INVALID_ARG
         assert status(lambda: pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 0)) == B.PL_ERR_INVALID_ARG
