@@ -305,7 +305,9 @@ def main(args=None):
             for algo in ("ring", "tree", "oneshot", "direct", "fused"):
                 if algo == "oneshot" and size > 64 * MIB:
                     continue
-                chunk = max(16, min(MIB, size // 8))
+                # chunks of a partition (size / 8) for the partitioned algorithms, of the whole
+                # message for one-shot and tree
+                chunk = max(16, min(MIB, size if algo in ("oneshot", "tree") else size // 8))
                 b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30 if lg < 24 else 10,
                              graph=lg <= 21)
     if "c4" in which:

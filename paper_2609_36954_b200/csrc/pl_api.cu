@@ -232,7 +232,15 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
     delete S;
     return st;
   }
-  assign_queues(&S->L, comm->R, pol.n_ctas);
+  // Latency regime with the grid left to the library: one queue per op a rank can run at
+  // the same time, so that no ready op sits behind another in a queue.
+  const bool latency = rq.n_layers == 0 && !rq.staged && S->L.message_bytes <= (1u << 20);
+  if (requested == 0 && latency) {
+    const int per_rank = std::min(capacity / comm->R, std::max(pol.n_ctas / comm->R, level_width(S->L, comm->R)));
+    pol.n_ctas = std::max(1, per_rank) * comm->R;
+    S->pol = pol;
+  }
+  assign_queues(&S->L, comm->R, pol.n_ctas, latency);
   if (!(flags & PL_OPT_SKIP_VALIDATE)) {
     st = validate(S->L, comm->R, &err);
     if (st != PL_OK) {

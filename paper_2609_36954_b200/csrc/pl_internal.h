@@ -125,7 +125,10 @@ struct BuildRequest {
 
 // orchestrator (host only, no CUDA)
 pl_status_t lower(const BuildRequest& rq, Lowered* out, std::string* err);
-void assign_queues(Lowered* L, int R, int n_queues);
+void assign_queues(Lowered* L, int R, int n_queues, bool by_level = false);
+// Largest number of ops one rank has at the same depth of the flag-dependency graph: the
+// queues per rank a latency-bound schedule can keep busy at once.
+int level_width(const Lowered& L, int R);
 pl_status_t validate(const Lowered& L, int R, std::string* err);
 Policy default_policy(const BuildRequest& rq, int max_resident_ctas);
 

@@ -85,8 +85,8 @@ def run(ops, info, R, ins, seed=0, max_steps=None):
             kinds = {op.src[k].dtype for k in range(op.n_src)} | {op.dst.dtype}
             if first.dtype == B.PL_I32:
                 acc = np.zeros(n, np.uint32)
-            elif B.PL_F32X2 in kinds:
-                acc = np.zeros(n, np.float64)  # stands in for the compensated fp32 pair
+            elif B.PL_F32X2 in kinds or B.PL_F32 in kinds:
+                acc = np.zeros(n, np.float64)  # stands in for the compensated fp32 (sum, correction) pair
             else:
                 acc = np.zeros(n, np.float32)
             for k in range(op.n_src):

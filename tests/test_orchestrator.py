@@ -497,3 +497,52 @@ def test_rooted_collectives_replay(R, root):
                 B.pl_schedule_build_rooted(pl.comm, B.PL_ALLREDUCE, 0, n, 48, None)
         finally:
             pl.close()
+
+
+def test_tree_root_rotates_with_the_chunk_and_balances_the_ranks():
+    """Binomial tree: 2(R-1) ops per chunk over log2(R) + log2(R) stages; the op that writes the
+    reduced chunk (the root's) moves to rank c mod R with the chunk index, so every rank carries
+    the same bytes when the chunk count is a multiple of R; one chunk is the rank-0 tree."""
+    R, es = 8, 4
+    pl = Planner(R, "i32")
+    try:
+        n = 16 * 256  # 16 chunks of 1 KiB
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_TREE, n, 1024, n_ctas=R, slice_bytes=1 << 20)
+        ops = B.pl_schedule_dump(s)
+        assert len(ops) == 16 * 2 * (R - 1)
+        roots = {}
+        per_rank = [0] * R
+        for o in ops:
+            per_rank[o.exec_rank] += o.count * (es if o.kind != B.PL_OP_COPY else 1)
+            if o.kind == B.PL_OP_COPY_REDUCE and o.dst.buf == B.PL_BUF_OUT:
+                roots[int(o.dst.offset) // 1024] = o.exec_rank
+        assert roots == {c: c % R for c in range(16)}
+        assert len(set(per_rank)) == 1
+        # a single chunk: reduce ends on rank 0, which never receives a broadcast copy
+        s1 = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_TREE, 256, 1024, n_ctas=R, slice_bytes=1 << 20)
+        ops1 = B.pl_schedule_dump(s1)
+        assert len(ops1) == 2 * (R - 1)
+        assert [o.exec_rank for o in ops1 if o.kind == B.PL_OP_COPY_REDUCE and o.dst.buf == B.PL_BUF_OUT] == [0]
+        assert sorted(o.exec_rank for o in ops1 if o.kind == B.PL_OP_COPY) == list(range(1, R))
+    finally:
+        pl.close()
+
+
+def test_latency_regime_grid_follows_the_schedule_width():
+    """Small messages with the grid left to the library: a rank gets one queue per op it can run
+    at the same depth of the dependency graph (two-shot all-reduce: R - 1 gather copies)."""
+    R = 8
+    pl = Planner(R, "bf16")
+    try:
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 2048, 512)  # 4 KiB per rank
+        info = B.pl_schedule_info(s)
+        ops = B.pl_schedule_dump(s)
+        assert info.n_queues == R * (R - 1)
+        # no queue holds two ops of the same phase
+        seen = set()
+        for o in ops:
+            key = (o.queue, o.kind)
+            assert key not in seen
+            seen.add(key)
+    finally:
+        pl.close()
