@@ -35,6 +35,9 @@
  *     other until the wait limit reports PL_ERR_TIMEOUT.  Issuing all executes on one stream
  *     is always safe.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - A communicator belongs to the CUDA device that was current when it was created; its
+ *     schedules and plans live there.  Every later call on it must be made with that device
+ *     current, otherwise the call returns PL_ERR_INVALID_ARG and launches nothing.
  */
 #ifndef PURLIN_H_
 #define PURLIN_H_

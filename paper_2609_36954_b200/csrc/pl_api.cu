@@ -17,7 +17,18 @@ using namespace pl;
 
 namespace pl {
 std::atomic<uint64_t> g_launches{0};
+
+bool on_comm_device(pl_comm_s* comm) {
+  if (comm->planner) return true;
+  int d = -1;
+  if (cudaGetDevice(&d) != cudaSuccess) { cudaGetLastError(); return false; }
+  if (d != comm->device) {
+    comm->last_error = "the current CUDA device is not the communicator's";
+    return false;
+  }
+  return true;
 }
+}  // namespace pl
 
 struct pl_schedule_s {
   pl_comm_t comm = nullptr;
@@ -168,6 +179,7 @@ pl_status_t upload(pl_schedule_s* S, int R) {
 pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t* opts, pl_schedule_t* out) {
   if (!comm || !out) return PL_ERR_INVALID_ARG;
   *out = nullptr;
+  if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
   Policy pol{};
   uint64_t timeout = 2000000000ull;
   uint32_t flags = 0;
@@ -325,6 +337,7 @@ pl_status_t pl_comm_status(pl_comm_t comm, pl_devstatus_t* out) {
   if (!comm || !out) return PL_ERR_INVALID_ARG;
   std::memset(out, 0, sizeof(*out));
   if (comm->planner) return PL_OK;
+  if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
   int words[kStatusWords];
   if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
   if (cudaMemcpy(words, comm->d_status, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
@@ -342,6 +355,7 @@ const char* pl_comm_last_error(pl_comm_t comm) { return comm ? comm->last_error.
 pl_status_t pl_comm_reset(pl_comm_t comm, void* stream) {
   if (!comm) return PL_ERR_INVALID_ARG;
   if (comm->planner) return PL_OK;
+  if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(comm->d_status, 0, kStatusWords * sizeof(int), st) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
   std::lock_guard<std::mutex> g(comm->mu);
@@ -525,6 +539,7 @@ static pl_status_t check_bufs(pl_schedule_t s, const pl_bufs_t* b) {
 pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   if (!s || !bufs) return PL_ERR_INVALID_ARG;
   if (s->comm->planner || !s->d_blob) return PL_ERR_UNSUPPORTED;
+  if (!on_comm_device(s->comm)) return PL_ERR_INVALID_ARG;
   pl_status_t st = check_bufs(s, bufs);
   if (st != PL_OK) return st;
   ExecParams P;

@@ -25,4 +25,6 @@ struct pl_comm_s {
 
 namespace pl {
 extern std::atomic<uint64_t> g_launches;
+// true when the calling thread's current CUDA device is the communicator's (always for a planner)
+bool on_comm_device(pl_comm_s* comm);
 }

@@ -370,6 +370,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   if (!comm || !out) return PL_ERR_INVALID_ARG;
   *out = nullptr;
   if (comm->planner) return PL_ERR_UNSUPPORTED;
+  if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
   const int R = comm->R;
   if (tokens_per_rank < 1 || hidden < 1 || n_experts < R || topk < 1 || topk > kMaxTopk) return PL_ERR_INVALID_ARG;
   if (n_experts % R || n_experts > 4096 || topk > n_experts) return PL_ERR_INVALID_ARG;
@@ -472,6 +473,7 @@ pl_status_t pl_moe_plan_destroy(pl_moe_plan_t plan) {
 pl_status_t pl_moe_dispatch(pl_moe_plan_t plan, const void* const* x, const int32_t* const* topk_idx,
                             void* const* recv, int32_t* const* recv_meta, void* stream) {
   if (!plan || !x || !topk_idx || !recv) return PL_ERR_INVALID_ARG;
+  if (!on_comm_device(plan->comm)) return PL_ERR_INVALID_ARG;
   const MoeGeo& g = plan->g;
   DispatchPtrs P;
   std::memset(&P, 0, sizeof(P));
@@ -505,6 +507,7 @@ pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float
   if (!plan || !y || !gates || !out) return PL_ERR_INVALID_ARG;
   if (plan->comm->dtype != PL_BF16) return PL_ERR_UNSUPPORTED;
   if (!plan->dispatched) return PL_ERR_INVALID_ARG;
+  if (!on_comm_device(plan->comm)) return PL_ERR_INVALID_ARG;
   const MoeGeo& g = plan->g;
   CombinePtrs P;
   std::memset(&P, 0, sizeof(P));
@@ -551,6 +554,7 @@ pl_status_t pl_moe_plan_read(pl_moe_plan_t plan, int32_t* pos, int64_t* counts, 
 pl_status_t pl_moe_dispatch_dedup(pl_moe_plan_t plan, const void* const* x, const int32_t* const* topk_idx,
                                   void* const* recv, int32_t* const* recv_meta, void* stream) {
   if (!plan || !x || !topk_idx || !recv) return PL_ERR_INVALID_ARG;
+  if (!on_comm_device(plan->comm)) return PL_ERR_INVALID_ARG;
   const MoeGeo& g = plan->g;
   const MoeGeo& d = plan->gd;
   DispatchPtrs P0, P;
@@ -588,6 +592,7 @@ pl_status_t pl_moe_combine_dedup(pl_moe_plan_t plan, const void* const* z, void*
   if (!plan || !z || !out) return PL_ERR_INVALID_ARG;
   if (plan->comm->dtype != PL_BF16) return PL_ERR_UNSUPPORTED;
   if (!plan->dispatched_dedup) return PL_ERR_INVALID_ARG;
+  if (!on_comm_device(plan->comm)) return PL_ERR_INVALID_ARG;
   const MoeGeo& d = plan->gd;
   CombinePtrs P;
   std::memset(&P, 0, sizeof(P));

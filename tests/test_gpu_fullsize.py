@@ -179,3 +179,50 @@ def test_c4_moe_full_size_sampled(identity):
     finally:
         B.pl_moe_plan_destroy(plan)
         B.pl_comm_destroy(comm)
+
+
+def test_buffers_beyond_4gib_use_64_bit_offsets():
+    """Maximum sizes: per-rank buffers of 4.5 GiB, so ops address past the 32-bit byte range.
+    All-gather (8 x 576 MiB -> 8 x 4.5 GiB) is compared bit for bit on whole partitions at the
+    far end and on samples; reduce-scatter (8 x 4.5 GiB -> 8 x 576 MiB) on sampled sums."""
+    R = 8
+    m = 288 * MIB                      # bf16 elements per partition: 576 MiB
+    n = R * m                          # 4.5 GiB per rank
+    comm = B.pl_comm_create(R, B.PL_BF16)
+    try:
+        part = big_inputs(R, m, seed=7)
+        ag = B.pl_schedule_build(comm, B.PL_ALLGATHER, B.PL_ALGO_DIRECT, m, MIB, None)
+        out = [torch.full((n,), -1, dtype=torch.int16, device="cuda") for _ in range(R)]
+        run(ag, comm, R, part, out)
+        B.pl_schedule_destroy(ag)
+        idx = sample_idx(n, k=1 << 16)
+        assert idx[-1] * 2 > (1 << 32)
+        ti = torch.from_numpy(idx).cuda()
+        src_rank = torch.from_numpy(idx // m).cuda()
+        src_off = torch.from_numpy(idx % m).cuda()
+        stacked = torch.stack(part)                      # [R, m]
+        expect = stacked[src_rank, src_off]
+        for r in range(R):
+            assert torch.equal(out[r][ti], expect)
+            assert torch.equal(out[r][(R - 1) * m:], part[R - 1])   # the partition that lies past 4 GiB
+        del stacked, expect
+        # reduce-scatter over 4.5 GiB inputs: rank r's input is the gathered buffer rolled by 4099 r
+        x = []
+        for r in range(R):                               # roll one buffer at a time: peak memory stays ~45 GiB
+            x.append(torch.roll(out[r], 4099 * r))
+            out[r] = None
+        rs = B.pl_schedule_build(comm, B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, MIB, None)
+        red = [torch.full((m,), -1, dtype=torch.int16, device="cuda") for _ in range(R)]
+        run(rs, comm, R, x, red)
+        B.pl_schedule_destroy(rs)
+        for r in (0, R - 1):
+            loc = sample_idx(m, k=4096, seed=r)
+            gi = torch.from_numpy(loc + r * m).cuda()
+            samples = [x[p][gi].cpu().numpy().view(np.uint16) for p in range(R)]
+            ref = oracle.allreduce(samples, "bf16")[0]
+            got = gen.bf16_bits_to_f64(red[r][torch.from_numpy(loc).cuda()].cpu().numpy().view(np.uint16))
+            check_float(got, ref, "bf16")
+    finally:
+        B.pl_comm_destroy(comm)
+        part = out = x = red = None
+        torch.cuda.empty_cache()
