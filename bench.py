@@ -263,7 +263,7 @@ def run_purlin(args):
 
     if rank == 0:
         line = {
-            "metric": "effective_collective_bandwidth", "value": value, "unit": "GB/s", "n_gpus": world,
+            "metric": "effective collective GB/s", "value": value, "unit": "GB/s", "n_gpus": world,
             "steps": K, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "C2: reduce-scatter (64 MiB/rank in) then all-gather (64 MiB/rank out), "
@@ -376,7 +376,7 @@ def run_reference(args):
     eff = 2 * x[0].nbytes
     value = eff / dt / 1e9
     sample = f"{x[0].nbytes / MIB:.3f} MiB/rank of the 64 MiB/rank C2 step per step (R={R})"
-    line = {"impl": "reference", "metric": "effective_collective_bandwidth", "value": value, "unit": "GB/s",
+    line = {"impl": "reference", "metric": "effective collective GB/s", "value": value, "unit": "GB/s",
             "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K, "warmup": W, "ms_per_step": dt * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": "C2: reduce-scatter then all-gather, R=8, bf16 N(0,1) seed 0 (CPU oracle, "

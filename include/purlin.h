@@ -110,7 +110,8 @@ typedef enum {
  *                         into all R outputs (no gather step, fewest bytes).
  *   PL_ALGO_RING          textbook ring; partial sums of bf16 data travel in fp32, of fp32
  *                         data as compensated fp32 pairs (PL_F32X2), of int32 data in int32.
- *   PL_ALGO_TREE          all-reduce only: binomial reduce to rank 0, binomial broadcast.
+ *   PL_ALGO_TREE          all-reduce only: binomial reduce to a root, binomial broadcast from it;
+ *                         the root of chunk c is rank c mod R (rank 0 for a one-chunk message).
  * Ring and tree are not in the paper (its only pattern is the direct pull); they are the
  * classical algorithms the benchmark configurations name. */
 typedef enum {
