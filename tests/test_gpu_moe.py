@@ -249,3 +249,39 @@ def test_combine_with_gates_from_logits(K):
             check_float(got, want[p], "bf16")
     finally:
         run.close()
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_moe_shapes_match_the_oracle(seed):
+    """Seeded draws of rank count, tokens, row width, expert count and top-k, including one
+    token per rank, experts that nobody selects and rows of a single 16-byte vector."""
+    rng = np.random.default_rng(500 + seed)
+    R = int(rng.choice([2, 3, 4, 8, 16]))
+    epr = int(rng.choice([1, 2, 5, 32]))
+    E = R * epr
+    K = int(rng.choice([k for k in (1, 2, 4, 8, 32) if k <= E]))
+    T = int(rng.choice([1, 2, 31, 256, 257, 600]))
+    H = int(rng.choice([8, 24, 512, 1000, 7168]))
+    ident = bool(rng.integers(0, 2))
+    idx, gates = gen.moe_routing(R, T, E, K, seed=seed, identity_perm=ident)
+    x = gen.moe_tokens_bf16(R, T, H, seed=seed + 1)
+    cap = R * T * K
+    ref = oracle.moe_dispatch(x, idx, E, recv_capacity_rows=cap)
+    run = MoeRun(R, T, H, E, K, cap)
+    try:
+        st, recv, meta, pos, counts, ecounts = run.dispatch(x, idx)
+        assert st == B.PL_OK
+        assert np.array_equal(counts, ref["counts"]) and np.array_equal(ecounts, ref["expert_counts"])
+        for p in range(R):
+            assert np.array_equal(pos[p], ref["pos"][p])
+        for r in range(R):
+            nrows = int(counts[:, r].sum())
+            assert np.array_equal(recv[r].view(np.uint16).reshape(cap, H)[:nrows], ref["recv"][r][:nrows])
+            assert np.array_equal(meta[r][:nrows], ref["meta"][r][:nrows])
+            assert np.all(recv[r].reshape(cap, -1)[nrows:] == 0xFF)
+        out = run.combine(run.d_recv, gates)
+        want = oracle.moe_combine(ref["recv"], idx, ref["pos"], gates, E, H)
+        for p in range(R):
+            check_float(gen.bf16_bits_to_f64(out[p]), want[p], "bf16")
+    finally:
+        run.close()
