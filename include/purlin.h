@@ -168,6 +168,13 @@ typedef struct {
 /* Record, for every op, when its waits were satisfied and when its signal was about to be
  * released (%globaltimer, ns) into a schedule-owned buffer: see pl_schedule_trace_read. */
 #define PL_OPT_TRACE 8u
+/* Launch pl_execute's kernel with CUDA's programmatic stream serialization attribute, so that
+ * when the kernel in front of it on the stream is another execute, its CTAs may be set up
+ * while that one drains (the kernel waits for the completion of everything in front of it
+ * before it reads anything an earlier launch wrote, so stream order is kept as seen by the
+ * data).  Shortens back-to-back executes; no effect after any other kind of work.  The paper
+ * has no counterpart (it measures calls inside a CUDA graph, Sec. 5). */
+#define PL_OPT_OVERLAP_LAUNCH 16u
 #define PL_OPT_NO_L2_HINTS 2u  /* bulk copies without L2 eviction hints (default: stores evict-first,
                                   sources of copy ops evict-last; measured 7 % on all-gather) */
 

@@ -310,6 +310,10 @@ def main(args=None):
                 chunk = max(16, min(MIB, size if algo in ("oneshot", "tree") else size // 8))
                 b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30 if lg < 24 else 10,
                              graph=lg <= 21)
+                # latency-bound sizes again with overlapped launches (CTAs of call i+1 set up while call i drains)
+                if lg <= 20 and algo in ("oneshot", "fused"):
+                    b.collective("C3-overlap", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30, graph=True,
+                                 flags=B.PL_OPT_OVERLAP_LAUNCH)
     if "c4" in which:
         T = int(os.environ.get("PL_MOE_TOKENS", 4096))  # fewer tokens per rank for profiler captures
         b.moe("C4", T=T, identity=False)

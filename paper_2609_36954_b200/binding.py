@@ -37,6 +37,7 @@ PL_OPT_SKIP_VALIDATE = 1
 PL_OPT_NO_L2_HINTS = 2
 PL_OPT_STAGED = 4
 PL_OPT_TRACE = 8
+PL_OPT_OVERLAP_LAUNCH = 16
 
 
 class PurlinError(RuntimeError):

@@ -38,6 +38,7 @@ struct pl_schedule_s {
   uint64_t timeout_ns = 0;
   bool no_l2_hints = false;
   bool trace = false;
+  bool overlap_launch = false;
   size_t off_trace = 0;
   float out_scale = 1.0f;
   // host copies in device (queue-major) order
@@ -236,6 +237,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   S->timeout_ns = timeout;
   S->no_l2_hints = (flags & PL_OPT_NO_L2_HINTS) != 0;
   S->trace = (flags & PL_OPT_TRACE) != 0;
+  S->overlap_launch = (flags & PL_OPT_OVERLAP_LAUNCH) != 0;
   S->out_scale = out_scale;
   std::string err;
   pl_status_t st = lower(rq, &S->L, &err);
@@ -567,6 +569,7 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   // bulk stores stream out (evict-first), sources of copies are re-read by other ranks (evict-last)
   P.hints = s->no_l2_hints ? 0u : 6u;
   P.out_scale = s->out_scale;
+  P.overlap_launch = s->overlap_launch ? 1u : 0u;
   cudaError_t le = s->pol.datapath == PL_DP_TMA
                        ? launch_exec_tma(s->comm->dtype, P, s->pol.n_ctas, static_cast<cudaStream_t>(stream))
                        : launch_exec(s->comm->dtype, P, s->pol.n_ctas, s->pol.threads, static_cast<cudaStream_t>(stream));

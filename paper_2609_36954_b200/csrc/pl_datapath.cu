@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   // advanced after all CTAs reported, so all of them see the same value; a schedule without
   // flags needs no epoch at all
   const bool has_flags = P.flags != nullptr;
-  const unsigned long long epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
+  pdl_launch_dependents();
   if (tid == 0) s_abort[0] = s_abort[1] = 0;
   bool aborted = false;
 
@@ -236,10 +236,10 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   uint4 r_op = make_uint4(0, 0, 0, 0);
   uint64_t r_src = 0;
   DevWait r_wait = {0, 0};
-  if (tid < 32) {
-    fetch(0, r_op, r_src, r_wait);
-    stash(0, r_op, r_src, r_wait);
-  }
+  if (tid < 32) fetch(0, r_op, r_src, r_wait);  // descriptors are immutable: fetched before the wait below
+  pdl_wait();
+  const unsigned long long epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
+  if (tid < 32) stash(0, r_op, r_src, r_wait);
   __syncthreads();
   // the first descriptor tells how many ops the queue holds (a placeholder marks an empty one)
   const uint32_t n_ops = s_slot[0].op.kind == kNopKind ? 0u : s_slot[0].op.remaining + 1u;
@@ -316,8 +316,16 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
 
 template <int DT>
 cudaError_t launch_t(const ExecParams& P, int grid, int threads, cudaStream_t stream) {
-  pl_exec_kernel<DT><<<grid, threads, 0, stream>>>(P);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = P.overlap_launch ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, pl_exec_kernel<DT>, P);
 }
 
 }  // namespace

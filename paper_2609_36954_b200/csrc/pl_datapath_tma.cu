@@ -18,6 +18,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "pl_device.cuh"
 #include "pl_internal.h"
 #include "pl_kernels.h"
@@ -180,7 +182,7 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, q = blockIdx.x;
   const uint32_t S = (uint32_t)P.stages, slot_bytes = P.stage_bytes;
   const bool has_flags = P.flags != nullptr;
-  const unsigned long long epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
+  pdl_launch_dependents();
 
   if (tid == 0) {
     for (uint32_t s = 0; s < S; ++s) {
@@ -191,6 +193,8 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
     c->abort = 0;
     ptx::mbar_init_fence();
   }
+  pdl_wait();  // from here on memory written by earlier launches may be read
+  const unsigned long long epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
   __syncthreads();
 
   if (warp == 0) {
@@ -429,14 +433,28 @@ __global__ void __launch_bounds__(kThreads, 1) pl_exec_tma_kernel(const __grid_c
 template <int DT>
 cudaError_t launch_t(const ExecParams& P, int grid, cudaStream_t stream) {
   const size_t smem = exec_tma_smem_bytes(P.stages, P.stage_bytes);
-  static bool configured = false;  // per instantiation
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(pl_exec_tma_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  // the shared-memory opt-in is a per-device attribute of the function: one bit per device
+  static std::atomic<unsigned long long> configured{0};  // per instantiation
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (!(configured.load(std::memory_order_acquire) & bit)) {
+    e = cudaFuncSetAttribute(pl_exec_tma_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured.fetch_or(bit, std::memory_order_release);
   }
-  pl_exec_tma_kernel<DT><<<grid, kThreads, smem, stream>>>(P);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = P.overlap_launch ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, pl_exec_tma_kernel<DT>, P);
 }
 
 template <int DT>

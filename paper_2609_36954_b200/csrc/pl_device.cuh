@@ -20,6 +20,14 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 __device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
+// Programmatic dependent launch (kernels launched with the programmatic stream serialization
+// attribute): launch_dependents lets the next such kernel in the stream start its CTAs while
+// this grid still runs; wait returns once every grid this one depends on has completed and
+// its writes are visible.  Both are no-ops for a plain launch.  Nothing written by an earlier
+// launch (epoch, flags, status, data) may be read before the wait; descriptors are immutable.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));

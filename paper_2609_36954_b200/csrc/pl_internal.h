@@ -90,6 +90,7 @@ struct ExecParams {
   uint32_t stage_bytes;  // bytes per ring slot
   float out_scale;       // multiplies every final (element-typed) sum; 1 = plain sum
   uint32_t hints;        // L2 policy bits for bulk copies: 1 loads evict-first, 2 stores evict-first, 4 copy loads evict-last
+  uint32_t overlap_launch;  // host side only: launch with the programmatic stream serialization attribute
 };
 
 struct Policy {

@@ -585,3 +585,60 @@ def test_register_path_and_bulk_copy_ring_agree_bit_for_bit():
                     assert torch.equal(ref, out0), (algo, dp, n_ctas, sl)
     finally:
         ses.close()
+
+
+# ---- overlapped launches (programmatic stream serialization) ----------------------------------
+@pytest.mark.parametrize("dp", DATAPATHS)
+def test_overlapped_launches_keep_stream_order(dp):
+    """With PL_OPT_OVERLAP_LAUNCH a kernel's CTAs may start while its predecessor drains; the
+    data must still see stream order.  A chain x -> y -> z of two all-reduces where the second
+    reads what the first wrote, re-run back to back on poisoned buffers (eagerly and inside a
+    CUDA graph), must give all-reduce(all-reduce(x)) every time; repeated executes of ONE
+    flagged schedule must keep their epochs apart."""
+    import torch
+    from gpu_harness import poison
+    R, n = 8, 8 * 5000
+    x = gen.rank_inputs(R, n, "i32", seed=0)
+    y_ref = oracle.allreduce(x, "i32")
+    z_ref = oracle.allreduce(y_ref, "i32")
+    ses = Session(R, "i32")
+    try:
+        flags = B.PL_OPT_OVERLAP_LAUNCH
+        a = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 2048, datapath=dp, flags=flags)
+        b = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, n, 4096, datapath=dp, flags=flags)
+        nb = n * 4
+        d_x = [to_dev(v) for v in x]
+        d_y = [poison(nb) for _ in range(R)]
+        d_z = [poison(nb) for _ in range(R)]
+        bufs_a = B.make_bufs([t.data_ptr() for t in d_x], [t.data_ptr() for t in d_y], [nb] * R, [nb] * R)
+        bufs_b = B.make_bufs([t.data_ptr() for t in d_y], [t.data_ptr() for t in d_z], [nb] * R, [nb] * R)
+
+        def chain(h, reps):
+            for _ in range(reps):
+                B.pl_execute(a, bufs_a, h)
+                B.pl_execute(b, bufs_b, h)
+
+        def check():
+            torch.cuda.synchronize()
+            assert B.pl_comm_status(ses.comm).code == B.PL_OK
+            for r in range(R):
+                assert np.array_equal(d_y[r].cpu().numpy().view(np.int32), y_ref[r])
+                assert np.array_equal(d_z[r].cpu().numpy().view(np.int32), z_ref[r])
+
+        for _ in range(5):
+            for t in d_y + d_z:
+                t.fill_(0xFF)
+            chain(torch.cuda.current_stream().cuda_stream, 6)
+            check()
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.graph(g, stream=side):
+            chain(torch.cuda.current_stream().cuda_stream, 8)
+        for _ in range(3):
+            for t in d_y + d_z:
+                t.fill_(0xFF)
+            g.replay()
+            check()
+    finally:
+        ses.close()
