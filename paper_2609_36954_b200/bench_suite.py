@@ -165,7 +165,7 @@ class Bench:
         graph_us = _time_graph(lambda h: B.pl_execute(s, bufs, h)) if info.message_bytes <= 2 * MIB else None
         sched_bytes = info.bytes_read + info.bytes_written
         self.emit({"cfg": cfg, "coll": int(coll), "algo": "direct", "R": R, "message_bytes": int(info.message_bytes),
-                   "us": p50, "us_graph128": graph_us, "layer_us_in_kernel": in_kernel, "eff_gbs": info.message_bytes / p50 / 1e3,
+                   "us": p50, "us_graph128": graph_us, "eff_gbs": info.message_bytes / p50 / 1e3,
                    "sched_gbs": sched_bytes / p50 / 1e3, "hbm_frac_measured": sched_bytes / p50 / 1e3 / self.peak,
                    "n_ops": int(info.n_ops), "grid": int(info.grid), "datapath": int(info.datapath),
                    "status": int(B.pl_comm_status(comm).code)})

@@ -263,12 +263,14 @@ void scatter_direct(Emitter& em, const Geo& g, int root) {
                   {ref(root, PL_BUF_IN, PL_U8, (r * g.P + c * g.chunk) * g.es)}, g.clen(c) * g.es, {}, -1);
 }
 
-// gather: only the root consumes; it copies every rank's packed contribution to slot p.
+// gather: only the root consumes.  Rank p writes its packed contribution into slot p of the
+// root's output (a push): the copies then run on every rank's queues.  Left to the root as
+// pulls they would all sit on the root's queues, one eighth of the CTAs at R = 8.
 void gather_direct(Emitter& em, const Geo& g, int root) {
-  em.phase_chunks = g.n_c * g.R;
+  em.phase_chunks = g.n_c;
   for (uint64_t c = 0; c < g.n_c; ++c)
     for (int p = 0; p < g.R; ++p)
-      em.chunk_op(PL_OP_COPY, root, 0, ref(root, PL_BUF_OUT, PL_U8, (p * g.P + c * g.chunk) * g.es), false,
+      em.chunk_op(PL_OP_COPY, p, 0, ref(root, PL_BUF_OUT, PL_U8, (p * g.P + c * g.chunk) * g.es), false,
                   {ref(p, PL_BUF_IN, PL_U8, c * g.chunk * g.es)}, g.clen(c) * g.es, {}, -1);
 }
 
@@ -296,29 +298,17 @@ void broadcast_composed(Emitter& em, const Geo& g, int root) {
 }
 
 // reduce = compose<reduce-scatter, gather>: rank k reduces chunk c of partition k (ascending
-// rank order) into its scratch -- the root straight into its output -- and the root gathers.
+// rank order) and, the gather being a push, writes the result straight into partition k of
+// the root's output: one pass, no intermediate buffer, no flags.
 void reduce_composed(Emitter& em, const Geo& g, int root) {
-  std::vector<int> reduced(g.R * g.n_c, -1);
   em.phase_chunks = g.n_c;
   for (uint64_t c = 0; c < g.n_c; ++c)
     for (int k = 0; k < g.R; ++k) {
       std::vector<pl_ref_t> src;
       const uint64_t off = (k * g.P + c * g.chunk) * g.es;
       for (int p = 0; p < g.R; ++p) src.push_back(ref(p, PL_BUF_IN, g.dtype, off));
-      pl_ref_t d = (k == root) ? ref(root, PL_BUF_OUT, g.dtype, off) : ref(k, PL_BUF_SCRATCH, g.dtype, c * g.chunk * g.es);
-      int f = -1;
-      if (k != root) f = reduced[k * g.n_c + c] = em.new_flag();
-      em.chunk_op(PL_OP_REDUCE, k, 0, d, false, src, g.clen(c), {}, f);
+      em.chunk_op(PL_OP_REDUCE, k, 0, ref(root, PL_BUF_OUT, g.dtype, off), false, src, g.clen(c), {}, -1);
     }
-  em.phase_chunks = g.n_c * (g.R - 1);
-  for (uint64_t c = 0; c < g.n_c; ++c)
-    for (int k = 0; k < g.R; ++k) {
-      if (k == root) continue;
-      em.chunk_op(PL_OP_COPY, root, 0, ref(root, PL_BUF_OUT, PL_U8, (k * g.P + c * g.chunk) * g.es), false,
-                  {ref(k, PL_BUF_SCRATCH, PL_U8, c * g.chunk * g.es)}, g.clen(c) * g.es, {reduced[k * g.n_c + c]}, -1);
-    }
-  for (int k = 0; k < g.R; ++k)
-    if (k != root) em.L->scratch_per_rank[k] = g.P * g.es;
 }
 
 // all-reduce, one-shot: every rank reduces the whole message from all R inputs.
