@@ -39,6 +39,13 @@ struct Emitter {
   uint32_t min_slice = 16384, max_slice = 131072;
   double op_overhead_us = 1.5, wait_overhead_us = 0.5;
   int role = 0;  // role stamped on emitted ops
+  // Non-zero: COPY ops are cut into slices of exactly this many bytes (short tail), dealt
+  // round-robin over the rank's queues.  Set for all-to-all on the bulk-copy datapath, where
+  // every byte is read once from HBM and written once: the CTAs of a rank then sweep one
+  // compact window of the source and one of the destination instead of 18 separate regions
+  // (measured on B200, R = 8: 64 MiB per rank 185 -> 169 us, 256 MiB 694 -> 644 us; all-gather,
+  // whose sources are re-read from L2, prefers the coarse slices of the cost model).
+  uint32_t stream_slice = 0;
 
   int new_flag() { return L->n_flags++; }
 
@@ -56,7 +63,9 @@ struct Emitter {
     const uint64_t unit16 = kind == PL_OP_COPY ? 16 : 16 / elem_size(dtype);
     uint64_t wide = count * max_es;
     uint64_t n_slices = 1;
-    if (slice_bytes) {
+    if (stream_slice && kind == PL_OP_COPY && !slice_bytes) {
+      n_slices = std::max<uint64_t>(1, (wide + stream_slice - 1) / stream_slice);
+    } else if (slice_bytes) {
       if (wide > (uint64_t)slice_bytes + slice_bytes / 2) n_slices = (wide + slice_bytes - 1) / slice_bytes;
     } else {
       // Pick the slice count that minimises the time of the phase under a simple model: a rank
@@ -85,6 +94,7 @@ struct Emitter {
     uint64_t per = (count + n_slices - 1) / n_slices;
     uint64_t unit = (per >= 64 * unit16) ? 8 * unit16 : unit16;
     per = (per + unit - 1) / unit * unit;
+    if (stream_slice && kind == PL_OP_COPY && !slice_bytes && n_slices > 1) per = stream_slice;  // COPY counts are bytes
     for (uint64_t b = 0; b < count; b += per) {
       HostOp op;
       op.kind = kind;
@@ -804,6 +814,7 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
       }
     L->message_bytes = total / R;
     em.phase_chunks = 0;
+    if (rq.pol.datapath == PL_DP_TMA) em.stream_slice = 32768;
     a2av_direct(em, R, dt, rq.counts_v, rq.chunk_bytes);
     return PL_OK;
   }
@@ -868,7 +879,10 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
       for (int r = 0; r < R; ++r) L->in_bytes[r] = L->out_bytes[r] = bytes;
       L->message_bytes = bytes;
       if (rq.staged) a2a_direct_staged(em, g, rq.staging_bytes);
-      else a2a_direct(em, g);
+      else {
+        if (rq.pol.datapath == PL_DP_TMA) em.stream_slice = 32768;
+        a2a_direct(em, g);
+      }
       return PL_OK;
     }
     case PL_REDUCE_SCATTER: {
