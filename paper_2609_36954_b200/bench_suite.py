@@ -235,7 +235,7 @@ def probe(b):
 
 
 def main(args=None):
-    which = os.environ.get("PL_SUITE", "probe,c1,c2,staged,varlen,rooted,c3,c4,c5").split(",")
+    which = os.environ.get("PL_SUITE", "probe,c1,c2,a2a,staged,varlen,rooted,c3,c4,c5").split(",")
     out = os.environ.get("PL_SUITE_OUT")  # optional file that receives the JSON lines too
     if out and os.path.dirname(out):
         os.makedirs(os.path.dirname(out), exist_ok=True)
@@ -269,6 +269,14 @@ def main(args=None):
             for name, coll, count in (("broadcast", B.PL_BROADCAST, size // 2), ("reduce", B.PL_REDUCE, size // 2),
                                       ("scatter", B.PL_SCATTER, size // 16), ("gather", B.PL_GATHER, size // 16)):
                 b.collective("rooted-" + name, 8, B.PL_BF16, coll, "direct", count, MIB, root=0, graph=size < MIB)
+    if "a2a" in which:
+        # all-to-all: a pure copy, every byte read once from HBM and written once (64 MiB per rank first:
+        # the case the profiler summary under profiles/ captures)
+        for mib in (64, 16, 256):
+            b.collective("A2A", 8, B.PL_BF16, B.PL_ALLTOALL, "direct", mib * MIB // 2, MIB)
+        # slice size of the copy ops: the cost model's coarse slices against the 32 KiB sweep
+        for sl in (262144, 131072, 65536, 32768, 16384):
+            b.collective(f"A2A-slice{sl >> 10}K", 8, B.PL_BF16, B.PL_ALLTOALL, "direct", 32 * MIB, MIB, slice_bytes=sl)
     if "ablation" in which:
         # (a) pipeline depth at a fixed CTA count: the analogue of the paper's copy ablation
         #     (Sec. 5, "ablation": bandwidth vs. number of stages S at fixed stage size)
