@@ -642,3 +642,35 @@ def test_overlapped_launches_keep_stream_order(dp):
             check()
     finally:
         ses.close()
+
+
+def test_two_schedules_overlap_on_two_streams_when_co_resident():
+    """Executes of different schedules may overlap on the GPU when their grids fit together
+    (32 + 32 CTAs here): both chains of flag waits make progress and both results are right."""
+    import torch
+    from gpu_harness import poison
+    R, n = 4, 4 * 20000
+    x1 = gen.rank_inputs(R, n, "i32", seed=0)
+    x2 = [v + 7 for v in x1]
+    ref1, ref2 = oracle.allreduce(x1, "i32"), oracle.allreduce(x2, "i32")
+    ses = Session(R, "i32")
+    try:
+        s1 = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 4096, n_ctas=32, datapath=B.PL_DP_LDST)
+        s2 = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_TREE, n, 4096, n_ctas=32, datapath=B.PL_DP_LDST)
+        nb = n * 4
+        d1, d2 = [to_dev(v) for v in x1], [to_dev(v) for v in x2]
+        o1, o2 = [poison(nb) for _ in range(R)], [poison(nb) for _ in range(R)]
+        b1 = B.make_bufs([t.data_ptr() for t in d1], [t.data_ptr() for t in o1], [nb] * R, [nb] * R)
+        b2 = B.make_bufs([t.data_ptr() for t in d2], [t.data_ptr() for t in o2], [nb] * R, [nb] * R)
+        st1, st2 = torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+        for _ in range(50):
+            B.pl_execute(s1, b1, st1.cuda_stream)
+            B.pl_execute(s2, b2, st2.cuda_stream)
+        torch.cuda.synchronize()
+        assert B.pl_comm_status(ses.comm).code == B.PL_OK
+        for r in range(R):
+            assert np.array_equal(o1[r].cpu().numpy().view(np.int32), ref1[r])
+            assert np.array_equal(o2[r].cpu().numpy().view(np.int32), ref2[r])
+    finally:
+        ses.close()
