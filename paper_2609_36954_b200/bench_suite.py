@@ -317,7 +317,7 @@ def main(args=None):
                 # message for one-shot and tree
                 chunk = max(16, min(MIB, size if algo in ("oneshot", "tree") else size // 8))
                 b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30 if lg < 24 else 10,
-                             graph=lg <= 21)
+                             graph=lg <= 24)
                 # latency-bound sizes again with overlapped launches (CTAs of call i+1 set up while call i drains)
                 if lg <= 20 and algo in ("oneshot", "fused"):
                     b.collective("C3-overlap", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30, graph=True,

@@ -84,11 +84,18 @@ __global__ void __launch_bounds__(1024) moe_scan_kernel(const __grid_constant__ 
   for (int pe = tid; pe < g.R * g.E; pe += n) {
     const int p = pe / g.E, e = pe % g.E;
     int run = 0;
-    for (int b = 0; b < g.NB; ++b) {
-      int32_t* c = g.blockcnt + ((size_t)p * g.NB + b) * g.E + e;
-      const int v = *c;
-      *c = run;
-      run += v;
+    // exclusive scan over the token blocks, eight independent loads at a time
+    for (int b0 = 0; b0 < g.NB; b0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        v[i] = (b0 + i < g.NB) ? g.blockcnt[((size_t)p * g.NB + b0 + i) * g.E + e] : 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (b0 + i < g.NB) {
+          g.blockcnt[((size_t)p * g.NB + b0 + i) * g.E + e] = run;
+          run += v[i];
+        }
     }
     g.ecounts[pe] = run;
   }
