@@ -461,6 +461,21 @@ pl_status_t pl_moe_combine_dedup(pl_moe_plan_t plan, const void* const* z, void*
  * [R][T][R] = row of (p, t) at rank r or -1; counts int64 [R][R].  Synchronises `stream`. */
 pl_status_t pl_moe_plan_read_dedup(pl_moe_plan_t plan, int32_t* pos, int64_t* counts, void* stream);
 
+/* ---- diagnostic: stream ceilings of the bulk-copy machinery ------------------------ */
+
+/* NOT PART OF THE PAPER'S METHOD.  Enqueues one kernel on `stream` that streams `bytes` with
+ * the instructions the executors use (bulk asynchronous copies through a shared-memory ring,
+ * one CTA per SM): kind 0 reads src and drops the data, kind 1 writes zeros to dst, kind 2
+ * copies src to dst.  Timed with CUDA events by the caller it gives the pure-read, pure-write
+ * and copy bandwidth that bound the read-dominated (reduce-scatter, MoE combine), write-
+ * dominated (all-gather, MoE dispatch) and balanced (all-to-all) collectives on this GPU.
+ *   src, dst  DEVICE pointers, 16-byte aligned, `bytes` long (src unused for kind 1, dst for
+ *             kind 0); bytes a positive multiple of 32768
+ *   status    optional DEVICE word of the caller: cleared on `stream`, set to PL_ERR_TIMEOUT if
+ *             a wait inside the kernel gave up (2 s); may be NULL
+ * Errors (before any launch): PL_ERR_INVALID_ARG, PL_ERR_ALIGNMENT, PL_ERR_CUDA. */
+pl_status_t pl_probe_hbm(int kind, const void* src, void* dst, size_t bytes, int32_t* status, void* stream);
+
 const char* pl_status_string(pl_status_t st);
 
 /* Number of kernels this library has launched in the calling process (all entry points). */

@@ -232,6 +232,11 @@ def probe(b):
                              ("torch sum fp32 (read)", lambda: af.sum(), n)):
         us, _, _ = _time(fn, 20)
         b.emit({"cfg": "probe", "what": name, "gbs": nbytes / us / 1e3})
+    # the same three streams through the library's own bulk-copy ring (pl_probe_hbm)
+    h = torch.cuda.current_stream().cuda_stream
+    for name, kind, nbytes in (("bulk-copy ring: read", 0, n), ("bulk-copy ring: write", 1, n), ("bulk-copy ring: copy", 2, 2 * n)):
+        us, _, _ = _time(lambda: B.pl_probe_hbm(kind, a.data_ptr(), c.data_ptr(), n, 0, h), 20)
+        b.emit({"cfg": "probe", "what": name, "gbs": nbytes / us / 1e3})
 
 
 def main(args=None):

@@ -89,7 +89,7 @@ class pl_devstatus_t(C.Structure):
 
 EXPORTS = [
     "pl_comm_create", "pl_comm_create_planner", "pl_comm_destroy", "pl_comm_status", "pl_comm_reset",
-    "pl_comm_last_error",
+    "pl_comm_last_error", "pl_probe_hbm",
     "pl_schedule_build", "pl_schedule_build_v", "pl_schedule_build_layers", "pl_schedule_build_rooted", "pl_schedule_info",
     "pl_schedule_dump", "pl_schedule_validate", "pl_schedule_debug_break_wait", "pl_schedule_debug_drop_wait",
     "pl_schedule_trace_read", "pl_schedule_destroy",
@@ -157,6 +157,7 @@ def load():
     L.pl_status_string.restype = C.c_char_p
     L.pl_comm_last_error.argtypes = [vp]
     L.pl_comm_last_error.restype = C.c_char_p
+    L.pl_probe_hbm.argtypes = [C.c_int, vp, vp, C.c_size_t, vp, vp]
     L.pl_launch_count.argtypes = []
     L.pl_launch_count.restype = C.c_uint64
     _lib = L
@@ -220,6 +221,11 @@ def pl_comm_status(comm):
 
 def pl_comm_last_error(comm) -> str:
     return load().pl_comm_last_error(comm).decode()
+
+
+def pl_probe_hbm(kind: int, src: int, dst: int, nbytes: int, status: int = 0, stream=0) -> None:
+    """kind 0 read, 1 write, 2 copy; src / dst / status are device addresses (0 = unused)."""
+    _check(load().pl_probe_hbm(kind, src or None, dst or None, nbytes, status or None, stream), "pl_probe_hbm")
 
 
 def pl_comm_reset(comm, stream=0):

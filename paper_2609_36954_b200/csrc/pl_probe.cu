@@ -1,0 +1,131 @@
+// Diagnostic: what the bulk-copy machinery of the executors reaches on plain streams.
+//
+// Not part of the paper's method.  The roofline fractions of the collectives are quoted against
+// a library copy; this probe measures, with the same instructions the executors use
+// (cp.async.bulk global->shared with mbarrier completion, cp.async.bulk shared->global), the
+// three ceilings that bound them: a pure read (reduce-scatter and MoE combine are 8 reads to
+// 1 write), a pure write (all-gather and MoE dispatch are write dominated) and a copy.
+//
+// One warp per CTA, one CTA per SM, a ring of 6 tiles of 32 KiB.  CTA c handles tiles
+// c, c + G, c + 2G, ...: at any moment the grid sweeps one compact window of the buffer.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "pl_api_internal.h"
+#include "pl_ptx.cuh"
+#include "purlin.h"
+
+using namespace pl;
+
+namespace {
+
+constexpr uint32_t kTile = 32768;
+constexpr uint32_t kSlots = 6;
+constexpr size_t kSmem = 128 + (size_t)kSlots * kTile;
+constexpr unsigned long long kLimitNs = 2000000000ull;
+
+__device__ __forceinline__ unsigned long long now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// bounded wait on a "tile landed" barrier; false when the time limit passed
+__device__ __forceinline__ bool wait_full(uint64_t* bar, uint32_t parity) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = now_ns();
+  for (uint32_t tries = 1;; ++tries) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((tries & 1023u) == 0 && now_ns() - t0 > kLimitNs) return false;
+  }
+}
+
+// kind 0: read (tiles are loaded and dropped), 1: write (tiles of zeros are stored), 2: copy
+__global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src, char* dst, unsigned long long n_tiles,
+                                                      int* status) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);
+  unsigned char* tiles = smem + 128;
+  const int lane = threadIdx.x;
+  if (kind == 1) {
+    for (uint32_t i = lane; i < kSlots * kTile / 16; i += 32) reinterpret_cast<uint4*>(tiles)[i] = make_uint4(0, 0, 0, 0);
+    ptx::fence_proxy_async_smem();
+  }
+  if (lane == 0) {
+    for (uint32_t s = 0; s < kSlots; ++s) ptx::mbar_init(full + s, 1);
+    ptx::mbar_init_fence();
+  }
+  __syncwarp();
+  if (lane != 0) return;
+  const unsigned long long c = blockIdx.x, G = gridDim.x;
+  if (c >= n_tiles) return;
+  const unsigned long long n_my = (n_tiles - c + G - 1) / G;
+  auto tile_off = [&](unsigned long long n) { return (c + n * G) * (unsigned long long)kTile; };
+  unsigned long long issued = 0;  // loads issued so far (tiles 0 .. issued-1 of this CTA)
+  auto load = [&](unsigned long long n) {
+    const uint32_t s = (uint32_t)(n % kSlots);
+    ptx::mbar_expect_tx(full + s, kTile);
+    ptx::bulk_g2s(tiles + (size_t)s * kTile, src + tile_off(n), kTile, full + s);
+    issued = n + 1;
+  };
+  bool ok = true;
+  unsigned long long n = 0;
+  if (kind != 1)
+    for (unsigned long long k = 0; k < n_my && k < kSlots; ++k) load(k);
+  for (; n < n_my; ++n) {
+    const uint32_t s = (uint32_t)(n % kSlots), parity = (uint32_t)((n / kSlots) & 1);
+    if (kind != 1 && !(ok = wait_full(full + s, parity))) break;
+    if (kind == 0) {
+      if (n + kSlots < n_my) load(n + kSlots);  // the tile is dropped: its slot is free at once
+      continue;
+    }
+    ptx::bulk_s2g(dst + tile_off(n), tiles + (size_t)s * kTile, kTile);
+    ptx::bulk_commit();
+    if (kind == 2 && n >= 2) {
+      ptx::bulk_wait_read<2>();  // the store of tile n-2 no longer reads its slot
+      if (n - 2 + kSlots < n_my) load(n - 2 + kSlots);
+    } else if (kind == 1) {
+      ptx::bulk_wait_read<8>();  // bounds the stores in flight; the zero tiles are never rewritten
+    }
+  }
+  ptx::bulk_wait<0>();
+  if (!ok) {
+    if (status) *status = PL_ERR_TIMEOUT;
+    // loads already issued may still land: give each a bounded chance before leaving
+    for (unsigned long long k = n; k < issued; ++k) {
+      const uint32_t s = (uint32_t)(k % kSlots), parity = (uint32_t)((k / kSlots) & 1);
+      for (uint32_t tries = 0; tries < (1u << 20) && !ptx::mbar_try_wait(full + s, parity); ++tries) {}
+    }
+  }
+}
+
+}  // namespace
+
+extern "C" pl_status_t pl_probe_hbm(int kind, const void* src, void* dst, size_t bytes, int32_t* status, void* stream) {
+  if (kind < 0 || kind > 2 || bytes == 0 || bytes % kTile) return PL_ERR_INVALID_ARG;
+  if ((kind != 1 && !src) || (kind != 0 && !dst)) return PL_ERR_INVALID_ARG;
+  if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15)) return PL_ERR_ALIGNMENT;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return PL_ERR_CUDA;
+  }
+  static std::atomic<unsigned long long> configured{0};  // shared-memory opt-in, one bit per device
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (!(configured.load(std::memory_order_acquire) & bit)) {
+    if (cudaFuncSetAttribute(pl_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem) != cudaSuccess) {
+      cudaGetLastError();
+      return PL_ERR_CUDA;
+    }
+    configured.fetch_or(bit, std::memory_order_release);
+  }
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (status && cudaMemsetAsync(status, 0, sizeof(int32_t), cs) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  pl_probe_kernel<<<sms, 32, kSmem, cs>>>(kind, static_cast<const char*>(src), static_cast<char*>(dst),
+                                          (unsigned long long)(bytes / kTile), reinterpret_cast<int*>(status));
+  if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return PL_OK;
+}

@@ -674,3 +674,27 @@ def test_two_schedules_overlap_on_two_streams_when_co_resident():
             assert np.array_equal(o2[r].cpu().numpy().view(np.int32), ref2[r])
     finally:
         ses.close()
+
+
+def test_stream_probe_copies_and_zero_fills():
+    """pl_probe_hbm: the copy stream reproduces its source bit for bit, the write stream leaves
+    zeros, the read stream leaves its source alone; no wait gives up; bad sizes are refused."""
+    import torch
+    n = 32768 * 301  # ragged against the 148-CTA sweep
+    src = torch.randint(0, 255, (n,), dtype=torch.uint8, device="cuda")
+    keep = src.clone()
+    dst = torch.full((n + 32768,), 7, dtype=torch.uint8, device="cuda")
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    h = torch.cuda.current_stream().cuda_stream
+    B.pl_probe_hbm(2, src.data_ptr(), dst.data_ptr(), n, status.data_ptr(), h)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(dst[:n], src) and bool((dst[n:] == 7).all())
+    B.pl_probe_hbm(1, 0, dst.data_ptr(), n, status.data_ptr(), h)
+    B.pl_probe_hbm(0, src.data_ptr(), 0, n, status.data_ptr(), h)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and bool((dst[:n] == 0).all()) and bool((dst[n:] == 7).all())
+    assert torch.equal(src, keep)
+    with pytest.raises(B.PurlinError):
+        B.pl_probe_hbm(2, src.data_ptr(), dst.data_ptr(), n - 16, 0, h)
+    with pytest.raises(B.PurlinError):
+        B.pl_probe_hbm(2, 0, dst.data_ptr(), n, 0, h)
