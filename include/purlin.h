@@ -465,8 +465,8 @@ pl_status_t pl_moe_plan_read_dedup(pl_moe_plan_t plan, int32_t* pos, int64_t* co
 
 /* NOT PART OF THE PAPER'S METHOD.  Enqueues one kernel on `stream` that streams `bytes` with
  * the instructions the executors use (bulk asynchronous copies through a shared-memory ring,
- * one CTA per SM): kind 0 reads src and drops the data, kind 1 writes zeros to dst, kind 2
- * copies src to dst.  Timed with CUDA events by the caller it gives the pure-read, pure-write
+ * one CTA per SM): kind 0 reads src and drops the data, kind 1 fills dst with a fixed pattern
+ * (32-bit word j of every 32 KiB tile = j * 2654435761 mod 2^32), kind 2 copies src to dst.  Timed with CUDA events by the caller it gives the pure-read, pure-write
  * and copy bandwidth that bound the read-dominated (reduce-scatter, MoE combine), write-
  * dominated (all-gather, MoE dispatch) and balanced (all-to-all) collectives on this GPU.
  *   src, dst  DEVICE pointers, 16-byte aligned, `bytes` long (src unused for kind 1, dst for

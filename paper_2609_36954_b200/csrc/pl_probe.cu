@@ -42,7 +42,7 @@ __device__ __forceinline__ bool wait_full(uint64_t* bar, uint32_t parity) {
   }
 }
 
-// kind 0: read (tiles are loaded and dropped), 1: write (tiles of zeros are stored), 2: copy
+// kind 0: read (tiles are loaded and dropped), 1: write (a fixed pattern tile is stored), 2: copy
 __global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src, char* dst, unsigned long long n_tiles,
                                                       int* status) {
   extern __shared__ __align__(128) unsigned char smem[];
@@ -50,7 +50,8 @@ __global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src,
   unsigned char* tiles = smem + 128;
   const int lane = threadIdx.x;
   if (kind == 1) {
-    for (uint32_t i = lane; i < kSlots * kTile / 16; i += 32) reinterpret_cast<uint4*>(tiles)[i] = make_uint4(0, 0, 0, 0);
+    // every tile carries the same non-constant pattern: 32-bit word j of a tile = j * 2654435761
+    for (uint32_t i = lane; i < kSlots * kTile / 4; i += 32) reinterpret_cast<uint32_t*>(tiles)[i] = (i % (kTile / 4)) * 2654435761u;
     ptx::fence_proxy_async_smem();
   }
   if (lane == 0) {
@@ -87,7 +88,7 @@ __global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src,
       ptx::bulk_wait_read<2>();  // the store of tile n-2 no longer reads its slot
       if (n - 2 + kSlots < n_my) load(n - 2 + kSlots);
     } else if (kind == 1) {
-      ptx::bulk_wait_read<8>();  // bounds the stores in flight; the zero tiles are never rewritten
+      ptx::bulk_wait_read<8>();  // bounds the stores in flight; the pattern tiles are never rewritten
     }
   }
   ptx::bulk_wait<0>();

@@ -678,7 +678,7 @@ def test_two_schedules_overlap_on_two_streams_when_co_resident():
 
 def test_stream_probe_copies_and_zero_fills():
     """pl_probe_hbm: the copy stream reproduces its source bit for bit, the write stream leaves
-    zeros, the read stream leaves its source alone; no wait gives up; bad sizes are refused."""
+    its pattern, the read stream leaves its source alone; no wait gives up; bad sizes are refused."""
     import torch
     n = 32768 * 301  # ragged against the 148-CTA sweep
     src = torch.randint(0, 255, (n,), dtype=torch.uint8, device="cuda")
@@ -692,7 +692,8 @@ def test_stream_probe_copies_and_zero_fills():
     B.pl_probe_hbm(1, 0, dst.data_ptr(), n, status.data_ptr(), h)
     B.pl_probe_hbm(0, src.data_ptr(), 0, n, status.data_ptr(), h)
     torch.cuda.synchronize()
-    assert int(status.item()) == 0 and bool((dst[:n] == 0).all()) and bool((dst[n:] == 7).all())
+    pattern = torch.from_numpy(((np.arange(8192, dtype=np.uint64) * 2654435761) % (1 << 32)).astype(np.uint32).view(np.int32)).cuda()
+    assert int(status.item()) == 0 and bool((dst[:n].view(torch.int32).view(-1, 8192) == pattern).all()) and bool((dst[n:] == 7).all())
     assert torch.equal(src, keep)
     with pytest.raises(B.PurlinError):
         B.pl_probe_hbm(2, src.data_ptr(), dst.data_ptr(), n - 16, 0, h)
