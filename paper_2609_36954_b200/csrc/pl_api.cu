@@ -39,6 +39,7 @@ struct pl_schedule_s {
   bool no_l2_hints = false;
   bool trace = false;
   bool overlap_launch = false;
+  bool pipelined_reduce = false;  // bulk-copy datapath: every reduce op is plain, run the 12-warp variant
   size_t off_trace = 0;
   float out_scale = 1.0f;
   // host copies in device (queue-major) order
@@ -215,7 +216,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   if (pol.datapath == PL_DP_TMA) {
     if (pol.stages < 2 || pol.stages > 8 || pol.stage_bytes < 1024 || exec_tma_smem_bytes(pol.stages, pol.stage_bytes) > 227 * 1024)
       return PL_ERR_INVALID_ARG;
-    pol.threads = exec_tma_threads();
+    pol.threads = exec_tma_threads(false);
     rq.pol.threads = pol.threads;
   }
   int capacity = 148 * (pol.datapath == PL_DP_TMA ? 2 : 1);
@@ -262,6 +263,20 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
       delete S;
       return st;
     }
+  }
+  if (pol.datapath == PL_DP_TMA && comm->dtype != PL_U8) {
+    // Plain reduce ops only (element-typed sources and destination, one destination, at most 8
+    // sources): the kernel variant with the software-pipelined consumers applies.
+    bool any = false, plain = true;
+    for (const HostOp& op : S->L.ops) {
+      if (op.kind == PL_OP_COPY) continue;
+      any = true;
+      if (op.bcast || op.src.size() > 8 || op.dst.dtype != comm->dtype) plain = false;
+      for (const pl_ref_t& r : op.src)
+        if (r.dtype != comm->dtype) plain = false;
+    }
+    S->pipelined_reduce = any && plain;
+    S->pol.threads = exec_tma_threads(S->pipelined_reduce);
   }
   fill_info(S, comm->R);
   flatten(S, comm->dtype);
@@ -570,6 +585,7 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   P.hints = s->no_l2_hints ? 0u : 6u;
   P.out_scale = s->out_scale;
   P.overlap_launch = s->overlap_launch ? 1u : 0u;
+  P.pipelined_reduce = s->pipelined_reduce ? 1u : 0u;
   cudaError_t le = s->pol.datapath == PL_DP_TMA
                        ? launch_exec_tma(s->comm->dtype, P, s->pol.n_ctas, static_cast<cudaStream_t>(stream))
                        : launch_exec(s->comm->dtype, P, s->pol.n_ctas, s->pol.threads, static_cast<cudaStream_t>(stream));

@@ -15,7 +15,8 @@ int exec_max_threads();
 // TMA (bulk-copy, shared-memory ring) executor
 cudaError_t launch_exec_tma(int dtype, const ExecParams& P, int grid, cudaStream_t stream);
 int exec_tma_max_ctas_per_sm(int dtype, int stages, uint32_t stage_bytes);
-int exec_tma_threads();
+// threads per CTA of the two variants: general (16 consumer warps) and pipelined reduce (12)
+int exec_tma_threads(bool pipelined);
 size_t exec_tma_smem_bytes(int stages, uint32_t stage_bytes);
 
 }  // namespace pl
