@@ -273,7 +273,9 @@ const char* pl_comm_last_error(pl_comm_t comm);
  *                   all-reduce, reduce-scatter and all-to-all; the per-rank CONTRIBUTION
  *                   for all-gather (output = R * count_per_rank).
  *   chunk_bytes     chunk size in bytes of the element type (multiple of 16); clipped to
- *                   the partition size; the last chunk of a partition may be short.
+ *                   the partition size; the last chunk of a partition may be short.  It is
+ *                   the granularity of the flags; a schedule whose ops neither wait nor
+ *                   signal (direct all-gather) may be cut into smaller chunks.
  * Partitioned collectives need count_per_rank * elem_size divisible by R*16
  * (PL_ERR_INVALID_ARG).  PL_ERR_UNSUPPORTED for algorithm/collective pairs that do not
  * exist (tree, one-shot and fused are all-reduce only; PL_U8 cannot be reduced).

@@ -872,8 +872,14 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
       L->message_bytes = bytes * R;
       if (rq.staged && rq.algo != PL_ALGO_DIRECT) return fail(PL_ERR_UNSUPPORTED, "staged schedules are direct only");
       if (rq.staged) ag_direct_staged(em, g, rq.staging_bytes);
-      else if (rq.algo == PL_ALGO_DIRECT) ag_direct(em, g);
-      else if (rq.algo == PL_ALGO_RING) ag_ring(em, g, false, nullptr);
+      else if (rq.algo == PL_ALGO_DIRECT) {
+        // No op of a direct all-gather waits or signals, so the chunk size only orders the copy
+        // ops.  On the bulk-copy datapath at most 512 KiB per chunk: the ranks then walk the
+        // sources in step and the seven re-reads of a contribution hit L2 (measured, R = 8,
+        // 64 MiB gathered per rank: 108.5 us with 1 MiB chunks, 105 us with 256 or 512 KiB).
+        if (rq.pol.datapath == PL_DP_TMA && rq.chunk_bytes > (512u << 10)) g = make_geo(R, dt, n * R, n, 512u << 10);
+        ag_direct(em, g);
+      } else if (rq.algo == PL_ALGO_RING) ag_ring(em, g, false, nullptr);
       else return fail(PL_ERR_UNSUPPORTED, "all-gather supports direct and ring");
       return PL_OK;
     }
