@@ -36,6 +36,25 @@ __device__ __forceinline__ void body_copy(char* dst, const char* src, uint64_t b
   for (; i < n; i += nthr) st16(dst + (i << 4), ld16(src + (i << 4)));
 }
 
+// The same bytes to the same offset of every rank's output (a pushed all-gather contribution).
+__device__ __forceinline__ void body_copy_bcast(const ExecParams& P, uint64_t dst_off, const char* src, uint64_t bytes,
+                                                int tid, int nthr) {
+  const uint64_t n = bytes >> 4;
+  constexpr int U = 4;
+  for (uint64_t i = tid; i < n; i += (uint64_t)U * nthr) {
+    uint4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (i + (uint64_t)u * nthr < n) v[u] = ld16(src + ((i + (uint64_t)u * nthr) << 4));
+    for (int k = 0; k < P.n_ranks; ++k) {
+      char* d = static_cast<char*>(P.base[kSlotOut + k]) + dst_off;
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (i + (uint64_t)u * nthr < n) st16(d + ((i + (uint64_t)u * nthr) << 4), v[u]);
+    }
+  }
+}
+
 // Add NB same-typed sources (ascending) for U units at once: all loads first, then the adds.
 template <int DT, int NB, int U>
 __device__ __forceinline__ void accumulate_batch(Acc<DT> (&acc)[U], const char* const* src, const uint64_t (&off)[U]) {
@@ -280,7 +299,8 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
     const DevOp& op = S.op;
     if (P.trace && tid == 0) P.trace[2ull * op.topo] = globaltimer_ns();  // waits satisfied
     if (op.kind == PL_OP_COPY) {
-      body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
+      if (op.flags & kDstBcast) body_copy_bcast(P, op.dst & 0xFFFFFFFFFFFFull, S.src[0], op.count, tid, nthr);
+      else body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
     } else if (op.kind == PL_OP_REDUCE) {
       if constexpr (DT != PL_U8) body_reduce<DT>(P, op, S.src, tid, nthr);
     } else {

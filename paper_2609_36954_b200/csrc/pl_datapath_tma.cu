@@ -366,7 +366,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
         __syncwarp();
         if (lane < (int)n_src) {
           void* sdst = slots + (size_t)s * slot_bytes + my_tile_off;
-          if ((P.hints & 4u) && kind == PL_OP_COPY) ptx::bulk_g2s_hint(sdst, my_src + u0 * my_w, units * my_w, &c->full[s], ptx::policy_evict_last());
+          if ((P.hints & 4u) && kind == PL_OP_COPY && !(oflags & kDstBcast)) ptx::bulk_g2s_hint(sdst, my_src + u0 * my_w, units * my_w, &c->full[s], ptx::policy_evict_last());
           else if (P.hints & 1u) ptx::bulk_g2s_hint(sdst, my_src + u0 * my_w, units * my_w, &c->full[s], ptx::policy_evict_first());
           else ptx::bulk_g2s(sdst, my_src + u0 * my_w, units * my_w, &c->full[s]);
         }
@@ -402,6 +402,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
       const uint32_t kind = d.kind;
       if (kind == kEnd) break;
       const bool via_smem = leaves_via_smem(kind, d.flags, d.pmask);
+      const bool to_all = via_smem || (kind == PL_OP_COPY && (d.flags & kDstBcast));  // one tile, R destinations
       const bool uses_done = via_smem || (kind != PL_OP_COPY && (d.flags & kLastOfOp) && d.signal != kNoFlag);
       if (via_smem) {
         bool ready = true;
@@ -412,7 +413,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
       if (uses_done) done_parity ^= 1u << s;
       if (lane == 0) {
         if (kind == PL_OP_COPY || via_smem) {
-          if (via_smem) {
+          if (to_all) {
             for (int k = 0; k < P.n_ranks; ++k) {
               void* dk = static_cast<char*>(P.base[kSlotOut + k]) + d.dst_off;
               if (P.hints & 2u) ptx::bulk_s2g_hint(dk, slots + (size_t)s * slot_bytes, d.units * 16u, ptx::policy_evict_first());

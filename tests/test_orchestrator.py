@@ -203,12 +203,15 @@ def test_schedule_bytes_match_closed_forms_bf16_R8():
     n = M // 2
     pl = Planner(R, "bf16")
     try:
-        def total(coll, algo, count=n):
-            i = B.pl_schedule_info(pl.build(coll, algo, count, 1 << 16))
+        def total(coll, algo, count=n, **kw):
+            i = B.pl_schedule_info(pl.build(coll, algo, count, 1 << 16, **kw))
             return i.bytes_read + i.bytes_written
         assert total(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT) == (R + 1) * M
         assert total(B.PL_REDUCE_SCATTER, B.PL_ALGO_RING) == 33 * M  # fp32 partials: (16+10(R-3))/2 per byte
-        assert total(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R) == 2 * R * M  # per-rank-message M = gathered size
+        # per-rank-message M = gathered size; pulled (bulk-copy path): every rank reads and writes it all;
+        # pushed (register path): each contribution is read once and written R times
+        assert total(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, datapath=B.PL_DP_TMA) == 2 * R * M
+        assert total(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, datapath=B.PL_DP_LDST) == (R + 1) * M
         assert total(B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT) == R * (R + 1) * M
         assert total(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT) == (3 * R - 1) * M
         assert total(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT_FUSED) == 2 * R * M
