@@ -101,7 +101,9 @@ typedef enum {
 } pl_collective_t;
 
 /* Algorithms.
- *   PL_ALGO_DIRECT        every consumer pulls straight from the producers' buffers.  For
+ *   PL_ALGO_DIRECT        every consumer pulls straight from the producers' buffers (small
+ *                         all-gathers, whose working set sits in L2, are pushed instead: the
+ *                         producer writes its contribution into every output).  For
  *                         all-reduce this is Algorithm 1 without the staging role: rank k
  *                         reduces partition k from all inputs into its own output,
  *                         publishes reduced(k, c), and every other rank copies that chunk.

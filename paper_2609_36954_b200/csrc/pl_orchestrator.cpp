@@ -311,27 +311,18 @@ void gather_direct(Emitter& em, const Geo& g, int root) {
                   {ref(p, PL_BUF_IN, PL_U8, c * g.chunk * g.es)}, g.clen(c) * g.es, {}, -1);
 }
 
-// broadcast = compose<scatter, all-gather>: rank k pulls chunk c of partition k from the root
-// into its own output and publishes it; every other rank then pulls it from rank k.
+// broadcast = compose<scatter, all-gather> with both copies folded into one op: rank k takes
+// chunk c of partition k from the root's input (the scatter) and writes it into every rank's
+// output (the all-gather, as a push).  One phase, no flags, every rank's queues share the work;
+// the root's buffer is read once.
 void broadcast_composed(Emitter& em, const Geo& g, int root) {
-  std::vector<int> have(g.R * g.n_c);
   em.phase_chunks = g.n_c;
   for (uint64_t c = 0; c < g.n_c; ++c)
     for (int k = 0; k < g.R; ++k) {
       const uint64_t off = (k * g.P + c * g.chunk) * g.es;
-      have[k * g.n_c + c] = em.new_flag();
-      em.chunk_op(PL_OP_COPY, k, 0, ref(k, PL_BUF_OUT, PL_U8, off), false, {ref(root, PL_BUF_IN, PL_U8, off)},
-                  g.clen(c) * g.es, {}, have[k * g.n_c + c]);
+      em.chunk_op(PL_OP_COPY, k, 0, ref(k, PL_BUF_OUT, PL_U8, off), true, {ref(root, PL_BUF_IN, PL_U8, off)},
+                  g.clen(c) * g.es, {}, -1);
     }
-  em.phase_chunks = g.n_c * (g.R - 1);
-  for (uint64_t c = 0; c < g.n_c; ++c)
-    for (int i = 1; i < g.R; ++i)
-      for (int r = 0; r < g.R; ++r) {
-        const int k = (r + i) % g.R;
-        const uint64_t off = (k * g.P + c * g.chunk) * g.es;
-        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, off), false, {ref(k, PL_BUF_OUT, PL_U8, off)},
-                    g.clen(c) * g.es, {have[k * g.n_c + c]}, -1);
-      }
 }
 
 // reduce = compose<reduce-scatter, gather>: rank k reduces chunk c of partition k (ascending
@@ -758,9 +749,12 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
     footprint = (uint64_t)(rq.R + 1) * msg;
   if (rq.coll == PL_ALLTOALLV) footprint = 2 * (uint64_t)rq.R * msg;
   // Register path while the working set is L2 sized (and for layered latency schedules);
-  // bulk-copy ring once it has to stream from HBM.  Measured crossover on B200: all-reduce of
-  // 16-32 MiB per rank at R=8.
-  const bool stream = footprint >= (256ull << 20) && rq.n_layers == 0;
+  // bulk-copy ring once it has to stream from HBM.  Measured crossovers on B200 at R=8
+  // (128-call CUDA graphs): reduce-scatter, all-gather, all-to-all, scatter, gather, broadcast
+  // between 72 and 144 MiB of inputs + outputs (the L2 holds 126 MB); all-reduce between 128
+  // and 256 MiB (its outputs are written once and never re-read).
+  const uint64_t knee = rq.coll == PL_ALLREDUCE ? (256ull << 20) : (128ull << 20);
+  const bool stream = footprint >= knee && rq.n_layers == 0;
   if (p.datapath == PL_DP_AUTO) p.datapath = stream ? PL_DP_TMA : PL_DP_LDST;
   if (p.threads <= 0) p.threads = 512;
   if (p.stages <= 0) p.stages = 4;
