@@ -6,11 +6,12 @@
 //                     cp.async.bulk loads (one per source), running ahead of the consumers
 //                     across op boundaries (Algorithm 2 of the paper: prime / steady / drain,
 //                     here as a free-running ring with full / empty mbarriers);
-//   warp 1  copier    for COPY stages: one bulk store shared -> global per stage, no
-//                     registers touched by the payload;
-//   warps 2..17 consumers  for REDUCE / COPY_REDUCE stages: read the source tiles from
-//                     shared memory 16 bytes at a time, accumulate in fp32 in ascending
-//                     source order, store the result with 128-bit global stores.
+//   warp 1  copier    for COPY stages: one bulk store shared -> global per stage (R stores
+//                     for a broadcast copy), no registers touched by the payload;
+//   warps 2..  consumers (16, or 12 in the variant for plain reduce schedules)  for REDUCE /
+//                     COPY_REDUCE stages: read the source tiles from shared memory 16 bytes
+//                     at a time, accumulate in fp32 in ascending source order, store the
+//                     result with 128-bit global stores.
 // A stage descriptor travels with every slot.  The last stage of an op carries its signal:
 // the warps that wrote report on an mbarrier, then one thread fences and does the release
 // increment.  Every wait (flag, full, empty, done) is bounded; on expiry the CTA records a
