@@ -236,6 +236,13 @@ void a2av_direct(Emitter& em, int R, int dtype, const uint64_t* counts, uint64_t
   uint64_t max_seg = 0;
   for (int i = 0; i < R * R; ++i) max_seg = std::max(max_seg, counts[i] * es);
   uint64_t chunk = std::max<uint64_t>(16, chunk_bytes);
+  uint64_t busiest = 1;  // chunk ops of the rank that receives the most
+  for (int r = 0; r < R; ++r) {
+    uint64_t c = 0;
+    for (int p = 0; p < R; ++p) c += (counts[p * R + r] * es + chunk - 1) / chunk;
+    busiest = std::max(busiest, c);
+  }
+  em.phase_chunks = busiest;
   for (uint64_t b = 0; b < max_seg; b += chunk)
     for (int i = 0; i < R; ++i)
       for (int r = 0; r < R; ++r) {
@@ -256,6 +263,7 @@ void rsv_direct(Emitter& em, int R, int dtype, const uint64_t* n, uint64_t chunk
   uint64_t max_n = 0;
   std::vector<uint64_t> off(R, 0);
   for (int k = 0; k < R; ++k) { max_n = std::max(max_n, n[k]); if (k) off[k] = off[k - 1] + n[k - 1]; }
+  em.phase_chunks = std::max<uint64_t>(1, (max_n + chunk - 1) / chunk);  // chunk ops of the busiest rank
   for (uint64_t b = 0; b < max_n; b += chunk)
     for (int k = 0; k < R; ++k) {
       if (b >= n[k]) continue;
@@ -267,10 +275,17 @@ void rsv_direct(Emitter& em, int R, int dtype, const uint64_t* n, uint64_t chunk
 
 void agv_direct(Emitter& em, int R, int dtype, const uint64_t* n, uint64_t chunk_bytes, bool push) {
   const int es = elem_size(dtype);
-  const uint64_t chunk = std::max<uint64_t>(16, chunk_bytes);
-  uint64_t max_b = 0;
+  // pulled (bulk-copy path): at most 512 KiB per chunk, as for the fixed-size all-gather
+  const uint64_t chunk = std::max<uint64_t>(16, push ? chunk_bytes : std::min<uint64_t>(chunk_bytes, 512u << 10));
+  uint64_t max_b = 0, all_chunks = 0;
   std::vector<uint64_t> off(R, 0);
-  for (int p = 0; p < R; ++p) { max_b = std::max(max_b, n[p] * es); if (p) off[p] = off[p - 1] + n[p - 1] * es; }
+  for (int p = 0; p < R; ++p) {
+    max_b = std::max(max_b, n[p] * es);
+    all_chunks += (n[p] * es + chunk - 1) / chunk;
+    if (p) off[p] = off[p - 1] + n[p - 1] * es;
+  }
+  // chunk ops per rank: its own contribution when pushed, everybody's when pulled
+  em.phase_chunks = std::max<uint64_t>(1, push ? (max_b + chunk - 1) / chunk : all_chunks);
   if (push) {  // rank p writes its contribution into every output (see ag_direct_push)
     for (uint64_t b = 0; b < max_b; b += chunk)
       for (int p = 0; p < R; ++p) {
