@@ -184,19 +184,44 @@ __device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDe
 // of 8 x 64 MiB: the ring held ~1.5 of its 4 slots for the consumers, which kept the bytes in
 // flight below what saturates HBM).
 struct PlainStage {
-  char* dst;        // destination of the thread's first unit
+  char* dst;        // destination of the stage's unit 0
   uint32_t units;   // units in the stage
   uint32_t ns;      // sources
   bool dpart;       // destination holds partials (twice as wide)
 };
 
+// A thread keeps 8 operand vectors of a stage: 1 unit of up to 8 sources, 2 units of up to 4
+// or 4 units of up to 2, unit j of thread t being unit t + j * (32 * CW) of the stage.  The producer sizes plain stages of
+// the pipelined variant accordingly (plain_unit_cap).
+__device__ __forceinline__ uint32_t plain_units_per_thread(uint32_t ns) { return ns > 4 ? 1u : ns > 2 ? 2u : 4u; }
+template <int CW>
+__device__ __forceinline__ uint32_t plain_unit_cap(uint32_t ns) { return (uint32_t)(32 * CW) * plain_units_per_thread(ns); }
+
 template <int CW>
 __device__ __forceinline__ bool stage_is_plain(const StageDesc& d) {
-  return d.kind != PL_OP_COPY && d.kind != kEnd && d.pmask == 0 && d.n_src <= 8 && !(d.flags & kDstBcast) &&
-         !((d.flags & kLastOfOp) && d.signal != kNoFlag) && d.units <= (uint32_t)(32 * CW);
+  return d.kind != PL_OP_COPY && d.kind != kEnd && d.pmask == 0 && d.n_src >= 1 && d.n_src <= 8 && !(d.flags & kDstBcast) &&
+         !((d.flags & kLastOfOp) && d.signal != kNoFlag) && d.units <= plain_unit_cap<CW>(d.n_src);
 }
 
-// Operands of this thread's unit into q[], descriptor fields into st, slot released.
+// Operands of this thread's units into q[]: NSMAX (8, 4 or 2) bounds the source count, so the
+// register index of every operand is a compile-time constant.
+template <int CW, int NSMAX>
+__device__ __forceinline__ void plain_load_ns(const unsigned char* slot, uint32_t tile, uint32_t units, uint32_t ns, int ctid,
+                                              uint4 (&q)[8]) {
+  constexpr int UPT = 8 / NSMAX;
+#pragma unroll
+  for (int j = 0; j < UPT; ++j) {
+    const uint32_t u = (uint32_t)ctid + (uint32_t)(j * 32 * CW);
+    if (u < units) {
+#pragma unroll
+      for (int k = 0; k < NSMAX; ++k)
+        if ((uint32_t)k < ns) q[j * NSMAX + k] = lds16(slot + (size_t)k * tile + (size_t)u * 16u);
+    }
+  }
+}
+
+// Descriptor fields into st, operands into q[], slot released.
+template <int CW>
 __device__ __forceinline__ void plain_load(const StageDesc& d, const unsigned char* slot, int ctid, uint64_t* empty,
                                            PlainStage& st, uint4 (&q)[8]) {
   st.units = d.units;
@@ -204,44 +229,53 @@ __device__ __forceinline__ void plain_load(const StageDesc& d, const unsigned ch
   st.dpart = d.flags & kDstF32;
   st.dst = d.dst;
   const uint32_t tile = d.ucap * 16u;
-  if ((uint32_t)ctid < st.units) {
-    const unsigned char* p = slot + (size_t)ctid * 16u;
-#pragma unroll
-    for (uint32_t k = 0; k < 8; ++k)
-      if (k < st.ns) q[k] = lds16(p + (size_t)k * tile);
-  }
+  if (st.ns > 4) plain_load_ns<CW, 8>(slot, tile, st.units, st.ns, ctid, q);
+  else if (st.ns > 2) plain_load_ns<CW, 4>(slot, tile, st.units, st.ns, ctid, q);
+  else plain_load_ns<CW, 2>(slot, tile, st.units, st.ns, ctid, q);
   __syncwarp();
   // the arrive is a release: this warp's shared-memory loads above are performed before it
   if ((ctid & 31) == 0) ptx::mbar_arrive(empty);
 }
 
-template <int DT>
-__device__ __forceinline__ void plain_finish(const ExecParams& P, const PlainStage& st, const uint4 (&q)[8], int ctid) {
-  if ((uint32_t)ctid >= st.units) return;
-  Acc<DT> acc;
-  acc.zero();
+template <int DT, int CW, int NSMAX>
+__device__ __forceinline__ void plain_finish_ns(const ExecParams& P, const PlainStage& st, const uint4 (&q)[8], int ctid) {
+  constexpr int UPT = 8 / NSMAX;
 #pragma unroll
-  for (uint32_t k = 0; k < 8; ++k)
-    if (k < st.ns) {
-      if constexpr (DT == PL_BF16) acc.add_bf16(q[k]);
-      else acc.add(q[k]);
+  for (int j = 0; j < UPT; ++j) {
+    const uint32_t u = (uint32_t)ctid + (uint32_t)(j * 32 * CW);
+    if (u >= st.units) continue;
+    Acc<DT> acc;
+    acc.zero();
+#pragma unroll
+    for (int k = 0; k < NSMAX; ++k)
+      if ((uint32_t)k < st.ns) {
+        if constexpr (DT == PL_BF16) acc.add_bf16(q[j * NSMAX + k]);
+        else acc.add(q[j * NSMAX + k]);
+      }
+    if (st.dpart) {
+      if constexpr (DT == PL_BF16) {
+        st16(st.dst + (size_t)u * 32u, make_uint4(__float_as_uint(acc.v[0]), __float_as_uint(acc.v[1]),
+                                                  __float_as_uint(acc.v[2]), __float_as_uint(acc.v[3])));
+        st16(st.dst + (size_t)u * 32u + 16u, make_uint4(__float_as_uint(acc.v[4]), __float_as_uint(acc.v[5]),
+                                                        __float_as_uint(acc.v[6]), __float_as_uint(acc.v[7])));
+      } else if constexpr (DT == PL_F32) {
+        st16(st.dst + (size_t)u * 32u, acc.sums());
+        st16(st.dst + (size_t)u * 32u + 16u, acc.corrections());
+      }
+    } else {
+      uint4 r;
+      if constexpr (DT == PL_BF16) r = acc.to_bf16(P.out_scale);
+      else r = acc.result(P.out_scale);
+      st16(st.dst + (size_t)u * 16u, r);
     }
-  if (st.dpart) {
-    if constexpr (DT == PL_BF16) {
-      st16(st.dst + (size_t)ctid * 32u, make_uint4(__float_as_uint(acc.v[0]), __float_as_uint(acc.v[1]),
-                                                   __float_as_uint(acc.v[2]), __float_as_uint(acc.v[3])));
-      st16(st.dst + (size_t)ctid * 32u + 16u, make_uint4(__float_as_uint(acc.v[4]), __float_as_uint(acc.v[5]),
-                                                         __float_as_uint(acc.v[6]), __float_as_uint(acc.v[7])));
-    } else if constexpr (DT == PL_F32) {
-      st16(st.dst + (size_t)ctid * 32u, acc.sums());
-      st16(st.dst + (size_t)ctid * 32u + 16u, acc.corrections());
-    }
-  } else {
-    uint4 r;
-    if constexpr (DT == PL_BF16) r = acc.to_bf16(P.out_scale);
-    else r = acc.result(P.out_scale);
-    st16(st.dst + (size_t)ctid * 16u, r);
   }
+}
+
+template <int DT, int CW>
+__device__ __forceinline__ void plain_finish(const ExecParams& P, const PlainStage& st, const uint4 (&q)[8], int ctid) {
+  if (st.ns > 4) plain_finish_ns<DT, CW, 8>(P, st, q, ctid);
+  else if (st.ns > 2) plain_finish_ns<DT, CW, 4>(P, st, q, ctid);
+  else plain_finish_ns<DT, CW, 2>(P, st, q, ctid);
 }
 
 // A REDUCE stage whose result leaves through shared memory (see consume_stage).
@@ -334,7 +368,12 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
       const char* my_src = (lane < (int)n_src) ? resolve(P, r_src) : nullptr;
       const bool my_part = (pmask >> lane) & 1u;
       const uint32_t unit_b = (kind == PL_OP_COPY) ? 16u : 16u * (n_src + __popc(pmask));  // slot bytes per unit
-      const uint32_t ucap = slot_bytes / unit_b;
+      uint32_t ucap = slot_bytes / unit_b;
+      if constexpr (CW == kWarpsPipelined) {
+        // plain reduce op: a stage holds what the consumer threads can keep in registers
+        if (kind != PL_OP_COPY && pmask == 0 && n_src >= 1 && n_src <= 8 && !(oflags & kDstBcast))
+          ucap = min(ucap, plain_unit_cap<CW>(n_src));
+      }
       const uint64_t n_units = (kind == PL_OP_COPY) ? (count >> 4) : count / Acc<DT == PL_U8 ? PL_I32 : DT>::kElems;
       // tile offset of my source inside a slot, and my bytes per unit
       const uint32_t my_w = my_part ? 32u : 16u;
@@ -475,14 +514,14 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
           if (next) {
             PlainStage st_b;
             uint4 q_b[8];
-            plain_load(c->desc[s], slots + (size_t)s * slot_bytes, ctid, &c->empty[s], st_b, q_b);
-            plain_finish<DT>(P, st_a, q_a, ctid);
+            plain_load<CW>(c->desc[s], slots + (size_t)s * slot_bytes, ctid, &c->empty[s], st_b, q_b);
+            plain_finish<DT, CW>(P, st_a, q_a, ctid);
             st_a = st_b;
 #pragma unroll
             for (int k = 0; k < 8; ++k) q_a[k] = q_b[k];
             continue;
           }
-          plain_finish<DT>(P, st_a, q_a, ctid);
+          plain_finish<DT, CW>(P, st_a, q_a, ctid);
           have = false;  // stage n is handled below
         }
       }
@@ -496,7 +535,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
       if (kind == kEnd) break;
       if constexpr (DT != PL_U8 && CW == kWarpsPipelined) {
         if (stage_is_plain<CW>(d)) {
-          plain_load(d, slots + (size_t)s * slot_bytes, ctid, &c->empty[s], st_a, q_a);
+          plain_load<CW>(d, slots + (size_t)s * slot_bytes, ctid, &c->empty[s], st_a, q_a);
           have = true;
           continue;
         }
