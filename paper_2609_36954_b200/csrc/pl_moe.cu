@@ -275,7 +275,8 @@ __global__ void __launch_bounds__(32) moe_move_kernel(const __grid_constant__ Di
 
 // combine: CTA per token (grid-strided), 16-byte column units across threads, the K source
 // rows and gates of the next token are fetched while the current one is summed.
-__global__ void __launch_bounds__(256) moe_combine_kernel(const __grid_constant__ CombinePtrs P, const __grid_constant__ MoeGeo g) {
+constexpr int kCombineThreads = 256;
+__global__ void __launch_bounds__(kCombineThreads) moe_combine_kernel(const __grid_constant__ CombinePtrs P, const __grid_constant__ MoeGeo g) {
   __shared__ const char* s_row[2][kMaxTopk];
   __shared__ float s_gate[2][kMaxTopk];
   const int tid = threadIdx.x;
@@ -310,7 +311,7 @@ __global__ void __launch_bounds__(256) moe_combine_kernel(const __grid_constant_
     if (tok + gridDim.x < n_tok) load_meta(tok + gridDim.x, buf ^ 1);
     const int p = (int)(tok / g.T);
     char* out = static_cast<char*>(P.out[p]) + (tok % g.T) * g.row_bytes;
-    for (uint32_t u = tid; u < units; u += 256) {
+    for (uint32_t u = tid; u < units; u += kCombineThreads) {
       float acc[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[i] = 0.f;
@@ -359,6 +360,7 @@ struct pl_moe_plan_s {
   char* d_blob = nullptr;
   size_t blob_bytes = 0;
   int sm_count = 148;
+  int combine_per_sm = 4;  // resident CTAs of the combine kernel per SM (occupancy query at plan creation)
   size_t move_smem = 0;
   bool dispatched = false;
   // deduplicated variant: the same machinery run over "one expert per rank" routing
@@ -389,6 +391,17 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   if (!pl) return PL_ERR_OOM;
   pl->comm = comm;
   pl->sm_count = comm->sm_count;
+  {
+    // The combine kernel deals tokens to CTAs by a fixed stride, so its grid must be exactly one
+    // resident wave: with 1.5 waves (6 CTAs per SM against 4 resident) the second half wave ran
+    // alone and the launch took 703 us instead of 612 us (C4 shape).
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, moe_combine_kernel, kCombineThreads, 0) != cudaSuccess || occ < 1) {
+      cudaGetLastError();
+      occ = 1;
+    }
+    pl->combine_per_sm = occ;
+  }
   MoeGeo& g = pl->g;
   g.R = R;
   g.T = tokens_per_rank;
@@ -526,8 +539,8 @@ pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float
     P.out[r] = out[r];
   }
   const unsigned long long n_tok = (unsigned long long)g.R * g.T;
-  const int grid = (int)std::min<unsigned long long>(n_tok, (unsigned long long)plan->sm_count * 6);
-  moe_combine_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(P, g);
+  const int grid = (int)std::min<unsigned long long>(n_tok, (unsigned long long)plan->sm_count * plan->combine_per_sm);
+  moe_combine_kernel<<<grid, kCombineThreads, 0, static_cast<cudaStream_t>(stream)>>>(P, g);
   if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
   g_launches.fetch_add(1);
   return PL_OK;
@@ -611,8 +624,8 @@ pl_status_t pl_moe_combine_dedup(pl_moe_plan_t plan, const void* const* z, void*
     P.out[r] = out[r];
   }
   const unsigned long long n_tok = (unsigned long long)d.R * d.T;
-  const int grid = (int)std::min<unsigned long long>(n_tok, (unsigned long long)plan->sm_count * 6);
-  moe_combine_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(P, d);
+  const int grid = (int)std::min<unsigned long long>(n_tok, (unsigned long long)plan->sm_count * plan->combine_per_sm);
+  moe_combine_kernel<<<grid, kCombineThreads, 0, static_cast<cudaStream_t>(stream)>>>(P, d);
   if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
   g_launches.fetch_add(1);
   return PL_OK;
