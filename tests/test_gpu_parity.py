@@ -6,7 +6,7 @@ from oracle import oracle
 from paper_2609_36954_b200 import binding as B
 from paper_2609_36954_b200 import inputs as gen
 
-from gpu_harness import Session, check_float, to_dev
+from gpu_harness import DT, Session, check_float, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -699,3 +699,33 @@ def test_stream_probe_copies_and_zero_fills():
         B.pl_probe_hbm(2, src.data_ptr(), dst.data_ptr(), n - 16, 0, h)
     with pytest.raises(B.PurlinError):
         B.pl_probe_hbm(2, 0, dst.data_ptr(), n, 0, h)
+
+
+@pytest.mark.parametrize("R", [2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("dtype", ["bf16", "f32", "i32"])
+def test_pipelined_reduce_variant_for_every_source_count(R, dtype):
+    """The bulk-copy executor's software-pipelined consumers keep 1, 2 or 4 units per thread
+    depending on the source count.  Reduce-scatter and the two-shot all-reduce over ops that
+    span several ring stages (and a ragged tail) must match the oracle and, bit for bit, the
+    register path, for every R up to 8."""
+    import torch
+    from gpu_harness import stream_handle
+    es = B.DTYPE_SIZE[DT[dtype]]
+    per_part = (200 * 1024 + 48) // es          # ~4 stages of 48 KiB per op at R = 8, ragged
+    n = R * per_part
+    x = gen.rank_inputs(R, n, dtype, seed=90 + R)
+    ses = Session(R, dtype)
+    try:
+        for coll in (B.PL_REDUCE_SCATTER, B.PL_ALLREDUCE):
+            ref = oracle.reduce_scatter(x, dtype) if coll == B.PL_REDUCE_SCATTER else oracle.allreduce(x, dtype)
+            outs = {}
+            for dp in (B.PL_DP_TMA, B.PL_DP_LDST):
+                s = ses.build(coll, B.PL_ALGO_DIRECT, n, 1 << 20, datapath=dp)
+                if dp == B.PL_DP_TMA:
+                    assert B.pl_schedule_info(s).threads == 448   # the 12-warp variant was chosen
+                outs[dp], _ = ses.execute(s, x, repeats=3)
+                compare_reduce(outs[dp], ref, dtype)
+            for r in range(R):
+                assert np.array_equal(outs[B.PL_DP_TMA][r], outs[B.PL_DP_LDST][r])
+    finally:
+        ses.close()
