@@ -9,6 +9,7 @@ for reduce-scatter, gathered output for all-gather; algorithm bandwidth = size /
 
   python bench.py [--gpus N] [--steps K] [--warmup W]            # the CUDA path
   python bench.py --impl reference [--steps K] [--warmup W]      # the CPU oracle, timed
+  python bench.py --cpu-suite                                    # the CPU oracle on samples of every configuration
   python bench.py --suite                                          # every configuration, one line each
 
 With N > 1 (torchrun) every rank runs an independent replica on its own GPU: the path has
@@ -388,6 +389,61 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ---------------------------------------------------------------------------------------------
+# the oracle timed per configuration (reported baseline: wall time per collective on the host)
+# ---------------------------------------------------------------------------------------------
+def run_cpu_suite(args):
+    """One JSON line per (configuration, thread count): the CPU oracle as it stands, on bounded
+    samples of every benchmark configuration, with 1 thread and with every available core.
+    No GPU is touched."""
+    import ctypes
+    from oracle import oracle
+    from paper_2609_36954_b200 import inputs as gen
+    omp = ctypes.CDLL("libgomp.so.1")
+    all_threads = oracle.num_threads()
+
+    def timed(fn, budget_s=2.0):
+        fn()
+        t0 = time.perf_counter()
+        reps = 0
+        while True:
+            fn()
+            reps += 1
+            dt = time.perf_counter() - t0
+            if reps >= 3 and dt >= budget_s or reps >= 50:
+                return dt / reps
+
+    def emit(cfg, what, threads, sec, eff_bytes):
+        print(json.dumps({"cfg": cfg, "impl": "cpu-oracle", "what": what, "threads": threads, "us": sec * 1e6,
+                          "eff_gbs": eff_bytes / sec / 1e9}), flush=True)
+
+    cases = []
+    x1 = gen.rank_inputs(4, 262144, "f32", seed=0)
+    cases.append(("C1", "all-reduce R=4 1 MiB fp32", lambda: oracle.allreduce(x1, "f32"), 1 << 20))
+    n2 = 4 * MIB  # 8 MiB per rank sample of the 64 MiB C2 message
+    x2 = [gen.normal_bf16(n2, 0, r) for r in range(8)]
+    cases.append(("C2", "reduce-scatter R=8, 8 MiB/rank sample", lambda: oracle.reduce_scatter(x2, "bf16"), n2 * 2))
+    part = [a[: n2 // 8].copy() for a in x2]
+    cases.append(("C2", "all-gather R=8, 8 MiB/rank sample", lambda: oracle.allgather(part), n2 * 2))
+    for kib in (4, 64, 1024, 16384):
+        n = kib * 1024 // 2
+        x = [gen.normal_bf16(n, 0, r) for r in range(8)]
+        cases.append(("C3", f"all-reduce R=8 {kib} KiB bf16", (lambda x=x: oracle.allreduce(x, "bf16")), n * 2))
+    R, T, H, E, K = 8, 256, 7168, 256, 8  # 256 of the 4096 tokens per rank
+    idx, gates = gen.moe_routing(R, T, E, K, seed=0)
+    xt = gen.moe_tokens_bf16(R, T, H, seed=2)
+    disp = oracle.moe_dispatch(xt, idx, E, recv_capacity_rows=R * T * K)
+    cases.append(("C4", "MoE dispatch, 256 tokens/rank sample", lambda: oracle.moe_dispatch(xt, idx, E, recv_capacity_rows=R * T * K), R * T * K * H * 2))
+    cases.append(("C4", "MoE combine, 256 tokens/rank sample", lambda: oracle.moe_combine(disp["recv"], idx, disp["pos"], gates, E, H), R * T * K * H * 2))
+    x5 = [gen.normal_bf16(8192, 0, r) for r in range(8)]
+    cases.append(("C5", "all-reduce R=8 16 KiB (one decode layer)", lambda: oracle.allreduce(x5, "bf16"), 16384))
+    for threads in sorted({1, all_threads}):
+        omp.omp_set_num_threads(threads)
+        for cfg, what, fn, eff in cases:
+            emit(cfg, what, threads, timed(fn, budget_s=args.cpu_seconds / 12.0), eff)
+    omp.omp_set_num_threads(all_threads)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -395,6 +451,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="purlin", choices=["purlin", "reference"])
     ap.add_argument("--suite", action="store_true", help="run every configuration (paper_2609_36954_b200/bench_suite.py)")
+    ap.add_argument("--cpu-suite", action="store_true", help="time the CPU oracle on samples of every configuration (1 thread and all cores)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-latency", action="store_true")
@@ -411,6 +468,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.cpu_suite:
+        run_cpu_suite(args)
     elif args.suite:
         from paper_2609_36954_b200 import bench_suite
         bench_suite.main(args)
