@@ -140,7 +140,9 @@ typedef struct pl_moe_plan_s* pl_moe_plan_t;
 typedef struct {
   uint32_t struct_size;
   int32_t n_ctas;        /* persistent CTAs = op queues; rounded down to a multiple of R  */
-  int32_t threads;       /* threads per CTA (multiple of 32, <= 1024)                     */
+  int32_t threads;       /* threads per CTA of the register datapath (multiple of 32, <=  */
+                         /* 512); the bulk-copy datapath fixes its own (576, or 448 for   */
+                         /* schedules of plain reduce ops: see pl_sched_info_t.threads)   */
   int32_t datapath;      /* pl_datapath_t                                                 */
   int32_t stages;        /* shared-memory ring depth S of the TMA pipeline                */
   uint32_t stage_bytes;  /* bytes per ring slot B_stage (multiple of 16)                  */
