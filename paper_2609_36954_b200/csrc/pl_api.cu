@@ -39,6 +39,7 @@ struct pl_schedule_s {
   bool no_l2_hints = false;
   bool trace = false;
   bool overlap_launch = false;
+  bool bcast_copies = false;      // some COPY op writes every rank's output
   bool pipelined_reduce = false;  // bulk-copy datapath: every reduce op is plain, run the 12-warp variant
   size_t off_trace = 0;
   float out_scale = 1.0f;
@@ -278,6 +279,8 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
     S->pipelined_reduce = any && plain;
     S->pol.threads = exec_tma_threads(S->pipelined_reduce);
   }
+  for (const HostOp& op : S->L.ops)
+    if (op.kind == PL_OP_COPY && op.bcast) S->bcast_copies = true;
   fill_info(S, comm->R);
   flatten(S, comm->dtype);
   if (!comm->planner) {
@@ -586,6 +589,7 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   P.out_scale = s->out_scale;
   P.overlap_launch = s->overlap_launch ? 1u : 0u;
   P.pipelined_reduce = s->pipelined_reduce ? 1u : 0u;
+  P.bcast_copies = s->bcast_copies ? 1u : 0u;
   cudaError_t le = s->pol.datapath == PL_DP_TMA
                        ? launch_exec_tma(s->comm->dtype, P, s->pol.n_ctas, static_cast<cudaStream_t>(stream))
                        : launch_exec(s->comm->dtype, P, s->pol.n_ctas, s->pol.threads, static_cast<cudaStream_t>(stream));

@@ -225,7 +225,11 @@ struct OpSlot {
   DevWait wait[PL_MAX_WAITS];
 };
 
-template <int DT>
+// BC: the variant that also runs broadcast copies (pushed all-gather, broadcast).  It is a
+// kernel of its own because the mere presence of that body in the function changed the code
+// generated for the reduce loops (one-shot all-reduce of 8 MiB per rank: 71 -> 88 us);
+// schedules with broadcast copies hold no reduce ops, schedules with reduce ops run BC = false.
+template <int DT, bool BC>
 __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_constant__ ExecParams P) {
   __shared__ OpSlot s_slot[2];
   __shared__ int s_abort[2];  // indexed by iteration parity: written during wait i, read after barrier i
@@ -299,8 +303,12 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
     const DevOp& op = S.op;
     if (P.trace && tid == 0) P.trace[2ull * op.topo] = globaltimer_ns();  // waits satisfied
     if (op.kind == PL_OP_COPY) {
-      if (op.flags & kDstBcast) body_copy_bcast(P, op.dst & 0xFFFFFFFFFFFFull, S.src[0], op.count, tid, nthr);
-      else body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
+      if constexpr (BC) {
+        if (op.flags & kDstBcast) body_copy_bcast(P, op.dst & 0xFFFFFFFFFFFFull, S.src[0], op.count, tid, nthr);
+        else body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
+      } else {
+        body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
+      }
     } else if (op.kind == PL_OP_REDUCE) {
       if constexpr (DT != PL_U8) body_reduce<DT>(P, op, S.src, tid, nthr);
     } else {
@@ -334,7 +342,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   }
 }
 
-template <int DT>
+template <int DT, bool BC>
 cudaError_t launch_t(const ExecParams& P, int grid, int threads, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
@@ -345,17 +353,25 @@ cudaError_t launch_t(const ExecParams& P, int grid, int threads, cudaStream_t st
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = P.overlap_launch ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, pl_exec_kernel<DT>, P);
+  return cudaLaunchKernelEx(&cfg, pl_exec_kernel<DT, BC>, P);
 }
 
 }  // namespace
 
 cudaError_t launch_exec(int dtype, const ExecParams& P, int grid, int threads, cudaStream_t stream) {
+  if (P.bcast_copies) {
+    switch (dtype) {
+      case PL_BF16: return launch_t<PL_BF16, true>(P, grid, threads, stream);
+      case PL_F32: return launch_t<PL_F32, true>(P, grid, threads, stream);
+      case PL_I32: return launch_t<PL_I32, true>(P, grid, threads, stream);
+      default: return launch_t<PL_U8, true>(P, grid, threads, stream);
+    }
+  }
   switch (dtype) {
-    case PL_BF16: return launch_t<PL_BF16>(P, grid, threads, stream);
-    case PL_F32: return launch_t<PL_F32>(P, grid, threads, stream);
-    case PL_I32: return launch_t<PL_I32>(P, grid, threads, stream);
-    default: return launch_t<PL_U8>(P, grid, threads, stream);
+    case PL_BF16: return launch_t<PL_BF16, false>(P, grid, threads, stream);
+    case PL_F32: return launch_t<PL_F32, false>(P, grid, threads, stream);
+    case PL_I32: return launch_t<PL_I32, false>(P, grid, threads, stream);
+    default: return launch_t<PL_U8, false>(P, grid, threads, stream);
   }
 }
 
@@ -363,10 +379,10 @@ int exec_max_ctas_per_sm(int dtype, int threads) {
   int n = 0;
   cudaError_t e;
   switch (dtype) {
-    case PL_BF16: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_BF16>, threads, 0); break;
-    case PL_F32: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_F32>, threads, 0); break;
-    case PL_I32: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_I32>, threads, 0); break;
-    default: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_U8>, threads, 0); break;
+    case PL_BF16: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_BF16, true>, threads, 0); break;
+    case PL_F32: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_F32, true>, threads, 0); break;
+    case PL_I32: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_I32, true>, threads, 0); break;
+    default: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_U8, true>, threads, 0); break;
   }
   if (e != cudaSuccess) { cudaGetLastError(); return 0; }
   return n;
