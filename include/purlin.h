@@ -121,7 +121,12 @@ typedef enum {
   PL_ALGO_TREE = 1,
   PL_ALGO_DIRECT = 2,
   PL_ALGO_ONESHOT = 3,
-  PL_ALGO_DIRECT_FUSED = 4
+  PL_ALGO_DIRECT_FUSED = 4,
+  /* The library's pick for the collective and size, from the measurements on B200 (R = 8):
+   * all-reduce: one-shot up to 32 KiB per rank, direct-fused above (the fastest of the five at
+   * every size from 4 KiB to 256 MiB); everything else: direct.  pl_schedule_info does not
+   * report the pick; pl_schedule_dump shows the ops. */
+  PL_ALGO_AUTO = 5
 } pl_algo_t;
 
 typedef enum { PL_OP_COPY = 0, PL_OP_REDUCE = 1, PL_OP_COPY_REDUCE = 2 } pl_op_kind_t;

@@ -28,7 +28,7 @@ DTYPE_SIZE = {PL_BF16: 2, PL_F32: 4, PL_I32: 4, PL_U8: 1, PL_F32X2: 8}
 PL_ALLREDUCE, PL_REDUCE_SCATTER, PL_ALLGATHER, PL_ALLTOALL, PL_ALLTOALLV, PL_ALLGATHERV, PL_REDUCE_SCATTERV, \
     PL_BROADCAST, PL_REDUCE, PL_SCATTER, PL_GATHER = range(11)
 # algorithms
-PL_ALGO_RING, PL_ALGO_TREE, PL_ALGO_DIRECT, PL_ALGO_ONESHOT, PL_ALGO_DIRECT_FUSED = range(5)
+PL_ALGO_RING, PL_ALGO_TREE, PL_ALGO_DIRECT, PL_ALGO_ONESHOT, PL_ALGO_DIRECT_FUSED, PL_ALGO_AUTO = range(6)
 # op kinds / buffer kinds / datapaths
 PL_OP_COPY, PL_OP_REDUCE, PL_OP_COPY_REDUCE = range(3)
 PL_BUF_IN, PL_BUF_OUT, PL_BUF_SCRATCH = range(3)

@@ -390,6 +390,10 @@ pl_status_t pl_schedule_build(pl_comm_t comm, pl_collective_t coll, pl_algo_t al
   BuildRequest rq{};
   rq.coll = coll;
   rq.algo = algo;
+  if (algo == PL_ALGO_AUTO && comm) {
+    const size_t bytes = count_per_rank * (size_t)elem_size(comm->dtype);
+    rq.algo = coll != PL_ALLREDUCE ? PL_ALGO_DIRECT : bytes <= (32u << 10) ? PL_ALGO_ONESHOT : PL_ALGO_DIRECT_FUSED;
+  }
   rq.count_per_rank = count_per_rank;
   rq.chunk_bytes = chunk_bytes;
   return build_common(comm, rq, opts, out);
@@ -403,7 +407,7 @@ pl_status_t pl_schedule_build_v(pl_comm_t comm, pl_collective_t coll, pl_algo_t 
   for (size_t i = 0; i < c.size(); ++i) c[i] = counts[i];
   BuildRequest rq{};
   rq.coll = coll;
-  rq.algo = algo;
+  rq.algo = algo == PL_ALGO_AUTO ? PL_ALGO_DIRECT : algo;
   rq.chunk_bytes = chunk_bytes;
   rq.counts_v = c.data();
   return build_common(comm, rq, opts, out);
@@ -428,7 +432,7 @@ pl_status_t pl_schedule_build_layers(pl_comm_t comm, pl_algo_t algo, size_t coun
   if (n_layers < 1) return PL_ERR_INVALID_ARG;
   BuildRequest rq{};
   rq.coll = PL_ALLREDUCE;
-  rq.algo = algo;
+  rq.algo = algo == PL_ALGO_AUTO ? PL_ALGO_DIRECT_FUSED : algo;  // the fastest layered form at 16 KiB - 1 MiB
   rq.count_per_rank = count_per_rank;
   rq.n_layers = n_layers;
   // a layer is one chunk per partition: the latency path does not pipeline inside a layer

@@ -549,3 +549,28 @@ def test_latency_regime_grid_follows_the_schedule_width():
             seen.add(key)
     finally:
         pl.close()
+
+
+def test_algo_auto_picks_by_collective_and_size():
+    """PL_ALGO_AUTO: one-shot for all-reduces up to 32 KiB per rank, direct-fused above, direct for
+    everything else; the schedules are the same as the explicitly named ones."""
+    R = 8
+    pl = Planner(R, "bf16")
+    try:
+        def same(coll, count, named):
+            a = B.pl_schedule_dump(pl.build(coll, B.PL_ALGO_AUTO, count, 1 << 20))
+            b = B.pl_schedule_dump(pl.build(coll, named, count, 1 << 20))
+            key = lambda o: (o.kind, o.exec_rank, o.queue, int(o.count), int(o.dst.offset), o.n_src, o.dst_bcast)
+            assert [key(o) for o in a] == [key(o) for o in b]
+        same(B.PL_ALLREDUCE, 8192, B.PL_ALGO_ONESHOT)           # 16 KiB
+        same(B.PL_ALLREDUCE, 16384, B.PL_ALGO_ONESHOT)          # 32 KiB
+        same(B.PL_ALLREDUCE, 32768, B.PL_ALGO_DIRECT_FUSED)     # 64 KiB
+        same(B.PL_ALLREDUCE, 1 << 24, B.PL_ALGO_DIRECT_FUSED)
+        same(B.PL_REDUCE_SCATTER, 1 << 20, B.PL_ALGO_DIRECT)
+        same(B.PL_ALLGATHER, 1 << 17, B.PL_ALGO_DIRECT)
+        same(B.PL_ALLTOALL, 1 << 20, B.PL_ALGO_DIRECT)
+        s = B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_AUTO, 8192, 4, None)
+        pl.scheds.append(s)
+        assert all(o.dst_bcast for o in B.pl_schedule_dump(s))  # direct-fused layers
+    finally:
+        pl.close()
