@@ -412,7 +412,8 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   g.row_bytes = (uint32_t)row_bytes;
   g.n_tiles = (uint32_t)((row_bytes + kMaxTile - 1) / kMaxTile);
   g.tile_bytes = (uint32_t)align_up((row_bytes + g.n_tiles - 1) / g.n_tiles, 16);
-  g.slots = (uint32_t)std::min<size_t>(8, std::max<size_t>(2, (96 * 1024) / g.tile_bytes));
+  // at least 4: the move kernel keeps 2 store groups reading their tiles while it refills others
+  g.slots = (uint32_t)std::min<size_t>(8, std::max<size_t>(4, (96 * 1024) / g.tile_bytes));
   g.cap = recv_capacity_rows;
   pl->move_smem = 128 + (size_t)g.slots * g.tile_bytes;
   size_t off = 0;
