@@ -72,3 +72,85 @@ def test_random_case_matches_the_oracle(seed):
                 check_float(outs[r].view(np.float32).astype(np.float64), ref[r], dtype)
     finally:
         s.close()
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_v_and_rooted_case_matches_the_oracle(seed):
+    """Seeded draws for the variable-size collectives (ragged per-rank sizes with empty ranks)
+    and the rooted ones (any root), over rank count, element type, chunk size and datapath."""
+    rng = np.random.default_rng(7000 + seed)
+    R = int(rng.choice([2, 3, 5, 8, 11, 16]))
+    dtype = str(rng.choice(["i32", "bf16", "f32"]))
+    es = B.DTYPE_SIZE[DT[dtype]]
+    dp = int(rng.choice([B.PL_DP_AUTO, B.PL_DP_LDST, B.PL_DP_TMA]))
+    chunk = 16 * int(rng.choice([1, 7, 256, 4096, 1 << 16]))
+    kind = str(rng.choice(["agv", "rsv", "a2av", "broadcast", "reduce", "scatter", "gather"]))
+    vec = 16 // es
+    s = Session(R, dtype)
+    try:
+        if kind in ("agv", "rsv"):
+            sizes = [int(v) * vec for v in rng.choice([0, 1, 3, 64, 1000, 5000], size=R)]
+            if sum(sizes) == 0:
+                sizes[0] = vec
+            total = sum(sizes)
+            x = gen.rank_inputs(R, total, dtype, seed=seed)
+            if kind == "rsv":
+                outs, _ = s.execute(s.build_v(sizes, chunk, coll=B.PL_REDUCE_SCATTERV, datapath=dp), x, repeats=2)
+                ref = oracle.reduce_scatterv(x, sizes, dtype)
+                for r in range(R):
+                    assert outs[r].size == sizes[r] * es
+                    if not sizes[r]:
+                        continue
+                    if dtype == "i32":
+                        assert np.array_equal(outs[r].view(np.int32), ref[r])
+                    elif dtype == "bf16":
+                        check_float(gen.bf16_bits_to_f64(outs[r].view(np.uint16)), ref[r], dtype)
+                    else:
+                        check_float(outs[r].view(np.float32).astype(np.float64), ref[r], dtype)
+            else:
+                contrib = [x[p][: sizes[p]].copy() for p in range(R)]
+                outs, _ = s.execute(s.build_v(sizes, chunk, coll=B.PL_ALLGATHERV, datapath=dp), contrib, repeats=2)
+                ref = oracle.allgatherv(contrib)
+                for r in range(R):
+                    assert np.array_equal(outs[r], ref[r].view(np.uint8))
+        elif kind == "a2av":
+            counts = (rng.choice([0, 1, 2, 40, 700], size=(R, R)) * vec).astype(np.int64)
+            x = [gen.rank_inputs(1, max(int(counts[p].sum()), vec), dtype, seed=seed * 31 + p)[0] for p in range(R)]
+            outs, _ = s.execute(s.build_v(counts.reshape(-1).tolist(), chunk, datapath=dp), x, repeats=2)
+            ref = oracle.alltoallv([a[: int(counts[p].sum())] for p, a in enumerate(x)], counts)
+            for r in range(R):
+                assert np.array_equal(outs[r][: ref[r].size * es], ref[r].view(np.uint8))
+        else:
+            root = int(rng.integers(0, R))
+            m = int(rng.choice([1, 5, 300, 4099])) * vec
+            n = R * m
+            x = gen.rank_inputs(R, n, dtype, seed=seed)
+            empty = np.zeros(0, x[0].dtype)
+            coll = {"broadcast": B.PL_BROADCAST, "reduce": B.PL_REDUCE, "scatter": B.PL_SCATTER, "gather": B.PL_GATHER}[kind]
+            count = n if kind in ("broadcast", "reduce") else m
+            sched = B.pl_schedule_build_rooted(s.comm, coll, root, count, chunk, B.make_opts(datapath=dp))
+            s.scheds.append(sched)
+            if kind == "broadcast":
+                outs, _ = s.execute(sched, [x[r] if r == root else empty for r in range(R)], repeats=2)
+                for r in range(R):
+                    assert np.array_equal(outs[r], x[root].view(np.uint8))
+            elif kind == "reduce":
+                outs, _ = s.execute(sched, x, repeats=2)
+                ref = oracle.reduce(x, root, dtype)[root]
+                if dtype == "i32":
+                    assert np.array_equal(outs[root].view(np.int32), ref)
+                elif dtype == "bf16":
+                    check_float(gen.bf16_bits_to_f64(outs[root].view(np.uint16)), ref, dtype)
+                else:
+                    check_float(outs[root].view(np.float32).astype(np.float64), ref, dtype)
+            elif kind == "scatter":
+                outs, _ = s.execute(sched, [x[r] if r == root else empty for r in range(R)], repeats=2)
+                ref = oracle.scatter(x, root)
+                for r in range(R):
+                    assert np.array_equal(outs[r], ref[r].view(np.uint8))
+            else:
+                contrib = [a[:m].copy() for a in x]
+                outs, _ = s.execute(sched, contrib, repeats=2)
+                assert np.array_equal(outs[root], oracle.gather(contrib, root)[root].view(np.uint8))
+    finally:
+        s.close()
