@@ -2,9 +2,10 @@
 // only known on the device (Table 2 of the paper names the pattern; Sec. 4 uses prefix sums
 // for the variable-length offsets).
 //
-// dispatch = count (per 256-token block, per expert, via bit masks) -> scan (exclusive
-// prefix sums: receive offsets in (source rank, expert, token) order) -> place (row index
-// of every (token, slot) + receive metadata) -> move (each token row is read once into
+// dispatch = count (per 256-token block, per expert, via bit masks) -> scan (one CTA per
+// source rank: exclusive prefix sums over its blocks, totals per expert and destination) ->
+// place (segment bases in (source rank, expert, token) order, row index of every
+// (token, slot), receive metadata) -> move (each token row is read once into
 // shared memory by a bulk async copy and written to its K destinations by K bulk stores).
 // combine = gate-weighted fp32 sum of the K expert rows of every token, ascending slot.
 #include <cuda_bf16.h>
@@ -43,7 +44,6 @@ struct MoeGeo {
   uint32_t row_bytes, tile_bytes, n_tiles, slots;
   unsigned long long cap;
   int32_t* blockcnt;   // [R][NB][E]: per-block counts, turned into exclusive block offsets by scan
-  int32_t* base;       // [R][E]: first row of segment (p, e) in the destination's receive buffer
   long long* counts;   // [R][R]
   long long* ecounts;  // [R][E]
   int32_t* pos;        // [R][T][K] row in the destination's receive buffer, -1 if dropped
@@ -78,11 +78,13 @@ __global__ void __launch_bounds__(kTB) moe_count_kernel(const __grid_constant__ 
   }
 }
 
-__global__ void __launch_bounds__(1024) moe_scan_kernel(const __grid_constant__ MoeGeo g) {
-  const int tid = threadIdx.x, n = blockDim.x;
-  if (tid < 3) g.flags[tid] = 0;
-  for (int pe = tid; pe < g.R * g.E; pe += n) {
-    const int p = pe / g.E, e = pe % g.E;
+// One CTA per source rank p: exclusive scan of the per-block counts of every expert, the totals
+// per expert (ecounts) and per destination rank (counts).  Segment bases, which need the counts
+// of all source ranks, are computed by the place kernel.
+__global__ void __launch_bounds__(256) moe_scan_kernel(const __grid_constant__ MoeGeo g) {
+  const int tid = threadIdx.x, n = blockDim.x, p = blockIdx.x;
+  if (p == 0 && tid < 3) g.flags[tid] = 0;
+  for (int e = tid; e < g.E; e += n) {
     int run = 0;
     // exclusive scan over the token blocks, eight independent loads at a time
     for (int b0 = 0; b0 < g.NB; b0 += 8) {
@@ -97,35 +99,36 @@ __global__ void __launch_bounds__(1024) moe_scan_kernel(const __grid_constant__ 
           run += v[i];
         }
     }
-    g.ecounts[pe] = run;
+    g.ecounts[p * g.E + e] = run;
   }
-  __syncthreads();
-  for (int pr = tid; pr < g.R * g.R; pr += n) {
-    const int p = pr / g.R, r = pr % g.R;
+  __syncthreads();  // this CTA's ecounts are visible to its own threads
+  for (int r = tid; r < g.R; r += n) {
     long long s = 0;
     for (int e = r * g.epr; e < (r + 1) * g.epr; ++e) s += g.ecounts[p * g.E + e];
-    g.counts[pr] = s;
-  }
-  __syncthreads();
-  for (int pe = tid; pe < g.R * g.E; pe += n) {
-    const int p = pe / g.E, e = pe % g.E, r = e / g.epr;
-    long long off = 0;
-    for (int q = 0; q < p; ++q) off += g.counts[q * g.R + r];
-    for (int e2 = r * g.epr; e2 < e; ++e2) off += g.ecounts[p * g.E + e2];
-    g.base[pe] = (int32_t)off;
-  }
-  for (int r = tid; r < g.R; r += n) {
-    long long total = 0;
-    for (int p = 0; p < g.R; ++p) total += g.counts[p * g.R + r];
-    if ((unsigned long long)total > g.cap) g.flags[0] = 1;
+    g.counts[p * g.R + r] = s;
   }
 }
 
 __global__ void __launch_bounds__(kTB) moe_place_kernel(const __grid_constant__ DispatchPtrs P, const __grid_constant__ MoeGeo g) {
   extern __shared__ uint32_t mask[];
+  int32_t* s_base = reinterpret_cast<int32_t*>(mask + (size_t)g.E * kMaskWords);  // [E] row of this source's segments
   const int b = blockIdx.x, p = blockIdx.y, tid = threadIdx.x, t = b * kTB + tid;
   const int32_t* idx = P.idx[p];
-  build_mask(g, idx, mask, t, tid);
+  // first row of expert e's run inside the receive buffer of its rank: everything sources
+  // q < p send to that rank, then this source's rows for the rank's earlier experts
+  for (int e = tid; e < g.E; e += kTB) {
+    const int r = e / g.epr;
+    long long off = 0;
+    for (int q = 0; q < p; ++q) off += g.counts[q * g.R + r];
+    for (int e2 = r * g.epr; e2 < e; ++e2) off += g.ecounts[p * g.E + e2];
+    s_base[e] = (int32_t)off;
+  }
+  if (b == 0 && p == 0 && tid < g.R) {  // capacity check, once
+    long long total = 0;
+    for (int q = 0; q < g.R; ++q) total += g.counts[q * g.R + tid];
+    if ((unsigned long long)total > g.cap) g.flags[0] = 1;
+  }
+  build_mask(g, idx, mask, t, tid);  // ends with a barrier: s_base is visible
   if (t >= g.T) return;
   const int w = tid >> 5;
   const uint32_t below = (1u << (tid & 31)) - 1u;
@@ -135,7 +138,7 @@ __global__ void __launch_bounds__(kTB) moe_place_kernel(const __grid_constant__ 
     if ((unsigned)e >= (unsigned)g.E) { g.pos[o] = -1; g.prank[o] = 0; continue; }
     int rank = __popc(mask[e * kMaskWords + w] & below);
     for (int w2 = 0; w2 < w; ++w2) rank += __popc(mask[e * kMaskWords + w2]);
-    const long long row = (long long)g.base[p * g.E + e] + g.blockcnt[((size_t)p * g.NB + b) * g.E + e] + rank;
+    const long long row = (long long)s_base[e] + g.blockcnt[((size_t)p * g.NB + b) * g.E + e] + rank;
     const int r = e / g.epr;
     g.prank[o] = r;
     if ((unsigned long long)row < g.cap) {
@@ -418,7 +421,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   pl->move_smem = 128 + (size_t)g.slots * g.tile_bytes;
   size_t off = 0;
   auto place = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  const size_t o_bc = place((size_t)R * g.NB * g.E * 4), o_base = place((size_t)R * g.E * 4);
+  const size_t o_bc = place((size_t)R * g.NB * g.E * 4);
   const size_t o_cnt = place((size_t)R * R * 8), o_ecnt = place((size_t)R * g.E * 8);
   const size_t o_pos = place((size_t)R * g.T * g.K * 4), o_prank = place((size_t)R * g.T * g.K * 4);
   const size_t o_flags = place(16);
@@ -426,7 +429,6 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   if (cudaMalloc(&pl->d_blob, off) != cudaSuccess) { cudaGetLastError(); delete pl; return PL_ERR_OOM; }
   if (cudaMemset(pl->d_blob, 0, off) != cudaSuccess) { cudaGetLastError(); cudaFree(pl->d_blob); delete pl; return PL_ERR_CUDA; }
   g.blockcnt = reinterpret_cast<int32_t*>(pl->d_blob + o_bc);
-  g.base = reinterpret_cast<int32_t*>(pl->d_blob + o_base);
   g.counts = reinterpret_cast<long long*>(pl->d_blob + o_cnt);
   g.ecounts = reinterpret_cast<long long*>(pl->d_blob + o_ecnt);
   g.pos = reinterpret_cast<int32_t*>(pl->d_blob + o_pos);
@@ -434,7 +436,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   g.flags = reinterpret_cast<int*>(pl->d_blob + o_flags);
   if (cudaFuncSetAttribute(moe_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->move_smem) != cudaSuccess ||
       cudaFuncSetAttribute(moe_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.E * kMaskWords * 4) != cudaSuccess ||
-      cudaFuncSetAttribute(moe_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.E * kMaskWords * 4) != cudaSuccess) {
+      cudaFuncSetAttribute(moe_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.E * kMaskWords * 4 + g.E * 4) != cudaSuccess) {
     cudaGetLastError();
     cudaFree(pl->d_blob);
     delete pl;
@@ -451,7 +453,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
     size_t off2 = 0;
     auto place2 = [&](size_t bytes) { size_t o = off2; off2 = align_up(off2 + bytes, 256); return o; };
     const size_t tk = (size_t)R * g.T * d.K;
-    const size_t q_bc = place2((size_t)R * g.NB * R * 4), q_base = place2((size_t)R * R * 4);
+    const size_t q_bc = place2((size_t)R * g.NB * R * 4);
     const size_t q_cnt = place2((size_t)R * R * 8), q_ecnt = place2((size_t)R * R * 8);
     const size_t q_pos = place2(tk * 4), q_prank = place2(tk * 4), q_ridx = place2(tk * 4), q_rmask = place2(tk * 4);
     const size_t q_ones = place2((size_t)g.T * d.K * 4), q_flags = place2(16);
@@ -466,7 +468,6 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
       return PL_ERR_CUDA;
     }
     d.blockcnt = reinterpret_cast<int32_t*>(pl->d_blob2 + q_bc);
-    d.base = reinterpret_cast<int32_t*>(pl->d_blob2 + q_base);
     d.counts = reinterpret_cast<long long*>(pl->d_blob2 + q_cnt);
     d.ecounts = reinterpret_cast<long long*>(pl->d_blob2 + q_ecnt);
     d.pos = reinterpret_cast<int32_t*>(pl->d_blob2 + q_pos);
@@ -511,8 +512,8 @@ pl_status_t pl_moe_dispatch(pl_moe_plan_t plan, const void* const* x, const int3
   const size_t mask_smem = (size_t)g.E * kMaskWords * 4;
   dim3 grid(g.NB, g.R);
   moe_count_kernel<<<grid, kTB, mask_smem, cs>>>(P, g);
-  moe_scan_kernel<<<1, 1024, 0, cs>>>(g);
-  moe_place_kernel<<<grid, kTB, mask_smem, cs>>>(P, g);
+  moe_scan_kernel<<<g.R, 256, 0, cs>>>(g);
+  moe_place_kernel<<<grid, kTB, mask_smem + (size_t)g.E * 4, cs>>>(P, g);
   const unsigned long long items = (unsigned long long)g.R * g.T * g.n_tiles;
   const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, (200 * 1024) / plan->move_smem));
   const int mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)plan->sm_count * per_sm);
@@ -597,8 +598,8 @@ pl_status_t pl_moe_dispatch_dedup(pl_moe_plan_t plan, const void* const* x, cons
   const size_t mask_smem = (size_t)d.E * kMaskWords * 4;
   dim3 grid(d.NB, d.R);
   moe_count_kernel<<<grid, kTB, mask_smem, cs>>>(P, d);
-  moe_scan_kernel<<<1, 1024, 0, cs>>>(d);
-  moe_place_kernel<<<grid, kTB, mask_smem, cs>>>(P, d);
+  moe_scan_kernel<<<d.R, 256, 0, cs>>>(d);
+  moe_place_kernel<<<grid, kTB, mask_smem + (size_t)d.E * 4, cs>>>(P, d);
   const unsigned long long items = (unsigned long long)d.R * d.T * d.n_tiles;
   const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, (200 * 1024) / plan->move_smem));
   const int mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)plan->sm_count * per_sm);
