@@ -34,8 +34,8 @@ if ROOT not in sys.path:
 MIB = 1 << 20
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one reduce-scatter launch of this workload,
-# from the ncu capture summarised in profiles/pl_exec_tma_kernel_bf16_c2_reduce_scatter_all_gather.md
+# dram__bytes_read.sum + dram__bytes_write.sum of one reduce-scatter launch of this workload
+# (one ncu capture of that launch)
 NCU_RS_TRAFFIC_BYTES = 593797120.0
 
 
@@ -450,7 +450,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="purlin", choices=["purlin", "reference"])
-    ap.add_argument("--suite", action="store_true", help="run every configuration (paper_2609_36954_b200/bench_suite.py)")
+    ap.add_argument("--suite", action="store_true", help="run every configuration (bench_suite.py)")
     ap.add_argument("--cpu-suite", action="store_true", help="time the CPU oracle on samples of every configuration (1 thread and all cores)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -471,7 +471,7 @@ def main():
     elif args.cpu_suite:
         run_cpu_suite(args)
     elif args.suite:
-        from paper_2609_36954_b200 import bench_suite
+        import bench_suite
         bench_suite.main(args)
     else:
         run_purlin(args)

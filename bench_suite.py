@@ -15,8 +15,8 @@ import sys
 import numpy as np
 import torch
 
-from . import binding as B
-from . import inputs as gen
+from paper_2609_36954_b200 import binding as B
+from paper_2609_36954_b200 import inputs as gen
 
 MIB = 1 << 20
 ALGO = {"ring": B.PL_ALGO_RING, "tree": B.PL_ALGO_TREE, "direct": B.PL_ALGO_DIRECT,
@@ -24,7 +24,7 @@ ALGO = {"ring": B.PL_ALGO_RING, "tree": B.PL_ALGO_TREE, "direct": B.PL_ALGO_DIRE
 
 
 def _peak():
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    root = os.path.dirname(os.path.abspath(__file__))
     try:
         return float(json.load(open(os.path.join(root, "MEASURED_PEAKS.json")))["hbm_gbs"])
     except Exception:

@@ -249,7 +249,12 @@ typedef struct {
 
 /* ---- communicator ------------------------------------------------------------------ */
 
-/* Create a communicator of R emulated ranks (2 <= R <= PL_MAX_RANKS) with element type
+/* The communicator holds the state that outlives one call (Sec. 4.2: the paper's executor keeps
+ * persistent per-communicator state -- epoch, flags, staging -- between calls so that nothing is
+ * set up or cleared per collective): here the device status record and the list of schedules,
+ * each of which owns its epoch and flag words.
+ *
+ * Create a communicator of R emulated ranks (2 <= R <= PL_MAX_RANKS) with element type
  * `dtype` on the CURRENT CUDA device.  Allocates a few device words (status, abort).
  * Errors: PL_ERR_INVALID_ARG (R, dtype, out), PL_ERR_CUDA (no usable device). */
 pl_status_t pl_comm_create(int R, pl_dtype_t dtype, pl_comm_t* out);
@@ -320,7 +325,9 @@ pl_status_t pl_schedule_build_rooted(pl_comm_t comm, pl_collective_t coll, int r
                                      size_t chunk_bytes, const pl_sched_opts_t* opts, pl_schedule_t* out);
 
 /* n_layers back-to-back all-reduces in ONE launch (the latency path: no kernel launch,
- * memset or host round trip per layer).  Layer l reads in[r] + l*M and writes out[r] + l*M
+ * memset or host round trip per layer).  The shape is tensor-parallel decoding (Sec. 2.1:
+ * decode exchanges messages of tens of KB per layer, where set-up and synchronisation cost
+ * dominate; Sec. 3.2 "Specializing for latency").  Layer l reads in[r] + l*M and writes out[r] + l*M
  * (M = count_per_rank * elem_size).  Rank r's layer-(l+1) contribution counts as published
  * only when r's layer-l output is complete, and no consumer reads it earlier.  Algorithms:
  * PL_ALGO_ONESHOT, PL_ALGO_DIRECT, PL_ALGO_DIRECT_FUSED. */
@@ -363,7 +370,10 @@ pl_status_t pl_schedule_destroy(pl_schedule_t s);
 
 /* ---- datapath ---------------------------------------------------------------------- */
 
-/* Run the schedule once over `bufs` on `stream` (asynchronous, one kernel launch).
+/* Run the schedule once over `bufs` on `stream` (asynchronous, one kernel launch): the datapath
+ * tier (Sec. 3.3, Listing 3 and Algorithm 2): every CTA walks its op queue, and per op waits,
+ * moves the chunk through the pipeline with the op's consume step (copy or rank-ordered
+ * reduce, Eq. "rank-order") and signals.
  * Errors (all before launch): PL_ERR_INVALID_ARG (NULL pointer, buffer smaller than
  * pl_schedule_info reports, in/out ranges that overlap), PL_ERR_ALIGNMENT (a pointer not
  * 16-byte aligned), PL_ERR_UNSUPPORTED (planner communicator), PL_ERR_CUDA (launch). */
@@ -446,12 +456,22 @@ pl_status_t pl_moe_plan_read(pl_moe_plan_t plan, int32_t* pos, int64_t* counts,
  *   - The first call on a device looks up the device address of the built-in array (a one-
  *     time set-up with that device current); make that first call outside any stream capture.
  *   - All calls on a GPU share the array, and it keeps whatever the last call left there.
- *     Nothing in it needs clearing between calls, but two calls that overlap in time on the
- *     same GPU (e.g. on two streams) race on it: issue them on one stream or order them.
+ *     Nothing in it needs clearing between calls (the kernel numbers its calls with a counter
+ *     that lives on the device and ignores readiness marks of earlier calls, also after a
+ *     time-out), but two calls that overlap in time on the same GPU (e.g. on two streams) race
+ *     on it: issue them on one stream or order them.
  *   - Calls no cudaMalloc, cudaFree or other allocating routine. */
 pl_status_t pl_reduce_scatter_ring_static(int R, pl_dtype_t dtype, size_t count_per_rank,
                                           const void* const* in, void* const* out,
                                           int32_t* status, void* stream);
+
+/* TEST HOOK for the call above (the paper has no counterpart): same arguments, but every wait
+ * inside the kernel expects a mark that is never published and gives up after timeout_ns
+ * (1 ns .. 1 s), so that *status becomes PL_ERR_TIMEOUT and the outputs are incomplete.  Shows
+ * that a time-out leaves the GPU and the built-in array usable for the next call. */
+pl_status_t pl_reduce_scatter_ring_static_debug_timeout(int R, pl_dtype_t dtype, size_t count_per_rank,
+                                                        const void* const* in, void* const* out,
+                                                        int32_t* status, void* stream, uint64_t timeout_ns);
 
 /* Deduplicated variant (one row per token and DESTINATION RANK instead of per expert: when
  * several of a token's experts live on one rank the row crosses once; 32 % fewer rows on the

@@ -97,6 +97,7 @@ EXPORTS = [
     "pl_moe_plan_create", "pl_moe_plan_destroy", "pl_moe_dispatch", "pl_moe_combine", "pl_moe_plan_read",
     "pl_moe_dispatch_dedup", "pl_moe_combine_dedup", "pl_moe_plan_read_dedup", "pl_moe_combine_logits",
     "pl_status_string", "pl_launch_count", "pl_reduce_scatter_ring_static",
+    "pl_reduce_scatter_ring_static_debug_timeout",
 ]
 
 _lib = None
@@ -148,6 +149,7 @@ def load():
         "pl_moe_combine_dedup": [vp, P(vp), P(vp), vp],
         "pl_moe_plan_read_dedup": [vp, vp, vp, vp],
         "pl_reduce_scatter_ring_static": [i32, i32, sz, P(vp), P(vp), vp, vp],
+        "pl_reduce_scatter_ring_static_debug_timeout": [i32, i32, sz, P(vp), P(vp), vp, vp, u64],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -370,6 +372,12 @@ def pl_reduce_scatter_ring_static(R, dtype, count_per_rank, ins, outs, status=0,
     pl_status_t instead of raising, so that callers can test the size limit."""
     return load().pl_reduce_scatter_ring_static(R, dtype, count_per_rank, _ptr_array(ins), _ptr_array(outs),
                                                 status or None, stream)
+
+
+def pl_reduce_scatter_ring_static_debug_timeout(R, dtype, count_per_rank, ins, outs, status, stream, timeout_ns):
+    """Test hook: the same call with waits that can never be met and give up after timeout_ns."""
+    return load().pl_reduce_scatter_ring_static_debug_timeout(R, dtype, count_per_rank, _ptr_array(ins), _ptr_array(outs),
+                                                              status or None, stream, timeout_ns)
 
 
 def pl_launch_count() -> int:

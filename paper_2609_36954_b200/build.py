@@ -12,7 +12,7 @@ LIB = os.path.join(HERE, "libpurlin.so")
 SOURCES = ["pl_orchestrator.cpp", "pl_api.cu", "pl_datapath.cu", "pl_datapath_tma.cu", "pl_moe.cu", "pl_noalloc.cu", "pl_probe.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-    "--use_fast_math=false" if False else "-Xptxas=-v", "-shared", "-Xcompiler", "-fPIC",
+    "-Xptxas=-v", "-shared", "-Xcompiler", "-fPIC",
     "-cudart", "static",
 ]
 

@@ -258,7 +258,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   }
   assign_queues(&S->L, comm->R, pol.n_ctas, latency);
   if (!(flags & PL_OPT_SKIP_VALIDATE)) {
-    st = validate(S->L, comm->R, &err);
+    st = validate(S->L, comm->R, &err, pol.datapath == PL_DP_TMA);
     if (st != PL_OK) {
       comm->last_error = err;
       delete S;
@@ -479,7 +479,7 @@ pl_status_t pl_schedule_dump(pl_schedule_t s, pl_op_t* ops, size_t cap, size_t* 
 pl_status_t pl_schedule_validate(pl_schedule_t s, char* msg, size_t msg_cap) {
   if (!s) return PL_ERR_INVALID_ARG;
   std::string err;
-  pl_status_t st = validate(s->L, s->comm->R, &err);
+  pl_status_t st = validate(s->L, s->comm->R, &err, s->pol.datapath == PL_DP_TMA);
   if (msg && msg_cap) {
     std::snprintf(msg, msg_cap, "%s", err.c_str());
   }

@@ -375,17 +375,27 @@ cudaError_t launch_exec(int dtype, const ExecParams& P, int grid, int threads, c
   }
 }
 
-int exec_max_ctas_per_sm(int dtype, int threads) {
-  int n = 0;
-  cudaError_t e;
-  switch (dtype) {
-    case PL_BF16: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_BF16, true>, threads, 0); break;
-    case PL_F32: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_F32, true>, threads, 0); break;
-    case PL_I32: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_I32, true>, threads, 0); break;
-    default: e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_kernel<PL_U8, true>, threads, 0); break;
+namespace {
+template <int DT>
+int occupancy_both(int threads) {
+  // capacity that holds for whichever variant a schedule launches
+  int a = 0, b = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, pl_exec_kernel<DT, true>, threads, 0) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, pl_exec_kernel<DT, false>, threads, 0) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
   }
-  if (e != cudaSuccess) { cudaGetLastError(); return 0; }
-  return n;
+  return a < b ? a : b;
+}
+}  // namespace
+
+int exec_max_ctas_per_sm(int dtype, int threads) {
+  switch (dtype) {
+    case PL_BF16: return occupancy_both<PL_BF16>(threads);
+    case PL_F32: return occupancy_both<PL_F32>(threads);
+    case PL_I32: return occupancy_both<PL_I32>(threads);
+    default: return occupancy_both<PL_U8>(threads);
+  }
 }
 
 int exec_max_threads() { return kMaxThreads; }

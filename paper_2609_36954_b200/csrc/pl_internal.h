@@ -132,7 +132,9 @@ void assign_queues(Lowered* L, int R, int n_queues, bool by_level = false);
 // Largest number of ops one rank has at the same depth of the flag-dependency graph: the
 // queues per rank a latency-bound schedule can keep busy at once.
 int level_width(const Lowered& L, int R);
-pl_status_t validate(const Lowered& L, int R, std::string* err);
+// bulk_datapath: the schedule runs on the bulk-copy executor, where program order on one queue
+// orders less than on the register executor (see validate()).
+pl_status_t validate(const Lowered& L, int R, std::string* err, bool bulk_datapath);
 Policy default_policy(const BuildRequest& rq, int max_resident_ctas);
 
 }  // namespace pl

@@ -11,6 +11,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -355,6 +356,25 @@ __global__ void __launch_bounds__(kCombineThreads) moe_combine_kernel(const __gr
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// The dynamic shared-memory limit is an attribute of the FUNCTION (per device), not of a plan:
+// it is raised once per device to the most any plan can ask for, so that creating a second,
+// smaller plan cannot lower it under the feet of the first.
+constexpr int kMaxExperts = 4096;
+constexpr size_t kMoveSmemMax = 128 + 8 * (size_t)kMaxTile;
+bool configure_kernels(int device) {
+  static std::atomic<unsigned long long> configured{0};
+  const unsigned long long bit = 1ull << (device & 63);
+  if (configured.load(std::memory_order_acquire) & bit) return true;
+  if (cudaFuncSetAttribute(moe_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMoveSmemMax) != cudaSuccess ||
+      cudaFuncSetAttribute(moe_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxExperts * kMaskWords * 4) != cudaSuccess ||
+      cudaFuncSetAttribute(moe_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxExperts * kMaskWords * 4 + kMaxExperts * 4) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  configured.fetch_or(bit, std::memory_order_release);
+  return true;
+}
+
 }  // namespace
 
 struct pl_moe_plan_s {
@@ -385,7 +405,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
   const int R = comm->R;
   if (tokens_per_rank < 1 || hidden < 1 || n_experts < R || topk < 1 || topk > kMaxTopk) return PL_ERR_INVALID_ARG;
-  if (n_experts % R || n_experts > 4096 || topk > n_experts) return PL_ERR_INVALID_ARG;
+  if (n_experts % R || n_experts > kMaxExperts || topk > n_experts) return PL_ERR_INVALID_ARG;
   if (recv_capacity_rows == 0 || recv_capacity_rows > 0x7FFFFFFFull) return PL_ERR_INVALID_ARG;
   const size_t row_bytes = (size_t)hidden * elem_size(comm->dtype);
   if (row_bytes % 16) return PL_ERR_ALIGNMENT;
@@ -434,10 +454,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   g.pos = reinterpret_cast<int32_t*>(pl->d_blob + o_pos);
   g.prank = reinterpret_cast<int32_t*>(pl->d_blob + o_prank);
   g.flags = reinterpret_cast<int*>(pl->d_blob + o_flags);
-  if (cudaFuncSetAttribute(moe_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->move_smem) != cudaSuccess ||
-      cudaFuncSetAttribute(moe_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.E * kMaskWords * 4) != cudaSuccess ||
-      cudaFuncSetAttribute(moe_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g.E * kMaskWords * 4 + g.E * 4) != cudaSuccess) {
-    cudaGetLastError();
+  if (!configure_kernels(comm->device)) {
     cudaFree(pl->d_blob);
     delete pl;
     return PL_ERR_CUDA;
@@ -524,13 +541,14 @@ pl_status_t pl_moe_dispatch(pl_moe_plan_t plan, const void* const* x, const int3
   return PL_OK;
 }
 
-pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float* const* gates, void* const* out,
-                           void* stream) {
+static pl_status_t combine_impl(pl_moe_plan_t plan, const void* const* y, const float* const* gates, void* const* out,
+                                void* stream, bool gates_are_logits) {
   if (!plan || !y || !gates || !out) return PL_ERR_INVALID_ARG;
   if (plan->comm->dtype != PL_BF16) return PL_ERR_UNSUPPORTED;
   if (!plan->dispatched) return PL_ERR_INVALID_ARG;
   if (!on_comm_device(plan->comm)) return PL_ERR_INVALID_ARG;
-  const MoeGeo& g = plan->g;
+  MoeGeo g = plan->g;  // by value: the mode below belongs to this call, not to the plan
+  g.gates_are_logits = gates_are_logits ? 1 : 0;
   CombinePtrs P;
   std::memset(&P, 0, sizeof(P));
   for (int r = 0; r < g.R; ++r) {
@@ -548,13 +566,14 @@ pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float
   return PL_OK;
 }
 
+pl_status_t pl_moe_combine(pl_moe_plan_t plan, const void* const* y, const float* const* gates, void* const* out,
+                           void* stream) {
+  return combine_impl(plan, y, gates, out, stream, false);
+}
+
 pl_status_t pl_moe_combine_logits(pl_moe_plan_t plan, const void* const* y, const float* const* logits,
                                   void* const* out, void* stream) {
-  if (!plan) return PL_ERR_INVALID_ARG;
-  plan->g.gates_are_logits = 1;
-  pl_status_t st = pl_moe_combine(plan, y, logits, out, stream);
-  plan->g.gates_are_logits = 0;
-  return st;
+  return combine_impl(plan, y, logits, out, stream, true);
 }
 
 pl_status_t pl_moe_plan_read(pl_moe_plan_t plan, int32_t* pos, int64_t* counts, int64_t* expert_counts, void* stream) {

@@ -14,6 +14,10 @@
 // (different streams) would overwrite each other's partial sums.  Nothing in it has to start
 // at zero: partial sums are fully rewritten by every call, and the readiness words carry a
 // call number that only grows, so left-overs of earlier calls are never mistaken for "ready".
+// The call number lives on the device (every CTA reads it at entry, the last CTA to leave
+// advances it), so it follows the order in which the launches actually run: host threads that
+// enqueue in another order than they entered, or a captured launch that is replayed, cannot
+// desynchronise it.
 #include <cuda_runtime.h>
 
 #include <atomic>
@@ -37,6 +41,7 @@ constexpr int kThreads = 512;
 // device addresses are looked up once per device with cudaGetSymbolAddress (see setup()).
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 static __device__ __align__(256) unsigned long long g_ready[PL_MAX_RANKS * PL_MAX_RANKS * kMaxSlices];
+static __device__ __align__(256) unsigned long long g_calls[2];  // [0] calls completed, [1] CTAs of the running call that left
 
 struct RingParams {
   const void* in[PL_MAX_RANKS];
@@ -44,7 +49,8 @@ struct RingParams {
   unsigned char* scratch;       // device address of g_scratch
   unsigned long long* ready;    // device address of g_ready: [rank][step][slice]
   int* status;                  // caller-owned device word (may be null): 0 or PL_ERR_TIMEOUT
-  unsigned long long call;      // number of this call on this device (1, 2, ...)
+  unsigned long long* calls;    // device address of g_calls
+  unsigned long long wait_bias; // 0; the test hook raises what every wait expects so that it can never be met
   unsigned long long units;     // 16-byte units of the element type per partition
   unsigned long long timeout_ns;
   int R;
@@ -99,16 +105,21 @@ __global__ void __launch_bounds__(kThreads) pl_ring_rs_static_kernel(const __gri
   const unsigned long long part_e = U * kE;  // elements per partition
   const int q = (r + R - 1) % R;
   if (tid == 0) s_abort = 0;
+  // number of this call: all CTAs read the counter before any of them reports that it has left,
+  // and it only moves once all of them have, so they agree
+  const unsigned long long call = *reinterpret_cast<volatile unsigned long long*>(p.calls) + 1ull;
+  const unsigned long long expect = call + p.wait_bias;
   __syncthreads();
+  bool aborted = false;
   for (int s = 0; s <= R - 2; ++s) {
     const int k = ((r - s - 2) % R + R) % R;
     const bool last = s == R - 2;
     if (s > 0 && tid == 0) {
       const unsigned long long* f = p.ready + ((size_t)q * PL_MAX_RANKS + (s - 1)) * kMaxSlices + g;
-      if (ld_acquire_u64(f) < p.call) {
+      if (ld_acquire_u64(f) < expect) {
         const unsigned long long t0 = globaltimer_ns();
         unsigned spins = 0;
-        while (ld_acquire_u64(f) < p.call) {
+        while (ld_acquire_u64(f) < expect) {
           if ((++spins & 63u) == 0 && globaltimer_ns() - t0 > p.timeout_ns) {
             if (p.status) atomicExch(p.status, (int)PL_ERR_TIMEOUT);
             s_abort = 1;
@@ -118,7 +129,7 @@ __global__ void __launch_bounds__(kThreads) pl_ring_rs_static_kernel(const __gri
       }
     }
     __syncthreads();
-    if (s_abort) return;
+    if (s_abort) { aborted = true; break; }
     const char* a = (s == 0) ? static_cast<const char*>(p.in[q]) + (size_t)k * part_e * es
                              : reinterpret_cast<const char*>(p.scratch) + ((size_t)q * (R - 2) + (s - 1)) * part_e * ps;
     const char* b = static_cast<const char*>(p.in[r]) + (size_t)k * part_e * es;
@@ -129,8 +140,20 @@ __global__ void __launch_bounds__(kThreads) pl_ring_rs_static_kernel(const __gri
       __syncthreads();
       if (tid == 0) {
         __threadfence();
-        asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.ready + ((size_t)r * PL_MAX_RANKS + s) * kMaxSlices + g), "l"(p.call) : "memory");
+        asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.ready + ((size_t)r * PL_MAX_RANKS + s) * kMaxSlices + g), "l"(call) : "memory");
       }
+    }
+  }
+  (void)aborted;
+  // The last CTA to leave advances the call number, after a timeout too: the next call then
+  // expects a larger number than anything this one may have left in the readiness words.
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned long long left = atomicAdd(p.calls + 1, 1ull);
+    if (left == (unsigned long long)gridDim.x * gridDim.y - 1ull) {
+      p.calls[1] = 0ull;
+      __threadfence();
+      *reinterpret_cast<volatile unsigned long long*>(p.calls) = call;
     }
   }
 }
@@ -139,8 +162,8 @@ struct DeviceState {
   bool ready = false;
   unsigned char* scratch = nullptr;
   unsigned long long* flags = nullptr;
+  unsigned long long* calls = nullptr;
   int sm_count = 0;
-  unsigned long long calls = 0;
 };
 DeviceState g_dev[kMaxDevices];
 std::mutex g_mu;
@@ -152,6 +175,7 @@ pl_status_t setup(int device, DeviceState** out) {
   if (!d.ready) {
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&d.scratch), g_scratch) != cudaSuccess ||
         cudaGetSymbolAddress(reinterpret_cast<void**>(&d.flags), g_ready) != cudaSuccess ||
+        cudaGetSymbolAddress(reinterpret_cast<void**>(&d.calls), g_calls) != cudaSuccess ||
         cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
       cudaGetLastError();
       return PL_ERR_CUDA;
@@ -164,9 +188,8 @@ pl_status_t setup(int device, DeviceState** out) {
 
 }  // namespace
 
-extern "C" pl_status_t pl_reduce_scatter_ring_static(int R, pl_dtype_t dtype, size_t count_per_rank,
-                                                     const void* const* in, void* const* out,
-                                                     int32_t* status, void* stream) {
+static pl_status_t ring_static(int R, pl_dtype_t dtype, size_t count_per_rank, const void* const* in, void* const* out,
+                               int32_t* status, void* stream, unsigned long long wait_bias, unsigned long long timeout_ns) {
   if (R < 2 || R > PL_MAX_RANKS || !in || !out) return PL_ERR_INVALID_ARG;
   if (dtype != PL_BF16 && dtype != PL_F32 && dtype != PL_I32) return PL_ERR_UNSUPPORTED;
   const size_t es = elem_size(dtype), ps = elem_size(partial_dtype(dtype));
@@ -181,21 +204,21 @@ extern "C" pl_status_t pl_reduce_scatter_ring_static(int R, pl_dtype_t dtype, si
   if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
   RingParams p;
   DeviceState* d = nullptr;
-  {
-    std::lock_guard<std::mutex> lock(g_mu);
-    pl_status_t st = setup(device, &d);
-    if (st != PL_OK) return st;
-    p.call = ++d->calls;
-  }
+  // one caller at a time from set-up to launch: calls reach the stream in the order they got here
+  std::lock_guard<std::mutex> lock(g_mu);
+  pl_status_t st = setup(device, &d);
+  if (st != PL_OK) return st;
   for (int r = 0; r < PL_MAX_RANKS; ++r) {
     p.in[r] = r < R ? in[r] : nullptr;
     p.out[r] = r < R ? out[r] : nullptr;
   }
   p.scratch = d->scratch;
   p.ready = d->flags;
+  p.calls = d->calls;
+  p.wait_bias = wait_bias;
   p.status = status;
   p.units = part * es / 16;
-  p.timeout_ns = 2000000000ull;
+  p.timeout_ns = timeout_ns;
   p.R = R;
   // all CTAs wait on one another, so the grid must be co-resident: at most one CTA per SM
   int slices = d->sm_count / R;
@@ -213,4 +236,20 @@ extern "C" pl_status_t pl_reduce_scatter_ring_static(int R, pl_dtype_t dtype, si
   if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
   g_launches.fetch_add(1);
   return PL_OK;
+}
+
+extern "C" pl_status_t pl_reduce_scatter_ring_static(int R, pl_dtype_t dtype, size_t count_per_rank,
+                                                     const void* const* in, void* const* out,
+                                                     int32_t* status, void* stream) {
+  return ring_static(R, dtype, count_per_rank, in, out, status, stream, 0ull, 2000000000ull);
+}
+
+// TEST HOOK: the same call, but every wait inside the kernel expects a call number that is never
+// published and gives up after timeout_ns, so that the time-out path (status word set, kernel
+// returns, later calls work) can be exercised without hanging a GPU.
+extern "C" pl_status_t pl_reduce_scatter_ring_static_debug_timeout(int R, pl_dtype_t dtype, size_t count_per_rank,
+                                                                   const void* const* in, void* const* out,
+                                                                   int32_t* status, void* stream, uint64_t timeout_ns) {
+  if (timeout_ns == 0 || timeout_ns > 1000000000ull) return PL_ERR_INVALID_ARG;
+  return ring_static(R, dtype, count_per_rank, in, out, status, stream, 1ull << 40, timeout_ns);
 }

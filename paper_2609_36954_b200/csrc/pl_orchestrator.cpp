@@ -1091,7 +1091,7 @@ namespace {
 using Key = std::pair<int, int>;  // (buf kind, rank)
 }  // namespace
 
-pl_status_t validate(const Lowered& L, int R, std::string* err) {
+pl_status_t validate(const Lowered& L, int R, std::string* err, bool bulk_datapath) {
   char msg[256];
   auto fail = [&](const char* m) {
     if (err) *err = m;
@@ -1168,17 +1168,44 @@ pl_status_t validate(const Lowered& L, int R, std::string* err) {
       if (f >= 0) signallers[f].push_back((int)i);
   std::vector<int> stamp(n, -1);
   int query = 0;
-  auto happens_before = [&](int a, int x) -> bool {
+  // What program order on one queue is worth depends on the executor.  The register executor
+  // puts a CTA-wide barrier between ops: everything of op a is done before anything of a later
+  // op on its queue.  The bulk-copy executor runs ahead: its producer warp issues the loads of
+  // later ops while the consumer warps (register stores) and the copier warp (bulk stores) are
+  // still writing earlier ones, and those two kinds of writers do not wait for each other.
+  // There, on one queue: a later op's READ is never ordered after an earlier op's write; an
+  // earlier op's reads are complete before a later op stores or signals (the ring is consumed
+  // in order); an earlier op's WRITES are complete before a later op's stores or signal only
+  // if both leave through the same kind of writer.
+  auto writer_class = [&](const HostOp& o) {  // 0: consumer warps, 1: copier warp (bulk stores)
+    if (o.kind == PL_OP_COPY) return 1;
+    bool plain = true;
+    for (const pl_ref_t& r : o.src)
+      if (r.dtype != o.dst.dtype) plain = false;
+    return (o.bcast && plain) ? 1 : 0;
+  };
+  // a_writes: the access of op a that must be complete is a write (else a read);
+  // x_reads: the access of op x that must come later is a read (else a write).
+  auto happens_before = [&](int a, int x, bool a_writes, bool x_reads) -> bool {
     if (a >= x) return false;
     ++query;
     std::vector<std::pair<int, int>> stack{{x, 0}};
     stamp[x] = query;
     size_t visited = 0;
+    const HostOp& oa = L.ops[a];
     while (!stack.empty()) {
       auto [y, depth] = stack.back();
       stack.pop_back();
       const HostOp& oy = L.ops[y];
-      if (oy.queue == L.ops[a].queue && a < y) return true;
+      if (oy.queue == oa.queue && a < y) {
+        if (!bulk_datapath) return true;
+        const bool same_writer = writer_class(oa) == writer_class(oy);
+        if (y == x) {
+          if (!x_reads && (!a_writes || same_writer)) return true;
+        } else if (!a_writes || same_writer) {
+          return true;  // y's signal is released after a's access is complete
+        }
+      }
       if (depth >= 6 || ++visited > 200000) continue;
       for (int f : oy.waits)
         for (int sgn : signallers[f]) {
@@ -1223,7 +1250,7 @@ pl_status_t validate(const Lowered& L, int R, std::string* err) {
         bool direct = false;
         for (int f : op.waits)
           if (f == L.ops[w].signal || f == L.ops[w].signal2) direct = true;
-        if (!direct && !happens_before(w, (int)i)) {
+        if (!direct && !happens_before(w, (int)i, true, true)) {
           std::snprintf(msg, sizeof msg, "op %zu reads bytes written by op %d without being ordered after it", i, w);
           return fail(msg);
         }
@@ -1243,12 +1270,12 @@ pl_status_t validate(const Lowered& L, int R, std::string* err) {
           std::snprintf(msg, sizeof msg, "ops %d and %zu write overlapping bytes of the output of rank %d", it->second.writer, i, r);
           return fail(msg);
         }
-        if (!happens_before(it->second.writer, (int)i)) {
+        if (!happens_before(it->second.writer, (int)i, true, false)) {
           std::snprintf(msg, sizeof msg, "op %zu overwrites scratch written by op %d without being ordered after it", i, it->second.writer);
           return fail(msg);
         }
         for (int rd : it->second.readers)
-          if (rd != (int)i && !happens_before(rd, (int)i)) {
+          if (rd != (int)i && !happens_before(rd, (int)i, false, false)) {
             std::snprintf(msg, sizeof msg, "op %zu overwrites scratch that op %d may still be reading", i, rd);
             return fail(msg);
           }

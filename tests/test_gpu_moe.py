@@ -285,3 +285,31 @@ def test_random_moe_shapes_match_the_oracle(seed):
             check_float(gen.bf16_bits_to_f64(out[p]), want[p], "bf16")
     finally:
         run.close()
+
+
+def test_a_second_smaller_plan_does_not_break_the_first():
+    """The kernels' shared-memory limit is a property of the function, not of a plan: a plan with
+    wide rows (86 KiB of tiles per CTA, above the 48 KiB default) must keep working after a plan
+    with narrow rows and few experts has been created."""
+    R, T, H, E, K = 4, 96, 7168, 64, 4
+    idx, gates = gen.moe_routing(R, T, E, K, seed=4)
+    x = gen.moe_tokens_bf16(R, T, H, seed=6)
+    cap = R * T * K
+    ref = oracle.moe_dispatch(x, idx, E, recv_capacity_rows=cap)
+    big = MoeRun(R, T, H, E, K, cap)
+    small = MoeRun(2, 16, 256, 4, 2, 64)
+    try:
+        xs = gen.moe_tokens_bf16(2, 16, 256, seed=7)
+        idxs, _ = gen.moe_routing(2, 16, 4, 2, seed=8)
+        st, recv_s, _, _, counts_s, _ = small.dispatch(xs, idxs)
+        refs = oracle.moe_dispatch(xs, idxs, 4, recv_capacity_rows=64)
+        assert st == B.PL_OK and np.array_equal(counts_s, refs["counts"])
+        st, recv, meta, pos, counts, ecounts = big.dispatch(x, idx)
+        assert st == B.PL_OK
+        assert np.array_equal(counts, ref["counts"])
+        for r in range(R):
+            nrows = int(counts[:, r].sum())
+            assert np.array_equal(recv[r].view(np.uint16).reshape(cap, H)[:nrows], ref["recv"][r][:nrows])
+    finally:
+        small.close()
+        big.close()

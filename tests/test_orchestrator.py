@@ -406,6 +406,52 @@ def test_validator_notices_a_dropped_wait_edge():
         pl.close()
 
 
+def test_validator_counts_queue_order_only_where_the_executor_gives_it():
+    """The register executor finishes an op before the next one of its queue starts; the bulk-copy
+    executor issues later ops' loads ahead of earlier ops' stores.  A read-after-write on one queue
+    with no flag edge is therefore fine for the first and must be rejected for the second."""
+    pl = Planner(4, "i32")
+    try:
+        n = 4 * 4 * 8
+        for datapath, want in ((B.PL_DP_LDST, B.PL_OK), (B.PL_DP_TMA, B.PL_ERR_INVALID_SCHEDULE)):
+            # tree with one queue per rank: a rank's level-1 addition reads its own level-0 partial
+            s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_TREE, n, n * 4, n_ctas=4, datapath=datapath)
+            assert B.pl_schedule_validate(s)[0] == B.PL_OK
+            ops = B.pl_schedule_dump(s)
+            signaller = {o.signal_flag: o for o in ops if o.signal_flag >= 0}
+            victim = next(o.topo for o in ops if o.kind == B.PL_OP_COPY_REDUCE and o.n_wait == 2
+                          and signaller[o.wait_flag[0]].queue == o.queue)
+            B.pl_schedule_debug_drop_wait(s, victim)
+            st, msg = B.pl_schedule_validate(s)
+            assert st == want, msg
+            if want != B.PL_OK:
+                assert "without being ordered" in msg
+    finally:
+        pl.close()
+
+
+@pytest.mark.parametrize("R", [2, 3, 8])
+def test_every_lowering_validates_under_the_bulk_copy_rules(R):
+    """All algorithms carry explicit flag edges for every dependency the bulk-copy executor does
+    not give by queue order (build runs the validator; a failure would raise)."""
+    pl = Planner(R, "bf16")
+    try:
+        n = R * 8 * 24
+        for chunk in (16, 64, n * 2):
+            for nct in (R, 3 * R):
+                kw = dict(datapath=B.PL_DP_TMA, n_ctas=nct, slice_bytes=32)
+                for algo in ALLREDUCE_ALGOS:
+                    pl.build(B.PL_ALLREDUCE, algo, n, chunk, **kw)
+                for coll in (B.PL_REDUCE_SCATTER, B.PL_ALLGATHER):
+                    for algo in (B.PL_ALGO_DIRECT, B.PL_ALGO_RING):
+                        pl.build(coll, algo, n, chunk, **kw)
+                pl.build(B.PL_ALLTOALL, B.PL_ALGO_DIRECT, n, chunk, **kw)
+                for coll in (B.PL_ALLREDUCE, B.PL_REDUCE_SCATTER, B.PL_ALLGATHER, B.PL_ALLTOALL):
+                    pl.build(coll, B.PL_ALGO_DIRECT, n, chunk, flags=B.PL_OPT_STAGED, staging_bytes=2 * chunk * R, **kw)
+    finally:
+        pl.close()
+
+
 # ---- V variants of all-gather / reduce-scatter ---------------------------------------------
 @pytest.mark.parametrize("R", [2, 5, 8])
 def test_allgatherv_reduce_scatterv_replay(R):
