@@ -497,11 +497,13 @@ pl_status_t pl_moe_plan_read_dedup(pl_moe_plan_t plan, int32_t* pos, int64_t* co
 /* NOT PART OF THE PAPER'S METHOD.  Enqueues one kernel on `stream` that streams `bytes` with
  * the instructions the executors use (bulk asynchronous copies through a shared-memory ring,
  * one CTA per SM): kind 0 reads src and drops the data, kind 1 fills dst with a fixed pattern
- * (32-bit word j of every 32 KiB tile = j * 2654435761 mod 2^32), kind 2 copies src to dst.  Timed with CUDA events by the caller it gives the pure-read, pure-write
- * and copy bandwidth that bound the read-dominated (reduce-scatter, MoE combine), write-
- * dominated (all-gather, MoE dispatch) and balanced (all-to-all) collectives on this GPU.
+ * (32-bit word j of every 32 KiB tile = j * 2654435761 mod 2^32), kind 2 copies src to dst,
+ * kind 3 writes every tile of src to the same offset of 8 consecutive regions of dst (one read
+ * to eight writes).  Timed with CUDA events by the caller it gives the pure-read, pure-write,
+ * copy and 1:8 bandwidth that bound the read-dominated (reduce-scatter, MoE combine), balanced
+ * (all-to-all) and write-dominated (all-gather, MoE dispatch) collectives on this GPU.
  *   src, dst  DEVICE pointers, 16-byte aligned, `bytes` long (src unused for kind 1, dst for
- *             kind 0); bytes a positive multiple of 32768
+ *             kind 0; dst 8 * bytes long for kind 3); bytes a positive multiple of 32768
  *   status    optional DEVICE word of the caller: cleared on `stream`, set to PL_ERR_TIMEOUT if
  *             a wait inside the kernel gave up (2 s); may be NULL
  * Errors (before any launch): PL_ERR_INVALID_ARG, PL_ERR_ALIGNMENT, PL_ERR_CUDA. */

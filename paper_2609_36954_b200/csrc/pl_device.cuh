@@ -152,17 +152,21 @@ struct Acc<PL_I32> {
 };
 
 // Record a timeout (first writer wins) and raise the abort word.
-static __device__ __noinline__ void record_timeout(const ExecParams& P, int queue, uint32_t topo, uint32_t flag,
-                                            unsigned long long expected, unsigned long long observed) {
-  if (atomicCAS(P.status, 0, (int)PL_ERR_TIMEOUT) == 0) {
-    P.status[1] = queue;
-    P.status[2] = (int)topo;
-    P.status[3] = (int)flag;
-    *reinterpret_cast<unsigned long long*>(P.status + 4) = expected;
-    *reinterpret_cast<unsigned long long*>(P.status + 6) = observed;
+static __device__ __noinline__ void record_timeout_at(int* status, int queue, uint32_t topo, uint32_t flag,
+                                                      unsigned long long expected, unsigned long long observed) {
+  if (atomicCAS(status, 0, (int)PL_ERR_TIMEOUT) == 0) {
+    status[1] = queue;
+    status[2] = (int)topo;
+    status[3] = (int)flag;
+    *reinterpret_cast<unsigned long long*>(status + 4) = expected;
+    *reinterpret_cast<unsigned long long*>(status + 6) = observed;
   }
   __threadfence();
-  atomicExch(P.status + 8, 1);
+  atomicExch(status + 8, 1);
+}
+static __device__ __forceinline__ void record_timeout(const ExecParams& P, int queue, uint32_t topo, uint32_t flag,
+                                                      unsigned long long expected, unsigned long long observed) {
+  record_timeout_at(P.status, queue, topo, flag, expected, observed);
 }
 
 }  // namespace dev

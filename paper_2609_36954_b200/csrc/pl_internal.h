@@ -95,6 +95,20 @@ struct ExecParams {
   uint32_t pipelined_reduce;  // host side only: every reduce op is plain (element-typed operands), use the 12-warp variant
 };
 
+// Parameters of the packet executor (layered one-shot all-reduce, see pl_datapath_packet.cu).
+struct PacketParams {
+  const void* in[PL_MAX_RANKS];
+  void* out[PL_MAX_RANKS];
+  void* pkt[PL_MAX_RANKS];      // per rank: two packet buffers (even / odd global layer), 2 * message bytes each
+  unsigned long long* epoch;    // [0] executes completed, [1] CTAs finished in this execute
+  int* status;                  // pl_devstatus_t words + abort word (comm-owned)
+  unsigned long long* trace;    // optional: per op [start, end] %globaltimer stamps
+  unsigned long long timeout_ns;
+  unsigned long long units_per_rank;  // 16-byte vectors of one layer's message
+  int n_ranks, n_layers, ctas_per_rank;
+  float out_scale;
+};
+
 struct Policy {
   int n_ctas, threads, datapath, stages;
   uint32_t stage_bytes, slice_bytes;
@@ -112,6 +126,7 @@ struct Lowered {
   uint64_t message_bytes = 0;
   int n_layers = 1;
   int role_queues[4] = {0, 0, 0, 0};  // queues per rank reserved for each role (0 = roles unused)
+  bool queues_preassigned = false;    // the lowering fixed op.queue itself (packet schedules)
 };
 
 struct BuildRequest {
@@ -123,6 +138,7 @@ struct BuildRequest {
   int root;                  // rooted collectives
   bool staged;               // stage through schedule-owned memory (ordinary application buffers)
   uint64_t staging_bytes;    // staging capacity per rank (0 = default)
+  int packet_ctas_per_rank;  // > 0: layered all-reduce on the packet datapath with this many CTAs per rank
   Policy pol;
 };
 

@@ -19,4 +19,10 @@ int exec_tma_max_ctas_per_sm(int dtype, int stages, uint32_t stage_bytes);
 int exec_tma_threads(bool pipelined);
 size_t exec_tma_smem_bytes(int stages, uint32_t stage_bytes);
 
+// packet executor (latency path): rank = cluster of ctas_per_rank CTAs
+cudaError_t launch_exec_packet(int dtype, const PacketParams& P, int threads, bool overlap, cudaStream_t stream);
+int exec_packet_max_groups(int dtype, int ctas_per_rank, int threads);
+int exec_packet_max_units_per_thread();
+int exec_packet_max_threads();
+
 }  // namespace pl

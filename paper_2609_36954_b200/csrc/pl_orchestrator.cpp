@@ -376,6 +376,44 @@ void ar_oneshot(Emitter& em, const Geo& g, int layer, uint64_t in_off, uint64_t 
     }
 }
 
+// Layered one-shot all-reduce for the packet datapath (Sec. 3.2, "Specializing for latency").
+// Rank r is a group of G CTAs; CTA (r, j) reduces slice j of every layer's message from all R
+// contributions.  The op list states the data movement and the ordering rules, with logical
+// flags: done[r][l] is signalled by the G ops of rank r in layer l and every op of layer l+1
+// waits for done[p][l] of all p (rank p's contribution to layer l+1 counts as published once
+// p's layer-l output is complete).  On the device no flag word exists: the G CTAs of a rank
+// join with a cluster barrier, then copy their slice of the next layer's input into 16-byte
+// packets (8 B payload + 8 B layer tag), and consumers poll the packets themselves.
+void ar_oneshot_packets(Emitter& em, const Geo& g, int n_layers, int G) {
+  const int R = g.R;
+  const uint64_t msg = g.n * g.es, per = g.n / (uint64_t)G;
+  std::vector<int> prev, cur;
+  for (int l = 0; l < n_layers; ++l) {
+    cur.assign(R, -1);
+    if (l + 1 < n_layers)
+      for (int r = 0; r < R; ++r) cur[r] = em.new_flag();
+    for (int r = 0; r < R; ++r)
+      for (int j = 0; j < G; ++j) {
+        HostOp op;
+        op.kind = PL_OP_REDUCE;
+        op.exec_rank = r;
+        op.layer = l;
+        op.count = per;
+        const uint64_t off = (uint64_t)l * msg + (uint64_t)j * per * g.es;
+        op.dst = ref(r, PL_BUF_OUT, g.dtype, off);
+        for (int p = 0; p < R; ++p) op.src.push_back(ref(p, PL_BUF_IN, g.dtype, off));
+        if (l > 0) op.waits = prev;
+        op.signal = cur[r];
+        op.queue = j * R + r;
+        em.L->ops.push_back(std::move(op));
+      }
+    prev = cur;
+  }
+  em.L->queues_preassigned = true;
+  // two packet buffers per rank, alternated by layer parity, each the message as packets (2x)
+  for (int r = 0; r < R; ++r) em.L->scratch_per_rank[r] = 4 * msg;
+}
+
 // all-reduce, direct fused: the reducer of partition k writes each result into all R outputs.
 void ar_fused(Emitter& em, const Geo& g, int layer, uint64_t in_off, uint64_t out_off, const LayerEdges* le) {
   em.phase_chunks = g.n_c;
@@ -967,6 +1005,12 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
       L->message_bytes = bytes;
       Geo gp = make_geo(R, dt, n, n / R, rq.chunk_bytes);  // partitioned view
       Geo gw = make_geo(R, dt, n, n, rq.chunk_bytes);      // whole-message view
+      if (rq.packet_ctas_per_rank > 0) {
+        if (rq.n_layers < 1 || rq.algo != PL_ALGO_ONESHOT) return fail(PL_ERR_UNSUPPORTED, "the packet datapath runs layered one-shot all-reduces");
+        if ((bytes / 16) % (uint64_t)rq.packet_ctas_per_rank) return fail(PL_ERR_INVALID_ARG, "message vectors must divide evenly over a rank's CTAs");
+        ar_oneshot_packets(em, gw, n_layers, rq.packet_ctas_per_rank);
+        return PL_OK;
+      }
       if (rq.n_layers > 0) {
         LayerEdges le;
         le.pub.assign(R, -1);
@@ -1056,8 +1100,12 @@ void assign_queues(Lowered* L, int R, int n_queues, bool by_level) {
       return std::make_pair(same, load[q]);
     };
     int best = lo[role];
-    for (int j = lo[role] + 1; j < hi[role]; ++j)
-      if (key(j) < key(best)) best = j;
+    if (L->queues_preassigned) {
+      best = op.queue / R;
+    } else {
+      for (int j = lo[role] + 1; j < hi[role]; ++j)
+        if (key(j) < key(best)) best = j;
+    }
     load[(size_t)best * R + op.exec_rank] += cost;
     if (by_level) {
       std::vector<int>& al = at_level[(size_t)best * R + op.exec_rank];

@@ -3,8 +3,8 @@
 // Not part of the paper's method.  The roofline fractions of the collectives are quoted against
 // a library copy; this probe measures, with the same instructions the executors use
 // (cp.async.bulk global->shared with mbarrier completion, cp.async.bulk shared->global), the
-// three ceilings that bound them: a pure read (reduce-scatter and MoE combine are 8 reads to
-// 1 write), a pure write (all-gather and MoE dispatch are write dominated) and a copy.
+// ceilings that bound them: a pure read (reduce-scatter and MoE combine are 8 reads to
+// 1 write), a pure write, a copy, and one read to eight writes (all-gather and MoE dispatch).
 //
 // One warp per CTA, one CTA per SM, a ring of 6 tiles of 32 KiB.  CTA c handles tiles
 // c, c + G, c + 2G, ...: at any moment the grid sweeps one compact window of the buffer.
@@ -42,7 +42,9 @@ __device__ __forceinline__ bool wait_full(uint64_t* bar, uint32_t parity) {
   }
 }
 
-// kind 0: read (tiles are loaded and dropped), 1: write (a fixed pattern tile is stored), 2: copy
+// kind 0: read (tiles are loaded and dropped), 1: write (a fixed pattern tile is stored), 2: copy,
+// 3: one read to eight writes (every tile is stored to the same offset of 8 consecutive regions of
+// dst, each as long as src): the mix of the all-gather and of the MoE dispatch
 __global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src, char* dst, unsigned long long n_tiles,
                                                       int* status) {
   extern __shared__ __align__(128) unsigned char smem[];
@@ -82,9 +84,14 @@ __global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src,
       if (n + kSlots < n_my) load(n + kSlots);  // the tile is dropped: its slot is free at once
       continue;
     }
-    ptx::bulk_s2g(dst + tile_off(n), tiles + (size_t)s * kTile, kTile);
+    if (kind == 3) {
+      for (unsigned long long j = 0; j < 8; ++j)
+        ptx::bulk_s2g(dst + j * n_tiles * kTile + tile_off(n), tiles + (size_t)s * kTile, kTile);
+    } else {
+      ptx::bulk_s2g(dst + tile_off(n), tiles + (size_t)s * kTile, kTile);
+    }
     ptx::bulk_commit();
-    if (kind == 2 && n >= 2) {
+    if (kind >= 2 && n >= 2) {
       ptx::bulk_wait_read<2>();  // the store of tile n-2 no longer reads its slot
       if (n - 2 + kSlots < n_my) load(n - 2 + kSlots);
     } else if (kind == 1) {
@@ -105,7 +112,7 @@ __global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src,
 }  // namespace
 
 extern "C" pl_status_t pl_probe_hbm(int kind, const void* src, void* dst, size_t bytes, int32_t* status, void* stream) {
-  if (kind < 0 || kind > 2 || bytes == 0 || bytes % kTile) return PL_ERR_INVALID_ARG;
+  if (kind < 0 || kind > 3 || bytes == 0 || bytes % kTile) return PL_ERR_INVALID_ARG;
   if ((kind != 1 && !src) || (kind != 0 && !dst)) return PL_ERR_INVALID_ARG;
   if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15)) return PL_ERR_ALIGNMENT;
   int dev = 0, sms = 0;
