@@ -335,6 +335,17 @@ def main(args=None):
         for batch in (1, 8, 64):
             for algo in ("oneshot", "direct", "fused"):
                 b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, batch * 8192, 0, iters=50, layers=80)
+    if "c5p" in which or "c5" in which:
+        # the two latency protocols side by side: per-rank flags (register executor) against
+        # 16-byte packets (8 B payload + 8 B tag), per layer, 80 layers in one launch
+        for kib in (4, 16, 64):
+            b.collective("C5-flags", 8, B.PL_BF16, B.PL_ALLREDUCE, "oneshot", kib * 512, 0, iters=100, layers=80)
+            b.collective("C5-flags", 8, B.PL_BF16, B.PL_ALLREDUCE, "fused", kib * 512, 0, iters=100, layers=80)
+            for g in (8, 4, 2, 1):
+                if kib * 1024 // 16 // g <= 1024:  # at most 4 vectors per thread
+                    b.collective("C5-packets G=%d" % g, 8, B.PL_BF16, B.PL_ALLREDUCE, "oneshot", kib * 512, 0, iters=100, layers=80,
+                                 datapath=B.PL_DP_PACKET, n_ctas=8 * g)
+    if "c5" in which:
         # the same with in-kernel time stamps: distribution of the per-layer latency inside one launch
         for batch in (1, 8, 64):
             b.collective("C5-trace", 8, B.PL_BF16, B.PL_ALLREDUCE, "fused", batch * 8192, 0, iters=20, layers=80,

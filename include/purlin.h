@@ -134,7 +134,22 @@ typedef enum { PL_BUF_IN = 0, PL_BUF_OUT = 1, PL_BUF_SCRATCH = 2 } pl_buf_kind_t
 /* How an op body moves bytes (Sec. 3.3).  TMA = cp.async.bulk staged through a
  * shared-memory ring of `stages` slots of `stage_bytes` (Algorithm 2: prime / steady /
  * drain).  LDST = 128-bit register loads/stores, unrolled (the paper's register path). */
-typedef enum { PL_DP_AUTO = 0, PL_DP_LDST = 1, PL_DP_TMA = 2 } pl_datapath_t;
+typedef enum {
+  PL_DP_AUTO = 0,
+  PL_DP_LDST = 1,
+  PL_DP_TMA = 2,
+  /* Sec. 3.2, "Specializing for latency": data travels as 16-byte packets of 8 bytes of payload
+   * and an 8-byte tag written with one store; the consumer polls the packet itself, so there is
+   * no separate flag, fence or acquire on the path.  Only for pl_schedule_build_layers with
+   * PL_ALGO_ONESHOT (or PL_ALGO_AUTO) and small messages (at most 128 KiB per rank; meant for
+   * up to 64 KiB): rank r runs as a thread-block cluster of n_ctas / R CTAs (1, 2, 4 or 8) that
+   * joins with a cluster barrier when its layer's output is complete and then publishes its
+   * next contribution; the schedule owns two packet buffers per rank, alternated by layer
+   * parity (Sec. 4.2, epoch-parity double buffering), tags are global layer numbers that only
+   * grow, nothing is reset between executes.  pl_schedule_dump shows the same data movement
+   * with the ordering rules as logical flags (no flag words exist on the device). */
+  PL_DP_PACKET = 3
+} pl_datapath_t;
 
 typedef struct pl_comm_s* pl_comm_t;
 typedef struct pl_schedule_s* pl_schedule_t;

@@ -32,7 +32,7 @@ PL_ALGO_RING, PL_ALGO_TREE, PL_ALGO_DIRECT, PL_ALGO_ONESHOT, PL_ALGO_DIRECT_FUSE
 # op kinds / buffer kinds / datapaths
 PL_OP_COPY, PL_OP_REDUCE, PL_OP_COPY_REDUCE = range(3)
 PL_BUF_IN, PL_BUF_OUT, PL_BUF_SCRATCH = range(3)
-PL_DP_AUTO, PL_DP_LDST, PL_DP_TMA = range(3)
+PL_DP_AUTO, PL_DP_LDST, PL_DP_TMA, PL_DP_PACKET = range(4)
 PL_OPT_SKIP_VALIDATE = 1
 PL_OPT_NO_L2_HINTS = 2
 PL_OPT_STAGED = 4

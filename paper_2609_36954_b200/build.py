@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpurlin.so")
-SOURCES = ["pl_orchestrator.cpp", "pl_api.cu", "pl_datapath.cu", "pl_datapath_tma.cu", "pl_moe.cu", "pl_noalloc.cu", "pl_probe.cu"]
+SOURCES = ["pl_orchestrator.cpp", "pl_api.cu", "pl_datapath.cu", "pl_datapath_tma.cu", "pl_datapath_packet.cu", "pl_moe.cu", "pl_noalloc.cu", "pl_probe.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
     "-Xptxas=-v", "-shared", "-Xcompiler", "-fPIC",

@@ -41,6 +41,8 @@ struct pl_schedule_s {
   bool overlap_launch = false;
   bool bcast_copies = false;      // some COPY op writes every rank's output
   bool pipelined_reduce = false;  // bulk-copy datapath: every reduce op is plain, run the 12-warp variant
+  int packet_ctas_per_rank = 0;   // > 0: packet datapath (layered one-shot all-reduce), CTAs per rank
+  long long packet_break_op = -1; // test hook (pl_schedule_debug_break_wait on a packet schedule)
   size_t off_trace = 0;
   float out_scale = 1.0f;
   // host copies in device (queue-major) order
@@ -56,6 +58,7 @@ struct pl_schedule_s {
   size_t sync_bytes = 0;  // flags + epoch, zeroed at build and by reset
   char* d_scratch = nullptr;
   uint64_t scratch_off[PL_MAX_RANKS] = {0};
+  uint64_t scratch_total = 0;
 };
 
 namespace {
@@ -173,9 +176,94 @@ pl_status_t upload(pl_schedule_s* S, int R) {
     S->scratch_off[r] = total;
     total += align_up(S->L.scratch_per_rank[r], 256);
   }
+  S->scratch_total = total;
   if (total) {
     if (cudaMalloc(&S->d_scratch, total) != cudaSuccess) { cudaGetLastError(); return PL_ERR_OOM; }
+    // packet buffers: a tag left over from whoever used this memory before must never match
+    if (S->packet_ctas_per_rank && cudaMemset(S->d_scratch, 0, total) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
   }
+  return PL_OK;
+}
+
+// Packet datapath (layered one-shot all-reduce of a small message): pick the CTAs per rank and
+// the CTA size, lower, check that all rank groups can be resident at once, upload.
+pl_status_t build_packets(pl_comm_t comm, BuildRequest rq, Policy pol, uint64_t timeout, uint32_t flags, float out_scale,
+                          pl_schedule_t* out) {
+  auto fail = [&](pl_status_t st, const char* m) {
+    comm->last_error = m;
+    return st;
+  };
+  const int R = comm->R, es = elem_size(comm->dtype);
+  if (rq.n_layers < 1 || rq.coll != PL_ALLREDUCE) return fail(PL_ERR_UNSUPPORTED, "the packet datapath runs layered all-reduces (pl_schedule_build_layers)");
+  if (rq.algo != PL_ALGO_ONESHOT) return fail(PL_ERR_UNSUPPORTED, "the packet datapath is one-shot");
+  if (comm->dtype == PL_U8) return fail(PL_ERR_UNSUPPORTED, "bytes cannot be reduced");
+  if (rq.staged || (flags & PL_OPT_STAGED)) return fail(PL_ERR_UNSUPPORTED, "packets are their own staging");
+  const uint64_t bytes = rq.count_per_rank * (uint64_t)es;
+  if (bytes == 0 || bytes % 16) return fail(PL_ERR_INVALID_ARG, "message bytes must be a positive multiple of 16");
+  const uint64_t units = bytes / 16;
+  int G = 0;
+  if (pol.n_ctas > 0) {
+    G = pol.n_ctas / R;
+    if (G * R != pol.n_ctas || (G != 1 && G != 2 && G != 4 && G != 8) || units % (uint64_t)G)
+      return fail(PL_ERR_INVALID_ARG, "n_ctas must be R times 1, 2, 4 or 8 and divide the message vectors");
+  } else {
+    for (G = 8; G > 1; G /= 2)
+      if (units % (uint64_t)G == 0 && units / (uint64_t)G >= 8) break;
+  }
+  const uint64_t per_cta = units / (uint64_t)G;
+  int threads = pol.threads > 0 ? pol.threads : (int)std::min<uint64_t>(exec_packet_max_threads(), (per_cta + 31) / 32 * 32);
+  if (threads > exec_packet_max_threads()) return fail(PL_ERR_INVALID_ARG, "at most 256 threads per CTA on the packet datapath");
+  if ((per_cta + threads - 1) / threads > (uint64_t)exec_packet_max_units_per_thread())
+    return fail(PL_ERR_UNSUPPORTED, "message too large for the packet datapath (at most 4 vectors per thread)");
+  if (!comm->planner) {
+    const int groups = exec_packet_max_groups(comm->dtype, G, threads);
+    if (groups <= 0) return PL_ERR_CUDA;
+    if (groups < R) return fail(PL_ERR_OVERSUBSCRIBED, "the rank groups of the packet datapath cannot all be resident");
+  }
+  pol.datapath = PL_DP_PACKET;
+  pol.n_ctas = G * R;
+  pol.threads = threads;
+  pol.stages = 0;
+  pol.stage_bytes = 0;
+  pol.slice_bytes = (uint32_t)(per_cta * 16);
+  rq.pol = pol;
+  rq.packet_ctas_per_rank = G;
+  rq.chunk_bytes = ((uint64_t)1 << 40);
+
+  pl_schedule_s* S = new (std::nothrow) pl_schedule_s();
+  if (!S) return PL_ERR_OOM;
+  S->comm = comm;
+  S->pol = pol;
+  S->timeout_ns = timeout;
+  S->trace = (flags & PL_OPT_TRACE) != 0;
+  S->overlap_launch = (flags & PL_OPT_OVERLAP_LAUNCH) != 0;
+  S->out_scale = out_scale;
+  S->packet_ctas_per_rank = G;
+  std::string err;
+  pl_status_t st = lower(rq, &S->L, &err);
+  if (st == PL_OK) {
+    assign_queues(&S->L, R, pol.n_ctas, false);
+    if (!(flags & PL_OPT_SKIP_VALIDATE)) st = validate(S->L, R, &err, false);
+  }
+  if (st != PL_OK) {
+    comm->last_error = err;
+    delete S;
+    return st;
+  }
+  fill_info(S, R);
+  flatten(S, comm->dtype);
+  if (!comm->planner) {
+    st = upload(S, R);
+    if (st != PL_OK) {
+      pl_schedule_destroy(S);
+      return st;
+    }
+  }
+  {
+    std::lock_guard<std::mutex> g(comm->mu);
+    comm->schedules.push_back(S);
+  }
+  *out = S;
   return PL_OK;
 }
 
@@ -205,10 +293,11 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
     }
     if (pol.threads < 0 || pol.threads % 32 || pol.threads > exec_max_threads()) return PL_ERR_INVALID_ARG;
     if (pol.n_ctas < 0 || pol.stages < 0 || pol.stage_bytes % 16 || pol.slice_bytes % 16) return PL_ERR_INVALID_ARG;
-    if (pol.datapath < PL_DP_AUTO || pol.datapath > PL_DP_TMA) return PL_ERR_INVALID_ARG;
+    if (pol.datapath < PL_DP_AUTO || pol.datapath > PL_DP_PACKET) return PL_ERR_INVALID_ARG;
   }
   rq.R = comm->R;
   rq.dtype = comm->dtype;
+  if (pol.datapath == PL_DP_PACKET) return build_packets(comm, rq, pol, timeout, flags, out_scale, out);
   rq.pol = pol;
   const int requested = pol.n_ctas;
   pol = default_policy(rq, 0);  // datapath, threads, ring geometry
@@ -379,8 +468,11 @@ pl_status_t pl_comm_reset(pl_comm_t comm, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(comm->d_status, 0, kStatusWords * sizeof(int), st) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
   std::lock_guard<std::mutex> g(comm->mu);
-  for (pl_schedule_s* S : comm->schedules)
+  for (pl_schedule_s* S : comm->schedules) {
     if (S->d_blob && cudaMemsetAsync(S->d_blob + S->off_flags, 0, S->sync_bytes, st) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+    // packet tags restart with the epoch: old packets must not match them
+    if (S->packet_ctas_per_rank && S->d_scratch && cudaMemsetAsync(S->d_scratch, 0, S->scratch_total, st) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  }
   return PL_OK;
 }
 
@@ -433,6 +525,7 @@ pl_status_t pl_schedule_build_layers(pl_comm_t comm, pl_algo_t algo, size_t coun
   BuildRequest rq{};
   rq.coll = PL_ALLREDUCE;
   rq.algo = algo == PL_ALGO_AUTO ? PL_ALGO_DIRECT_FUSED : algo;  // the fastest layered form at 16 KiB - 1 MiB
+  if (algo == PL_ALGO_AUTO && opts && opts->struct_size == sizeof(pl_sched_opts_t) && opts->datapath == PL_DP_PACKET) rq.algo = PL_ALGO_ONESHOT;
   rq.count_per_rank = count_per_rank;
   rq.n_layers = n_layers;
   // a layer is one chunk per partition: the latency path does not pipeline inside a layer
@@ -509,6 +602,10 @@ pl_status_t pl_schedule_debug_break_wait(pl_schedule_t s, size_t op_index) {
   if (!s || op_index >= s->L.ops.size()) return PL_ERR_INVALID_ARG;
   const HostOp& h = s->L.ops[op_index];
   if (h.waits.empty()) return PL_ERR_INVALID_ARG;
+  if (s->packet_ctas_per_rank) {  // no wait entries on the device: the op's polls expect a tag nobody publishes
+    s->packet_break_op = (long long)op_index;
+    return PL_OK;
+  }
   const size_t pos = (size_t)s->topo_to_dev[op_index];
   DevWait& w = s->waits[pos * s->wait_stride];
   w.need += 1;  // one more signal than the schedule will ever produce
@@ -566,6 +663,32 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   if (!on_comm_device(s->comm)) return PL_ERR_INVALID_ARG;
   pl_status_t st = check_bufs(s, bufs);
   if (st != PL_OK) return st;
+  if (s->packet_ctas_per_rank) {
+    PacketParams K;
+    std::memset(&K, 0, sizeof(K));
+    const int R = s->comm->R;
+    for (int r = 0; r < R; ++r) {
+      K.in[r] = bufs->in[r];
+      K.out[r] = bufs->out[r];
+      K.pkt[r] = s->d_scratch + s->scratch_off[r];
+    }
+    K.epoch = reinterpret_cast<unsigned long long*>(s->d_blob + s->off_epoch);
+    K.status = s->comm->d_status;
+    K.trace = s->trace ? reinterpret_cast<unsigned long long*>(s->d_blob + s->off_trace) : nullptr;
+    K.timeout_ns = s->timeout_ns;
+    K.units_per_rank = s->L.message_bytes / 16;
+    K.n_ranks = R;
+    K.n_layers = s->L.n_layers;
+    K.ctas_per_rank = s->packet_ctas_per_rank;
+    K.out_scale = s->out_scale;
+    K.break_op = s->packet_break_op;
+    if (launch_exec_packet(s->comm->dtype, K, s->pol.threads, s->overlap_launch, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+      cudaGetLastError();
+      return PL_ERR_CUDA;
+    }
+    g_launches.fetch_add(1);
+    return PL_OK;
+  }
   ExecParams P;
   std::memset(&P, 0, sizeof(P));
   const int R = s->comm->R;

@@ -1,9 +1,11 @@
 // Packet datapath: the latency specialisation of the paper (Sec. 3.2, "Specializing for
 // latency").  L back-to-back one-shot all-reduces of a small message run in one launch.
 //
-// A packet is 16 bytes: 8 bytes of payload and an 8-byte tag, written with one 16-byte store
-// and read with one 16-byte load, so data and "data is ready" arrive together and no separate
-// flag word, fence or acquire sits on the path.  The tag is the global layer number (executes
+// A packet is 16 bytes: 8 bytes of payload and an 8-byte tag that travel in one store and one
+// load, so data and "data is ready" arrive together and no separate flag word, fence or acquire
+// sits on the path.  A thread owns 16 bytes of the message, i.e. two neighbouring packets (one
+// 32-byte sector), and moves both with one 256-bit access; each packet carries its own tag and
+// both tags are checked.  The tag is the global layer number (executes
 // completed * L + layer + 1): it only grows, nothing is ever reset, and a consumer accepts a
 // packet only when the tag is exactly the one it expects.
 //
@@ -50,8 +52,20 @@ __device__ __forceinline__ Packet ld_packet(const void* p) {
   asm volatile("ld.relaxed.gpu.global.v2.u64 {%0,%1}, [%2];" : "=l"(k.payload), "=l"(k.tag) : "l"(p) : "memory");
   return k;
 }
-__device__ __forceinline__ void st_packet(void* p, unsigned long long payload, unsigned long long tag) {
-  asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1,%2};" ::"l"(p), "l"(payload), "l"(tag) : "memory");
+// Two neighbouring packets (one 32-byte sector) with one 256-bit access.
+struct Packet2 {
+  Packet lo, hi;
+};
+__device__ __forceinline__ Packet2 ld_packet2(const void* p) {
+  Packet2 k;
+  asm volatile("ld.relaxed.gpu.global.v4.u64 {%0,%1,%2,%3}, [%4];"
+               : "=l"(k.lo.payload), "=l"(k.lo.tag), "=l"(k.hi.payload), "=l"(k.hi.tag)
+               : "l"(p)
+               : "memory");
+  return k;
+}
+__device__ __forceinline__ void st_packet2(void* p, unsigned long long pay0, unsigned long long pay1, unsigned long long tag) {
+  asm volatile("st.relaxed.gpu.global.v4.u64 [%0], {%1,%2,%3,%4};" ::"l"(p), "l"(pay0), "l"(tag), "l"(pay1), "l"(tag) : "memory");
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -89,8 +103,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_packet_kernel(const __gri
       const uint64_t u = (uint64_t)tid + (uint64_t)k * nthr;
       if (u < UC) {
         char* at = base + (u0 + u) * 32ull;
-        st_packet(at, ((unsigned long long)pub[k].y << 32) | pub[k].x, gl + 1ull);
-        st_packet(at + 16, ((unsigned long long)pub[k].w << 32) | pub[k].z, gl + 1ull);
+        st_packet2(at, ((unsigned long long)pub[k].y << 32) | pub[k].x, ((unsigned long long)pub[k].w << 32) | pub[k].z, gl + 1ull);
       }
     }
   };
@@ -99,26 +112,64 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_packet_kernel(const __gri
   publish(gl0);
   bool aborted = false;
   for (int l = 0; l < L; ++l) {
-    const unsigned long long gl = gl0 + (unsigned long long)l, want = gl + 1ull;
+    const unsigned long long gl = gl0 + (unsigned long long)l;
+    // test hook: the op named by break_op expects a tag nobody publishes
+    const unsigned long long want = gl + 1ull + (((long long)l * R + r) * G + j == P.break_op ? (1ull << 40) : 0ull);
     if (l + 1 < L) fetch_pub(l + 1);
     if (!aborted) {
+      const int lane = tid & 31;
 #pragma unroll 1
       for (int k = 0; k < kMaxUnitsPerThread; ++k) {
+        // control flow is uniform per warp from here to the end of the iteration
+        const uint64_t warp_first = (uint64_t)(tid & ~31) + (uint64_t)k * nthr;  // this warp's first vector
+        if (warp_first >= UC) break;
         const uint64_t u = (uint64_t)tid + (uint64_t)k * nthr;
-        if (u >= UC) break;
+        const bool mine = u < UC;
+        // ---- watch one packet per source first.  Polling every packet of every thread re-reads
+        // the whole message per round: that is bound by the SM's L2 bandwidth, not by latency,
+        // and the flood of loads delays the very stores it waits for.  The warp that publishes
+        // this warp's vectors for rank p is the same warp of the same CTA index in rank p, and
+        // the last packet it stores is the second packet of its last lane: lane p polls that one
+        // packet of rank p.  When all R are there, the full read below almost always finds
+        // everything in place (and polls on for whatever is not).
+        {
+          const uint64_t warp_last = min(UC - 1, warp_first + 31);
+          const bool poller = lane < R;
+          const char* sentinel = static_cast<const char*>(P.pkt[poller ? lane : 0]) + (gl & 1ull) * half + (u0 + warp_last) * 32ull + 16;
+          bool here = !poller || ld_packet(sentinel).tag == want;
+          if (!__all_sync(0xFFFFFFFFu, here)) {
+            const unsigned long long t0 = globaltimer_ns();
+            uint32_t spins = 0;
+            for (;;) {
+              if (!here) here = ld_packet(sentinel).tag == want;
+              if (__all_sync(0xFFFFFFFFu, here)) break;
+              if ((++spins & 63u) == 0) {
+                bool give_up = ld_volatile_s32(P.status + 8) != 0;
+                if (!give_up && !here && globaltimer_ns() - t0 > P.timeout_ns) {
+                  record_timeout_at(P.status, blockIdx.x, (uint32_t)((l * R + r) * G + j), (uint32_t)lane, want,
+                                    ld_packet(sentinel).tag);
+                  give_up = true;
+                }
+                if (__any_sync(0xFFFFFFFFu, give_up)) { aborted = true; break; }
+              }
+            }
+          }
+        }
+        if (aborted) break;  // warp-uniform
         Acc<DT> acc;
         acc.zero();
         const uint64_t at = (gl & 1ull) * half + (u0 + u) * 32ull;
+        bool failed = false;
 #pragma unroll 1
-        for (int p0 = 0; p0 < R && !aborted; p0 += kBatch) {
+        for (int p0 = 0; p0 < R && mine && !failed; p0 += kBatch) {
           Packet lo[kBatch], hi[kBatch];
           uint32_t pending = 0;
 #pragma unroll
           for (int b = 0; b < kBatch; ++b)
             if (p0 + b < R) {
-              const char* a = static_cast<const char*>(P.pkt[p0 + b]) + at;
-              lo[b] = ld_packet(a);
-              hi[b] = ld_packet(a + 16);
+              const Packet2 two = ld_packet2(static_cast<const char*>(P.pkt[p0 + b]) + at);
+              lo[b] = two.lo;
+              hi[b] = two.hi;
             }
 #pragma unroll
           for (int b = 0; b < kBatch; ++b)
@@ -127,27 +178,34 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_packet_kernel(const __gri
             const unsigned long long t0 = globaltimer_ns();
             uint32_t spins = 0;
             while (pending) {
+              // all missing packets are asked for again before any answer is looked at: one
+              // round trip per round, not one per source
 #pragma unroll
               for (int b = 0; b < kBatch; ++b)
                 if ((pending >> b) & 1u) {
-                  const char* a = static_cast<const char*>(P.pkt[p0 + b]) + at;
-                  lo[b] = ld_packet(a);
-                  hi[b] = ld_packet(a + 16);
-                  if (lo[b].tag == want && hi[b].tag == want) pending &= ~(1u << b);
+                  const Packet2 two = ld_packet2(static_cast<const char*>(P.pkt[p0 + b]) + at);
+                  lo[b] = two.lo;
+                  hi[b] = two.hi;
                 }
+#pragma unroll
+              for (int b = 0; b < kBatch; ++b)
+                if (((pending >> b) & 1u) && lo[b].tag == want && hi[b].tag == want) pending &= ~(1u << b);
               if (pending && (++spins & 63u) == 0) {
-                if (ld_volatile_s32(P.status + 8)) { aborted = true; break; }
+                if (ld_volatile_s32(P.status + 8)) { failed = true; break; }
                 if (globaltimer_ns() - t0 > P.timeout_ns) {
-                  const int b = __ffs(pending) - 1;
-                  record_timeout_at(P.status, blockIdx.x, (uint32_t)((l * R + r) * G + j), (uint32_t)(p0 + b), want,
-                                    lo[b].tag != want ? lo[b].tag : hi[b].tag);
-                  aborted = true;
+                  const int first = __ffs(pending) - 1;  // the lowest rank whose packets are missing
+                  unsigned long long seen = 0;
+#pragma unroll
+                  for (int b = 0; b < kBatch; ++b)
+                    if (b == first) seen = lo[b].tag != want ? lo[b].tag : hi[b].tag;
+                  record_timeout_at(P.status, blockIdx.x, (uint32_t)((l * R + r) * G + j), (uint32_t)(p0 + first), want, seen);
+                  failed = true;
                   break;
                 }
               }
             }
           }
-          if (!aborted) {
+          if (!failed) {
 #pragma unroll
             for (int b = 0; b < kBatch; ++b)
               if (p0 + b < R) {
@@ -158,11 +216,13 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_packet_kernel(const __gri
               }
           }
         }
-        if (aborted) break;
-        uint4 res;
-        if constexpr (DT == PL_BF16) res = acc.to_bf16(P.out_scale);
-        else res = acc.result(P.out_scale);
-        st16(static_cast<char*>(P.out[r]) + (uint64_t)l * msg + (u0 + u) * 16ull, res);
+        if (mine && !failed) {
+          uint4 res;
+          if constexpr (DT == PL_BF16) res = acc.to_bf16(P.out_scale);
+          else res = acc.result(P.out_scale);
+          st16(static_cast<char*>(P.out[r]) + (uint64_t)l * msg + (u0 + u) * 16ull, res);
+        }
+        if (__any_sync(0xFFFFFFFFu, failed)) { aborted = true; break; }
       }
       if (aborted) s_abort = 1;
     }

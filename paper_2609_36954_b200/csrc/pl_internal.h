@@ -105,6 +105,7 @@ struct PacketParams {
   unsigned long long* trace;    // optional: per op [start, end] %globaltimer stamps
   unsigned long long timeout_ns;
   unsigned long long units_per_rank;  // 16-byte vectors of one layer's message
+  long long break_op;                 // test hook: index of an op whose polls can never be satisfied, -1 = none
   int n_ranks, n_layers, ctas_per_rank;
   float out_scale;
 };

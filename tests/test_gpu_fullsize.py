@@ -101,14 +101,16 @@ def test_c3_allreduce_256mib_sampled(algo):
         B.pl_comm_destroy(comm)
 
 
-@pytest.mark.parametrize("batch,algo", [(1, B.PL_ALGO_DIRECT_FUSED), (1, B.PL_ALGO_ONESHOT), (64, B.PL_ALGO_DIRECT_FUSED)])
-def test_c5_decode_allreduce_80_layers(batch, algo):
+@pytest.mark.parametrize("batch,algo,datapath", [(1, B.PL_ALGO_DIRECT_FUSED, B.PL_DP_AUTO), (1, B.PL_ALGO_ONESHOT, B.PL_DP_AUTO),
+                                                 (64, B.PL_ALGO_DIRECT_FUSED, B.PL_DP_AUTO),
+                                                 (1, B.PL_ALGO_ONESHOT, B.PL_DP_PACKET), (4, B.PL_ALGO_ONESHOT, B.PL_DP_PACKET)])
+def test_c5_decode_allreduce_80_layers(batch, algo, datapath):
     R, hidden, layers = 8, 8192, 80
     n = batch * hidden
     comm = B.pl_comm_create(R, B.PL_BF16)
     try:
         x = big_inputs(R, n * layers, seed=5, block=1 << 18)
-        s = B.pl_schedule_build_layers(comm, algo, n, layers, None)
+        s = B.pl_schedule_build_layers(comm, algo, n, layers, B.make_opts(datapath=datapath))
         out = [torch.full((n * layers,), -1, dtype=torch.int16, device="cuda") for _ in range(R)]
         for _ in range(2):  # twice: flags carry over between executes
             run(s, comm, R, x, out)

@@ -172,6 +172,82 @@ def test_layered_allreduce_replay_and_program_order(algo):
         pl.close()
 
 
+@pytest.mark.parametrize("R,units,G", [(4, 24, 0), (8, 64, 8), (3, 5, 0), (2, 16, 2)])
+def test_packet_schedule_replay_program_order_and_geometry(R, units, G):
+    """The packet datapath's schedule: the op list states the data movement and the ordering rules
+    (as logical flags); replayed on the CPU it must give the oracle's all-reduce per layer, every
+    cross-layer edge must be there, and op (layer, rank, slice) must sit at the index the kernel
+    derives from its block index."""
+    dtype, Lyr = "bf16", 4
+    n = units * 8
+    pl = Planner(R, dtype)
+    try:
+        x = [np.concatenate([gen.normal_bf16(n, 0, l * R + r) for l in range(Lyr)]) for r in range(R)]
+        s = B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_AUTO, n, Lyr, B.make_opts(datapath=B.PL_DP_PACKET, n_ctas=G * R))
+        pl.scheds.append(s)
+        assert B.pl_schedule_validate(s)[0] == B.PL_OK
+        info = B.pl_schedule_info(s)
+        assert info.datapath == B.PL_DP_PACKET and info.n_layers == Lyr
+        g = int(info.grid) // R
+        assert g in (1, 2, 4, 8) and units % g == 0 and (G == 0 or g == G)
+        assert info.scratch_bytes == R * 4 * n * 2          # two packet buffers of twice the message per rank
+        ops = B.pl_schedule_dump(s)
+        assert len(ops) == Lyr * R * g
+        for o in ops:
+            r, j = o.exec_rank, o.queue // R
+            assert o.topo == (o.layer * R + r) * g + j and o.queue % R == r
+            assert o.count == n // g and o.dst.offset == (o.layer * n + j * (n // g)) * 2
+            assert o.n_wait == (R if o.layer else 0)
+        outs = interp_run(ops, info, R, x, seed=9)
+        for l in range(Lyr):
+            ref = oracle.allreduce([a[l * n:(l + 1) * n] for a in x], dtype)
+            for r in range(R):
+                check_float(gen.bf16_bits_to_f64(outs[r].view(np.uint16)[l * n:(l + 1) * n]), ref[r], dtype)
+        writers = {}
+        for o in ops:
+            if o.signal_flag >= 0:
+                writers.setdefault(o.signal_flag, []).append(o)
+        for o in ops:
+            if o.layer:
+                waited = {o.wait_flag[k] for k in range(o.n_wait)}
+                for w in ops:
+                    if w.layer == o.layer - 1:
+                        assert w.signal_flag in waited
+    finally:
+        pl.close()
+
+
+def test_packet_schedule_rejections():
+    pl = Planner(4, "bf16")
+    try:
+        pk = B.make_opts(datapath=B.PL_DP_PACKET)
+        for algo in (B.PL_ALGO_DIRECT, B.PL_ALGO_DIRECT_FUSED, B.PL_ALGO_RING):
+            with pytest.raises(B.PurlinError) as e:
+                B.pl_schedule_build_layers(pl.comm, algo, 1024, 3, pk)
+            assert e.value.status == B.PL_ERR_UNSUPPORTED
+        with pytest.raises(B.PurlinError) as e:   # not a layered build
+            B.pl_schedule_build(pl.comm, B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT, 1024, 1024, pk)
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+        with pytest.raises(B.PurlinError) as e:   # 1 MiB per rank: beyond what a CTA's threads can hold
+            B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_ONESHOT, 512 * 1024, 2, pk)
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+        with pytest.raises(B.PurlinError) as e:   # 3 CTAs per rank
+            B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_ONESHOT, 1024, 2, B.make_opts(datapath=B.PL_DP_PACKET, n_ctas=12))
+        assert e.value.status == B.PL_ERR_INVALID_ARG
+        with pytest.raises(B.PurlinError) as e:   # 24 bytes
+            B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_ONESHOT, 12, 2, pk)
+        assert e.value.status == B.PL_ERR_INVALID_ARG
+    finally:
+        pl.close()
+    pu = Planner(4, "u8")
+    try:
+        with pytest.raises(B.PurlinError) as e:
+            B.pl_schedule_build_layers(pu.comm, B.PL_ALGO_ONESHOT, 1024, 2, B.make_opts(datapath=B.PL_DP_PACKET))
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+    finally:
+        pu.close()
+
+
 def test_config1_op_counts_and_bytes():
     # all-reduce, R=4, 262144 fp32 per rank, ring, 64 KiB chunks, unsliced:
     # 3 reduce-scatter hops + 3 all-gather hops, 4 ranks, 4 chunks per partition
