@@ -237,6 +237,10 @@ def probe(b):
     for name, kind, nbytes in (("bulk-copy ring: read", 0, n), ("bulk-copy ring: write", 1, n), ("bulk-copy ring: copy", 2, 2 * n)):
         us, _, _ = _time(lambda: B.pl_probe_hbm(kind, a.data_ptr(), c.data_ptr(), n, 0, h), 20)
         b.emit({"cfg": "probe", "what": name, "gbs": nbytes / us / 1e3})
+    # one read to eight writes (the mix of the all-gather and of the MoE dispatch): 128 MiB in, 1 GiB out
+    m = n // 8
+    us, _, _ = _time(lambda: B.pl_probe_hbm(3, a.data_ptr(), c.data_ptr(), m, 0, h), 20)
+    b.emit({"cfg": "probe", "what": "bulk-copy ring: 1 read : 8 writes", "gbs": 9 * m / us / 1e3})
 
 
 def main(args=None):

@@ -49,7 +49,8 @@ struct MoeGeo {
   long long* ecounts;  // [R][E]
   int32_t* pos;        // [R][T][K] row in the destination's receive buffer, -1 if dropped
   int32_t* prank;      // [R][T][K] destination rank
-  int* flags;          // [0] overflow, [1] invalid expert id, [2] copy engine wait gave up
+  int* flags;          // [0] overflow, [1] invalid expert id, [2] copy engine wait gave up, [3] grid barrier gave up (sticky)
+  unsigned int* sync;  // fused bookkeeping: [0] CTAs that reached the grid barrier, [1] CTAs that left the kernel
   const int32_t* slotmask;  // optional [R][T][K]: written into the metadata instead of the slot index
   int gates_are_logits;     // combine: the gate input holds the K selected logits; softmax them first
 };
@@ -151,6 +152,179 @@ __global__ void __launch_bounds__(kTB) moe_place_kernel(const __grid_constant__ 
   }
 }
 
+
+// ---- fused bookkeeping: count -> (grid barrier) -> offsets -> place in ONE launch ------------
+// Grid (NB, R), all CTAs co-resident (checked on the host).  Phase 1: the block's expert masks
+// stay in shared memory and its per-expert counts go to global memory.  After a grid-wide
+// barrier every CTA reads all R * NB * E counts (128 KiB at the C4 shape, from L2), derives the
+// per-source totals, the segment bases of its own source rank and its own block offsets, and
+// places its tokens.  The barrier is an arrival counter with a bounded wait; the last CTA to
+// leave the kernel clears it, so nothing has to be reset between dispatches (or graph replays).
+__global__ void __launch_bounds__(kTB) moe_plan_kernel(const __grid_constant__ DispatchPtrs P, const __grid_constant__ MoeGeo g) {
+  extern __shared__ __align__(16) uint32_t mask[];
+  int32_t* s_base = reinterpret_cast<int32_t*>(mask + (size_t)g.E * kMaskWords);  // [E]
+  int32_t* s_ecnt = s_base + g.E;                                                 // [R][E] totals per (source, expert)
+  int32_t* s_cnt = s_ecnt + (size_t)g.R * g.E;                                    // [R][R] rows source -> destination
+  __shared__ int s_bad, s_giveup;
+  const int b = blockIdx.x, p = blockIdx.y, tid = threadIdx.x, t = b * kTB + tid;
+  const int32_t* idx = P.idx[p];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (tid == 0) { s_bad = 0; s_giveup = 0; }
+  // ---- phase 1: masks and counts of this block
+  for (int i = tid; i < g.E * kMaskWords; i += kTB) mask[i] = 0u;
+  __syncthreads();
+  if (t < g.T)
+    for (int j0 = 0; j0 < g.K; j0 += 8) {
+      int ev[8];  // eight slots at a time: the loads are independent of one another
+#pragma unroll
+      for (int k = 0; k < 8; ++k) ev[k] = (j0 + k < g.K) ? __ldg(&idx[(size_t)t * g.K + j0 + k]) : -1;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int e = ev[k];
+        if (e < 0) continue;  // empty slot (deduplicated routing pads with -1)
+        if (e < g.E) atomicOr(&mask[e * kMaskWords + (tid >> 5)], 1u << (tid & 31));
+        else s_bad = 1;
+      }
+    }
+  __syncthreads();
+  for (int e = tid; e < g.E; e += kTB) {
+    int c = 0;
+#pragma unroll
+    for (int w = 0; w < kMaskWords; ++w) c += __popc(mask[e * kMaskWords + w]);
+    g.blockcnt[((size_t)p * g.NB + b) * g.E + e] = c;
+  }
+  if (b == 0 && p == 0 && tid < 3) g.flags[tid] = 0;  // ordered before every later flag write by the barrier
+  // ---- grid barrier
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned int n_ctas = gridDim.x * gridDim.y;
+    __threadfence();
+    atomicAdd(g.sync, 1u);
+    unsigned int seen;
+    unsigned long long t0 = 0;
+    uint32_t spins = 0;
+    for (;;) {
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(g.sync) : "memory");
+      if (seen >= n_ctas) break;
+      if ((++spins & 63u) == 0) {
+        unsigned long long now;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
+        if (t0 == 0) t0 = now;
+        if (now - t0 > 2000000000ull) { s_giveup = 1; g.flags[3] = 1; break; }
+      }
+    }
+  }
+  __syncthreads();
+  if (!s_giveup) {
+    // ---- phase 2: totals per (source, expert); this block's offset inside its source's run.
+    // Loads go out eight blocks at a time (independent, so one L2 latency per batch).
+    if ((g.E & 3) == 0) {
+      const int E4 = g.E >> 2;
+      for (int i = tid; i < g.R * E4; i += kTB) {
+        const int q = i / E4, e = (i - q * E4) << 2;
+        int4 total = make_int4(0, 0, 0, 0), before = total;
+        for (int b0 = 0; b0 < g.NB; b0 += 8) {
+          int4 v[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            v[k] = (b0 + k < g.NB) ? __ldcg(reinterpret_cast<const int4*>(&g.blockcnt[((size_t)q * g.NB + b0 + k) * g.E + e]))
+                                   : make_int4(0, 0, 0, 0);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            if (b0 + k == b) before = total;
+            total.x += v[k].x; total.y += v[k].y; total.z += v[k].z; total.w += v[k].w;
+          }
+        }
+        *reinterpret_cast<int4*>(&s_ecnt[q * g.E + e]) = total;
+        if (q == p) *reinterpret_cast<int4*>(&s_base[e]) = before;
+      }
+    } else {
+      for (int i = tid; i < g.R * g.E; i += kTB) {
+        const int q = i / g.E, e = i - q * g.E;
+        int total = 0, before = 0;
+        for (int b0 = 0; b0 < g.NB; b0 += 8) {
+          int v[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) v[k] = (b0 + k < g.NB) ? __ldcg(&g.blockcnt[((size_t)q * g.NB + b0 + k) * g.E + e]) : 0;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            if (b0 + k == b) before = total;
+            total += v[k];
+          }
+        }
+        s_ecnt[i] = total;
+        if (q == p) s_base[e] = before;
+      }
+    }
+    __syncthreads();
+    for (int i = tid; i < g.R * g.R; i += kTB) {
+      const int q = i / g.R, r = i - q * g.R;
+      int c = 0;
+      for (int e = r * g.epr; e < (r + 1) * g.epr; ++e) c += s_ecnt[q * g.E + e];
+      s_cnt[i] = c;
+    }
+    __syncthreads();
+    // first row of expert e's run in the receive buffer of its rank: what sources q < p send
+    // there, then this source's rows for the rank's earlier experts, then the earlier blocks
+    for (int e = tid; e < g.E; e += kTB) {
+      const int r = e / g.epr;
+      long long off = s_base[e];
+      for (int q = 0; q < p; ++q) off += s_cnt[q * g.R + r];
+      for (int e2 = r * g.epr; e2 < e; ++e2) off += s_ecnt[p * g.E + e2];
+      s_base[e] = (int32_t)off;
+      if (b == 0) g.ecounts[p * g.E + e] = s_ecnt[p * g.E + e];
+    }
+    if (b == 0 && tid < g.R) g.counts[p * g.R + tid] = s_cnt[p * g.R + tid];
+    if (b == 0 && p == 0 && tid < g.R) {  // capacity check, once
+      long long total = 0;
+      for (int q = 0; q < g.R; ++q) total += s_cnt[q * g.R + tid];
+      if ((unsigned long long)total > g.cap) g.flags[0] = 1;
+    }
+    if (tid == 0 && s_bad) g.flags[1] = 1;
+    __syncthreads();
+    // ---- phase 3: place this block's tokens
+    if (t < g.T) {
+      const int w = tid >> 5;
+      const uint32_t below = (1u << (tid & 31)) - 1u;
+      for (int j0 = 0; j0 < g.K; j0 += 8) {
+        int ev[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) ev[k] = (j0 + k < g.K) ? __ldg(&idx[(size_t)t * g.K + j0 + k]) : -1;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int j = j0 + k;
+          if (j >= g.K) break;
+          const int e = ev[k];
+          const size_t o = ((size_t)p * g.T + t) * g.K + j;
+          if ((unsigned)e >= (unsigned)g.E) { g.pos[o] = -1; g.prank[o] = 0; continue; }
+          int rank = __popc(mask[e * kMaskWords + w] & below);
+          for (int w2 = 0; w2 < w; ++w2) rank += __popc(mask[e * kMaskWords + w2]);
+          const long long row = (long long)s_base[e] + rank;
+          const int r = e / g.epr;
+          g.prank[o] = r;
+          if ((unsigned long long)row < g.cap) {
+            g.pos[o] = (int32_t)row;
+            if (P.meta[r]) reinterpret_cast<int4*>(P.meta[r])[row] = make_int4(p, t, g.slotmask ? g.slotmask[o] : j, e);
+          } else {
+            g.pos[o] = -1;
+          }
+        }
+      }
+    }
+  }
+  // ---- the last CTA to leave clears the barrier words for the next dispatch
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned int n_ctas = gridDim.x * gridDim.y;
+    __threadfence();
+    if (atomicAdd(g.sync + 1, 1u) == n_ctas - 1u) {
+      g.sync[0] = 0u;
+      g.sync[1] = 0u;
+      __threadfence();
+    }
+  }
+}
+
 // Deduplicated routing: for every token the distinct destination ranks in ascending order
 // (padded with -1) and, per destination, the mask of slots whose expert lives there.
 __global__ void __launch_bounds__(256) moe_derive_ranks_kernel(const __grid_constant__ DispatchPtrs P, int R, int T, int K,
@@ -198,6 +372,9 @@ __global__ void __launch_bounds__(32) moe_move_kernel(const __grid_constant__ Di
     ptx::mbar_init_fence();
   }
   __syncwarp();
+  // launched with programmatic stream serialization: set up above while the bookkeeping kernel
+  // drains, wait here for it to complete before anything it wrote (pos, prank) is read
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const unsigned long long n_items = (unsigned long long)g.R * g.T * g.n_tiles;
   const unsigned long long c = blockIdx.x, G = gridDim.x;
   if (c >= n_items) return;
@@ -361,13 +538,19 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // smaller plan cannot lower it under the feet of the first.
 constexpr int kMaxExperts = 4096;
 constexpr size_t kMoveSmemMax = 128 + 8 * (size_t)kMaxTile;
+constexpr size_t kPlanSmemMax = 200 * 1024;  // the fused bookkeeping kernel is used while its tables fit this
+
+size_t plan_smem_bytes(const MoeGeo& g) {
+  return ((size_t)g.E * kMaskWords + (size_t)g.E + (size_t)g.R * g.E + (size_t)g.R * g.R) * 4;
+}
 bool configure_kernels(int device) {
   static std::atomic<unsigned long long> configured{0};
   const unsigned long long bit = 1ull << (device & 63);
   if (configured.load(std::memory_order_acquire) & bit) return true;
   if (cudaFuncSetAttribute(moe_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMoveSmemMax) != cudaSuccess ||
       cudaFuncSetAttribute(moe_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxExperts * kMaskWords * 4) != cudaSuccess ||
-      cudaFuncSetAttribute(moe_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxExperts * kMaskWords * 4 + kMaxExperts * 4) != cudaSuccess) {
+      cudaFuncSetAttribute(moe_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxExperts * kMaskWords * 4 + kMaxExperts * 4) != cudaSuccess ||
+      cudaFuncSetAttribute(moe_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPlanSmemMax) != cudaSuccess) {
     cudaGetLastError();
     return false;
   }
@@ -385,6 +568,7 @@ struct pl_moe_plan_s {
   int sm_count = 148;
   int combine_per_sm = 4;  // resident CTAs of the combine kernel per SM (occupancy query at plan creation)
   size_t move_smem = 0;
+  bool fused = false, fused_dedup = false;  // bookkeeping in one launch (grid co-resident, tables fit shared memory)
   bool dispatched = false;
   // deduplicated variant: the same machinery run over "one expert per rank" routing
   MoeGeo gd{};
@@ -444,7 +628,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   const size_t o_bc = place((size_t)R * g.NB * g.E * 4);
   const size_t o_cnt = place((size_t)R * R * 8), o_ecnt = place((size_t)R * g.E * 8);
   const size_t o_pos = place((size_t)R * g.T * g.K * 4), o_prank = place((size_t)R * g.T * g.K * 4);
-  const size_t o_flags = place(16);
+  const size_t o_flags = place(32);  // 4 flag words + 2 barrier words
   pl->blob_bytes = off;
   if (cudaMalloc(&pl->d_blob, off) != cudaSuccess) { cudaGetLastError(); delete pl; return PL_ERR_OOM; }
   if (cudaMemset(pl->d_blob, 0, off) != cudaSuccess) { cudaGetLastError(); cudaFree(pl->d_blob); delete pl; return PL_ERR_CUDA; }
@@ -454,6 +638,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   g.pos = reinterpret_cast<int32_t*>(pl->d_blob + o_pos);
   g.prank = reinterpret_cast<int32_t*>(pl->d_blob + o_prank);
   g.flags = reinterpret_cast<int*>(pl->d_blob + o_flags);
+  g.sync = reinterpret_cast<unsigned int*>(pl->d_blob + o_flags + 16);
   if (!configure_kernels(comm->device)) {
     cudaFree(pl->d_blob);
     delete pl;
@@ -473,7 +658,7 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
     const size_t q_bc = place2((size_t)R * g.NB * R * 4);
     const size_t q_cnt = place2((size_t)R * R * 8), q_ecnt = place2((size_t)R * R * 8);
     const size_t q_pos = place2(tk * 4), q_prank = place2(tk * 4), q_ridx = place2(tk * 4), q_rmask = place2(tk * 4);
-    const size_t q_ones = place2((size_t)g.T * d.K * 4), q_flags = place2(16);
+    const size_t q_ones = place2((size_t)g.T * d.K * 4), q_flags = place2(32);
     if (cudaMalloc(&pl->d_blob2, off2) != cudaSuccess) { cudaGetLastError(); cudaFree(pl->d_blob); delete pl; return PL_ERR_OOM; }
     std::vector<float> ones((size_t)g.T * d.K, 1.0f);
     if (cudaMemset(pl->d_blob2, 0, off2) != cudaSuccess ||
@@ -490,10 +675,26 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
     d.pos = reinterpret_cast<int32_t*>(pl->d_blob2 + q_pos);
     d.prank = reinterpret_cast<int32_t*>(pl->d_blob2 + q_prank);
     d.flags = reinterpret_cast<int*>(pl->d_blob2 + q_flags);
+    d.sync = reinterpret_cast<unsigned int*>(pl->d_blob2 + q_flags + 16);
     pl->d_ridx = reinterpret_cast<int32_t*>(pl->d_blob2 + q_ridx);
     pl->d_rmask = reinterpret_cast<int32_t*>(pl->d_blob2 + q_rmask);
     pl->d_ones = reinterpret_cast<float*>(pl->d_blob2 + q_ones);
     d.slotmask = pl->d_rmask;
+  }
+  {
+    // one-launch bookkeeping needs every CTA of its grid resident at once (they meet at a barrier)
+    auto feasible = [&](const MoeGeo& q) {
+      const size_t smem = plan_smem_bytes(q);
+      if (smem > kPlanSmemMax) return false;
+      int per_sm = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, moe_plan_kernel, kTB, smem) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+      }
+      return (long long)q.NB * q.R <= (long long)per_sm * comm->sm_count;
+    };
+    pl->fused = feasible(pl->g);
+    pl->fused_dedup = feasible(pl->gd);
   }
   comm->n_plans += 1;
   *out = pl;
@@ -507,6 +708,39 @@ pl_status_t pl_moe_plan_destroy(pl_moe_plan_t plan) {
   plan->comm->n_plans -= 1;
   delete plan;
   return PL_OK;
+}
+
+// count / scan / place (or the fused kernel), then the row mover launched so that its set-up
+// overlaps the tail of the bookkeeping.  Returns the number of kernels launched, 0 on error.
+static int launch_dispatch(pl_moe_plan_t plan, const DispatchPtrs& P, const MoeGeo& g, bool fused, cudaStream_t cs) {
+  int launched = 0;
+  const size_t mask_smem = (size_t)g.E * kMaskWords * 4;
+  dim3 grid(g.NB, g.R);
+  if (fused) {
+    moe_plan_kernel<<<grid, kTB, plan_smem_bytes(g), cs>>>(P, g);
+    launched = 1;
+  } else {
+    moe_count_kernel<<<grid, kTB, mask_smem, cs>>>(P, g);
+    moe_scan_kernel<<<g.R, 256, 0, cs>>>(g);
+    moe_place_kernel<<<grid, kTB, mask_smem + (size_t)g.E * 4, cs>>>(P, g);
+    launched = 3;
+  }
+  if (cudaGetLastError() != cudaSuccess) return 0;
+  const unsigned long long items = (unsigned long long)g.R * g.T * g.n_tiles;
+  const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, (200 * 1024) / plan->move_smem));
+  const int mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)plan->sm_count * per_sm);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)mgrid);
+  cfg.blockDim = dim3(32);
+  cfg.dynamicSmemBytes = plan->move_smem;
+  cfg.stream = cs;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = fused ? 1 : 0;  // only the fused kernel releases its dependents early
+  if (cudaLaunchKernelEx(&cfg, moe_move_kernel, P, g) != cudaSuccess) { cudaGetLastError(); return 0; }
+  return launched + 1;
 }
 
 pl_status_t pl_moe_dispatch(pl_moe_plan_t plan, const void* const* x, const int32_t* const* topk_idx,
@@ -525,18 +759,9 @@ pl_status_t pl_moe_dispatch(pl_moe_plan_t plan, const void* const* x, const int3
     P.recv[r] = recv[r];
     P.meta[r] = recv_meta ? recv_meta[r] : nullptr;
   }
-  cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  const size_t mask_smem = (size_t)g.E * kMaskWords * 4;
-  dim3 grid(g.NB, g.R);
-  moe_count_kernel<<<grid, kTB, mask_smem, cs>>>(P, g);
-  moe_scan_kernel<<<g.R, 256, 0, cs>>>(g);
-  moe_place_kernel<<<grid, kTB, mask_smem + (size_t)g.E * 4, cs>>>(P, g);
-  const unsigned long long items = (unsigned long long)g.R * g.T * g.n_tiles;
-  const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, (200 * 1024) / plan->move_smem));
-  const int mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)plan->sm_count * per_sm);
-  moe_move_kernel<<<mgrid, 32, plan->move_smem, cs>>>(P, g);
-  if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
-  g_launches.fetch_add(4);
+  const int launched = launch_dispatch(plan, P, g, plan->fused, static_cast<cudaStream_t>(stream));
+  if (!launched) return PL_ERR_CUDA;
+  g_launches.fetch_add(launched);
   plan->dispatched = true;
   return PL_OK;
 }
@@ -581,7 +806,11 @@ pl_status_t pl_moe_plan_read(pl_moe_plan_t plan, int32_t* pos, int64_t* counts, 
   const MoeGeo& g = plan->g;
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
   int flags[4] = {0, 0, 0, 0};
-  bool ok = cudaMemcpy(flags, g.flags, 12, cudaMemcpyDeviceToHost) == cudaSuccess;
+  bool ok = cudaMemcpy(flags, g.flags, 16, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (ok && flags[3]) {  // the grid barrier of the bookkeeping kernel gave up: report once, clear barrier state
+    flags[2] = 1;
+    ok = cudaMemset(g.flags + 3, 0, 4 + 8) == cudaSuccess;  // flags[3] and the two barrier words behind it
+  }
   if (ok && pos) ok = cudaMemcpy(pos, g.pos, (size_t)g.R * g.T * g.K * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
   if (ok && counts) ok = cudaMemcpy(counts, g.counts, (size_t)g.R * g.R * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
   if (ok && expert_counts) ok = cudaMemcpy(expert_counts, g.ecounts, (size_t)g.R * g.E * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
@@ -614,17 +843,10 @@ pl_status_t pl_moe_dispatch_dedup(pl_moe_plan_t plan, const void* const* x, cons
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   const long long n_tok = (long long)g.R * g.T;
   moe_derive_ranks_kernel<<<(unsigned)((n_tok + 255) / 256), 256, 0, cs>>>(P0, g.R, g.T, g.K, g.epr, d.K, plan->d_ridx, plan->d_rmask);
-  const size_t mask_smem = (size_t)d.E * kMaskWords * 4;
-  dim3 grid(d.NB, d.R);
-  moe_count_kernel<<<grid, kTB, mask_smem, cs>>>(P, d);
-  moe_scan_kernel<<<d.R, 256, 0, cs>>>(d);
-  moe_place_kernel<<<grid, kTB, mask_smem + (size_t)d.E * 4, cs>>>(P, d);
-  const unsigned long long items = (unsigned long long)d.R * d.T * d.n_tiles;
-  const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, (200 * 1024) / plan->move_smem));
-  const int mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)plan->sm_count * per_sm);
-  moe_move_kernel<<<mgrid, 32, plan->move_smem, cs>>>(P, d);
   if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
-  g_launches.fetch_add(5);
+  const int launched = launch_dispatch(plan, P, d, plan->fused_dedup, cs);
+  if (!launched) return PL_ERR_CUDA;
+  g_launches.fetch_add(1 + launched);
   plan->dispatched_dedup = true;
   return PL_OK;
 }
@@ -657,7 +879,11 @@ pl_status_t pl_moe_plan_read_dedup(pl_moe_plan_t plan, int32_t* pos, int64_t* co
   const MoeGeo& d = plan->gd;
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
   int flags[4] = {0, 0, 0, 0};
-  bool ok = cudaMemcpy(flags, d.flags, 12, cudaMemcpyDeviceToHost) == cudaSuccess;
+  bool ok = cudaMemcpy(flags, d.flags, 16, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (ok && flags[3]) {
+    flags[2] = 1;
+    ok = cudaMemset(d.flags + 3, 0, 4 + 8) == cudaSuccess;
+  }
   if (ok && counts) ok = cudaMemcpy(counts, d.counts, (size_t)d.R * d.R * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
   if (ok && pos) {
     const size_t tk = (size_t)d.R * d.T * d.K;
