@@ -164,32 +164,45 @@ def run_purlin(args):
     assert B.pl_comm_status(comm).code == B.PL_OK
 
     # ---- device-timed region --------------------------------------------------------------
+    # A block is exactly K steps bracketed by a barrier and a device synchronisation on both
+    # sides.  The block is repeated until the timed region lasts at least half a second, so that
+    # the clock record holds more than one sample whatever K is; the median block is reported.
     K = args.steps
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
     sampler = ClockSampler(local)
     launches0 = B.pl_launch_count()
-    replicas.barrier()
-    torch.cuda.synchronize()
+
+    def one_block():
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+        replicas.barrier()
+        torch.cuda.synchronize()
+        for i in range(K):
+            ev[i][0].record()
+            B.pl_execute(rs, b_rs, stream)
+            ev[i][1].record()
+            B.pl_execute(ag, b_ag, stream)
+            ev[i][2].record()
+        torch.cuda.synchronize()
+        replicas.barrier()
+        return (ev[0][0].elapsed_time(ev[K - 1][2]),
+                [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)], [ev[i][1].elapsed_time(ev[i][2]) for i in range(K)])
+
     sampler.start()
-    t_begin = torch.cuda.Event(enable_timing=True)
-    t_end = torch.cuda.Event(enable_timing=True)
-    t_begin.record()
-    for i in range(K):
-        ev[i][0].record()
-        B.pl_execute(rs, b_rs, stream)
-        ev[i][1].record()
-        B.pl_execute(ag, b_ag, stream)
-        ev[i][2].record()
-    t_end.record()
-    torch.cuda.synchronize()
+    block_ms, rs_all, ag_all = [], [], []
+    spent = 0.0
+    while True:
+        ms, r_ms, a_ms = one_block()
+        block_ms.append(replicas.max_over_ranks(ms))   # the job's block time is its slowest replica's
+        rs_all += r_ms
+        ag_all += a_ms
+        spent += block_ms[-1]
+        if (spent >= args.min_timed_ms and len(block_ms) >= 1) or len(block_ms) >= 2000:
+            break
     clocks = sampler.stop()
-    launches = B.pl_launch_count() - launches0
-    total_ms = t_begin.elapsed_time(t_end)
-    rs_ms = np.array([ev[i][0].elapsed_time(ev[i][1]) for i in range(K)])
-    ag_ms = np.array([ev[i][1].elapsed_time(ev[i][2]) for i in range(K)])
+    n_blocks = len(block_ms)
+    launches = (B.pl_launch_count() - launches0) // n_blocks       # kernels launched per timed block of K steps
+    total_ms = float(np.median(block_ms))
+    rs_ms, ag_ms = np.array(rs_all), np.array(ag_all)
     assert B.pl_comm_status(comm).code == B.PL_OK
-    replicas.barrier()
-    total_ms = replicas.max_over_ranks(total_ms)
 
     ms_per_step = total_ms / K
     eff_bytes = irs.message_bytes + iag.message_bytes  # 64 MiB + 64 MiB per step
@@ -257,6 +270,21 @@ def run_purlin(args):
         "datapath": int(irs.datapath), "n_ops_rs": int(irs.n_ops), "n_ops_ag": int(iag.n_ops),
     }
 
+    detail["timed_region"] = {"blocks": n_blocks, "steps_per_block": K, "block_ms_median": total_ms,
+                              "block_ms_min": float(min(block_ms)), "block_ms_max": float(max(block_ms))}
+
+    # ---- the same step with overlapped launches (no events between the two executes) ---------
+    if not args.no_detail:
+        detail["step_overlapped_launches"] = measure_overlapped_step(B, torch, comm, n, chunk, R, b_rs, b_ag, stream, ms_per_step)
+
+    # free the headline buffers before the other configurations allocate theirs
+    del d_in, d_mid, d_out, b_rs, b_ag, pinned_in
+    torch.cuda.empty_cache()
+
+    # ---- every other configuration, measured in this same process -----------------------------
+    if rank == 0 and world == 1 and not args.no_detail:
+        detail["configs"] = measure_all_configs(peak)
+
     # ---- the oracle timed on this machine's host cores (rank 0, N=1 only) -----------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -279,6 +307,116 @@ def run_purlin(args):
     B.pl_schedule_destroy(ag)
     B.pl_comm_destroy(comm)
     replicas.finalize()
+
+
+def measure_overlapped_step(B, torch, comm, n, chunk, R, b_rs, b_ag, stream, plain_ms):
+    """The C2 step built with PL_OPT_OVERLAP_LAUNCH (the CTAs of a launch are set up while the one
+    in front of it drains) and timed without events between the two launches."""
+    opts = B.make_opts(flags=B.PL_OPT_OVERLAP_LAUNCH)
+    rs = B.pl_schedule_build(comm, B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, chunk, opts)
+    ag = B.pl_schedule_build(comm, B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, chunk, opts)
+    for _ in range(5):
+        B.pl_execute(rs, b_rs, stream)
+        B.pl_execute(ag, b_ag, stream)
+    torch.cuda.synchronize()
+    reps = 300
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        B.pl_execute(rs, b_rs, stream)
+        B.pl_execute(ag, b_ag, stream)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    B.pl_schedule_destroy(rs)
+    B.pl_schedule_destroy(ag)
+    return {"ms_per_step": ms, "steps": reps, "vs_plain_step": ms / plain_ms}
+
+
+def measure_all_configs(peak):
+    """C1, C3 (three sizes x five algorithms), C4 (both routings), C5 (three sizes, both latency
+    protocols) and the stream ceilings of the bulk-copy ring, each timed with CUDA events in this
+    process.  Every entry carries its algorithmic bytes (pl_schedule_info), the fraction of the
+    measured copy peak and of 8 TB/s, and the fraction of the matching stream ceiling."""
+    import bench_suite as S
+    from paper_2609_36954_b200 import binding as B
+    b = S.Bench(quiet=True)
+    streams = S.probe(b)
+    ceil = {"read": streams["bulk-copy ring: read"], "write": streams["bulk-copy ring: write"],
+            "copy": streams["bulk-copy ring: copy"], "mix_1r_8w": streams["bulk-copy ring: 1 read : 8 writes"]}
+    out = {"stream_ceilings_gbs": {k: round(v, 1) for k, v in streams.items()}}
+
+    def which_ceiling(read_b, write_b):
+        share = read_b / max(1, read_b + write_b)
+        return "read" if share >= 0.8 else "mix_1r_8w" if share <= 0.2 else "copy"
+
+    def entry(rec, note=None):
+        if rec is None or "error" in rec:
+            return {"error": (rec or {}).get("error", "not built")}
+        alg = rec["bytes_read"] + rec["bytes_written"]
+        comp = rec["compulsory_bytes"]
+        us = rec["us"] * max(1, rec["layers"])
+        gbs = comp / us / 1e3
+        c = which_ceiling(comp - rec["bytes_written"], rec["bytes_written"])
+        e = {"us": round(rec["us"], 3), "us_p10": round(rec["us_p10"], 3), "us_p90": round(rec["us_p90"], 3),
+             "message_bytes": rec["message_bytes"], "algorithmic_bytes": alg, "hbm_bytes": comp,
+             "algbw_gbs": round(rec["eff_gbs"], 1), "hbm_gbs": round(gbs, 1),
+             "frac_measured": round(gbs / peak, 4), "frac_8TBps": round(gbs / NOMINAL_HBM_GBS, 4),
+             "ceiling": c, "frac_of_ceiling": round(gbs / ceil[c], 4),
+             "grid": rec["grid"], "threads": rec["threads"], "datapath": rec["datapath"], "status": rec["status"]}
+        if rec.get("us_graph128") is not None:
+            e["us_in_128_call_graph"] = round(rec["us_graph128"], 3)
+        if note:
+            e["note"] = note
+        return e
+
+    l2 = "working set sits in L2: the HBM fractions do not apply"
+    # C1: all-reduce, R = 4, 1 MiB per rank, ring, 64 KiB chunks
+    out["C1"] = {name: entry(b.collective("C1", 4, dt, B.PL_ALLREDUCE, "ring", 262144, 65536, iters=50, graph=True), l2)
+                 for name, dt in (("f32", B.PL_F32), ("i32", B.PL_I32))}
+    # C3: all-reduce sweep points
+    out["C3"] = {}
+    for label, size, graph, iters in (("64KiB", 64 << 10, True, 30), ("16MiB", 16 << 20, False, 20), ("256MiB", 256 << 20, False, 8)):
+        out["C3"][label] = {}
+        for algo in ("ring", "tree", "oneshot", "direct", "fused"):
+            chunk = max(16, min(MIB, size if algo in ("oneshot", "tree") else size // 8))
+            rec = b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=iters, graph=graph)
+            out["C3"][label][algo] = entry(rec, l2 if size < (32 << 20) else None)
+    # all-to-all and the stand-alone C2 collectives (no neighbour launch dirtying L2)
+    out["C2_alone"] = {
+        "reduce_scatter": entry(b.collective("C2-RS", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "direct", 32 * MIB, MIB)),
+        "all_gather": entry(b.collective("C2-AG", 8, B.PL_BF16, B.PL_ALLGATHER, "direct", 4 * MIB, MIB)),
+        "reduce_scatter_ring": entry(b.collective("C2-RS", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "ring", 32 * MIB, 256 << 10)),
+        "all_gather_ring": entry(b.collective("C2-AG", 8, B.PL_BF16, B.PL_ALLGATHER, "ring", 4 * MIB, 256 << 10)),
+        "all_to_all": entry(b.collective("A2A", 8, B.PL_BF16, B.PL_ALLTOALL, "direct", 32 * MIB, MIB)),
+    }
+    # C4: MoE dispatch / combine at the full shape, both routings
+    out["C4"] = {}
+    for name, ident in (("permuted", False), ("identity", True)):
+        r = b.moe("C4", identity=ident, dedup=False)
+        out["C4"][name] = {
+            "dispatch_us": round(r["dispatch_us"], 1), "combine_us": round(r["combine_us"], 1),
+            "algorithmic_bytes_each": r["dispatch_bytes"], "rows": r["rows"], "max_over_mean_rows": round(r["max_over_mean_rows"], 2),
+            "dispatch_hbm_gbs": round(r["dispatch_gbs"], 1), "combine_hbm_gbs": round(r["combine_gbs"], 1),
+            "dispatch_frac_measured": round(r["dispatch_frac_measured"], 4), "combine_frac_measured": round(r["combine_frac_measured"], 4),
+            "dispatch_frac_8TBps": round(r["dispatch_gbs"] / NOMINAL_HBM_GBS, 4), "combine_frac_8TBps": round(r["combine_gbs"] / NOMINAL_HBM_GBS, 4),
+            "dispatch_frac_of_ceiling": round(r["dispatch_gbs"] / ceil["mix_1r_8w"], 4), "dispatch_ceiling": "mix_1r_8w",
+            "combine_frac_of_ceiling": round(r["combine_gbs"] / ceil["read"], 4), "combine_ceiling": "read", "status": r["status"]}
+    # C5: 80 layers per launch; per layer.  Flags (register executor) at the three benchmark sizes,
+    # then the two latency protocols side by side at 4 / 16 / 64 KiB.
+    out["C5"] = {}
+    for label, count in (("16KiB", 8192), ("128KiB", 65536), ("1MiB", 524288)):
+        out["C5"][label] = {algo: entry(b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, count, 0, iters=100, layers=80), l2)
+                            for algo in ("oneshot", "fused")}
+    out["C5_protocols"] = {}
+    for kib in (4, 16, 64):
+        flags = [b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, kib * 512, 0, iters=200, layers=80) for algo in ("oneshot", "fused")]
+        best = min(flags, key=lambda r: r["us"])
+        pk = b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, "oneshot", kib * 512, 0, iters=200, layers=80, datapath=B.PL_DP_PACKET)
+        out["C5_protocols"]["%dKiB" % kib] = {
+            "flags": {"algo": best["algo"], "p50_us": round(best["us"], 3), "p10_us": round(best["us_p10"], 3), "p90_us": round(best["us_p90"], 3), "grid": best["grid"]},
+            "packets": {"algo": "oneshot", "p50_us": round(pk["us"], 3), "p10_us": round(pk["us_p10"], 3), "p90_us": round(pk["us_p90"], 3), "grid": pk["grid"]}}
+    return out
 
 
 def measure_small_allreduce(B, torch, stream, R=8, hidden=8192, layers=80, steps=200):
@@ -447,7 +585,7 @@ def run_cpu_suite(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="purlin", choices=["purlin", "reference"])
     ap.add_argument("--suite", action="store_true", help="run every configuration (bench_suite.py)")
@@ -455,6 +593,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-latency", action="store_true")
+    ap.add_argument("--no-detail", action="store_true", help="skip the other configurations (C1, C3, C4, C5, stream ceilings)")
+    ap.add_argument("--min-timed-ms", type=float, default=500.0, help="repeat the K-step block until the timed region lasts this long")
     ap.add_argument("--fast-inputs", action="store_true", help="tile 4 Mi generated elements instead of generating all")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--n-ctas", type=int, default=0)
@@ -465,7 +605,29 @@ def main():
     ap.add_argument("--stage-bytes", type=int, default=0)
     ap.add_argument("--ncu-traffic", type=float, default=NCU_RS_TRAFFIC_BYTES,
                     help="dram bytes per reduce-scatter launch from the committed ncu capture")
+    ap.add_argument("--replica-selftest", action="store_true",
+                    help="only join the process group (gloo), take a barrier and a max over ranks, print one line: "
+                         "checks the multi-process plumbing without a GPU")
     args = ap.parse_args()
+    # --gpus N: N independent replicas, one process per GPU.  Under a launcher (torchrun) the
+    # environment describes the group and must agree with --gpus; without one, this process starts
+    # the N replicas itself.
+    env_world = os.environ.get("WORLD_SIZE")
+    if env_world is not None and int(env_world) != args.gpus and args.impl != "reference":
+        raise SystemExit(f"bench.py: --gpus {args.gpus} disagrees with WORLD_SIZE={env_world} of the launcher")
+    if env_world is None and args.gpus > 1 and args.impl != "reference" and not args.cpu_suite and not args.suite:
+        from paper_2609_36954_b200 import replicas
+        raise SystemExit(replicas.launch_local(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:]))
+    if args.replica_selftest:
+        from paper_2609_36954_b200 import replicas
+        n, rank, _ = replicas.init("gloo")
+        replicas.barrier()
+        slow = replicas.max_over_ranks(1.0 + rank)
+        replicas.barrier()
+        if rank == 0:
+            print(json.dumps({"selftest": True, "n_gpus": n, "max_over_ranks": slow}))
+        replicas.finalize()
+        return
     if args.impl == "reference":
         run_reference(args)
     elif args.cpu_suite:

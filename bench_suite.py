@@ -86,13 +86,18 @@ def _time_graph(launch, calls=128, replays=8):
 
 
 class Bench:
-    def __init__(self, out_path=None, opts_kw=None):
+    def __init__(self, out_path=None, opts_kw=None, quiet=False):
         self.peak = _peak()
         self.out = open(out_path, "w") if out_path else None
         self.stream = torch.cuda.current_stream().cuda_stream
         self.opts_kw = opts_kw or {}
+        self.quiet = quiet       # collect the records instead of printing them (bench.py's detail section)
+        self.records = []
 
     def emit(self, rec):
+        self.records.append(rec)
+        if self.quiet:
+            return
         line = json.dumps(rec)
         print(line, flush=True)
         if self.out:
@@ -139,7 +144,11 @@ class Bench:
                          "p90_us": float(np.percentile(gaps, 90))}
         nl = max(1, layers)
         sched_bytes = info.bytes_read + info.bytes_written
-        rec = {"cfg": cfg, "coll": int(coll), "algo": algo, "R": R, "dtype": int(dtype),
+        # bytes that must cross the HBM interface when nothing is cached between launches: every
+        # input byte once, every output byte once (an all-gather re-reads its sources from L2)
+        compulsory = sum(int(info.in_bytes[r]) for r in range(R)) + int(info.bytes_written)
+        rec = {"cfg": cfg, "bytes_read": int(info.bytes_read), "bytes_written": int(info.bytes_written),
+               "compulsory_bytes": int(min(compulsory, sched_bytes)), "coll": int(coll), "algo": algo, "R": R, "dtype": int(dtype),
                "message_bytes": int(info.message_bytes), "chunk": int(min(chunk, 1 << 40)), "layers": layers,
                "us": p50 / nl, "us_p10": p10 / nl, "us_p90": p90 / nl, "us_graph128": graph_us, "layer_us_in_kernel": in_kernel,
                "eff_gbs": info.message_bytes * nl / p50 / 1e3, "sched_gbs": sched_bytes / p50 / 1e3,
@@ -172,7 +181,7 @@ class Bench:
         B.pl_schedule_destroy(s)
         B.pl_comm_destroy(comm)
 
-    def moe(self, cfg, R=8, T=4096, H=7168, E=256, K=8, identity=False, iters=10):
+    def moe(self, cfg, R=8, T=4096, H=7168, E=256, K=8, identity=False, iters=10, dedup=True):
         idx, gates = gen.moe_routing(R, T, E, K, identity_perm=identity)
         counts = np.zeros((R, R), np.int64)
         for p in range(R):
@@ -195,33 +204,38 @@ class Bench:
         disp, _, _ = _time(lambda: B.pl_moe_dispatch(plan, px, pi, pr, pm, self.stream), iters, per_call_events=True)
         comb, _, _ = _time(lambda: B.pl_moe_combine(plan, pr, pg, po, self.stream), iters, per_call_events=True)
         st = B.pl_moe_plan_read(plan, 0, 0, 0, self.stream)
-        # deduplicated variant on the same plan: one row per (token, destination rank)
-        dd, _, _ = _time(lambda: B.pl_moe_dispatch_dedup(plan, px, pi, pr, pm, self.stream), iters, per_call_events=True)
-        dc, _, _ = _time(lambda: B.pl_moe_combine_dedup(plan, pr, po, self.stream), iters, per_call_events=True)
-        cnt = np.zeros((R, R), np.int64)
-        B.pl_moe_plan_read_dedup(plan, 0, cnt.ctypes.data, self.stream)
-        rows_dd = int(cnt.sum())
         rows = R * T * K
         row_b = H * 2
         d_bytes = R * T * row_b + rows * row_b
         c_bytes = rows * row_b + R * T * row_b
-        self.emit({"cfg": cfg, "routing": "identity" if identity else "permuted", "rows": rows, "cap": cap,
-                   "max_over_mean_rows": float(counts.sum(axis=0).max() / counts.sum(axis=0).mean()),
-                   "dispatch_us": disp, "combine_us": comb,
-                   "dispatch_gbs": d_bytes / disp / 1e3, "combine_gbs": c_bytes / comb / 1e3,
-                   "dispatch_frac_measured": d_bytes / disp / 1e3 / self.peak,
-                   "combine_frac_measured": c_bytes / comb / 1e3 / self.peak, "status": int(st),
-                   "dedup_rows": rows_dd, "dedup_dispatch_us": dd, "dedup_combine_us": dc,
-                   "dedup_dispatch_gbs": (R * T + rows_dd) * H * 2 / dd / 1e3,
-                   "dedup_combine_gbs": (R * T + rows_dd) * H * 2 / dc / 1e3})
+        rec = {"cfg": cfg, "routing": "identity" if identity else "permuted", "rows": rows, "cap": cap,
+               "max_over_mean_rows": float(counts.sum(axis=0).max() / counts.sum(axis=0).mean()),
+               "dispatch_us": disp, "combine_us": comb, "dispatch_bytes": d_bytes, "combine_bytes": c_bytes,
+               "dispatch_gbs": d_bytes / disp / 1e3, "combine_gbs": c_bytes / comb / 1e3,
+               "dispatch_frac_measured": d_bytes / disp / 1e3 / self.peak,
+               "combine_frac_measured": c_bytes / comb / 1e3 / self.peak, "status": int(st)}
+        if dedup:
+            # deduplicated variant on the same plan: one row per (token, destination rank)
+            dd, _, _ = _time(lambda: B.pl_moe_dispatch_dedup(plan, px, pi, pr, pm, self.stream), iters, per_call_events=True)
+            dc, _, _ = _time(lambda: B.pl_moe_combine_dedup(plan, pr, po, self.stream), iters, per_call_events=True)
+            cnt = np.zeros((R, R), np.int64)
+            B.pl_moe_plan_read_dedup(plan, 0, cnt.ctypes.data, self.stream)
+            rows_dd = int(cnt.sum())
+            rec.update({"dedup_rows": rows_dd, "dedup_dispatch_us": dd, "dedup_combine_us": dc,
+                        "dedup_dispatch_gbs": (R * T + rows_dd) * H * 2 / dd / 1e3,
+                        "dedup_combine_gbs": (R * T + rows_dd) * H * 2 / dc / 1e3})
+        self.emit(rec)
         B.pl_moe_plan_destroy(plan)
         B.pl_comm_destroy(comm)
+        return rec
 
 
 def probe(b):
     """Reference points from library kernels on the same GPU (context for the roofline
-    fractions, not part of the product path): plain copy, fill and read over 1 GiB."""
+    fractions, not part of the product path): plain copy, fill and read over 1 GiB.  Returns
+    {stream name: GB/s}."""
     n = 1 << 30
+    found = {}
     a = torch.empty(n, dtype=torch.uint8, device="cuda")
     c = torch.empty(n, dtype=torch.uint8, device="cuda")
     a.zero_()
@@ -232,15 +246,19 @@ def probe(b):
                              ("torch sum fp32 (read)", lambda: af.sum(), n)):
         us, _, _ = _time(fn, 20)
         b.emit({"cfg": "probe", "what": name, "gbs": nbytes / us / 1e3})
+        found[name] = nbytes / us / 1e3
     # the same three streams through the library's own bulk-copy ring (pl_probe_hbm)
     h = torch.cuda.current_stream().cuda_stream
     for name, kind, nbytes in (("bulk-copy ring: read", 0, n), ("bulk-copy ring: write", 1, n), ("bulk-copy ring: copy", 2, 2 * n)):
         us, _, _ = _time(lambda: B.pl_probe_hbm(kind, a.data_ptr(), c.data_ptr(), n, 0, h), 20)
         b.emit({"cfg": "probe", "what": name, "gbs": nbytes / us / 1e3})
+        found[name] = nbytes / us / 1e3
     # one read to eight writes (the mix of the all-gather and of the MoE dispatch): 128 MiB in, 1 GiB out
     m = n // 8
     us, _, _ = _time(lambda: B.pl_probe_hbm(3, a.data_ptr(), c.data_ptr(), m, 0, h), 20)
     b.emit({"cfg": "probe", "what": "bulk-copy ring: 1 read : 8 writes", "gbs": 9 * m / us / 1e3})
+    found["bulk-copy ring: 1 read : 8 writes"] = 9 * m / us / 1e3
+    return found
 
 
 def main(args=None):

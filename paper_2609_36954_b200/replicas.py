@@ -57,3 +57,28 @@ def aggregate_throughput(units_per_replica: float, ms_per_step: float, n_replica
 def finalize():
     if dist.is_initialized():
         dist.destroy_process_group()
+
+
+def launch_local(n: int, argv: list, timeout_s: float = 3600.0) -> int:
+    """Start n replica processes of `argv` on this node, one per GPU index, with the environment a
+    launcher would give them (RANK / LOCAL_RANK / WORLD_SIZE / MASTER_ADDR / MASTER_PORT on
+    127.0.0.1).  Rank 0 inherits stdout; returns the first non-zero exit code, else 0."""
+    import socket
+    import subprocess
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), WORLD_SIZE=str(n), RANK=str(rank),
+                   LOCAL_RANK=str(rank))
+        procs.append(subprocess.Popen(argv, env=env, stdout=None if rank == 0 else subprocess.DEVNULL))
+    rc = 0
+    for p in procs:
+        try:
+            code = p.wait(timeout=timeout_s)
+        except subprocess.TimeoutExpired:
+            p.kill()
+            code = 124
+        rc = rc or code
+    return rc

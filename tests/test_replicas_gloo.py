@@ -65,3 +65,23 @@ def test_reference_arm_runs_on_rank0_only():
     assert rec["impl"] == "reference" and rec["cpu_baseline"]["kind"] == "oracle"
     assert rec["e2e"]["h2d_bytes_per_step"] == 0 and rec["value"] > 0
     assert rec["steps"] == 2 and rec["warmup"] == 1
+
+
+def test_bench_gpus_n_starts_n_replicas_itself():
+    """Without a launcher, `bench.py --gpus N` must start the N replica processes itself (here with the
+    self-test that needs no GPU): rank 0 prints one line for the whole job."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, "bench.py", "--gpus", "2", "--replica-selftest"], env=env, cwd=ROOT,
+                         capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec == {"selftest": True, "n_gpus": 2, "max_over_ranks": 2.0}
+
+
+def test_bench_refuses_a_launcher_that_disagrees_with_gpus():
+    env = dict(os.environ, WORLD_SIZE="3", RANK="0", LOCAL_RANK="0", MASTER_ADDR="127.0.0.1", MASTER_PORT="29999")
+    out = subprocess.run([sys.executable, "bench.py", "--gpus", "2", "--replica-selftest"], env=env, cwd=ROOT,
+                         capture_output=True, text=True, timeout=120)
+    assert out.returncode != 0 and "disagrees with WORLD_SIZE" in out.stderr
