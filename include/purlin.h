@@ -176,7 +176,23 @@ typedef struct {
                          /* registers"): every final sum is multiplied by this in fp32 before   */
                          /* the one conversion to the element type, e.g. 1/R for an average.    */
                          /* 0 = no scaling.  Float element types only (PL_ERR_UNSUPPORTED).     */
+  uint32_t hook;         /* PL_HOOK_* bits: further steps of the processing phase (below)        */
 } pl_sched_opts_t;
+/* The processing phase as a small family (Sec. 3.3: the phase between the last addition and the
+ * store is configurable while the sum sits in registers).  With s = out_scale (1 if unset):
+ *   out_r[i] = cvt( s * sum_p x_p[i]  [+ aux_r[i]] )
+ * PL_HOOK_RESIDUAL  adds a second operand per rank, aux[r] (pl_bufs_t), laid out like out[r] and
+ *                   of the element type, in fp32 before the one conversion (the residual
+ *                   connection that follows a tensor-parallel all-reduce).
+ * PL_HOOK_F32_OUT   bf16 schedules only: no conversion, out[r] holds fp32 (twice the bytes;
+ *                   pl_schedule_info reports them).
+ * Both need a collective whose outputs are written by its reduce ops and by nothing else:
+ * reduce-scatter (direct, ring, staged), one-shot and direct-fused all-reduce (also layered),
+ * reduce-scatter-v, rooted reduce.  Collectives that finish with a copy phase (ring / tree /
+ * two-shot all-reduce) return PL_ERR_UNSUPPORTED: a copied result cannot differ per rank.
+ * Float element types only; not on the packet datapath. */
+#define PL_HOOK_RESIDUAL 1u
+#define PL_HOOK_F32_OUT 2u
 #define PL_OPT_SKIP_VALIDATE 1u /* do not run the static validator inside build */
 /* Treat in/out as ORDINARY application buffers that peers must not touch (Sec. 3.2, "Protocol
  * operations": stage -> notify -> consume; Algorithm 1 with its staging role).  Every rank
@@ -224,7 +240,8 @@ typedef struct {
   int32_t n_wait;
   int32_t signal_flag; /* flag incremented (release) when the op's writes are done, -1 none */
   int32_t signal_flag2;/* optional second flag incremented the same way, -1 none */
-  int32_t dst_bcast;   /* 1: dst is replicated at the same offset into out[0..R) */
+  int32_t dst_bcast;   /* 1: dst is replicated at the same offset into out[0..R); 3: and the op is final */
+                       /* bit 1 (value 2): the op writes final output and runs the processing phase    */
   uint64_t count;      /* elements; COPY ops count bytes (dtype PL_U8) */
   pl_ref_t dst;
   pl_ref_t src[PL_MAX_SRC];
@@ -243,14 +260,21 @@ typedef struct {
   uint64_t out_bytes[PL_MAX_RANKS];    /* bytes pl_execute requires in bufs->out[r]         */
   int32_t grid, threads, smem_bytes, datapath, stages;
   uint32_t stage_bytes, slice_bytes;
+  uint64_t aux_bytes[PL_MAX_RANKS];    /* bytes pl_execute requires in bufs->aux[r] (PL_HOOK_RESIDUAL) */
+  int32_t out_dtype;                   /* element type stored in out[r]: PL_F32 under PL_HOOK_F32_OUT  */
+  uint32_t hook;                       /* PL_HOOK_* bits of the schedule                               */
 } pl_sched_info_t;
 
-/* Device buffers of one execute: in[r] / out[r] for r < R, 16-byte aligned, non-overlapping. */
+/* Device buffers of one execute: in[r] / out[r] for r < R, 16-byte aligned, non-overlapping.
+ * aux[r] is only read by schedules built with PL_HOOK_RESIDUAL (second operand of the
+ * processing phase, laid out like out[r]); it may overlap nothing that is written. */
 typedef struct {
   const void* in[PL_MAX_RANKS];
   void* out[PL_MAX_RANKS];
   size_t in_bytes[PL_MAX_RANKS];
   size_t out_bytes[PL_MAX_RANKS];
+  const void* aux[PL_MAX_RANKS];
+  size_t aux_bytes[PL_MAX_RANKS];
 } pl_bufs_t;
 
 /* Device-side status record (first writer wins).  code == PL_OK when nothing happened. */

@@ -199,6 +199,37 @@ def reduce(inputs, root, dtype):
     return out
 
 
+# ---- processing phase (Sec. 3.3: the step between the last addition and the store is
+# configurable): out_r[i] = scale * sum_p x_p[i] + aux_r[i], all in fp64 here.  The element type of
+# the stored result (bf16, or fp32 when no conversion is asked for) is the caller's business: the
+# oracle returns the exact fp64 value either way.
+def _to_f64(a, dtype):
+    if dtype == "bf16":
+        assert a.dtype == np.uint16
+        return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    return a.astype(np.float64)
+
+
+def processed(sums, dtype, scale=1.0, aux=None):
+    """sums[r]: fp64 arrays (an fp64 collective result); aux[r]: element-typed second operands laid
+    out like the outputs, or None."""
+    out = []
+    for r, acc in enumerate(sums):
+        v = np.float64(scale) * acc
+        if aux is not None:
+            v = v + _to_f64(aux[r], dtype)
+        out.append(v)
+    return out
+
+
+def allreduce_processed(inputs, dtype, scale=1.0, aux=None):
+    return processed(allreduce(inputs, dtype), dtype, scale, aux)
+
+
+def reduce_scatter_processed(inputs, dtype, scale=1.0, aux=None):
+    return processed(reduce_scatter(inputs, dtype), dtype, scale, aux)
+
+
 def moe_dispatch(x, idx, E, recv_capacity_rows=None):
     """x[p]: [T, W] row arrays (any dtype), idx[p]: int32 [T, K].
     Returns dict(recv, meta, pos, counts, expert_counts); recv[r] has capacity rows,

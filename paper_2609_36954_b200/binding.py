@@ -38,6 +38,8 @@ PL_OPT_NO_L2_HINTS = 2
 PL_OPT_STAGED = 4
 PL_OPT_TRACE = 8
 PL_OPT_OVERLAP_LAUNCH = 16
+PL_HOOK_RESIDUAL = 1
+PL_HOOK_F32_OUT = 2
 
 
 class PurlinError(RuntimeError):
@@ -50,7 +52,7 @@ class pl_sched_opts_t(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("n_ctas", C.c_int32), ("threads", C.c_int32),
                 ("datapath", C.c_int32), ("stages", C.c_int32), ("stage_bytes", C.c_uint32),
                 ("slice_bytes", C.c_uint32), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32),
-                ("staging_bytes", C.c_uint64), ("out_scale", C.c_float)]
+                ("staging_bytes", C.c_uint64), ("out_scale", C.c_float), ("hook", C.c_uint32)]
 
 
 class pl_ref_t(C.Structure):
@@ -74,12 +76,14 @@ class pl_sched_info_t(C.Structure):
                 ("in_bytes", C.c_uint64 * PL_MAX_RANKS), ("out_bytes", C.c_uint64 * PL_MAX_RANKS),
                 ("grid", C.c_int32), ("threads", C.c_int32), ("smem_bytes", C.c_int32),
                 ("datapath", C.c_int32), ("stages", C.c_int32),
-                ("stage_bytes", C.c_uint32), ("slice_bytes", C.c_uint32)]
+                ("stage_bytes", C.c_uint32), ("slice_bytes", C.c_uint32),
+                ("aux_bytes", C.c_uint64 * PL_MAX_RANKS), ("out_dtype", C.c_int32), ("hook", C.c_uint32)]
 
 
 class pl_bufs_t(C.Structure):
     _fields_ = [("in_", C.c_void_p * PL_MAX_RANKS), ("out", C.c_void_p * PL_MAX_RANKS),
-                ("in_bytes", C.c_size_t * PL_MAX_RANKS), ("out_bytes", C.c_size_t * PL_MAX_RANKS)]
+                ("in_bytes", C.c_size_t * PL_MAX_RANKS), ("out_bytes", C.c_size_t * PL_MAX_RANKS),
+                ("aux", C.c_void_p * PL_MAX_RANKS), ("aux_bytes", C.c_size_t * PL_MAX_RANKS)]
 
 
 class pl_devstatus_t(C.Structure):
@@ -176,19 +180,24 @@ def _check(st, where):
 
 
 def make_opts(n_ctas=0, threads=0, datapath=PL_DP_AUTO, stages=0, stage_bytes=0, slice_bytes=0,
-              timeout_ns=0, flags=0, staging_bytes=0, out_scale=0.0):
+              timeout_ns=0, flags=0, staging_bytes=0, out_scale=0.0, hook=0):
     o = pl_sched_opts_t()
     o.struct_size = C.sizeof(pl_sched_opts_t)
     o.n_ctas, o.threads, o.datapath, o.stages = n_ctas, threads, datapath, stages
     o.stage_bytes, o.slice_bytes, o.timeout_ns, o.flags = stage_bytes, slice_bytes, timeout_ns, flags
     o.staging_bytes = staging_bytes
     o.out_scale = out_scale
+    o.hook = hook
     return o
 
 
-def make_bufs(ins, outs, in_bytes, out_bytes):
-    """ins/outs: integer addresses per rank (device or host, as the callee expects)."""
+def make_bufs(ins, outs, in_bytes, out_bytes, aux=None, aux_bytes=None):
+    """ins/outs (and aux, for PL_HOOK_RESIDUAL): integer addresses per rank (device or host, as the
+    callee expects)."""
     b = pl_bufs_t()
+    for r, (a, n) in enumerate(zip(aux or [], aux_bytes or [])):
+        b.aux[r] = a
+        b.aux_bytes[r] = n
     for r, (a, n) in enumerate(zip(ins, in_bytes)):
         b.in_[r] = a
         b.in_bytes[r] = n

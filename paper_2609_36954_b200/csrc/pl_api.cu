@@ -45,6 +45,7 @@ struct pl_schedule_s {
   long long packet_break_op = -1; // test hook (pl_schedule_debug_break_wait on a packet schedule)
   size_t off_trace = 0;
   float out_scale = 1.0f;
+  uint32_t hook = 0;  // PL_HOOK_* bits
   // host copies in device (queue-major) order
   std::vector<DevOp> dev_ops;
   std::vector<uint64_t> srcs;
@@ -82,13 +83,17 @@ void fill_info(pl_schedule_s* S, int R) {
     I.n_waits += op.waits.size();
     for (const pl_ref_t& s : op.src) I.bytes_read += op.count * elem_size(s.dtype);
     I.bytes_written += op.count * elem_size(op.dst.dtype) * (op.bcast ? R : 1);
+    if (op.final_hook && (S->hook & PL_HOOK_RESIDUAL)) I.bytes_read += op.count * elem_size(S->comm->dtype) * (op.bcast ? R : 1);
   }
   I.message_bytes = L.message_bytes;
   for (int r = 0; r < R; ++r) {
     I.scratch_bytes += L.scratch_per_rank[r];
     I.in_bytes[r] = L.in_bytes[r];
     I.out_bytes[r] = L.out_bytes[r];
+    I.aux_bytes[r] = L.aux_bytes[r];
   }
+  I.out_dtype = (S->hook & PL_HOOK_F32_OUT) ? PL_F32 : S->comm->dtype;
+  I.hook = S->hook;
   I.grid = S->pol.n_ctas;
   I.threads = S->pol.threads;
   I.smem_bytes = S->pol.datapath == PL_DP_TMA ? (int32_t)exec_tma_smem_bytes(S->pol.stages, S->pol.stage_bytes) : 0;
@@ -134,7 +139,8 @@ void flatten(pl_schedule_s* S, int dtype) {
     d.n_wait = (uint32_t)op.waits.size();
     d.signal = op.signal >= 0 ? (uint32_t)op.signal : kNoFlag;
     d.signal2 = op.signal2 >= 0 ? (uint32_t)op.signal2 : kNoFlag;
-    d.flags = (op.bcast ? kDstBcast : 0u) | ((op.kind != PL_OP_COPY && op.dst.dtype != dtype) ? kDstF32 : 0u);
+    d.flags = (op.bcast ? kDstBcast : 0u) | ((op.kind != PL_OP_COPY && op.dst.dtype != dtype) ? kDstF32 : 0u) |
+              (op.final_hook ? kFinal : 0u);
     d.count = op.count;
     d.dst = pack(*S, op.dst);
     d.topo = (uint32_t)op.topo;
@@ -273,7 +279,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
   Policy pol{};
   uint64_t timeout = 2000000000ull;
-  uint32_t flags = 0;
+  uint32_t flags = 0, hook = 0;
   float out_scale = 1.0f;
   if (opts) {
     if (opts->struct_size != sizeof(pl_sched_opts_t)) return PL_ERR_INVALID_ARG;
@@ -291,12 +297,20 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
       if (comm->dtype != PL_BF16 && comm->dtype != PL_F32) return PL_ERR_UNSUPPORTED;
       out_scale = opts->out_scale;
     }
+    hook = opts->hook;
+    if (hook & ~(PL_HOOK_RESIDUAL | PL_HOOK_F32_OUT)) return PL_ERR_INVALID_ARG;
+    if (hook && comm->dtype != PL_BF16 && comm->dtype != PL_F32) return PL_ERR_UNSUPPORTED;
     if (pol.threads < 0 || pol.threads % 32 || pol.threads > exec_max_threads()) return PL_ERR_INVALID_ARG;
     if (pol.n_ctas < 0 || pol.stages < 0 || pol.stage_bytes % 16 || pol.slice_bytes % 16) return PL_ERR_INVALID_ARG;
     if (pol.datapath < PL_DP_AUTO || pol.datapath > PL_DP_PACKET) return PL_ERR_INVALID_ARG;
   }
   rq.R = comm->R;
   rq.dtype = comm->dtype;
+  rq.hook = hook;
+  if (pol.datapath == PL_DP_PACKET && hook) {
+    comm->last_error = "processing hooks are not offered on the packet datapath";
+    return PL_ERR_UNSUPPORTED;
+  }
   if (pol.datapath == PL_DP_PACKET) return build_packets(comm, rq, pol, timeout, flags, out_scale, out);
   rq.pol = pol;
   const int requested = pol.n_ctas;
@@ -330,6 +344,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   S->trace = (flags & PL_OPT_TRACE) != 0;
   S->overlap_launch = (flags & PL_OPT_OVERLAP_LAUNCH) != 0;
   S->out_scale = out_scale;
+  S->hook = hook;
   std::string err;
   pl_status_t st = lower(rq, &S->L, &err);
   if (st != PL_OK) {
@@ -365,7 +380,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
       for (const pl_ref_t& r : op.src)
         if (r.dtype != comm->dtype) plain = false;
     }
-    S->pipelined_reduce = any && plain;
+    S->pipelined_reduce = any && plain && !hook;  // the processing phase lives in the general variant
     S->pol.threads = exec_tma_threads(S->pipelined_reduce);
   }
   for (const HostOp& op : S->L.ops)
@@ -557,7 +572,7 @@ pl_status_t pl_schedule_dump(pl_schedule_t s, pl_op_t* ops, size_t cap, size_t* 
     o.n_wait = (int32_t)h.waits.size();
     o.signal_flag = h.signal;
     o.signal_flag2 = h.signal2;
-    o.dst_bcast = h.bcast ? 1 : 0;
+    o.dst_bcast = (h.bcast ? 1 : 0) | (h.final_hook ? 2 : 0);
     o.count = h.count;
     o.dst = h.dst;
     for (size_t k = 0; k < h.src.size(); ++k) o.src[k] = h.src[k];
@@ -641,6 +656,11 @@ static pl_status_t check_bufs(pl_schedule_t s, const pl_bufs_t* b) {
     if (((uintptr_t)b->in[r] & 15) || ((uintptr_t)b->out[r] & 15)) return PL_ERR_ALIGNMENT;
     if (b->in_bytes[r] < s->info.in_bytes[r] || b->out_bytes[r] < s->info.out_bytes[r]) return PL_ERR_INVALID_ARG;
   }
+  for (int r = 0; r < R; ++r) {
+    if (!s->info.aux_bytes[r]) continue;
+    if (!b->aux[r] || b->aux_bytes[r] < s->info.aux_bytes[r]) return PL_ERR_INVALID_ARG;
+    if ((uintptr_t)b->aux[r] & 15) return PL_ERR_ALIGNMENT;
+  }
   // outputs must not overlap any input or another output (all collectives are out of place)
   for (int r = 0; r < R; ++r) {
     const uintptr_t olo = (uintptr_t)b->out[r], ohi = olo + s->info.out_bytes[r];
@@ -648,6 +668,8 @@ static pl_status_t check_bufs(pl_schedule_t s, const pl_bufs_t* b) {
     for (int p = 0; p < R; ++p) {
       const uintptr_t ilo = (uintptr_t)b->in[p], ihi = ilo + s->info.in_bytes[p];
       if (ilo < ohi && olo < ihi) return PL_ERR_INVALID_ARG;
+      const uintptr_t alo = (uintptr_t)b->aux[p], ahi = alo + s->info.aux_bytes[p];
+      if (s->info.aux_bytes[p] && alo < ohi && olo < ahi) return PL_ERR_INVALID_ARG;
       if (p != r) {
         const uintptr_t qlo = (uintptr_t)b->out[p], qhi = qlo + s->info.out_bytes[p];
         if (qlo < ohi && olo < qhi) return PL_ERR_INVALID_ARG;
@@ -696,7 +718,9 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
     P.base[kSlotIn + r] = const_cast<void*>(bufs->in[r]);
     P.base[kSlotOut + r] = bufs->out[r];
     P.base[kSlotScratch + r] = s->d_scratch ? s->d_scratch + s->scratch_off[r] : nullptr;
+    P.base[kSlotAux + r] = s->info.aux_bytes[r] ? const_cast<void*>(bufs->aux[r]) : nullptr;
   }
+  P.hook = s->hook;
   P.ops = reinterpret_cast<const DevOp*>(s->d_blob + s->off_ops);
   P.n_queues = (uint32_t)s->pol.n_ctas;
   P.srcs = reinterpret_cast<const uint64_t*>(s->d_blob + s->off_srcs);
@@ -742,6 +766,14 @@ pl_status_t pl_execute_host(pl_schedule_t s, const pl_bufs_t* host, const pl_buf
       cudaGetLastError();
       return PL_ERR_CUDA;
     }
+  for (int r = 0; r < R; ++r) {
+    if (!s->info.aux_bytes[r]) continue;
+    if (!host->aux[r] || host->aux_bytes[r] < s->info.aux_bytes[r]) return PL_ERR_INVALID_ARG;
+    if (cudaMemcpyAsync(const_cast<void*>(dev->aux[r]), host->aux[r], s->info.aux_bytes[r], cudaMemcpyHostToDevice, cs) != cudaSuccess) {
+      cudaGetLastError();
+      return PL_ERR_CUDA;
+    }
+  }
   st = pl_execute(s, dev, stream);
   if (st != PL_OK) return st;
   for (int r = 0; r < R; ++r)

@@ -73,9 +73,10 @@ __device__ __forceinline__ void accumulate_batch(Acc<DT> (&acc)[U], const char* 
 }
 
 // Reduce U units (unit index first + u*stride) from ns sources and store the result.
-template <int DT, int U>
+template <int DT, int U, bool HOOK>
 __device__ __forceinline__ void reduce_units(const ExecParams& P, const char* const* s_src, int ns, char* dst,
-                                             uint64_t dst_off, bool bcast, uint64_t first, uint64_t stride) {
+                                             uint64_t dst_off, bool bcast, uint64_t first, uint64_t stride,
+                                             uint64_t dst_slot, bool final_op) {
   Acc<DT> acc[U];
   uint64_t off[U];
 #pragma unroll
@@ -88,6 +89,13 @@ __device__ __forceinline__ void reduce_units(const ExecParams& P, const char* co
   for (; s + 4 <= ns; s += 4) accumulate_batch<DT, 4, U>(acc, s_src + s, off);
   if (s + 2 <= ns) { accumulate_batch<DT, 2, U>(acc, s_src + s, off); s += 2; }
   if (s < ns) accumulate_batch<DT, 1, U>(acc, s_src + s, off);
+  if constexpr (HOOK) {
+    if (final_op) {  // the processing phase: scale, second operand, output type
+#pragma unroll
+      for (int u = 0; u < U; ++u) store_final_unit<DT>(P, acc[u], dst_slot, dst_off, bcast, first + (uint64_t)u * stride);
+      return;
+    }
+  }
 #pragma unroll
   for (int u = 0; u < U; ++u) {
     uint4 r;
@@ -103,10 +111,12 @@ __device__ __forceinline__ void reduce_units(const ExecParams& P, const char* co
 
 // REDUCE with n same-typed sources -> element-typed destination (optionally replicated to
 // every rank's output).  s_src holds the resolved source pointers in shared memory.
-template <int DT>
+template <int DT, bool HOOK>
 __device__ __forceinline__ void body_reduce(const ExecParams& P, const DevOp& op, const char* const* s_src, int tid,
                                             int nthr) {
   constexpr int U = 2;
+  const uint64_t dst_slot = op.dst >> 48;
+  const bool final_op = op.flags & kFinal;
   const uint64_t n_units = op.count / Acc<DT>::kElems;  // 16 bytes of every operand each
   const bool bcast = op.flags & kDstBcast;
   char* dst = resolve(P, op.dst);
@@ -114,12 +124,37 @@ __device__ __forceinline__ void body_reduce(const ExecParams& P, const DevOp& op
   const int ns = op.n_src;
   uint64_t base = tid;
   for (; base + (uint64_t)(U - 1) * nthr < n_units; base += (uint64_t)U * nthr)
-    reduce_units<DT, U>(P, s_src, ns, dst, dst_off, bcast, base, nthr);
-  for (; base < n_units; base += nthr) reduce_units<DT, 1>(P, s_src, ns, dst, dst_off, bcast, base, nthr);
+    reduce_units<DT, U, HOOK>(P, s_src, ns, dst, dst_off, bcast, base, nthr, dst_slot, final_op);
+  for (; base < n_units; base += nthr) reduce_units<DT, 1, HOOK>(P, s_src, ns, dst, dst_off, bcast, base, nthr, dst_slot, final_op);
 }
 
 // COPY_REDUCE: dst = a + b where a and/or b may hold fp32 partials of a bf16 reduction and
 // dst may be a partial too.  For fp32 / int32 data every operand has the element type.
+// Final hop of a travelling sum in a hooked schedule: dst = process(a + b).
+template <int DT>
+__device__ __forceinline__ void body_copy_reduce_final(const ExecParams& P, const DevOp& op, const char* const* s_src,
+                                                       int tid, int nthr) {
+  if constexpr (DT == PL_BF16 || DT == PL_F32) {
+    const uint64_t n_units = op.count / Acc<DT>::kElems;
+    const char* a = s_src[0];
+    const char* b = s_src[1];
+    const bool ap = op.src_f32_mask & 1u, bp = op.src_f32_mask & 2u;
+    const uint64_t dst_slot = op.dst >> 48, dst_off = op.dst & 0xFFFFFFFFFFFFull;
+    for (uint64_t i = tid; i < n_units; i += nthr) {
+      Acc<DT> acc;
+      acc.zero();
+      if constexpr (DT == PL_BF16) {
+        if (ap) acc.add_f32(ld16(a + (i << 5)), ld16(a + (i << 5) + 16)); else acc.add_bf16(ld16(a + (i << 4)));
+        if (bp) acc.add_f32(ld16(b + (i << 5)), ld16(b + (i << 5) + 16)); else acc.add_bf16(ld16(b + (i << 4)));
+      } else {
+        if (ap) acc.add_pair(ld16(a + (i << 5)), ld16(a + (i << 5) + 16)); else acc.add(ld16(a + (i << 4)));
+        if (bp) acc.add_pair(ld16(b + (i << 5)), ld16(b + (i << 5) + 16)); else acc.add(ld16(b + (i << 4)));
+      }
+      store_final_unit<DT>(P, acc, dst_slot, dst_off, false, i);
+    }
+  }
+}
+
 template <int DT>
 __device__ __forceinline__ void body_copy_reduce(const ExecParams& P, const DevOp& op, const char* const* s_src,
                                                  int tid, int nthr) {
@@ -229,7 +264,10 @@ struct OpSlot {
 // kernel of its own because the mere presence of that body in the function changed the code
 // generated for the reduce loops (one-shot all-reduce of 8 MiB per rank: 71 -> 88 us);
 // schedules with broadcast copies hold no reduce ops, schedules with reduce ops run BC = false.
-template <int DT, bool BC>
+// HOOK: the variant for schedules with a processing phase beyond the scale (PL_HOOK_*): its
+// final reduce ops add the second operand and / or keep fp32.  A kernel of its own for the
+// same reason as BC: the plain variants keep the code they have.
+template <int DT, bool BC, bool HOOK = false>
 __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_constant__ ExecParams P) {
   __shared__ OpSlot s_slot[2];
   __shared__ int s_abort[2];  // indexed by iteration parity: written during wait i, read after barrier i
@@ -310,9 +348,12 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
         body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
       }
     } else if (op.kind == PL_OP_REDUCE) {
-      if constexpr (DT != PL_U8) body_reduce<DT>(P, op, S.src, tid, nthr);
+      if constexpr (DT != PL_U8) body_reduce<DT, HOOK>(P, op, S.src, tid, nthr);
     } else {
-      if constexpr (DT != PL_U8) body_copy_reduce<DT>(P, op, S.src, tid, nthr);
+      if constexpr (DT != PL_U8) {
+        if (HOOK && (op.flags & kFinal)) body_copy_reduce_final<DT>(P, op, S.src, tid, nthr);
+        else body_copy_reduce<DT>(P, op, S.src, tid, nthr);
+      }
     }
 
     if (op.signal != kNoFlag || P.trace) {
@@ -342,7 +383,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   }
 }
 
-template <int DT, bool BC>
+template <int DT, bool BC, bool HOOK = false>
 cudaError_t launch_t(const ExecParams& P, int grid, int threads, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
@@ -353,12 +394,19 @@ cudaError_t launch_t(const ExecParams& P, int grid, int threads, cudaStream_t st
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = P.overlap_launch ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, pl_exec_kernel<DT, BC>, P);
+  return cudaLaunchKernelEx(&cfg, pl_exec_kernel<DT, BC, HOOK>, P);
 }
 
 }  // namespace
 
 cudaError_t launch_exec(int dtype, const ExecParams& P, int grid, int threads, cudaStream_t stream) {
+  if (P.hook) {  // float schedules with reduce ops only (checked at build)
+    switch (dtype) {
+      case PL_BF16: return launch_t<PL_BF16, false, true>(P, grid, threads, stream);
+      case PL_F32: return launch_t<PL_F32, false, true>(P, grid, threads, stream);
+      default: return cudaErrorInvalidValue;
+    }
+  }
   if (P.bcast_copies) {
     switch (dtype) {
       case PL_BF16: return launch_t<PL_BF16, true>(P, grid, threads, stream);
@@ -379,13 +427,19 @@ namespace {
 template <int DT>
 int occupancy_both(int threads) {
   // capacity that holds for whichever variant a schedule launches
-  int a = 0, b = 0;
+  int a = 0, b = 0, c = 1 << 30;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, pl_exec_kernel<DT, true>, threads, 0) != cudaSuccess ||
       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, pl_exec_kernel<DT, false>, threads, 0) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
-  return a < b ? a : b;
+  if constexpr (DT == PL_BF16 || DT == PL_F32) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c, pl_exec_kernel<DT, false, true>, threads, 0) != cudaSuccess) {
+      cudaGetLastError();
+      return 0;
+    }
+  }
+  return a < b ? (a < c ? a : c) : (b < c ? b : c);
 }
 }  // namespace
 

@@ -53,7 +53,7 @@ struct StageDesc {
   char* dst;       // destination of this stage
   uint64_t dst_off;  // byte offset inside every rank's output (broadcast destinations)
   uint32_t topo;   // the op's topological index (trace)
-  uint32_t pad;
+  uint32_t dst_slot;  // pointer-table slot of the destination (hooked schedules: finds the second operand)
 };
 static_assert(sizeof(StageDesc) == 56, "StageDesc layout");
 
@@ -97,11 +97,12 @@ __device__ __forceinline__ uint4 lds16(const unsigned char* p) {
 }
 
 // Consumer work for one stage of a REDUCE / COPY_REDUCE op.
-template <int DT, int CW>
+template <int DT, int CW, bool HOOK>
 __device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDesc& d, const unsigned char* slot, int ctid) {
   const uint32_t units = d.units, ns = d.n_src, pmask = d.pmask;
   const uint32_t tile = d.ucap * 16u;  // bytes of an element-typed tile; partial tiles are twice that
   const bool dpart = d.flags & kDstF32, bcast = d.flags & kDstBcast;
+  const bool final_op = HOOK && (d.flags & kFinal);
   for (uint32_t u = ctid; u < units; u += 32 * CW) {
     Acc<DT> acc;
     acc.zero();
@@ -141,7 +142,11 @@ __device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDe
         }
       }
     }
-    if (dpart) {
+    if (final_op) {
+      // processing phase of a hooked schedule: scale, second operand, output type; one store
+      // per destination (the results may differ per rank, so nothing leaves through the slot)
+      if constexpr (HOOK && (DT == PL_BF16 || DT == PL_F32)) store_final_unit<DT>(P, acc, d.dst_slot, d.dst_off, bcast, u);
+    } else if (dpart) {
       if constexpr (DT == PL_BF16) {
         st16(d.dst + (size_t)u * 32u, make_uint4(__float_as_uint(acc.v[0]), __float_as_uint(acc.v[1]),
                                                   __float_as_uint(acc.v[2]), __float_as_uint(acc.v[3])));
@@ -170,7 +175,7 @@ __device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDe
       }
     }
   }
-  if (bcast && pmask == 0) ptx::fence_proxy_async_smem();  // generic writes above -> the copier's bulk stores
+  if (bcast && pmask == 0 && !final_op) ptx::fence_proxy_async_smem();  // generic writes above -> the copier's bulk stores
 }
 
 // ---- software-pipelined path for plain reduce stages ---------------------------------------
@@ -280,10 +285,11 @@ __device__ __forceinline__ void plain_finish(const ExecParams& P, const PlainSta
 
 // A REDUCE stage whose result leaves through shared memory (see consume_stage).
 __device__ __forceinline__ bool leaves_via_smem(uint32_t kind, uint32_t flags, uint32_t pmask) {
-  return kind != PL_OP_COPY && (flags & kDstBcast) && !(flags & kDstF32) && pmask == 0;
+  return kind != PL_OP_COPY && (flags & kDstBcast) && !(flags & (kDstF32 | kFinal)) && pmask == 0;
 }
 
-template <int DT, int CW>
+// HOOK: the variant for schedules with a processing phase beyond the scale (general consumers only).
+template <int DT, int CW, bool HOOK = false>
 __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __grid_constant__ ExecParams P) {
   extern __shared__ __align__(1024) unsigned char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
@@ -401,6 +407,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
           d.dst = dst + u0 * dst_w;
           d.dst_off = dst_off + u0 * dst_w;
           d.topo = topo;
+          d.dst_slot = (uint32_t)(dstp >> 48);
           ptx::mbar_expect_tx(&c->full[s], units * unit_b);
         }
         __syncwarp();
@@ -541,7 +548,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
         }
       }
       if (kind != PL_OP_COPY) {
-        if constexpr (DT != PL_U8) consume_stage<DT, CW>(P, d, slots + (size_t)s * slot_bytes, ctid);
+        if constexpr (DT != PL_U8) consume_stage<DT, CW, HOOK>(P, d, slots + (size_t)s * slot_bytes, ctid);
         const bool last = d.flags & kLastOfOp;
         const uint32_t signal = d.signal, signal2 = d.signal2, topo = d.topo;
         __syncwarp();
@@ -579,7 +586,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
   }
 }
 
-template <int DT, int CW>
+template <int DT, int CW, bool HOOK = false>
 cudaError_t launch_t(const ExecParams& P, int grid, cudaStream_t stream) {
   const size_t smem = exec_tma_smem_bytes(P.stages, P.stage_bytes);
   // the shared-memory opt-in is a per-device attribute of the function: one bit per device
@@ -589,7 +596,7 @@ cudaError_t launch_t(const ExecParams& P, int grid, cudaStream_t stream) {
   if (e != cudaSuccess) return e;
   const unsigned long long bit = 1ull << (dev & 63);
   if (!(configured.load(std::memory_order_acquire) & bit)) {
-    e = cudaFuncSetAttribute(pl_exec_tma_kernel<DT, CW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    e = cudaFuncSetAttribute(pl_exec_tma_kernel<DT, CW, HOOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     configured.fetch_or(bit, std::memory_order_release);
   }
@@ -603,14 +610,14 @@ cudaError_t launch_t(const ExecParams& P, int grid, cudaStream_t stream) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = P.overlap_launch ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, pl_exec_tma_kernel<DT, CW>, P);
+  return cudaLaunchKernelEx(&cfg, pl_exec_tma_kernel<DT, CW, HOOK>, P);
 }
 
-template <int DT, int CW>
+template <int DT, int CW, bool HOOK = false>
 int occupancy_t(size_t smem) {
   int n = 0;
-  if (cudaFuncSetAttribute(pl_exec_tma_kernel<DT, CW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_tma_kernel<DT, CW>, 32 * (2 + CW), smem) != cudaSuccess) {
+  if (cudaFuncSetAttribute(pl_exec_tma_kernel<DT, CW, HOOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_tma_kernel<DT, CW, HOOK>, 32 * (2 + CW), smem) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
@@ -624,6 +631,13 @@ int exec_tma_threads(bool pipelined) { return 32 * (2 + (pipelined ? kWarpsPipel
 
 cudaError_t launch_exec_tma(int dtype, const ExecParams& P, int grid, cudaStream_t stream) {
   if (P.stages < 2 || P.stages > kMaxStages) return cudaErrorInvalidValue;
+  if (P.hook) {
+    switch (dtype) {
+      case PL_BF16: return launch_t<PL_BF16, kWarpsGeneral, true>(P, grid, stream);
+      case PL_F32: return launch_t<PL_F32, kWarpsGeneral, true>(P, grid, stream);
+      default: return cudaErrorInvalidValue;
+    }
+  }
   if (P.pipelined_reduce) {
     switch (dtype) {
       case PL_BF16: return launch_t<PL_BF16, kWarpsPipelined>(P, grid, stream);
@@ -645,8 +659,10 @@ int exec_tma_max_ctas_per_sm(int dtype, int stages, uint32_t stage_bytes) {
   const size_t smem = exec_tma_smem_bytes(stages, stage_bytes);
   if (smem > 227 * 1024) return 0;
   switch (dtype) {
-    case PL_BF16: return std::min(occupancy_t<PL_BF16, kWarpsGeneral>(smem), occupancy_t<PL_BF16, kWarpsPipelined>(smem));
-    case PL_F32: return std::min(occupancy_t<PL_F32, kWarpsGeneral>(smem), occupancy_t<PL_F32, kWarpsPipelined>(smem));
+    case PL_BF16: return std::min({occupancy_t<PL_BF16, kWarpsGeneral>(smem), occupancy_t<PL_BF16, kWarpsPipelined>(smem),
+                                   occupancy_t<PL_BF16, kWarpsGeneral, true>(smem)});
+    case PL_F32: return std::min({occupancy_t<PL_F32, kWarpsGeneral>(smem), occupancy_t<PL_F32, kWarpsPipelined>(smem),
+                                  occupancy_t<PL_F32, kWarpsGeneral, true>(smem)});
     case PL_I32: return std::min(occupancy_t<PL_I32, kWarpsGeneral>(smem), occupancy_t<PL_I32, kWarpsPipelined>(smem));
     default: return occupancy_t<PL_U8, kWarpsGeneral>(smem);
   }

@@ -151,6 +151,74 @@ struct Acc<PL_I32> {
   __device__ __forceinline__ uint4 result(float = 1.0f) const { return make_uint4(v[0], v[1], v[2], v[3]); }
 };
 
+// ---- processing phase of a final reduce op (Sec. 3.3: configurable while the sum is in registers)
+// value = scale * sum [+ residual], then one conversion to the element type, or none (fp32 out).
+// `dst` points at this unit in the destination (16 bytes per unit; 32 for fp32 output of a bf16
+// schedule), `res` at the same unit of the second operand (element-typed) or is unused.
+template <int DT>
+__device__ __forceinline__ void store_final(const Acc<DT>& acc, float scale, uint32_t hook, char* dst, const char* res) {
+  if constexpr (DT == PL_BF16) {
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __fmul_rn(acc.v[i], scale);
+    if (hook & PL_HOOK_RESIDUAL) {
+      const uint4 q = ld16(res);
+      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __fadd_rn(v[2 * i], __uint_as_float(w[i] << 16));
+        v[2 * i + 1] = __fadd_rn(v[2 * i + 1], __uint_as_float(w[i] & 0xFFFF0000u));
+      }
+    }
+    if (hook & PL_HOOK_F32_OUT) {
+      st16(dst, make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])));
+      st16(dst + 16, make_uint4(__float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7])));
+    } else {
+      uint4 q;
+      __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+      __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
+      q.x = *reinterpret_cast<uint32_t*>(&a);
+      q.y = *reinterpret_cast<uint32_t*>(&b);
+      q.z = *reinterpret_cast<uint32_t*>(&c);
+      q.w = *reinterpret_cast<uint32_t*>(&d);
+      st16(dst, q);
+    }
+  } else if constexpr (DT == PL_F32) {
+    float v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = __fmul_rn(__fadd_rn(acc.v[i], acc.c[i]), scale);
+    if (hook & PL_HOOK_RESIDUAL) {
+      const uint4 q = ld16(res);
+      v[0] = __fadd_rn(v[0], __uint_as_float(q.x));
+      v[1] = __fadd_rn(v[1], __uint_as_float(q.y));
+      v[2] = __fadd_rn(v[2], __uint_as_float(q.z));
+      v[3] = __fadd_rn(v[3], __uint_as_float(q.w));
+    }
+    st16(dst, make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])));
+  }
+}
+
+// A final op of a hooked schedule stores unit `unit` of its result to one destination or to all
+// ranks' outputs.  dst_packed = (slot << 48) | byte offset of the op's destination; the second
+// operand of rank k sits in slot kSlotAux + k, laid out like the (element-typed) output.
+template <int DT>
+__device__ __forceinline__ void store_final_unit(const ExecParams& P, const Acc<DT>& acc, uint64_t dst_slot, uint64_t dst_off,
+                                                 bool bcast, uint64_t unit) {
+  const uint32_t hook = P.hook;
+  const bool f32 = (DT == PL_BF16) && (hook & PL_HOOK_F32_OUT);
+  const uint64_t d_off = dst_off + unit * (f32 ? 32ull : 16ull);       // bytes into the output
+  const uint64_t r_off = (f32 ? dst_off >> 1 : dst_off) + unit * 16ull;  // bytes into the second operand
+  if (!bcast) {
+    const char* res = (hook & PL_HOOK_RESIDUAL) ? static_cast<const char*>(P.base[kSlotAux + (dst_slot - kSlotOut)]) + r_off : nullptr;
+    store_final<DT>(acc, P.out_scale, hook, static_cast<char*>(P.base[dst_slot]) + d_off, res);
+  } else {
+    for (int k = 0; k < P.n_ranks; ++k) {
+      const char* res = (hook & PL_HOOK_RESIDUAL) ? static_cast<const char*>(P.base[kSlotAux + k]) + r_off : nullptr;
+      store_final<DT>(acc, P.out_scale, hook, static_cast<char*>(P.base[kSlotOut + k]) + d_off, res);
+    }
+  }
+}
+
 // Record a timeout (first writer wins) and raise the abort word.
 static __device__ __noinline__ void record_timeout_at(int* status, int queue, uint32_t topo, uint32_t flag,
                                                       unsigned long long expected, unsigned long long observed) {

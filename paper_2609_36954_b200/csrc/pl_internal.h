@@ -34,6 +34,7 @@ struct HostOp {
   std::vector<int> waits;  // flag ids
   int signal = -1;
   int signal2 = -1;
+  bool final_hook = false;  // writes final output: the processing phase (residual, fp32 output) applies
   int role = 0;  // 0 = any queue of the rank; 1 stage, 2 reduce, 3 gather: CTA groups per role (Sec. 3.2)
   int queue = -1;
   int topo = -1;
@@ -42,8 +43,8 @@ struct HostOp {
 // ---- device-resident schedule ------------------------------------------------------
 // A buffer address is packed as (slot << 48) | byte offset; slot indexes the pointer
 // table passed by value in the kernel parameters: in[0..16), out[16..32), scratch[32..48).
-constexpr int kSlotIn = 0, kSlotOut = PL_MAX_RANKS, kSlotScratch = 2 * PL_MAX_RANKS;
-constexpr int kNumSlots = 3 * PL_MAX_RANKS;
+constexpr int kSlotIn = 0, kSlotOut = PL_MAX_RANKS, kSlotScratch = 2 * PL_MAX_RANKS, kSlotAux = 3 * PL_MAX_RANKS;
+constexpr int kNumSlots = 4 * PL_MAX_RANKS;
 constexpr uint32_t kNoFlag = 0xFFFFFFFFu;
 constexpr uint32_t kNopKind = 0xFFu;  // placeholder op of an empty queue
 
@@ -55,7 +56,7 @@ struct alignas(16) DevOp {
   uint32_t rsv1;
   uint32_t n_wait;
   uint32_t signal;      // flag index or kNoFlag
-  uint32_t flags;       // bit0: dst holds partials; bit1: dst broadcast
+  uint32_t flags;       // bit0: dst holds partials (or fp32 output); bit1: dst broadcast; bit2: final op of a hooked schedule
   uint64_t count;       // elements (bytes for COPY)
   uint64_t dst;         // packed address
   uint32_t topo;
@@ -63,7 +64,7 @@ struct alignas(16) DevOp {
   uint32_t pad[2];
 };
 static_assert(sizeof(DevOp) == 64, "DevOp must stay 64 bytes");
-constexpr uint32_t kDstF32 = 1u, kDstBcast = 2u;
+constexpr uint32_t kDstF32 = 1u, kDstBcast = 2u, kFinal = 4u;  // kFinal: processing phase applies (hooked schedules)
 
 struct DevWait {
   uint32_t flag;
@@ -89,6 +90,7 @@ struct ExecParams {
   int stages;            // shared-memory ring depth of the TMA executor
   uint32_t stage_bytes;  // bytes per ring slot
   float out_scale;       // multiplies every final (element-typed) sum; 1 = plain sum
+  uint32_t hook;         // PL_HOOK_* bits (host side: selects the kernel variant; device: what final ops do)
   uint32_t hints;        // L2 policy bits for bulk copies: 1 loads evict-first, 2 stores evict-first, 4 copy loads evict-last
   uint32_t overlap_launch;  // host side only: launch with the programmatic stream serialization attribute
   uint32_t bcast_copies;      // host side only: the schedule holds broadcast copy ops (register executor variant)
@@ -124,6 +126,7 @@ struct Lowered {
   uint64_t scratch_per_rank[PL_MAX_RANKS] = {0};
   uint64_t in_bytes[PL_MAX_RANKS] = {0};
   uint64_t out_bytes[PL_MAX_RANKS] = {0};
+  uint64_t aux_bytes[PL_MAX_RANKS] = {0};
   uint64_t message_bytes = 0;
   int n_layers = 1;
   int role_queues[4] = {0, 0, 0, 0};  // queues per rank reserved for each role (0 = roles unused)
@@ -140,6 +143,7 @@ struct BuildRequest {
   bool staged;               // stage through schedule-owned memory (ordinary application buffers)
   uint64_t staging_bytes;    // staging capacity per rank (0 = default)
   int packet_ctas_per_rank;  // > 0: layered all-reduce on the packet datapath with this many CTAs per rank
+  uint32_t hook;             // PL_HOOK_* bits
   Policy pol;
 };
 

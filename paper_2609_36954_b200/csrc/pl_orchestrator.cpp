@@ -843,7 +843,54 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
   return p;
 }
 
+namespace {
+pl_status_t lower_collective(const BuildRequest& rq, Lowered* L, std::string* err);
+
+// Processing phase (PL_HOOK_*): mark the reduce ops that write final output, give their
+// destinations the output type, size the second operand.  Only collectives whose outputs are
+// written by reduce ops alone qualify: a result that is copied on cannot differ per rank.
+pl_status_t apply_hooks(const BuildRequest& rq, Lowered* L, std::string* err) {
+  auto fail = [&](pl_status_t st, const char* m) {
+    if (err) *err = m;
+    return st;
+  };
+  const int es = elem_size(rq.dtype);
+  if (rq.dtype != PL_BF16 && rq.dtype != PL_F32) return fail(PL_ERR_UNSUPPORTED, "processing hooks need a float element type");
+  if ((rq.hook & PL_HOOK_F32_OUT) && rq.dtype != PL_BF16) return fail(PL_ERR_UNSUPPORTED, "fp32 output is for bf16 schedules");
+  if (rq.packet_ctas_per_rank > 0) return fail(PL_ERR_UNSUPPORTED, "processing hooks are not offered on the packet datapath");
+  for (const HostOp& op : L->ops) {
+    bool touches_out = op.kind == PL_OP_COPY && op.dst.buf == PL_BUF_OUT;
+    for (const pl_ref_t& s : op.src) touches_out = touches_out || s.buf == PL_BUF_OUT;
+    if (touches_out)
+      return fail(PL_ERR_UNSUPPORTED, "processing hooks need a collective whose outputs are written by its reduce ops only "
+                                      "(reduce-scatter, one-shot or fused all-reduce, rooted reduce)");
+  }
+  const bool f32 = rq.hook & PL_HOOK_F32_OUT;
+  for (HostOp& op : L->ops) {
+    if (op.dst.buf != PL_BUF_OUT) continue;
+    if (op.dst.dtype != rq.dtype) return fail(PL_ERR_UNSUPPORTED, "an op writes non-element-typed output");
+    op.final_hook = true;
+    if (f32) {
+      op.dst.dtype = PL_F32;
+      op.dst.offset = op.dst.offset / es * 4;
+    }
+  }
+  for (int r = 0; r < rq.R; ++r) {
+    if (rq.hook & PL_HOOK_RESIDUAL) L->aux_bytes[r] = L->out_bytes[r];  // element-typed, laid out like the output
+    if (f32) L->out_bytes[r] = L->out_bytes[r] / es * 4;
+  }
+  return PL_OK;
+}
+}  // namespace
+
 pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
+  pl_status_t st = lower_collective(rq, L, err);
+  if (st == PL_OK && rq.hook) st = apply_hooks(rq, L, err);
+  return st;
+}
+
+namespace {
+pl_status_t lower_collective(const BuildRequest& rq, Lowered* L, std::string* err) {
   const int R = rq.R, dt = rq.dtype, es = elem_size(dt);
   auto fail = [&](pl_status_t st, const char* m) {
     if (err) *err = m;
@@ -1057,6 +1104,7 @@ pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
     default: return fail(PL_ERR_INVALID_ARG, "unknown collective");
   }
 }
+}  // namespace
 
 // Place ops on queues.  Rank r owns queues {q : q % R == r}; its ops go, in topological
 // order, to the least-loaded of its queues (ties to the lowest queue).  Each queue's order is
@@ -1230,7 +1278,7 @@ pl_status_t validate(const Lowered& L, int R, std::string* err, bool bulk_datapa
     bool plain = true;
     for (const pl_ref_t& r : o.src)
       if (r.dtype != o.dst.dtype) plain = false;
-    return (o.bcast && plain) ? 1 : 0;
+    return (o.bcast && plain && !o.final_hook) ? 1 : 0;
   };
   // a_writes: the access of op a that must be complete is a write (else a read);
   // x_reads: the access of op x that must come later is a read (else a write).

@@ -48,8 +48,10 @@ def _store(buf, off, vals, dtype):
     buf[off:off + raw.size] = raw
 
 
-def run(ops, info, R, ins, seed=0, max_steps=None):
-    """ins[r]: numpy arrays (any dtype).  Returns list of uint8 output buffers."""
+def run(ops, info, R, ins, seed=0, max_steps=None, aux=None, scale=1.0, elem_dtype=None):
+    """ins[r]: numpy arrays (any dtype).  Returns list of uint8 output buffers.  aux / scale /
+    elem_dtype: second operand per rank (element-typed, laid out like the output), output scale and
+    element type of a schedule with a processing phase (applied by ops flagged final)."""
     rng = random.Random(seed)
     bufs = {B.PL_BUF_IN: [np.ascontiguousarray(a).view(np.uint8).reshape(-1) for a in ins],
             B.PL_BUF_OUT: [np.full(int(info.out_bytes[r]), 0xFF, np.uint8) for r in range(R)],
@@ -93,9 +95,16 @@ def run(ops, info, R, ins, seed=0, max_steps=None):
                 s = op.src[k]
                 acc = acc + _load(bufs[s.buf][s.rank], int(s.offset), n, s.dtype)
             result, rdt = acc, op.dst.dtype
-        targets = range(R) if op.dst_bcast else [op.dst.rank]
+        targets = range(R) if (op.dst_bcast & 1) else [op.dst.rank]
+        final = bool(op.dst_bcast & 2)
         for r in targets:
-            _store(bufs[op.dst.buf][r], int(op.dst.offset), result, rdt)
+            val = result
+            if final:
+                val = np.float64(scale) * result.astype(np.float64)
+                if aux is not None:  # the second operand is element-typed and indexed like the (unconverted) output
+                    e_off = int(op.dst.offset) // _ES[rdt] * _ES[elem_dtype]
+                    val = val + _load(np.ascontiguousarray(aux[r]).view(np.uint8).reshape(-1), e_off, n, elem_dtype).astype(np.float64)
+            _store(bufs[op.dst.buf][r], int(op.dst.offset), val, rdt)
         for f in (op.signal_flag, op.signal_flag2):
             if f >= 0:
                 flags[f] += 1

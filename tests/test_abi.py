@@ -28,7 +28,7 @@ def test_struct_layouts_match_header_sizes():
     # sizes implied by the header's field lists (natural alignment, LP64)
     assert ctypes.sizeof(B.pl_ref_t) == 24
     assert ctypes.sizeof(B.pl_op_t) == 40 + 8 + 24 + 24 * 16 + 4 * 16 + 4 * 16
-    assert ctypes.sizeof(B.pl_bufs_t) == 4 * 16 * 8
+    assert ctypes.sizeof(B.pl_bufs_t) == 6 * 16 * 8
     assert ctypes.sizeof(B.pl_devstatus_t) == 32
     assert ctypes.sizeof(B.pl_sched_opts_t) == 64
 

@@ -11,6 +11,7 @@ import pytest
 
 from oracle import oracle
 from paper_2609_36954_b200 import inputs
+from paper_2609_36954_b200 import inputs as gen
 
 
 # ----------------------------------------------------------------------------- #
@@ -427,3 +428,38 @@ def test_moe_dedup_dispatch_and_combine():
     for r in range(R):
         n = int(a["counts"][:, r].sum())
         assert np.array_equal(a["recv"][r][:n], b["recv"][r][:n]) and np.array_equal(a["counts"], b["counts"])
+
+
+# ---- processing phase: scale, second operand, unconverted output ---------------------------------
+def test_processed_sum_closed_forms():
+    """Pins that a dropped term, a wrong sign or a scale applied to the wrong operand would break:
+    residual = -sum gives exactly zero; equal inputs give R * x exactly (so the fp32 image of the
+    result is R * x bit for bit); scale 1/R on equal inputs returns x; the residual is NOT scaled."""
+    R, n = 8, 64
+    ints = [gen.f32_to_bf16_bits(((np.arange(n) % 7) - 3 + r).astype(np.float32)) for r in range(R)]  # small integers: exact
+    exact = sum(gen.bf16_bits_to_f64(a) for a in ints)
+    res = [gen.f32_to_bf16_bits((-exact).astype(np.float32)) for _ in range(R)]
+    assert np.array_equal(gen.bf16_bits_to_f64(res[0]), -exact)          # representable: |sum| <= 88
+    out = oracle.allreduce_processed(ints, "bf16", 1.0, res)
+    for r in range(R):
+        assert np.all(out[r] == 0.0)
+    x = gen.normal_bf16(n, 3, 0)
+    same = [x.copy() for _ in range(R)]
+    out = oracle.allreduce_processed(same, "bf16")
+    assert np.array_equal(out[0], R * gen.bf16_bits_to_f64(x))
+    assert np.array_equal(out[0].astype(np.float32).astype(np.float64), out[0])   # exact in fp32: R is a power of two
+    out = oracle.allreduce_processed(same, "bf16", 1.0 / R)
+    assert np.array_equal(out[5], gen.bf16_bits_to_f64(x))
+    # scale applies to the sum only: with a zero sum the output is the second operand itself
+    zero = [np.zeros(n, np.uint16) for _ in range(R)]
+    aux = [gen.normal_bf16(n, 4, r) for r in range(R)]
+    out = oracle.allreduce_processed(zero, "bf16", 0.125, aux)
+    for r in range(R):
+        assert np.array_equal(out[r], gen.bf16_bits_to_f64(aux[r]))
+    # reduce-scatter form: rank r gets partition r, its own second operand, laid out like its output
+    xs = [gen.normal_f32(R * 16, 9, r) for r in range(R)]
+    aux = [gen.normal_f32(16, 10, r) for r in range(R)]
+    out = oracle.reduce_scatter_processed(xs, "f32", 0.5, aux)
+    stacked = np.stack([a.astype(np.float64) for a in xs]).sum(axis=0)
+    for r in range(R):
+        assert np.allclose(out[r], 0.5 * stacked[r * 16:(r + 1) * 16] + aux[r].astype(np.float64), rtol=0, atol=1e-12)

@@ -248,6 +248,70 @@ def test_packet_schedule_rejections():
         pu.close()
 
 
+@pytest.mark.parametrize("hook", [B.PL_HOOK_RESIDUAL, B.PL_HOOK_F32_OUT, B.PL_HOOK_RESIDUAL | B.PL_HOOK_F32_OUT])
+def test_processing_hooks_lowering_and_replay(hook):
+    """Schedules with a processing phase: the reduce ops that write output are flagged final, fp32
+    output doubles the output bytes and offsets of a bf16 schedule, the second operand is sized like
+    the element-typed output; replayed on the CPU the schedule gives scale * sum + aux."""
+    R, dtype = 4, "bf16"
+    n = R * 8 * 5
+    scale = 0.25
+    x = [gen.normal_bf16(n, 0, r) for r in range(R)]
+    pl = Planner(R, dtype)
+    try:
+        cases = [(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n // R), (B.PL_REDUCE_SCATTER, B.PL_ALGO_RING, n // R),
+                 (B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT, n), (B.PL_ALLREDUCE, B.PL_ALGO_DIRECT_FUSED, n)]
+        for coll, algo, n_out in cases:
+            s = pl.build(coll, algo, n, 32, hook=hook, out_scale=scale, slice_bytes=16)
+            info = B.pl_schedule_info(s)
+            f32 = bool(hook & B.PL_HOOK_F32_OUT)
+            assert info.hook == hook and info.out_dtype == (B.PL_F32 if f32 else B.PL_BF16)
+            for r in range(R):
+                assert info.out_bytes[r] == n_out * (4 if f32 else 2)
+                assert info.aux_bytes[r] == (n_out * 2 if hook & B.PL_HOOK_RESIDUAL else 0)
+            ops = B.pl_schedule_dump(s)
+            finals = [o for o in ops if o.dst_bcast & 2]
+            assert finals and all(o.kind != B.PL_OP_COPY and o.dst.buf == B.PL_BUF_OUT for o in finals)
+            assert all(bool(o.dst_bcast & 2) == (o.dst.buf == B.PL_BUF_OUT) for o in ops)
+            assert all(o.dst.dtype == (B.PL_F32 if f32 else B.PL_BF16) for o in finals)
+            aux = [gen.normal_bf16(n_out, 5, r) for r in range(R)] if hook & B.PL_HOOK_RESIDUAL else None
+            outs = interp_run(ops, info, R, x, seed=3, aux=aux, scale=scale, elem_dtype=B.PL_BF16)
+            ref = (oracle.allreduce_processed if coll == B.PL_ALLREDUCE else oracle.reduce_scatter_processed)(x, dtype, scale, aux)
+            for r in range(R):
+                got = outs[r].view(np.float32).astype(np.float64) if f32 else gen.bf16_bits_to_f64(outs[r].view(np.uint16))
+                check_float(got, ref[r], "bf16")
+    finally:
+        pl.close()
+
+
+def test_processing_hooks_rejections():
+    pl = Planner(4, "bf16")
+    try:
+        for algo in (B.PL_ALGO_RING, B.PL_ALGO_TREE, B.PL_ALGO_DIRECT):   # all-reduces that end with copies
+            with pytest.raises(B.PurlinError) as e:
+                pl.build(B.PL_ALLREDUCE, algo, 1024, 256, hook=B.PL_HOOK_RESIDUAL)
+            assert e.value.status == B.PL_ERR_UNSUPPORTED
+        with pytest.raises(B.PurlinError) as e:
+            pl.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, 1024, 256, hook=B.PL_HOOK_F32_OUT)
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+        with pytest.raises(B.PurlinError) as e:
+            pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, 1024, 256, hook=8)
+        assert e.value.status == B.PL_ERR_INVALID_ARG
+        with pytest.raises(B.PurlinError) as e:
+            B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_ONESHOT, 1024, 2, B.make_opts(datapath=B.PL_DP_PACKET, hook=B.PL_HOOK_RESIDUAL))
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+    finally:
+        pl.close()
+    for dt, hook in (("i32", B.PL_HOOK_RESIDUAL), ("f32", B.PL_HOOK_F32_OUT)):
+        p2 = Planner(4, dt)
+        try:
+            with pytest.raises(B.PurlinError) as e:
+                p2.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, 1024, 256, hook=hook)
+            assert e.value.status == B.PL_ERR_UNSUPPORTED
+        finally:
+            p2.close()
+
+
 def test_config1_op_counts_and_bytes():
     # all-reduce, R=4, 262144 fp32 per rank, ring, 64 KiB chunks, unsliced:
     # 3 reduce-scatter hops + 3 all-gather hops, 4 ranks, 4 chunks per partition
