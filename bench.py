@@ -390,6 +390,21 @@ def measure_all_configs(peak):
         "all_gather_ring": entry(b.collective("C2-AG", 8, B.PL_BF16, B.PL_ALLGATHER, "ring", 4 * MIB, 256 << 10)),
         "all_to_all": entry(b.collective("A2A", 8, B.PL_BF16, B.PL_ALLTOALL, "direct", 32 * MIB, MIB)),
     }
+    # staged schedules (ordinary application buffers), back-to-back executes without events in between:
+    # one staging buffer, overlapped launches, two buffers alternated by launch parity (stage ahead)
+    out["staged_back_to_back"] = {}
+    for label, coll, count in (("allreduce_64MiB", B.PL_ALLREDUCE, 32 * MIB), ("reduce_scatter_64MiB", B.PL_REDUCE_SCATTER, 32 * MIB),
+                               ("allreduce_1MiB", B.PL_ALLREDUCE, MIB // 2)):
+        out["staged_back_to_back"][label] = {}
+        for name, fl in (("one_buffer", B.PL_OPT_STAGED), ("one_buffer_overlapped_launches", B.PL_OPT_STAGED | B.PL_OPT_OVERLAP_LAUNCH),
+                         ("two_buffers_stage_ahead", B.PL_OPT_STAGED | B.PL_OPT_OVERLAP_LAUNCH | B.PL_OPT_STAGE_AHEAD)):
+            rec = b.collective("staged", 8, B.PL_BF16, coll, "direct", count, max(16, min(MIB, count * 2 // 8)), iters=50, back_to_back=True, flags=fl)
+            out["staged_back_to_back"][label][name] = entry(rec)
+    # processing phase folded into the reduce (scale, residual, fp32 output): fused all-reduce, 64 MiB per rank
+    out["processing_phase"] = {}
+    for name, kw in (("plain", {}), ("scale", dict(out_scale=0.125)), ("scale_residual", dict(out_scale=0.125, hook=B.PL_HOOK_RESIDUAL)),
+                     ("f32_out", dict(hook=B.PL_HOOK_F32_OUT))):
+        out["processing_phase"][name] = entry(b.collective("hook", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "direct", 32 * MIB, MIB, **kw))
     # C4: MoE dispatch / combine at the full shape, both routings
     out["C4"] = {}
     for name, ident in (("permuted", False), ("identity", True)):

@@ -104,7 +104,8 @@ class Bench:
             self.out.write(line + "\n")
             self.out.flush()
 
-    def collective(self, cfg, R, dtype, coll, algo, count, chunk, iters=20, layers=0, graph=False, root=None, **kw):
+    def collective(self, cfg, R, dtype, coll, algo, count, chunk, iters=20, layers=0, graph=False, root=None,
+                   back_to_back=False, **kw):
         comm = B.pl_comm_create(R, dtype)
         okw = dict(self.opts_kw)
         okw.update(kw)
@@ -123,9 +124,12 @@ class Bench:
         info = B.pl_schedule_info(s)
         d_in = [_fill(int(info.in_bytes[r]), r) for r in range(R)]
         d_out = [torch.empty(max(16, int(info.out_bytes[r])), dtype=torch.uint8, device="cuda") for r in range(R)]
+        d_aux = [_fill(int(info.aux_bytes[r]), 100 + r) for r in range(R)] if any(info.aux_bytes[r] for r in range(R)) else None
         bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
-                           [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
-        p50, p10, p90 = _time(lambda: B.pl_execute(s, bufs, self.stream), iters, per_call_events=True)
+                           [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)],
+                           [t.data_ptr() for t in d_aux] if d_aux else None, [int(info.aux_bytes[r]) for r in range(R)] if d_aux else None)
+        # back_to_back: no event between the launches, so that overlapped launches can overlap
+        p50, p10, p90 = _time(lambda: B.pl_execute(s, bufs, self.stream), iters, per_call_events=not back_to_back)
         graph_us = None
         if graph:
             graph_us = _time_graph(lambda h: B.pl_execute(s, bufs, h)) / max(1, layers)
@@ -291,6 +295,15 @@ def main(args=None):
             for size in (MIB, 16 * MIB, 64 * MIB, 256 * MIB):
                 b.collective("staged-AR cap=%d" % cap, 8, B.PL_BF16, B.PL_ALLREDUCE, "direct", size // 2,
                              max(16, min(MIB, size // 8)), iters=10, **kw)
+    if "stage_ahead" in which:
+        # back-to-back staged executes: one staging buffer, overlapped launches, and two staging
+        # buffers alternated by launch parity with the stage role running ahead (Sec. 4.1-4.2)
+        for name, coll, count in (("AR", B.PL_ALLREDUCE, 32 * MIB), ("RS", B.PL_REDUCE_SCATTER, 32 * MIB), ("AR-1MiB", B.PL_ALLREDUCE, MIB // 2),
+                                  ("AR-16MiB", B.PL_ALLREDUCE, 8 * MIB)):
+            for label, fl in (("one buffer", B.PL_OPT_STAGED), ("one buffer, overlapped launches", B.PL_OPT_STAGED | B.PL_OPT_OVERLAP_LAUNCH),
+                              ("two buffers, stage ahead", B.PL_OPT_STAGED | B.PL_OPT_OVERLAP_LAUNCH | B.PL_OPT_STAGE_AHEAD)):
+                b.collective("staged-%s %s" % (name, label), 8, B.PL_BF16, coll, "direct", count, max(16, min(MIB, count * 2 // 8)), iters=50,
+                             back_to_back=True, flags=fl)
     if "rooted" in which:
         for size in (64 * 1024, 64 * MIB):
             for name, coll, count in (("broadcast", B.PL_BROADCAST, size // 2), ("reduce", B.PL_REDUCE, size // 2),

@@ -201,9 +201,8 @@ typedef struct {
  * its reduced chunks Y_k[c] in staging and the gather role publishes consumed(r,k,c).  Staging
  * holds staging_bytes per rank: when the message needs more, chunk slots are reused cyclically
  * (Sec. 4.1) and a stage op waits until the slot's previous chunk has been consumed.  Only
- * PL_ALGO_DIRECT.  (The paper alternates two staging buffers by epoch parity so that a rank
- * can start the next call early; here a launch ends only when every rank has drained, so one
- * buffer is enough.) */
+ * PL_ALGO_DIRECT.  One staging buffer per rank, unless PL_OPT_STAGE_AHEAD asks for the paper's
+ * two buffers alternated by epoch parity. */
 #define PL_OPT_STAGED 4u
 /* Record, for every op, when its waits were satisfied and when its signal was about to be
  * released (%globaltimer, ns) into a schedule-owned buffer: see pl_schedule_trace_read. */
@@ -215,6 +214,19 @@ typedef struct {
  * data).  Shortens back-to-back executes; no effect after any other kind of work.  The paper
  * has no counterpart (it measures calls inside a CUDA graph, Sec. 5). */
 #define PL_OPT_OVERLAP_LAUNCH 16u
+/* Epoch-parity double buffering of the staging memory (Sec. 4.1-4.2: two staging buffers
+ * alternated by the parity of a persistent epoch, so that a rank can enter call n+1 while peers
+ * still consume call n).  Needs PL_OPT_STAGED and PL_OPT_OVERLAP_LAUNCH.  The schedule owns two
+ * staging buffers and two flag sets per rank; launch i uses set i mod 2 (the launch number is a
+ * device-resident counter taken at kernel entry, so CUDA-graph replays stay consistent).  The
+ * stage role of execute n+1 -- the leading stage ops of a queue that wait for nothing: they only
+ * read the caller's inputs and write the other staging buffer -- runs BEFORE the kernel waits for
+ * execute n to complete; everything else runs after it.  The caller promises that the inputs of
+ * an execute are not written by the launch directly in front of it on the stream (an execute
+ * that consumes the previous execute's outputs must not use this option).  The paper advances
+ * its epoch by the chunk count rounded to an odd number so that the parity flips on every call;
+ * here the launch counter itself is the epoch and its lowest bit the parity. */
+#define PL_OPT_STAGE_AHEAD 32u
 #define PL_OPT_NO_L2_HINTS 2u  /* bulk copies without L2 eviction hints (default: stores evict-first,
                                   sources of copy ops evict-last; measured 7 % on all-gather) */
 
@@ -242,6 +254,8 @@ typedef struct {
   int32_t signal_flag2;/* optional second flag incremented the same way, -1 none */
   int32_t dst_bcast;   /* 1: dst is replicated at the same offset into out[0..R); 3: and the op is final */
                        /* bit 1 (value 2): the op writes final output and runs the processing phase    */
+                       /* bit 2 (value 4): stage op that PL_OPT_STAGE_AHEAD may run before the launch  */
+                       /* in front has completed                                                       */
   uint64_t count;      /* elements; COPY ops count bytes (dtype PL_U8) */
   pl_ref_t dst;
   pl_ref_t src[PL_MAX_SRC];

@@ -38,6 +38,7 @@ PL_OPT_NO_L2_HINTS = 2
 PL_OPT_STAGED = 4
 PL_OPT_TRACE = 8
 PL_OPT_OVERLAP_LAUNCH = 16
+PL_OPT_STAGE_AHEAD = 32
 PL_HOOK_RESIDUAL = 1
 PL_HOOK_F32_OUT = 2
 

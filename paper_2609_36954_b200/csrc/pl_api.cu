@@ -41,6 +41,8 @@ struct pl_schedule_s {
   bool overlap_launch = false;
   bool bcast_copies = false;      // some COPY op writes every rank's output
   bool pipelined_reduce = false;  // bulk-copy datapath: every reduce op is plain, run the 12-warp variant
+  bool stage_ahead = false;       // double-buffered staging: two scratch halves and flag sets, chosen by launch parity
+  uint64_t scratch_half = 0;      // bytes of one half (all ranks)
   int packet_ctas_per_rank = 0;   // > 0: packet datapath (layered one-shot all-reduce), CTAs per rank
   long long packet_break_op = -1; // test hook (pl_schedule_debug_break_wait on a packet schedule)
   size_t off_trace = 0;
@@ -87,7 +89,7 @@ void fill_info(pl_schedule_s* S, int R) {
   }
   I.message_bytes = L.message_bytes;
   for (int r = 0; r < R; ++r) {
-    I.scratch_bytes += L.scratch_per_rank[r];
+    I.scratch_bytes += L.scratch_per_rank[r] * (S->stage_ahead ? 2 : 1);
     I.in_bytes[r] = L.in_bytes[r];
     I.out_bytes[r] = L.out_bytes[r];
     I.aux_bytes[r] = L.aux_bytes[r];
@@ -140,7 +142,7 @@ void flatten(pl_schedule_s* S, int dtype) {
     d.signal = op.signal >= 0 ? (uint32_t)op.signal : kNoFlag;
     d.signal2 = op.signal2 >= 0 ? (uint32_t)op.signal2 : kNoFlag;
     d.flags = (op.bcast ? kDstBcast : 0u) | ((op.kind != PL_OP_COPY && op.dst.dtype != dtype) ? kDstF32 : 0u) |
-              (op.final_hook ? kFinal : 0u);
+              (op.final_hook ? kFinal : 0u) | (op.stage_ahead ? kStageAhead : 0u);
     d.count = op.count;
     d.dst = pack(*S, op.dst);
     d.topo = (uint32_t)op.topo;
@@ -163,8 +165,8 @@ pl_status_t upload(pl_schedule_s* S, int R) {
   S->off_ops = place(S->dev_ops.size() * sizeof(DevOp));
   S->off_srcs = place(S->srcs.size() * sizeof(uint64_t));
   S->off_waits = place(S->waits.size() * sizeof(DevWait));
-  S->off_flags = place((size_t)std::max(1, S->L.n_flags) * sizeof(unsigned long long));
-  S->off_epoch = place(2 * sizeof(unsigned long long));
+  S->off_flags = place((size_t)std::max(1, S->L.n_flags) * sizeof(unsigned long long) * (S->stage_ahead ? 2 : 1));
+  S->off_epoch = place(4 * sizeof(unsigned long long));
   S->sync_bytes = off - S->off_flags;
   if (S->trace) S->off_trace = place(2 * S->L.ops.size() * sizeof(unsigned long long));
   S->blob_bytes = off;
@@ -181,6 +183,10 @@ pl_status_t upload(pl_schedule_s* S, int R) {
   for (int r = 0; r < R; ++r) {
     S->scratch_off[r] = total;
     total += align_up(S->L.scratch_per_rank[r], 256);
+  }
+  if (S->stage_ahead) {  // second staging buffer of every rank, one half behind the first
+    S->scratch_half = total;
+    total *= 2;
   }
   S->scratch_total = total;
   if (total) {
@@ -307,6 +313,11 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   rq.R = comm->R;
   rq.dtype = comm->dtype;
   rq.hook = hook;
+  rq.stage_ahead = (flags & PL_OPT_STAGE_AHEAD) != 0;
+  if (rq.stage_ahead && (!(flags & PL_OPT_STAGED) || !(flags & PL_OPT_OVERLAP_LAUNCH) || (flags & PL_OPT_TRACE) || hook)) {
+    comm->last_error = "PL_OPT_STAGE_AHEAD needs PL_OPT_STAGED and PL_OPT_OVERLAP_LAUNCH (and neither trace nor hooks)";
+    return PL_ERR_INVALID_ARG;
+  }
   if (pol.datapath == PL_DP_PACKET && hook) {
     comm->last_error = "processing hooks are not offered on the packet datapath";
     return PL_ERR_UNSUPPORTED;
@@ -343,6 +354,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   S->no_l2_hints = (flags & PL_OPT_NO_L2_HINTS) != 0;
   S->trace = (flags & PL_OPT_TRACE) != 0;
   S->overlap_launch = (flags & PL_OPT_OVERLAP_LAUNCH) != 0;
+  S->stage_ahead = (flags & PL_OPT_STAGE_AHEAD) != 0;
   S->out_scale = out_scale;
   S->hook = hook;
   std::string err;
@@ -572,7 +584,7 @@ pl_status_t pl_schedule_dump(pl_schedule_t s, pl_op_t* ops, size_t cap, size_t* 
     o.n_wait = (int32_t)h.waits.size();
     o.signal_flag = h.signal;
     o.signal_flag2 = h.signal2;
-    o.dst_bcast = (h.bcast ? 1 : 0) | (h.final_hook ? 2 : 0);
+    o.dst_bcast = (h.bcast ? 1 : 0) | (h.final_hook ? 2 : 0) | (h.stage_ahead ? 4 : 0);
     o.count = h.count;
     o.dst = h.dst;
     for (size_t k = 0; k < h.src.size(); ++k) o.src[k] = h.src[k];
@@ -721,6 +733,9 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
     P.base[kSlotAux + r] = s->info.aux_bytes[r] ? const_cast<void*>(bufs->aux[r]) : nullptr;
   }
   P.hook = s->hook;
+  P.stage_ahead = s->stage_ahead ? 1u : 0u;
+  P.n_flags = (uint32_t)s->L.n_flags;
+  P.scratch_half = s->scratch_half;
   P.ops = reinterpret_cast<const DevOp*>(s->d_blob + s->off_ops);
   P.n_queues = (uint32_t)s->pol.n_ctas;
   P.srcs = reinterpret_cast<const uint64_t*>(s->d_blob + s->off_srcs);

@@ -10,6 +10,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
+
 #include "pl_device.cuh"
 #include "pl_internal.h"
 #include "pl_kernels.h"
@@ -112,14 +114,13 @@ __device__ __forceinline__ void reduce_units(const ExecParams& P, const char* co
 // REDUCE with n same-typed sources -> element-typed destination (optionally replicated to
 // every rank's output).  s_src holds the resolved source pointers in shared memory.
 template <int DT, bool HOOK>
-__device__ __forceinline__ void body_reduce(const ExecParams& P, const DevOp& op, const char* const* s_src, int tid,
+__device__ __forceinline__ void body_reduce(const ExecParams& P, const DevOp& op, const char* const* s_src, char* dst, int tid,
                                             int nthr) {
   constexpr int U = 2;
   const uint64_t dst_slot = op.dst >> 48;
   const bool final_op = op.flags & kFinal;
   const uint64_t n_units = op.count / Acc<DT>::kElems;  // 16 bytes of every operand each
   const bool bcast = op.flags & kDstBcast;
-  char* dst = resolve(P, op.dst);
   const uint64_t dst_off = op.dst & 0xFFFFFFFFFFFFull;
   const int ns = op.n_src;
   uint64_t base = tid;
@@ -156,10 +157,9 @@ __device__ __forceinline__ void body_copy_reduce_final(const ExecParams& P, cons
 }
 
 template <int DT>
-__device__ __forceinline__ void body_copy_reduce(const ExecParams& P, const DevOp& op, const char* const* s_src,
+__device__ __forceinline__ void body_copy_reduce(const ExecParams& P, const DevOp& op, const char* const* s_src, char* dst,
                                                  int tid, int nthr) {
   const uint64_t n_units = op.count / Acc<DT>::kElems;
-  char* dst = resolve(P, op.dst);
   const char* a = s_src[0];
   const char* b = s_src[1];
   if constexpr (DT == PL_I32) {
@@ -267,19 +267,25 @@ struct OpSlot {
 // HOOK: the variant for schedules with a processing phase beyond the scale (PL_HOOK_*): its
 // final reduce ops add the second operand and / or keep fp32.  A kernel of its own for the
 // same reason as BC: the plain variants keep the code they have.
-template <int DT, bool BC, bool HOOK = false>
+// DBUF: the variant for staged schedules with two staging buffers (PL_OPT_STAGE_AHEAD): flag set
+// and staging buffer follow the parity of a launch counter taken at entry, and the leading
+// stage ops of a queue run before the kernel waits for the launch in front of it.
+template <int DT, bool BC, bool HOOK = false, bool DBUF = false>
 __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_constant__ ExecParams P) {
   __shared__ OpSlot s_slot[2];
   __shared__ int s_abort[2];  // indexed by iteration parity: written during wait i, read after barrier i
+  __shared__ unsigned long long s_launch;
   const int tid = threadIdx.x, nthr = blockDim.x, q = blockIdx.x;
   const uint32_t nq = P.n_queues;
   // every CTA reads the epoch before it reports completion, and the epoch word is only
   // advanced after all CTAs reported, so all of them see the same value; a schedule without
   // flags needs no epoch at all
   const bool has_flags = P.flags != nullptr;
-  pdl_launch_dependents();
+  if constexpr (!DBUF) pdl_launch_dependents();
   if (tid == 0) s_abort[0] = s_abort[1] = 0;
   bool aborted = false;
+  unsigned long long scratch_shift = 0ull;       // DBUF: distance to this launch's staging buffer
+  const unsigned long long* flag_base = P.flags;  // DBUF: this launch's flag set
 
   // descriptor fetch by warp 0: lanes 0-3 carry the op, lane k source k and wait entry k
   auto fetch = [&](uint32_t i, uint4& r_op, uint64_t& r_src, DevWait& r_wait) {
@@ -290,7 +296,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   };
   auto stash = [&](int slot, const uint4& r_op, uint64_t r_src, const DevWait& r_wait) {
     if (tid < 4) reinterpret_cast<uint4*>(&s_slot[slot].op)[tid] = r_op;
-    if (tid < (int)P.src_stride) s_slot[slot].src[tid] = resolve(P, r_src);
+    if (tid < (int)P.src_stride) s_slot[slot].src[tid] = DBUF ? resolve(P, r_src, scratch_shift) : resolve(P, r_src);
     if (tid < (int)P.wait_stride) s_slot[slot].wait[tid] = r_wait;
   };
 
@@ -298,8 +304,24 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   uint64_t r_src = 0;
   DevWait r_wait = {0, 0};
   if (tid < 32) fetch(0, r_op, r_src, r_wait);  // descriptors are immutable: fetched before the wait below
-  pdl_wait();
-  const unsigned long long epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
+  unsigned long long epoch;
+  bool waited = !DBUF;  // DBUF: griddepcontrol.wait is still to come (before the first op that is not an early stage op)
+  if constexpr (DBUF) {
+    // Launch number: every CTA of launch i takes its ticket before it lets launch i+1 start, so
+    // ticket / grid is i for all of them (also under graph replay).  Parity picks the flag set
+    // and the staging buffer; a set is used by every second launch, hence its own epoch i / 2.
+    if (tid == 0) s_launch = atomicAdd(P.epoch + 2, 1ull) / gridDim.x;
+    __syncthreads();
+    const unsigned long long launch = s_launch;
+    epoch = (launch >> 1) + 1ull;
+    if (launch & 1ull) {
+      scratch_shift = P.scratch_half;
+      flag_base = P.flags + P.n_flags;
+    }
+  } else {
+    pdl_wait();
+    epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
+  }
   if (tid < 32) stash(0, r_op, r_src, r_wait);
   __syncthreads();
   // the first descriptor tells how many ops the queue holds (a placeholder marks an empty one)
@@ -308,13 +330,22 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   for (uint32_t i = 0; i < n_ops; ++i) {
     const int slot = i & 1;
     OpSlot& S = s_slot[slot];
+    if constexpr (DBUF) {
+      // everything but the leading early-stage ops runs after the launch in front has completed;
+      // only then may the launch behind this one start (it shares this launch's other buffer)
+      if (!waited && !(S.op.flags & kStageAhead)) {
+        pdl_wait();
+        pdl_launch_dependents();
+        waited = true;
+      }
+    }
     if (tid < 32) {
       // ---- wait: lane k polls wait entry k (acquire), bounded by the time limit
       const uint32_t nw = S.op.n_wait;
       if (tid < (int)nw) {
         const DevWait w = S.wait[tid];
         const unsigned long long need = epoch * (unsigned long long)w.need;
-        const unsigned long long* fp = P.flags + w.flag;
+        const unsigned long long* fp = flag_base + w.flag;
         unsigned long long seen = ld_acquire_u64(fp);
         if (seen < need) {
           const unsigned long long t0 = globaltimer_ns();
@@ -340,19 +371,20 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
 
     const DevOp& op = S.op;
     if (P.trace && tid == 0) P.trace[2ull * op.topo] = globaltimer_ns();  // waits satisfied
+    char* const op_dst = DBUF ? resolve(P, op.dst, scratch_shift) : resolve(P, op.dst);
     if (op.kind == PL_OP_COPY) {
       if constexpr (BC) {
         if (op.flags & kDstBcast) body_copy_bcast(P, op.dst & 0xFFFFFFFFFFFFull, S.src[0], op.count, tid, nthr);
-        else body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
+        else body_copy(op_dst, S.src[0], op.count, tid, nthr);
       } else {
-        body_copy(resolve(P, op.dst), S.src[0], op.count, tid, nthr);
+        body_copy(op_dst, S.src[0], op.count, tid, nthr);
       }
     } else if (op.kind == PL_OP_REDUCE) {
-      if constexpr (DT != PL_U8) body_reduce<DT, HOOK>(P, op, S.src, tid, nthr);
+      if constexpr (DT != PL_U8) body_reduce<DT, HOOK>(P, op, S.src, op_dst, tid, nthr);
     } else {
       if constexpr (DT != PL_U8) {
         if (HOOK && (op.flags & kFinal)) body_copy_reduce_final<DT>(P, op, S.src, tid, nthr);
-        else body_copy_reduce<DT>(P, op, S.src, tid, nthr);
+        else body_copy_reduce<DT>(P, op, S.src, op_dst, tid, nthr);
       }
     }
 
@@ -361,8 +393,8 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
       if (tid == 0 && P.trace) P.trace[2ull * op.topo + 1] = globaltimer_ns();
       if (tid == 0 && op.signal != kNoFlag) {
         __threadfence();
-        red_release_add_u64(P.flags + op.signal, 1ull);
-        if (op.signal2 != kNoFlag) red_release_add_u64(P.flags + op.signal2, 1ull);
+        red_release_add_u64(const_cast<unsigned long long*>(flag_base) + op.signal, 1ull);
+        if (op.signal2 != kNoFlag) red_release_add_u64(const_cast<unsigned long long*>(flag_base) + op.signal2, 1ull);
       }
     }
     if (tid < 32 && has_next) {
@@ -371,8 +403,14 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
     }
   }
 
+  if constexpr (DBUF) {
+    if (!waited) {  // a queue of early stage ops only (or an empty one): still ordered behind the launch in front
+      pdl_wait();
+      pdl_launch_dependents();
+    }
+  }
   __syncthreads();
-  if (tid == 0 && !aborted && has_flags) {
+  if (tid == 0 && !aborted && has_flags && !DBUF) {
     // last CTA to finish advances the epoch for the next execute
     const unsigned long long prev = atomicAdd(P.epoch + 1, 1ull);
     if (prev == (unsigned long long)gridDim.x - 1ull) {
@@ -383,7 +421,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
   }
 }
 
-template <int DT, bool BC, bool HOOK = false>
+template <int DT, bool BC, bool HOOK = false, bool DBUF = false>
 cudaError_t launch_t(const ExecParams& P, int grid, int threads, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
@@ -394,7 +432,7 @@ cudaError_t launch_t(const ExecParams& P, int grid, int threads, cudaStream_t st
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = P.overlap_launch ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, pl_exec_kernel<DT, BC, HOOK>, P);
+  return cudaLaunchKernelEx(&cfg, pl_exec_kernel<DT, BC, HOOK, DBUF>, P);
 }
 
 }  // namespace
@@ -405,6 +443,14 @@ cudaError_t launch_exec(int dtype, const ExecParams& P, int grid, int threads, c
       case PL_BF16: return launch_t<PL_BF16, false, true>(P, grid, threads, stream);
       case PL_F32: return launch_t<PL_F32, false, true>(P, grid, threads, stream);
       default: return cudaErrorInvalidValue;
+    }
+  }
+  if (P.stage_ahead) {  // staged schedules: copies and plain reduces, no broadcast copies, no hooks (checked at build)
+    switch (dtype) {
+      case PL_BF16: return launch_t<PL_BF16, false, false, true>(P, grid, threads, stream);
+      case PL_F32: return launch_t<PL_F32, false, false, true>(P, grid, threads, stream);
+      case PL_I32: return launch_t<PL_I32, false, false, true>(P, grid, threads, stream);
+      default: return launch_t<PL_U8, false, false, true>(P, grid, threads, stream);
     }
   }
   if (P.bcast_copies) {
@@ -439,7 +485,12 @@ int occupancy_both(int threads) {
       return 0;
     }
   }
-  return a < b ? (a < c ? a : c) : (b < c ? b : c);
+  int d = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d, pl_exec_kernel<DT, false, false, true>, threads, 0) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return std::min(std::min(a, b), std::min(c, d));
 }
 }  // namespace
 

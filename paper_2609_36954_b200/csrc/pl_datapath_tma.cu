@@ -66,6 +66,7 @@ struct Ctrl {
   uint64_t done[kMaxStages];
   int abort;
   int pad;
+  unsigned long long launch;  // double-buffered staging: number of this launch (taken at entry by thread 0)
   StageDesc desc[kMaxStages];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
@@ -289,7 +290,11 @@ __device__ __forceinline__ bool leaves_via_smem(uint32_t kind, uint32_t flags, u
 }
 
 // HOOK: the variant for schedules with a processing phase beyond the scale (general consumers only).
-template <int DT, int CW, bool HOOK = false>
+// DBUF: the variant for staged schedules with two staging buffers (PL_OPT_STAGE_AHEAD): flag set
+// and staging buffer follow the parity of a launch counter taken at entry; the producer runs the
+// leading stage ops of its queue (copies from the caller's input into the staging buffer of this
+// parity) before it waits for the launch in front, the copier ships them, the consumers wait.
+template <int DT, int CW, bool HOOK = false, bool DBUF = false>
 __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __grid_constant__ ExecParams P) {
   extern __shared__ __align__(1024) unsigned char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
@@ -297,9 +302,10 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, q = blockIdx.x;
   const uint32_t S = (uint32_t)P.stages, slot_bytes = P.stage_bytes;
   const bool has_flags = P.flags != nullptr;
-  pdl_launch_dependents();
+  if constexpr (!DBUF) pdl_launch_dependents();
 
   if (tid == 0) {
+    if constexpr (DBUF) c->launch = atomicAdd(P.epoch + 2, 1ull) / gridDim.x;  // ticket: see the register executor
     for (uint32_t s = 0; s < S; ++s) {
       ptx::mbar_init(&c->full[s], 1);
       ptx::mbar_init(&c->empty[s], 1 + CW);  // copier + every consumer warp
@@ -308,9 +314,26 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
     c->abort = 0;
     ptx::mbar_init_fence();
   }
-  pdl_wait();  // from here on memory written by earlier launches may be read
-  const unsigned long long epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
-  __syncthreads();
+  unsigned long long epoch = 0ull, scratch_shift = 0ull;
+  unsigned long long* flag_base = P.flags;
+  if constexpr (DBUF) {
+    __syncthreads();
+    const unsigned long long launch = c->launch;
+    epoch = (launch >> 1) + 1ull;
+    if (launch & 1ull) {
+      scratch_shift = P.scratch_half;
+      flag_base = P.flags + P.n_flags;
+    }
+    // consumers only ever handle reduce stages, which come after the producer's wait: they may
+    // block here; the producer waits later (below), the copier not at all (it reads shared
+    // memory only, and what it stores or signals belongs to this launch's own buffer and flag set
+    // until the producer has waited)
+    if (warp >= 2) pdl_wait();
+  } else {
+    pdl_wait();  // from here on memory written by earlier launches may be read
+    epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
+    __syncthreads();
+  }
 
   if (warp == 0) {
     // ================================ producer =========================================
@@ -330,11 +353,21 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
     // the first descriptor tells how many ops the queue holds (a placeholder marks an empty one)
     const uint32_t first_kind = __shfl_sync(0xFFFFFFFFu, r_op_next.x, 0);
     const uint32_t n_ops = first_kind == kNopKind ? 0u : __shfl_sync(0xFFFFFFFFu, r_op_next.z, 0) + 1u;
+    bool waited = !DBUF;
     for (uint32_t i = 0; i < n_ops && ok; ++i) {
       r_op = r_op_next;
       r_src = r_src_next;
       r_wait = r_wait_next;
       if (i + 1 < n_ops) fetch(i + 1, r_op_next, r_src_next, r_wait_next);
+      if constexpr (DBUF) {
+        // the first op that is not an early stage op: wait for the launch in front, then let the
+        // launch behind start (it will write the staging buffer this launch's predecessor used)
+        if (!waited && !(__shfl_sync(0xFFFFFFFFu, r_op.w, 1) & kStageAhead)) {
+          pdl_wait();
+          pdl_launch_dependents();
+          waited = true;
+        }
+      }
       // op words: lane 0: kind n_src remaining pmask | lane 1: rsv n_wait signal flags | lane 2: count dst | lane 3: topo signal2
       const uint32_t kind = __shfl_sync(0xFFFFFFFFu, r_op.x, 0), n_src = __shfl_sync(0xFFFFFFFFu, r_op.y, 0);
       const uint32_t pmask = __shfl_sync(0xFFFFFFFFu, r_op.w, 0);
@@ -348,7 +381,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
       bool lane_ok = true;
       if (lane < (int)n_wait) {
         const unsigned long long need = epoch * (unsigned long long)r_wait.need;
-        const unsigned long long* fp = P.flags + r_wait.flag;
+        const unsigned long long* fp = flag_base + r_wait.flag;
         unsigned long long seen = ld_acquire_u64(fp);
         if (seen < need) {
           const unsigned long long t0 = globaltimer_ns();
@@ -371,7 +404,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
       if (P.trace && lane == 0) P.trace[2ull * topo] = globaltimer_ns();  // waits satisfied
 
       // ---- cut the op into stages
-      const char* my_src = (lane < (int)n_src) ? resolve(P, r_src) : nullptr;
+      const char* my_src = (lane < (int)n_src) ? (DBUF ? resolve(P, r_src, scratch_shift) : resolve(P, r_src)) : nullptr;
       const bool my_part = (pmask >> lane) & 1u;
       const uint32_t unit_b = (kind == PL_OP_COPY) ? 16u : 16u * (n_src + __popc(pmask));  // slot bytes per unit
       uint32_t ucap = slot_bytes / unit_b;
@@ -385,7 +418,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
       const uint32_t my_w = my_part ? 32u : 16u;
       const uint32_t my_tile_off = ucap * 16u * (lane + __popc(pmask & ((1u << lane) - 1u)));
       const uint32_t dst_w = (kind == PL_OP_COPY) ? 16u : ((oflags & kDstF32) ? 32u : 16u);
-      char* dst = resolve(P, dstp);
+      char* dst = DBUF ? resolve(P, dstp, scratch_shift) : resolve(P, dstp);
       const uint64_t dst_off = dstp & 0xFFFFFFFFFFFFull;
       for (uint64_t u0 = 0; u0 < n_units; u0 += ucap) {
         const uint32_t units = (uint32_t)min((uint64_t)ucap, n_units - u0);
@@ -402,8 +435,9 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
           d.ucap = ucap;
           d.pmask = pmask;
           d.flags = oflags | ((u0 + ucap >= n_units) ? kLastOfOp : 0u);
-          d.signal = signal;
-          d.signal2 = signal2;
+          // signals go to this launch's flag set
+          d.signal = (DBUF && signal != kNoFlag && flag_base != P.flags) ? signal + P.n_flags : signal;
+          d.signal2 = (DBUF && signal2 != kNoFlag && flag_base != P.flags) ? signal2 + P.n_flags : signal2;
           d.dst = dst + u0 * dst_w;
           d.dst_off = dst_off + u0 * dst_w;
           d.topo = topo;
@@ -418,6 +452,12 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
           else ptx::bulk_g2s(sdst, my_src + u0 * my_w, units * my_w, &c->full[s]);
         }
         ++n;
+      }
+    }
+    if constexpr (DBUF) {
+      if (!waited) {  // a queue of early stage ops only (or an empty one)
+        pdl_wait();
+        pdl_launch_dependents();
       }
     }
     // ---- end of queue (or abort): tell the other warps, then make sure nothing is in flight
@@ -576,7 +616,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
   }
 
   __syncthreads();
-  if (tid == 0 && has_flags && !*reinterpret_cast<volatile int*>(&c->abort)) {
+  if (tid == 0 && has_flags && !DBUF && !*reinterpret_cast<volatile int*>(&c->abort)) {
     const unsigned long long prev = atomicAdd(P.epoch + 1, 1ull);
     if (prev == (unsigned long long)gridDim.x - 1ull) {
       P.epoch[1] = 0ull;
@@ -586,7 +626,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
   }
 }
 
-template <int DT, int CW, bool HOOK = false>
+template <int DT, int CW, bool HOOK = false, bool DBUF = false>
 cudaError_t launch_t(const ExecParams& P, int grid, cudaStream_t stream) {
   const size_t smem = exec_tma_smem_bytes(P.stages, P.stage_bytes);
   // the shared-memory opt-in is a per-device attribute of the function: one bit per device
@@ -596,7 +636,7 @@ cudaError_t launch_t(const ExecParams& P, int grid, cudaStream_t stream) {
   if (e != cudaSuccess) return e;
   const unsigned long long bit = 1ull << (dev & 63);
   if (!(configured.load(std::memory_order_acquire) & bit)) {
-    e = cudaFuncSetAttribute(pl_exec_tma_kernel<DT, CW, HOOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    e = cudaFuncSetAttribute(pl_exec_tma_kernel<DT, CW, HOOK, DBUF>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     configured.fetch_or(bit, std::memory_order_release);
   }
@@ -610,14 +650,14 @@ cudaError_t launch_t(const ExecParams& P, int grid, cudaStream_t stream) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = P.overlap_launch ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, pl_exec_tma_kernel<DT, CW, HOOK>, P);
+  return cudaLaunchKernelEx(&cfg, pl_exec_tma_kernel<DT, CW, HOOK, DBUF>, P);
 }
 
-template <int DT, int CW, bool HOOK = false>
+template <int DT, int CW, bool HOOK = false, bool DBUF = false>
 int occupancy_t(size_t smem) {
   int n = 0;
-  if (cudaFuncSetAttribute(pl_exec_tma_kernel<DT, CW, HOOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_tma_kernel<DT, CW, HOOK>, 32 * (2 + CW), smem) != cudaSuccess) {
+  if (cudaFuncSetAttribute(pl_exec_tma_kernel<DT, CW, HOOK, DBUF>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_tma_kernel<DT, CW, HOOK, DBUF>, 32 * (2 + CW), smem) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
@@ -631,6 +671,14 @@ int exec_tma_threads(bool pipelined) { return 32 * (2 + (pipelined ? kWarpsPipel
 
 cudaError_t launch_exec_tma(int dtype, const ExecParams& P, int grid, cudaStream_t stream) {
   if (P.stages < 2 || P.stages > kMaxStages) return cudaErrorInvalidValue;
+  if (P.stage_ahead) {
+    switch (dtype) {
+      case PL_BF16: return launch_t<PL_BF16, kWarpsGeneral, false, true>(P, grid, stream);
+      case PL_F32: return launch_t<PL_F32, kWarpsGeneral, false, true>(P, grid, stream);
+      case PL_I32: return launch_t<PL_I32, kWarpsGeneral, false, true>(P, grid, stream);
+      default: return launch_t<PL_U8, kWarpsGeneral, false, true>(P, grid, stream);
+    }
+  }
   if (P.hook) {
     switch (dtype) {
       case PL_BF16: return launch_t<PL_BF16, kWarpsGeneral, true>(P, grid, stream);
@@ -660,11 +708,12 @@ int exec_tma_max_ctas_per_sm(int dtype, int stages, uint32_t stage_bytes) {
   if (smem > 227 * 1024) return 0;
   switch (dtype) {
     case PL_BF16: return std::min({occupancy_t<PL_BF16, kWarpsGeneral>(smem), occupancy_t<PL_BF16, kWarpsPipelined>(smem),
-                                   occupancy_t<PL_BF16, kWarpsGeneral, true>(smem)});
+                                   occupancy_t<PL_BF16, kWarpsGeneral, true>(smem), occupancy_t<PL_BF16, kWarpsGeneral, false, true>(smem)});
     case PL_F32: return std::min({occupancy_t<PL_F32, kWarpsGeneral>(smem), occupancy_t<PL_F32, kWarpsPipelined>(smem),
-                                  occupancy_t<PL_F32, kWarpsGeneral, true>(smem)});
-    case PL_I32: return std::min(occupancy_t<PL_I32, kWarpsGeneral>(smem), occupancy_t<PL_I32, kWarpsPipelined>(smem));
-    default: return occupancy_t<PL_U8, kWarpsGeneral>(smem);
+                                  occupancy_t<PL_F32, kWarpsGeneral, true>(smem), occupancy_t<PL_F32, kWarpsGeneral, false, true>(smem)});
+    case PL_I32: return std::min({occupancy_t<PL_I32, kWarpsGeneral>(smem), occupancy_t<PL_I32, kWarpsPipelined>(smem),
+                                  occupancy_t<PL_I32, kWarpsGeneral, false, true>(smem)});
+    default: return std::min(occupancy_t<PL_U8, kWarpsGeneral>(smem), occupancy_t<PL_U8, kWarpsGeneral, false, true>(smem));
   }
 }
 

@@ -50,6 +50,13 @@ __device__ __forceinline__ void st16(void* p, const uint4& v) {
 __device__ __forceinline__ char* resolve(const ExecParams& P, uint64_t packed) {
   return static_cast<char*>(P.base[packed >> 48]) + (packed & 0xFFFFFFFFFFFFull);
 }
+// The same for a schedule with two staging buffers: scratch addresses move by `scratch_shift`
+// (0 or the distance to the second buffer, by launch parity); inputs and outputs stay.
+__device__ __forceinline__ char* resolve(const ExecParams& P, uint64_t packed, unsigned long long scratch_shift) {
+  const uint64_t slot = packed >> 48;
+  return static_cast<char*>(P.base[slot]) + (packed & 0xFFFFFFFFFFFFull) +
+         ((slot >= (uint64_t)kSlotScratch && slot < (uint64_t)kSlotAux) ? scratch_shift : 0ull);
+}
 
 // ---- element arithmetic ----------------------------------------------------------------
 // A "unit" is the group of elements one 16-byte vector of the narrowest operand holds:

@@ -34,6 +34,7 @@ struct HostOp {
   std::vector<int> waits;  // flag ids
   int signal = -1;
   int signal2 = -1;
+  bool stage_ahead = false;  // a stage op that waits for nothing (double-buffered staging may run it early)
   bool final_hook = false;  // writes final output: the processing phase (residual, fp32 output) applies
   int role = 0;  // 0 = any queue of the rank; 1 stage, 2 reduce, 3 gather: CTA groups per role (Sec. 3.2)
   int queue = -1;
@@ -65,6 +66,7 @@ struct alignas(16) DevOp {
 };
 static_assert(sizeof(DevOp) == 64, "DevOp must stay 64 bytes");
 constexpr uint32_t kDstF32 = 1u, kDstBcast = 2u, kFinal = 4u;  // kFinal: processing phase applies (hooked schedules)
+constexpr uint32_t kStageAhead = 8u;  // stage op that waits for nothing: may run before the previous launch has completed
 
 struct DevWait {
   uint32_t flag;
@@ -82,9 +84,13 @@ struct ExecParams {
   const DevWait* waits;         // wait_stride entries per op
   uint32_t src_stride, wait_stride;
   unsigned long long* flags;    // one 64-bit counter per flag, monotone across executes; null if the schedule has none
-  unsigned long long* epoch;    // [0] executes completed, [1] CTAs finished in this execute
+  unsigned long long* epoch;    // [0] executes completed, [1] CTAs finished in this execute, [2] CTAs started (double-buffered staging)
   int* status;                  // pl_devstatus_t words + abort word (comm-owned)
   unsigned long long* trace;    // optional: per op (topological index) [start, end] %globaltimer stamps
+  // Double-buffered staging (PL_OPT_STAGE_AHEAD): launch i uses flag set and scratch half i mod 2
+  uint32_t stage_ahead;         // 0 / 1
+  uint32_t n_flags;             // flags per set
+  unsigned long long scratch_half;  // bytes from a rank's first staging buffer to its second
   unsigned long long timeout_ns;
   int n_ranks;
   int stages;            // shared-memory ring depth of the TMA executor
@@ -131,6 +137,7 @@ struct Lowered {
   int n_layers = 1;
   int role_queues[4] = {0, 0, 0, 0};  // queues per rank reserved for each role (0 = roles unused)
   bool queues_preassigned = false;    // the lowering fixed op.queue itself (packet schedules)
+  bool double_buffered = false;       // two staging buffers and flag sets, alternated by launch parity
 };
 
 struct BuildRequest {
@@ -144,6 +151,7 @@ struct BuildRequest {
   uint64_t staging_bytes;    // staging capacity per rank (0 = default)
   int packet_ctas_per_rank;  // > 0: layered all-reduce on the packet datapath with this many CTAs per rank
   uint32_t hook;             // PL_HOOK_* bits
+  bool stage_ahead;          // PL_OPT_STAGE_AHEAD
   Policy pol;
 };
 

@@ -886,6 +886,18 @@ pl_status_t apply_hooks(const BuildRequest& rq, Lowered* L, std::string* err) {
 pl_status_t lower(const BuildRequest& rq, Lowered* L, std::string* err) {
   pl_status_t st = lower_collective(rq, L, err);
   if (st == PL_OK && rq.hook) st = apply_hooks(rq, L, err);
+  if (st == PL_OK && rq.stage_ahead) {
+    if (!rq.staged) {
+      if (err) *err = "PL_OPT_STAGE_AHEAD needs PL_OPT_STAGED";
+      return PL_ERR_INVALID_ARG;
+    }
+    // Stage ops that wait for nothing read only the caller's input and write only staging memory:
+    // with two staging buffers they may run while the previous execute still drains.
+    for (HostOp& op : L->ops)
+      op.stage_ahead = op.kind == PL_OP_COPY && !op.bcast && op.waits.empty() && op.dst.buf == PL_BUF_SCRATCH &&
+                       op.src.size() == 1 && op.src[0].buf == PL_BUF_IN;
+    L->double_buffered = true;
+  }
   return st;
 }
 
@@ -1250,6 +1262,19 @@ pl_status_t validate(const Lowered& L, int R, std::string* err, bool bulk_datapa
     }
     for (const pl_ref_t& s : op.src)
       if (const char* m = check(s, limit(s))) return fail(m);
+  }
+  // 3b. two staging buffers alternated by launch parity: an op that may run while the previous
+  //     execute still drains must touch nothing that execute can touch.  The previous execute
+  //     reads inputs, writes outputs and uses the OTHER staging buffer and flag set, so an early op
+  //     may only read the caller's input, write staging memory and signal; it cannot wait (its
+  //     flag set belongs to this execute, whose other ops have not started).
+  for (const HostOp& op : L.ops) {
+    if (!op.stage_ahead) continue;
+    if (!L.double_buffered) return fail("an op is marked for early staging in a schedule with one staging buffer");
+    if (!op.waits.empty()) return fail("an early stage op waits on a flag");
+    if (op.kind != PL_OP_COPY || op.bcast || op.dst.buf != PL_BUF_SCRATCH) return fail("an early stage op writes something other than staging memory");
+    for (const pl_ref_t& s : op.src)
+      if (s.buf != PL_BUF_IN) return fail("an early stage op reads something other than the caller's input");
   }
   // 4. memory hazards, replayed in topological order over a map of disjoint segments per
   //    buffer.  Outputs: every byte written exactly once and fully covered.  Scratch (staging

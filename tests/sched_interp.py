@@ -109,3 +109,75 @@ def run(ops, info, R, ins, seed=0, max_steps=None, aux=None, scale=1.0, elem_dty
             if f >= 0:
                 flags[f] += 1
     return bufs[B.PL_BUF_OUT]
+
+
+def run_two_overlapped(ops, info, R, ins_a, ins_b, seed=0):
+    """Two back-to-back executes of a schedule built with two staging buffers (PL_OPT_STAGE_AHEAD).
+    Execute B's early stage ops (flag value 4 in dst_bcast; only the leading ones of a queue) may
+    interleave freely with execute A's ops; everything else of B starts when A has finished.  Each
+    execute has its own staging memory and flag set (launch parity); they share the output buffers.
+    Returns (outputs after A, outputs after B)."""
+    rng = random.Random(seed)
+    nq = int(info.n_queues)
+    queues = [[] for _ in range(nq)]
+    for op in sorted(ops, key=lambda o: o.topo):
+        queues[op.queue].append(op)
+    outs = [np.full(int(info.out_bytes[r]), 0xFF, np.uint8) for r in range(R)]
+
+    class Exe:
+        def __init__(self, ins):
+            self.bufs = {B.PL_BUF_IN: [np.ascontiguousarray(a).view(np.uint8).reshape(-1) for a in ins], B.PL_BUF_OUT: outs,
+                         B.PL_BUF_SCRATCH: [np.full(int(info.scratch_bytes) + 16, 0xFF, np.uint8) for _ in range(R)]}
+            self.heads = [0] * nq
+            self.flags = [0] * int(info.n_flags)
+            self.left = len(ops)
+
+        def runnable(self, early_only):
+            out = []
+            for q in range(nq):
+                if self.heads[q] < len(queues[q]):
+                    op = queues[q][self.heads[q]]
+                    if early_only and not (op.dst_bcast & 4):
+                        continue
+                    if all(self.flags[op.wait_flag[k]] >= op.wait_need[k] for k in range(op.n_wait)):
+                        out.append(q)
+            return out
+
+        def step(self, q):
+            op = queues[q][self.heads[q]]
+            self.heads[q] += 1
+            self.left -= 1
+            n = int(op.count)
+            if op.kind == B.PL_OP_COPY:
+                result, rdt = _load(self.bufs[op.src[0].buf][op.src[0].rank], int(op.src[0].offset), n, B.PL_U8), B.PL_U8
+            else:
+                first = op.src[0]
+                acc = np.zeros(n, np.uint32 if first.dtype == B.PL_I32 else np.float32)
+                for k in range(op.n_src):
+                    sk = op.src[k]
+                    acc = acc + _load(self.bufs[sk.buf][sk.rank], int(sk.offset), n, sk.dtype)
+                result, rdt = acc, op.dst.dtype
+            for r in (range(R) if (op.dst_bcast & 1) else [op.dst.rank]):
+                _store(self.bufs[op.dst.buf][r], int(op.dst.offset), result, rdt)
+            for f in (op.signal_flag, op.signal_flag2):
+                if f >= 0:
+                    self.flags[f] += 1
+
+    a, b = Exe(ins_a), Exe(ins_b)
+    early_steps = 0
+    while a.left:
+        ra, rb = a.runnable(False), b.runnable(True)
+        assert ra, "execute A deadlocks"
+        if rb and rng.random() < 0.5:
+            b.step(rng.choice(rb))
+            early_steps += 1
+        else:
+            a.step(rng.choice(ra))
+    after_a = [o.copy() for o in outs]
+    for o in outs:
+        o[:] = 0xFF
+    while b.left:
+        rb = b.runnable(False)
+        assert rb, "execute B deadlocks"
+        b.step(rng.choice(rb))
+    return after_a, [o.copy() for o in outs], early_steps

@@ -312,6 +312,58 @@ def test_processing_hooks_rejections():
             p2.close()
 
 
+@pytest.mark.parametrize("coll", [B.PL_ALLREDUCE, B.PL_REDUCE_SCATTER, B.PL_ALLGATHER, B.PL_ALLTOALL])
+@pytest.mark.parametrize("cap_chunks", [0, 2])
+def test_double_buffered_staging_two_overlapped_executes(coll, cap_chunks):
+    """Two staging buffers alternated by launch parity (the paper's epoch-parity double buffering):
+    the early stage ops of execute B interleave with execute A on the CPU replay; both results must
+    be the oracle's, with different inputs per execute."""
+    from sched_interp import run_two_overlapped
+    R, dtype = 4, "i32"
+    chunk = 32
+    per = R * 8 * 6 if coll != B.PL_ALLGATHER else 8 * 6
+    flags = B.PL_OPT_STAGED | B.PL_OPT_OVERLAP_LAUNCH | B.PL_OPT_STAGE_AHEAD
+    pl = Planner(R, dtype)
+    try:
+        s = pl.build(coll, B.PL_ALGO_DIRECT, per, chunk, flags=flags, staging_bytes=cap_chunks * chunk * (R if coll != B.PL_ALLGATHER else 1),
+                     n_ctas=3 * R, slice_bytes=16)
+        assert B.pl_schedule_validate(s)[0] == B.PL_OK
+        info = B.pl_schedule_info(s)
+        ops = B.pl_schedule_dump(s)
+        early = [o for o in ops if o.dst_bcast & 4]
+        assert early and all(o.kind == B.PL_OP_COPY and o.n_wait == 0 and o.dst.buf == B.PL_BUF_SCRATCH
+                             and o.src[0].buf == B.PL_BUF_IN for o in early)
+        if cap_chunks:  # cyclic slots: later stage ops wait for their slot and are not early
+            assert any(o.kind == B.PL_OP_COPY and o.dst.buf == B.PL_BUF_SCRATCH and not (o.dst_bcast & 4) for o in ops)
+        xa = gen.rank_inputs(R, per, dtype)
+        xb = [(a.astype(np.int64) * 3 + 11).astype(np.int32) for a in xa]
+        got_a, got_b, early_steps = run_two_overlapped(ops, info, R, xa, xb, seed=4)
+        assert early_steps > 0
+        fn = {B.PL_ALLREDUCE: lambda x: oracle.allreduce(x, dtype), B.PL_REDUCE_SCATTER: lambda x: oracle.reduce_scatter(x, dtype),
+              B.PL_ALLGATHER: oracle.allgather, B.PL_ALLTOALL: oracle.alltoall}[coll]
+        for got, x in ((got_a, xa), (got_b, xb)):
+            ref = fn(x)
+            for r in range(R):
+                assert np.array_equal(got[r].view(np.int32), np.asarray(ref[r]).view(np.int32))
+    finally:
+        pl.close()
+
+
+def test_stage_ahead_needs_staging_and_overlapped_launches():
+    pl = Planner(4, "bf16")
+    try:
+        for flags in (B.PL_OPT_STAGE_AHEAD, B.PL_OPT_STAGE_AHEAD | B.PL_OPT_STAGED, B.PL_OPT_STAGE_AHEAD | B.PL_OPT_OVERLAP_LAUNCH,
+                      B.PL_OPT_STAGE_AHEAD | B.PL_OPT_STAGED | B.PL_OPT_OVERLAP_LAUNCH | B.PL_OPT_TRACE):
+            with pytest.raises(B.PurlinError) as e:
+                pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 256, flags=flags)
+            assert e.value.status == B.PL_ERR_INVALID_ARG
+        s = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 256, flags=B.PL_OPT_STAGED | B.PL_OPT_OVERLAP_LAUNCH | B.PL_OPT_STAGE_AHEAD)
+        one = pl.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, 1024, 256, flags=B.PL_OPT_STAGED | B.PL_OPT_OVERLAP_LAUNCH)
+        assert B.pl_schedule_info(s).scratch_bytes == 2 * B.pl_schedule_info(one).scratch_bytes   # two staging buffers
+    finally:
+        pl.close()
+
+
 def test_config1_op_counts_and_bytes():
     # all-reduce, R=4, 262144 fp32 per rank, ring, 64 KiB chunks, unsliced:
     # 3 reduce-scatter hops + 3 all-gather hops, 4 ranks, 4 chunks per partition
