@@ -150,7 +150,7 @@ class Bench:
         sched_bytes = info.bytes_read + info.bytes_written
         # bytes that must cross the HBM interface when nothing is cached between launches: every
         # input byte once, every output byte once (an all-gather re-reads its sources from L2)
-        compulsory = sum(int(info.in_bytes[r]) for r in range(R)) + int(info.bytes_written)
+        compulsory = sum(int(info.in_bytes[r]) + int(info.aux_bytes[r]) for r in range(R)) + int(info.bytes_written)
         rec = {"cfg": cfg, "bytes_read": int(info.bytes_read), "bytes_written": int(info.bytes_written),
                "compulsory_bytes": int(min(compulsory, sched_bytes)), "coll": int(coll), "algo": algo, "R": R, "dtype": int(dtype),
                "message_bytes": int(info.message_bytes), "chunk": int(min(chunk, 1 << 40)), "layers": layers,
@@ -370,6 +370,40 @@ def main(args=None):
         for batch in (1, 8, 64):
             for algo in ("oneshot", "direct", "fused"):
                 b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, batch * 8192, 0, iters=50, layers=80)
+    if "c5prof" in which:
+        # the three latency-path kernels at 16 KiB, one after the other (short: for profiler captures)
+        b.collective("C5-flags", 8, B.PL_BF16, B.PL_ALLREDUCE, "fused", 8192, 0, iters=20, layers=80)
+        b.collective("C5-flags", 8, B.PL_BF16, B.PL_ALLREDUCE, "oneshot", 8192, 0, iters=20, layers=80)
+        b.collective("C5-packets", 8, B.PL_BF16, B.PL_ALLREDUCE, "oneshot", 8192, 0, iters=20, layers=80, datapath=B.PL_DP_PACKET)
+    if "c5trace" in which:
+        # where a layer's time goes, from the in-kernel stamps of the last execute (PL_OPT_TRACE): for
+        # every op "start" = its waits are satisfied (flags seen / one packet of every rank seen) and
+        # "end" = its output is written and it is about to signal (flags) or to join its rank (packets)
+        for kib in (4, 16):
+            for name, algo, kw in (("flags fused", "fused", {}), ("flags oneshot", "oneshot", {}),
+                                   ("packets", "oneshot", dict(datapath=B.PL_DP_PACKET))):
+                comm = B.pl_comm_create(8, B.PL_BF16)
+                sched = B.pl_schedule_build_layers(comm, ALGO[algo], kib * 512, 80, B.make_opts(flags=B.PL_OPT_TRACE, **kw))
+                info = B.pl_schedule_info(sched)
+                d_in = [_fill(int(info.in_bytes[r]), r) for r in range(8)]
+                d_out = [torch.empty(int(info.out_bytes[r]), dtype=torch.uint8, device="cuda") for r in range(8)]
+                bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                                   [int(info.in_bytes[r]) for r in range(8)], [int(info.out_bytes[r]) for r in range(8)])
+                for _ in range(5):
+                    B.pl_execute(sched, bufs, b.stream)
+                ops = B.pl_schedule_dump(sched)
+                tr = B.pl_schedule_trace_read(sched, len(ops), b.stream).astype(np.int64)
+                lay = np.array([o.layer for o in ops])
+                start = np.array([tr[lay == l, 0].max() for l in range(80)])   # the last op of the layer to see its inputs
+                first = np.array([tr[lay == l, 0].min() for l in range(80)])
+                end = np.array([tr[lay == l, 1].max() for l in range(79)])      # the last op of the layer to finish writing
+                b.emit({"cfg": "C5-trace", "protocol": name, "message_bytes": kib * 1024, "grid": int(info.grid),
+                        "layer_ns_p50": float(np.median(np.diff(start)[5:])),
+                        "written_to_next_seen_ns_p50": float(np.median((start[1:] - end)[5:])),
+                        "written_to_first_seen_ns_p50": float(np.median((first[1:] - end)[5:])),
+                        "seen_to_written_ns_p50": float(np.median((end - start[:-1])[5:]))})
+                B.pl_schedule_destroy(sched)
+                B.pl_comm_destroy(comm)
     if "c5p" in which or "c5" in which:
         # the two latency protocols side by side: per-rank flags (register executor) against
         # 16-byte packets (8 B payload + 8 B tag), per layer, 80 layers in one launch

@@ -156,6 +156,7 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_packet_kernel(const __gri
           }
         }
         if (aborted) break;  // warp-uniform
+        if (P.trace && tid == 0 && k == 0) P.trace[2 * (((uint64_t)l * R + r) * G + j)] = globaltimer_ns();  // sentinels of every rank seen
         Acc<DT> acc;
         acc.zero();
         const uint64_t at = (gl & 1ull) * half + (u0 + u) * 32ull;
@@ -229,10 +230,8 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_packet_kernel(const __gri
     if (P.trace) {
       __syncthreads();
       if (tid == 0) {
-        const unsigned long long t = globaltimer_ns();
-        const uint64_t op = ((uint64_t)l * R + r) * G + j;
-        P.trace[2 * op] = t;      // all of the layer's packets seen (and the slice written)
-        P.trace[2 * op + 1] = t;  // about to join: nothing of this op happens after this stamp
+        // about to join: every thread has read its packets and stored its part of the slice
+        P.trace[2 * (((uint64_t)l * R + r) * G + j) + 1] = globaltimer_ns();
       }
     }
     // ---- join: rank r's layer-l output is complete when every CTA of the rank is here
