@@ -320,8 +320,9 @@ pl_status_t pl_comm_create_planner(int R, pl_dtype_t dtype, pl_comm_t* out);
  * (PL_ERR_INVALID_ARG otherwise). */
 pl_status_t pl_comm_destroy(pl_comm_t comm);
 
-/* Read the device status record.  Synchronises the device.  Returns PL_OK and fills *out;
- * out->code tells whether a wait timed out since the last reset. */
+/* Read the device status record as it stands at the time of the call (on an internal stream: the
+ * call waits for no other work, so synchronise the stream of the executes you ask about first).
+ * Returns PL_OK and fills *out; out->code tells whether a wait timed out since the last reset. */
 pl_status_t pl_comm_status(pl_comm_t comm, pl_devstatus_t* out);
 
 /* Clear the status record and re-zero the flags and epochs of every schedule of `comm`

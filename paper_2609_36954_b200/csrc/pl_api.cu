@@ -453,6 +453,9 @@ static pl_status_t comm_create(int R, pl_dtype_t dtype, bool planner, pl_comm_t*
     c->sm_count = prop.multiProcessorCount;
     if (cudaMalloc(&c->d_status, kStatusWords * sizeof(int)) != cudaSuccess) { cudaGetLastError(); delete c; return PL_ERR_OOM; }
     if (cudaMemset(c->d_status, 0, kStatusWords * sizeof(int)) != cudaSuccess) { cudaGetLastError(); cudaFree(c->d_status); delete c; return PL_ERR_CUDA; }
+    cudaStream_t st = nullptr;
+    if (cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); cudaFree(c->d_status); delete c; return PL_ERR_CUDA; }
+    c->status_stream = st;
   }
   *out = c;
   return PL_OK;
@@ -465,6 +468,7 @@ pl_status_t pl_comm_destroy(pl_comm_t comm) {
   if (!comm) return PL_ERR_INVALID_ARG;
   if (!comm->schedules.empty() || comm->n_plans != 0) return PL_ERR_INVALID_ARG;
   if (comm->d_status) cudaFree(comm->d_status);
+  if (comm->status_stream) cudaStreamDestroy(static_cast<cudaStream_t>(comm->status_stream));
   delete comm;
   return PL_OK;
 }
@@ -475,8 +479,13 @@ pl_status_t pl_comm_status(pl_comm_t comm, pl_devstatus_t* out) {
   if (comm->planner) return PL_OK;
   if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
   int words[kStatusWords];
-  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
-  if (cudaMemcpy(words, comm->d_status, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  // the record as it stands now, read on a stream of its own: no other stream is waited for
+  cudaStream_t st = static_cast<cudaStream_t>(comm->status_stream);
+  if (cudaMemcpyAsync(words, comm->d_status, sizeof(words), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return PL_ERR_CUDA;
+  }
   out->code = words[0];
   out->queue = words[1];
   out->op = words[2];

@@ -17,6 +17,7 @@ struct pl_comm_s {
   int device = -1;
   int sm_count = 148;
   int* d_status = nullptr;
+  void* status_stream = nullptr;  // non-blocking stream used only to read the status record
   std::mutex mu;
   std::vector<pl_schedule_s*> schedules;
   int n_plans = 0;

@@ -392,7 +392,8 @@ __global__ void __launch_bounds__(kMaxThreads) pl_exec_kernel(const __grid_const
       __syncthreads();  // every thread's writes are done
       if (tid == 0 && P.trace) P.trace[2ull * op.topo + 1] = globaltimer_ns();
       if (tid == 0 && op.signal != kNoFlag) {
-        __threadfence();
+        // the release is cumulative: it covers the other threads' stores, which this thread
+        // observed through the barrier above
         red_release_add_u64(const_cast<unsigned long long*>(flag_base) + op.signal, 1ull);
         if (op.signal2 != kNoFlag) red_release_add_u64(const_cast<unsigned long long*>(flag_base) + op.signal2, 1ull);
       }
