@@ -154,3 +154,132 @@ def test_random_v_and_rooted_case_matches_the_oracle(seed):
                 assert np.array_equal(outs[root], oracle.gather(contrib, root)[root].view(np.uint8))
     finally:
         s.close()
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_random_hook_stage_ahead_and_packet_cases_match_the_oracle(seed):
+    """Seeded draws over the options of the processing phase (scale, second operand, fp32 output),
+    double-buffered staging (back-to-back executes with different inputs) and the packet datapath
+    (layered one-shot all-reduce), with ragged sizes, odd rank counts, both executors."""
+    import torch
+    from gpu_harness import poison, stream_handle, to_dev
+    rng = np.random.default_rng(9000 + seed)
+    kind = str(rng.choice(["hook", "stage_ahead", "packets"]))
+    R = int(rng.choice([2, 3, 4, 5, 7, 8, 12, 16]))
+    vecs = int(rng.choice([1, 3, 17, 64, 257, 1031]))
+    dp = int(rng.choice([B.PL_DP_AUTO, B.PL_DP_LDST, B.PL_DP_TMA]))
+
+    def run(sched, ses, x, aux=None):
+        info = B.pl_schedule_info(sched)
+        d_in = [to_dev(a) for a in x]
+        d_aux = [to_dev(a) for a in aux] if aux is not None else None
+        d_out = [poison(info.out_bytes[r]) for r in range(R)]
+        bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                           [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)],
+                           [t.data_ptr() for t in d_aux] if d_aux else None,
+                           [int(info.aux_bytes[r]) for r in range(R)] if d_aux else None)
+        B.pl_execute(sched, bufs, stream_handle())
+        return d_in, d_aux, d_out, info
+
+    if kind == "hook":
+        dtype = str(rng.choice(["bf16", "f32"]))
+        es = B.DTYPE_SIZE[DT[dtype]]
+        coll, algo = [(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT), (B.PL_REDUCE_SCATTER, B.PL_ALGO_RING),
+                      (B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT), (B.PL_ALLREDUCE, B.PL_ALGO_DIRECT_FUSED)][int(rng.integers(0, 4))]
+        hook = int(rng.choice([1, 2, 3])) if dtype == "bf16" else 1
+        scale = float(rng.choice([1.0, 0.5, 1.0 / R, -2.0]))
+        n = R * vecs * (16 // es)
+        n_out = n // R if coll == B.PL_REDUCE_SCATTER else n
+        x = gen.rank_inputs(R, n, "f32n" if dtype == "f32" else dtype, seed=seed)
+        aux = gen.rank_inputs(R, n_out, "f32n" if dtype == "f32" else dtype, seed=seed + 500) if hook & 1 else None
+        ref = (oracle.allreduce_processed if coll == B.PL_ALLREDUCE else oracle.reduce_scatter_processed)(x, dtype, scale, aux)
+        ses = Session(R, dtype)
+        try:
+            sched = ses.build(coll, algo, n, 16 * int(rng.choice([1, 5, 64, 3000])), datapath=dp, hook=hook, out_scale=scale,
+                              slice_bytes=16 * int(rng.choice([0, 1, 128])))
+            keep = run(sched, ses, x, aux)
+            torch.cuda.synchronize()
+            assert B.pl_comm_status(ses.comm).code == B.PL_OK
+            d_out, info = keep[2], keep[3]
+            for r in range(R):
+                got = d_out[r][: int(info.out_bytes[r])].cpu().numpy()
+                if hook & 2:
+                    lo, hi = (r * n_out, (r + 1) * n_out) if coll == B.PL_REDUCE_SCATTER else (0, n)
+                    mag = abs(scale) * sum(np.abs(gen.bf16_bits_to_f64(a[lo:hi])) for a in x)
+                    if aux is not None:
+                        mag = mag + np.abs(gen.bf16_bits_to_f64(aux[r]))
+                    assert np.all(np.abs(got.view(np.float32).astype(np.float64) - ref[r]) <= (R + 1) * 2.0 ** -24 * mag + 1e-30)
+                elif dtype == "bf16":
+                    # the scale may enlarge the sum: the bf16 bound is relative to the processed value
+                    check_float(gen.bf16_bits_to_f64(got.view(np.uint16)), ref[r], "bf16")
+                else:
+                    a64 = aux[r].astype(np.float64)
+                    assert np.all(np.abs(got.view(np.float32).astype(np.float64) - ref[r]) <= 1e-6 * (np.abs(ref[r] - a64) + np.abs(a64)) + 1e-7)
+        finally:
+            ses.close()
+    elif kind == "stage_ahead":
+        dtype = str(rng.choice(["i32", "bf16"]))
+        es = B.DTYPE_SIZE[DT[dtype]]
+        coll = int(rng.choice([B.PL_ALLREDUCE, B.PL_REDUCE_SCATTER, B.PL_ALLGATHER, B.PL_ALLTOALL]))
+        chunk_vecs = int(rng.choice([1, 5, 64, 512]))
+        n = R * vecs * (16 // es)
+        count = n // R if coll == B.PL_ALLGATHER else n
+        cap = int(rng.choice([0, 2])) * 16 * min(chunk_vecs, vecs) * (1 if coll == B.PL_ALLGATHER else R)
+        ses = Session(R, dtype)
+        try:
+            sched = ses.build(coll, B.PL_ALGO_DIRECT, count, 16 * chunk_vecs, datapath=dp, staging_bytes=cap,
+                              flags=B.PL_OPT_STAGED | B.PL_OPT_OVERLAP_LAUNCH | B.PL_OPT_STAGE_AHEAD)
+            calls, kept = 3, []
+            xs = []
+            for k in range(calls):
+                x = gen.rank_inputs(R, n, dtype, seed=seed * 7 + k)
+                if dtype == "i32":
+                    x = [(a.astype(np.int64) * (k + 2) + k).astype(np.int32) for a in x]
+                if coll == B.PL_ALLGATHER:
+                    x = [a[:count].copy() for a in x]
+                xs.append(x)
+                kept.append(run(sched, ses, x))     # back to back, no synchronisation in between
+            torch.cuda.synchronize()
+            assert B.pl_comm_status(ses.comm).code == B.PL_OK
+            for k in range(calls):
+                x, (_, _, d_out, info) = xs[k], kept[k]
+                ref = {B.PL_ALLREDUCE: lambda: oracle.allreduce(x, dtype), B.PL_REDUCE_SCATTER: lambda: oracle.reduce_scatter(x, dtype),
+                       B.PL_ALLGATHER: lambda: oracle.allgather(x), B.PL_ALLTOALL: lambda: oracle.alltoall(x)}[coll]()
+                for r in range(R):
+                    got = d_out[r][: int(info.out_bytes[r])].cpu().numpy()
+                    if coll in (B.PL_ALLGATHER, B.PL_ALLTOALL) or dtype == "i32":
+                        assert np.array_equal(got, np.ascontiguousarray(ref[r]).view(np.uint8).reshape(-1)), (k, r)
+                    else:
+                        check_float(gen.bf16_bits_to_f64(got.view(np.uint16)), ref[r], "bf16")
+        finally:
+            ses.close()
+    else:
+        dtype = str(rng.choice(["i32", "bf16", "f32"]))
+        es = B.DTYPE_SIZE[DT[dtype]]
+        layers = int(rng.choice([1, 2, 5, 9]))
+        vecs = min(vecs, 257)     # a CTA's threads hold at most 4 vectors each: 1024 per CTA
+        n = vecs * (16 // es)
+        ses = Session(R, dtype)
+        try:
+            g = int(rng.choice([0, 1, 2, 4, 8]))
+            if g and vecs % g:
+                g = 1
+            sched = ses.build_layers(B.PL_ALGO_ONESHOT, n, layers, datapath=B.PL_DP_PACKET, n_ctas=g * R)
+            for rep in range(2):
+                x = [np.concatenate([gen.rank_inputs(R, n, "f32n" if dtype == "f32" else dtype, seed=seed * 13 + rep, stream_base=l * R)[r]
+                                     for l in range(layers)]) for r in range(R)]
+                if dtype == "i32":
+                    x = [(a.astype(np.int64) * (rep + 1) + np.repeat(np.arange(layers), n) * 101).astype(np.int32) for a in x]
+                outs, _ = ses.execute(sched, x)
+                for l in range(layers):
+                    ref = oracle.allreduce([a[l * n:(l + 1) * n] for a in x], dtype)
+                    for r in range(R):
+                        got = outs[r][l * n * es:(l + 1) * n * es]
+                        if dtype == "i32":
+                            assert np.array_equal(got.view(np.int32), ref[r])
+                        elif dtype == "bf16":
+                            check_float(gen.bf16_bits_to_f64(got.view(np.uint16)), ref[r], "bf16")
+                        else:
+                            check_float(got.view(np.float32).astype(np.float64), ref[r], "f32")
+        finally:
+            ses.close()
