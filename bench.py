@@ -250,7 +250,7 @@ def run_purlin(args):
 
     # ---- roofline of the dominant kernel (the reduce-scatter launch) -----------------------
     rs_alg = irs.bytes_read + irs.bytes_written            # (R+1) * M: every byte touched once
-    ag_floor = iag.in_bytes[0] * R + iag.bytes_written     # compulsory DRAM traffic (R+1) * M
+    ag_floor = iag.hbm_bytes                               # compulsory DRAM traffic (R+1) * M
     rs_gbs = rs_alg / (rs_ms.mean() * 1e-3) / 1e9
     ag_gbs = ag_floor / (ag_ms.mean() * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "pl_exec_tma_kernel<bf16> (reduce-scatter launch)",

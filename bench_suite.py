@@ -148,11 +148,10 @@ class Bench:
                          "p90_us": float(np.percentile(gaps, 90))}
         nl = max(1, layers)
         sched_bytes = info.bytes_read + info.bytes_written
-        # bytes that must cross the HBM interface when nothing is cached between launches: every
-        # input byte once, every output byte once (an all-gather re-reads its sources from L2)
-        compulsory = sum(int(info.in_bytes[r]) + int(info.aux_bytes[r]) for r in range(R)) + int(info.bytes_written)
+        # bytes that must cross the HBM interface when nothing is cached between launches
+        # (pl_sched_info_t.hbm_bytes: input bytes once however often they are read, everything else as scheduled)
         rec = {"cfg": cfg, "bytes_read": int(info.bytes_read), "bytes_written": int(info.bytes_written),
-               "compulsory_bytes": int(min(compulsory, sched_bytes)), "coll": int(coll), "algo": algo, "R": R, "dtype": int(dtype),
+               "compulsory_bytes": int(info.hbm_bytes), "coll": int(coll), "algo": algo, "R": R, "dtype": int(dtype),
                "message_bytes": int(info.message_bytes), "chunk": int(min(chunk, 1 << 40)), "layers": layers,
                "us": p50 / nl, "us_p10": p10 / nl, "us_p90": p90 / nl, "us_graph128": graph_us, "layer_us_in_kernel": in_kernel,
                "eff_gbs": info.message_bytes * nl / p50 / 1e3, "sched_gbs": sched_bytes / p50 / 1e3,

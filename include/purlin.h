@@ -277,6 +277,10 @@ typedef struct {
   uint64_t aux_bytes[PL_MAX_RANKS];    /* bytes pl_execute requires in bufs->aux[r] (PL_HOOK_RESIDUAL) */
   int32_t out_dtype;                   /* element type stored in out[r]: PL_F32 under PL_HOOK_F32_OUT  */
   uint32_t hook;                       /* PL_HOOK_* bits of the schedule                               */
+  uint64_t hbm_bytes;                  /* bytes that must cross the memory interface when nothing is   */
+                                       /* cached between launches: bytes_read with every byte of the   */
+                                       /* caller's inputs (and second operands) counted once, however  */
+                                       /* many ops read it, plus bytes_written                         */
 } pl_sched_info_t;
 
 /* Device buffers of one execute: in[r] / out[r] for r < R, 16-byte aligned, non-overlapping.

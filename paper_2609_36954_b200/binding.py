@@ -78,7 +78,8 @@ class pl_sched_info_t(C.Structure):
                 ("grid", C.c_int32), ("threads", C.c_int32), ("smem_bytes", C.c_int32),
                 ("datapath", C.c_int32), ("stages", C.c_int32),
                 ("stage_bytes", C.c_uint32), ("slice_bytes", C.c_uint32),
-                ("aux_bytes", C.c_uint64 * PL_MAX_RANKS), ("out_dtype", C.c_int32), ("hook", C.c_uint32)]
+                ("aux_bytes", C.c_uint64 * PL_MAX_RANKS), ("out_dtype", C.c_int32), ("hook", C.c_uint32),
+                ("hbm_bytes", C.c_uint64)]
 
 
 class pl_bufs_t(C.Structure):

@@ -1,6 +1,7 @@
 // C-ABI layer: handles, argument checks, device upload of a lowered schedule, launches.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstring>
@@ -93,6 +94,32 @@ void fill_info(pl_schedule_s* S, int R) {
     I.in_bytes[r] = L.in_bytes[r];
     I.out_bytes[r] = L.out_bytes[r];
     I.aux_bytes[r] = L.aux_bytes[r];
+  }
+  // Compulsory traffic: what the ops read from the caller's inputs counts once per byte (the union
+  // of the ranges per rank), what they read from outputs or scratch was produced by this launch
+  // and counts every time, like every write.
+  {
+    std::vector<std::vector<std::pair<uint64_t, uint64_t>>> ranges(R);
+    uint64_t other_reads = 0;
+    for (const HostOp& op : L.ops)
+      for (const pl_ref_t& s : op.src) {
+        const uint64_t b = op.count * elem_size(s.dtype);
+        if (s.buf == PL_BUF_IN) ranges[s.rank].emplace_back(s.offset, s.offset + b);
+        else other_reads += b;
+      }
+    uint64_t in_once = 0;
+    for (auto& v : ranges) {
+      std::sort(v.begin(), v.end());
+      uint64_t hi = 0;
+      for (const auto& iv : v) {
+        if (iv.second <= hi) continue;
+        in_once += iv.second - std::max(iv.first, hi);
+        hi = iv.second;
+      }
+    }
+    uint64_t aux_reads = 0;
+    for (int r = 0; r < R; ++r) aux_reads += L.aux_bytes[r];
+    I.hbm_bytes = in_once + other_reads + aux_reads + I.bytes_written;
   }
   I.out_dtype = (S->hook & PL_HOOK_F32_OUT) ? PL_F32 : S->comm->dtype;
   I.hook = S->hook;

@@ -364,6 +364,33 @@ def test_stage_ahead_needs_staging_and_overlapped_launches():
         pl.close()
 
 
+def test_hbm_bytes_count_every_input_byte_once():
+    """pl_sched_info_t.hbm_bytes: bytes_read with the caller's inputs counted once, plus bytes_written."""
+    R, M = 8, 1 << 20            # bf16, 1 MiB per rank
+    pl = Planner(R, "bf16")
+    try:
+        n = M // 2
+        want = {
+            (B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n): (R + 1) * M,                 # read everything once, write M / R per rank
+            (B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R): (R + 1) * M,                 # contributions once, R * M written
+            (B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT, n): 2 * R * M,                       # inputs once (not R times), R * M written
+            (B.PL_ALLREDUCE, B.PL_ALGO_DIRECT_FUSED, n): 2 * R * M,
+            (B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, n): R * M + M + (R - 1) * M + (R - 1) * M,  # + reduced partitions re-read by R - 1 ranks
+            (B.PL_ALLTOALL, B.PL_ALGO_DIRECT, n): 2 * R * M,
+        }
+        for (coll, algo, count), bytes_ in want.items():
+            info = B.pl_schedule_info(pl.build(coll, algo, count, 65536, datapath=B.PL_DP_TMA))
+            assert info.hbm_bytes == bytes_, (coll, algo, info.hbm_bytes, bytes_)
+            assert info.hbm_bytes <= info.bytes_read + info.bytes_written
+        # ring reduce-scatter: every input partition once (the chain start reads two inputs of the same
+        # partition from two ranks), the travelling fp32 partials written and read once per hop
+        info = B.pl_schedule_info(pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_RING, n, 65536, datapath=B.PL_DP_TMA))
+        P = M // R
+        assert info.hbm_bytes == R * M + 2 * R * (R - 2) * 2 * P + R * P
+    finally:
+        pl.close()
+
+
 def test_config1_op_counts_and_bytes():
     # all-reduce, R=4, 262144 fp32 per rank, ring, 64 KiB chunks, unsliced:
     # 3 reduce-scatter hops + 3 all-gather hops, 4 ranks, 4 chunks per partition
