@@ -424,7 +424,7 @@ def measure_all_configs(peak):
         out["C5"][label] = {algo: entry(b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, count, 0, iters=100, layers=80), l2)
                             for algo in ("oneshot", "fused")}
     out["C5_protocols"] = {}
-    for kib in (4, 16, 64):
+    for kib in (1, 4, 16, 64):
         flags = [b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, kib * 512, 0, iters=200, layers=80) for algo in ("oneshot", "fused")]
         best = min(flags, key=lambda r: r["us"])
         pk = b.collective("C5", 8, B.PL_BF16, B.PL_ALLREDUCE, "oneshot", kib * 512, 0, iters=200, layers=80, datapath=B.PL_DP_PACKET)

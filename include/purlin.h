@@ -142,9 +142,9 @@ typedef enum {
    * and an 8-byte tag written with one store; the consumer polls the packet itself, so there is
    * no separate flag, fence or acquire on the path.  Only for pl_schedule_build_layers with
    * PL_ALGO_ONESHOT (or PL_ALGO_AUTO) and small messages (at most 128 KiB per rank; meant for
-   * up to 64 KiB): rank r runs as a thread-block cluster of n_ctas / R CTAs (1, 2, 4 or 8) that
-   * joins with a cluster barrier when its layer's output is complete and then publishes its
-   * next contribution; the schedule owns two packet buffers per rank, alternated by layer
+   * up to 64 KiB): rank r runs as a thread-block cluster of n_ctas / R CTAs (1, 2, 4 or 8; the
+   * library picks 1 up to 4 KiB, else up to 8) that joins with a cluster barrier (a CTA barrier
+   * for one CTA) when its layer's output is complete and then publishes its next contribution; the schedule owns two packet buffers per rank, alternated by layer
    * parity (Sec. 4.2, epoch-parity double buffering), tags are global layer numbers that only
    * grow, nothing is reset between executes.  pl_schedule_dump shows the same data movement
    * with the ordering rules as logical flags (no flag words exist on the device). */
@@ -388,7 +388,9 @@ pl_status_t pl_schedule_build_rooted(pl_comm_t comm, pl_collective_t coll, int r
  * dominate; Sec. 3.2 "Specializing for latency").  Layer l reads in[r] + l*M and writes out[r] + l*M
  * (M = count_per_rank * elem_size).  Rank r's layer-(l+1) contribution counts as published
  * only when r's layer-l output is complete, and no consumer reads it earlier.  Algorithms:
- * PL_ALGO_ONESHOT, PL_ALGO_DIRECT, PL_ALGO_DIRECT_FUSED. */
+ * PL_ALGO_ONESHOT, PL_ALGO_DIRECT, PL_ALGO_DIRECT_FUSED; PL_ALGO_AUTO picks direct-fused on the
+ * register executor, and for messages of at most 4 KiB (with grid, datapath and hooks left to the
+ * library) one-shot on the packet datapath with one CTA per rank, the fastest form there. */
 pl_status_t pl_schedule_build_layers(pl_comm_t comm, pl_algo_t algo, size_t count_per_rank,
                                      int n_layers, const pl_sched_opts_t* opts,
                                      pl_schedule_t* out);

@@ -217,6 +217,27 @@ def test_packet_schedule_replay_program_order_and_geometry(R, units, G):
         pl.close()
 
 
+def test_layers_auto_picks_packets_for_tiny_messages_only():
+    pl = Planner(8, "bf16")
+    try:
+        for n, want_dp, want_grid in ((512, B.PL_DP_PACKET, 8), (2048, B.PL_DP_PACKET, 8), (4096, B.PL_DP_LDST, None), (8192, B.PL_DP_LDST, None)):
+            s = B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_AUTO, n, 4, None)
+            pl.scheds.append(s)
+            info = B.pl_schedule_info(s)
+            assert info.datapath == want_dp, (n, info.datapath)
+            if want_grid:
+                assert info.grid == want_grid          # one CTA per rank
+        # anything the caller pins keeps the flag path
+        s = B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_AUTO, 512, 4, B.make_opts(n_ctas=16))
+        pl.scheds.append(s)
+        assert B.pl_schedule_info(s).datapath == B.PL_DP_LDST
+        s = B.pl_schedule_build_layers(pl.comm, B.PL_ALGO_DIRECT_FUSED, 512, 4, None)
+        pl.scheds.append(s)
+        assert B.pl_schedule_info(s).datapath == B.PL_DP_LDST
+    finally:
+        pl.close()
+
+
 def test_packet_schedule_rejections():
     pl = Planner(4, "bf16")
     try:
