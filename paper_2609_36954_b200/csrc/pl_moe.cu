@@ -43,6 +43,7 @@ struct CombinePtrs {
 struct MoeGeo {
   int R, T, E, K, NB, epr;
   uint32_t row_bytes, tile_bytes, n_tiles, slots;
+  uint32_t rows_per_item, slot_bytes;  // mover: consecutive token rows per bulk load, bytes per ring slot
   unsigned long long cap;
   int32_t* blockcnt;   // [R][NB][E]: per-block counts, turned into exclusive block offsets by scan
   long long* counts;   // [R][R]
@@ -360,7 +361,13 @@ __global__ void __launch_bounds__(256) moe_derive_ranks_kernel(const __grid_cons
 
 // One warp per CTA drives a ring of `slots` shared-memory tiles: lane 0 issues the bulk loads
 // (prime, then refill as tiles drain: the paper's Algorithm 2 with the processing step being
-// "store to K places"), lane j issues the bulk store to destination j.
+// "store to K places"), the lanes share the bulk stores.  A work item is a group of `rows`
+// consecutive token rows of one source rank, which are contiguous in its input: one bulk load of
+// up to 56 KiB, then rows x K bulk stores of one row each (rows wider than 16 KiB are moved in
+// tiles, one row per item).  The write-dominated stream this kernel is runs fastest with large
+// loads and 128-136 CTAs on this GPU (1 read : 8 writes through the same ring: 6.15-6.3 TB/s with
+// 128-136 CTAs and 32-64 KiB tiles, 5.65-5.73 TB/s with 140-148 CTAs, 5.55 TB/s with 296 CTAs and
+// 14 KiB tiles), so the grid is a property of the GPU's memory system, not of the row count.
 __global__ void __launch_bounds__(32) moe_move_kernel(const __grid_constant__ DispatchPtrs P, const __grid_constant__ MoeGeo g) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int lane = threadIdx.x;
@@ -375,29 +382,35 @@ __global__ void __launch_bounds__(32) moe_move_kernel(const __grid_constant__ Di
   // launched with programmatic stream serialization: set up above while the bookkeeping kernel
   // drains, wait here for it to complete before anything it wrote (pos, prank) is read
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const unsigned long long n_items = (unsigned long long)g.R * g.T * g.n_tiles;
+  const uint32_t rows = g.rows_per_item;  // > 1 only when a row is one tile
+  const unsigned long long groups_per_rank = ((unsigned long long)g.T + rows - 1) / rows;
+  const unsigned long long n_items = (unsigned long long)g.R * groups_per_rank * g.n_tiles;
   const unsigned long long c = blockIdx.x, G = gridDim.x;
   if (c >= n_items) return;
   const unsigned long long n_my = (n_items - c + G - 1) / G;
   constexpr int L = 2;  // store groups allowed to be still reading shared memory
 
-  auto item = [&](unsigned long long n, unsigned long long& tok, uint32_t& off, uint32_t& bytes) {
+  // item n of this CTA: tokens [tok, tok + nrows) of one rank, bytes [off, off + bytes) of each row
+  auto item = [&](unsigned long long n, unsigned long long& tok, uint32_t& nrows, uint32_t& off, uint32_t& bytes) {
     const unsigned long long w = c + n * G;
-    tok = w / g.n_tiles;
+    const unsigned long long grp = w / g.n_tiles;
     const uint32_t tile = (uint32_t)(w % g.n_tiles);
+    const unsigned long long p = grp / groups_per_rank, t0 = (grp % groups_per_rank) * rows;
+    tok = p * g.T + t0;
+    nrows = (uint32_t)min((unsigned long long)rows, (unsigned long long)g.T - t0);
     off = tile * g.tile_bytes;
-    bytes = min(g.tile_bytes, g.row_bytes - off);
+    bytes = (rows > 1) ? g.row_bytes : min(g.tile_bytes, g.row_bytes - off);
   };
   auto issue_load = [&](unsigned long long n) {
     unsigned long long tok;
-    uint32_t off, bytes;
-    item(n, tok, off, bytes);
+    uint32_t nrows, off, bytes;
+    item(n, tok, nrows, off, bytes);
     const int p = (int)(tok / g.T);
     const unsigned long long t = tok % g.T;
     const char* src = static_cast<const char*>(P.x[p]) + t * g.row_bytes + off;
     const uint32_t s = (uint32_t)(n % S);
-    ptx::mbar_expect_tx(full + s, bytes);
-    ptx::bulk_g2s_hint(tiles + (size_t)s * g.tile_bytes, src, bytes, full + s, ptx::policy_evict_first());
+    ptx::mbar_expect_tx(full + s, nrows * bytes);
+    ptx::bulk_g2s_hint(tiles + (size_t)s * g.slot_bytes, src, nrows * bytes, full + s, ptx::policy_evict_first());
   };
 
   unsigned long long issued = 0;
@@ -408,10 +421,12 @@ __global__ void __launch_bounds__(32) moe_move_kernel(const __grid_constant__ Di
   unsigned long long n = 0;
   for (; n < n_my; ++n) {
     unsigned long long tok;
-    uint32_t off, bytes;
-    item(n, tok, off, bytes);
+    uint32_t nrows, off, bytes;
+    item(n, tok, nrows, off, bytes);
+    // this lane's first store of the item: (row i of the group, slot j); fetched before the wait
+    const uint32_t n_st = nrows * (uint32_t)g.K;
     int row = -1, r = 0;
-    if (lane < g.K) {
+    if ((uint32_t)lane < n_st) {
       row = g.pos[tok * g.K + lane];
       r = g.prank[tok * g.K + lane];
     }
@@ -432,8 +447,16 @@ __global__ void __launch_bounds__(32) moe_move_kernel(const __grid_constant__ Di
     ok = __all_sync(0xFFFFFFFFu, ok);
     if (!ok) { failed = true; break; }
     // every token row is read once and every received row written once: both stream through L2
-    if (row >= 0) ptx::bulk_s2g_hint(static_cast<char*>(P.recv[r]) + (size_t)row * g.row_bytes + off,
-                                     tiles + (size_t)s * g.tile_bytes, bytes, ptx::policy_evict_first());
+    const unsigned char* tile = tiles + (size_t)s * g.slot_bytes;
+    for (uint32_t idx = lane; idx < n_st; idx += 32) {
+      if (idx >= 32) {
+        row = g.pos[tok * g.K + idx];
+        r = g.prank[tok * g.K + idx];
+      }
+      if (row >= 0)
+        ptx::bulk_s2g_hint(static_cast<char*>(P.recv[r]) + (size_t)row * g.row_bytes + off,
+                           tile + (size_t)(idx / (uint32_t)g.K) * bytes, bytes, ptx::policy_evict_first());
+    }
     ptx::bulk_commit();
     if (n >= (unsigned long long)L) {
       ptx::bulk_wait_read<L>();
@@ -537,7 +560,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // it is raised once per device to the most any plan can ask for, so that creating a second,
 // smaller plan cannot lower it under the feet of the first.
 constexpr int kMaxExperts = 4096;
-constexpr size_t kMoveSmemMax = 128 + 8 * (size_t)kMaxTile;
+constexpr size_t kMoveSmemMax = 227 * 1024;
 constexpr size_t kPlanSmemMax = 200 * 1024;  // the fused bookkeeping kernel is used while its tables fit this
 
 size_t plan_smem_bytes(const MoeGeo& g) {
@@ -619,10 +642,17 @@ pl_status_t pl_moe_plan_create(pl_comm_t comm, int tokens_per_rank, int hidden, 
   g.row_bytes = (uint32_t)row_bytes;
   g.n_tiles = (uint32_t)((row_bytes + kMaxTile - 1) / kMaxTile);
   g.tile_bytes = (uint32_t)align_up((row_bytes + g.n_tiles - 1) / g.n_tiles, 16);
-  // at least 4: the move kernel keeps 2 store groups reading their tiles while it refills others
-  g.slots = (uint32_t)std::min<size_t>(8, std::max<size_t>(4, (96 * 1024) / g.tile_bytes));
+  // Rows of at most one tile are moved in groups of consecutive tokens, up to 56 KiB per bulk load,
+  // through exactly three slots: two store groups may still read their tiles while the third tile
+  // is loaded.  Measured at the C4 shape (14,336-byte rows, 8 stores per row): 4 rows x 3 slots
+  // 722-726 us; 4 slots 787 us, 2 or 3 rows per load with 4-6 slots 785-793 us, one row per load
+  // 771 us: the write-dominated stream wants large loads and few bytes in flight.  Wider rows go
+  // tile by tile through at least 4 slots.
+  g.rows_per_item = g.n_tiles == 1 ? (uint32_t)std::max<size_t>(1, std::min<size_t>(32, 57344 / g.tile_bytes)) : 1u;
+  g.slot_bytes = g.rows_per_item * g.tile_bytes;
+  g.slots = g.rows_per_item > 1 ? 3u : (uint32_t)std::min<size_t>(8, std::max<size_t>(4, (96 * 1024) / g.tile_bytes));
   g.cap = recv_capacity_rows;
-  pl->move_smem = 128 + (size_t)g.slots * g.tile_bytes;
+  pl->move_smem = 128 + (size_t)g.slots * g.slot_bytes;
   size_t off = 0;
   auto place = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const size_t o_bc = place((size_t)R * g.NB * g.E * 4);
@@ -726,9 +756,13 @@ static int launch_dispatch(pl_moe_plan_t plan, const DispatchPtrs& P, const MoeG
     launched = 3;
   }
   if (cudaGetLastError() != cudaSuccess) return 0;
-  const unsigned long long items = (unsigned long long)g.R * g.T * g.n_tiles;
-  const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, (200 * 1024) / plan->move_smem));
-  const int mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)plan->sm_count * per_sm);
+  const unsigned long long items = (unsigned long long)g.R * ((g.T + g.rows_per_item - 1) / g.rows_per_item) * g.n_tiles;
+  const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, (227 * 1024) / plan->move_smem));
+  int mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)plan->sm_count * per_sm);
+  // Grouped rows: about 8/9 of the SMs, one CTA each (132 on a B200).  The 1 read : K writes stream
+  // is fastest there: 722-726 us at the C4 shape with 128-132 CTAs, 734-744 us with 136-148, 737 us
+  // with 296 (two per SM), 749-794 us with 112-120.
+  if (g.rows_per_item > 1) mgrid = (int)std::min<unsigned long long>(items, (unsigned long long)((plan->sm_count * 8 / 9 + 3) & ~3));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)mgrid);
   cfg.blockDim = dim3(32);
