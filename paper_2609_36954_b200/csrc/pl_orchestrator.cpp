@@ -188,23 +188,9 @@ void rs_direct(Emitter& em, const Geo& g) {
     }
 }
 
-// all-gather, direct: rank r copies chunk c of every peer's packed input to
-// out + peer*partBytes + offset (Listing 2, scattered output).  Peers are visited starting
-// at r so that the R consumers do not all hit the same producer at once.
-void ag_direct(Emitter& em, const Geo& g) {
-  em.phase_chunks = g.n_c * g.R;
-  for (uint64_t c = 0; c < g.n_c; ++c)
-    for (int i = 0; i < g.R; ++i)
-      for (int r = 0; r < g.R; ++r) {
-        int p = (r + i) % g.R;
-        uint64_t bytes = g.clen(c) * g.es;
-        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, (p * g.P + c * g.chunk) * g.es), false,
-                    {ref(p, PL_BUF_IN, PL_U8, c * g.chunk * g.es)}, bytes, {}, -1);
-      }
-}
-
-// all-gather as a push: rank p writes chunk c of its contribution into slot p of every rank's
-// output (one load, R stores per tile).  Same result as the pull above; the contribution is
+// all-gather, direct, as a push: rank p writes chunk c of its contribution into slot p of every
+// rank's output (one load, R stores per tile; Listing 2's scattered output, out + peer*partBytes +
+// offset, written by the producer).  Same result as a pull by every consumer; the contribution is
 // read once instead of R times, which on one GPU takes the R-1 re-reads out of L2 and the
 // load queue.  (The paper pulls because a pull over NVLink is cheaper than a push, Sec. 3.2;
 // between buffers of one HBM the store count is the same either way.)
@@ -282,36 +268,24 @@ void rsv_direct(Emitter& em, int R, int dtype, const uint64_t* n, uint64_t chunk
     }
 }
 
-void agv_direct(Emitter& em, int R, int dtype, const uint64_t* n, uint64_t chunk_bytes, bool push) {
+void agv_direct(Emitter& em, int R, int dtype, const uint64_t* n, uint64_t chunk_bytes) {
   const int es = elem_size(dtype);
-  // pulled (bulk-copy path): at most 512 KiB per chunk, as for the fixed-size all-gather
-  const uint64_t chunk = std::max<uint64_t>(16, push ? chunk_bytes : std::min<uint64_t>(chunk_bytes, 512u << 10));
-  uint64_t max_b = 0, all_chunks = 0;
+  const uint64_t chunk = std::max<uint64_t>(16, chunk_bytes);
+  uint64_t max_b = 0;
   std::vector<uint64_t> off(R, 0);
   for (int p = 0; p < R; ++p) {
     max_b = std::max(max_b, n[p] * es);
-    all_chunks += (n[p] * es + chunk - 1) / chunk;
     if (p) off[p] = off[p - 1] + n[p - 1] * es;
   }
-  // chunk ops per rank: its own contribution when pushed, everybody's when pulled
-  em.phase_chunks = std::max<uint64_t>(1, push ? (max_b + chunk - 1) / chunk : all_chunks);
-  if (push) {  // rank p writes its contribution into every output (see ag_direct_push)
-    for (uint64_t b = 0; b < max_b; b += chunk)
-      for (int p = 0; p < R; ++p) {
-        if (b >= n[p] * es) continue;
-        em.chunk_op(PL_OP_COPY, p, 0, ref(p, PL_BUF_OUT, PL_U8, off[p] + b), true, {ref(p, PL_BUF_IN, PL_U8, b)},
-                    std::min(chunk, n[p] * es - b), {}, -1);
-      }
-    return;
-  }
+  // chunk ops per rank: its own contribution
+  em.phase_chunks = std::max<uint64_t>(1, (max_b + chunk - 1) / chunk);
+  // rank p writes its contribution into every output (see ag_direct_push)
   for (uint64_t b = 0; b < max_b; b += chunk)
-    for (int i = 0; i < R; ++i)
-      for (int r = 0; r < R; ++r) {
-        const int p = (r + i) % R;
-        if (b >= n[p] * es) continue;
-        em.chunk_op(PL_OP_COPY, r, 0, ref(r, PL_BUF_OUT, PL_U8, off[p] + b), false, {ref(p, PL_BUF_IN, PL_U8, b)},
-                    std::min(chunk, n[p] * es - b), {}, -1);
-      }
+    for (int p = 0; p < R; ++p) {
+      if (b >= n[p] * es) continue;
+      em.chunk_op(PL_OP_COPY, p, 0, ref(p, PL_BUF_OUT, PL_U8, off[p] + b), true, {ref(p, PL_BUF_IN, PL_U8, b)},
+                  std::min(chunk, n[p] * es - b), {}, -1);
+    }
 }
 
 // ---- rooted collectives (Appendix B of the paper: layouts plus a Root role) ----------------
@@ -829,7 +803,13 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
   p.max_slice = latency ? 32768 : (p.datapath == PL_DP_TMA ? 262144 : 131072);
   if (max_resident_ctas <= 0) return p;
   if (p.n_ctas <= 0) {
-    const int full = std::max(rq.R, max_resident_ctas / rq.R * rq.R);
+    int full = std::max(rq.R, max_resident_ctas / rq.R * rq.R);
+    // Pushed copies on the bulk-copy datapath (all-gather(-v), broadcast) are a 1 read : R writes
+    // stream, which this GPU's memory system serves fastest with about 9 of 10 SMs writing
+    // (measured, 148 SMs: 128-136 CTAs 6.15-6.3 TB/s, 140-148 CTAs 5.65-5.73 TB/s): 136 of 148.
+    if (p.datapath == PL_DP_TMA && (rq.coll == PL_ALLGATHER || rq.coll == PL_ALLGATHERV || rq.coll == PL_BROADCAST) &&
+        rq.algo == PL_ALGO_DIRECT && !rq.staged)
+      full = std::max(rq.R, (max_resident_ctas * 92 / 100) / rq.R * rq.R);
     // bytes a rank produces in its busiest phase
     uint64_t per_rank = msg;
     if (rq.coll == PL_REDUCE_SCATTER || rq.coll == PL_REDUCE_SCATTERV) per_rank = msg / rq.R;
@@ -938,7 +918,7 @@ pl_status_t lower_collective(const BuildRequest& rq, Lowered* L, std::string* er
     }
     L->message_bytes = total;
     em.phase_chunks = 0;
-    if (rq.coll == PL_ALLGATHERV) agv_direct(em, R, dt, rq.counts_v, rq.chunk_bytes, rq.pol.datapath == PL_DP_LDST);
+    if (rq.coll == PL_ALLGATHERV) agv_direct(em, R, dt, rq.counts_v, rq.chunk_bytes);
     else rsv_direct(em, R, dt, rq.counts_v, rq.chunk_bytes);
     return PL_OK;
   }
@@ -1014,16 +994,13 @@ pl_status_t lower_collective(const BuildRequest& rq, Lowered* L, std::string* er
       if (rq.staged && rq.algo != PL_ALGO_DIRECT) return fail(PL_ERR_UNSUPPORTED, "staged schedules are direct only");
       if (rq.staged) ag_direct_staged(em, g, rq.staging_bytes);
       else if (rq.algo == PL_ALGO_DIRECT) {
-        // No op of a direct all-gather waits or signals, so the chunk size only orders the copy
-        // ops.  On the bulk-copy datapath at most 512 KiB per chunk: the ranks then walk the
-        // sources in step and the seven re-reads of a contribution hit L2 (measured, R = 8,
-        // 64 MiB gathered per rank: 108.5 us with 1 MiB chunks, 105 us with 256 or 512 KiB).
-        if (rq.pol.datapath == PL_DP_TMA && rq.chunk_bytes > (512u << 10)) g = make_geo(R, dt, n * R, n, 512u << 10);
-        // Register path (working set in L2): push, one read per contribution (measured, R = 8,
-        // 8 MiB gathered per rank: 19.9 -> 12.0 us per call; 1 MiB: 4.4 -> 3.2 us).  Bulk-copy
-        // path (streaming from HBM): pull; there the push is slower (64 MiB: 113 vs 106 us).
-        if (rq.pol.datapath == PL_DP_LDST) ag_direct_push(em, g);
-        else ag_direct(em, g);
+        // A push on both datapaths: rank p reads each chunk of its contribution once and writes
+        // it into all R outputs.  Register path (working set in L2), R = 8: 8 MiB gathered per rank
+        // 19.9 -> 12.0 us against the pull, 1 MiB 4.4 -> 3.2 us.  Bulk-copy path (streaming from
+        // HBM), 64 MiB gathered per rank: 101 us with 128-136 CTAs (the grid the policy picks for
+        // this 1 read : R writes stream) against 104-106 us for the pull with 144 CTAs; with 144
+        // CTAs the push takes 112 us, which is why the grid matters.
+        ag_direct_push(em, g);
       } else if (rq.algo == PL_ALGO_RING) ag_ring(em, g, false, nullptr);
       else return fail(PL_ERR_UNSUPPORTED, "all-gather supports direct and ring");
       return PL_OK;

@@ -6,7 +6,7 @@
 // ceilings that bound them: a pure read (reduce-scatter and MoE combine are 8 reads to
 // 1 write), a pure write, a copy, and one read to eight writes (all-gather and MoE dispatch).
 //
-// One warp per CTA, one CTA per SM, a ring of 6 tiles of 32 KiB.  CTA c handles tiles
+// One warp per CTA, one CTA per SM (132 CTAs for the 1 : 8 stream), a ring of 6 tiles of 32 KiB.  CTA c handles tiles
 // c, c + G, c + 2G, ...: at any moment the grid sweeps one compact window of the buffer.
 #include <cuda_runtime.h>
 
@@ -131,7 +131,10 @@ extern "C" pl_status_t pl_probe_hbm(int kind, const void* src, void* dst, size_t
   }
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   if (status && cudaMemsetAsync(status, 0, sizeof(int32_t), cs) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
-  pl_probe_kernel<<<sms, 32, kSmem, cs>>>(kind, static_cast<const char*>(src), static_cast<char*>(dst),
+  // The write-dominated stream is fastest with about 8/9 of the SMs writing (132 of 148: 6.15 TB/s
+  // against 5.7 TB/s with one CTA on every SM); the other streams want them all.
+  const int grid = kind == 3 ? ((sms * 8 / 9 + 3) & ~3) : sms;
+  pl_probe_kernel<<<grid, 32, kSmem, cs>>>(kind, static_cast<const char*>(src), static_cast<char*>(dst),
                                           (unsigned long long)(bytes / kTile), reinterpret_cast<int*>(status));
   if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
   g_launches.fetch_add(1);

@@ -394,6 +394,7 @@ def test_hbm_bytes_count_every_input_byte_once():
         want = {
             (B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n): (R + 1) * M,                 # read everything once, write M / R per rank
             (B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R): (R + 1) * M,                 # contributions once, R * M written
+            (B.PL_ALLGATHER, B.PL_ALGO_RING, n // R): (R + 1) * M + (R - 2) * M,      # + what the hops re-read from outputs
             (B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT, n): 2 * R * M,                       # inputs once (not R times), R * M written
             (B.PL_ALLREDUCE, B.PL_ALGO_DIRECT_FUSED, n): 2 * R * M,
             (B.PL_ALLREDUCE, B.PL_ALGO_DIRECT, n): R * M + M + (R - 1) * M + (R - 1) * M,  # + reduced partitions re-read by R - 1 ranks
@@ -448,10 +449,11 @@ def test_schedule_bytes_match_closed_forms_bf16_R8():
             return i.bytes_read + i.bytes_written
         assert total(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT) == (R + 1) * M
         assert total(B.PL_REDUCE_SCATTER, B.PL_ALGO_RING) == 33 * M  # fp32 partials: (16+10(R-3))/2 per byte
-        # per-rank-message M = gathered size; pulled (bulk-copy path): every rank reads and writes it all;
-        # pushed (register path): each contribution is read once and written R times
-        assert total(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, datapath=B.PL_DP_TMA) == 2 * R * M
+        # per-rank-message M = gathered size; the direct all-gather is a push on both datapaths: each
+        # contribution is read once and written R times; the ring copies it hop by hop
+        assert total(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, datapath=B.PL_DP_TMA) == (R + 1) * M
         assert total(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, datapath=B.PL_DP_LDST) == (R + 1) * M
+        assert total(B.PL_ALLGATHER, B.PL_ALGO_RING, n // R) == 2 * R * M
         assert total(B.PL_ALLREDUCE, B.PL_ALGO_ONESHOT) == R * (R + 1) * M
         assert total(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT) == (3 * R - 1) * M
         assert total(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT_FUSED) == 2 * R * M
