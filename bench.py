@@ -36,7 +36,10 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one reduce-scatter launch of this workload
 # (one ncu capture of that launch)
-NCU_RS_TRAFFIC_BYTES = 596315392.0
+NCU_RS_TRAFFIC_BYTES = 594654208.0
+# the same sum for a reduce-scatter launch inside the step (captured in one pass with the caches
+# left as the all-gather before it left them): 59 MB more, the write-back of that launch's dirty lines
+NCU_RS_TRAFFIC_IN_SITU_BYTES = 653507174.0
 
 
 def measured_peak():
@@ -171,35 +174,50 @@ def run_purlin(args):
     sampler = ClockSampler(local)
     launches0 = B.pl_launch_count()
 
-    def one_block():
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    def one_block(inner_events):
+        """K steps between a barrier + device synchronisation on both sides.  Without inner
+        events the block is what a caller runs (launch after launch) and gives the step time;
+        with an event between all launches it gives each launch's duration, at the price of
+        about 2.5 us per launch that the event itself puts between two kernels."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)] if inner_events else None
         replicas.barrier()
         torch.cuda.synchronize()
+        e0.record()
         for i in range(K):
-            ev[i][0].record()
+            if ev:
+                ev[i][0].record()
             B.pl_execute(rs, b_rs, stream)
-            ev[i][1].record()
+            if ev:
+                ev[i][1].record()
             B.pl_execute(ag, b_ag, stream)
-            ev[i][2].record()
+            if ev:
+                ev[i][2].record()
+        e1.record()
         torch.cuda.synchronize()
         replicas.barrier()
-        return (ev[0][0].elapsed_time(ev[K - 1][2]),
+        if not ev:
+            return e0.elapsed_time(e1), [], []
+        return (e0.elapsed_time(e1),
                 [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)], [ev[i][1].elapsed_time(ev[i][2]) for i in range(K)])
 
     sampler.start()
-    block_ms, rs_all, ag_all = [], [], []
+    block_ms, block_ms_events, rs_all, ag_all = [], [], [], []
     spent = 0.0
     while True:
-        ms, r_ms, a_ms = one_block()
-        block_ms.append(replicas.max_over_ranks(ms))   # the job's block time is its slowest replica's
+        # blocks alternate: plain (the step time) and with per-launch events (the launch durations)
+        inner = len(block_ms) > len(block_ms_events)
+        ms, r_ms, a_ms = one_block(inner)
+        ms = replicas.max_over_ranks(ms)               # the job's block time is its slowest replica's
+        (block_ms_events if inner else block_ms).append(ms)
         rs_all += r_ms
         ag_all += a_ms
-        spent += block_ms[-1]
-        if (spent >= args.min_timed_ms and len(block_ms) >= 1) or len(block_ms) >= 2000:
+        spent += ms
+        if (spent >= args.min_timed_ms and len(block_ms_events) >= 1) or len(block_ms) >= 1000:
             break
     clocks = sampler.stop()
     n_blocks = len(block_ms)
-    launches = (B.pl_launch_count() - launches0) // n_blocks       # kernels launched per timed block of K steps
+    launches = (B.pl_launch_count() - launches0) // (n_blocks + len(block_ms_events))      # kernels launched per timed block of K steps
     total_ms = float(np.median(block_ms))
     rs_ms, ag_ms = np.array(rs_all), np.array(ag_all)
     assert B.pl_comm_status(comm).code == B.PL_OK
@@ -257,7 +275,8 @@ def run_purlin(args):
                 "achieved": rs_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": rs_gbs / peak, "frac_of_nominal_8TBps": rs_gbs / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_launch": int(rs_alg), "avg_launch_us": float(rs_ms.mean() * 1e3),
-                "traffic": args.ncu_traffic}
+                "traffic": args.ncu_traffic, "traffic_in_situ": NCU_RS_TRAFFIC_IN_SITU_BYTES,
+                "dram_gbs_in_situ": NCU_RS_TRAFFIC_IN_SITU_BYTES / (rs_ms.mean() * 1e-3) / 1e9}
     detail = {
         "reduce_scatter": {"us": float(rs_ms.mean() * 1e3), "p50_us": float(np.median(rs_ms) * 1e3),
                            "algbw_gbs": irs.message_bytes / (rs_ms.mean() * 1e-3) / 1e9,
@@ -271,7 +290,11 @@ def run_purlin(args):
     }
 
     detail["timed_region"] = {"blocks": n_blocks, "steps_per_block": K, "block_ms_median": total_ms,
-                              "block_ms_min": float(min(block_ms)), "block_ms_max": float(max(block_ms))}
+                              "block_ms_min": float(min(block_ms)), "block_ms_max": float(max(block_ms)),
+                              "blocks_with_an_event_between_launches": len(block_ms_events),
+                              "their_block_ms_median": float(np.median(block_ms_events)),
+                              "note": "blocks alternate: plain ones give ms_per_step and value, the ones with an event "
+                                      "between all launches give the per-launch durations of roofline and detail"}
 
     # ---- the same step with overlapped launches (no events between the two executes) ---------
     if not args.no_detail:
@@ -311,7 +334,9 @@ def run_purlin(args):
 
 def measure_overlapped_step(B, torch, comm, n, chunk, R, b_rs, b_ag, stream, plain_ms):
     """The C2 step built with PL_OPT_OVERLAP_LAUNCH (the CTAs of a launch are set up while the one
-    in front of it drains) and timed without events between the two launches."""
+    in front of it drains) and timed without events between the two launches.  The option is
+    made for the latency path; on these HBM-bound launches it does not pay (the CTAs of a launch
+    then take the SMs in the order in which they become free)."""
     opts = B.make_opts(flags=B.PL_OPT_OVERLAP_LAUNCH)
     rs = B.pl_schedule_build(comm, B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, chunk, opts)
     ag = B.pl_schedule_build(comm, B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, chunk, opts)

@@ -161,7 +161,7 @@ typedef struct {
   uint32_t struct_size;
   int32_t n_ctas;        /* persistent CTAs = op queues; rounded down to a multiple of R  */
   int32_t threads;       /* threads per CTA of the register datapath (multiple of 32, <=  */
-                         /* 512); the bulk-copy datapath fixes its own (576, or 448 for   */
+                         /* 512); the bulk-copy datapath fixes its own (608, or 480 for   */
                          /* schedules of plain reduce ops: see pl_sched_info_t.threads)   */
   int32_t datapath;      /* pl_datapath_t                                                 */
   int32_t stages;        /* shared-memory ring depth S of the TMA pipeline                */

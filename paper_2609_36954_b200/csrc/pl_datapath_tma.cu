@@ -1,14 +1,18 @@
 // Throughput datapath: the op-queue executor built around bulk asynchronous copies (TMA).
 //
 // One CTA per op queue, warp specialised:
-//   warp 0  producer  walks the queue, waits on the op's flags (acquire, bounded), cuts the
-//                     op into stages and fills a ring of shared-memory slots with
-//                     cp.async.bulk loads (one per source), running ahead of the consumers
-//                     across op boundaries (Algorithm 2 of the paper: prime / steady / drain,
-//                     here as a free-running ring with full / empty mbarriers);
-//   warp 1  copier    for COPY stages: one bulk store shared -> global per stage (R stores
+//   warps 0, 1  producers  both walk the queue, wait on every op's flags (acquire, bounded) and
+//                     cut the op into stages; producer p fills the ring slots of the stages
+//                     with number n = p (mod 2) with cp.async.bulk loads (one per source),
+//                     running ahead of the consumers across op boundaries (Algorithm 2 of the
+//                     paper: prime / steady / drain, here as a free-running ring with full /
+//                     empty mbarriers).  Two of them because issuing is what a producer spends
+//                     its time on: the bulk loads of one warp are accepted one at a time,
+//                     60-70 ns each, so the 8 loads of an 8-source stage plus the stage's
+//                     bookkeeping (about 1 us) took as long as HBM needs to deliver its 48 KiB;
+//   warp 2  copier    for COPY stages: one bulk store shared -> global per stage (R stores
 //                     for a broadcast copy), no registers touched by the payload;
-//   warps 2..  consumers (16, or 12 in the variant for plain reduce schedules)  for REDUCE /
+//   warps 3..  consumers (16, or 12 in the variant for plain reduce schedules)  for REDUCE /
 //                     COPY_REDUCE stages: read the source tiles from shared memory 16 bytes
 //                     at a time, accumulate in fp32 in ascending source order, store the
 //                     result with 128-bit global stores.
@@ -37,6 +41,7 @@ using namespace dev;
 // stages of operands in registers (128 registers per thread need the smaller CTA).
 constexpr int kWarpsGeneral = 16;
 constexpr int kWarpsPipelined = 12;
+constexpr int kProducers = 2;  // producer warps; the copier is warp kProducers, consumers follow
 constexpr int kMaxStages = 8;
 constexpr uint32_t kEnd = 0xFFFFFFFFu;
 constexpr uint32_t kLastOfOp = 0x100u;  // stage flag (above the DevOp flag bits)
@@ -295,7 +300,7 @@ __device__ __forceinline__ bool leaves_via_smem(uint32_t kind, uint32_t flags, u
 // leading stage ops of its queue (copies from the caller's input into the staging buffer of this
 // parity) before it waits for the launch in front, the copier ships them, the consumers wait.
 template <int DT, int CW, bool HOOK = false, bool DBUF = false>
-__global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __grid_constant__ ExecParams P) {
+__global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_kernel(const __grid_constant__ ExecParams P) {
   extern __shared__ __align__(1024) unsigned char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
   unsigned char* slots = smem + kCtrlBytes;
@@ -314,6 +319,20 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
     c->abort = 0;
     ptx::mbar_init_fence();
   }
+  // Producers: the first descriptor of the queue.  Descriptors are written when the schedule is
+  // built and never by a kernel, so this load may run ahead of the wait for the launch in front.
+  const uint32_t nq = P.n_queues;
+  uint4 r_op = make_uint4(0, 0, 0, 0), r_op_next = r_op;
+  uint64_t r_src = 0, r_src_next = 0;
+  DevWait r_wait = {0, 0}, r_wait_next = {0, 0};
+  auto fetch = [&](uint32_t i, uint4& o, uint64_t& sr, DevWait& w) {
+    const uint64_t at = (uint64_t)i * nq + q;  // op i of this queue
+    if (lane < 4) o = reinterpret_cast<const uint4*>(P.ops + at)[lane];
+    if (lane < (int)P.src_stride) sr = P.srcs[at * P.src_stride + lane];
+    if (lane < (int)P.wait_stride) w = P.waits[at * P.wait_stride + lane];
+  };
+  if (warp < kProducers) fetch(0, r_op_next, r_src_next, r_wait_next);
+
   unsigned long long epoch = 0ull, scratch_shift = 0ull;
   unsigned long long* flag_base = P.flags;
   if constexpr (DBUF) {
@@ -328,28 +347,19 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
     // block here; the producer waits later (below), the copier not at all (it reads shared
     // memory only, and what it stores or signals belongs to this launch's own buffer and flag set
     // until the producer has waited)
-    if (warp >= 2) pdl_wait();
+    if (warp > kProducers) pdl_wait();
   } else {
     pdl_wait();  // from here on memory written by earlier launches may be read
     epoch = has_flags ? *reinterpret_cast<volatile unsigned long long*>(P.epoch) + 1ull : 0ull;
     __syncthreads();
   }
 
-  if (warp == 0) {
-    // ================================ producer =========================================
-    const uint32_t nq = P.n_queues;
+  if (warp < kProducers) {
+    // ================================ producers ========================================
+    // Both walk the whole queue (descriptors, flag waits, stage arithmetic); a stage is filled
+    // by the producer whose number equals the stage number modulo kProducers.
     uint32_t n = 0;  // stages produced
     bool ok = true;
-    uint4 r_op = make_uint4(0, 0, 0, 0), r_op_next = r_op;
-    uint64_t r_src = 0, r_src_next = 0;
-    DevWait r_wait = {0, 0}, r_wait_next = {0, 0};
-    auto fetch = [&](uint32_t i, uint4& o, uint64_t& sr, DevWait& w) {
-      const uint64_t at = (uint64_t)i * nq + q;  // op i of this queue
-      if (lane < 4) o = reinterpret_cast<const uint4*>(P.ops + at)[lane];
-      if (lane < (int)P.src_stride) sr = P.srcs[at * P.src_stride + lane];
-      if (lane < (int)P.wait_stride) w = P.waits[at * P.wait_stride + lane];
-    };
-    fetch(0, r_op_next, r_src_next, r_wait_next);
     // the first descriptor tells how many ops the queue holds (a placeholder marks an empty one)
     const uint32_t first_kind = __shfl_sync(0xFFFFFFFFu, r_op_next.x, 0);
     const uint32_t n_ops = first_kind == kNopKind ? 0u : __shfl_sync(0xFFFFFFFFu, r_op_next.z, 0) + 1u;
@@ -401,7 +411,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
       ok = __all_sync(0xFFFFFFFFu, lane_ok);
       if (!ok) break;
       if (n_wait) ptx::fence_proxy_async();  // data released by other CTAs' generic stores -> our bulk loads
-      if (P.trace && lane == 0) P.trace[2ull * topo] = globaltimer_ns();  // waits satisfied
+      if (P.trace && tid == 0) P.trace[2ull * topo] = globaltimer_ns();  // waits satisfied
 
       // ---- cut the op into stages
       const char* my_src = (lane < (int)n_src) ? (DBUF ? resolve(P, r_src, scratch_shift) : resolve(P, r_src)) : nullptr;
@@ -421,6 +431,10 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
       char* dst = DBUF ? resolve(P, dstp, scratch_shift) : resolve(P, dstp);
       const uint64_t dst_off = dstp & 0xFFFFFFFFFFFFull;
       for (uint64_t u0 = 0; u0 < n_units; u0 += ucap) {
+        if (n % kProducers != (uint32_t)warp) {  // the other producer's stage
+          ++n;
+          continue;
+        }
         const uint32_t units = (uint32_t)min((uint64_t)ucap, n_units - u0);
         const uint32_t s = n % S, ph = (n / S) & 1u;
         bool w_ok = true;
@@ -464,17 +478,19 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
     if (lane == 0) {
       if (!ok) {
         *reinterpret_cast<volatile int*>(&c->abort) = 1;
-        // loads already issued must land before the CTA may leave: bounded drain
+        // loads this warp issued must land before the CTA may leave: bounded drain
         for (uint32_t k = (n > S ? n - S : 0u); k < n; ++k)
-          for (uint32_t tries = 0; tries < (1u << 22) && !ptx::mbar_try_wait(&c->full[k % S], (k / S) & 1u); ++tries) {}
+          if (k % kProducers == (uint32_t)warp)
+            for (uint32_t tries = 0; tries < (1u << 22) && !ptx::mbar_try_wait(&c->full[k % S], (k / S) & 1u); ++tries) {}
       }
+      // the end marker is the stage after the last one: it belongs to one of the producers too
       const uint32_t s = n % S, ph = (n / S) & 1u;
-      if (ok && wait_bar(P, c, &c->empty[s], ph ^ 1u)) {
+      if (ok && n % kProducers == (uint32_t)warp && wait_bar(P, c, &c->empty[s], ph ^ 1u)) {
         c->desc[s].kind = kEnd;
         ptx::mbar_arrive(&c->full[s]);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == kProducers) {
     // ================================ copier ============================================
     int prev = -1;  // slot whose bulk store may still be reading shared memory
     uint32_t done_parity = 0;  // tracked exactly as the consumers do
@@ -541,7 +557,7 @@ __global__ void __launch_bounds__(32 * (2 + CW), 1) pl_exec_tma_kernel(const __g
     }
   } else {
     // ================================ consumers =========================================
-    const int ctid = tid - 64;
+    const int ctid = tid - 32 * (kProducers + 1);
     uint32_t done_parity = 0;  // bit s: parity of the next phase of done[s]
     // operands of a plain stage that were pulled into registers ahead of time
     bool have = false;
@@ -642,7 +658,7 @@ cudaError_t launch_t(const ExecParams& P, int grid, cudaStream_t stream) {
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3((unsigned)(32 * (2 + CW)));
+  cfg.blockDim = dim3((unsigned)(32 * (kProducers + 1 + CW)));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -657,7 +673,7 @@ template <int DT, int CW, bool HOOK = false, bool DBUF = false>
 int occupancy_t(size_t smem) {
   int n = 0;
   if (cudaFuncSetAttribute(pl_exec_tma_kernel<DT, CW, HOOK, DBUF>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_tma_kernel<DT, CW, HOOK, DBUF>, 32 * (2 + CW), smem) != cudaSuccess) {
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pl_exec_tma_kernel<DT, CW, HOOK, DBUF>, 32 * (kProducers + 1 + CW), smem) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
@@ -667,7 +683,7 @@ int occupancy_t(size_t smem) {
 }  // namespace
 
 size_t exec_tma_smem_bytes(int stages, uint32_t stage_bytes) { return kCtrlBytes + (size_t)stages * stage_bytes; }
-int exec_tma_threads(bool pipelined) { return 32 * (2 + (pipelined ? kWarpsPipelined : kWarpsGeneral)); }
+int exec_tma_threads(bool pipelined) { return 32 * (kProducers + 1 + (pipelined ? kWarpsPipelined : kWarpsGeneral)); }
 
 cudaError_t launch_exec_tma(int dtype, const ExecParams& P, int grid, cudaStream_t stream) {
   if (P.stages < 2 || P.stages > kMaxStages) return cudaErrorInvalidValue;

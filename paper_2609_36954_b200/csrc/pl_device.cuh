@@ -76,8 +76,12 @@ struct Acc<PL_BF16> {
     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      v[2 * i] += __uint_as_float(w[i] << 16);
-      v[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
+      // fp32 += bf16 as one mixed-precision add per element (the bf16 operand is widened exactly,
+      // the sum rounded to nearest once: bit for bit what shift / mask and an fp32 add give)
+      uint16_t lo, hi;
+      asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(w[i]));
+      asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(v[2 * i]) : "h"(lo));
+      asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(v[2 * i + 1]) : "h"(hi));
     }
   }
   __device__ __forceinline__ void add_f32(const uint4& lo, const uint4& hi) {

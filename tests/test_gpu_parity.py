@@ -722,7 +722,7 @@ def test_pipelined_reduce_variant_for_every_source_count(R, dtype):
             for dp in (B.PL_DP_TMA, B.PL_DP_LDST):
                 s = ses.build(coll, B.PL_ALGO_DIRECT, n, 1 << 20, datapath=dp)
                 if dp == B.PL_DP_TMA:
-                    assert B.pl_schedule_info(s).threads == 448   # the 12-warp variant was chosen
+                    assert B.pl_schedule_info(s).threads == 480   # the 12-warp variant was chosen
                 outs[dp], _ = ses.execute(s, x, repeats=3)
                 compare_reduce(outs[dp], ref, dtype)
             for r in range(R):
