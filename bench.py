@@ -37,9 +37,10 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one reduce-scatter launch of this workload
 # (one ncu capture of that launch)
 NCU_RS_TRAFFIC_BYTES = 594654208.0
-# the same sum for a reduce-scatter launch inside the step (captured in one pass with the caches
-# left as the all-gather before it left them): 59 MB more, the write-back of that launch's dirty lines
-NCU_RS_TRAFFIC_IN_SITU_BYTES = 653507174.0
+# the same sum for a reduce-scatter launch inside the step (one pass, caches left as the
+# all-gather before it left them, both schedules with PL_OPT_INPUTS_LAST_USE): 20 MB more, the
+# write-back of dirty lines it inherits
+NCU_RS_TRAFFIC_IN_SITU_BYTES = 615150000.0
 
 
 def measured_peak():
@@ -140,8 +141,11 @@ def run_purlin(args):
     # the full-size inputs are generated exactly (seeded, per rank) unless --fast-inputs
     x = c2_inputs(R, n, seed=0, unique=(4 * MIB if args.fast_inputs else None))
     comm = B.pl_comm_create(R, B.PL_BF16)
+    # Both launches read their inputs for the last time (the reduce-scatter consumes the
+    # contributions, the all-gather the reduced partition): PL_OPT_INPUTS_LAST_USE says so.
+    step_flags = 0 if args.plain_options else B.PL_OPT_INPUTS_LAST_USE
     opts = B.make_opts(n_ctas=args.n_ctas, threads=args.threads, slice_bytes=args.slice_bytes,
-                       datapath=args.datapath, stages=args.stages, stage_bytes=args.stage_bytes)
+                       datapath=args.datapath, stages=args.stages, stage_bytes=args.stage_bytes, flags=step_flags)
     rs = B.pl_schedule_build(comm, B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, chunk, opts)
     ag = B.pl_schedule_build(comm, B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, chunk, opts)
     irs, iag = B.pl_schedule_info(rs), B.pl_schedule_info(ag)
@@ -298,7 +302,9 @@ def run_purlin(args):
 
     # ---- the same step with overlapped launches (no events between the two executes) ---------
     if not args.no_detail:
-        detail["step_overlapped_launches"] = measure_overlapped_step(B, torch, comm, n, chunk, R, b_rs, b_ag, stream, ms_per_step)
+        detail["step_overlapped_launches"] = measure_step_variant(B, torch, comm, n, chunk, R, b_rs, b_ag, stream, ms_per_step,
+                                                                  step_flags | B.PL_OPT_OVERLAP_LAUNCH)
+        detail["step_without_last_use_hint"] = measure_step_variant(B, torch, comm, n, chunk, R, b_rs, b_ag, stream, ms_per_step, 0)
 
     # free the headline buffers before the other configurations allocate theirs
     del d_in, d_mid, d_out, b_rs, b_ag, pinned_in
@@ -320,6 +326,7 @@ def run_purlin(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "C2: reduce-scatter (64 MiB/rank in) then all-gather (64 MiB/rank out), "
                                    "R=8 emulated ranks in one HBM, bf16 N(0,1) seed 0, direct schedules, 1 MiB chunks",
+                       "options": "default" if args.plain_options else "PL_OPT_INPUTS_LAST_USE on both schedules (inputs loaded evict-first)",
                        "l2": "inputs_larger_than_l2 (512 MiB of inputs per step; no flush)",
                        "replicas": world, "parallelism": "replicas only (no inter-GPU exchange on this path)"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
@@ -332,12 +339,13 @@ def run_purlin(args):
     replicas.finalize()
 
 
-def measure_overlapped_step(B, torch, comm, n, chunk, R, b_rs, b_ag, stream, plain_ms):
-    """The C2 step built with PL_OPT_OVERLAP_LAUNCH (the CTAs of a launch are set up while the one
-    in front of it drains) and timed without events between the two launches.  The option is
-    made for the latency path; on these HBM-bound launches it does not pay (the CTAs of a launch
-    then take the SMs in the order in which they become free)."""
-    opts = B.make_opts(flags=B.PL_OPT_OVERLAP_LAUNCH)
+def measure_step_variant(B, torch, comm, n, chunk, R, b_rs, b_ag, stream, plain_ms, flags):
+    """The C2 step built with other schedule options and timed without events between the two
+    launches.  PL_OPT_OVERLAP_LAUNCH (the CTAs of a launch are set up while the one in front of it
+    drains) is made for the latency path; on these HBM-bound launches it does not pay (the CTAs of
+    a launch then take the SMs in the order in which they become free).  flags = 0 is the step
+    without PL_OPT_INPUTS_LAST_USE."""
+    opts = B.make_opts(flags=flags)
     rs = B.pl_schedule_build(comm, B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, chunk, opts)
     ag = B.pl_schedule_build(comm, B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, chunk, opts)
     for _ in range(5):
@@ -355,7 +363,7 @@ def measure_overlapped_step(B, torch, comm, n, chunk, R, b_rs, b_ag, stream, pla
     ms = e0.elapsed_time(e1) / reps
     B.pl_schedule_destroy(rs)
     B.pl_schedule_destroy(ag)
-    return {"ms_per_step": ms, "steps": reps, "vs_plain_step": ms / plain_ms}
+    return {"ms_per_step": ms, "steps": reps, "vs_headline_step": ms / plain_ms}
 
 
 def measure_all_configs(peak):
@@ -634,6 +642,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-latency", action="store_true")
     ap.add_argument("--no-detail", action="store_true", help="skip the other configurations (C1, C3, C4, C5, stream ceilings)")
+    ap.add_argument("--plain-options", action="store_true", help="build the two schedules of the step without PL_OPT_INPUTS_LAST_USE")
     ap.add_argument("--min-timed-ms", type=float, default=500.0, help="repeat the K-step block until the timed region lasts this long")
     ap.add_argument("--fast-inputs", action="store_true", help="tile 4 Mi generated elements instead of generating all")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)

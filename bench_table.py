@@ -41,7 +41,14 @@ def main(path):
           f"end to end {f(line['e2e']['value'], 2)} GB/s; clocks {line['clocks']['sm_mhz']} MHz {line['clocks']['reasons']}.")
     if "step_overlapped_launches" in d:
         o = d["step_overlapped_launches"]
-        print(f"Step with overlapped launches: {f(o['ms_per_step'] * 1e3, 1)} us ({f(o['vs_plain_step'], 3)} of the plain step).")
+        print(f"Step with overlapped launches: {f(o['ms_per_step'] * 1e3, 1)} us ({f(o['vs_headline_step'], 3)} of the headline step).")
+    if "step_without_last_use_hint" in d:
+        o = d["step_without_last_use_hint"]
+        print(f"Step without PL_OPT_INPUTS_LAST_USE: {f(o['ms_per_step'] * 1e3, 1)} us ({f(o['vs_headline_step'], 3)} of the headline step).")
+    r = line["roofline"]
+    if "traffic_in_situ" in r:
+        print(f"Reduce-scatter DRAM traffic per launch: {f(r['traffic'] / 1e6, 1)} MB captured alone, {f(r['traffic_in_situ'] / 1e6, 1)} MB inside the step "
+              f"({f(r['dram_gbs_in_situ'], 0)} GB/s of DRAM traffic in situ).")
     c = d.get("configs")
     if not c:
         return

@@ -228,7 +228,18 @@ typedef struct {
  * here the launch counter itself is the epoch and its lowest bit the parity. */
 #define PL_OPT_STAGE_AHEAD 32u
 #define PL_OPT_NO_L2_HINTS 2u  /* bulk copies without L2 eviction hints (default: stores evict-first,
-                                  sources of copy ops evict-last; measured 7 % on all-gather) */
+                                  sources of copy ops evict-last) */
+/* The caller's input buffers are read here for the last time (gradients that the reduce-scatter
+ * consumes, the partition an all-gather spreads): the bulk-copy datapath then loads them with an
+ * L2 evict-first hint, so that the stream of inputs displaces itself from L2 and not what this
+ * launch writes or what the launch behind it is about to read.  Measured on the reduce-scatter ->
+ * all-gather step (8 x 64 MiB): the all-gather finds the reduce-scatter's 64 MiB of results in L2
+ * (6 MB of DRAM reads instead of 67 MB) and the step takes 5 % less; a launch repeated on its own
+ * is 1-2 % slower with the hint, which is why it is not the default.  Ignored by schedules that
+ * read an input byte more than once (one-shot all-reduce), by the register and packet datapaths
+ * and together with PL_OPT_NO_L2_HINTS.  Nothing in the paper corresponds to this option (its
+ * inputs live in other GPUs' memories). */
+#define PL_OPT_INPUTS_LAST_USE 64u
 
 /* A buffer reference inside an op: rank's in/out/scratch buffer, byte offset, and the
  * element type stored there (partials of a bf16 reduction are PL_F32). */

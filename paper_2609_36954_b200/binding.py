@@ -39,6 +39,7 @@ PL_OPT_STAGED = 4
 PL_OPT_TRACE = 8
 PL_OPT_OVERLAP_LAUNCH = 16
 PL_OPT_STAGE_AHEAD = 32
+PL_OPT_INPUTS_LAST_USE = 64
 PL_HOOK_RESIDUAL = 1
 PL_HOOK_F32_OUT = 2
 

@@ -38,6 +38,7 @@ struct pl_schedule_s {
   pl_sched_info_t info{};
   uint64_t timeout_ns = 0;
   bool no_l2_hints = false;
+  bool inputs_last_use = false;   // PL_OPT_INPUTS_LAST_USE asked for and every input byte is read once
   bool trace = false;
   bool overlap_launch = false;
   bool bcast_copies = false;      // some COPY op writes every rank's output
@@ -107,7 +108,9 @@ void fill_info(pl_schedule_s* S, int R) {
         if (s.buf == PL_BUF_IN) ranges[s.rank].emplace_back(s.offset, s.offset + b);
         else other_reads += b;
       }
-    uint64_t in_once = 0;
+    uint64_t in_once = 0, in_reads = 0;
+    for (const auto& v : ranges)
+      for (const auto& iv : v) in_reads += iv.second - iv.first;
     for (auto& v : ranges) {
       std::sort(v.begin(), v.end());
       uint64_t hi = 0;
@@ -120,6 +123,7 @@ void fill_info(pl_schedule_s* S, int R) {
     uint64_t aux_reads = 0;
     for (int r = 0; r < R; ++r) aux_reads += L.aux_bytes[r];
     I.hbm_bytes = in_once + other_reads + aux_reads + I.bytes_written;
+    if (in_reads != in_once) S->inputs_last_use = false;  // some input byte is read more than once
   }
   I.out_dtype = (S->hook & PL_HOOK_F32_OUT) ? PL_F32 : S->comm->dtype;
   I.hook = S->hook;
@@ -385,6 +389,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   S->pol = pol;
   S->timeout_ns = timeout;
   S->no_l2_hints = (flags & PL_OPT_NO_L2_HINTS) != 0;
+  S->inputs_last_use = (flags & PL_OPT_INPUTS_LAST_USE) && !S->no_l2_hints;
   S->trace = (flags & PL_OPT_TRACE) != 0;
   S->overlap_launch = (flags & PL_OPT_OVERLAP_LAUNCH) != 0;
   S->stage_ahead = (flags & PL_OPT_STAGE_AHEAD) != 0;
@@ -807,7 +812,7 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   P.stages = s->pol.stages;
   P.stage_bytes = s->pol.stage_bytes;
   // bulk stores stream out (evict-first), sources of copies are re-read by other ranks (evict-last)
-  P.hints = s->no_l2_hints ? 0u : 6u;
+  P.hints = s->no_l2_hints ? 0u : (6u | (s->inputs_last_use ? 1u : 0u));
   P.out_scale = s->out_scale;
   P.overlap_launch = s->overlap_launch ? 1u : 0u;
   P.pipelined_reduce = s->pipelined_reduce ? 1u : 0u;

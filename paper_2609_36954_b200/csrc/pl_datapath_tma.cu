@@ -462,7 +462,7 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
         if (lane < (int)n_src) {
           void* sdst = slots + (size_t)s * slot_bytes + my_tile_off;
           if ((P.hints & 4u) && kind == PL_OP_COPY && !(oflags & kDstBcast)) ptx::bulk_g2s_hint(sdst, my_src + u0 * my_w, units * my_w, &c->full[s], ptx::policy_evict_last());
-          else if (P.hints & 1u) ptx::bulk_g2s_hint(sdst, my_src + u0 * my_w, units * my_w, &c->full[s], ptx::policy_evict_first());
+          else if ((P.hints & 1u) && (r_src >> 48) < (uint64_t)kSlotOut) ptx::bulk_g2s_hint(sdst, my_src + u0 * my_w, units * my_w, &c->full[s], ptx::policy_evict_first());
           else ptx::bulk_g2s(sdst, my_src + u0 * my_w, units * my_w, &c->full[s]);
         }
         ++n;

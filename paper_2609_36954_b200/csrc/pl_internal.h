@@ -97,7 +97,7 @@ struct ExecParams {
   uint32_t stage_bytes;  // bytes per ring slot
   float out_scale;       // multiplies every final (element-typed) sum; 1 = plain sum
   uint32_t hook;         // PL_HOOK_* bits (host side: selects the kernel variant; device: what final ops do)
-  uint32_t hints;        // L2 policy bits for bulk copies: 1 loads evict-first, 2 stores evict-first, 4 copy loads evict-last
+  uint32_t hints;        // L2 policy bits for bulk copies: 1 loads of the caller's inputs evict-first, 2 stores evict-first, 4 copy loads evict-last
   uint32_t overlap_launch;  // host side only: launch with the programmatic stream serialization attribute
   uint32_t bcast_copies;      // host side only: the schedule holds broadcast copy ops (register executor variant)
   uint32_t pipelined_reduce;  // host side only: every reduce op is plain (element-typed operands), use the 12-warp variant
