@@ -335,6 +335,20 @@ pl_status_t pl_comm_create_planner(int R, pl_dtype_t dtype, pl_comm_t* out);
  * (PL_ERR_INVALID_ARG otherwise). */
 pl_status_t pl_comm_destroy(pl_comm_t comm);
 
+/* Measure, on this communicator's GPU, the grid with which the write-dominated direct schedules
+ * of the bulk-copy datapath (all-gather, all-gather-v, broadcast: 1 read : R writes) run fastest,
+ * and make it the default of later builds on this communicator (opts.n_ctas still overrides; the
+ * schedules already built keep theirs).  Such a stream is served best with fewer than all SMs
+ * writing, and how many differs from one GPU to the next of the same model (of two B200s one ran
+ * the 8 x 64 MiB all-gather fastest with 136 CTAs, the other with 128: 113 us with 136).  Runs an
+ * all-gather of 64 MiB with every multiple of R between 3/4 of the resident CTAs and all of them
+ * (2 + 6 launches each) on `stream`, on buffers it allocates and frees ((R + 1) x 64 MiB), and
+ * synchronises: a call for set-up time, not for the hot path.  Nothing in the paper corresponds
+ * to it.  *push_ctas_out (may be NULL) receives the chosen grid.
+ * Errors: PL_ERR_UNSUPPORTED (planner communicator), PL_ERR_OOM, PL_ERR_CUDA, PL_ERR_INVALID_ARG
+ * (the current device is not the communicator's). */
+pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out);
+
 /* Read the device status record as it stands at the time of the call (on an internal stream: the
  * call waits for no other work, so synchronise the stream of the executes you ask about first).
  * Returns PL_OK and fills *out; out->code tells whether a wait timed out since the last reset. */
@@ -456,6 +470,28 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream);
  * staging buffers (caller-owned).  Sizes come from pl_schedule_info. */
 pl_status_t pl_execute_host(pl_schedule_t s, const pl_bufs_t* host, const pl_bufs_t* dev,
                             void* stream);
+
+/* Pipelined form of pl_execute_host for a sequence of host executes on one communicator (no
+ * counterpart in the paper, whose data never leaves the GPUs): the uploads run on an upload
+ * stream of the communicator, the schedule on `stream`, the downloads on a download stream, tied
+ * together by events, so that the download of one call overlaps the upload of the next (the host
+ * link carries both directions at once).  What is ordered: an upload waits for the schedule of
+ * the previous async host execute (which read the device inputs it overwrites) and for every
+ * download still in flight that writes a host range it reads or reads a device range it
+ * overwrites; the schedule waits for its uploads and for every download that still reads device
+ * outputs it overwrites; downloads run in call order.  What is NOT ordered: other work the caller
+ * puts on `stream` between two async host executes is waited for only by the first call and
+ * after a change of stream, so the device staging buffers in `dev` must not be touched by such
+ * work; and `stream` does not wait for the downloads: the host outputs are complete after
+ * pl_comm_host_sync (host blocks) or behind pl_comm_host_fence (the given stream waits).
+ * Allocates nothing after the first call (two streams and a fixed set of events).  Arguments and
+ * errors as pl_execute_host. */
+pl_status_t pl_execute_host_async(pl_schedule_t s, const pl_bufs_t* host, const pl_bufs_t* dev,
+                                  void* stream);
+/* Make `stream` wait (asynchronously) for all downloads of earlier pl_execute_host_async calls. */
+pl_status_t pl_comm_host_fence(pl_comm_t comm, void* stream);
+/* Block the calling thread until all downloads of earlier pl_execute_host_async calls are done. */
+pl_status_t pl_comm_host_sync(pl_comm_t comm);
 
 /* ---- MoE expert-parallel dispatch / combine (all-to-all-v of token rows) ------------ */
 

@@ -100,7 +100,7 @@ EXPORTS = [
     "pl_schedule_build", "pl_schedule_build_v", "pl_schedule_build_layers", "pl_schedule_build_rooted", "pl_schedule_info",
     "pl_schedule_dump", "pl_schedule_validate", "pl_schedule_debug_break_wait", "pl_schedule_debug_drop_wait",
     "pl_schedule_trace_read", "pl_schedule_destroy",
-    "pl_execute", "pl_execute_host",
+    "pl_execute", "pl_execute_host", "pl_execute_host_async", "pl_comm_host_fence", "pl_comm_host_sync", "pl_comm_tune",
     "pl_moe_plan_create", "pl_moe_plan_destroy", "pl_moe_dispatch", "pl_moe_combine", "pl_moe_plan_read",
     "pl_moe_dispatch_dedup", "pl_moe_combine_dedup", "pl_moe_plan_read_dedup", "pl_moe_combine_logits",
     "pl_status_string", "pl_launch_count", "pl_reduce_scatter_ring_static",
@@ -146,6 +146,10 @@ def load():
         "pl_schedule_destroy": [vp],
         "pl_execute": [vp, P(pl_bufs_t), vp],
         "pl_execute_host": [vp, P(pl_bufs_t), P(pl_bufs_t), vp],
+        "pl_execute_host_async": [vp, P(pl_bufs_t), P(pl_bufs_t), vp],
+        "pl_comm_host_fence": [vp, vp],
+        "pl_comm_host_sync": [vp],
+        "pl_comm_tune": [vp, vp, P(C.c_int32)],
         "pl_moe_plan_create": [vp, i32, i32, i32, i32, sz, P(vp)],
         "pl_moe_plan_destroy": [vp],
         "pl_moe_dispatch": [vp, P(vp), P(vp), P(vp), P(vp), vp],
@@ -326,6 +330,25 @@ def pl_execute(s, bufs, stream=0):
 
 def pl_execute_host(s, host_bufs, dev_bufs, stream=0):
     _check(load().pl_execute_host(s, C.byref(host_bufs), C.byref(dev_bufs), stream), "pl_execute_host")
+
+
+def pl_execute_host_async(s, host_bufs, dev_bufs, stream=0):
+    _check(load().pl_execute_host_async(s, C.byref(host_bufs), C.byref(dev_bufs), stream), "pl_execute_host_async")
+
+
+def pl_comm_host_fence(comm, stream=0):
+    _check(load().pl_comm_host_fence(comm, stream), "pl_comm_host_fence")
+
+
+def pl_comm_tune(comm, stream=0):
+    """Returns the grid chosen for pushed copies on the bulk-copy datapath."""
+    g = C.c_int32(0)
+    _check(load().pl_comm_tune(comm, stream, C.byref(g)), "pl_comm_tune")
+    return int(g.value)
+
+
+def pl_comm_host_sync(comm):
+    _check(load().pl_comm_host_sync(comm), "pl_comm_host_sync")
 
 
 def _ptr_array(addrs):

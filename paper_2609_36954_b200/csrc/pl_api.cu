@@ -361,6 +361,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   }
   if (pol.datapath == PL_DP_PACKET) return build_packets(comm, rq, pol, timeout, flags, out_scale, out);
   rq.pol = pol;
+  rq.tuned_push_ctas = comm->tuned_push_ctas;
   const int requested = pol.n_ctas;
   pol = default_policy(rq, 0);  // datapath, threads, ring geometry
   rq.pol = pol;
@@ -455,6 +456,99 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
 }  // namespace
 
 extern "C" {
+static pl_status_t check_bufs(pl_schedule_t s, const pl_bufs_t* b);
+}
+
+namespace {
+
+void host_pipeline_destroy(pl_comm_s* comm) {
+  if (comm->down_stream) cudaStreamSynchronize(static_cast<cudaStream_t>(comm->down_stream));
+  if (comm->up_stream) cudaStreamSynchronize(static_cast<cudaStream_t>(comm->up_stream));
+  auto drop = [](void** ev) {
+    if (*ev) cudaEventDestroy(static_cast<cudaEvent_t>(*ev));
+    *ev = nullptr;
+  };
+  drop(&comm->ev_entry);
+  for (int i = 0; i < pl_comm_s::kHostSlots; ++i) {
+    drop(&comm->ev_up[i]);
+    drop(&comm->ev_kernel[i]);
+    drop(&comm->downloads[i].done);
+    comm->downloads[i].live = false;
+  }
+  if (comm->up_stream) cudaStreamDestroy(static_cast<cudaStream_t>(comm->up_stream));
+  if (comm->down_stream) cudaStreamDestroy(static_cast<cudaStream_t>(comm->down_stream));
+  comm->up_stream = comm->down_stream = nullptr;
+  comm->last_download = -1;
+  comm->host_calls = 0;
+}
+
+// Argument checks shared by the two host entry points.
+pl_status_t check_host_bufs(pl_schedule_s* s, const pl_bufs_t* host, const pl_bufs_t* dev) {
+  if (!s || !host || !dev) return PL_ERR_INVALID_ARG;
+  if (s->comm->planner || !s->d_blob) return PL_ERR_UNSUPPORTED;
+  pl_status_t st = check_bufs(s, dev);
+  if (st != PL_OK) return st;
+  for (int r = 0; r < s->comm->R; ++r) {
+    if (host->in_bytes[r] < s->info.in_bytes[r] || host->out_bytes[r] < s->info.out_bytes[r]) return PL_ERR_INVALID_ARG;
+    if ((s->info.in_bytes[r] && !host->in[r]) || (s->info.out_bytes[r] && !host->out[r])) return PL_ERR_INVALID_ARG;
+    if (s->info.aux_bytes[r] && (!host->aux[r] || host->aux_bytes[r] < s->info.aux_bytes[r])) return PL_ERR_INVALID_ARG;
+  }
+  return PL_OK;
+}
+
+// host -> device copies of inputs and second operands (upload) or device -> host copies of outputs.
+bool copy_all(pl_schedule_s* s, int R, const pl_bufs_t* host, const pl_bufs_t* dev, bool upload, cudaStream_t on) {
+  bool ok = true;
+  for (int r = 0; r < R && ok; ++r) {
+    if (upload) {
+      if (s->info.in_bytes[r])
+        ok = cudaMemcpyAsync(const_cast<void*>(dev->in[r]), host->in[r], s->info.in_bytes[r], cudaMemcpyHostToDevice, on) == cudaSuccess;
+      if (ok && s->info.aux_bytes[r])
+        ok = cudaMemcpyAsync(const_cast<void*>(dev->aux[r]), host->aux[r], s->info.aux_bytes[r], cudaMemcpyHostToDevice, on) == cudaSuccess;
+    } else if (s->info.out_bytes[r]) {
+      ok = cudaMemcpyAsync(host->out[r], dev->out[r], s->info.out_bytes[r], cudaMemcpyDeviceToHost, on) == cudaSuccess;
+    }
+  }
+  if (!ok) cudaGetLastError();
+  return ok;
+}
+
+bool ranges_overlap(const std::vector<pl_comm_s::Range>& a, const std::vector<pl_comm_s::Range>& b) {
+  for (const auto& x : a)
+    for (const auto& y : b)
+      if (x.lo < y.hi && y.lo < x.hi) return true;
+  return false;
+}
+
+// Streams and events of the pipelined host entry point, created at its first use.
+bool host_pipeline_init(pl_comm_s* comm) {
+  if (comm->up_stream) return true;
+  cudaStream_t up = nullptr, down = nullptr;
+  bool ok = cudaStreamCreateWithFlags(&up, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&down, cudaStreamNonBlocking) == cudaSuccess;
+  auto make = [&](void** ev) {
+    cudaEvent_t e = nullptr;
+    ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+    *ev = e;
+  };
+  make(&comm->ev_entry);
+  for (int i = 0; i < pl_comm_s::kHostSlots; ++i) {
+    make(&comm->ev_up[i]);
+    make(&comm->ev_kernel[i]);
+    make(&comm->downloads[i].done);
+  }
+  comm->up_stream = up;
+  comm->down_stream = down;
+  if (!ok) {
+    cudaGetLastError();
+    host_pipeline_destroy(comm);
+  }
+  return ok;
+}
+
+}  // namespace
+
+extern "C" {
 
 const char* pl_status_string(pl_status_t st) {
   switch (st) {
@@ -507,8 +601,81 @@ pl_status_t pl_comm_destroy(pl_comm_t comm) {
   if (!comm->schedules.empty() || comm->n_plans != 0) return PL_ERR_INVALID_ARG;
   if (comm->d_status) cudaFree(comm->d_status);
   if (comm->status_stream) cudaStreamDestroy(static_cast<cudaStream_t>(comm->status_stream));
+  host_pipeline_destroy(comm);
   delete comm;
   return PL_OK;
+}
+
+pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out) {
+  if (!comm) return PL_ERR_INVALID_ARG;
+  if (push_ctas_out) *push_ctas_out = 0;
+  if (comm->planner) return PL_ERR_UNSUPPORTED;
+  if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
+  const int R = comm->R;
+  const size_t es = (size_t)elem_size(comm->dtype);
+  // the measured case: an all-gather of 64 MiB (R contributions of 64 MiB / R), far beyond L2
+  const size_t part = ((size_t)64 << 20) / (size_t)R / (16 * es) * (16 * es);
+  const size_t count = part / es;
+  char *d_in = nullptr, *d_out = nullptr;
+  if (cudaMalloc(&d_in, part * R) != cudaSuccess || cudaMalloc(&d_out, part * R * R) != cudaSuccess) {
+    cudaGetLastError();
+    if (d_in) cudaFree(d_in);
+    return PL_ERR_OOM;
+  }
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  cudaMemsetAsync(d_in, 0, part * R, cs);
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaEventCreate(&e0);
+  cudaEventCreate(&e1);
+  pl_bufs_t bufs;
+  std::memset(&bufs, 0, sizeof(bufs));
+  for (int r = 0; r < R; ++r) {
+    bufs.in[r] = d_in + (size_t)r * part;
+    bufs.in_bytes[r] = part;
+    bufs.out[r] = d_out + (size_t)r * part * R;
+    bufs.out_bytes[r] = part * R;
+  }
+  const int per_sm = exec_tma_max_ctas_per_sm(comm->dtype, 4, 48 * 1024);
+  const int resident = std::max(1, per_sm) * comm->sm_count;
+  int best = 0;
+  float best_ms = 0.f;
+  pl_status_t result = PL_OK;
+  const int saved = comm->tuned_push_ctas;
+  for (int g = resident / R * R; g >= resident * 3 / 4 && g >= R; g -= R) {
+    pl_sched_opts_t o;
+    std::memset(&o, 0, sizeof(o));
+    o.struct_size = sizeof(o);
+    o.n_ctas = g;
+    o.datapath = PL_DP_TMA;
+    pl_schedule_t s = nullptr;
+    if (pl_schedule_build(comm, PL_ALLGATHER, PL_ALGO_DIRECT, count, (size_t)1 << 20, &o, &s) != PL_OK) continue;
+    bool ok = true;
+    for (int i = 0; i < 2 && ok; ++i) ok = pl_execute(s, &bufs, stream) == PL_OK;
+    const int reps = 6;
+    ok = ok && cudaEventRecord(e0, cs) == cudaSuccess;
+    for (int i = 0; i < reps && ok; ++i) ok = pl_execute(s, &bufs, stream) == PL_OK;
+    ok = ok && cudaEventRecord(e1, cs) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess;
+    float ms = 0.f;
+    ok = ok && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess;
+    pl_schedule_destroy(s);
+    if (!ok) {
+      cudaGetLastError();
+      result = PL_ERR_CUDA;
+      break;
+    }
+    if (best == 0 || ms < best_ms) {
+      best = g;
+      best_ms = ms;
+    }
+  }
+  cudaStreamSynchronize(cs);
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  cudaFree(d_in);
+  cudaFree(d_out);
+  comm->tuned_push_ctas = (result == PL_OK && best > 0) ? best : saved;
+  if (push_ctas_out) *push_ctas_out = comm->tuned_push_ctas;
+  return result;
 }
 
 pl_status_t pl_comm_status(pl_comm_t comm, pl_devstatus_t* out) {
@@ -826,38 +993,118 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
 }
 
 pl_status_t pl_execute_host(pl_schedule_t s, const pl_bufs_t* host, const pl_bufs_t* dev, void* stream) {
-  if (!s || !host || !dev) return PL_ERR_INVALID_ARG;
-  if (s->comm->planner || !s->d_blob) return PL_ERR_UNSUPPORTED;
-  pl_status_t st = check_bufs(s, dev);
+  pl_status_t st = check_host_bufs(s, host, dev);
   if (st != PL_OK) return st;
   const int R = s->comm->R;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  for (int r = 0; r < R; ++r) {
-    if (host->in_bytes[r] < s->info.in_bytes[r] || host->out_bytes[r] < s->info.out_bytes[r]) return PL_ERR_INVALID_ARG;
-    if ((s->info.in_bytes[r] && !host->in[r]) || (s->info.out_bytes[r] && !host->out[r])) return PL_ERR_INVALID_ARG;
-  }
-  for (int r = 0; r < R; ++r)
-    if (s->info.in_bytes[r] &&
-        cudaMemcpyAsync(const_cast<void*>(dev->in[r]), host->in[r], s->info.in_bytes[r], cudaMemcpyHostToDevice, cs) != cudaSuccess) {
-      cudaGetLastError();
-      return PL_ERR_CUDA;
-    }
-  for (int r = 0; r < R; ++r) {
-    if (!s->info.aux_bytes[r]) continue;
-    if (!host->aux[r] || host->aux_bytes[r] < s->info.aux_bytes[r]) return PL_ERR_INVALID_ARG;
-    if (cudaMemcpyAsync(const_cast<void*>(dev->aux[r]), host->aux[r], s->info.aux_bytes[r], cudaMemcpyHostToDevice, cs) != cudaSuccess) {
-      cudaGetLastError();
-      return PL_ERR_CUDA;
-    }
-  }
+  // downloads of earlier pipelined host executes may still read or write what this call touches
+  st = pl_comm_host_fence(s->comm, stream);
+  if (st != PL_OK) return st;
+  if (!copy_all(s, R, host, dev, /*upload=*/true, cs)) return PL_ERR_CUDA;
   st = pl_execute(s, dev, stream);
   if (st != PL_OK) return st;
-  for (int r = 0; r < R; ++r)
-    if (s->info.out_bytes[r] &&
-        cudaMemcpyAsync(host->out[r], dev->out[r], s->info.out_bytes[r], cudaMemcpyDeviceToHost, cs) != cudaSuccess) {
-      cudaGetLastError();
-      return PL_ERR_CUDA;
+  if (!copy_all(s, R, host, dev, /*upload=*/false, cs)) return PL_ERR_CUDA;
+  return PL_OK;
+}
+
+pl_status_t pl_execute_host_async(pl_schedule_t s, const pl_bufs_t* host, const pl_bufs_t* dev, void* stream) {
+  pl_status_t st = check_host_bufs(s, host, dev);
+  if (st != PL_OK) return st;
+  pl_comm_s* comm = s->comm;
+  if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> host_guard(comm->host_mu);
+  if (!host_pipeline_init(comm)) return PL_ERR_CUDA;
+  const int R = comm->R;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  cudaStream_t up = static_cast<cudaStream_t>(comm->up_stream), down = static_cast<cudaStream_t>(comm->down_stream);
+  const int slot = (int)(comm->host_calls % pl_comm_s::kHostSlots);
+  bool ok = true;
+  auto wait = [&](cudaStream_t on, void* ev) { ok = ok && cudaStreamWaitEvent(on, static_cast<cudaEvent_t>(ev), 0) == cudaSuccess; };
+
+  // The slot's events are about to be recorded again: whoever still waits for the download that
+  // used it kHostSlots calls ago must have seen it first.
+  pl_comm_s::Download& mine = comm->downloads[slot];
+  if (mine.live) {
+    wait(up, mine.done);
+    wait(cs, mine.done);
+    mine.live = false;
+  }
+  // Uploads overwrite the device inputs: the schedule of the previous host execute (and, on a
+  // stream in order, everything before it) must have finished reading them.  The first call, or a
+  // change of stream, also orders them behind what the caller has put on `stream` so far.
+  if (comm->host_calls == 0 || comm->host_stream_last != stream) {
+    ok = ok && cudaEventRecord(static_cast<cudaEvent_t>(comm->ev_entry), cs) == cudaSuccess;
+    wait(up, comm->ev_entry);
+  }
+  if (comm->host_calls > 0) wait(up, comm->ev_kernel[(comm->host_calls - 1) % pl_comm_s::kHostSlots]);
+  // Hazards with downloads still in flight: an upload must not read a host range, nor overwrite a
+  // device range, that a download has yet to finish with; the schedule must not overwrite device
+  // outputs that a download still reads.
+  std::vector<pl_comm_s::Range> h_in, d_in, d_out, h_out;
+  for (int r = 0; r < R; ++r) {
+    auto add = [](std::vector<pl_comm_s::Range>& v, const void* p, size_t n) {
+      if (p && n) v.push_back({static_cast<const char*>(p), static_cast<const char*>(p) + n});
+    };
+    add(h_in, host->in[r], s->info.in_bytes[r]);
+    add(h_in, host->aux[r], s->info.aux_bytes[r]);
+    add(d_in, dev->in[r], s->info.in_bytes[r]);
+    add(d_in, dev->aux[r], s->info.aux_bytes[r]);
+    add(d_out, dev->out[r], s->info.out_bytes[r]);
+    add(h_out, host->out[r], s->info.out_bytes[r]);
+  }
+  for (pl_comm_s::Download& d : comm->downloads) {
+    if (!d.live) continue;
+    if (cudaEventQuery(static_cast<cudaEvent_t>(d.done)) == cudaSuccess) {
+      d.live = false;
+      continue;
     }
+    cudaGetLastError();  // cudaErrorNotReady is not an error here
+    if (ranges_overlap(h_in, d.host_out) || ranges_overlap(d_in, d.dev_out)) wait(up, d.done);
+    if (ranges_overlap(d_out, d.dev_out) || ranges_overlap(d_in, d.dev_out)) wait(cs, d.done);
+  }
+  if (!ok) { cudaGetLastError(); return PL_ERR_CUDA; }
+
+  if (!copy_all(s, R, host, dev, /*upload=*/true, up)) return PL_ERR_CUDA;
+  ok = cudaEventRecord(static_cast<cudaEvent_t>(comm->ev_up[slot]), up) == cudaSuccess;
+  wait(cs, comm->ev_up[slot]);
+  if (!ok) { cudaGetLastError(); return PL_ERR_CUDA; }
+  st = pl_execute(s, dev, stream);
+  if (st != PL_OK) return st;
+  ok = cudaEventRecord(static_cast<cudaEvent_t>(comm->ev_kernel[slot]), cs) == cudaSuccess;
+  wait(down, comm->ev_kernel[slot]);
+  if (!ok) { cudaGetLastError(); return PL_ERR_CUDA; }
+  ++comm->host_calls;                 // ev_kernel[slot] is what the next upload waits for
+  comm->host_stream_last = stream;
+  if (!copy_all(s, R, host, dev, /*upload=*/false, down)) return PL_ERR_CUDA;
+  if (cudaEventRecord(static_cast<cudaEvent_t>(mine.done), down) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
+  mine.host_out = std::move(h_out);
+  mine.dev_out = std::move(d_out);
+  mine.live = true;
+  comm->last_download = slot;
+  return PL_OK;
+}
+
+pl_status_t pl_comm_host_fence(pl_comm_t comm, void* stream) {
+  if (!comm) return PL_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> host_guard(comm->host_mu);
+  if (comm->last_download < 0) return PL_OK;
+  // downloads run in order on one stream: the last one's event covers them all
+  if (cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), static_cast<cudaEvent_t>(comm->downloads[comm->last_download].done), 0) != cudaSuccess) {
+    cudaGetLastError();
+    return PL_ERR_CUDA;
+  }
+  return PL_OK;
+}
+
+pl_status_t pl_comm_host_sync(pl_comm_t comm) {
+  if (!comm) return PL_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> host_guard(comm->host_mu);
+  if (comm->last_download < 0) return PL_OK;
+  if (cudaEventSynchronize(static_cast<cudaEvent_t>(comm->downloads[comm->last_download].done)) != cudaSuccess) {
+    cudaGetLastError();
+    return PL_ERR_CUDA;
+  }
+  for (pl_comm_s::Download& d : comm->downloads) d.live = false;
   return PL_OK;
 }
 

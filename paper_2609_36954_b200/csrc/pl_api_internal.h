@@ -21,7 +21,28 @@ struct pl_comm_s {
   std::mutex mu;
   std::vector<pl_schedule_s*> schedules;
   int n_plans = 0;
+  int tuned_push_ctas = 0;  // pl_comm_tune: best grid for pushed copies on the bulk-copy datapath (0 = not measured)
   std::string last_error;
+  // pl_execute_host_async: an upload and a download stream, and the downloads still in flight
+  // with the host and device ranges they touch (hazards are resolved with their events)
+  struct Range { const char* lo; const char* hi; };
+  struct Download {
+    void* done = nullptr;          // cudaEvent_t recorded behind the download's last copy
+    std::vector<Range> host_out;   // host ranges the download writes
+    std::vector<Range> dev_out;    // device ranges it reads
+    bool live = false;
+  };
+  static constexpr int kHostSlots = 8;
+  void* up_stream = nullptr;
+  void* down_stream = nullptr;
+  void* ev_up[kHostSlots] = {};      // uploads of call n complete
+  void* ev_kernel[kHostSlots] = {};  // schedule of call n complete
+  void* ev_entry = nullptr;
+  Download downloads[kHostSlots];
+  uint64_t host_calls = 0;           // async host executes so far
+  void* host_stream_last = nullptr;  // the caller's stream of the previous async host execute
+  int last_download = -1;            // slot of the most recent download
+  std::mutex host_mu;                // serialises the host-pipeline entry points
 };
 
 namespace pl {

@@ -152,6 +152,7 @@ struct BuildRequest {
   int packet_ctas_per_rank;  // > 0: layered all-reduce on the packet datapath with this many CTAs per rank
   uint32_t hook;             // PL_HOOK_* bits
   bool stage_ahead;          // PL_OPT_STAGE_AHEAD
+  int tuned_push_ctas;       // > 0: grid that pl_comm_tune measured for pushed copies on the bulk-copy datapath
   Policy pol;
 };
 

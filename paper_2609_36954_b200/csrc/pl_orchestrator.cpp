@@ -805,11 +805,16 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
   if (p.n_ctas <= 0) {
     int full = std::max(rq.R, max_resident_ctas / rq.R * rq.R);
     // Pushed copies on the bulk-copy datapath (all-gather(-v), broadcast) are a 1 read : R writes
-    // stream, which this GPU's memory system serves fastest with about 9 of 10 SMs writing
-    // (measured, 148 SMs: 128-136 CTAs 6.15-6.3 TB/s, 140-148 CTAs 5.65-5.73 TB/s): 136 of 148.
+    // stream, which the memory system serves fastest with fewer than all SMs writing.  How many
+    // depends on the individual GPU (which SMs a grid smaller than the SM count leaves idle follows
+    // the chip's own SM layout): of two B200s one ran the 8 x 64 MiB all-gather in 101 us with 136
+    // CTAs and 102 with 128, the other in 113 us with 136 and 102-104 with 128 (144: 106 and 110).
+    // pl_comm_tune measures it; untuned, 87 % of the resident CTAs (128 of 148) is the safe choice.
     if (p.datapath == PL_DP_TMA && (rq.coll == PL_ALLGATHER || rq.coll == PL_ALLGATHERV || rq.coll == PL_BROADCAST) &&
-        rq.algo == PL_ALGO_DIRECT && !rq.staged)
-      full = std::max(rq.R, (max_resident_ctas * 92 / 100) / rq.R * rq.R);
+        rq.algo == PL_ALGO_DIRECT && !rq.staged) {
+      if (rq.tuned_push_ctas > 0 && rq.tuned_push_ctas <= max_resident_ctas) full = std::max(rq.R, rq.tuned_push_ctas / rq.R * rq.R);
+      else full = std::max(rq.R, (max_resident_ctas * 87 / 100) / rq.R * rq.R);
+    }
     // bytes a rank produces in its busiest phase
     uint64_t per_rank = msg;
     if (rq.coll == PL_REDUCE_SCATTER || rq.coll == PL_REDUCE_SCATTERV) per_rank = msg / rq.R;

@@ -66,3 +66,26 @@ def test_last_use_is_accepted_and_ignored_off_the_bulk_copy_datapath():
                 assert np.array_equal(outs[r].view(np.int32), ref[r])
     finally:
         ses.close()
+
+
+def test_comm_tune_picks_a_grid_and_later_builds_use_it():
+    """pl_comm_tune measures the all-gather's grid on this GPU; the pick is a multiple of R within
+    the resident CTAs, later default builds of the pushed all-gather use it, and it computes the
+    same bytes as any other grid."""
+    R = 8
+    ses = Session(R, "bf16")
+    try:
+        g = B.pl_comm_tune(ses.comm, 0)
+        assert g % R == 0 and 96 <= g <= 148
+        n = R * (3 << 20)                      # 6 MiB per contribution: the bulk-copy datapath by default
+        x = gen.rank_inputs(R, n // R, "bf16", seed=17)
+        s = ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 20, datapath=B.PL_DP_TMA)
+        outs, info = ses.execute(s, x)
+        assert info.grid == g
+        ref = oracle.allgather(x)
+        for r in range(R):
+            assert np.array_equal(outs[r].view(np.uint16), ref[r])
+        s2 = ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 20, datapath=B.PL_DP_TMA, n_ctas=104)
+        assert B.pl_schedule_info(s2).grid == 104                 # an explicit grid still wins
+    finally:
+        ses.close()
