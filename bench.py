@@ -35,12 +35,12 @@ MIB = 1 << 20
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one reduce-scatter launch of this workload
-# (one ncu capture of that launch)
-NCU_RS_TRAFFIC_BYTES = 594654208.0
+# (one ncu capture of that launch, caches flushed before it: 537.7 MB read, 18.1 MB written; three
+# quarters of the 64 MiB of results are still in L2 when the kernel ends)
+NCU_RS_TRAFFIC_BYTES = 555785728.0
 # the same sum for a reduce-scatter launch inside the step (one pass, caches left as the
-# all-gather before it left them, both schedules with PL_OPT_INPUTS_LAST_USE): 20 MB more, the
-# write-back of dirty lines it inherits
-NCU_RS_TRAFFIC_IN_SITU_BYTES = 615150000.0
+# all-gather before it left them): 537.1 MB read, 76.9 MB written
+NCU_RS_TRAFFIC_IN_SITU_BYTES = 614000000.0
 
 
 def measured_peak():
@@ -142,14 +142,19 @@ def run_purlin(args):
     x = c2_inputs(R, n, seed=0, unique=(4 * MIB if args.fast_inputs else None))
     comm = B.pl_comm_create(R, B.PL_BF16)
     # set-up: which grid this GPU's memory system serves the all-gather's 1 read : 8 writes stream best with
-    tuned_grid = B.pl_comm_tune(comm, stream)
+    tuned_grid = 0 if (args.no_tune or args.ag_grid) else B.pl_comm_tune(comm, stream)
     # Both launches read their inputs for the last time (the reduce-scatter consumes the
     # contributions, the all-gather the reduced partition): PL_OPT_INPUTS_LAST_USE says so.
     step_flags = 0 if args.plain_options else B.PL_OPT_INPUTS_LAST_USE
     opts = B.make_opts(n_ctas=args.n_ctas, threads=args.threads, slice_bytes=args.slice_bytes,
                        datapath=args.datapath, stages=args.stages, stage_bytes=args.stage_bytes, flags=step_flags)
     rs = B.pl_schedule_build(comm, B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, chunk, opts)
-    ag = B.pl_schedule_build(comm, B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, chunk, opts)
+    if args.ag_grid:    # profiling runs: the all-gather's grid given instead of measured (no tuning launches)
+        opts_ag = B.make_opts(n_ctas=args.ag_grid, threads=args.threads, slice_bytes=args.slice_bytes, datapath=args.datapath,
+                              stages=args.stages, stage_bytes=args.stage_bytes, flags=step_flags)
+    else:
+        opts_ag = opts
+    ag = B.pl_schedule_build(comm, B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, chunk, opts_ag)
     irs, iag = B.pl_schedule_info(rs), B.pl_schedule_info(ag)
 
     pinned_in = [torch.from_numpy(a.view(np.int16)).pin_memory() for a in x]
@@ -648,6 +653,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-latency", action="store_true")
     ap.add_argument("--no-detail", action="store_true", help="skip the other configurations (C1, C3, C4, C5, stream ceilings)")
+    ap.add_argument("--ag-grid", type=int, default=0, help="grid of the all-gather schedule (skips pl_comm_tune); for profiling runs")
+    ap.add_argument("--no-tune", action="store_true", help="skip pl_comm_tune (the all-gather then runs with the untuned default grid)")
     ap.add_argument("--plain-options", action="store_true", help="build the two schedules of the step without PL_OPT_INPUTS_LAST_USE")
     ap.add_argument("--min-timed-ms", type=float, default=500.0, help="repeat the K-step block until the timed region lasts this long")
     ap.add_argument("--fast-inputs", action="store_true", help="tile 4 Mi generated elements instead of generating all")
