@@ -45,6 +45,7 @@ constexpr int kProducers = 2;  // producer warps; the copier is warp kProducers,
 constexpr int kMaxStages = 8;
 constexpr uint32_t kEnd = 0xFFFFFFFFu;
 constexpr uint32_t kLastOfOp = 0x100u;  // stage flag (above the DevOp flag bits)
+constexpr uint32_t kAuxInSlot = 0x200u;  // stage flag: the second operand's tile sits in the slot behind the sources
 constexpr int kCtrlBytes = 1024;        // barriers + stage descriptors ahead of the slots
 
 struct StageDesc {
@@ -151,7 +152,16 @@ __device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDe
     if (final_op) {
       // processing phase of a hooked schedule: scale, second operand, output type; one store
       // per destination (the results may differ per rank, so nothing leaves through the slot)
-      if constexpr (HOOK && (DT == PL_BF16 || DT == PL_F32)) store_final_unit<DT>(P, acc, d.dst_slot, d.dst_off, bcast, u);
+      if constexpr (HOOK && (DT == PL_BF16 || DT == PL_F32)) {
+        if (d.flags & kAuxInSlot) {
+          // one destination: the producer brought the second operand's tile along with the sources
+          const uint4 rq = lds16(slot + (size_t)(ns + __popc(pmask)) * tile + (size_t)u * 16u);
+          const bool f32 = (DT == PL_BF16) && (P.hook & PL_HOOK_F32_OUT);
+          store_final_q<DT>(acc, P.out_scale, P.hook, static_cast<char*>(P.base[d.dst_slot]) + d.dst_off + (size_t)u * (f32 ? 32u : 16u), rq);
+        } else {
+          store_final_unit<DT>(P, acc, d.dst_slot, d.dst_off, bcast, u);
+        }
+      }
     } else if (dpart) {
       if constexpr (DT == PL_BF16) {
         st16(d.dst + (size_t)u * 32u, make_uint4(__float_as_uint(acc.v[0]), __float_as_uint(acc.v[1]),
@@ -416,7 +426,12 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
       // ---- cut the op into stages
       const char* my_src = (lane < (int)n_src) ? (DBUF ? resolve(P, r_src, scratch_shift) : resolve(P, r_src)) : nullptr;
       const bool my_part = (pmask >> lane) & 1u;
-      const uint32_t unit_b = (kind == PL_OP_COPY) ? 16u : 16u * (n_src + __popc(pmask));  // slot bytes per unit
+      // Final op of a schedule with a second operand and one destination: that operand's tile
+      // rides in the slot behind the sources (one more bulk load per stage), so that no consumer
+      // waits for a global load with the slot in its hands.
+      bool aux_tile = false;
+      if constexpr (HOOK) aux_tile = kind != PL_OP_COPY && (oflags & kFinal) && !(oflags & kDstBcast) && (P.hook & PL_HOOK_RESIDUAL);
+      const uint32_t unit_b = (kind == PL_OP_COPY) ? 16u : 16u * (n_src + __popc(pmask) + (aux_tile ? 1u : 0u));  // slot bytes per unit
       uint32_t ucap = slot_bytes / unit_b;
       if constexpr (CW == kWarpsPipelined) {
         // plain reduce op: a stage holds what the consumer threads can keep in registers
@@ -430,6 +445,12 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
       const uint32_t dst_w = (kind == PL_OP_COPY) ? 16u : ((oflags & kDstF32) ? 32u : 16u);
       char* dst = DBUF ? resolve(P, dstp, scratch_shift) : resolve(P, dstp);
       const uint64_t dst_off = dstp & 0xFFFFFFFFFFFFull;
+      const char* aux_src = nullptr;
+      if (aux_tile) {
+        const bool f32 = (DT == PL_BF16) && (P.hook & PL_HOOK_F32_OUT);  // the output is twice as wide as the operand
+        aux_src = static_cast<const char*>(P.base[kSlotAux + ((dstp >> 48) - kSlotOut)]) + (f32 ? dst_off >> 1 : dst_off);
+      }
+      const uint32_t aux_tile_off = ucap * 16u * (n_src + __popc(pmask));
       for (uint64_t u0 = 0; u0 < n_units; u0 += ucap) {
         if (n % kProducers != (uint32_t)warp) {  // the other producer's stage
           ++n;
@@ -448,7 +469,7 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
           d.units = units;
           d.ucap = ucap;
           d.pmask = pmask;
-          d.flags = oflags | ((u0 + ucap >= n_units) ? kLastOfOp : 0u);
+          d.flags = oflags | ((u0 + ucap >= n_units) ? kLastOfOp : 0u) | (aux_tile ? kAuxInSlot : 0u);
           // signals go to this launch's flag set
           d.signal = (DBUF && signal != kNoFlag && flag_base != P.flags) ? signal + P.n_flags : signal;
           d.signal2 = (DBUF && signal2 != kNoFlag && flag_base != P.flags) ? signal2 + P.n_flags : signal2;
@@ -465,6 +486,8 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
           else if ((P.hints & 1u) && (r_src >> 48) < (uint64_t)kSlotOut) ptx::bulk_g2s_hint(sdst, my_src + u0 * my_w, units * my_w, &c->full[s], ptx::policy_evict_first());
           else ptx::bulk_g2s(sdst, my_src + u0 * my_w, units * my_w, &c->full[s]);
         }
+        if (aux_tile && lane == (int)n_src)
+          ptx::bulk_g2s(slots + (size_t)s * slot_bytes + aux_tile_off, aux_src + u0 * 16u, units * 16u, &c->full[s]);
         ++n;
       }
     }

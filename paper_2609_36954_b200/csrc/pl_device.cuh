@@ -166,14 +166,14 @@ struct Acc<PL_I32> {
 // value = scale * sum [+ residual], then one conversion to the element type, or none (fp32 out).
 // `dst` points at this unit in the destination (16 bytes per unit; 32 for fp32 output of a bf16
 // schedule), `res` at the same unit of the second operand (element-typed) or is unused.
+// `q` is the unit of the second operand, already loaded (ignored without PL_HOOK_RESIDUAL).
 template <int DT>
-__device__ __forceinline__ void store_final(const Acc<DT>& acc, float scale, uint32_t hook, char* dst, const char* res) {
+__device__ __forceinline__ void store_final_q(const Acc<DT>& acc, float scale, uint32_t hook, char* dst, const uint4& q) {
   if constexpr (DT == PL_BF16) {
     float v[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = __fmul_rn(acc.v[i], scale);
     if (hook & PL_HOOK_RESIDUAL) {
-      const uint4 q = ld16(res);
       const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -199,7 +199,6 @@ __device__ __forceinline__ void store_final(const Acc<DT>& acc, float scale, uin
 #pragma unroll
     for (int i = 0; i < 4; ++i) v[i] = __fmul_rn(__fadd_rn(acc.v[i], acc.c[i]), scale);
     if (hook & PL_HOOK_RESIDUAL) {
-      const uint4 q = ld16(res);
       v[0] = __fadd_rn(v[0], __uint_as_float(q.x));
       v[1] = __fadd_rn(v[1], __uint_as_float(q.y));
       v[2] = __fadd_rn(v[2], __uint_as_float(q.z));
@@ -207,6 +206,13 @@ __device__ __forceinline__ void store_final(const Acc<DT>& acc, float scale, uin
     }
     st16(dst, make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])));
   }
+}
+
+template <int DT>
+__device__ __forceinline__ void store_final(const Acc<DT>& acc, float scale, uint32_t hook, char* dst, const char* res) {
+  uint4 q = make_uint4(0, 0, 0, 0);
+  if (hook & PL_HOOK_RESIDUAL) q = ld16(res);
+  store_final_q<DT>(acc, scale, hook, dst, q);
 }
 
 // A final op of a hooked schedule stores unit `unit` of its result to one destination or to all
