@@ -46,6 +46,10 @@ constexpr int kMaxStages = 8;
 constexpr uint32_t kEnd = 0xFFFFFFFFu;
 constexpr uint32_t kLastOfOp = 0x100u;  // stage flag (above the DevOp flag bits)
 constexpr uint32_t kAuxInSlot = 0x200u;  // stage flag: the second operand's tile sits in the slot behind the sources
+// Stage flag of a final op with R destinations (fused all-reduce with a processing phase): the
+// consumers leave the results in the slot at res_off (+ k * res_stride for rank k when the
+// results differ per rank) and the copier ships them with bulk stores.
+constexpr uint32_t kResInSlot = 0x400u;
 constexpr int kCtrlBytes = 1024;        // barriers + stage descriptors ahead of the slots
 
 struct StageDesc {
@@ -62,6 +66,13 @@ struct StageDesc {
   uint32_t dst_slot;  // pointer-table slot of the destination (hooked schedules: finds the second operand)
 };
 static_assert(sizeof(StageDesc) == 56, "StageDesc layout");
+// kResInSlot stages: the result region starts right behind the n_src source tiles; with a second
+// operand (PL_HOOK_RESIDUAL) it is one tile per rank (rank k's result over rank k's operand
+// tile), otherwise one region of 32 bytes per unit.
+__device__ __forceinline__ uint32_t res_off(const StageDesc& d) { return d.ucap * 16u * d.n_src; }
+__device__ __forceinline__ uint32_t res_stride(const ExecParams& P, const StageDesc& d) {
+  return (P.hook & PL_HOOK_RESIDUAL) ? d.ucap * 16u : 0u;
+}
 
 struct Ctrl {
   uint64_t full[kMaxStages];
@@ -153,7 +164,28 @@ __device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDe
       // processing phase of a hooked schedule: scale, second operand, output type; one store
       // per destination (the results may differ per rank, so nothing leaves through the slot)
       if constexpr (HOOK && (DT == PL_BF16 || DT == PL_F32)) {
-        if (d.flags & kAuxInSlot) {
+        if (d.flags & kResInSlot) {
+          // R destinations: results go into the slot, the copier stores them.  With a second
+          // operand (one tile per rank, brought by the producer) rank k's result replaces unit u
+          // of rank k's operand tile, which only this thread reads; otherwise one result of 32
+          // bytes per unit (fp32 output) goes to a region of its own behind the sources.
+          unsigned char* res = const_cast<unsigned char*>(slot) + res_off(d);
+          const uint32_t stride = res_stride(P, d);
+          if (stride) {
+            for (int k = 0; k < P.n_ranks; ++k) {
+              unsigned char* at = res + (size_t)k * stride + (size_t)u * 16u;
+              uint4 lo, hi;
+              final_value<DT>(acc, P.out_scale, P.hook, lds16(at), lo, hi);
+              asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(ptx::smem_u32(at)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
+            }
+          } else {
+            uint4 lo, hi = make_uint4(0, 0, 0, 0);
+            final_value<DT>(acc, P.out_scale, P.hook, make_uint4(0, 0, 0, 0), lo, hi);
+            unsigned char* at = res + (size_t)u * 32u;
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(ptx::smem_u32(at)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(ptx::smem_u32(at + 16)), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+          }
+        } else if (d.flags & kAuxInSlot) {
           // one destination: the producer brought the second operand's tile along with the sources
           const uint4 rq = lds16(slot + (size_t)(ns + __popc(pmask)) * tile + (size_t)u * 16u);
           const bool f32 = (DT == PL_BF16) && (P.hook & PL_HOOK_F32_OUT);
@@ -191,7 +223,7 @@ __device__ __forceinline__ void consume_stage(const ExecParams& P, const StageDe
       }
     }
   }
-  if (bcast && pmask == 0 && !final_op) ptx::fence_proxy_async_smem();  // generic writes above -> the copier's bulk stores
+  if ((bcast && pmask == 0 && !final_op) || (HOOK && (d.flags & kResInSlot))) ptx::fence_proxy_async_smem();  // generic writes above -> the copier's bulk stores
 }
 
 // ---- software-pipelined path for plain reduce stages ---------------------------------------
@@ -300,8 +332,11 @@ __device__ __forceinline__ void plain_finish(const ExecParams& P, const PlainSta
 }
 
 // A REDUCE stage whose result leaves through shared memory (see consume_stage).
+template <bool HOOK>
 __device__ __forceinline__ bool leaves_via_smem(uint32_t kind, uint32_t flags, uint32_t pmask) {
-  return kind != PL_OP_COPY && (flags & kDstBcast) && !(flags & (kDstF32 | kFinal)) && pmask == 0;
+  if (kind == PL_OP_COPY) return false;
+  if (HOOK && (flags & kResInSlot)) return true;
+  return (flags & kDstBcast) && !(flags & (kDstF32 | kFinal)) && pmask == 0;
 }
 
 // HOOK: the variant for schedules with a processing phase beyond the scale (general consumers only).
@@ -431,7 +466,22 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
       // waits for a global load with the slot in its hands.
       bool aux_tile = false;
       if constexpr (HOOK) aux_tile = kind != PL_OP_COPY && (oflags & kFinal) && !(oflags & kDstBcast) && (P.hook & PL_HOOK_RESIDUAL);
-      const uint32_t unit_b = (kind == PL_OP_COPY) ? 16u : 16u * (n_src + __popc(pmask) + (aux_tile ? 1u : 0u));  // slot bytes per unit
+      // Final op with R destinations: results leave through the slot (kResInSlot) when the slot
+      // can hold them: a second operand per rank and element-typed output (R operand tiles,
+      // overwritten in place by the R results), or fp32 output without a second operand (one
+      // result region of 32 bytes per unit).  Both at once would leave too few units per stage:
+      // those schedules keep the consumers' per-destination global stores.
+      uint32_t res_mode = 0;  // 1: per-rank results over the operand tiles, 2: one wide result region
+      if constexpr (HOOK) {
+        if (kind != PL_OP_COPY && (oflags & kFinal) && (oflags & kDstBcast) && pmask == 0) {
+          const bool residual = P.hook & PL_HOOK_RESIDUAL, wide = (DT == PL_BF16) && (P.hook & PL_HOOK_F32_OUT);
+          if (residual && !wide && n_src + (uint32_t)P.n_ranks <= 32u) res_mode = 1;
+          else if (!residual && wide) res_mode = 2;
+        }
+      }
+      const uint32_t extra_b = aux_tile ? 16u : res_mode == 1 ? 16u * (uint32_t)P.n_ranks : res_mode == 2 ? 32u : 0u;
+      const uint32_t unit_b = (kind == PL_OP_COPY) ? 16u : 16u * (n_src + __popc(pmask)) + extra_b;  // slot bytes per unit
+      const uint32_t load_b = unit_b - (res_mode == 2 ? 32u : 0u);  // of which the bulk loads fill (a result region is not loaded)
       uint32_t ucap = slot_bytes / unit_b;
       if constexpr (CW == kWarpsPipelined) {
         // plain reduce op: a stage holds what the consumer threads can keep in registers
@@ -450,7 +500,7 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
         const bool f32 = (DT == PL_BF16) && (P.hook & PL_HOOK_F32_OUT);  // the output is twice as wide as the operand
         aux_src = static_cast<const char*>(P.base[kSlotAux + ((dstp >> 48) - kSlotOut)]) + (f32 ? dst_off >> 1 : dst_off);
       }
-      const uint32_t aux_tile_off = ucap * 16u * (n_src + __popc(pmask));
+      const uint32_t aux_tile_off = HOOK ? ucap * 16u * (n_src + __popc(pmask)) : 0u;
       for (uint64_t u0 = 0; u0 < n_units; u0 += ucap) {
         if (n % kProducers != (uint32_t)warp) {  // the other producer's stage
           ++n;
@@ -469,7 +519,7 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
           d.units = units;
           d.ucap = ucap;
           d.pmask = pmask;
-          d.flags = oflags | ((u0 + ucap >= n_units) ? kLastOfOp : 0u) | (aux_tile ? kAuxInSlot : 0u);
+          d.flags = oflags | ((u0 + ucap >= n_units) ? kLastOfOp : 0u) | (aux_tile ? kAuxInSlot : 0u) | (res_mode ? kResInSlot : 0u);
           // signals go to this launch's flag set
           d.signal = (DBUF && signal != kNoFlag && flag_base != P.flags) ? signal + P.n_flags : signal;
           d.signal2 = (DBUF && signal2 != kNoFlag && flag_base != P.flags) ? signal2 + P.n_flags : signal2;
@@ -477,7 +527,7 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
           d.dst_off = dst_off + u0 * dst_w;
           d.topo = topo;
           d.dst_slot = (uint32_t)(dstp >> 48);
-          ptx::mbar_expect_tx(&c->full[s], units * unit_b);
+          ptx::mbar_expect_tx(&c->full[s], units * load_b);
         }
         __syncwarp();
         if (lane < (int)n_src) {
@@ -488,6 +538,12 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
         }
         if (aux_tile && lane == (int)n_src)
           ptx::bulk_g2s(slots + (size_t)s * slot_bytes + aux_tile_off, aux_src + u0 * 16u, units * 16u, &c->full[s]);
+        if (res_mode == 1 && lane >= (int)n_src && lane < (int)n_src + P.n_ranks) {
+          // rank k's second operand for this stage (laid out like the element-typed output)
+          const int k = lane - (int)n_src;
+          ptx::bulk_g2s(slots + (size_t)s * slot_bytes + aux_tile_off + (size_t)k * ucap * 16u,
+                        static_cast<const char*>(P.base[kSlotAux + k]) + dst_off + u0 * 16u, units * 16u, &c->full[s]);
+        }
         ++n;
       }
     }
@@ -527,7 +583,7 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
       const StageDesc& d = c->desc[s];
       const uint32_t kind = d.kind;
       if (kind == kEnd) break;
-      const bool via_smem = leaves_via_smem(kind, d.flags, d.pmask);
+      const bool via_smem = leaves_via_smem<HOOK>(kind, d.flags, d.pmask);
       const bool to_all = via_smem || (kind == PL_OP_COPY && (d.flags & kDstBcast));  // one tile, R destinations
       const bool uses_done = via_smem || (kind != PL_OP_COPY && (d.flags & kLastOfOp) && d.signal != kNoFlag);
       if (via_smem) {
@@ -540,10 +596,14 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
       if (lane == 0) {
         if (kind == PL_OP_COPY || via_smem) {
           if (to_all) {
+            const bool res = HOOK && (d.flags & kResInSlot);
+            const uint32_t stride = res ? res_stride(P, d) : 0u;
+            const uint32_t bytes = d.units * ((res && !stride) ? 32u : 16u);
             for (int k = 0; k < P.n_ranks; ++k) {
               void* dk = static_cast<char*>(P.base[kSlotOut + k]) + d.dst_off;
-              if (P.hints & 2u) ptx::bulk_s2g_hint(dk, slots + (size_t)s * slot_bytes, d.units * 16u, ptx::policy_evict_first());
-              else ptx::bulk_s2g(dk, slots + (size_t)s * slot_bytes, d.units * 16u);
+              const unsigned char* from = slots + (size_t)s * slot_bytes + (res ? res_off(d) + (size_t)k * stride : 0u);
+              if (P.hints & 2u) ptx::bulk_s2g_hint(dk, from, bytes, ptx::policy_evict_first());
+              else ptx::bulk_s2g(dk, from, bytes);
             }
           } else if (P.hints & 2u) {
             ptx::bulk_s2g_hint(d.dst, slots + (size_t)s * slot_bytes, d.units * 16u, ptx::policy_evict_first());
@@ -631,7 +691,7 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
         const bool last = d.flags & kLastOfOp;
         const uint32_t signal = d.signal, signal2 = d.signal2, topo = d.topo;
         __syncwarp();
-        if (leaves_via_smem(kind, d.flags, d.pmask)) {
+        if (leaves_via_smem<HOOK>(kind, d.flags, d.pmask)) {
           // the copier ships the tile (and signals, if this is the op's last stage)
           if (lane == 0) ptx::mbar_arrive(&c->done[s]);
           done_parity ^= 1u << s;

@@ -167,8 +167,10 @@ struct Acc<PL_I32> {
 // `dst` points at this unit in the destination (16 bytes per unit; 32 for fp32 output of a bf16
 // schedule), `res` at the same unit of the second operand (element-typed) or is unused.
 // `q` is the unit of the second operand, already loaded (ignored without PL_HOOK_RESIDUAL).
+// final_value computes the unit's result: 16 bytes in `lo`, or 32 bytes in `lo`, `hi` for the
+// fp32 output of a bf16 schedule (returns true then).
 template <int DT>
-__device__ __forceinline__ void store_final_q(const Acc<DT>& acc, float scale, uint32_t hook, char* dst, const uint4& q) {
+__device__ __forceinline__ bool final_value(const Acc<DT>& acc, float scale, uint32_t hook, const uint4& q, uint4& lo, uint4& hi) {
   if constexpr (DT == PL_BF16) {
     float v[8];
 #pragma unroll
@@ -182,18 +184,17 @@ __device__ __forceinline__ void store_final_q(const Acc<DT>& acc, float scale, u
       }
     }
     if (hook & PL_HOOK_F32_OUT) {
-      st16(dst, make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])));
-      st16(dst + 16, make_uint4(__float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7])));
-    } else {
-      uint4 q;
-      __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
-      __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
-      q.x = *reinterpret_cast<uint32_t*>(&a);
-      q.y = *reinterpret_cast<uint32_t*>(&b);
-      q.z = *reinterpret_cast<uint32_t*>(&c);
-      q.w = *reinterpret_cast<uint32_t*>(&d);
-      st16(dst, q);
+      lo = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+      hi = make_uint4(__float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7]));
+      return true;
     }
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+    __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
+    lo.x = *reinterpret_cast<uint32_t*>(&a);
+    lo.y = *reinterpret_cast<uint32_t*>(&b);
+    lo.z = *reinterpret_cast<uint32_t*>(&c);
+    lo.w = *reinterpret_cast<uint32_t*>(&d);
+    return false;
   } else if constexpr (DT == PL_F32) {
     float v[4];
 #pragma unroll
@@ -204,8 +205,19 @@ __device__ __forceinline__ void store_final_q(const Acc<DT>& acc, float scale, u
       v[2] = __fadd_rn(v[2], __uint_as_float(q.z));
       v[3] = __fadd_rn(v[3], __uint_as_float(q.w));
     }
-    st16(dst, make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])));
+    lo = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+    return false;
+  } else {
+    return false;
   }
+}
+
+template <int DT>
+__device__ __forceinline__ void store_final_q(const Acc<DT>& acc, float scale, uint32_t hook, char* dst, const uint4& q) {
+  uint4 lo, hi;
+  const bool wide = final_value<DT>(acc, scale, hook, q, lo, hi);
+  st16(dst, lo);
+  if (wide) st16(dst + 16, hi);
 }
 
 template <int DT>
