@@ -39,9 +39,9 @@ def main(path):
           f"({f(d['reduce_scatter']['frac_measured'], 3)} of measured, {f(d['reduce_scatter']['frac_8TBps'], 3)} of 8 TB/s), "
           f"all-gather launch {f(d['all_gather']['us'], 1)} us ({f(d['all_gather']['frac_measured'], 3)} of measured on compulsory bytes); "
           f"end to end {f(line['e2e']['value'], 2)} GB/s; clocks {line['clocks']['sm_mhz']} MHz {line['clocks']['reasons']}.")
-    if "step_overlapped_launches" in d:
-        o = d["step_overlapped_launches"]
-        print(f"Step with overlapped launches: {f(o['ms_per_step'] * 1e3, 1)} us ({f(o['vs_headline_step'], 3)} of the headline step).")
+    if "step_both_launches_overlapped" in d:
+        o = d["step_both_launches_overlapped"]
+        print(f"Step with both launches overlapped: {f(o['ms_per_step'] * 1e3, 1)} us ({f(o['vs_headline_step'], 3)} of the headline step).")
     if "step_without_last_use_hint" in d:
         o = d["step_without_last_use_hint"]
         print(f"Step without PL_OPT_INPUTS_LAST_USE: {f(o['ms_per_step'] * 1e3, 1)} us ({f(o['vs_headline_step'], 3)} of the headline step).")
