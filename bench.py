@@ -431,7 +431,7 @@ def measure_all_configs(peak):
     for label, size, graph, iters in (("64KiB", 64 << 10, True, 30), ("16MiB", 16 << 20, False, 20), ("256MiB", 256 << 20, False, 8)):
         out["C3"][label] = {}
         for algo in ("ring", "tree", "oneshot", "direct", "fused"):
-            chunk = max(16, min(MIB, size if algo in ("oneshot", "tree") else size // 8))
+            chunk = max(16, min(MIB, size if (algo == "oneshot" or (algo == "tree" and size <= (128 << 10))) else size // 8))
             rec = b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=iters, graph=graph)
             out["C3"][label][algo] = entry(rec, l2 if size < (32 << 20) else None)
     # all-to-all and the stand-alone C2 collectives (no neighbour launch dirtying L2)
@@ -441,6 +441,12 @@ def measure_all_configs(peak):
         "reduce_scatter_ring": entry(b.collective("C2-RS", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "ring", 32 * MIB, 256 << 10)),
         "all_gather_ring": entry(b.collective("C2-AG", 8, B.PL_BF16, B.PL_ALLGATHER, "ring", 4 * MIB, 256 << 10)),
         "all_to_all": entry(b.collective("A2A", 8, B.PL_BF16, B.PL_ALLTOALL, "direct", 32 * MIB, MIB)),
+    }
+    # the same two collectives at 256 MiB per rank: what the datapath sustains once launch, ramp and
+    # tail (about 9 us per launch) stop mattering
+    out["C2_alone_256MiB"] = {
+        "reduce_scatter": entry(b.collective("C2-RS", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "direct", 128 * MIB, MIB, iters=10)),
+        "all_gather": entry(b.collective("C2-AG", 8, B.PL_BF16, B.PL_ALLGATHER, "direct", 16 * MIB, MIB, iters=10)),
     }
     # staged schedules (ordinary application buffers), back-to-back executes without events in between:
     # one staging buffer, overlapped launches, two buffers alternated by launch parity (stage ahead)

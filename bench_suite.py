@@ -352,9 +352,10 @@ def main(args=None):
             for algo in ("ring", "tree", "oneshot", "direct", "fused"):
                 if algo == "oneshot" and size > 64 * MIB:
                     continue
-                # chunks of a partition (size / 8) for the partitioned algorithms, of the whole
-                # message for one-shot and tree
-                chunk = max(16, min(MIB, size if algo in ("oneshot", "tree") else size // 8))
+                # chunks of a partition (size / 8) for the partitioned algorithms and for trees above
+                # 128 KiB (a tree pipelines its levels over the chunks: 1 MiB in one chunk takes
+                # 51 us, in eight 23 us), of the whole message for one-shot and small trees
+                chunk = max(16, min(MIB, size if (algo == "oneshot" or (algo == "tree" and size <= (128 << 10))) else size // 8))
                 b.collective("C3", 8, B.PL_BF16, B.PL_ALLREDUCE, algo, size // 2, chunk, iters=30 if lg < 24 else 10,
                              graph=lg <= 24)
                 # latency-bound sizes again with overlapped launches (CTAs of call i+1 set up while call i drains)

@@ -59,6 +59,8 @@ def main(path):
         print(collective_rows(f"C1 ring all-reduce R=4 1 MiB {k}", e))
     for k, e in c["C2_alone"].items():
         print(collective_rows(f"C2 {k} alone, 64 MiB", e))
+    for k, e in c.get("C2_alone_256MiB", {}).items():
+        print(collective_rows(f"C2 {k} alone, 256 MiB", e))
     for size, algos in c["C3"].items():
         for k, e in algos.items():
             print(collective_rows(f"C3 all-reduce {size} {k}", e))
