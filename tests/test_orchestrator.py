@@ -862,3 +862,30 @@ def test_algo_auto_picks_by_collective_and_size():
         assert all(o.dst_bcast for o in B.pl_schedule_dump(s))  # direct-fused layers
     finally:
         pl.close()
+
+
+def test_pushed_all_gather_default_grid_and_option_flags_on_the_planner():
+    """Policy, no GPU: the pushed all-gather of the bulk-copy datapath asks for fewer CTAs than a
+    reduce-scatter of the same size (a 1 read : R writes stream wants fewer writers), a multiple
+    of R either way; the L2 options change nothing in what is lowered; tuning needs a GPU."""
+    R = 8
+    pl = Planner(R, "bf16")
+    try:
+        n = R * (4 << 20)
+        ag = pl.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 20, datapath=B.PL_DP_TMA)
+        rs = pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, 1 << 20, datapath=B.PL_DP_TMA)
+        ia, ir = B.pl_schedule_info(ag), B.pl_schedule_info(rs)
+        assert ia.grid % R == 0 and ir.grid % R == 0
+        assert ia.grid < ir.grid and 0.80 * ir.grid <= ia.grid <= 0.90 * ir.grid
+        plain = B.pl_schedule_dump(rs)
+        for flags in (B.PL_OPT_INPUTS_LAST_USE, B.PL_OPT_NO_L2_HINTS, B.PL_OPT_INPUTS_LAST_USE | B.PL_OPT_NO_L2_HINTS):
+            s = pl.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, 1 << 20, datapath=B.PL_DP_TMA, flags=flags)
+            i2 = B.pl_schedule_info(s)
+            assert (i2.grid, i2.n_ops, i2.bytes_read, i2.bytes_written, i2.hbm_bytes) == (ir.grid, ir.n_ops, ir.bytes_read, ir.bytes_written, ir.hbm_bytes)
+            ops = B.pl_schedule_dump(s)
+            assert [(o.kind, o.queue, o.count) for o in ops] == [(o.kind, o.queue, o.count) for o in plain]
+        with pytest.raises(B.PurlinError) as e:
+            B.pl_comm_tune(pl.comm, 0)
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+    finally:
+        pl.close()
