@@ -148,3 +148,30 @@ def test_hooked_execute_needs_the_second_operand():
         assert e.value.status == B.PL_ERR_ALIGNMENT
     finally:
         ses.close()
+
+
+@pytest.mark.parametrize("R", [3, 16])
+@pytest.mark.parametrize("hook", [B.PL_HOOK_RESIDUAL, B.PL_HOOK_F32_OUT])
+def test_hooked_fused_allreduce_on_the_bulk_copy_executor_at_other_rank_counts(R, hook):
+    """The results of a hooked fused all-reduce leave through the ring slot (one operand / result
+    tile per rank, or one wide result region): 16 ranks fill all 32 producer lanes, 3 ranks leave
+    odd tile counts; sizes ragged against the stage capacity."""
+    part = 21 * 1024 + 32
+    n = R * part // 2
+    scale = 0.5
+    x = gen.rank_inputs(R, n, "bf16", seed=80 + R)
+    aux = gen.rank_inputs(R, n, "bf16", seed=81 + R) if hook & B.PL_HOOK_RESIDUAL else None
+    ref = oracle.allreduce_processed(x, "bf16", scale, aux)
+    ses = Session(R, "bf16")
+    try:
+        s = ses.build(B.PL_ALLREDUCE, B.PL_ALGO_DIRECT_FUSED, n, 8192, datapath=B.PL_DP_TMA, hook=hook, out_scale=scale)
+        outs, info = run_hooked(ses, s, x, aux)
+        assert info.datapath == B.PL_DP_TMA
+        for r in range(R):
+            if hook & B.PL_HOOK_F32_OUT:
+                got = outs[r].view(np.float32).astype(np.float64)
+                assert np.all(np.abs(got - ref[r]) <= f32_out_tolerance(x, None, scale, R))
+            else:
+                check_float(gen.bf16_bits_to_f64(outs[r].view(np.uint16)), ref[r], "bf16")
+    finally:
+        ses.close()
