@@ -281,6 +281,11 @@ def main(args=None):
             for chunk in (256 * 1024, MIB):
                 b.collective("C2-RS", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, algo, n, chunk)
                 b.collective("C2-AG", 8, B.PL_BF16, B.PL_ALLGATHER, algo, n // 8, chunk)
+    if "c2big" in which:
+        # the same two collectives at 256 MiB per rank: the sustained rate, launch edges amortised
+        n = 128 * MIB
+        b.collective("C2-RS-256MiB", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "direct", n, MIB, iters=10)
+        b.collective("C2-AG-256MiB", 8, B.PL_BF16, B.PL_ALLGATHER, "direct", n // 8, MIB, iters=10)
     if "staged" in which:
         # the paper's default setting: ordinary application buffers, so the work of staging is
         # included (Sec. 5, "Collective Microbenchmarks"); full and restricted staging capacity
