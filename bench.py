@@ -142,7 +142,7 @@ def run_purlin(args):
     x = c2_inputs(R, n, seed=0, unique=(4 * MIB if args.fast_inputs else None))
     comm = B.pl_comm_create(R, B.PL_BF16)
     # set-up: which grid this GPU's memory system serves the all-gather's 1 read : 8 writes stream best with
-    tuned_grid = 0 if (args.no_tune or args.ag_grid) else B.pl_comm_tune(comm, stream)
+    tuned_grid = 0 if (args.no_tune or args.ag_grid) else B.pl_comm_tune(comm, stream)   # later builds on comm use what it measured
     # Both launches read their inputs for the last time (the reduce-scatter consumes the
     # contributions, the all-gather the reduced partition): PL_OPT_INPUTS_LAST_USE says so.
     step_flags = 0 if args.plain_options else B.PL_OPT_INPUTS_LAST_USE
@@ -157,8 +157,9 @@ def run_purlin(args):
         stage_bytes=args.stage_bytes, flags=step_flags | B.PL_OPT_OVERLAP_LAUNCH)
     rs = B.pl_schedule_build(comm, B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, chunk, opts_rs)
     if args.ag_grid:    # profiling runs: the all-gather's grid given instead of measured (no tuning launches)
+        first, count = (int(v) for v in args.ag_idle.split(":")) if args.ag_idle else (0, 0)
         opts_ag = B.make_opts(n_ctas=args.ag_grid, threads=args.threads, slice_bytes=args.slice_bytes, datapath=args.datapath,
-                              stages=args.stages, stage_bytes=args.stage_bytes, flags=step_flags)
+                              stages=args.stages, stage_bytes=args.stage_bytes, flags=step_flags, idle_sm_first=first, idle_sm_count=count)
     else:
         opts_ag = opts
     ag = B.pl_schedule_build(comm, B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, chunk, opts_ag)
@@ -307,7 +308,8 @@ def run_purlin(args):
                        "algbw_gbs": iag.message_bytes / (ag_ms.mean() * 1e-3) / 1e9,
                        "hbm_gbs_compulsory": ag_gbs, "frac_measured": ag_gbs / peak,
                        "schedule_gbs": (iag.bytes_read + iag.bytes_written) / (ag_ms.mean() * 1e-3) / 1e9},
-        "grid": int(irs.grid), "grid_all_gather": int(iag.grid), "grid_all_gather_tuned": int(tuned_grid), "threads": int(irs.threads), "slice_bytes": int(irs.slice_bytes),
+        "grid": int(irs.grid), "grid_all_gather": int(iag.grid), "grid_all_gather_tuned": int(tuned_grid),
+        "idle_sms_all_gather": {"first": int(iag.idle_sm_first), "count": int(iag.idle_sm_count)}, "threads": int(irs.threads), "slice_bytes": int(irs.slice_bytes),
         "datapath": int(irs.datapath), "n_ops_rs": int(irs.n_ops), "n_ops_ag": int(iag.n_ops),
     }
 
@@ -668,6 +670,7 @@ def main():
     ap.add_argument("--no-latency", action="store_true")
     ap.add_argument("--no-detail", action="store_true", help="skip the other configurations (C1, C3, C4, C5, stream ceilings)")
     ap.add_argument("--ag-grid", type=int, default=0, help="grid of the all-gather schedule (skips pl_comm_tune); for profiling runs")
+    ap.add_argument("--ag-idle", default="", help="with --ag-grid: window of idle SMs of the all-gather launch as first:count")
     ap.add_argument("--no-tune", action="store_true", help="skip pl_comm_tune (the all-gather then runs with the untuned default grid)")
     ap.add_argument("--plain-options", action="store_true", help="build the two schedules of the step without PL_OPT_INPUTS_LAST_USE")
     ap.add_argument("--min-timed-ms", type=float, default=500.0, help="repeat the K-step block until the timed region lasts this long")

@@ -177,6 +177,15 @@ typedef struct {
                          /* the one conversion to the element type, e.g. 1/R for an average.    */
                          /* 0 = no scaling.  Float element types only (PL_ERR_UNSUPPORTED).     */
   uint32_t hook;         /* PL_HOOK_* bits: further steps of the processing phase (below)        */
+  int32_t idle_sm_first; /* SM-window launch (bulk-copy datapath, schedules without flags): one  */
+  int32_t idle_sm_count; /* CTA per SM is launched and the CTAs on SMs idle_sm_first ..          */
+                         /* idle_sm_first + idle_sm_count - 1 return at once; the others claim   */
+                         /* the queues.  n_ctas must be 0 or the SM count minus idle_sm_count,   */
+                         /* which must be a multiple of R.  0 = the library decides (a plain     */
+                         /* launch, or the window pl_comm_tune measured / the default one for    */
+                         /* pushed all-gathers).  Which SMs take part decides how fast a write-  */
+                         /* dominated stream runs (pl_comm_tune).  PL_ERR_UNSUPPORTED where it   */
+                         /* does not apply.  No counterpart in the paper.                        */
 } pl_sched_opts_t;
 /* The processing phase as a small family (Sec. 3.3: the phase between the last addition and the
  * store is configurable while the sum sits in registers).  With s = out_scale (1 if unset):
@@ -292,6 +301,7 @@ typedef struct {
                                        /* cached between launches: bytes_read with every byte of the   */
                                        /* caller's inputs (and second operands) counted once, however  */
                                        /* many ops read it, plus bytes_written                         */
+  int32_t idle_sm_first, idle_sm_count; /* SM-window launch: the SMs that sit out (count 0: plain launch of `grid` CTAs) */
 } pl_sched_info_t;
 
 /* Device buffers of one execute: in[r] / out[r] for r < R, 16-byte aligned, non-overlapping.
@@ -335,19 +345,25 @@ pl_status_t pl_comm_create_planner(int R, pl_dtype_t dtype, pl_comm_t* out);
  * (PL_ERR_INVALID_ARG otherwise). */
 pl_status_t pl_comm_destroy(pl_comm_t comm);
 
-/* Measure, on this communicator's GPU, the grid with which the write-dominated direct schedules
- * of the bulk-copy datapath (all-gather, all-gather-v, broadcast: 1 read : R writes) run fastest,
- * and make it the default of later builds on this communicator (opts.n_ctas still overrides; the
- * schedules already built keep theirs).  Such a stream is served best with fewer than all SMs
- * writing, and how many differs from one GPU to the next of the same model (of two B200s one ran
- * the 8 x 64 MiB all-gather fastest with 136 CTAs, the other with 128: 113 us with 136).  Runs an
- * all-gather of 64 MiB with every multiple of R between 3/4 of the resident CTAs and all of them
- * (2 + 6 launches each) on `stream`, on buffers it allocates and frees ((R + 1) x 64 MiB), and
- * synchronises: a call for set-up time, not for the hot path.  Nothing in the paper corresponds
- * to it.  *push_ctas_out (may be NULL) receives the chosen grid.
+/* Measure, on this communicator's GPU, with how many CTAs and on WHICH SMs the write-dominated
+ * direct schedules of the bulk-copy datapath (all-gather, all-gather-v, broadcast: 1 read : R
+ * writes) run fastest, and make the result the default of later builds on this communicator
+ * (opts.n_ctas / opts.idle_sm_count still override; schedules already built keep theirs).  Such
+ * a stream is served best with fewer than all SMs writing, and with the right ones sitting out:
+ * 16-20 idle SMs taken from SM ids 0-31 or 64-79 gave 97-103 us for the 8 x 64 MiB all-gather on
+ * every B200 tried, the same number anywhere else 108-116 us; which SMs a plain launch of fewer
+ * CTAs leaves idle is up to the hardware and differs from one GPU to the next of the same model
+ * (plain launches: 101 us at best on some, 107 us on others).  Candidates: plain launches of
+ * every multiple of R between 3/4 of the resident CTAs and all of them, and the same grids
+ * launched as one CTA per SM with the idle SMs as a window starting at SM 0, 8, 16 or 64; each
+ * runs an all-gather of 64 MiB (2 + 6 launches) on `stream`, on buffers this call allocates and
+ * frees ((R + 1) x 64 MiB).  Synchronises: a call for set-up time, not for the hot path.  Nothing
+ * in the paper corresponds to it.  The outputs (each may be NULL) receive the chosen grid and
+ * window (count 0: a plain launch).
  * Errors: PL_ERR_UNSUPPORTED (planner communicator), PL_ERR_OOM, PL_ERR_CUDA, PL_ERR_INVALID_ARG
  * (the current device is not the communicator's). */
-pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out);
+pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out, int32_t* idle_sm_first_out,
+                         int32_t* idle_sm_count_out);
 
 /* Read the device status record as it stands at the time of the call (on an internal stream: the
  * call waits for no other work, so synchronise the stream of the executes you ask about first).

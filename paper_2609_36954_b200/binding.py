@@ -54,7 +54,8 @@ class pl_sched_opts_t(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("n_ctas", C.c_int32), ("threads", C.c_int32),
                 ("datapath", C.c_int32), ("stages", C.c_int32), ("stage_bytes", C.c_uint32),
                 ("slice_bytes", C.c_uint32), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32),
-                ("staging_bytes", C.c_uint64), ("out_scale", C.c_float), ("hook", C.c_uint32)]
+                ("staging_bytes", C.c_uint64), ("out_scale", C.c_float), ("hook", C.c_uint32),
+                ("idle_sm_first", C.c_int32), ("idle_sm_count", C.c_int32)]
 
 
 class pl_ref_t(C.Structure):
@@ -80,7 +81,7 @@ class pl_sched_info_t(C.Structure):
                 ("datapath", C.c_int32), ("stages", C.c_int32),
                 ("stage_bytes", C.c_uint32), ("slice_bytes", C.c_uint32),
                 ("aux_bytes", C.c_uint64 * PL_MAX_RANKS), ("out_dtype", C.c_int32), ("hook", C.c_uint32),
-                ("hbm_bytes", C.c_uint64)]
+                ("hbm_bytes", C.c_uint64), ("idle_sm_first", C.c_int32), ("idle_sm_count", C.c_int32)]
 
 
 class pl_bufs_t(C.Structure):
@@ -149,7 +150,7 @@ def load():
         "pl_execute_host_async": [vp, P(pl_bufs_t), P(pl_bufs_t), vp],
         "pl_comm_host_fence": [vp, vp],
         "pl_comm_host_sync": [vp],
-        "pl_comm_tune": [vp, vp, P(C.c_int32)],
+        "pl_comm_tune": [vp, vp, P(C.c_int32), P(C.c_int32), P(C.c_int32)],
         "pl_moe_plan_create": [vp, i32, i32, i32, i32, sz, P(vp)],
         "pl_moe_plan_destroy": [vp],
         "pl_moe_dispatch": [vp, P(vp), P(vp), P(vp), P(vp), vp],
@@ -187,7 +188,7 @@ def _check(st, where):
 
 
 def make_opts(n_ctas=0, threads=0, datapath=PL_DP_AUTO, stages=0, stage_bytes=0, slice_bytes=0,
-              timeout_ns=0, flags=0, staging_bytes=0, out_scale=0.0, hook=0):
+              timeout_ns=0, flags=0, staging_bytes=0, out_scale=0.0, hook=0, idle_sm_first=0, idle_sm_count=0):
     o = pl_sched_opts_t()
     o.struct_size = C.sizeof(pl_sched_opts_t)
     o.n_ctas, o.threads, o.datapath, o.stages = n_ctas, threads, datapath, stages
@@ -195,6 +196,7 @@ def make_opts(n_ctas=0, threads=0, datapath=PL_DP_AUTO, stages=0, stage_bytes=0,
     o.staging_bytes = staging_bytes
     o.out_scale = out_scale
     o.hook = hook
+    o.idle_sm_first, o.idle_sm_count = idle_sm_first, idle_sm_count
     return o
 
 
@@ -340,11 +342,12 @@ def pl_comm_host_fence(comm, stream=0):
     _check(load().pl_comm_host_fence(comm, stream), "pl_comm_host_fence")
 
 
-def pl_comm_tune(comm, stream=0):
-    """Returns the grid chosen for pushed copies on the bulk-copy datapath."""
-    g = C.c_int32(0)
-    _check(load().pl_comm_tune(comm, stream, C.byref(g)), "pl_comm_tune")
-    return int(g.value)
+def pl_comm_tune(comm, stream=0, full=False):
+    """Returns the grid chosen for pushed copies on the bulk-copy datapath; with full=True the
+    tuple (grid, first idle SM, idle SMs) (idle SMs = 0: a plain launch)."""
+    g, f, n = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    _check(load().pl_comm_tune(comm, stream, C.byref(g), C.byref(f), C.byref(n)), "pl_comm_tune")
+    return (int(g.value), int(f.value), int(n.value)) if full else int(g.value)
 
 
 def pl_comm_host_sync(comm):

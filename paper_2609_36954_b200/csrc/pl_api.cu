@@ -38,6 +38,9 @@ struct pl_schedule_s {
   pl_sched_info_t info{};
   uint64_t timeout_ns = 0;
   bool no_l2_hints = false;
+  bool sm_window = false;         // launch one CTA per SM; the SMs outside sm_mask sit out (pol.idle_first / idle_count)
+  uint32_t sm_mask[5] = {0, 0, 0, 0, 0};
+  size_t off_sm_state = 0;
   bool inputs_last_use = false;   // PL_OPT_INPUTS_LAST_USE asked for and every input byte is read once
   bool trace = false;
   bool overlap_launch = false;
@@ -128,6 +131,8 @@ void fill_info(pl_schedule_s* S, int R) {
   I.out_dtype = (S->hook & PL_HOOK_F32_OUT) ? PL_F32 : S->comm->dtype;
   I.hook = S->hook;
   I.grid = S->pol.n_ctas;
+  I.idle_sm_first = S->sm_window ? S->pol.idle_first : 0;
+  I.idle_sm_count = S->sm_window ? S->pol.idle_count : 0;
   I.threads = S->pol.threads;
   I.smem_bytes = S->pol.datapath == PL_DP_TMA ? (int32_t)exec_tma_smem_bytes(S->pol.stages, S->pol.stage_bytes) : 0;
   I.datapath = S->pol.datapath;
@@ -198,6 +203,7 @@ pl_status_t upload(pl_schedule_s* S, int R) {
   S->off_waits = place(S->waits.size() * sizeof(DevWait));
   S->off_flags = place((size_t)std::max(1, S->L.n_flags) * sizeof(unsigned long long) * (S->stage_ahead ? 2 : 1));
   S->off_epoch = place(4 * sizeof(unsigned long long));
+  S->off_sm_state = place(3 * sizeof(unsigned long long));   // claim words of SM-window launches (zeroed with the flags)
   S->sync_bytes = off - S->off_flags;
   if (S->trace) S->off_trace = place(2 * S->L.ops.size() * sizeof(unsigned long long));
   S->blob_bytes = off;
@@ -324,6 +330,7 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   uint64_t timeout = 2000000000ull;
   uint32_t flags = 0, hook = 0;
   float out_scale = 1.0f;
+  bool idle_asked = false;  // opts name a window of idle SMs
   if (opts) {
     if (opts->struct_size != sizeof(pl_sched_opts_t)) return PL_ERR_INVALID_ARG;
     pol.n_ctas = opts->n_ctas;
@@ -341,6 +348,17 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
       out_scale = opts->out_scale;
     }
     hook = opts->hook;
+    if (opts->idle_sm_count < 0 || opts->idle_sm_first < 0) return PL_ERR_INVALID_ARG;
+    if (opts->idle_sm_count > 0) {
+      // an explicit window: the grid is every other SM
+      const int active = comm->sm_count - opts->idle_sm_count;
+      if (opts->idle_sm_first + opts->idle_sm_count > comm->sm_count || active < comm->R || active % comm->R) return PL_ERR_INVALID_ARG;
+      if (pol.n_ctas != 0 && pol.n_ctas != active) return PL_ERR_INVALID_ARG;
+      pol.n_ctas = active;
+      pol.idle_first = opts->idle_sm_first;
+      pol.idle_count = opts->idle_sm_count;
+      idle_asked = true;
+    }
     if (hook & ~(PL_HOOK_RESIDUAL | PL_HOOK_F32_OUT)) return PL_ERR_INVALID_ARG;
     if (hook && comm->dtype != PL_BF16 && comm->dtype != PL_F32) return PL_ERR_UNSUPPORTED;
     if (pol.threads < 0 || pol.threads % 32 || pol.threads > exec_max_threads()) return PL_ERR_INVALID_ARG;
@@ -362,6 +380,9 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   if (pol.datapath == PL_DP_PACKET) return build_packets(comm, rq, pol, timeout, flags, out_scale, out);
   rq.pol = pol;
   rq.tuned_push_ctas = comm->tuned_push_ctas;
+  rq.tuned_idle_first = comm->tuned_idle_first;
+  rq.tuned_idle_count = comm->tuned_idle_count;
+  rq.sm_count = comm->sm_count;
   const int requested = pol.n_ctas;
   pol = default_policy(rq, 0);  // datapath, threads, ring geometry
   rq.pol = pol;
@@ -436,6 +457,24 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   }
   for (const HostOp& op : S->L.ops)
     if (op.kind == PL_OP_COPY && op.bcast) S->bcast_copies = true;
+  // A window of idle SMs needs: the bulk-copy datapath with one CTA per SM, no flags (a queue
+  // may be claimed late, so no queue may wait for another), one staging buffer, at most 160 SMs.
+  if (S->pol.idle_count > 0) {
+    const bool fits = pol.datapath == PL_DP_TMA && !comm->planner && S->L.n_flags == 0 && !S->stage_ahead && comm->sm_count <= 160 &&
+                      exec_tma_max_ctas_per_sm(comm->dtype, pol.stages, pol.stage_bytes) == 1 &&
+                      S->pol.n_ctas + S->pol.idle_count == comm->sm_count;
+    if (!fits && idle_asked) {
+      comm->last_error = "a window of idle SMs needs the bulk-copy datapath with one CTA per SM and a schedule without flags";
+      delete S;
+      return PL_ERR_UNSUPPORTED;
+    }
+    if (!fits) S->pol.idle_count = 0;
+  }
+  if (S->pol.idle_count > 0) {
+    S->sm_window = true;
+    for (int sm = 0; sm < comm->sm_count; ++sm)
+      if (sm < S->pol.idle_first || sm >= S->pol.idle_first + S->pol.idle_count) S->sm_mask[sm >> 5] |= 1u << (sm & 31);
+  }
   fill_info(S, comm->R);
   flatten(S, comm->dtype);
   if (!comm->planner) {
@@ -606,9 +645,11 @@ pl_status_t pl_comm_destroy(pl_comm_t comm) {
   return PL_OK;
 }
 
-pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out) {
+pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out, int32_t* idle_sm_first_out, int32_t* idle_sm_count_out) {
   if (!comm) return PL_ERR_INVALID_ARG;
   if (push_ctas_out) *push_ctas_out = 0;
+  if (idle_sm_first_out) *idle_sm_first_out = 0;
+  if (idle_sm_count_out) *idle_sm_count_out = 0;
   if (comm->planner) return PL_ERR_UNSUPPORTED;
   if (!on_comm_device(comm)) return PL_ERR_INVALID_ARG;
   const int R = comm->R;
@@ -637,16 +678,30 @@ pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out) {
   }
   const int per_sm = exec_tma_max_ctas_per_sm(comm->dtype, 4, 48 * 1024);
   const int resident = std::max(1, per_sm) * comm->sm_count;
-  int best = 0;
+  // candidates: plain launches of every multiple of R down to 3/4 of the resident CTAs, and, with
+  // one CTA per SM, the same grids with the idle SMs as a window at a few places of the SM range
+  struct Cand { int n_ctas, idle_first, idle_count; };
+  std::vector<Cand> cands;
+  const int firsts[] = {0, 8, 16, 64};
+  for (int g = resident / R * R; g >= resident * 3 / 4 && g >= R; g -= R) {
+    cands.push_back({g, 0, 0});
+    const int idle = comm->sm_count - g;
+    if (per_sm == 1 && comm->sm_count <= 160 && idle >= 12 && idle <= 40)
+      for (int f : firsts)
+        if (f + idle <= comm->sm_count) cands.push_back({g, f, idle});
+  }
+  Cand best{0, 0, 0};
   float best_ms = 0.f;
   pl_status_t result = PL_OK;
-  const int saved = comm->tuned_push_ctas;
-  for (int g = resident / R * R; g >= resident * 3 / 4 && g >= R; g -= R) {
+  const Cand saved{comm->tuned_push_ctas, comm->tuned_idle_first, comm->tuned_idle_count};
+  for (const Cand& cd : cands) {
     pl_sched_opts_t o;
     std::memset(&o, 0, sizeof(o));
     o.struct_size = sizeof(o);
-    o.n_ctas = g;
+    o.n_ctas = cd.n_ctas;
     o.datapath = PL_DP_TMA;
+    o.idle_sm_first = cd.idle_first;
+    o.idle_sm_count = cd.idle_count;
     pl_schedule_t s = nullptr;
     if (pl_schedule_build(comm, PL_ALLGATHER, PL_ALGO_DIRECT, count, (size_t)1 << 20, &o, &s) != PL_OK) continue;
     bool ok = true;
@@ -663,8 +718,11 @@ pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out) {
       result = PL_ERR_CUDA;
       break;
     }
-    if (best == 0 || ms < best_ms) {
-      best = g;
+    // a window launch costs its CTAs a claim (an atomic's round trip) in front of their first
+    // load: it has to beat the best plain launch by more than that to be taken
+    const float handicap = cd.idle_count > 0 ? 1.015f : 1.0f;
+    if (best.n_ctas == 0 || ms * handicap < best_ms * (best.idle_count > 0 ? 1.015f : 1.0f)) {
+      best = cd;
       best_ms = ms;
     }
   }
@@ -673,8 +731,13 @@ pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out) {
   cudaEventDestroy(e1);
   cudaFree(d_in);
   cudaFree(d_out);
-  comm->tuned_push_ctas = (result == PL_OK && best > 0) ? best : saved;
-  if (push_ctas_out) *push_ctas_out = comm->tuned_push_ctas;
+  const Cand pick = (result == PL_OK && best.n_ctas > 0) ? best : saved;
+  comm->tuned_push_ctas = pick.n_ctas;
+  comm->tuned_idle_first = pick.idle_first;
+  comm->tuned_idle_count = pick.idle_count;
+  if (push_ctas_out) *push_ctas_out = pick.n_ctas;
+  if (idle_sm_first_out) *idle_sm_first_out = pick.idle_first;
+  if (idle_sm_count_out) *idle_sm_count_out = pick.idle_count;
   return result;
 }
 
@@ -974,6 +1037,8 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   P.epoch = reinterpret_cast<unsigned long long*>(s->d_blob + s->off_epoch);
   P.status = s->comm->d_status;
   P.trace = s->trace ? reinterpret_cast<unsigned long long*>(s->d_blob + s->off_trace) : nullptr;
+  P.sm_state = s->sm_window ? reinterpret_cast<unsigned long long*>(s->d_blob + s->off_sm_state) : nullptr;
+  for (int i = 0; i < 5; ++i) P.sm_mask[i] = s->sm_mask[i];
   P.timeout_ns = s->timeout_ns;
   P.n_ranks = R;
   P.stages = s->pol.stages;
@@ -985,7 +1050,7 @@ pl_status_t pl_execute(pl_schedule_t s, const pl_bufs_t* bufs, void* stream) {
   P.pipelined_reduce = s->pipelined_reduce ? 1u : 0u;
   P.bcast_copies = s->bcast_copies ? 1u : 0u;
   cudaError_t le = s->pol.datapath == PL_DP_TMA
-                       ? launch_exec_tma(s->comm->dtype, P, s->pol.n_ctas, static_cast<cudaStream_t>(stream))
+                       ? launch_exec_tma(s->comm->dtype, P, s->sm_window ? s->comm->sm_count : s->pol.n_ctas, static_cast<cudaStream_t>(stream))
                        : launch_exec(s->comm->dtype, P, s->pol.n_ctas, s->pol.threads, static_cast<cudaStream_t>(stream));
   if (le != cudaSuccess) return PL_ERR_CUDA;
   g_launches.fetch_add(1);

@@ -22,6 +22,7 @@ struct pl_comm_s {
   std::vector<pl_schedule_s*> schedules;
   int n_plans = 0;
   int tuned_push_ctas = 0;  // pl_comm_tune: best grid for pushed copies on the bulk-copy datapath (0 = not measured)
+  int tuned_idle_first = 0, tuned_idle_count = 0;  // and the idle SM window measured with it (count 0: plain launch)
   std::string last_error;
   // pl_execute_host_async: an upload and a download stream, and the downloads still in flight
   // with the host and device ranges they touch (hazards are resolved with their events)

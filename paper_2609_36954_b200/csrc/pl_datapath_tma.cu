@@ -84,6 +84,7 @@ struct Ctrl {
   int abort;
   int pad;
   unsigned long long launch;  // double-buffered staging: number of this launch (taken at entry by thread 0)
+  int q;                      // SM-window launches: the queue this CTA claimed (-1: its SM sits out)
   StageDesc desc[kMaxStages];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
@@ -100,7 +101,7 @@ __device__ __forceinline__ bool wait_bar(const ExecParams& P, Ctrl* c, uint64_t*
     if ((spins & 255u) == 0) {
       if (*reinterpret_cast<volatile int*>(&c->abort)) return false;
       if (globaltimer_ns() - t0 > 2ull * P.timeout_ns + 1000000ull) {
-        record_timeout(P, blockIdx.x, 0xFFFFFFFFu, 0xFFFFFFFFu, parity, 0);
+        record_timeout(P, c->q, 0xFFFFFFFFu, 0xFFFFFFFFu, parity, 0);
         *reinterpret_cast<volatile int*>(&c->abort) = 1;
         return false;
       }
@@ -344,12 +345,72 @@ __device__ __forceinline__ bool leaves_via_smem(uint32_t kind, uint32_t flags, u
 // and staging buffer follow the parity of a launch counter taken at entry; the producer runs the
 // leading stage ops of its queue (copies from the caller's input into the staging buffer of this
 // parity) before it waits for the launch in front, the copier ships them, the consumers wait.
+// SM-window launches (write-dominated schedules without flags).  One CTA is launched per SM; a CTA
+// whose SM lies in the idle window sits the launch out, every other CTA claims the next queue.
+// How fast a 1 read : R writes stream runs depends on WHICH SMs take part (see pl_comm_tune), and
+// a plain launch of fewer CTAs than SMs leaves that choice to the hardware.
+// State (three words, zero between launches): [0] arrivals << 32 | queues claimed by CTAs on
+// active SMs, [1] queues claimed afterwards, [2] (low half) CTAs that have left.  Every CTA adds
+// itself to [0] with ONE atomic (no compare-and-swap loop: 148 CTAs contending for one word would
+// take tens of microseconds).  A CTA on an active SM runs the queue it drew.  A CTA on an idle SM
+// waits until all CTAs have arrived, normally a microsecond, and leaves; should the CTAs not have
+// landed one per SM (other work on the GPU), queues are left over then and the waiting CTAs draw
+// them from [1], so every queue runs exactly once.  The last CTA to leave zeroes the state.
+__device__ __forceinline__ int claim_queue(const ExecParams& P) {
+  uint32_t sm;
+  asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+  const bool active = sm >= 160u || ((P.sm_mask[sm >> 5] >> (sm & 31u)) & 1u);
+  const uint32_t total = gridDim.x;
+  const unsigned long long mine = (1ull << 32) | (active ? 1ull : 0ull);
+  const unsigned long long old = atomicAdd(P.sm_state, mine);
+  if (active) {
+    const uint32_t taken = (uint32_t)old;
+    return taken < P.n_queues ? (int)taken : -1;  // a surplus CTA on an active SM has nothing to do
+  }
+  // idle SM: wait for the count of arrivals to be complete (bounded), then look for leftovers
+  unsigned long long now = old + mine;
+  const unsigned long long t0 = globaltimer_ns();
+  for (uint32_t spins = 1; (uint32_t)(now >> 32) < total; ++spins) {
+    now = *reinterpret_cast<volatile unsigned long long*>(P.sm_state);
+    if ((spins & 63u) == 0 && globaltimer_ns() - t0 > 2ull * P.timeout_ns + 1000000ull) break;
+  }
+  const uint32_t by_active = (uint32_t)now;
+  if ((uint32_t)(now >> 32) < total || by_active >= P.n_queues) return -1;
+  const uint32_t extra = atomicAdd(reinterpret_cast<unsigned int*>(P.sm_state + 1), 1u);
+  return by_active + extra < P.n_queues ? (int)(by_active + extra) : -1;
+}
+// A CTA of an SM-window launch leaves: the last one puts the state back to zero.
+__device__ __forceinline__ void leave_window(const ExecParams& P) {
+  __threadfence();
+  const unsigned int left = atomicAdd(reinterpret_cast<unsigned int*>(P.sm_state + 2), 1u);
+  if (left == gridDim.x - 1u) {
+    P.sm_state[0] = 0ull;
+    P.sm_state[1] = 0ull;
+    P.sm_state[2] = 0ull;
+    __threadfence();
+  }
+}
+
 template <int DT, int CW, bool HOOK = false, bool DBUF = false>
 __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_kernel(const __grid_constant__ ExecParams P) {
   extern __shared__ __align__(1024) unsigned char smem[];
   Ctrl* c = reinterpret_cast<Ctrl*>(smem);
   unsigned char* slots = smem + kCtrlBytes;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, q = blockIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int q = blockIdx.x;
+  uint32_t n_cta = gridDim.x;  // CTAs that work in this launch
+  if constexpr (!DBUF) {
+    if (P.sm_state != nullptr) {
+      if (tid == 0) c->q = claim_queue(P);
+      __syncthreads();
+      q = c->q;
+      n_cta = P.n_queues;
+      if (q < 0) {  // this SM sits the launch out (an exited CTA counts as having let dependents go)
+        if (tid == 0) leave_window(P);
+        return;
+      }
+    }
+  }
   const uint32_t S = (uint32_t)P.stages, slot_bytes = P.stage_bytes;
   const bool has_flags = P.flags != nullptr;
   if constexpr (!DBUF) pdl_launch_dependents();
@@ -362,6 +423,7 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
     }
     for (uint32_t s = 0; s < S; ++s) ptx::mbar_init(&c->done[s], CW);
     c->abort = 0;
+    c->q = q;
     ptx::mbar_init_fence();
   }
   // Producers: the first descriptor of the queue.  Descriptors are written when the schedule is
@@ -715,9 +777,12 @@ __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_ker
   }
 
   __syncthreads();
+  if constexpr (!DBUF) {
+    if (tid == 0 && P.sm_state != nullptr) leave_window(P);
+  }
   if (tid == 0 && has_flags && !DBUF && !*reinterpret_cast<volatile int*>(&c->abort)) {
     const unsigned long long prev = atomicAdd(P.epoch + 1, 1ull);
-    if (prev == (unsigned long long)gridDim.x - 1ull) {
+    if (prev == (unsigned long long)n_cta - 1ull) {
       P.epoch[1] = 0ull;
       __threadfence();
       *reinterpret_cast<volatile unsigned long long*>(P.epoch) = epoch;

@@ -87,6 +87,10 @@ struct ExecParams {
   unsigned long long* epoch;    // [0] executes completed, [1] CTAs finished in this execute, [2] CTAs started (double-buffered staging)
   int* status;                  // pl_devstatus_t words + abort word (comm-owned)
   unsigned long long* trace;    // optional: per op (topological index) [start, end] %globaltimer stamps
+  // SM-window launches of the bulk-copy executor: one CTA per SM is launched, the CTAs on SMs
+  // whose bit is clear in sm_mask return, the others claim queues through sm_state (null: plain launch)
+  unsigned long long* sm_state;
+  uint32_t sm_mask[5];
   // Double-buffered staging (PL_OPT_STAGE_AHEAD): launch i uses flag set and scratch half i mod 2
   uint32_t stage_ahead;         // 0 / 1
   uint32_t n_flags;             // flags per set
@@ -120,6 +124,7 @@ struct PacketParams {
 
 struct Policy {
   int n_ctas, threads, datapath, stages;
+  int idle_first, idle_count;  // SM-window launch: SMs that sit out (count 0: plain launch); idle_count < 0: asked for "none" 
   uint32_t stage_bytes, slice_bytes;
   // automatic slicing (slice_bytes == 0): bounds of a slice
   uint32_t min_slice, max_slice;
@@ -153,6 +158,8 @@ struct BuildRequest {
   uint32_t hook;             // PL_HOOK_* bits
   bool stage_ahead;          // PL_OPT_STAGE_AHEAD
   int tuned_push_ctas;       // > 0: grid that pl_comm_tune measured for pushed copies on the bulk-copy datapath
+  int tuned_idle_first, tuned_idle_count;  // and the window of idle SMs it measured with it (count 0: plain launch)
+  int sm_count;              // SMs of the communicator's GPU
   Policy pol;
 };
 

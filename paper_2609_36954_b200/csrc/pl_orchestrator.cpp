@@ -812,8 +812,23 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
     // pl_comm_tune measures it; untuned, 87 % of the resident CTAs (128 of 148) is the safe choice.
     if (p.datapath == PL_DP_TMA && (rq.coll == PL_ALLGATHER || rq.coll == PL_ALLGATHERV || rq.coll == PL_BROADCAST) &&
         rq.algo == PL_ALGO_DIRECT && !rq.staged) {
-      if (rq.tuned_push_ctas > 0 && rq.tuned_push_ctas <= max_resident_ctas) full = std::max(rq.R, rq.tuned_push_ctas / rq.R * rq.R);
-      else full = std::max(rq.R, (max_resident_ctas * 87 / 100) / rq.R * rq.R);
+      const bool one_per_sm = rq.sm_count > 0 && max_resident_ctas == rq.sm_count;
+      if (rq.tuned_push_ctas > 0 && rq.tuned_push_ctas <= max_resident_ctas) {
+        full = std::max(rq.R, rq.tuned_push_ctas / rq.R * rq.R);
+        if (p.idle_count == 0 && one_per_sm && rq.tuned_idle_count > 0 && full + rq.tuned_idle_count == rq.sm_count) {
+          p.idle_first = rq.tuned_idle_first;
+          p.idle_count = rq.tuned_idle_count;
+        }
+      } else {
+        full = std::max(rq.R, (max_resident_ctas * 87 / 100) / rq.R * rq.R);
+        // Untuned: WHICH SMs sit out matters as much as how many (pl_comm_tune); a window of idle
+        // SMs that starts at SM 8 was among the fast ones on every B200 tried (97-100 us for the
+        // 8 x 64 MiB all-gather), the SMs a plain launch leaves idle were not (98-107 us).
+        if (p.idle_count == 0 && one_per_sm && rq.sm_count == 148 && full < rq.sm_count) {
+          p.idle_first = 8;
+          p.idle_count = rq.sm_count - full;
+        }
+      }
     }
     // bytes a rank produces in its busiest phase
     uint64_t per_rank = msg;
@@ -825,6 +840,8 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
     p.n_ctas = (int)std::min<uint64_t>(full, std::max<uint64_t>(rq.R, want));
   }
   p.n_ctas = std::max(rq.R, p.n_ctas / rq.R * rq.R);
+  // a window of idle SMs goes with a grid of exactly the other SMs
+  if (p.idle_count > 0 && (rq.sm_count <= 0 || p.n_ctas + p.idle_count != rq.sm_count)) p.idle_count = 0;
   return p;
 }
 

@@ -30,7 +30,7 @@ def test_struct_layouts_match_header_sizes():
     assert ctypes.sizeof(B.pl_op_t) == 40 + 8 + 24 + 24 * 16 + 4 * 16 + 4 * 16
     assert ctypes.sizeof(B.pl_bufs_t) == 6 * 16 * 8
     assert ctypes.sizeof(B.pl_devstatus_t) == 32
-    assert ctypes.sizeof(B.pl_sched_opts_t) == 64
+    assert ctypes.sizeof(B.pl_sched_opts_t) == 72
 
 
 def test_status_strings():
