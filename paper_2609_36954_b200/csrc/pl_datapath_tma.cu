@@ -375,7 +375,12 @@ __device__ __forceinline__ int claim_queue(const ExecParams& P) {
     if ((spins & 63u) == 0 && globaltimer_ns() - t0 > 2ull * P.timeout_ns + 1000000ull) break;
   }
   const uint32_t by_active = (uint32_t)now;
-  if ((uint32_t)(now >> 32) < total || by_active >= P.n_queues) return -1;
+  if ((uint32_t)(now >> 32) < total) {
+    // CTAs of this launch are still missing after the time limit: queues may go unclaimed, say so
+    record_timeout(P, (int)blockIdx.x, 0xFFFFFFFFu, 0xFFFFFFFFu, total, (uint32_t)(now >> 32));
+    return -1;
+  }
+  if (by_active >= P.n_queues) return -1;
   const uint32_t extra = atomicAdd(reinterpret_cast<unsigned int*>(P.sm_state + 1), 1u);
   return by_active + extra < P.n_queues ? (int)(by_active + extra) : -1;
 }

@@ -3,12 +3,13 @@ schedules built with PL_OPT_INPUTS_LAST_USE (inputs loaded evict-first) or PL_OP
 the same bits as the default ones, and match the oracle."""
 import numpy as np
 import pytest
+import torch
 
 from oracle import oracle
 from paper_2609_36954_b200 import binding as B
 from paper_2609_36954_b200 import inputs as gen
 
-from gpu_harness import Session, check_float
+from gpu_harness import Session, check_float, poison, stream_handle, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -87,5 +88,93 @@ def test_comm_tune_picks_a_grid_and_later_builds_use_it():
             assert np.array_equal(outs[r].view(np.uint16), ref[r])
         s2 = ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 20, datapath=B.PL_DP_TMA, n_ctas=104)
         assert B.pl_schedule_info(s2).grid == 104                 # an explicit grid still wins
+    finally:
+        ses.close()
+
+
+def test_sm_window_launch_matches_the_oracle_and_reports_its_window():
+    """One CTA per SM is launched, the SMs of the window sit out, the others claim the queues:
+    the bytes are those of a plain launch, whatever window is asked for."""
+    R = 8
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n = R * (3 << 20) + R * 4096 * 3
+    x = gen.rank_inputs(R, n // R, "bf16", seed=23)
+    ref = oracle.allgather(x)
+    ses = Session(R, "bf16")
+    try:
+        for first, count in ((0, sms - 128), (8, sms - 128), (sms - 36, 36), (64, 12)):
+            if count <= 0 or (sms - count) % R:
+                continue
+            s = ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 20, datapath=B.PL_DP_TMA, idle_sm_first=first, idle_sm_count=count)
+            info = B.pl_schedule_info(s)
+            assert (info.grid, info.idle_sm_first, info.idle_sm_count) == (sms - count, first, count)
+            for rep in range(3):                       # the claim words must be back at zero after every launch
+                outs, _ = ses.execute(s, x)
+                for r in range(R):
+                    assert np.array_equal(outs[r].view(np.uint16), ref[r]), (first, count, rep, r)
+        # a reduce-scatter (no flags either) under a window, against the oracle
+        xr = gen.rank_inputs(R, n, "bf16", seed=24)
+        s = ses.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, 1 << 20, datapath=B.PL_DP_TMA, idle_sm_first=16, idle_sm_count=sms - 128)
+        outs, _ = ses.execute(s, xr, repeats=2)
+        rref = oracle.reduce_scatter(xr, "bf16")
+        for r in range(R):
+            check_float(gen.bf16_bits_to_f64(outs[r].view(np.uint16)), rref[r], "bf16")
+    finally:
+        ses.close()
+
+
+def test_sm_window_launch_keeps_every_queue_when_the_gpu_is_busy():
+    """Other work holds SMs while the window launch starts, so its CTAs do not land one per SM at
+    once: CTAs on idle SMs that arrive late must pick up what is left, none may run twice."""
+    R = 8
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n = R * (2 << 20)
+    x = gen.rank_inputs(R, n // R, "bf16", seed=29)
+    ref = oracle.allgather(x)
+    ses = Session(R, "bf16")
+    try:
+        s = ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 20, datapath=B.PL_DP_TMA, idle_sm_first=8, idle_sm_count=sms - 128)
+        info = B.pl_schedule_info(s)
+        d_in = [to_dev(a) for a in x]
+        d_out = [poison(info.out_bytes[r]) for r in range(R)]
+        bufs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out],
+                           [int(info.in_bytes[r]) for r in range(R)], [int(info.out_bytes[r]) for r in range(R)])
+        side = torch.cuda.Stream()
+        a = torch.randn(4096, 4096, device="cuda")
+        for rep in range(6):
+            for t in d_out:
+                t.fill_(0x5A)
+            torch.cuda.synchronize()
+            with torch.cuda.stream(side):               # a few milliseconds of work on every SM
+                for _ in range(4):
+                    a = torch.tanh(a @ a * 1e-4)
+            B.pl_execute(s, bufs, stream_handle())
+            B.pl_execute(s, bufs, stream_handle())
+            torch.cuda.synchronize()
+            assert B.pl_comm_status(ses.comm).code == B.PL_OK
+            for r in range(R):
+                assert np.array_equal(d_out[r][: int(info.out_bytes[r])].cpu().numpy().view(np.uint16), ref[r]), (rep, r)
+    finally:
+        ses.close()
+
+
+def test_sm_window_is_rejected_where_it_does_not_apply():
+    R = 8
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    ses = Session(R, "bf16")
+    try:
+        n = R * (1 << 20)
+        with pytest.raises(B.PurlinError) as e:       # a ring all-reduce has flags
+            ses.build(B.PL_ALLREDUCE, B.PL_ALGO_RING, n, 1 << 18, datapath=B.PL_DP_TMA, idle_sm_first=0, idle_sm_count=sms - 128)
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+        with pytest.raises(B.PurlinError) as e:       # the register datapath has no window launch
+            ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 18, datapath=B.PL_DP_LDST, idle_sm_first=0, idle_sm_count=sms - 128)
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+        with pytest.raises(B.PurlinError) as e:       # grid and window must add up to the SM count
+            ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 18, datapath=B.PL_DP_TMA, n_ctas=64, idle_sm_first=0, idle_sm_count=sms - 128)
+        assert e.value.status == B.PL_ERR_INVALID_ARG
+        with pytest.raises(B.PurlinError) as e:       # the other SMs must be a multiple of R
+            ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 18, datapath=B.PL_DP_TMA, idle_sm_first=0, idle_sm_count=sms - 127)
+        assert e.value.status == B.PL_ERR_INVALID_ARG
     finally:
         ses.close()
