@@ -345,56 +345,15 @@ __device__ __forceinline__ bool leaves_via_smem(uint32_t kind, uint32_t flags, u
 // and staging buffer follow the parity of a launch counter taken at entry; the producer runs the
 // leading stage ops of its queue (copies from the caller's input into the staging buffer of this
 // parity) before it waits for the launch in front, the copier ships them, the consumers wait.
-// SM-window launches (write-dominated schedules without flags).  One CTA is launched per SM; a CTA
-// whose SM lies in the idle window sits the launch out, every other CTA claims the next queue.
-// How fast a 1 read : R writes stream runs depends on WHICH SMs take part (see pl_comm_tune), and
-// a plain launch of fewer CTAs than SMs leaves that choice to the hardware.
-// State (three words, zero between launches): [0] arrivals << 32 | queues claimed by CTAs on
-// active SMs, [1] queues claimed afterwards, [2] (low half) CTAs that have left.  Every CTA adds
-// itself to [0] with ONE atomic (no compare-and-swap loop: 148 CTAs contending for one word would
-// take tens of microseconds).  A CTA on an active SM runs the queue it drew.  A CTA on an idle SM
-// waits until all CTAs have arrived, normally a microsecond, and leaves; should the CTAs not have
-// landed one per SM (other work on the GPU), queues are left over then and the waiting CTAs draw
-// them from [1], so every queue runs exactly once.  The last CTA to leave zeroes the state.
+// SM-window launches (write-dominated schedules without flags): see window_claim in pl_device.cuh.
 __device__ __forceinline__ int claim_queue(const ExecParams& P) {
-  uint32_t sm;
-  asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
-  const bool active = sm >= 160u || ((P.sm_mask[sm >> 5] >> (sm & 31u)) & 1u);
-  const uint32_t total = gridDim.x;
-  const unsigned long long mine = (1ull << 32) | (active ? 1ull : 0ull);
-  const unsigned long long old = atomicAdd(P.sm_state, mine);
-  if (active) {
-    const uint32_t taken = (uint32_t)old;
-    return taken < P.n_queues ? (int)taken : -1;  // a surplus CTA on an active SM has nothing to do
-  }
-  // idle SM: wait for the count of arrivals to be complete (bounded), then look for leftovers
-  unsigned long long now = old + mine;
-  const unsigned long long t0 = globaltimer_ns();
-  for (uint32_t spins = 1; (uint32_t)(now >> 32) < total; ++spins) {
-    now = *reinterpret_cast<volatile unsigned long long*>(P.sm_state);
-    if ((spins & 63u) == 0 && globaltimer_ns() - t0 > 2ull * P.timeout_ns + 1000000ull) break;
-  }
-  const uint32_t by_active = (uint32_t)now;
-  if ((uint32_t)(now >> 32) < total) {
-    // CTAs of this launch are still missing after the time limit: queues may go unclaimed, say so
-    record_timeout(P, (int)blockIdx.x, 0xFFFFFFFFu, 0xFFFFFFFFu, total, (uint32_t)(now >> 32));
-    return -1;
-  }
-  if (by_active >= P.n_queues) return -1;
-  const uint32_t extra = atomicAdd(reinterpret_cast<unsigned int*>(P.sm_state + 1), 1u);
-  return by_active + extra < P.n_queues ? (int)(by_active + extra) : -1;
+  bool timed_out = false;
+  const int q = window_claim(P.sm_state, P.sm_mask, P.n_queues, 2ull * P.timeout_ns + 1000000ull, &timed_out);
+  // CTAs of this launch still missing after the time limit: queues may go unclaimed, say so
+  if (timed_out) record_timeout(P, (int)blockIdx.x, 0xFFFFFFFFu, 0xFFFFFFFFu, gridDim.x, 0);
+  return q;
 }
-// A CTA of an SM-window launch leaves: the last one puts the state back to zero.
-__device__ __forceinline__ void leave_window(const ExecParams& P) {
-  __threadfence();
-  const unsigned int left = atomicAdd(reinterpret_cast<unsigned int*>(P.sm_state + 2), 1u);
-  if (left == gridDim.x - 1u) {
-    P.sm_state[0] = 0ull;
-    P.sm_state[1] = 0ull;
-    P.sm_state[2] = 0ull;
-    __threadfence();
-  }
-}
+__device__ __forceinline__ void leave_window(const ExecParams& P) { window_leave(P.sm_state); }
 
 template <int DT, int CW, bool HOOK = false, bool DBUF = false>
 __global__ void __launch_bounds__(32 * (kProducers + 1 + CW), 1) pl_exec_tma_kernel(const __grid_constant__ ExecParams P) {

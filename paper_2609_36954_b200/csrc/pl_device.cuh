@@ -248,6 +248,59 @@ __device__ __forceinline__ void store_final_unit(const ExecParams& P, const Acc<
   }
 }
 
+// ---- SM-window launches -------------------------------------------------------------------
+// One CTA is launched per SM; a CTA whose SM lies in the idle window (bit clear in `mask`, one bit
+// per SM id, 160 bits) sits the launch out, every other CTA claims the next of n_slots work slots
+// (op queues of a schedule, strides of a stream).  How fast a 1 read : R writes stream runs depends
+// on WHICH SMs take part (see pl_comm_tune), and a plain launch of fewer CTAs than SMs leaves that
+// choice to the hardware.
+// State (three 64-bit words, zero between launches): [0] arrivals << 32 | slots claimed by CTAs on
+// active SMs, [1] slots claimed afterwards, [2] CTAs that have left.  Every CTA adds itself to [0]
+// with ONE atomic (no compare-and-swap loop: 148 CTAs contending for one word would take tens of
+// microseconds).  A CTA on an active SM takes the slot it drew.  A CTA on an idle SM waits until
+// all CTAs have arrived, normally a microsecond, and leaves; should the CTAs not have landed one
+// per SM (other work on the GPU), slots are left over then and the waiting CTAs draw them from
+// [1], so every slot is taken exactly once.  The last CTA to leave zeroes the state.
+// Returns the slot, or -1 (nothing to do).  *timed_out: arrivals still incomplete after limit_ns.
+__device__ __forceinline__ int window_claim(unsigned long long* state, const uint32_t* mask, uint32_t n_slots,
+                                            unsigned long long limit_ns, bool* timed_out) {
+  uint32_t sm;
+  asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+  const bool active = sm >= 160u || ((mask[sm >> 5] >> (sm & 31u)) & 1u);
+  const uint32_t total = gridDim.x;
+  const unsigned long long mine = (1ull << 32) | (active ? 1ull : 0ull);
+  const unsigned long long old = atomicAdd(state, mine);
+  if (active) {
+    const uint32_t taken = (uint32_t)old;
+    return taken < n_slots ? (int)taken : -1;  // a surplus CTA on an active SM has nothing to do
+  }
+  unsigned long long now = old + mine;
+  const unsigned long long t0 = globaltimer_ns();
+  for (uint32_t spins = 1; (uint32_t)(now >> 32) < total; ++spins) {
+    now = *reinterpret_cast<volatile unsigned long long*>(state);
+    if ((spins & 63u) == 0 && globaltimer_ns() - t0 > limit_ns) break;
+  }
+  if ((uint32_t)(now >> 32) < total) {
+    *timed_out = true;
+    return -1;
+  }
+  const uint32_t by_active = (uint32_t)now;
+  if (by_active >= n_slots) return -1;
+  const uint32_t extra = atomicAdd(reinterpret_cast<unsigned int*>(state + 1), 1u);
+  return by_active + extra < n_slots ? (int)(by_active + extra) : -1;
+}
+// A CTA of an SM-window launch leaves: the last one puts the state back to zero.
+__device__ __forceinline__ void window_leave(unsigned long long* state) {
+  __threadfence();
+  const unsigned int left = atomicAdd(reinterpret_cast<unsigned int*>(state + 2), 1u);
+  if (left == gridDim.x - 1u) {
+    state[0] = 0ull;
+    state[1] = 0ull;
+    state[2] = 0ull;
+    __threadfence();
+  }
+}
+
 // Record a timeout (first writer wins) and raise the abort word.
 static __device__ __noinline__ void record_timeout_at(int* status, int queue, uint32_t topo, uint32_t flag,
                                                       unsigned long long expected, unsigned long long observed) {

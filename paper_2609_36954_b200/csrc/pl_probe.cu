@@ -14,6 +14,8 @@
 #include <cstdint>
 
 #include "pl_api_internal.h"
+#include "pl_device.cuh"
+#include "pl_internal.h"
 #include "pl_ptx.cuh"
 #include "purlin.h"
 
@@ -45,8 +47,12 @@ __device__ __forceinline__ bool wait_full(uint64_t* bar, uint32_t parity) {
 // kind 0: read (tiles are loaded and dropped), 1: write (a fixed pattern tile is stored), 2: copy,
 // 3: one read to eight writes (every tile is stored to the same offset of 8 consecutive regions of
 // dst, each as long as src): the mix of the all-gather and of the MoE dispatch
+// idle_count > 0: an SM-window launch (one CTA per SM; the CTAs on SMs idle_first .. idle_first +
+// idle_count - 1 sit out, the others claim the n_active strides of the stream): see window_claim.
+__device__ unsigned long long g_probe_window[3];
+
 __global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src, char* dst, unsigned long long n_tiles,
-                                                      int* status) {
+                                                      int* status, int idle_first, int idle_count, int n_active) {
   extern __shared__ __align__(128) unsigned char smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);
   unsigned char* tiles = smem + 128;
@@ -62,8 +68,30 @@ __global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src,
   }
   __syncwarp();
   if (lane != 0) return;
-  const unsigned long long c = blockIdx.x, G = gridDim.x;
-  if (c >= n_tiles) return;
+  unsigned long long c = blockIdx.x, G = gridDim.x;
+  if (idle_count > 0) {
+    uint32_t mask[5];
+    for (int w = 0; w < 5; ++w) {
+      mask[w] = 0xFFFFFFFFu;
+      for (int b = 0; b < 32; ++b) {
+        const int sm = w * 32 + b;
+        if (sm >= idle_first && sm < idle_first + idle_count) mask[w] &= ~(1u << b);
+      }
+    }
+    bool timed_out = false;
+    const int slot = dev::window_claim(g_probe_window, mask, (uint32_t)n_active, kLimitNs, &timed_out);
+    if (timed_out && status) *status = PL_ERR_TIMEOUT;
+    if (slot < 0) {
+      dev::window_leave(g_probe_window);
+      return;
+    }
+    c = (unsigned long long)slot;
+    G = (unsigned long long)n_active;
+  }
+  if (c >= n_tiles) {
+    if (idle_count > 0) dev::window_leave(g_probe_window);
+    return;
+  }
   const unsigned long long n_my = (n_tiles - c + G - 1) / G;
   auto tile_off = [&](unsigned long long n) { return (c + n * G) * (unsigned long long)kTile; };
   unsigned long long issued = 0;  // loads issued so far (tiles 0 .. issued-1 of this CTA)
@@ -107,6 +135,7 @@ __global__ void __launch_bounds__(32) pl_probe_kernel(int kind, const char* src,
       for (uint32_t tries = 0; tries < (1u << 20) && !ptx::mbar_try_wait(full + s, parity); ++tries) {}
     }
   }
+  if (idle_count > 0) dev::window_leave(g_probe_window);
 }
 
 }  // namespace
@@ -131,11 +160,16 @@ extern "C" pl_status_t pl_probe_hbm(int kind, const void* src, void* dst, size_t
   }
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   if (status && cudaMemsetAsync(status, 0, sizeof(int32_t), cs) != cudaSuccess) { cudaGetLastError(); return PL_ERR_CUDA; }
-  // The write-dominated stream is fastest with about 8/9 of the SMs writing (132 of 148: 6.15 TB/s
-  // against 5.7 TB/s with one CTA on every SM); the other streams want them all.
-  const int grid = kind == 3 ? ((sms * 8 / 9 + 3) & ~3) : sms;
-  pl_probe_kernel<<<grid, 32, kSmem, cs>>>(kind, static_cast<const char*>(src), static_cast<char*>(dst),
-                                          (unsigned long long)(bytes / kTile), reinterpret_cast<int*>(status));
+  // The write-dominated stream is fastest with about 8/9 of the SMs writing (132 of 148: 6.15-6.35 TB/s
+  // against 5.7 TB/s with one CTA on every SM), and with the right ones sitting out: SMs 8-23 were a
+  // good window on every B200 tried, the SMs a plain launch of 132 CTAs leaves idle only on some
+  // (5.4 TB/s on the others).  The other streams want all SMs.  (Concurrent kind-3 probes on
+  // different streams would share the window's claim words: the probe is a one-at-a-time tool.)
+  const int active = kind == 3 ? ((sms * 8 / 9 + 3) & ~3) : sms;
+  const bool window = kind == 3 && sms == 148 && active < sms;
+  pl_probe_kernel<<<window ? sms : active, 32, kSmem, cs>>>(kind, static_cast<const char*>(src), static_cast<char*>(dst),
+                                                             (unsigned long long)(bytes / kTile), reinterpret_cast<int*>(status),
+                                                             8, window ? sms - active : 0, active);
   if (cudaGetLastError() != cudaSuccess) return PL_ERR_CUDA;
   g_launches.fetch_add(1);
   return PL_OK;
