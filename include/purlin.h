@@ -356,8 +356,11 @@ pl_status_t pl_comm_destroy(pl_comm_t comm);
  * (plain launches: 101 us at best on some, 107 us on others).  Candidates: plain launches of
  * every multiple of R between 3/4 of the resident CTAs and all of them, and the same grids
  * launched as one CTA per SM with the idle SMs as a window starting at SM 0, 8, 16 or 64; each
- * runs an all-gather of 64 MiB (2 + 6 launches) on `stream`, on buffers this call allocates and
- * frees ((R + 1) x 64 MiB).  Synchronises: a call for set-up time, not for the hot path.  Nothing
+ * runs an all-gather of 64 MiB behind the reduce-scatter that produces its input, both with
+ * PL_OPT_INPUTS_LAST_USE (2 + 6 pairs of launches): where an all-gather usually runs, its input
+ * is in L2 and its DRAM traffic almost purely writes, and the fastest candidate is not always the
+ * one that is fastest alone.  Runs on `stream`, on buffers this call allocates and frees
+ * ((2 R + 1) x 64 MiB).  Synchronises: a call for set-up time, not for the hot path.  Nothing
  * in the paper corresponds to it.  The outputs (each may be NULL) receive the chosen grid and
  * window (count 0: a plain launch).
  * Errors: PL_ERR_UNSUPPORTED (planner communicator), PL_ERR_OOM, PL_ERR_CUDA, PL_ERR_INVALID_ARG
