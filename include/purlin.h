@@ -185,7 +185,9 @@ typedef struct {
                          /* launch, or the window pl_comm_tune measured / the default one for    */
                          /* pushed all-gathers).  Which SMs take part decides how fast a write-  */
                          /* dominated stream runs (pl_comm_tune).  PL_ERR_UNSUPPORTED where it   */
-                         /* does not apply.  No counterpart in the paper.                        */
+                         /* does not apply (flags, register or packet datapath, more than one    */
+                         /* CTA per SM, PL_OPT_OVERLAP_LAUNCH: the claim words serve one launch  */
+                         /* at a time).  No counterpart in the paper.                            */
 } pl_sched_opts_t;
 /* The processing phase as a small family (Sec. 3.3: the phase between the last addition and the
  * store is configurable while the sum sits in registers).  With s = out_scale (1 if unset):

@@ -458,13 +458,16 @@ pl_status_t build_common(pl_comm_t comm, BuildRequest rq, const pl_sched_opts_t*
   for (const HostOp& op : S->L.ops)
     if (op.kind == PL_OP_COPY && op.bcast) S->bcast_copies = true;
   // A window of idle SMs needs: the bulk-copy datapath with one CTA per SM, no flags (a queue
-  // may be claimed late, so no queue may wait for another), one staging buffer, at most 160 SMs.
+  // may be claimed late, so no queue may wait for another), one staging buffer, at most 160 SMs,
+  // and ordinary launches: the claim words serve one launch at a time, and only a launch that
+  // waits for everything in front of it is sure not to meet its own predecessor still running.
   if (S->pol.idle_count > 0) {
-    const bool fits = pol.datapath == PL_DP_TMA && !comm->planner && S->L.n_flags == 0 && !S->stage_ahead && comm->sm_count <= 160 &&
+    const bool fits = pol.datapath == PL_DP_TMA && !comm->planner && S->L.n_flags == 0 && !S->stage_ahead && !S->overlap_launch &&
+                      comm->sm_count <= 160 &&
                       exec_tma_max_ctas_per_sm(comm->dtype, pol.stages, pol.stage_bytes) == 1 &&
                       S->pol.n_ctas + S->pol.idle_count == comm->sm_count;
     if (!fits && idle_asked) {
-      comm->last_error = "a window of idle SMs needs the bulk-copy datapath with one CTA per SM and a schedule without flags";
+      comm->last_error = "a window of idle SMs needs the bulk-copy datapath with one CTA per SM, a schedule without flags and no PL_OPT_OVERLAP_LAUNCH";
       delete S;
       return PL_ERR_UNSUPPORTED;
     }

@@ -178,3 +178,39 @@ def test_sm_window_is_rejected_where_it_does_not_apply():
         assert e.value.status == B.PL_ERR_INVALID_ARG
     finally:
         ses.close()
+
+
+def test_overlapped_launches_never_use_an_sm_window():
+    """The claim words of a window launch serve one launch at a time, so a schedule built for
+    overlapped launches is a plain launch whatever the tuner found, an explicit window with it is
+    refused, and back-to-back overlapped executes of reduce-scatter and all-gather stay correct."""
+    R = 8
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n = R * (2 << 20)
+    ses = Session(R, "bf16")
+    try:
+        with pytest.raises(B.PurlinError) as e:
+            ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 20, datapath=B.PL_DP_TMA, flags=B.PL_OPT_OVERLAP_LAUNCH,
+                      idle_sm_first=8, idle_sm_count=sms - 128)
+        assert e.value.status == B.PL_ERR_UNSUPPORTED
+        ag = ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 20, datapath=B.PL_DP_TMA, flags=B.PL_OPT_OVERLAP_LAUNCH)
+        assert B.pl_schedule_info(ag).idle_sm_count == 0
+        rs = ses.build(B.PL_REDUCE_SCATTER, B.PL_ALGO_DIRECT, n, 1 << 20, datapath=B.PL_DP_TMA, flags=B.PL_OPT_OVERLAP_LAUNCH)
+        ag_w = ses.build(B.PL_ALLGATHER, B.PL_ALGO_DIRECT, n // R, 1 << 20, datapath=B.PL_DP_TMA)   # default: a window launch
+        x = gen.rank_inputs(R, n, "bf16", seed=31)
+        irs, iag = B.pl_schedule_info(rs), B.pl_schedule_info(ag_w)
+        d_in = [to_dev(a) for a in x]
+        d_mid = [poison(irs.out_bytes[r]) for r in range(R)]
+        d_out = [poison(iag.out_bytes[r]) for r in range(R)]
+        b_rs = B.make_bufs([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_mid], [int(irs.in_bytes[r]) for r in range(R)], [int(irs.out_bytes[r]) for r in range(R)])
+        b_ag = B.make_bufs([t.data_ptr() for t in d_mid], [t.data_ptr() for t in d_out], [int(iag.in_bytes[r]) for r in range(R)], [int(iag.out_bytes[r]) for r in range(R)])
+        for _ in range(20):                        # overlapped reduce-scatter in front of a window-launched all-gather
+            B.pl_execute(rs, b_rs, stream_handle())
+            B.pl_execute(ag_w, b_ag, stream_handle())
+        torch.cuda.synchronize()
+        assert B.pl_comm_status(ses.comm).code == B.PL_OK
+        ref = oracle.allreduce(x, "bf16")
+        for r in (0, 5):
+            check_float(gen.bf16_bits_to_f64(d_out[r][: int(iag.out_bytes[r])].cpu().numpy().view(np.uint16)), ref[r], "bf16")
+    finally:
+        ses.close()
