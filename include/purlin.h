@@ -359,7 +359,8 @@ pl_status_t pl_comm_destroy(pl_comm_t comm);
  * every multiple of R between 3/4 of the resident CTAs and all of them, and the same grids
  * launched as one CTA per SM with the idle SMs as a window starting at SM 0, 8, 16 or 64; each
  * runs an all-gather of 64 MiB behind the reduce-scatter that produces its input, both with
- * PL_OPT_INPUTS_LAST_USE (2 + 6 pairs of launches): where an all-gather usually runs, its input
+ * PL_OPT_INPUTS_LAST_USE (2 + 10 pairs of launches; a candidate replaces the pick only if it is
+ * 0.5 % faster, so equal ones resolve to the larger grid and the plain launch): where an all-gather usually runs, its input
  * is in L2 and its DRAM traffic almost purely writes, and the fastest candidate is not always the
  * one that is fastest alone.  Runs on `stream`, on buffers this call allocates and frees
  * ((2 R + 1) x 64 MiB).  Synchronises: a call for set-up time, not for the hot path.  Nothing

@@ -733,7 +733,7 @@ pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out, i
     bool ok = true;
     auto pair = [&]() { return (!rs || pl_execute(rs, &rs_bufs, stream) == PL_OK) && pl_execute(s, &bufs, stream) == PL_OK; };
     for (int i = 0; i < 2 && ok; ++i) ok = pair();
-    const int reps = 6;
+    const int reps = 10;
     ok = ok && cudaEventRecord(e0, cs) == cudaSuccess;
     for (int i = 0; i < reps && ok; ++i) ok = pair();
     ok = ok && cudaEventRecord(e1, cs) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess;
@@ -745,10 +745,10 @@ pl_status_t pl_comm_tune(pl_comm_t comm, void* stream, int32_t* push_ctas_out, i
       result = PL_ERR_CUDA;
       break;
     }
-    // at equal speed the plain launch is kept (a window launch puts an atomic in front of every
-    // CTA's first load: the measurement contains it, the margin keeps noise from deciding)
-    const float handicap = cd.idle_count > 0 ? 1.003f : 1.0f;
-    if (best.n_ctas == 0 || ms * handicap < best_ms * (best.idle_count > 0 ? 1.003f : 1.0f)) {
+    // Candidates run from the largest grid down, plain launch first: a later one replaces the
+    // pick only if it is faster by more than the noise of the measurement (0.5 %), so that equal
+    // candidates resolve to the larger grid and to the plain launch.
+    if (best.n_ctas == 0 || ms < best_ms * 0.995f) {
       best = cd;
       best_ms = ms;
     }
