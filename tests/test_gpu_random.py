@@ -283,3 +283,52 @@ def test_random_hook_stage_ahead_and_packet_cases_match_the_oracle(seed):
                             check_float(got.view(np.float32).astype(np.float64), ref[r], "f32")
         finally:
             ses.close()
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_sm_window_and_l2_option_cases_match_the_oracle(seed):
+    """Flag-free schedules of the bulk-copy datapath (direct reduce-scatter, all-gather, all-to-all)
+    under random idle-SM windows and L2 options, odd rank counts and ragged sizes included: the
+    grid must be every SM outside the window and a multiple of R."""
+    import torch
+    rng = np.random.default_rng(5000 + seed)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    R = int(rng.choice([2, 3, 4, 5, 7, 8, 12, 16]))
+    dtype = str(rng.choice(["i32", "bf16", "f32"]))
+    coll = int(rng.choice([B.PL_REDUCE_SCATTER, B.PL_ALLGATHER, B.PL_ALLTOALL]))
+    es = B.DTYPE_SIZE[DT[dtype]]
+    vecs = int(rng.choice([17, 257, 1031, 4099, 20011]))
+    n = R * vecs * (16 // es)
+    count = n // R if coll == B.PL_ALLGATHER else n
+    # a window whose complement is a multiple of R
+    active = int(rng.integers(max(1, (sms * 3 // 4) // R), sms // R + 1)) * R
+    idle = sms - active
+    flags = int(rng.choice([0, B.PL_OPT_INPUTS_LAST_USE, B.PL_OPT_NO_L2_HINTS]))
+    kw = dict(datapath=B.PL_DP_TMA, flags=flags, slice_bytes=16 * int(rng.choice([0, 64, 1024])))
+    if idle > 0:
+        kw.update(idle_sm_first=int(rng.integers(0, sms - idle + 1)), idle_sm_count=idle)
+    s = Session(R, dtype)
+    try:
+        sched = s.build(coll, B.PL_ALGO_DIRECT, count, 16 * int(rng.choice([64, 512, 1 << 20])), **kw)
+        info = B.pl_schedule_info(sched)
+        if idle > 0:
+            assert (info.grid, info.idle_sm_count) == (active, idle)
+        x = gen.rank_inputs(R, n, dtype, seed=seed)
+        if coll == B.PL_ALLGATHER:
+            x = [a[:count].copy() for a in x]
+        outs, _ = s.execute(sched, x, repeats=3)
+        if coll == B.PL_REDUCE_SCATTER:
+            ref = oracle.reduce_scatter(x, dtype)
+        elif coll == B.PL_ALLGATHER:
+            ref = oracle.allgather(x)
+        else:
+            ref = oracle.alltoall(x)
+        for r in range(R):
+            if coll != B.PL_REDUCE_SCATTER or dtype == "i32":
+                assert np.array_equal(outs[r], np.ascontiguousarray(ref[r]).view(np.uint8).reshape(-1)), (seed, r)
+            elif dtype == "bf16":
+                check_float(gen.bf16_bits_to_f64(outs[r].view(np.uint16)), ref[r], dtype)
+            else:
+                check_float(outs[r].view(np.float32).astype(np.float64), ref[r], dtype)
+    finally:
+        s.close()
