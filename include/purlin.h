@@ -628,7 +628,9 @@ pl_status_t pl_moe_plan_read_dedup(pl_moe_plan_t plan, int32_t* pos, int64_t* co
  * one CTA per SM): kind 0 reads src and drops the data, kind 1 fills dst with a fixed pattern
  * (32-bit word j of every 32 KiB tile = j * 2654435761 mod 2^32), kind 2 copies src to dst,
  * kind 3 writes every tile of src to the same offset of 8 consecutive regions of dst (one read
- * to eight writes).  Timed with CUDA events by the caller it gives the pure-read, pure-write,
+ * to eight writes; on a 148-SM part 132 CTAs work and SMs 8-23 sit out, the kind of SM window the
+ * write-dominated schedules use: kind-3 probes must not run concurrently with one another, they
+ * share the window's claim words).  Timed with CUDA events by the caller it gives the pure-read, pure-write,
  * copy and 1:8 bandwidth that bound the read-dominated (reduce-scatter, MoE combine), balanced
  * (all-to-all) and write-dominated (all-gather, MoE dispatch) collectives on this GPU.
  *   src, dst  DEVICE pointers, 16-byte aligned, `bytes` long (src unused for kind 1, dst for
