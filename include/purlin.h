@@ -510,6 +510,14 @@ pl_status_t pl_execute_host(pl_schedule_t s, const pl_bufs_t* host, const pl_buf
  * errors as pl_execute_host. */
 pl_status_t pl_execute_host_async(pl_schedule_t s, const pl_bufs_t* host, const pl_bufs_t* dev,
                                   void* stream);
+/* Bytes the host entry points of this communicator have copied so far, host to device and
+ * device to host (either pointer may be NULL).  pl_execute_host_async does not upload an input
+ * that is already on the device: when a call's host input buffer is exactly the host output
+ * buffer of the immediately preceding call, that call's download is still in flight, and the
+ * device input buffer is the device buffer that download reads (a reduce-scatter's result handed
+ * to an all-gather through a host buffer), the bytes are the ones the previous schedule left
+ * there, and neither copy nor wait is needed. */
+pl_status_t pl_comm_host_stats(pl_comm_t comm, uint64_t* h2d_bytes, uint64_t* d2h_bytes);
 /* Make `stream` wait (asynchronously) for all downloads of earlier pl_execute_host_async calls. */
 pl_status_t pl_comm_host_fence(pl_comm_t comm, void* stream);
 /* Block the calling thread until all downloads of earlier pl_execute_host_async calls are done. */

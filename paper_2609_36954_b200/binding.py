@@ -101,7 +101,7 @@ EXPORTS = [
     "pl_schedule_build", "pl_schedule_build_v", "pl_schedule_build_layers", "pl_schedule_build_rooted", "pl_schedule_info",
     "pl_schedule_dump", "pl_schedule_validate", "pl_schedule_debug_break_wait", "pl_schedule_debug_drop_wait",
     "pl_schedule_trace_read", "pl_schedule_destroy",
-    "pl_execute", "pl_execute_host", "pl_execute_host_async", "pl_comm_host_fence", "pl_comm_host_sync", "pl_comm_tune",
+    "pl_execute", "pl_execute_host", "pl_execute_host_async", "pl_comm_host_fence", "pl_comm_host_sync", "pl_comm_host_stats", "pl_comm_tune",
     "pl_moe_plan_create", "pl_moe_plan_destroy", "pl_moe_dispatch", "pl_moe_combine", "pl_moe_plan_read",
     "pl_moe_dispatch_dedup", "pl_moe_combine_dedup", "pl_moe_plan_read_dedup", "pl_moe_combine_logits",
     "pl_status_string", "pl_launch_count", "pl_reduce_scatter_ring_static",
@@ -150,6 +150,7 @@ def load():
         "pl_execute_host_async": [vp, P(pl_bufs_t), P(pl_bufs_t), vp],
         "pl_comm_host_fence": [vp, vp],
         "pl_comm_host_sync": [vp],
+        "pl_comm_host_stats": [vp, P(C.c_uint64), P(C.c_uint64)],
         "pl_comm_tune": [vp, vp, P(C.c_int32), P(C.c_int32), P(C.c_int32)],
         "pl_moe_plan_create": [vp, i32, i32, i32, i32, sz, P(vp)],
         "pl_moe_plan_destroy": [vp],
@@ -348,6 +349,13 @@ def pl_comm_tune(comm, stream=0, full=False):
     g, f, n = C.c_int32(0), C.c_int32(0), C.c_int32(0)
     _check(load().pl_comm_tune(comm, stream, C.byref(g), C.byref(f), C.byref(n)), "pl_comm_tune")
     return (int(g.value), int(f.value), int(n.value)) if full else int(g.value)
+
+
+def pl_comm_host_stats(comm):
+    """(bytes copied host to device, bytes copied device to host) by the host entry points so far."""
+    a, b = C.c_uint64(0), C.c_uint64(0)
+    _check(load().pl_comm_host_stats(comm, C.byref(a), C.byref(b)), "pl_comm_host_stats")
+    return int(a.value), int(b.value)
 
 
 def pl_comm_host_sync(comm):

@@ -539,16 +539,22 @@ pl_status_t check_host_bufs(pl_schedule_s* s, const pl_bufs_t* host, const pl_bu
 }
 
 // host -> device copies of inputs and second operands (upload) or device -> host copies of outputs.
-bool copy_all(pl_schedule_s* s, int R, const pl_bufs_t* host, const pl_bufs_t* dev, bool upload, cudaStream_t on) {
+// skip_in: bit r set = rank r's input is already in dev->in[r] (see pl_execute_host_async).
+bool copy_all(pl_schedule_s* s, int R, const pl_bufs_t* host, const pl_bufs_t* dev, bool upload, cudaStream_t on, uint32_t skip_in = 0) {
   bool ok = true;
   for (int r = 0; r < R && ok; ++r) {
     if (upload) {
-      if (s->info.in_bytes[r])
+      if (s->info.in_bytes[r] && !((skip_in >> r) & 1u)) {
         ok = cudaMemcpyAsync(const_cast<void*>(dev->in[r]), host->in[r], s->info.in_bytes[r], cudaMemcpyHostToDevice, on) == cudaSuccess;
-      if (ok && s->info.aux_bytes[r])
+        s->comm->host_h2d_bytes += s->info.in_bytes[r];
+      }
+      if (ok && s->info.aux_bytes[r]) {
         ok = cudaMemcpyAsync(const_cast<void*>(dev->aux[r]), host->aux[r], s->info.aux_bytes[r], cudaMemcpyHostToDevice, on) == cudaSuccess;
+        s->comm->host_h2d_bytes += s->info.aux_bytes[r];
+      }
     } else if (s->info.out_bytes[r]) {
       ok = cudaMemcpyAsync(host->out[r], dev->out[r], s->info.out_bytes[r], cudaMemcpyDeviceToHost, on) == cudaSuccess;
+      s->comm->host_d2h_bytes += s->info.out_bytes[r];
     }
   }
   if (!ok) cudaGetLastError();
@@ -1134,14 +1140,37 @@ pl_status_t pl_execute_host_async(pl_schedule_t s, const pl_bufs_t* host, const 
   // Hazards with downloads still in flight: an upload must not read a host range, nor overwrite a
   // device range, that a download has yet to finish with; the schedule must not overwrite device
   // outputs that a download still reads.
+  // Forwarding: an input whose host buffer is exactly what the previous call's download is still
+  // writing, and whose device buffer is exactly what that download reads, is already where the
+  // upload would put it (the previous schedule wrote it there): no upload, and nothing to wait
+  // for (a reduce-scatter's result handed to an all-gather through a host buffer).  Only the
+  // immediately preceding call is looked at, and only while its download is in flight: once it
+  // has completed the caller may have rewritten the host buffer.
+  uint32_t fwd = 0;
+  if (comm->last_download >= 0 && comm->host_stream_last == stream) {  // same stream: the previous schedule is ordered in front of this one
+    pl_comm_s::Download& d = comm->downloads[comm->last_download];
+    if (d.live && cudaEventQuery(static_cast<cudaEvent_t>(d.done)) != cudaSuccess && d.host_out.size() == d.dev_out.size()) {
+      for (int r = 0; r < R; ++r) {
+        const size_t n = s->info.in_bytes[r];
+        if (!n) continue;
+        for (size_t k = 0; k < d.host_out.size(); ++k)
+          if (d.host_out[k].lo == static_cast<const char*>(host->in[r]) && (size_t)(d.host_out[k].hi - d.host_out[k].lo) == n &&
+              d.dev_out[k].lo == static_cast<const char*>(dev->in[r]) && (size_t)(d.dev_out[k].hi - d.dev_out[k].lo) == n)
+            fwd |= 1u << r;
+      }
+    }
+    cudaGetLastError();  // cudaErrorNotReady is not an error here
+  }
   std::vector<pl_comm_s::Range> h_in, d_in, d_out, h_out;
   for (int r = 0; r < R; ++r) {
     auto add = [](std::vector<pl_comm_s::Range>& v, const void* p, size_t n) {
       if (p && n) v.push_back({static_cast<const char*>(p), static_cast<const char*>(p) + n});
     };
-    add(h_in, host->in[r], s->info.in_bytes[r]);
+    if (!((fwd >> r) & 1u)) {
+      add(h_in, host->in[r], s->info.in_bytes[r]);
+      add(d_in, dev->in[r], s->info.in_bytes[r]);
+    }
     add(h_in, host->aux[r], s->info.aux_bytes[r]);
-    add(d_in, dev->in[r], s->info.in_bytes[r]);
     add(d_in, dev->aux[r], s->info.aux_bytes[r]);
     add(d_out, dev->out[r], s->info.out_bytes[r]);
     add(h_out, host->out[r], s->info.out_bytes[r]);
@@ -1158,7 +1187,7 @@ pl_status_t pl_execute_host_async(pl_schedule_t s, const pl_bufs_t* host, const 
   }
   if (!ok) { cudaGetLastError(); return PL_ERR_CUDA; }
 
-  if (!copy_all(s, R, host, dev, /*upload=*/true, up)) return PL_ERR_CUDA;
+  if (!copy_all(s, R, host, dev, /*upload=*/true, up, fwd)) return PL_ERR_CUDA;
   ok = cudaEventRecord(static_cast<cudaEvent_t>(comm->ev_up[slot]), up) == cudaSuccess;
   wait(cs, comm->ev_up[slot]);
   if (!ok) { cudaGetLastError(); return PL_ERR_CUDA; }
@@ -1175,6 +1204,14 @@ pl_status_t pl_execute_host_async(pl_schedule_t s, const pl_bufs_t* host, const 
   mine.dev_out = std::move(d_out);
   mine.live = true;
   comm->last_download = slot;
+  return PL_OK;
+}
+
+pl_status_t pl_comm_host_stats(pl_comm_t comm, uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
+  if (!comm) return PL_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> host_guard(comm->host_mu);
+  if (h2d_bytes) *h2d_bytes = comm->host_h2d_bytes;
+  if (d2h_bytes) *d2h_bytes = comm->host_d2h_bytes;
   return PL_OK;
 }
 

@@ -43,6 +43,7 @@ struct pl_comm_s {
   uint64_t host_calls = 0;           // async host executes so far
   void* host_stream_last = nullptr;  // the caller's stream of the previous async host execute
   int last_download = -1;            // slot of the most recent download
+  uint64_t host_h2d_bytes = 0, host_d2h_bytes = 0;  // bytes the host entry points have copied so far
   std::mutex host_mu;                // serialises the host-pipeline entry points
 };
 

@@ -50,6 +50,12 @@ def test_reduce_scatter_all_gather_steps_chained_through_host_buffers():
             B.pl_execute_host_async(ag, make(h_mid, h_out[k], iag), b_ag, stream_handle())
         B.pl_comm_host_sync(comm)
         assert B.pl_comm_status(comm).code == B.PL_OK
+        # the library's own count of what it copied: every output is downloaded; the all-gather's
+        # input is not uploaded again while the reduce-scatter's download of it is in flight
+        h2d, d2h = B.pl_comm_host_stats(comm)
+        full_up = steps * (sum(int(irs.in_bytes[r]) for r in range(R)) + sum(int(iag.in_bytes[r]) for r in range(R)))
+        assert d2h == steps * (sum(int(irs.out_bytes[r]) for r in range(R)) + sum(int(iag.out_bytes[r]) for r in range(R)))
+        assert steps * sum(int(irs.in_bytes[r]) for r in range(R)) <= h2d <= full_up
         for k in range(steps):
             ref = oracle.allreduce(xs[k], "bf16")
             for r in (0, 3, 7):
