@@ -471,6 +471,10 @@ def measure_all_configs(peak):
     for name, kw in (("plain", {}), ("scale", dict(out_scale=0.125)), ("scale_residual", dict(out_scale=0.125, hook=B.PL_HOOK_RESIDUAL)),
                      ("f32_out", dict(hook=B.PL_HOOK_F32_OUT))):
         out["processing_phase"][name] = entry(b.collective("hook", 8, B.PL_BF16, B.PL_REDUCE_SCATTER, "direct", 32 * MIB, MIB, **kw))
+    # the same phase on the fused all-reduce, whose results go to all 8 outputs
+    for name, kw in (("fused_allreduce_plain", {}), ("fused_allreduce_scale_residual", dict(out_scale=0.125, hook=B.PL_HOOK_RESIDUAL)),
+                     ("fused_allreduce_f32_out", dict(hook=B.PL_HOOK_F32_OUT))):
+        out["processing_phase"][name] = entry(b.collective("hook", 8, B.PL_BF16, B.PL_ALLREDUCE, "fused", 32 * MIB, MIB, iters=10, **kw))
     # C4: MoE dispatch / combine at the full shape, both routings
     out["C4"] = {}
     for name, ident in (("permuted", False), ("identity", True)):

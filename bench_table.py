@@ -71,7 +71,8 @@ def main(path):
         for a, ee in e.items():
             print(collective_rows(f"staged {k} {a}", ee))
     for k, e in c.get("processing_phase", {}).items():
-        print(collective_rows(f"reduce-scatter 64 MiB, processing phase: {k}", e))
+        what = "fused all-reduce" if k.startswith("fused_allreduce_") else "reduce-scatter"
+        print(collective_rows(f"{what} 64 MiB, processing phase: {k.replace('fused_allreduce_', '')}", e))
     print("\n" + row(["C4 routing", "dispatch us", "of measured", "of 8 TB/s", "of 1:8 ceiling", "combine us", "of measured", "of 8 TB/s", "of read ceiling"]))
     print(row(["---"] * 9))
     for k, e in c["C4"].items():
