@@ -794,7 +794,11 @@ Policy default_policy(const BuildRequest& rq, int max_resident_ctas) {
   if (p.datapath == PL_DP_AUTO) p.datapath = stream ? PL_DP_TMA : PL_DP_LDST;
   if (p.threads <= 0) p.threads = 512;
   if (p.stages <= 0) p.stages = 4;
-  if (p.stage_bytes == 0) p.stage_bytes = 49152;
+  // 48 KiB slots hold a full stage of 384 units of 8 sources; with a second operand per rank its
+  // tile rides in the slot as a ninth one, and 54 KiB keep the stage at 384 units (the general
+  // consumer path costs about a microsecond per stage whatever its size: reduce-scatter with
+  // residual 119 -> 111 us at 8 x 64 MiB; not the ring, whose stages hold partial sums and lose 2 %)
+  if (p.stage_bytes == 0) p.stage_bytes = ((rq.hook & PL_HOOK_RESIDUAL) && rq.algo != PL_ALGO_RING) ? 55296 : 49152;
   // Latency regime (at most 1 MiB per rank, and every layered schedule): slices down to 2 KiB,
   // one work item per queue, as many queues as there are items.  Measured on B200 with 80
   // layers in one launch: 16 KiB one-shot is fastest with 8 queues per rank of 2 KiB each.
